@@ -1,0 +1,216 @@
+/*
+ * draftexpert.h -- C ABI of the B200 (sm_100a) draft / verify MoE hot path of
+ * DraftExpert, expansion-aware self-speculative decoding for MoE models.
+ *
+ * What the library computes (paper notation):
+ *   - drafter,  Eq. 5 (Sec. 3.2):  y^d = S(h) + g_{e1} E_{e1}(h) + gamma E^d(h),  e1 = argmax_e R(h)_e
+ *   - verifier, Eq. 4 (Sec. 3.2):  y*_t = S(h_t) + sum_{e in TopK(h_t)} g_{t,e} E_e(h_t)   for a K-token block,
+ *     evaluated grouped by the block's expert set U(D) = union_t TopK(h_t) (Eq. 2, Eq. 3) so that each
+ *     expert's weights are read from HBM once per block
+ *   - exact greedy verification, Algorithm 1 last two steps: target tokens = vocabulary argmax, accepted
+ *     length = longest draft prefix that equals them
+ *   - the accelerator expert cache C and in-flight set P of Sec. 3.5 / Algorithm 1 (prefetch, wait, on-demand)
+ *
+ * Conventions
+ *   - Every function returns a dx_status; nothing throws, aborts or prints.
+ *   - "device pointer" = memory of the context's GPU, "host pointer" = ordinary host memory, "pinned host
+ *     pointer" = page-locked host memory.  All tensor pointers are BORROWED: the caller allocates and frees
+ *     them and keeps them alive until the stream work that uses them has finished.
+ *   - Handles (dx_ctx, dx_layer, dx_cache) are owned by the library; release them with the matching destroy.
+ *   - Compute calls only enqueue work on the caller's stream (a cudaStream_t passed as void*; NULL is the
+ *     default stream).  They do not synchronise the host, except where a function says so.
+ *   - A context carries one set of device scratch buffers; calls that share a context must be issued on one
+ *     stream (or otherwise ordered).  Use one context per concurrent stream.
+ *   - Matrices are row-major.  Hidden states, outputs, gate weights and logits are fp32; weights are fp32 or
+ *     bf16 as stated by weight_dtype; all accumulation is fp32.
+ *   - Limits: block length K <= 16, experts E <= 256, top-k <= 8, shared experts <= 8, every intermediate size
+ *     a multiple of 8; hidden a multiple of 256 up to 8192 for fp32 weights and one of 256, 512, 1024, 2048
+ *     for bf16 weights.  Outside them: DX_ERR_UNSUPPORTED.
+ *   - Device-side anomalies (an id out of range, a bounded wait that expired) never trap: the kernel records
+ *     a code in the context's device status word, readable with dx_last_device_status.
+ */
+#ifndef DRAFTEXPERT_H_
+#define DRAFTEXPERT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int32_t dx_status;
+enum {
+  DX_OK = 0,
+  DX_ERR_INVALID_ARG = 1,   /* NULL where a pointer is required, misaligned blob, index out of range */
+  DX_ERR_SHAPE = 2,         /* sizes inconsistent with the layer description */
+  DX_ERR_CUDA = 3,          /* a CUDA runtime call failed; see dx_last_cuda_error */
+  DX_ERR_OOM = 4,
+  DX_ERR_NOT_RESIDENT = 5,  /* an expert needed by the call has no weights attached / registered */
+  DX_ERR_TIMEOUT = 6,
+  DX_ERR_CACHE_FULL = 7,
+  DX_ERR_UNSUPPORTED = 8
+};
+
+enum { DX_SCORE_SOFTMAX = 0, DX_SCORE_SIGMOID = 1 };
+enum { DX_DTYPE_FP32 = 0, DX_DTYPE_BF16 = 1 };
+
+/* Codes a kernel may leave in the device status word (0 = clean). */
+enum {
+  DX_DEV_OK = 0,
+  DX_DEV_BAD_EXPERT_ID = 1,     /* a routed expert has no weight blob attached */
+  DX_DEV_WAIT_EXPIRED = 2,      /* a bounded wait inside a kernel gave up */
+  DX_DEV_WORKLIST_OVERFLOW = 3
+};
+
+typedef struct dx_ctx dx_ctx;
+typedef struct dx_layer dx_layer;
+typedef struct dx_cache dx_cache;
+
+/* One MoE layer.  score_fn / norm_topk / routed_scale define R(h) and g_{l,e} of Eq. 4 (the paper leaves
+ * them to the model: softmax or sigmoid scores, top-k weights renormalised or not, times a routed scaling
+ * factor that multiplies the routed sum only).  draft_gamma is gamma_l of Eq. 5. */
+typedef struct {
+  int32_t hidden;        /* H */
+  int32_t n_experts;     /* N_l (E) */
+  int32_t top_k;         /* k_l */
+  int32_t inter;         /* I of the routed experts */
+  int32_t n_shared;      /* number of shared experts making up S_l */
+  int32_t shared_inter;  /* I of each shared expert */
+  int32_t draft_inter;   /* I of the draft expert E^d_l (0 = none) */
+  int32_t score_fn;      /* DX_SCORE_* */
+  int32_t norm_topk;     /* 1: gate weights renormalised over the selected k */
+  int32_t weight_dtype;  /* DX_DTYPE_* of router and expert weights */
+  float routed_scale;
+  float draft_gamma;
+} dx_layer_desc;
+
+const char* dx_status_string(dx_status s);
+
+/* ---- context -------------------------------------------------------------------------------------------
+ * dx_create binds to CUDA device `device`, allocates the context's small device scratch (a few MB: work
+ * list, normalised block, router logits, argmax keys, status word) and returns the handle in *out.
+ * Synchronises the host.  dx_destroy frees it (device must be idle with respect to this context). */
+dx_status dx_create(int device, dx_ctx** out);
+dx_status dx_destroy(dx_ctx* ctx);
+/* Reads (and clears) the device status word.  Synchronises `stream` first. */
+dx_status dx_last_device_status(dx_ctx* ctx, void* stream, int32_t* dev_status_out);
+/* Last cudaError_t seen by this context as an int (0 = none). */
+int32_t dx_last_cuda_error(dx_ctx* ctx);
+/* Number of kernels this context has launched so far (for launch accounting by a caller). */
+int64_t dx_kernel_launches(dx_ctx* ctx);
+
+/* ---- expert weights ---------------------------------------------------------------------------------------
+ * An expert is a SwiGLU feed-forward E(h) = W_d ( silu(W_g h) * (W_u h) ), W_g,W_u [I,H], W_d [H,I]
+ * (the expert form the paper's parameter count in Sec. 2.1 implies: 3*H*I per expert).
+ * The kernels stream each expert from ONE contiguous "blob" in a tile-major layout of the library's choosing
+ * (the same number of bytes as the three matrices).  dx_expert_blob_bytes gives its size;
+ * dx_pack_expert fills a blob from the three canonical row-major matrices (all device pointers; the blob must
+ * be 128-byte aligned; runs on `stream`).  Blobs can be copied around freely (host pool, cache slots). */
+dx_status dx_expert_blob_bytes(const dx_layer_desc* desc, int32_t inter, size_t* bytes_out);
+dx_status dx_pack_expert(dx_ctx* ctx, const dx_layer_desc* desc, int32_t inter,
+                         const void* Wg, const void* Wu, const void* Wd, void* blob_out, void* stream);
+
+/* ---- layer ------------------------------------------------------------------------------------------------
+ * dx_layer_create copies the description and allocates the layer's device pointer table.
+ * set_router: W_r [E,H] in weight_dtype, optional fp32 bias[E] added to the router logits (NULL = none).
+ * set_shared / set_draft / set_expert attach packed blobs (device pointers, 128-byte aligned, borrowed).
+ * set_expert with blob == NULL detaches expert e (a block that then routes to it reports
+ * DX_DEV_BAD_EXPERT_ID in the device status word and skips that expert).
+ * The table is uploaded on the next compute call's stream, so set_* calls must not be interleaved with
+ * compute calls that are still being captured into a CUDA graph. */
+dx_status dx_layer_create(dx_ctx* ctx, const dx_layer_desc* desc, dx_layer** out);
+dx_status dx_layer_destroy(dx_layer* layer);
+dx_status dx_layer_set_router(dx_layer* layer, const void* W_r, const float* bias);
+dx_status dx_layer_set_shared(dx_layer* layer, int32_t s, const void* blob);
+dx_status dx_layer_set_draft(dx_layer* layer, const void* blob);
+dx_status dx_layer_set_expert(dx_layer* layer, int32_t e, const void* blob);
+/* Routed experts of this layer are looked up in cache slots of `cache` (layer index `layer_index` there)
+ * instead of the table filled by set_expert. */
+dx_status dx_layer_attach_cache(dx_layer* layer, dx_cache* cache, int32_t layer_index);
+
+/* ---- drafter: Eq. 5 -----------------------------------------------------------------------------------------
+ * One token.  h [H] fp32 in, y [H] fp32 out (overwritten), topk_ids [k] int32 and topk_w [k] fp32 out:
+ * the router's full top-k in descending score (ties: lower id first) with the gate weights of Eq. 4;
+ * e1 = topk_ids[0], and the k ids are the predicted verifier experts \hat{E}_{l,i} of Sec. 3.4.
+ * All device pointers. */
+dx_status moe_draft_step(dx_layer* layer, const float* h, float* y, int32_t* topk_ids, float* topk_w,
+                         void* stream);
+
+/* ---- verifier: Eq. 4 over a block, grouped by the union of Eq. 2 / Eq. 3 -----------------------------------
+ * h [K,H] in, y [K,H] out (overwritten).  Routing outputs (device pointers, each may be NULL if unwanted):
+ *   topk_ids [K,k] int32, topk_w [K,k] fp32;
+ *   union_mask [ceil(E/64)] uint64 (bit e set iff e in U); union_ids [min(E,K*k)] int32 ascending;
+ *   union_count [1] int32 = |U|;
+ *   offsets [E+1] int32 and perm [K*k] int32: the token-expert pairs p = t*k + j sorted by (expert, p);
+ *   expert e owns perm[offsets[e] .. offsets[e+1]).
+ * moe_verify_block = moe_verify_route followed by moe_verify_experts on the same stream; the two halves are
+ * exported so that a caller with offloaded experts can make them resident in between. */
+dx_status moe_verify_block(dx_layer* layer, const float* h, int32_t K, float* y,
+                           int32_t* topk_ids, float* topk_w, uint64_t* union_mask, int32_t* union_ids,
+                           int32_t* union_count, int32_t* offsets, int32_t* perm, void* stream);
+dx_status moe_verify_route(dx_layer* layer, const float* h, int32_t K, float* y,
+                           int32_t* topk_ids, float* topk_w, uint64_t* union_mask, int32_t* union_ids,
+                           int32_t* union_count, int32_t* offsets, int32_t* perm, void* stream);
+dx_status moe_verify_experts(dx_layer* layer, const float* h, int32_t K, float* y, void* stream);
+
+/* ---- pre-norm residual forms for layer stacks (synthetic stacks stub attention out) --------------------------
+ * h [K,H] is updated IN PLACE: h <- h + MoE(RMSNorm(h)) with unit gain and eps 1e-6, MoE = Eq. 4
+ * (verify) or Eq. 5 (draft, K = 1).  Routing outputs as above (NULL allowed). */
+dx_status moe_verify_block_residual(dx_layer* layer, float* h, int32_t K,
+                                    int32_t* topk_ids, float* topk_w, uint64_t* union_mask,
+                                    int32_t* union_ids, int32_t* union_count, int32_t* offsets,
+                                    int32_t* perm, void* stream);
+dx_status moe_draft_step_residual(dx_layer* layer, float* h, int32_t* topk_ids, float* topk_w, void* stream);
+
+/* ---- exact greedy verification: Algorithm 1, "verify" and "accept the target-consistent prefix" -------------
+ * h [M,H] fp32: row i is the hidden state that predicts draft token i (M = K, or K+1 to also get the token
+ * after a fully accepted block).  W_lm [V,H] in w_dtype.  draft [K] int32.  Outputs (device):
+ *   target [M] int32 = argmax_v <W_lm[v], h_i> (lowest v on ties);
+ *   n_accept [1] = length of the longest prefix with target[i] == draft[i];
+ *   next_token [1] = target[n_accept] if n_accept < M else -1.
+ * rms_norm != 0 applies RMSNorm (unit gain, eps 1e-6) to each row of h first.  M <= 16, H <= 8192. */
+dx_status spec_accept(dx_ctx* ctx, const float* h, int32_t M, const void* W_lm, int32_t V, int32_t H,
+                      int32_t w_dtype, const int32_t* draft, int32_t K, int32_t rms_norm,
+                      int32_t* target, int32_t* n_accept, int32_t* next_token, void* stream);
+
+/* ---- accelerator expert cache: C and P of Algorithm 1, Sec. 3.5 ----------------------------------------------
+ * A cache owns n_layers * slots_per_layer HBM slots of blob_bytes each (allocated in create), a side stream
+ * for transfers and one event per slot.  Routed experts live in a host pool the caller registers blob by
+ * blob (pinned host pointers, borrowed).  All id arrays are HOST pointers.
+ *   prefetch: for each id not cached and not in flight, pick the least-recently-used free slot and start a
+ *             non-blocking copy on the side stream (Algorithm 1: prefetch U_hat \ (C u P)); never blocks.
+ *   stage:    make ids resident now: cached ones are hits; in-flight ones are waited for; the rest are copied
+ *             on demand.  `stream` is made to wait (cudaStreamWaitEvent) for exactly the copies it needs.
+ *             n must not exceed slots_per_layer (DX_ERR_CACHE_FULL); larger unions are staged in waves.
+ *   wait:     like stage but never starts a copy: ids that are neither cached nor in flight give
+ *             DX_ERR_NOT_RESIDENT; host-polls outstanding copies up to timeout_s (DX_ERR_TIMEOUT).
+ * Results never depend on the cache: it only decides where a blob sits and when it moves. */
+typedef struct {
+  int64_t lookups;          /* ids asked for by stage / wait */
+  int64_t hits;             /* of those, already cached or in flight (no on-demand copy) */
+  int64_t on_demand;        /* copies started by stage */
+  int64_t prefetch_issued;  /* copies started by prefetch */
+  int64_t prefetch_used;    /* prefetched experts later asked for by stage / wait */
+  int64_t prefetch_wasted;  /* prefetched experts evicted before any use */
+  int64_t evictions;
+  int64_t bytes_h2d;
+} dx_cache_stats;
+
+dx_status expert_cache_create(dx_ctx* ctx, int32_t n_layers, int32_t n_experts, int32_t slots_per_layer,
+                              size_t blob_bytes, dx_cache** out);
+dx_status expert_cache_destroy(dx_cache* cache);
+dx_status expert_cache_register(dx_cache* cache, int32_t layer, int32_t expert, const void* pinned_host_blob);
+dx_status expert_cache_prefetch(dx_cache* cache, int32_t layer, const int32_t* host_ids, int32_t n);
+dx_status expert_cache_stage(dx_cache* cache, int32_t layer, const int32_t* host_ids, int32_t n, void* stream);
+dx_status expert_cache_wait(dx_cache* cache, int32_t layer, const int32_t* host_ids, int32_t n, void* stream,
+                            double timeout_s);
+dx_status expert_cache_stats(dx_cache* cache, dx_cache_stats* out);
+/* Slot currently holding `expert` of `layer` (-1 if none) and whether its copy is still in flight. */
+dx_status expert_cache_query(dx_cache* cache, int32_t layer, int32_t expert, int32_t* slot_out,
+                             int32_t* in_flight_out);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DRAFTEXPERT_H_ */

@@ -1,0 +1,315 @@
+"""Thin ctypes binding over ``libdraftexpert.so`` (the C ABI in ``include/draftexpert.h``).
+
+Argument marshalling only: PyTorch supplies device memory and the current
+stream, every step of the path (routing, union, grouped SwiGLU, argmax/accept,
+weight packing, cache transfers) runs inside the library.  Function names match
+the C entry points.  There is no fallback: if the shared library is missing or
+a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Dict, List, Optional, Sequence, Tuple
+
+import torch
+
+from .synth import DTYPE_BF16, LayerShape
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libdraftexpert.so")
+
+DX_OK = 0
+STATUS_NAMES = {0: "DX_OK", 1: "DX_ERR_INVALID_ARG", 2: "DX_ERR_SHAPE", 3: "DX_ERR_CUDA", 4: "DX_ERR_OOM",
+                5: "DX_ERR_NOT_RESIDENT", 6: "DX_ERR_TIMEOUT", 7: "DX_ERR_CACHE_FULL", 8: "DX_ERR_UNSUPPORTED"}
+
+
+class DxError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        super().__init__(f"{what}: {STATUS_NAMES.get(status, status)}")
+        self.status = status
+
+
+class LayerDesc(C.Structure):
+    _fields_ = [("hidden", C.c_int32), ("n_experts", C.c_int32), ("top_k", C.c_int32), ("inter", C.c_int32),
+                ("n_shared", C.c_int32), ("shared_inter", C.c_int32), ("draft_inter", C.c_int32),
+                ("score_fn", C.c_int32), ("norm_topk", C.c_int32), ("weight_dtype", C.c_int32),
+                ("routed_scale", C.c_float), ("draft_gamma", C.c_float)]
+
+
+class CacheStats(C.Structure):
+    _fields_ = [(n, C.c_int64) for n in ("lookups", "hits", "on_demand", "prefetch_issued", "prefetch_used",
+                                         "prefetch_wasted", "evictions", "bytes_h2d")]
+
+
+_P = C.c_void_p
+_I = C.c_int32
+# name -> (restype, argtypes): one line per declaration in include/draftexpert.h
+SIGNATURES = {
+    "dx_status_string": (C.c_char_p, [_I]),
+    "dx_create": (_I, [C.c_int, C.POINTER(_P)]),
+    "dx_destroy": (_I, [_P]),
+    "dx_last_device_status": (_I, [_P, _P, C.POINTER(_I)]),
+    "dx_last_cuda_error": (_I, [_P]),
+    "dx_kernel_launches": (C.c_int64, [_P]),
+    "dx_expert_blob_bytes": (_I, [C.POINTER(LayerDesc), _I, C.POINTER(C.c_size_t)]),
+    "dx_pack_expert": (_I, [_P, C.POINTER(LayerDesc), _I, _P, _P, _P, _P, _P]),
+    "dx_layer_create": (_I, [_P, C.POINTER(LayerDesc), C.POINTER(_P)]),
+    "dx_layer_destroy": (_I, [_P]),
+    "dx_layer_set_router": (_I, [_P, _P, _P]),
+    "dx_layer_set_shared": (_I, [_P, _I, _P]),
+    "dx_layer_set_draft": (_I, [_P, _P]),
+    "dx_layer_set_expert": (_I, [_P, _I, _P]),
+    "dx_layer_attach_cache": (_I, [_P, _P, _I]),
+    "moe_draft_step": (_I, [_P, _P, _P, _P, _P, _P]),
+    "moe_draft_step_residual": (_I, [_P, _P, _P, _P, _P]),
+    "moe_verify_block": (_I, [_P, _P, _I, _P, _P, _P, _P, _P, _P, _P, _P, _P]),
+    "moe_verify_route": (_I, [_P, _P, _I, _P, _P, _P, _P, _P, _P, _P, _P, _P]),
+    "moe_verify_experts": (_I, [_P, _P, _I, _P, _P]),
+    "moe_verify_block_residual": (_I, [_P, _P, _I, _P, _P, _P, _P, _P, _P, _P, _P]),
+    "spec_accept": (_I, [_P, _P, _I, _P, _I, _I, _I, _P, _I, _I, _P, _P, _P, _P]),
+    "expert_cache_create": (_I, [_P, _I, _I, _I, C.c_size_t, C.POINTER(_P)]),
+    "expert_cache_destroy": (_I, [_P]),
+    "expert_cache_register": (_I, [_P, _I, _I, _P]),
+    "expert_cache_prefetch": (_I, [_P, _I, _P, _I]),
+    "expert_cache_stage": (_I, [_P, _I, _P, _I, _P]),
+    "expert_cache_wait": (_I, [_P, _I, _P, _I, _P, C.c_double]),
+    "expert_cache_stats": (_I, [_P, C.POINTER(CacheStats)]),
+    "expert_cache_query": (_I, [_P, _I, _I, C.POINTER(_I), C.POINTER(_I)]),
+}
+
+_lib = None
+
+
+def load() -> C.CDLL:
+    """Loads the shared library (built by ``paper_2607_24434_b200/build.py``); raises if it is absent."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise FileNotFoundError(f"{LIB_PATH} not built: run `python -m paper_2607_24434_b200.build`")
+        lib = C.CDLL(LIB_PATH)
+        for name, (res, args) in SIGNATURES.items():
+            fn = getattr(lib, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = lib
+    return _lib
+
+
+def _check(status: int, what: str) -> None:
+    if status != DX_OK:
+        raise DxError(status, what)
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _desc(shape: LayerShape) -> LayerDesc:
+    return LayerDesc(shape.hidden, shape.n_experts, shape.top_k, shape.inter, shape.n_shared, shape.shared_inter,
+                     shape.draft_inter, shape.score_fn, shape.norm_topk, shape.weight_dtype, shape.routed_scale,
+                     shape.draft_gamma)
+
+
+class Context:
+    def __init__(self, device: int = 0):
+        self.lib = load()
+        self.device = device
+        h = _P()
+        _check(self.lib.dx_create(device, C.byref(h)), "dx_create")
+        self.handle = h
+
+    def close(self) -> None:
+        if self.handle:
+            self.lib.dx_destroy(self.handle)
+            self.handle = None
+
+    def device_status(self) -> int:
+        out = _I(0)
+        _check(self.lib.dx_last_device_status(self.handle, _stream(), C.byref(out)), "dx_last_device_status")
+        return out.value
+
+    def kernel_launches(self) -> int:
+        return int(self.lib.dx_kernel_launches(self.handle))
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def expert_blob_bytes(shape: LayerShape, inter: int) -> int:
+    n = C.c_size_t(0)
+    d = _desc(shape)
+    _check(load().dx_expert_blob_bytes(C.byref(d), inter, C.byref(n)), "dx_expert_blob_bytes")
+    return n.value
+
+
+def pack_expert(ctx: Context, shape: LayerShape, Wg: torch.Tensor, Wu: torch.Tensor, Wd: torch.Tensor,
+                out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """dx_pack_expert: canonical W_g [I,H], W_u [I,H], W_d [H,I] -> one streaming blob (uint8 tensor)."""
+    inter = Wg.shape[0]
+    nbytes = expert_blob_bytes(shape, inter)
+    if out is None:
+        out = torch.empty(nbytes, dtype=torch.uint8, device=Wg.device)
+    d = _desc(shape)
+    _check(ctx.lib.dx_pack_expert(ctx.handle, C.byref(d), inter, _ptr(Wg.contiguous()), _ptr(Wu.contiguous()),
+                                  _ptr(Wd.contiguous()), _ptr(out), _stream()), "dx_pack_expert")
+    return out
+
+
+class Layer:
+    """Handle of one MoE layer plus the tensors it borrows (kept alive here)."""
+
+    def __init__(self, ctx: Context, shape: LayerShape):
+        self.ctx, self.shape, self.lib = ctx, shape, ctx.lib
+        d = _desc(shape)
+        h = _P()
+        _check(self.lib.dx_layer_create(ctx.handle, C.byref(d), C.byref(h)), "dx_layer_create")
+        self.handle = h
+        self._keep: Dict[str, object] = {}
+
+    def close(self) -> None:
+        if self.handle:
+            self.lib.dx_layer_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def set_router(self, W_r: torch.Tensor, bias: Optional[torch.Tensor]) -> None:
+        self._keep["router"] = (W_r, bias)
+        _check(self.lib.dx_layer_set_router(self.handle, _ptr(W_r), _ptr(bias)), "dx_layer_set_router")
+
+    def set_shared(self, s: int, blob: torch.Tensor) -> None:
+        self._keep[f"shared{s}"] = blob
+        _check(self.lib.dx_layer_set_shared(self.handle, s, _ptr(blob)), "dx_layer_set_shared")
+
+    def set_draft(self, blob: torch.Tensor) -> None:
+        self._keep["draft"] = blob
+        _check(self.lib.dx_layer_set_draft(self.handle, _ptr(blob)), "dx_layer_set_draft")
+
+    def set_expert(self, e: int, blob: Optional[torch.Tensor]) -> None:
+        self._keep[f"expert{e}"] = blob
+        _check(self.lib.dx_layer_set_expert(self.handle, e, _ptr(blob)), "dx_layer_set_expert")
+
+    @classmethod
+    def from_weights(cls, ctx: Context, layer: Dict[str, object], routed_resident: bool = True) -> "Layer":
+        """Packs a canonical-layout layer (see ``synth.make_layer``) that already sits on the GPU and
+        attaches everything.  The routed experts share one [E, blob_bytes] allocation."""
+        shape: LayerShape = layer["shape"]
+        L = cls(ctx, shape)
+        L.set_router(layer["router"].contiguous(), None if layer["bias"] is None else layer["bias"].contiguous())
+        for s, (g, u, d) in enumerate(layer["shared"]):
+            L.set_shared(s, pack_expert(ctx, shape, g, u, d))
+        if layer["draft"] is not None:
+            L.set_draft(pack_expert(ctx, shape, *layer["draft"]))
+        Wg, Wu, Wd = layer["experts"]
+        nbytes = expert_blob_bytes(shape, shape.inter)
+        blobs = torch.empty((shape.n_experts, nbytes), dtype=torch.uint8, device=Wg.device)
+        for e in range(shape.n_experts):
+            pack_expert(ctx, shape, Wg[e], Wu[e], Wd[e], out=blobs[e])
+            if routed_resident:
+                L.set_expert(e, blobs[e])
+        L.blobs = blobs
+        return L
+
+
+def _routing_buffers(shape: LayerShape, K: int, device) -> Dict[str, torch.Tensor]:
+    E, k = shape.n_experts, shape.top_k
+    i32 = dict(dtype=torch.int32, device=device)
+    return {
+        "topk_ids": torch.empty((K, k), **i32),
+        "topk_w": torch.empty((K, k), dtype=torch.float32, device=device),
+        "union_mask": torch.empty(((E + 63) // 64,), dtype=torch.int64, device=device),
+        "union_ids": torch.full((min(E, K * k),), -1, **i32),
+        "union_count": torch.empty((1,), **i32),
+        "offsets": torch.empty((E + 1,), **i32),
+        "perm": torch.empty((K * k,), **i32),
+    }
+
+
+def moe_draft_step(layer: Layer, h: torch.Tensor, y: Optional[torch.Tensor] = None,
+                   out: Optional[Dict[str, torch.Tensor]] = None) -> Dict[str, torch.Tensor]:
+    """Eq. 5 for one token: h [H] (or [1,H]) fp32 -> y, topk_ids [k], topk_w [k]."""
+    sh = layer.shape
+    if out is None:
+        out = {"topk_ids": torch.empty((sh.top_k,), dtype=torch.int32, device=h.device),
+               "topk_w": torch.empty((sh.top_k,), dtype=torch.float32, device=h.device)}
+    if y is None:
+        y = torch.empty_like(h)
+    _check(layer.lib.moe_draft_step(layer.handle, _ptr(h), _ptr(y), _ptr(out["topk_ids"]), _ptr(out["topk_w"]),
+                                    _stream()), "moe_draft_step")
+    out["y"] = y
+    return out
+
+
+def moe_draft_step_residual(layer: Layer, h: torch.Tensor, out: Optional[Dict[str, torch.Tensor]] = None):
+    sh = layer.shape
+    if out is None:
+        out = {"topk_ids": torch.empty((sh.top_k,), dtype=torch.int32, device=h.device),
+               "topk_w": torch.empty((sh.top_k,), dtype=torch.float32, device=h.device)}
+    _check(layer.lib.moe_draft_step_residual(layer.handle, _ptr(h), _ptr(out["topk_ids"]), _ptr(out["topk_w"]),
+                                             _stream()), "moe_draft_step_residual")
+    return out
+
+
+def moe_verify_block(layer: Layer, h: torch.Tensor, y: Optional[torch.Tensor] = None,
+                     out: Optional[Dict[str, torch.Tensor]] = None) -> Dict[str, torch.Tensor]:
+    """Eq. 4 for a block h [K,H] fp32, grouped by the union of Eq. 2/3.  Returns y and the routing outputs."""
+    K = h.shape[0]
+    if out is None:
+        out = _routing_buffers(layer.shape, K, h.device)
+    if y is None:
+        y = torch.empty_like(h)
+    _check(layer.lib.moe_verify_block(layer.handle, _ptr(h), K, _ptr(y), _ptr(out["topk_ids"]), _ptr(out["topk_w"]),
+                                      _ptr(out["union_mask"]), _ptr(out["union_ids"]), _ptr(out["union_count"]),
+                                      _ptr(out["offsets"]), _ptr(out["perm"]), _stream()), "moe_verify_block")
+    out["y"] = y
+    return out
+
+
+def moe_verify_route(layer: Layer, h: torch.Tensor, y: torch.Tensor, out: Dict[str, torch.Tensor]) -> None:
+    _check(layer.lib.moe_verify_route(layer.handle, _ptr(h), h.shape[0], _ptr(y), _ptr(out["topk_ids"]),
+                                      _ptr(out["topk_w"]), _ptr(out["union_mask"]), _ptr(out["union_ids"]),
+                                      _ptr(out["union_count"]), _ptr(out["offsets"]), _ptr(out["perm"]), _stream()),
+           "moe_verify_route")
+
+
+def moe_verify_experts(layer: Layer, h: torch.Tensor, y: torch.Tensor) -> None:
+    _check(layer.lib.moe_verify_experts(layer.handle, _ptr(h), h.shape[0], _ptr(y), _stream()), "moe_verify_experts")
+
+
+def moe_verify_block_residual(layer: Layer, h: torch.Tensor, out: Optional[Dict[str, torch.Tensor]] = None):
+    """In place: h <- h + MoE(RMSNorm(h)) for the block."""
+    K = h.shape[0]
+    if out is None:
+        out = _routing_buffers(layer.shape, K, h.device)
+    _check(layer.lib.moe_verify_block_residual(layer.handle, _ptr(h), K, _ptr(out["topk_ids"]), _ptr(out["topk_w"]),
+                                               _ptr(out["union_mask"]), _ptr(out["union_ids"]),
+                                               _ptr(out["union_count"]), _ptr(out["offsets"]), _ptr(out["perm"]),
+                                               _stream()), "moe_verify_block_residual")
+    return out
+
+
+def spec_accept(ctx: Context, h: torch.Tensor, W_lm: torch.Tensor, draft: torch.Tensor, rms_norm: bool = False,
+                out: Optional[Dict[str, torch.Tensor]] = None) -> Dict[str, torch.Tensor]:
+    """Greedy exact verification: target [M], n_accept [1], next_token [1] (all int32, on the device)."""
+    M, H = h.shape
+    V = W_lm.shape[0]
+    if out is None:
+        out = {"target": torch.empty((M,), dtype=torch.int32, device=h.device),
+               "n_accept": torch.empty((1,), dtype=torch.int32, device=h.device),
+               "next_token": torch.empty((1,), dtype=torch.int32, device=h.device)}
+    wd = 1 if W_lm.dtype == torch.bfloat16 else 0
+    _check(ctx.lib.spec_accept(ctx.handle, _ptr(h), M, _ptr(W_lm), V, H, wd, _ptr(draft), int(draft.shape[0]),
+                               1 if rms_norm else 0, _ptr(out["target"]), _ptr(out["n_accept"]),
+                               _ptr(out["next_token"]), _stream()), "spec_accept")
+    return out

@@ -1,0 +1,266 @@
+// Exact greedy verification (Algorithm 1, "verify" + "accept the
+// target-consistent prefix"): target tokens t_i = argmax_v <W_lm[v], h_i> with
+// the lowest v winning ties, accepted length n = longest prefix with
+// t_i == d_i, next token = t_n.
+//
+// The LM head [V,H] is streamed from HBM exactly once for all M rows.  bf16
+// path: each warp owns 16 vocabulary rows at a time and multiplies them with
+// the M hidden rows on the tensor cores (mma.sync m16n8k16, vocabulary rows as
+// the 16-row operand, hidden rows as the 8-column operand, hidden rows fed as
+// bf16 high part + bf16 residual).  A lane loads 16 contiguous bytes of two
+// rows per step straight from global memory; the contraction index is permuted
+// consistently on both operands so those 16 bytes are exactly its fragment.
+// Every lane tracks the running maximum of the logits it owns; maxima are
+// merged as packed 64-bit keys (orderable logit << 32 | ~index) with
+// atomicMax, and the CTA that takes the last ticket turns the keys into
+// tokens, the accepted length and the next token.
+#include "dx_internal.cuh"
+
+namespace {
+
+__device__ __forceinline__ uint4 ldg_stream(const void* p) {
+  uint4 r;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
+               : "l"(p));
+  return r;
+}
+__device__ __forceinline__ void mma_k16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                        uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack2(__nv_bfloat16 lo16, __nv_bfloat16 hi16) {
+  return (uint32_t)__bfloat16_as_ushort(lo16) | ((uint32_t)__bfloat16_as_ushort(hi16) << 16);
+}
+__device__ __forceinline__ unsigned long long make_key(float v, int idx) {
+  return ((unsigned long long)dx_orderable(v) << 32) | (unsigned long long)(0xffffffffu - (unsigned)idx);
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+struct AcceptParams {
+  const float* h;
+  int M, V, H;
+  const void* W;
+  const int32_t* draft;
+  int K;
+  int rms_norm;
+  int32_t* target;
+  int32_t* n_accept;
+  int32_t* next_token;
+  unsigned long long* keys;
+  unsigned int* ticket;
+};
+
+// Shared tail: merge CTA maxima into the global keys; the last CTA decodes.
+__device__ __forceinline__ void finish(const AcceptParams& p, unsigned long long* s_keys) {
+  __shared__ int s_last;
+  __syncthreads();
+  if (threadIdx.x < p.M && s_keys[threadIdx.x] != 0ull) atomicMax(p.keys + threadIdx.x, s_keys[threadIdx.x]);
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) s_last = (atomicAdd(p.ticket, 1u) == gridDim.x - 1);
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  __shared__ int s_tok[DX_MAX_M];
+  if (threadIdx.x < p.M) {
+    unsigned long long kk = __ldcg(p.keys + threadIdx.x);
+    int tok = (int)(0xffffffffu - (unsigned)(kk & 0xffffffffull));
+    s_tok[threadIdx.x] = tok;
+    p.target[threadIdx.x] = tok;
+    p.keys[threadIdx.x] = 0ull;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int n = 0;
+    while (n < p.K && n < p.M && p.draft[n] == s_tok[n]) ++n;
+    *p.n_accept = n;
+    *p.next_token = n < p.M ? s_tok[n] : -1;
+    *p.ticket = 0u;
+  }
+}
+
+template <int NT>
+__global__ void __launch_bounds__(512, 1) dx_accept_bf16_kernel(AcceptParams p) {
+  extern __shared__ __align__(16) unsigned char smem[];
+  __shared__ float s_rstd[DX_MAX_M];
+  __shared__ unsigned long long s_keys[DX_MAX_M];
+  const int H = p.H, Q = H / 32;
+  uint4* hiF = reinterpret_cast<uint4*>(smem);        // [NT][Q][32]
+  uint4* loF = hiF + (size_t)NT * Q * 32;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, c = lane & 3;
+
+  if (warp < DX_MAX_M) {
+    float r = 1.0f;
+    if (p.rms_norm && warp < p.M) {
+      float ss = 0.f;
+      for (int j = lane * 4; j < H; j += 128) {
+        float4 v = *reinterpret_cast<const float4*>(p.h + (size_t)warp * H + j);
+        ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+      }
+      r = rsqrtf(warp_sum(ss) / (float)H + 1e-6f);
+    }
+    if (lane == 0) { s_rstd[warp] = r; s_keys[warp] = 0ull; }
+  }
+  __syncthreads();
+  // hidden-row fragments: lane (g,c) of column block q holds, for row nt*8+g,
+  // columns 32q+8c..+7 split into bf16 high part and residual
+  for (int idx = threadIdx.x; idx < NT * Q * 32; idx += blockDim.x) {
+    const int l = idx & 31, q = (idx >> 5) % Q, nt = idx / (32 * Q);
+    const int row = nt * 8 + (l >> 2);
+    uint4 oh = make_uint4(0u, 0u, 0u, 0u), ol = oh;
+    if (row < p.M) {
+      const float* src = p.h + (size_t)row * H + 32 * q + 8 * (l & 3);
+      const float4 v0 = *reinterpret_cast<const float4*>(src), v1 = *reinterpret_cast<const float4*>(src + 4);
+      const float rs = s_rstd[row];
+      const float x[8] = {v0.x * rs, v0.y * rs, v0.z * rs, v0.w * rs, v1.x * rs, v1.y * rs, v1.z * rs, v1.w * rs};
+      __nv_bfloat16 hb[8], lb[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        hb[i] = __float2bfloat16_rn(x[i]);
+        lb[i] = __float2bfloat16_rn(x[i] - __bfloat162float(hb[i]));
+      }
+      oh = make_uint4(pack2(hb[0], hb[1]), pack2(hb[2], hb[3]), pack2(hb[4], hb[5]), pack2(hb[6], hb[7]));
+      ol = make_uint4(pack2(lb[0], lb[1]), pack2(lb[2], lb[3]), pack2(lb[4], lb[5]), pack2(lb[6], lb[7]));
+    }
+    hiF[idx] = oh;
+    loF[idx] = ol;
+  }
+  __syncthreads();
+
+  float best_v[NT][2];
+  int best_i[NT][2];
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt) { best_v[nt][0] = best_v[nt][1] = -INFINITY; best_i[nt][0] = best_i[nt][1] = -1; }
+
+  const int tiles = (p.V + 15) / 16;
+  const int warps_total = gridDim.x * (blockDim.x >> 5);
+  const __nv_bfloat16* Wb = reinterpret_cast<const __nv_bfloat16*>(p.W);
+  for (int tile = blockIdx.x * (blockDim.x >> 5) + warp; tile < tiles; tile += warps_total) {
+    const int r0 = tile * 16 + g, r1 = r0 + 8;
+    const __nv_bfloat16* w0 = Wb + (size_t)min(r0, p.V - 1) * H + 8 * c;
+    const __nv_bfloat16* w1 = Wb + (size_t)min(r1, p.V - 1) * H + 8 * c;
+    float ch[NT][4], cl[NT][4];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+      for (int r = 0; r < 4; ++r) ch[nt][r] = cl[nt][r] = 0.f;
+#pragma unroll 8
+    for (int q = 0; q < Q; ++q) {
+      const uint4 a0 = ldg_stream(w0 + 32 * q);
+      const uint4 a1 = ldg_stream(w1 + 32 * q);
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) {
+        const uint4 bh = hiF[(nt * Q + q) * 32 + lane];
+        const uint4 bl = loF[(nt * Q + q) * 32 + lane];
+        mma_k16(ch[nt], a0.x, a1.x, a0.y, a1.y, bh.x, bh.y);
+        mma_k16(cl[nt], a0.x, a1.x, a0.y, a1.y, bl.x, bl.y);
+        mma_k16(ch[nt], a0.z, a1.z, a0.w, a1.w, bh.z, bh.w);
+        mma_k16(cl[nt], a0.z, a1.z, a0.w, a1.w, bl.z, bl.w);
+      }
+    }
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+      const float l00 = ch[nt][0] + cl[nt][0], l01 = ch[nt][1] + cl[nt][1];
+      const float l10 = ch[nt][2] + cl[nt][2], l11 = ch[nt][3] + cl[nt][3];
+      if (r0 < p.V) {
+        if (l00 > best_v[nt][0]) { best_v[nt][0] = l00; best_i[nt][0] = r0; }
+        if (l01 > best_v[nt][1]) { best_v[nt][1] = l01; best_i[nt][1] = r0; }
+      }
+      if (r1 < p.V) {
+        if (l10 > best_v[nt][0]) { best_v[nt][0] = l10; best_i[nt][0] = r1; }
+        if (l11 > best_v[nt][1]) { best_v[nt][1] = l11; best_i[nt][1] = r1; }
+      }
+    }
+  }
+  // lanes with equal c hold the same token columns: merge over g
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+      unsigned long long key = best_i[nt][j] >= 0 ? make_key(best_v[nt][j], best_i[nt][j]) : 0ull;
+#pragma unroll
+      for (int o = 4; o < 32; o <<= 1) {
+        unsigned long long other = __shfl_xor_sync(0xffffffffu, key, o);
+        key = other > key ? other : key;
+      }
+      const int row = nt * 8 + 2 * c + j;
+      if (g == 0 && row < p.M && key != 0ull) atomicMax(&s_keys[row], key);
+    }
+  finish(p, s_keys);
+}
+
+// fp32 LM head (small vocabularies): one warp per vocabulary row.
+__global__ void __launch_bounds__(256) dx_accept_fp32_kernel(AcceptParams p) {
+  __shared__ float s_rstd[DX_MAX_M];
+  __shared__ unsigned long long s_keys[DX_MAX_M];
+  const int H = p.H, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (int row = warp; row < DX_MAX_M; row += 8) {
+    float r = 1.0f;
+    if (p.rms_norm && row < p.M) {
+      float ss = 0.f;
+      for (int j = lane; j < H; j += 32) { float v = p.h[(size_t)row * H + j]; ss += v * v; }
+      r = rsqrtf(warp_sum(ss) / (float)H + 1e-6f);
+    }
+    if (lane == 0) { s_rstd[row] = r; s_keys[row] = 0ull; }
+  }
+  __syncthreads();
+  const float* Wf = reinterpret_cast<const float*>(p.W);
+  const int warps_total = gridDim.x * 8;
+  unsigned long long best[DX_MAX_M];
+#pragma unroll
+  for (int i = 0; i < DX_MAX_M; ++i) best[i] = 0ull;
+  for (int v = blockIdx.x * 8 + warp; v < p.V; v += warps_total) {
+    const float* wr = Wf + (size_t)v * H;
+#pragma unroll
+    for (int i = 0; i < DX_MAX_M; ++i) {
+      if (i < p.M) {
+        float acc = 0.f;
+        for (int j = lane; j < H; j += 32) acc = fmaf(wr[j], p.h[(size_t)i * H + j] * s_rstd[i], acc);
+        acc = warp_sum(acc);
+        unsigned long long key = make_key(acc, v);
+        best[i] = key > best[i] ? key : best[i];
+      }
+    }
+  }
+  if (lane == 0) {
+#pragma unroll
+    for (int i = 0; i < DX_MAX_M; ++i)
+      if (i < p.M && best[i] != 0ull) atomicMax(&s_keys[i], best[i]);
+  }
+  finish(p, s_keys);
+}
+
+}  // namespace
+
+cudaError_t dx_launch_accept(dx_ctx* ctx, const float* h, int M, const void* W_lm, int V, int H, int w_dtype,
+                             const int32_t* draft, int K, int rms_norm, int32_t* target, int32_t* n_accept,
+                             int32_t* next_token, cudaStream_t st) {
+  AcceptParams p{h, M, V, H, W_lm, draft, K, rms_norm, target, n_accept, next_token, ctx->keys, ctx->ticket + 1};
+  if (w_dtype == DX_DTYPE_FP32) {
+    int grid = (V + 7) / 8;
+    if (grid > ctx->sm_count * 8) grid = ctx->sm_count * 8;
+    dx_accept_fp32_kernel<<<grid, 256, 0, st>>>(p);
+    return cudaGetLastError();
+  }
+  const int NT = (M + 7) / 8;
+  const size_t smem = (size_t)NT * (H / 32) * 32 * 16 * 2;
+  cudaError_t e;
+  if (NT == 1) {
+    e = cudaFuncSetAttribute(dx_accept_bf16_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    dx_accept_bf16_kernel<1><<<ctx->sm_count, 512, smem, st>>>(p);
+  } else {
+    e = cudaFuncSetAttribute(dx_accept_bf16_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    dx_accept_bf16_kernel<2><<<ctx->sm_count, 512, smem, st>>>(p);
+  }
+  return cudaGetLastError();
+}

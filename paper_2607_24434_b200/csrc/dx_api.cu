@@ -1,0 +1,329 @@
+// C-ABI entry points: context and layer handles, argument checking, and the
+// launch sequences of the draft step (Eq. 5), the verify block (Eq. 4 grouped
+// by the union of Eq. 2 / Eq. 3) and greedy acceptance (Algorithm 1).
+#include <new>
+
+#include "dx_internal.cuh"
+
+bool dx_bf16_hidden_supported(int H);
+
+#define DX_CUDA(ctx, call)                 \
+  do {                                     \
+    cudaError_t e__ = (call);              \
+    if (e__ != cudaSuccess) {              \
+      if (ctx) (ctx)->last_cuda = e__;     \
+      return DX_ERR_CUDA;                  \
+    }                                      \
+  } while (0)
+
+extern "C" const char* dx_status_string(dx_status s) {
+  switch (s) {
+    case DX_OK: return "ok";
+    case DX_ERR_INVALID_ARG: return "invalid argument";
+    case DX_ERR_SHAPE: return "shape mismatch";
+    case DX_ERR_CUDA: return "CUDA runtime error";
+    case DX_ERR_OOM: return "out of memory";
+    case DX_ERR_NOT_RESIDENT: return "expert not resident";
+    case DX_ERR_TIMEOUT: return "timed out";
+    case DX_ERR_CACHE_FULL: return "expert cache full";
+    case DX_ERR_UNSUPPORTED: return "unsupported configuration";
+    default: return "unknown status";
+  }
+}
+
+extern "C" dx_status dx_create(int device, dx_ctx** out) {
+  if (!out) return DX_ERR_INVALID_ARG;
+  *out = nullptr;
+  int n = 0;
+  if (cudaGetDeviceCount(&n) != cudaSuccess || device < 0 || device >= n) return DX_ERR_CUDA;
+  dx_ctx* ctx = new (std::nothrow) dx_ctx();
+  if (!ctx) return DX_ERR_OOM;
+  ctx->device = device;
+  ctx->last_cuda = cudaSuccess;
+  ctx->launches = 0;
+  cudaError_t e = cudaSetDevice(device);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, device);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device);
+  if (e == cudaSuccess) e = cudaMalloc(&ctx->work, sizeof(DxWork));
+  if (e == cudaSuccess) e = cudaMalloc(&ctx->xn, sizeof(float) * DX_MAX_K * DX_MAX_H);
+  if (e == cudaSuccess) e = cudaMalloc(&ctx->z, sizeof(float) * DX_MAX_K * DX_MAX_E);
+  if (e == cudaSuccess) e = cudaMalloc(&ctx->ticket, sizeof(unsigned int) * 4);
+  if (e == cudaSuccess) e = cudaMalloc(&ctx->keys, sizeof(unsigned long long) * DX_MAX_M);
+  if (e == cudaSuccess) e = cudaMalloc(&ctx->dev_status, sizeof(int32_t));
+  if (e == cudaSuccess) e = cudaMemset(ctx->work, 0, sizeof(DxWork));
+  if (e == cudaSuccess) e = cudaMemset(ctx->ticket, 0, sizeof(unsigned int) * 4);
+  if (e == cudaSuccess) e = cudaMemset(ctx->keys, 0, sizeof(unsigned long long) * DX_MAX_M);
+  if (e == cudaSuccess) e = cudaMemset(ctx->dev_status, 0, sizeof(int32_t));
+  if (e == cudaSuccess) e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) {
+    dx_destroy(ctx);
+    return e == cudaErrorMemoryAllocation ? DX_ERR_OOM : DX_ERR_CUDA;
+  }
+  *out = ctx;
+  return DX_OK;
+}
+
+extern "C" dx_status dx_destroy(dx_ctx* ctx) {
+  if (!ctx) return DX_ERR_INVALID_ARG;
+  cudaFree(ctx->work);
+  cudaFree(ctx->xn);
+  cudaFree(ctx->z);
+  cudaFree(ctx->ticket);
+  cudaFree(ctx->keys);
+  cudaFree(ctx->dev_status);
+  delete ctx;
+  return DX_OK;
+}
+
+extern "C" dx_status dx_last_device_status(dx_ctx* ctx, void* stream, int32_t* out) {
+  if (!ctx || !out) return DX_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  DX_CUDA(ctx, cudaMemcpyAsync(out, ctx->dev_status, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+  DX_CUDA(ctx, cudaMemsetAsync(ctx->dev_status, 0, sizeof(int32_t), st));
+  DX_CUDA(ctx, cudaStreamSynchronize(st));
+  return DX_OK;
+}
+
+extern "C" int32_t dx_last_cuda_error(dx_ctx* ctx) { return ctx ? (int32_t)ctx->last_cuda : 0; }
+extern "C" int64_t dx_kernel_launches(dx_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+static dx_status check_desc(const dx_layer_desc* d) {
+  if (!d) return DX_ERR_INVALID_ARG;
+  if (d->hidden <= 0 || d->n_experts <= 0 || d->top_k <= 0 || d->inter <= 0 || d->n_shared < 0) return DX_ERR_SHAPE;
+  if (d->top_k > d->n_experts) return DX_ERR_SHAPE;
+  if (d->weight_dtype != DX_DTYPE_FP32 && d->weight_dtype != DX_DTYPE_BF16) return DX_ERR_INVALID_ARG;
+  if (d->score_fn != DX_SCORE_SOFTMAX && d->score_fn != DX_SCORE_SIGMOID) return DX_ERR_INVALID_ARG;
+  if (d->hidden > DX_MAX_H || d->hidden % 256 || d->n_experts > DX_MAX_E || d->top_k > DX_MAX_TOPK ||
+      d->n_shared > DX_MAX_SHARED)
+    return DX_ERR_UNSUPPORTED;
+  if (d->inter % DX_TILE_I || (d->n_shared && (d->shared_inter <= 0 || d->shared_inter % DX_TILE_I)) ||
+      d->draft_inter < 0 || d->draft_inter % DX_TILE_I)
+    return DX_ERR_UNSUPPORTED;
+  if (d->weight_dtype == DX_DTYPE_BF16 && !dx_bf16_hidden_supported(d->hidden)) return DX_ERR_UNSUPPORTED;
+  return DX_OK;
+}
+
+extern "C" dx_status dx_expert_blob_bytes(const dx_layer_desc* desc, int32_t inter, size_t* bytes_out) {
+  if (!desc || !bytes_out) return DX_ERR_INVALID_ARG;
+  if (inter <= 0 || inter % DX_TILE_I || desc->hidden <= 0 || desc->hidden % 256) return DX_ERR_UNSUPPORTED;
+  *bytes_out = (size_t)3 * desc->hidden * inter * (desc->weight_dtype == DX_DTYPE_BF16 ? 2 : 4);
+  return DX_OK;
+}
+
+extern "C" dx_status dx_pack_expert(dx_ctx* ctx, const dx_layer_desc* desc, int32_t inter, const void* Wg,
+                                    const void* Wu, const void* Wd, void* blob_out, void* stream) {
+  if (!ctx || !desc || !Wg || !Wu || !Wd || !blob_out) return DX_ERR_INVALID_ARG;
+  if (inter <= 0 || inter % DX_TILE_I || desc->hidden <= 0 || desc->hidden % 256) return DX_ERR_UNSUPPORTED;
+  if (((uintptr_t)blob_out) % 128) return DX_ERR_INVALID_ARG;
+  DX_CUDA(ctx, dx_launch_pack(desc->weight_dtype, desc->hidden, inter, Wg, Wu, Wd, blob_out, (cudaStream_t)stream));
+  ctx->launches++;
+  return DX_OK;
+}
+
+extern "C" dx_status dx_layer_create(dx_ctx* ctx, const dx_layer_desc* desc, dx_layer** out) {
+  if (!ctx || !out) return DX_ERR_INVALID_ARG;
+  *out = nullptr;
+  dx_status s = check_desc(desc);
+  if (s != DX_OK) return s;
+  dx_layer* L = new (std::nothrow) dx_layer();
+  if (!L) return DX_ERR_OOM;
+  L->ctx = ctx;
+  L->desc = *desc;
+  L->W_r = nullptr;
+  L->bias = nullptr;
+  L->table_len = desc->n_shared + 1 + desc->n_experts;
+  L->table_host = new (std::nothrow) const void*[L->table_len]();
+  L->table_dev = nullptr;
+  L->dirty = true;
+  L->cache = nullptr;
+  L->cache_layer = -1;
+  if (!L->table_host) { delete L; return DX_ERR_OOM; }
+  cudaError_t e = cudaMalloc((void**)&L->table_dev, sizeof(void*) * L->table_len);
+  if (e != cudaSuccess) {
+    ctx->last_cuda = e;
+    delete[] L->table_host;
+    delete L;
+    return DX_ERR_OOM;
+  }
+  *out = L;
+  return DX_OK;
+}
+
+extern "C" dx_status dx_layer_destroy(dx_layer* L) {
+  if (!L) return DX_ERR_INVALID_ARG;
+  cudaFree((void*)L->table_dev);
+  delete[] L->table_host;
+  delete L;
+  return DX_OK;
+}
+
+extern "C" dx_status dx_layer_set_router(dx_layer* L, const void* W_r, const float* bias) {
+  if (!L || !W_r) return DX_ERR_INVALID_ARG;
+  if (((uintptr_t)W_r) % 16 || ((uintptr_t)bias) % 4) return DX_ERR_INVALID_ARG;
+  L->W_r = W_r;
+  L->bias = bias;
+  return DX_OK;
+}
+
+static dx_status set_slot(dx_layer* L, int idx, const void* blob, bool allow_null) {
+  if (!blob && !allow_null) return DX_ERR_INVALID_ARG;
+  if (((uintptr_t)blob) % 128) return DX_ERR_INVALID_ARG;
+  L->table_host[idx] = blob;
+  L->dirty = true;
+  return DX_OK;
+}
+extern "C" dx_status dx_layer_set_shared(dx_layer* L, int32_t s, const void* blob) {
+  if (!L || s < 0 || s >= L->desc.n_shared) return DX_ERR_INVALID_ARG;
+  return set_slot(L, s, blob, false);
+}
+extern "C" dx_status dx_layer_set_draft(dx_layer* L, const void* blob) {
+  if (!L || L->desc.draft_inter <= 0) return DX_ERR_INVALID_ARG;
+  return set_slot(L, L->desc.n_shared, blob, false);
+}
+extern "C" dx_status dx_layer_set_expert(dx_layer* L, int32_t e, const void* blob) {
+  if (!L || e < 0 || e >= L->desc.n_experts) return DX_ERR_INVALID_ARG;
+  return set_slot(L, L->desc.n_shared + 1 + e, blob, true);
+}
+
+static dx_status upload_table(dx_layer* L, cudaStream_t st) {
+  if (!L->dirty) return DX_OK;
+  // pageable source: the runtime stages the bytes before returning, the copy itself is stream-ordered
+  DX_CUDA(L->ctx, cudaMemcpyAsync((void*)L->table_dev, L->table_host, sizeof(void*) * L->table_len,
+                                  cudaMemcpyHostToDevice, st));
+  L->dirty = false;
+  return DX_OK;
+}
+
+struct RouteOut {
+  int32_t* topk_ids;
+  float* topk_w;
+  uint64_t* union_mask;
+  int32_t* union_ids;
+  int32_t* union_count;
+  int32_t* offsets;
+  int32_t* perm;
+};
+
+static dx_status do_route(dx_layer* L, const float* h, int K, float* y, const RouteOut& o, bool draft, bool residual,
+                          cudaStream_t st) {
+  dx_ctx* ctx = L->ctx;
+  const dx_layer_desc& d = L->desc;
+  if (!h || !y) return DX_ERR_INVALID_ARG;
+  if (K < 1 || K > DX_MAX_K) return DX_ERR_UNSUPPORTED;
+  if (!L->W_r) return DX_ERR_NOT_RESIDENT;
+  for (int s = 0; s < d.n_shared; ++s)
+    if (!L->table_host[s]) return DX_ERR_NOT_RESIDENT;
+  if (draft && d.draft_inter > 0 && !L->table_host[d.n_shared]) return DX_ERR_NOT_RESIDENT;
+  if (((uintptr_t)h) % 16 || ((uintptr_t)y) % 16) return DX_ERR_INVALID_ARG;
+  dx_status s = upload_table(L, st);
+  if (s != DX_OK) return s;
+  DxRouteParams p{};
+  p.h = h; p.K = K; p.H = d.hidden; p.E = d.n_experts; p.k = d.top_k;
+  p.score_fn = d.score_fn; p.norm_topk = d.norm_topk; p.scale = d.routed_scale; p.gamma = d.draft_gamma;
+  p.W_r = L->W_r; p.bias = L->bias;
+  p.n_shared = d.n_shared;
+  p.shared_tiles = d.n_shared ? d.shared_inter / DX_TILE_I : 0;
+  p.routed_tiles = d.inter / DX_TILE_I;
+  p.draft_tiles = draft ? d.draft_inter / DX_TILE_I : 0;
+  p.draft_mode = draft ? 1 : 0;
+  p.top_r = 1;
+  p.rms_norm = residual ? 1 : 0;
+  p.accumulate = residual ? 1 : 0;
+  p.xn = ctx->xn; p.y = y; p.z = ctx->z; p.ticket = ctx->ticket; p.work = ctx->work; p.dev_status = ctx->dev_status;
+  p.topk_ids = o.topk_ids; p.topk_w = o.topk_w;
+  p.union_mask = (unsigned long long*)o.union_mask; p.union_ids = o.union_ids; p.union_count = o.union_count;
+  p.offsets = o.offsets; p.perm = o.perm;
+  DX_CUDA(ctx, dx_launch_route(p, d.weight_dtype, st));
+  ctx->launches++;
+  return DX_OK;
+}
+
+static dx_status do_experts(dx_layer* L, const float* h, int K, float* y, bool residual, cudaStream_t st) {
+  dx_ctx* ctx = L->ctx;
+  if (!h || !y) return DX_ERR_INVALID_ARG;
+  if (K < 1 || K > DX_MAX_K) return DX_ERR_UNSUPPORTED;
+  dx_status s = upload_table(L, st);
+  if (s != DX_OK) return s;
+  DxExpertParams p{};
+  p.x = residual ? ctx->xn : h;
+  p.y = y;
+  p.table = L->table_dev;
+  p.work = ctx->work;
+  p.dev_status = ctx->dev_status;
+  p.H = L->desc.hidden;
+  DX_CUDA(ctx, dx_launch_experts(ctx, p, L->desc.weight_dtype, K, st));
+  ctx->launches++;
+  if (L->cache) dx_cache_note_use(L->cache, L->cache_layer, st);
+  return DX_OK;
+}
+
+extern "C" dx_status moe_draft_step(dx_layer* L, const float* h, float* y, int32_t* topk_ids, float* topk_w,
+                                    void* stream) {
+  if (!L) return DX_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  RouteOut o{topk_ids, topk_w, nullptr, nullptr, nullptr, nullptr, nullptr};
+  dx_status s = do_route(L, h, 1, y, o, true, false, st);
+  if (s != DX_OK) return s;
+  return do_experts(L, h, 1, y, false, st);
+}
+
+extern "C" dx_status moe_draft_step_residual(dx_layer* L, float* h, int32_t* topk_ids, float* topk_w, void* stream) {
+  if (!L) return DX_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  RouteOut o{topk_ids, topk_w, nullptr, nullptr, nullptr, nullptr, nullptr};
+  dx_status s = do_route(L, h, 1, h, o, true, true, st);
+  if (s != DX_OK) return s;
+  return do_experts(L, h, 1, h, true, st);
+}
+
+extern "C" dx_status moe_verify_route(dx_layer* L, const float* h, int32_t K, float* y, int32_t* topk_ids,
+                                      float* topk_w, uint64_t* union_mask, int32_t* union_ids, int32_t* union_count,
+                                      int32_t* offsets, int32_t* perm, void* stream) {
+  if (!L) return DX_ERR_INVALID_ARG;
+  RouteOut o{topk_ids, topk_w, union_mask, union_ids, union_count, offsets, perm};
+  return do_route(L, h, K, y, o, false, false, (cudaStream_t)stream);
+}
+
+extern "C" dx_status moe_verify_experts(dx_layer* L, const float* h, int32_t K, float* y, void* stream) {
+  if (!L) return DX_ERR_INVALID_ARG;
+  return do_experts(L, h, K, y, false, (cudaStream_t)stream);
+}
+
+extern "C" dx_status moe_verify_block(dx_layer* L, const float* h, int32_t K, float* y, int32_t* topk_ids,
+                                      float* topk_w, uint64_t* union_mask, int32_t* union_ids, int32_t* union_count,
+                                      int32_t* offsets, int32_t* perm, void* stream) {
+  dx_status s = moe_verify_route(L, h, K, y, topk_ids, topk_w, union_mask, union_ids, union_count, offsets, perm,
+                                 stream);
+  if (s != DX_OK) return s;
+  return moe_verify_experts(L, h, K, y, stream);
+}
+
+extern "C" dx_status moe_verify_block_residual(dx_layer* L, float* h, int32_t K, int32_t* topk_ids, float* topk_w,
+                                               uint64_t* union_mask, int32_t* union_ids, int32_t* union_count,
+                                               int32_t* offsets, int32_t* perm, void* stream) {
+  if (!L) return DX_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  RouteOut o{topk_ids, topk_w, union_mask, union_ids, union_count, offsets, perm};
+  dx_status s = do_route(L, h, K, h, o, false, true, st);
+  if (s != DX_OK) return s;
+  return do_experts(L, h, K, h, true, st);
+}
+
+extern "C" dx_status spec_accept(dx_ctx* ctx, const float* h, int32_t M, const void* W_lm, int32_t V, int32_t H,
+                                 int32_t w_dtype, const int32_t* draft, int32_t K, int32_t rms_norm, int32_t* target,
+                                 int32_t* n_accept, int32_t* next_token, void* stream) {
+  if (!ctx || !h || !W_lm || !target || !n_accept || !next_token) return DX_ERR_INVALID_ARG;
+  if (K > 0 && !draft) return DX_ERR_INVALID_ARG;
+  if (M < 1 || V < 1 || K < 0) return DX_ERR_SHAPE;
+  if (w_dtype != DX_DTYPE_FP32 && w_dtype != DX_DTYPE_BF16) return DX_ERR_INVALID_ARG;
+  if (M > DX_MAX_M || K > DX_MAX_K || H <= 0 || H > DX_MAX_H || H % 256) return DX_ERR_UNSUPPORTED;
+  if (((uintptr_t)h) % 16 || ((uintptr_t)W_lm) % 16) return DX_ERR_INVALID_ARG;
+  if (w_dtype == DX_DTYPE_BF16) {
+    const size_t smem = (size_t)((M + 7) / 8) * H * 32;
+    if (smem > (size_t)ctx->smem_optin) return DX_ERR_UNSUPPORTED;
+  }
+  DX_CUDA(ctx, dx_launch_accept(ctx, h, M, W_lm, V, H, w_dtype, draft, K, rms_norm, target, n_accept, next_token,
+                                (cudaStream_t)stream));
+  ctx->launches++;
+  return DX_OK;
+}

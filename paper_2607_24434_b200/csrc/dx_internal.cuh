@@ -1,0 +1,128 @@
+// Internal declarations shared by the translation units of libdraftexpert.
+// Host-side handle structs, the device work list the routing kernel hands to
+// the expert kernels, and small device helpers.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "draftexpert.h"
+
+#define DX_MAX_K 16
+#define DX_MAX_E 256
+#define DX_MAX_TOPK 8
+#define DX_MAX_SHARED 8
+#define DX_MAX_H 8192
+#define DX_MAX_PAIRS (DX_MAX_K * DX_MAX_TOPK)
+#define DX_MAX_ENTRIES (DX_MAX_SHARED + 1 + DX_MAX_PAIRS)
+#define DX_TILE_I 8            // intermediate rows per streamed weight tile
+#define DX_MAX_M 16            // accept rows
+
+// One group of the grouped SwiGLU: an expert (by index into the layer's blob
+// table) together with the block tokens routed to it and their output weights.
+struct DxEntry {
+  int32_t table_index;   // index into the layer's device blob table
+  int32_t n_tiles;       // I / DX_TILE_I of this expert (0 = skip)
+  int32_t unit_begin;    // first global work-unit index of this entry
+  int32_t m;             // tokens in the group (<= K)
+  int32_t tok[DX_MAX_K]; // block row of each group token
+  float w[DX_MAX_K];     // weight of this expert's output in that row (g, 1 or gamma)
+};
+
+struct DxWork {
+  int32_t n_entries;
+  int32_t total_units;
+  int32_t K;
+  int32_t pad;
+  DxEntry entries[DX_MAX_ENTRIES];
+};
+
+struct dx_ctx {
+  int device;
+  int sm_count;
+  int smem_optin;
+  cudaError_t last_cuda;
+  int64_t launches;
+  // device scratch
+  DxWork* work;        // work list
+  float* xn;           // [DX_MAX_K, DX_MAX_H] normalised block
+  float* z;            // [DX_MAX_K, DX_MAX_E] router logits
+  unsigned int* ticket;        // last-CTA tickets (route, accept)
+  unsigned long long* keys;    // [DX_MAX_M] packed argmax keys
+  int32_t* dev_status;
+};
+
+struct dx_cache;
+
+struct dx_layer {
+  dx_ctx* ctx;
+  dx_layer_desc desc;
+  const void* W_r;
+  const float* bias;
+  // blob table: [0,n_shared) shared, [n_shared] draft, [n_shared+1, n_shared+1+E) routed
+  const void** table_host;
+  const void** table_dev;
+  int table_len;
+  bool dirty;
+  dx_cache* cache;
+  int cache_layer;
+};
+
+struct DxRouteParams {
+  const float* h;
+  int K, H, E, k;
+  int score_fn, norm_topk;
+  float scale, gamma;
+  const void* W_r;
+  const float* bias;
+  int n_shared, shared_tiles, routed_tiles, draft_tiles;
+  int draft_mode;   // 0: verify block, 1: drafter (shared + draft expert + top_r routed)
+  int top_r;
+  int rms_norm;     // 1: route and experts see RMSNorm(h)
+  int accumulate;   // 1: y is added to, not overwritten
+  float* xn;
+  float* y;
+  float* z;
+  unsigned int* ticket;
+  DxWork* work;
+  int32_t* dev_status;
+  int32_t* topk_ids;
+  float* topk_w;
+  unsigned long long* union_mask;
+  int32_t* union_ids;
+  int32_t* union_count;
+  int32_t* offsets;
+  int32_t* perm;
+};
+
+struct DxExpertParams {
+  const float* x;            // [K,H] block the experts see (h or the normalised copy)
+  float* y;                  // [K,H] accumulated into
+  const void* const* table;  // layer blob table (device)
+  const DxWork* work;
+  int32_t* dev_status;
+  int H;
+};
+
+// launchers (each returns the cudaError_t of the launch)
+cudaError_t dx_launch_route(const DxRouteParams& p, int weight_dtype, cudaStream_t st);
+cudaError_t dx_launch_experts(dx_ctx* ctx, const DxExpertParams& p, int weight_dtype, int K, cudaStream_t st);
+cudaError_t dx_launch_pack(int weight_dtype, int H, int I, const void* Wg, const void* Wu, const void* Wd,
+                           void* blob, cudaStream_t st);
+cudaError_t dx_launch_accept(dx_ctx* ctx, const float* h, int M, const void* W_lm, int V, int H, int w_dtype,
+                             const int32_t* draft, int K, int rms_norm, int32_t* target, int32_t* n_accept,
+                             int32_t* next_token, cudaStream_t st);
+cudaError_t dx_experts_prepare(dx_ctx* ctx);   // opt-in shared memory attributes, once per context
+
+// cache hooks used by the layer code
+const void** dx_cache_table(dx_cache* c, int layer);
+void dx_cache_note_use(dx_cache* c, int layer, cudaStream_t st);
+
+__device__ __forceinline__ float dx_silu(float x) { return x / (1.0f + expf(-x)); }
+
+// Monotone map from float to uint32 (larger float -> larger unsigned).
+__device__ __forceinline__ unsigned int dx_orderable(float f) {
+  unsigned int u = __float_as_uint(f);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
