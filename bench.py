@@ -1,0 +1,380 @@
+#!/usr/bin/env python
+"""Benchmark of the draft / verify MoE hot path on DeepSeek-V2-Lite-shaped synthetic layers.
+
+One *step* is one pass of the whole hot path over one block on one MoE layer:
+    moe_draft_step (1 token, Eq. 5)  ->  moe_verify_block (K tokens, Eq. 4 grouped by the expert union)
+    ->  spec_accept (greedy verification over the vocabulary).
+Steps rotate over independently seeded layers (default 8 x 1.16 GB of bf16 experts) so that no weight is
+ever re-read from L2 between timed iterations.
+
+Prints ONE JSON line (see README / DESIGN for the keys).  ``--impl reference`` times the CPU checker
+(``oracle/``) on the host cores on the same configuration instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2607_24434_b200 import synth
+
+METRIC = "verify_block_moe_tokens_per_s"
+UNIT = "tokens/s"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            return float(json.load(open(path))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index: int):
+        self.idx = device_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.idx}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            parts = [p.strip() for p in ln.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def build_workload(binding, ctx, shape, n_layers, K, V, seed0, device):
+    """Packed layers, hidden blocks, LM head and draft tokens, all resident on the GPU."""
+    layers, blocks, hosts = [], [], []
+    for i in range(n_layers):
+        w = synth.make_layer(shape, seed0 + i, device, zipf=True)
+        L = binding.Layer.from_weights(ctx, w)
+        torch.cuda.synchronize()
+        del w
+        layers.append(L)
+        blocks.append(synth.hidden_block(K, shape.hidden, seed0 + 100 + i, 0.0, device))
+    torch.cuda.empty_cache()
+    W_lm = synth.lm_head(V, shape.hidden, seed0 + 999, torch.bfloat16, device)
+    return layers, blocks, W_lm
+
+
+def run_gpu(args):
+    from paper_2607_24434_b200 import binding
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=device)
+
+    shape = synth.shape_v2lite()
+    K, V, NL = args.block, args.vocab, args.layers
+    ctx = binding.Context(local)
+    layers, blocks, W_lm = build_workload(binding, ctx, shape, NL, K, V, 1000 + 50 * rank, device)
+    H = shape.hidden
+    stream = torch.cuda.current_stream()
+
+    # persistent output buffers (one set per layer so results can be inspected afterwards)
+    rb = [binding._routing_buffers(shape, K, device) for _ in range(NL)]
+    ys = [torch.empty((K, H), device=device) for _ in range(NL)]
+    yd = torch.empty((1, H), device=device)
+    dbuf = {"topk_ids": torch.empty((shape.top_k,), dtype=torch.int32, device=device),
+            "topk_w": torch.empty((shape.top_k,), dtype=torch.float32, device=device)}
+    abuf = {"target": torch.empty((K,), dtype=torch.int32, device=device),
+            "n_accept": torch.empty((1,), dtype=torch.int32, device=device),
+            "next_token": torch.empty((1,), dtype=torch.int32, device=device)}
+    draft_tok = torch.zeros((K,), dtype=torch.int32, device=device)
+
+    def step(i):
+        li = i % NL
+        binding.moe_draft_step(layers[li], blocks[li][:1], yd, dbuf)
+        binding.moe_verify_block(layers[li], blocks[li], ys[li], rb[li])
+        binding.spec_accept(ctx, ys[li], W_lm, draft_tok, True, abuf)
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # draft tokens that agree with the target for a geometric(0.85) prefix (per layer 0's block)
+    step(0)
+    torch.cuda.synchronize()
+    tgt = abuf["target"].cpu().numpy()
+    draft_tok.copy_(torch.from_numpy(synth.draft_tokens_from_target(tgt, V, 7)).to(device))
+
+    for i in range(args.warmup):
+        step(i)
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    launches0 = ctx.kernel_launches()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(args.steps):
+        step(i)
+    e1.record(stream)
+    barrier()
+    launches = ctx.kernel_launches() - launches0
+    total_ms = e0.elapsed_time(e1)
+
+    # ---- per-kernel timing of the dominant kernel (grouped SwiGLU of the verify block) and the others
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    t_exp, t_route, t_draft, t_acc = [], [], [], []
+    for i in range(args.steps):
+        li = i % NL
+        a, b, c, d, e, f = ev(), ev(), ev(), ev(), ev(), ev()
+        a.record(stream)
+        binding.moe_draft_step(layers[li], blocks[li][:1], yd, dbuf)
+        b.record(stream)
+        binding.moe_verify_route(layers[li], blocks[li], ys[li], rb[li])
+        c.record(stream)
+        binding.moe_verify_experts(layers[li], blocks[li], ys[li])
+        d.record(stream)
+        binding.spec_accept(ctx, ys[li], W_lm, draft_tok, True, abuf)
+        e.record(stream)
+        t_exp.append((c, d, li)); t_route.append((b, c)); t_draft.append((a, b)); t_acc.append((d, e))
+    torch.cuda.synchronize()
+    clocks = sampler.stop() if rank == 0 else None
+    union = [int(rb[li]["union_count"].item()) for li in range(NL)]
+    exp_bytes = shape.expert_bytes()
+    exp_ms = [x.elapsed_time(y) for x, y, _ in t_exp]
+    exp_alg = [(union[li] + shape.n_shared) * exp_bytes + 2 * K * H * 4 for _, _, li in t_exp]
+    verify_gbs = sum(exp_alg) / (sum(exp_ms) * 1e-3) / 1e9
+    draft_ms = float(np.mean([x.elapsed_time(y) for x, y in t_draft]))
+    route_ms = float(np.mean([x.elapsed_time(y) for x, y in t_route]))
+    acc_ms = float(np.mean([x.elapsed_time(y) for x, y in t_acc]))
+    draft_bytes = (shape.n_shared + 2) * exp_bytes + shape.n_experts * H * 2
+    acc_bytes = V * H * 2
+
+    # ---- end to end through the binding with host buffers (pinned), copies inside the timed region
+    h_host = [b.cpu().pin_memory() for b in blocks]
+    d_host = draft_tok.cpu().pin_memory()
+    y_host = torch.empty((K, H), dtype=torch.float32).pin_memory()
+    res_host = torch.empty((2,), dtype=torch.int32).pin_memory()
+    tgt_host = torch.empty((K,), dtype=torch.int32).pin_memory()
+    h_dev = torch.empty((K, H), device=device)
+    d_dev = torch.empty((K,), dtype=torch.int32, device=device)
+
+    def e2e_step(i):
+        li = i % NL
+        h_dev.copy_(h_host[li], non_blocking=True)
+        d_dev.copy_(d_host, non_blocking=True)
+        binding.moe_draft_step(layers[li], h_dev[:1], yd, dbuf)
+        binding.moe_verify_block(layers[li], h_dev, ys[li], rb[li])
+        binding.spec_accept(ctx, ys[li], W_lm, d_dev, True, abuf)
+        y_host.copy_(ys[li], non_blocking=True)
+        tgt_host.copy_(abuf["target"], non_blocking=True)
+        res_host[0:1].copy_(abuf["n_accept"], non_blocking=True)
+        res_host[1:2].copy_(abuf["next_token"], non_blocking=True)
+        stream.synchronize()
+
+    for i in range(max(3, args.warmup)):
+        e2e_step(i)
+    barrier()
+    g0, g1 = ev(), ev()
+    g0.record(stream)
+    for i in range(args.steps):
+        e2e_step(i)
+    g1.record(stream)
+    barrier()
+    e2e_ms = g0.elapsed_time(g1)
+
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([total_ms, e2e_ms], device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms, e2e_ms = float(t[0]), float(t[1])
+        lt = torch.tensor([launches], device=device)
+        dist.all_reduce(lt)
+        launches = int(lt[0])
+
+    if rank != 0:
+        if world > 1:
+            torch.distributed.destroy_process_group()
+        return
+    peak, peak_kind = measured_peaks()
+    value = world * K * args.steps / (total_ms * 1e-3)
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16 weights, fp32 accumulate", "data": "synthetic",
+        "config": {"workload": "configs[1]: DeepSeek-V2-Lite-shaped MoE layer (H 2048, 64 experts x 1408, top-6, "
+                               "2 shared + 1 draft expert, Zipf(1.1) router bias); step = draft step (1 token) + "
+                               f"verify block K={K} + greedy accept over vocab {V}",
+                   "block_tokens": K, "vocab": V, "layers_rotated": NL,
+                   "l2": f"inputs larger than L2: steps rotate over {NL} independently seeded layers "
+                         f"({NL * (shape.n_experts + shape.n_shared + 1) * exp_bytes / 1e9:.1f} GB of weights)",
+                   "parallelism": "replicas only" if world > 1 else "single GPU"},
+        "gpu_launches": launches,
+        "e2e": {"value": world * K * args.steps / (e2e_ms * 1e-3), "unit": UNIT,
+                "h2d_bytes_per_step": K * H * 4 + K * 4, "d2h_bytes_per_step": K * H * 4 + K * 4 + 8,
+                "ms_per_step": e2e_ms / args.steps},
+        "roofline": {"kernel": "dx_experts_bf16_kernel (grouped SwiGLU of the verify block)", "bound": "hbm",
+                     "achieved": verify_gbs, "peak": peak, "unit": "GB/s", "frac": verify_gbs / peak,
+                     "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBs": verify_gbs / NOMINAL_HBM_GBS,
+                     "traffic": args.traffic, "ms_per_launch": float(np.mean(exp_ms)),
+                     "algorithmic_bytes_per_launch": float(np.mean(exp_alg)), "union_sizes": union},
+        "kernels": {"verify_experts_ms": float(np.mean(exp_ms)), "verify_route_ms": route_ms,
+                    "verify_tokens_per_s": K / ((float(np.mean(exp_ms)) + route_ms) * 1e-3),
+                    "draft_step_us": draft_ms * 1e3, "draft_gbs": draft_bytes / (draft_ms * 1e-3) / 1e9,
+                    "draft_frac_of_peak": draft_bytes / (draft_ms * 1e-3) / 1e9 / peak,
+                    "accept_ms": acc_ms, "accept_gbs": acc_bytes / (acc_ms * 1e-3) / 1e9,
+                    "accept_frac_of_peak": acc_bytes / (acc_ms * 1e-3) / 1e9 / peak},
+        "clocks": clocks,
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        out["cpu_baseline"] = cpu_baseline(shape, K, V, sample_vocab=args.cpu_vocab)
+    print(json.dumps(out))
+    if world > 1:
+        torch.distributed.destroy_process_group()
+
+
+def _blas_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        return max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def oracle_step(O, ref, h_np, W_np, draft, K):
+    """The same step on the CPU checker, as it stands: draft step, verify block, greedy accept."""
+    O.moe_draft(h_np[:1], ref)
+    y = O.moe_target(h_np, ref)[0]
+    return O.greedy_accept_fast(O.rmsnorm(y), W_np, draft)
+
+
+def cpu_baseline(shape, K, V, sample_vocab):
+    """Times the CPU checker on a bounded sample of the workload: one layer, one block, a vocabulary slice."""
+    from oracle import moe_oracle as O
+    layer = synth.make_layer(shape, 4242, "cpu", zipf=True)
+    ref = synth.layer_to_numpy(layer)
+    h_np = synth.hidden_block(K, shape.hidden, 4243, 0.0).numpy().astype(np.float64)
+    W_np = synth.to_numpy_f32(synth.lm_head(sample_vocab, shape.hidden, 4244, torch.bfloat16))
+    draft = np.zeros(K, np.int32)
+    t0 = time.perf_counter()
+    oracle_step(O, ref, h_np, W_np, draft, K)
+    dt = time.perf_counter() - t0
+    return {"value": K / dt, "unit": UNIT, "cores": _blas_threads(), "kind": "oracle",
+            "seconds": dt,
+            "sample": f"one step on one layer: draft step + verify block K={K} + greedy accept over the first "
+                      f"{sample_vocab} vocabulary rows (fp64 numpy)"}
+
+
+def run_reference(args):
+    """The reference arm: the CPU checker, as it stands, on the host cores (rank 0 only)."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    from oracle import moe_oracle as O
+    shape = synth.shape_v2lite()
+    K, V = args.block, args.cpu_vocab
+    n_layers = 1
+    refs = [synth.layer_to_numpy(synth.make_layer(shape, 1000 + i, "cpu", zipf=True)) for i in range(n_layers)]
+    hs = [synth.hidden_block(K, shape.hidden, 1100 + i, 0.0).numpy().astype(np.float64) for i in range(n_layers)]
+    W_np = synth.to_numpy_f32(synth.lm_head(V, shape.hidden, 1999, torch.bfloat16))
+    draft = np.zeros(K, np.int32)
+    for i in range(args.warmup):
+        oracle_step(O, refs[i % n_layers], hs[i % n_layers], W_np, draft, K)
+    t0 = time.perf_counter()
+    for i in range(args.steps):
+        oracle_step(O, refs[i % n_layers], hs[i % n_layers], W_np, draft, K)
+    dt = time.perf_counter() - t0
+    value = K * args.steps / dt
+    sample = (f"each step: draft step + verify block K={K} on one of {n_layers} layers + greedy accept over the "
+              f"first {V} vocabulary rows (fp64 numpy)")
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": int(os.environ.get(
+            "WORLD_SIZE", "1")), "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "configs[1]: DeepSeek-V2-Lite-shaped MoE layer; step = draft step + verify block "
+                               f"K={K} + greedy accept", "block_tokens": K, "vocab": V},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": _blas_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=40)
+    ap.add_argument("--warmup", type=int, default=8)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--block", type=int, default=4, help="verify block length K")
+    ap.add_argument("--vocab", type=int, default=102400)
+    ap.add_argument("--layers", type=int, default=8, help="independently seeded layers to rotate over")
+    ap.add_argument("--cpu-vocab", type=int, default=16384, help="vocabulary rows in the CPU-baseline sample")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--traffic", type=float, default=None,
+                    help="ncu DRAM bytes per launch of the dominant kernel, if known")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -94,29 +94,46 @@ __device__ __forceinline__ int find_entry(const DxWork* W, int n_entries, int u,
 }
 
 // ----------------------------------------------------- bf16 tensor-core path
+// Streaming layout.  A unit (8 gate rows, 8 up rows, 8 down columns; 48*H bytes)
+// is stored as eight equal "chunks", one per consumer warp: chunk w holds the
+// gate/up fragments of contraction steps [w*H/128, (w+1)*H/128) followed by the
+// down-projection fragments of output row tiles [w*H/128, (w+1)*H/128).  A chunk
+// is one bulk copy, one ring slot, one full/empty mbarrier pair, and is read by
+// exactly one warp, so slots recycle warp by warp and the producer can run
+// more than two units ahead of the consumers.
 constexpr int kConsumerWarps = 8;
 constexpr int kThreads = (kConsumerWarps + 1) * 32;
+constexpr int kMaxSlots = 24;
 
 struct SmemHeader {
-  unsigned long long full[8];
-  unsigned long long empty[8];
+  unsigned long long full[kMaxSlots];
+  unsigned long long empty[kMaxSlots];
   int abort_flag;
-  int pad[31];
+  int n_entries;
+  int pad[2];
+  int e_begin[DX_MAX_ENTRIES];       // first unit of each entry
+  int e_tiles[DX_MAX_ENTRIES];
+  int e_m[DX_MAX_ENTRIES];
+  const unsigned char* e_blob[DX_MAX_ENTRIES];
 };
 
 template <int H, int NT>
-__global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertParams p, int n_stages) {
-  constexpr int KW = H / 128;        // phase-1 k-steps per consumer warp
+__global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertParams p, int n_slots) {
+  constexpr int KW = H / 128;        // phase-1 contraction steps per consumer warp
   constexpr int PW = H / 256;        // phase-2 row-tile pairs per consumer warp
   constexpr int KSTEPS = H / 16;
-  constexpr uint32_t STAGE_BYTES = 16u * H;   // a third of a unit
-  constexpr uint32_t UNIT_BYTES = 48u * H;
+  constexpr uint32_t CHUNK_A = KW * 512u, CHUNK_D = PW * 512u, CHUNK = CHUNK_A + CHUNK_D;
+  constexpr uint32_t UNIT_BYTES = 8u * CHUNK;
+  constexpr bool kRegB = (NT == 1);  // token fragments live in registers (else in shared memory)
 
   extern __shared__ __align__(128) unsigned char smem[];
   SmemHeader* hdr = reinterpret_cast<SmemHeader*>(smem);
-  float4* partial = reinterpret_cast<float4*>(smem + sizeof(SmemHeader));                // [2][8][NT][32]
-  uint4* bfrag = reinterpret_cast<uint4*>(smem + sizeof(SmemHeader) + 2 * 8 * NT * 32 * 16);  // [NT][KSTEPS][32]
-  unsigned char* ring = reinterpret_cast<unsigned char*>(bfrag) + (size_t)NT * KSTEPS * 32 * 16;
+  constexpr size_t HDR = (sizeof(SmemHeader) + 127) / 128 * 128;
+  float4* partial = reinterpret_cast<float4*>(smem + HDR);                         // [2][8][NT][32]
+  constexpr size_t PART = (size_t)2 * 8 * NT * 32 * 16;
+  uint4* bfrag = reinterpret_cast<uint4*>(smem + HDR + PART);                       // [NT][KSTEPS][32] if !kRegB
+  constexpr size_t BF = kRegB ? 0 : (size_t)NT * KSTEPS * 32 * 16;
+  unsigned char* ring = smem + HDR + PART + BF;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const DxWork* W = p.work;
@@ -127,12 +144,21 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
   volatile int* abort_flag = &hdr->abort_flag;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < n_stages; ++s) {
+    for (int s = 0; s < n_slots; ++s) {
       mbar_init(smem_u32(&hdr->full[s]), 1);
-      mbar_init(smem_u32(&hdr->empty[s]), kConsumerWarps);
+      mbar_init(smem_u32(&hdr->empty[s]), 1);
     }
     hdr->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  for (int i = threadIdx.x; i < n_entries; i += kThreads) {
+    const DxEntry& en = W->entries[i];
+    const unsigned char* blob = reinterpret_cast<const unsigned char*>(p.table[en.table_index]);
+    hdr->e_begin[i] = en.unit_begin;
+    hdr->e_tiles[i] = en.n_tiles;
+    hdr->e_m[i] = en.m;
+    hdr->e_blob[i] = blob;
+    if (blob == nullptr && en.n_tiles > 0) atomicExch(p.dev_status, DX_DEV_BAD_EXPERT_ID);
   }
   __syncthreads();
   if (u_lo >= u_hi) return;
@@ -140,29 +166,30 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
   if (warp == kConsumerWarps) {
     // ------------------------------------------------------------ producer
     if (lane == 0) {
-      int ei = 0;
-      uint32_t it = 0;
-      for (int u = u_lo; u < u_hi; ++u) {
-        ei = find_entry(W, n_entries, u, ei);
-        const DxEntry& en = W->entries[ei];
-        const unsigned char* blob = reinterpret_cast<const unsigned char*>(p.table[en.table_index]);
-        if (blob == nullptr) continue;
-        const unsigned char* src = blob + (size_t)(u - en.unit_begin) * UNIT_BYTES;
+      uint32_t it = 0;   // chunk counter
+      for (int e = 0; e < n_entries; ++e) {
+        const int b = hdr->e_begin[e], nt = hdr->e_tiles[e];
+        const int lo = max(b, u_lo), hi = min(b + nt, u_hi);
+        const unsigned char* blob = hdr->e_blob[e];
+        if (lo >= hi || blob == nullptr) continue;
+        for (int u = lo; u < hi; ++u) {
+          const unsigned char* src = blob + (size_t)(u - b) * UNIT_BYTES;
 #pragma unroll 1
-        for (int part = 0; part < 3; ++part, ++it) {
-          const uint32_t s = it % (uint32_t)n_stages, ph = (it / (uint32_t)n_stages) & 1u;
-          mbar_wait(smem_u32(&hdr->empty[s]), ph ^ 1u, abort_flag);
-          const uint32_t fb = smem_u32(&hdr->full[s]);
-          mbar_arrive_expect_tx(fb, STAGE_BYTES);
-          bulk_g2s(smem_u32(ring + (size_t)s * STAGE_BYTES), src + (size_t)part * STAGE_BYTES, STAGE_BYTES, fb);
+          for (int w = 0; w < kConsumerWarps; ++w, ++it) {
+            const uint32_t s = it % (uint32_t)n_slots, ph = (it / (uint32_t)n_slots) & 1u;
+            mbar_wait(smem_u32(&hdr->empty[s]), ph ^ 1u, abort_flag);
+            const uint32_t fb = smem_u32(&hdr->full[s]);
+            mbar_arrive_expect_tx(fb, CHUNK);
+            bulk_g2s(smem_u32(ring + (size_t)s * CHUNK), src + (size_t)w * CHUNK, CHUNK, fb);
+          }
         }
       }
       if (*abort_flag) {
         // something gave up: make sure no copy is still landing in this CTA's
         // shared memory before it is released (bounded, ignores the flag)
-        const uint32_t n_back = it < (uint32_t)n_stages ? it : (uint32_t)n_stages;
-        for (uint32_t b = 1; b <= n_back; ++b) {
-          const uint32_t j = it - b, s = j % (uint32_t)n_stages, ph = (j / (uint32_t)n_stages) & 1u;
+        const uint32_t n_back = it < (uint32_t)n_slots ? it : (uint32_t)n_slots;
+        for (uint32_t k = 1; k <= n_back; ++k) {
+          const uint32_t j = it - k, s = j % (uint32_t)n_slots, ph = (j / (uint32_t)n_slots) & 1u;
           for (uint32_t spin = 0; spin < DX_WAIT_LIMIT; ++spin)
             if (mbar_try_wait(smem_u32(&hdr->full[s]), ph)) break;
         }
@@ -181,153 +208,159 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
     for (int j = 0; j < 2 * PW; ++j)
 #pragma unroll
       for (int r = 0; r < 4; ++r) acc[nt][j][r] = 0.f;
+  // register-resident token fragments: for contraction step i of this warp,
+  // {hi(k0,k1), hi(k2,k3), lo(k0,k1), lo(k2,k3)} of token slot g
+  uint32_t breg[kRegB ? KW : 1][4];
 
-  int ei = -1, cur_m = 0;
-  uint32_t it = 0;
+  uint32_t uc = 0;   // units consumed by this CTA so far
   int buf = 0;
+  // partial-exchange source lanes: lane (g,c) ends up holding the sums of rows i = 2c and 2c+1 for token g
+  const int src0 = (2 * c) * 4 + (g >> 1), src1 = src0 + 4;
+  const bool odd = g & 1;
 
-  auto flush = [&](int e_idx) {
-    const DxEntry& en = W->entries[e_idx];
+  for (int e = 0; e < n_entries; ++e) {
+    const int eb = hdr->e_begin[e], etiles = hdr->e_tiles[e];
+    const int lo = max(eb, u_lo), hi = min(eb + etiles, u_hi);
+    if (lo >= hi || hdr->e_blob[e] == nullptr) continue;
+    const DxEntry& en = W->entries[e];
+    const int m = hdr->e_m[e];
+
+    // ---- token fragments of this group
+    if constexpr (kRegB) {
+      const bool valid = g < m;
+      const float* xrow = p.x + (size_t)(valid ? en.tok[g] : 0) * H + 4 * c;
 #pragma unroll
-    for (int nt = 0; nt < NT; ++nt) {
-      const int s0 = nt * 8 + 2 * c, s1 = s0 + 1;
-      const bool v0 = s0 < en.m, v1 = s1 < en.m;
-      if (!v0) continue;
-      const float w0 = en.w[s0], w1 = v1 ? en.w[s1] : 0.f;
-      float* y0 = p.y + (size_t)en.tok[s0] * H;
-      float* y1 = v1 ? p.y + (size_t)en.tok[s1] * H : nullptr;
-#pragma unroll
-      for (int j = 0; j < 2 * PW; ++j) {
-        const int hh = (warp * 2 * PW + j) * 16 + g;
-        atomicAdd(y0 + hh, w0 * acc[nt][j][0]);
-        atomicAdd(y0 + hh + 8, w0 * acc[nt][j][2]);
-        if (v1) {
-          atomicAdd(y1 + hh, w1 * acc[nt][j][1]);
-          atomicAdd(y1 + hh + 8, w1 * acc[nt][j][3]);
-        }
+      for (int i = 0; i < KW; ++i) {
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (valid) v = *reinterpret_cast<const float4*>(xrow + 16 * (warp * KW + i));
+        __nv_bfloat16 h0, h1, h2, h3, l0, l1, l2, l3;
+        split_bf16(v.x, h0, l0); split_bf16(v.y, h1, l1); split_bf16(v.z, h2, l2); split_bf16(v.w, h3, l3);
+        breg[i][0] = pack2(h0, h1); breg[i][1] = pack2(h2, h3);
+        breg[i][2] = pack2(l0, l1); breg[i][3] = pack2(l2, l3);
       }
-    }
-#pragma unroll
-    for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-      for (int j = 0; j < 2 * PW; ++j)
-#pragma unroll
-        for (int r = 0; r < 4; ++r) acc[nt][j][r] = 0.f;
-  };
-
-  for (int u = u_lo; u < u_hi; ++u) {
-    const int ne = find_entry(W, n_entries, u, ei < 0 ? 0 : ei);
-    if (ne != ei) {
-      if (ei >= 0 && cur_m > 0) flush(ei);
-      ei = ne;
-      const DxEntry& en = W->entries[ei];
-      const bool present = p.table[en.table_index] != nullptr;
-      if (!present && threadIdx.x == 0) atomicExch(p.dev_status, DX_DEV_BAD_EXPERT_ID);
-      cur_m = present ? en.m : 0;
-      if (cur_m > 0) {
-        // token fragments of this group: lane (g,c) of k-step ks holds, for
-        // token slot nt*8+g, columns 16ks+4c..+3 as {hi01, hi23, lo01, lo23}
-        for (int idx = threadIdx.x; idx < NT * KSTEPS * 32; idx += kConsumerWarps * 32) {
-          const int l = idx & 31, ks = (idx >> 5) % KSTEPS, nt = idx / (32 * KSTEPS);
-          const int slot = nt * 8 + (l >> 2);
-          uint4 o = make_uint4(0u, 0u, 0u, 0u);
-          if (slot < cur_m) {
-            const float4 v =
-                *reinterpret_cast<const float4*>(p.x + (size_t)en.tok[slot] * H + 16 * ks + 4 * (l & 3));
-            __nv_bfloat16 h0, h1, h2, h3, l0, l1, l2, l3;
-            split_bf16(v.x, h0, l0); split_bf16(v.y, h1, l1); split_bf16(v.z, h2, l2); split_bf16(v.w, h3, l3);
-            o = make_uint4(pack2(h0, h1), pack2(h2, h3), pack2(l0, l1), pack2(l2, l3));
-          }
-          bfrag[idx] = o;
+    } else {
+      consumer_bar();   // everyone is done reading the previous group's fragments
+      for (int idx = threadIdx.x; idx < NT * KSTEPS * 32; idx += kConsumerWarps * 32) {
+        const int l = idx & 31, ks = (idx >> 5) % KSTEPS, nt = idx / (32 * KSTEPS);
+        const int slot = nt * 8 + (l >> 2);
+        uint4 o = make_uint4(0u, 0u, 0u, 0u);
+        if (slot < m) {
+          const float4 v = *reinterpret_cast<const float4*>(p.x + (size_t)en.tok[slot] * H + 16 * ks + 4 * (l & 3));
+          __nv_bfloat16 h0, h1, h2, h3, l0, l1, l2, l3;
+          split_bf16(v.x, h0, l0); split_bf16(v.y, h1, l1); split_bf16(v.z, h2, l2); split_bf16(v.w, h3, l3);
+          o = make_uint4(pack2(h0, h1), pack2(h2, h3), pack2(l0, l1), pack2(l2, l3));
         }
+        bfrag[idx] = o;
       }
       consumer_bar();
     }
-    if (cur_m == 0) continue;   // expert without weights: the producer skipped this unit too
 
-    // ---- phase 1: [8 gate rows ; 8 up rows] x tokens, k split over the warps
-    const uint32_t itA = it + (warp >> 2);
-    {
-      const uint32_t s = itA % (uint32_t)n_stages, ph = (itA / (uint32_t)n_stages) & 1u;
+    for (int u = lo; u < hi; ++u, ++uc) {
+      const uint32_t it = uc * kConsumerWarps + warp;
+      const uint32_t s = it % (uint32_t)n_slots, ph = (it / (uint32_t)n_slots) & 1u;
+      const uint4* A = reinterpret_cast<const uint4*>(ring + (size_t)s * CHUNK) + lane;
       mbar_wait(smem_u32(&hdr->full[s]), ph, abort_flag);
-      const uint4* A = reinterpret_cast<const uint4*>(ring + (size_t)s * STAGE_BYTES) + (warp & 3) * KW * 32 + lane;
-      float cacc[NT][2][4];
+
+      // ---- phase 1: [8 gate rows ; 8 up rows] x tokens over this warp's slice of the contraction
+      float ch[NT][2][4], cl[NT][2][4];
 #pragma unroll
       for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-        for (int r = 0; r < 4; ++r) cacc[nt][0][r] = cacc[nt][1][r] = 0.f;
+        for (int r = 0; r < 4; ++r) ch[nt][0][r] = ch[nt][1][r] = cl[nt][0][r] = cl[nt][1][r] = 0.f;
 #pragma unroll
       for (int i = 0; i < KW; ++i) {
         const uint4 a = A[i * 32];
+        if constexpr (kRegB) {
+          mma_k16(ch[0][i & 1], a, breg[i][0], breg[i][1]);
+          mma_k16(cl[0][i & 1], a, breg[i][2], breg[i][3]);
+        } else {
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt) {
-          if (nt > 0 && cur_m <= 8 * nt) continue;
-          const uint4 b = bfrag[(nt * KSTEPS + warp * KW + i) * 32 + lane];
-          mma_k16(cacc[nt][i & 1], a, b.x, b.y);
-          mma_k16(cacc[nt][i & 1], a, b.z, b.w);
+          for (int nt = 0; nt < NT; ++nt) {
+            if (nt > 0 && m <= 8 * nt) continue;
+            const uint4 b = bfrag[(nt * KSTEPS + warp * KW + i) * 32 + lane];
+            mma_k16(ch[nt][i & 1], a, b.x, b.y);
+            mma_k16(cl[nt][i & 1], a, b.z, b.w);
+          }
         }
       }
-      __syncwarp();
-      if (lane == 0) {
-        mbar_arrive(smem_u32(&hdr->empty[it % (uint32_t)n_stages]));
-        mbar_arrive(smem_u32(&hdr->empty[(it + 1) % (uint32_t)n_stages]));
-      }
+      // re-fragment: C holds (gate|up row g, tokens 2c,2c+1); phase 2 wants rows (2c,2c+1) of token g
 #pragma unroll
-      for (int nt = 0; nt < NT; ++nt)
+      for (int nt = 0; nt < NT; ++nt) {
+        float v[4];
+#pragma unroll
+        for (int r = 0; r < 4; ++r) v[r] = (ch[nt][0][r] + ch[nt][1][r]) + (cl[nt][0][r] + cl[nt][1][r]);
+        const float a0 = __shfl_sync(0xffffffffu, v[0], src0), a1 = __shfl_sync(0xffffffffu, v[1], src0);
+        const float a2 = __shfl_sync(0xffffffffu, v[2], src0), a3 = __shfl_sync(0xffffffffu, v[3], src0);
+        const float b0 = __shfl_sync(0xffffffffu, v[0], src1), b1 = __shfl_sync(0xffffffffu, v[1], src1);
+        const float b2 = __shfl_sync(0xffffffffu, v[2], src1), b3 = __shfl_sync(0xffffffffu, v[3], src1);
         partial[((buf * 8 + warp) * NT + nt) * 32 + lane] =
-            make_float4(cacc[nt][0][0] + cacc[nt][1][0], cacc[nt][0][1] + cacc[nt][1][1],
-                        cacc[nt][0][2] + cacc[nt][1][2], cacc[nt][0][3] + cacc[nt][1][3]);
-    }
-    consumer_bar();
-
-    // ---- reduce the k-split partials, activation, re-fragment for phase 2:
-    // lane (g,c) needs act[i = 2c, 2c+1][token slot g] which sits in source
-    // lane (i*4 + g/2), component g&1 (gate) / 2+(g&1) (up)
-    uint32_t bhi[NT], blo[NT];
-#pragma unroll
-    for (int nt = 0; nt < NT; ++nt) {
-      float G0 = 0.f, U0 = 0.f, G1 = 0.f, U1 = 0.f;
-      const int src0 = (2 * c) * 4 + (g >> 1), src1 = src0 + 4;
-#pragma unroll
-      for (int w = 0; w < 8; ++w) {
-        const float4 v0 = partial[((buf * 8 + w) * NT + nt) * 32 + src0];
-        const float4 v1 = partial[((buf * 8 + w) * NT + nt) * 32 + src1];
-        G0 += (g & 1) ? v0.y : v0.x; U0 += (g & 1) ? v0.w : v0.z;
-        G1 += (g & 1) ? v1.y : v1.x; U1 += (g & 1) ? v1.w : v1.z;
+            make_float4(odd ? a1 : a0, odd ? a3 : a2, odd ? b1 : b0, odd ? b3 : b2);
       }
-      const float a0 = dx_silu(G0) * U0, a1 = dx_silu(G1) * U1;
-      __nv_bfloat16 h0, l0, h1, l1;
-      split_bf16(a0, h0, l0);
-      split_bf16(a1, h1, l1);
-      bhi[nt] = pack2(h0, h1);
-      blo[nt] = pack2(l0, l1);
-    }
-    buf ^= 1;
+      consumer_bar();
 
-    // ---- phase 2: 8 columns of W_d x activations, output rows split over the warps
-    {
-      const uint32_t itD = it + 2;
-      const uint32_t s = itD % (uint32_t)n_stages, ph = (itD / (uint32_t)n_stages) & 1u;
-      mbar_wait(smem_u32(&hdr->full[s]), ph, abort_flag);
-      const uint4* D = reinterpret_cast<const uint4*>(ring + (size_t)s * STAGE_BYTES) + warp * PW * 32 + lane;
+      // ---- sum the eight slices, activation, phase-2 token fragment
+      uint32_t bhi[NT], blo[NT];
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) {
+        float4 t = partial[((buf * 8 + 0) * NT + nt) * 32 + lane];
+#pragma unroll
+        for (int w = 1; w < 8; ++w) {
+          const float4 q = partial[((buf * 8 + w) * NT + nt) * 32 + lane];
+          t.x += q.x; t.y += q.y; t.z += q.z; t.w += q.w;
+        }
+        const float a0 = dx_silu(t.x) * t.y, a1 = dx_silu(t.z) * t.w;
+        __nv_bfloat16 h0, l0, h1, l1;
+        split_bf16(a0, h0, l0);
+        split_bf16(a1, h1, l1);
+        bhi[nt] = pack2(h0, h1);
+        blo[nt] = pack2(l0, l1);
+      }
+      buf ^= 1;
+
+      // ---- phase 2: 8 columns of W_d x activations for this warp's output rows
+      const uint4* D = A + KW * 32;
 #pragma unroll
       for (int q = 0; q < PW; ++q) {
         const uint4 a = D[q * 32];
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
-          if (nt > 0 && cur_m <= 8 * nt) continue;
+          if (nt > 0 && m <= 8 * nt) continue;
           mma_k8(acc[nt][2 * q], a.x, a.y, bhi[nt]);
-          mma_k8(acc[nt][2 * q], a.x, a.y, blo[nt]);
           mma_k8(acc[nt][2 * q + 1], a.z, a.w, bhi[nt]);
+          mma_k8(acc[nt][2 * q], a.x, a.y, blo[nt]);
           mma_k8(acc[nt][2 * q + 1], a.z, a.w, blo[nt]);
         }
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&hdr->empty[s]));
     }
-    it += 3;
+
+    // ---- add this group's partial output rows to y (scaled by each token's weight), reset
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+      const int s0 = nt * 8 + 2 * c, s1 = s0 + 1;
+      const bool v0 = s0 < m, v1 = s1 < m;
+      if (v0) {
+        const float w0 = en.w[s0], w1 = v1 ? en.w[s1] : 0.f;
+        float* y0 = p.y + (size_t)en.tok[s0] * H;
+        float* y1 = p.y + (size_t)(v1 ? en.tok[s1] : 0) * H;
+#pragma unroll
+        for (int j = 0; j < 2 * PW; ++j) {
+          const int hh = (warp * 2 * PW + j) * 16 + g;
+          atomicAdd(y0 + hh, w0 * acc[nt][j][0]);
+          atomicAdd(y0 + hh + 8, w0 * acc[nt][j][2]);
+          if (v1) {
+            atomicAdd(y1 + hh, w1 * acc[nt][j][1]);
+            atomicAdd(y1 + hh + 8, w1 * acc[nt][j][3]);
+          }
+        }
+      }
+#pragma unroll
+      for (int j = 0; j < 2 * PW; ++j)
+#pragma unroll
+        for (int r = 0; r < 4; ++r) acc[nt][j][r] = 0.f;
+    }
   }
-  if (ei >= 0 && cur_m > 0) flush(ei);
   if (*abort_flag && threadIdx.x == 0) atomicExch(p.dev_status, DX_DEV_WAIT_EXPIRED);
 }
 
@@ -384,29 +417,30 @@ __global__ void __launch_bounds__(256) dx_experts_fp32_kernel(DxExpertParams p) 
 }
 
 // ------------------------------------------------------------ pack kernels
-// bf16 blob, unit j (24*H elements):
-//   gate/up part (16*H): k-step s, lane l=(g,c): 8 elements
+// bf16 blob, unit j (24*H elements) = 8 chunks of 3*H elements; chunk w:
+//   gate/up part (2*H): step i < H/128, contraction step s = w*H/128 + i, lane l=(g,c): 8 elements
 //       { Wg[8j+g][16s+4c+0..1], Wu[8j+g][16s+4c+0..1], Wg[8j+g][16s+4c+2..3], Wu[8j+g][16s+4c+2..3] }
-//   down part (8*H): row-tile pair q, lane l=(g,c): 8 elements
+//   down part (H): pair i < H/256, row-tile pair q = w*H/256 + i, lane l=(g,c): 8 elements
 //       { Wd[32q+g][8j+2c..+1], Wd[32q+8+g][..], Wd[32q+16+g][..], Wd[32q+24+g][..] }
 __global__ void dx_pack_bf16_kernel(const __nv_bfloat16* Wg, const __nv_bfloat16* Wu, const __nv_bfloat16* Wd,
                                     __nv_bfloat16* blob, int H, int I) {
   const size_t n = (size_t)3 * H * I;
+  const int KW = H / 128, PW = H / 256;
   for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < n; idx += (size_t)gridDim.x * blockDim.x) {
-    const size_t unit = idx / (24 * (size_t)H);
+    const int j = (int)(idx / (24 * (size_t)H));
     const int r = (int)(idx % (24 * (size_t)H));
-    const int j = (int)unit;
+    const int w = r / (3 * H), rr = r % (3 * H);
     __nv_bfloat16 v;
-    if (r < 16 * H) {
-      const int s = r / 256, l = (r % 256) / 8, el = r % 8;
-      const int g = l >> 2, c = l & 3;
+    if (rr < 2 * H) {
+      const int i = rr / 256, l = (rr % 256) / 8, el = rr % 8;
+      const int s = w * KW + i, g = l >> 2, c = l & 3;
       const int col = 16 * s + 4 * c + (el & 1) + ((el >> 2) << 1);
       const int row = 8 * j + g;
       v = ((el >> 1) & 1) ? Wu[(size_t)row * H + col] : Wg[(size_t)row * H + col];
     } else {
-      const int r2 = r - 16 * H;
-      const int q = r2 / 256, l = (r2 % 256) / 8, el = r2 % 8;
-      const int g = l >> 2, c = l & 3;
+      const int r2 = rr - 2 * H;
+      const int i = r2 / 256, l = (r2 % 256) / 8, el = r2 % 8;
+      const int q = w * PW + i, g = l >> 2, c = l & 3;
       const int row = 32 * q + 8 * (el >> 1) + g;
       const int col = 8 * j + 2 * c + (el & 1);
       v = Wd[(size_t)row * I + col];
@@ -431,22 +465,18 @@ __global__ void dx_pack_fp32_kernel(const float* Wg, const float* Wu, const floa
 }
 
 template <int H, int NT>
-size_t bf16_fixed_smem() {
-  return sizeof(SmemHeader) + (size_t)2 * 8 * NT * 32 * 16 + (size_t)NT * (H / 16) * 32 * 16;
-}
-
-template <int H, int NT>
 cudaError_t launch_bf16(dx_ctx* ctx, const DxExpertParams& p, cudaStream_t st) {
-  const size_t fixed = bf16_fixed_smem<H, NT>();
-  const size_t stage = (size_t)16 * H;
-  int n_stages = (int)(((size_t)ctx->smem_optin - fixed) / stage);
-  if (n_stages > 8) n_stages = 8;
-  if (n_stages < 2) return cudaErrorInvalidConfiguration;
-  const size_t smem = fixed + (size_t)n_stages * stage;
+  const size_t hdr = (sizeof(SmemHeader) + 127) / 128 * 128;
+  const size_t fixed = hdr + (size_t)2 * 8 * NT * 32 * 16 + (NT == 1 ? 0 : (size_t)NT * (H / 16) * 32 * 16);
+  const size_t chunk = (size_t)6 * H;
+  int n_slots = (int)(((size_t)ctx->smem_optin - fixed) / chunk);
+  if (n_slots > kMaxSlots) n_slots = kMaxSlots;
+  if (n_slots < 2) return cudaErrorInvalidConfiguration;
+  const size_t smem = fixed + (size_t)n_slots * chunk;
   cudaError_t e = cudaFuncSetAttribute(dx_experts_bf16_kernel<H, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)smem);
   if (e != cudaSuccess) return e;
-  dx_experts_bf16_kernel<H, NT><<<ctx->sm_count, kThreads, smem, st>>>(p, n_stages);
+  dx_experts_bf16_kernel<H, NT><<<ctx->sm_count, kThreads, smem, st>>>(p, n_slots);
   return cudaGetLastError();
 }
 

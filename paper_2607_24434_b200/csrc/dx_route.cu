@@ -220,15 +220,18 @@ __global__ void __launch_bounds__(256) dx_route_kernel(DxRouteParams p) {
     DxEntry& en = W->entries[me];
     en.table_index = me;
     en.n_tiles = p.shared_tiles;
+    en.unit_begin = me * p.shared_tiles;
     en.m = K;
     for (int i = 0; i < K; ++i) { en.tok[i] = i; en.w[i] = 1.0f; }
   }
-  int n_entries;
+  int n_entries, total_units;
+  const int routed_base = p.n_shared * p.shared_tiles;
   if (!p.draft_mode) {
     if (me < E && flag) {
       DxEntry& en = W->entries[p.n_shared + upos];
       en.table_index = p.n_shared + 1 + me;
       en.n_tiles = p.routed_tiles;
+      en.unit_begin = routed_base + upos * p.routed_tiles;
       en.m = cnt;
       for (int i = 0; i < cnt; ++i) {
         int q = s_perm[off + i];
@@ -237,6 +240,7 @@ __global__ void __launch_bounds__(256) dx_route_kernel(DxRouteParams p) {
       }
     }
     n_entries = p.n_shared + ucount;
+    total_units = routed_base + ucount * p.routed_tiles;
   } else {
     int base = p.n_shared;
     if (p.draft_tiles > 0) {
@@ -244,6 +248,7 @@ __global__ void __launch_bounds__(256) dx_route_kernel(DxRouteParams p) {
         DxEntry& en = W->entries[base];
         en.table_index = p.n_shared;
         en.n_tiles = p.draft_tiles;
+        en.unit_begin = routed_base;
         en.m = 1;
         en.tok[0] = 0;
         en.w[0] = p.gamma;
@@ -254,21 +259,17 @@ __global__ void __launch_bounds__(256) dx_route_kernel(DxRouteParams p) {
       DxEntry& en = W->entries[base + me];
       en.table_index = p.n_shared + 1 + s_ids[me];
       en.n_tiles = p.routed_tiles;
+      en.unit_begin = routed_base + p.draft_tiles + me * p.routed_tiles;
       en.m = 1;
       en.tok[0] = 0;
       en.w[0] = s_w[me];
     }
     n_entries = base + p.top_r;
+    total_units = routed_base + p.draft_tiles + p.top_r * p.routed_tiles;
   }
-  __syncthreads();
   if (me == 0) {
-    int u = 0;
-    for (int i = 0; i < n_entries; ++i) {
-      W->entries[i].unit_begin = u;
-      u += W->entries[i].n_tiles;
-    }
     W->n_entries = n_entries;
-    W->total_units = u;
+    W->total_units = total_units;
     W->K = K;
   }
 }
