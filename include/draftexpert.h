@@ -138,7 +138,7 @@ dx_status moe_draft_step(dx_layer* layer, const float* h, float* y, int32_t* top
                          void* stream);
 
 /* ---- verifier: Eq. 4 over a block, grouped by the union of Eq. 2 / Eq. 3 -----------------------------------
- * h [K,H] in, y [K,H] out (overwritten).  Routing outputs (device pointers, each may be NULL if unwanted):
+ * h [K,H] in, y [K,H] out (overwritten; must not overlap h).  Routing outputs (device pointers, each may be NULL if unwanted):
  *   topk_ids [K,k] int32, topk_w [K,k] fp32;
  *   union_mask [ceil(E/64)] uint64 (bit e set iff e in U); union_ids [min(E,K*k)] int32 ascending;
  *   union_count [1] int32 = |U|;
@@ -155,13 +155,14 @@ dx_status moe_verify_route(dx_layer* layer, const float* h, int32_t K, float* y,
 dx_status moe_verify_experts(dx_layer* layer, const float* h, int32_t K, float* y, void* stream);
 
 /* ---- pre-norm residual forms for layer stacks (synthetic stacks stub attention out) --------------------------
- * h [K,H] is updated IN PLACE: h <- h + MoE(RMSNorm(h)) with unit gain and eps 1e-6, MoE = Eq. 4
- * (verify) or Eq. 5 (draft, K = 1).  Routing outputs as above (NULL allowed). */
-dx_status moe_verify_block_residual(dx_layer* layer, float* h, int32_t K,
+ * h_out = h_in + MoE(RMSNorm(h_in)) with unit gain and eps 1e-6, MoE = Eq. 4 (verify, [K,H]) or Eq. 5 (draft,
+ * K = 1).  h_in and h_out must not overlap (a stack alternates two buffers).  Routing outputs as above. */
+dx_status moe_verify_block_residual(dx_layer* layer, const float* h_in, float* h_out, int32_t K,
                                     int32_t* topk_ids, float* topk_w, uint64_t* union_mask,
                                     int32_t* union_ids, int32_t* union_count, int32_t* offsets,
                                     int32_t* perm, void* stream);
-dx_status moe_draft_step_residual(dx_layer* layer, float* h, int32_t* topk_ids, float* topk_w, void* stream);
+dx_status moe_draft_step_residual(dx_layer* layer, const float* h_in, float* h_out, int32_t* topk_ids,
+                                  float* topk_w, void* stream);
 
 /* ---- exact greedy verification: Algorithm 1, "verify" and "accept the target-consistent prefix" -------------
  * h [M,H] fp32: row i is the hidden state that predicts draft token i (M = K, or K+1 to also get the token

@@ -62,11 +62,11 @@ SIGNATURES = {
     "dx_layer_set_expert": (_I, [_P, _I, _P]),
     "dx_layer_attach_cache": (_I, [_P, _P, _I]),
     "moe_draft_step": (_I, [_P, _P, _P, _P, _P, _P]),
-    "moe_draft_step_residual": (_I, [_P, _P, _P, _P, _P]),
+    "moe_draft_step_residual": (_I, [_P, _P, _P, _P, _P, _P]),
     "moe_verify_block": (_I, [_P, _P, _I, _P, _P, _P, _P, _P, _P, _P, _P, _P]),
     "moe_verify_route": (_I, [_P, _P, _I, _P, _P, _P, _P, _P, _P, _P, _P, _P]),
     "moe_verify_experts": (_I, [_P, _P, _I, _P, _P]),
-    "moe_verify_block_residual": (_I, [_P, _P, _I, _P, _P, _P, _P, _P, _P, _P, _P]),
+    "moe_verify_block_residual": (_I, [_P, _P, _P, _I, _P, _P, _P, _P, _P, _P, _P, _P]),
     "spec_accept": (_I, [_P, _P, _I, _P, _I, _I, _I, _P, _I, _I, _P, _P, _P, _P]),
     "expert_cache_create": (_I, [_P, _I, _I, _I, C.c_size_t, C.POINTER(_P)]),
     "expert_cache_destroy": (_I, [_P]),
@@ -251,13 +251,18 @@ def moe_draft_step(layer: Layer, h: torch.Tensor, y: Optional[torch.Tensor] = No
     return out
 
 
-def moe_draft_step_residual(layer: Layer, h: torch.Tensor, out: Optional[Dict[str, torch.Tensor]] = None):
+def moe_draft_step_residual(layer: Layer, h_in: torch.Tensor, h_out: Optional[torch.Tensor] = None,
+                            out: Optional[Dict[str, torch.Tensor]] = None) -> Dict[str, torch.Tensor]:
+    """h_out = h_in + Eq. 5 applied to RMSNorm(h_in), one token."""
     sh = layer.shape
     if out is None:
-        out = {"topk_ids": torch.empty((sh.top_k,), dtype=torch.int32, device=h.device),
-               "topk_w": torch.empty((sh.top_k,), dtype=torch.float32, device=h.device)}
-    _check(layer.lib.moe_draft_step_residual(layer.handle, _ptr(h), _ptr(out["topk_ids"]), _ptr(out["topk_w"]),
-                                             _stream()), "moe_draft_step_residual")
+        out = {"topk_ids": torch.empty((sh.top_k,), dtype=torch.int32, device=h_in.device),
+               "topk_w": torch.empty((sh.top_k,), dtype=torch.float32, device=h_in.device)}
+    if h_out is None:
+        h_out = torch.empty_like(h_in)
+    _check(layer.lib.moe_draft_step_residual(layer.handle, _ptr(h_in), _ptr(h_out), _ptr(out["topk_ids"]),
+                                             _ptr(out["topk_w"]), _stream()), "moe_draft_step_residual")
+    out["h"] = h_out
     return out
 
 
@@ -287,15 +292,19 @@ def moe_verify_experts(layer: Layer, h: torch.Tensor, y: torch.Tensor) -> None:
     _check(layer.lib.moe_verify_experts(layer.handle, _ptr(h), h.shape[0], _ptr(y), _stream()), "moe_verify_experts")
 
 
-def moe_verify_block_residual(layer: Layer, h: torch.Tensor, out: Optional[Dict[str, torch.Tensor]] = None):
-    """In place: h <- h + MoE(RMSNorm(h)) for the block."""
-    K = h.shape[0]
+def moe_verify_block_residual(layer: Layer, h_in: torch.Tensor, h_out: Optional[torch.Tensor] = None,
+                              out: Optional[Dict[str, torch.Tensor]] = None) -> Dict[str, torch.Tensor]:
+    """h_out = h_in + MoE(RMSNorm(h_in)) for the block (h_in and h_out distinct buffers)."""
+    K = h_in.shape[0]
     if out is None:
-        out = _routing_buffers(layer.shape, K, h.device)
-    _check(layer.lib.moe_verify_block_residual(layer.handle, _ptr(h), K, _ptr(out["topk_ids"]), _ptr(out["topk_w"]),
-                                               _ptr(out["union_mask"]), _ptr(out["union_ids"]),
+        out = _routing_buffers(layer.shape, K, h_in.device)
+    if h_out is None:
+        h_out = torch.empty_like(h_in)
+    _check(layer.lib.moe_verify_block_residual(layer.handle, _ptr(h_in), _ptr(h_out), K, _ptr(out["topk_ids"]),
+                                               _ptr(out["topk_w"]), _ptr(out["union_mask"]), _ptr(out["union_ids"]),
                                                _ptr(out["union_count"]), _ptr(out["offsets"]), _ptr(out["perm"]),
                                                _stream()), "moe_verify_block_residual")
+    out["h"] = h_out
     return out
 
 

@@ -96,6 +96,8 @@ __global__ void __launch_bounds__(512, 1) dx_accept_bf16_kernel(AcceptParams p) 
   uint4* hiF = reinterpret_cast<uint4*>(smem);        // [NT][Q][32]
   uint4* loF = hiF + (size_t)NT * Q * 32;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, c = lane & 3;
+  dx_pdl_wait();   // the hidden rows are usually the previous kernel's output
+  dx_pdl_trigger();
 
   if (warp < DX_MAX_M) {
     float r = 1.0f;
@@ -202,6 +204,8 @@ __global__ void __launch_bounds__(256) dx_accept_fp32_kernel(AcceptParams p) {
   __shared__ float s_rstd[DX_MAX_M];
   __shared__ unsigned long long s_keys[DX_MAX_M];
   const int H = p.H, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  dx_pdl_wait();
+  dx_pdl_trigger();
   for (int row = warp; row < DX_MAX_M; row += 8) {
     float r = 1.0f;
     if (p.rms_norm && row < p.M) {
@@ -247,8 +251,7 @@ cudaError_t dx_launch_accept(dx_ctx* ctx, const float* h, int M, const void* W_l
   if (w_dtype == DX_DTYPE_FP32) {
     int grid = (V + 7) / 8;
     if (grid > ctx->sm_count * 8) grid = ctx->sm_count * 8;
-    dx_accept_fp32_kernel<<<grid, 256, 0, st>>>(p);
-    return cudaGetLastError();
+    return dx_launch_pdl(DX_PDL_ACCEPT, dx_accept_fp32_kernel, dim3(grid), dim3(256), 0, st, p);
   }
   const int NT = (M + 7) / 8;
   const size_t smem = (size_t)NT * (H / 32) * 32 * 16 * 2;
@@ -256,11 +259,10 @@ cudaError_t dx_launch_accept(dx_ctx* ctx, const float* h, int M, const void* W_l
   if (NT == 1) {
     e = cudaFuncSetAttribute(dx_accept_bf16_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    dx_accept_bf16_kernel<1><<<ctx->sm_count, 512, smem, st>>>(p);
+    return dx_launch_pdl(DX_PDL_ACCEPT, dx_accept_bf16_kernel<1>, dim3(ctx->sm_count), dim3(512), smem, st, p);
   } else {
     e = cudaFuncSetAttribute(dx_accept_bf16_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    dx_accept_bf16_kernel<2><<<ctx->sm_count, 512, smem, st>>>(p);
+    return dx_launch_pdl(DX_PDL_ACCEPT, dx_accept_bf16_kernel<2>, dim3(ctx->sm_count), dim3(512), smem, st, p);
   }
-  return cudaGetLastError();
 }

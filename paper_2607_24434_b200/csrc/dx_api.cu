@@ -5,7 +5,17 @@
 
 #include "dx_internal.cuh"
 
+#include <cstdlib>
+
 bool dx_bf16_hidden_supported(int H);
+
+int dx_pdl_mask() {
+  static const int mask = [] {
+    const char* v = std::getenv("DX_PDL_MASK");
+    return v ? std::atoi(v) : (DX_PDL_ROUTE | DX_PDL_EXPERTS);
+  }();
+  return mask;
+}
 
 #define DX_CUDA(ctx, call)                 \
   do {                                     \
@@ -45,7 +55,6 @@ extern "C" dx_status dx_create(int device, dx_ctx** out) {
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, device);
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device);
   if (e == cudaSuccess) e = cudaMalloc(&ctx->work, sizeof(DxWork));
-  if (e == cudaSuccess) e = cudaMalloc(&ctx->xn, sizeof(float) * DX_MAX_K * DX_MAX_H);
   if (e == cudaSuccess) e = cudaMalloc(&ctx->z, sizeof(float) * DX_MAX_K * DX_MAX_E);
   if (e == cudaSuccess) e = cudaMalloc(&ctx->ticket, sizeof(unsigned int) * 4);
   if (e == cudaSuccess) e = cudaMalloc(&ctx->keys, sizeof(unsigned long long) * DX_MAX_M);
@@ -66,7 +75,6 @@ extern "C" dx_status dx_create(int device, dx_ctx** out) {
 extern "C" dx_status dx_destroy(dx_ctx* ctx) {
   if (!ctx) return DX_ERR_INVALID_ARG;
   cudaFree(ctx->work);
-  cudaFree(ctx->xn);
   cudaFree(ctx->z);
   cudaFree(ctx->ticket);
   cudaFree(ctx->keys);
@@ -208,7 +216,7 @@ static dx_status do_route(dx_layer* L, const float* h, int K, float* y, const Ro
                           cudaStream_t st) {
   dx_ctx* ctx = L->ctx;
   const dx_layer_desc& d = L->desc;
-  if (!h || !y) return DX_ERR_INVALID_ARG;
+  if (!h || !y || h == y) return DX_ERR_INVALID_ARG;
   if (K < 1 || K > DX_MAX_K) return DX_ERR_UNSUPPORTED;
   if (!L->W_r) return DX_ERR_NOT_RESIDENT;
   for (int s = 0; s < d.n_shared; ++s)
@@ -228,8 +236,8 @@ static dx_status do_route(dx_layer* L, const float* h, int K, float* y, const Ro
   p.draft_mode = draft ? 1 : 0;
   p.top_r = 1;
   p.rms_norm = residual ? 1 : 0;
-  p.accumulate = residual ? 1 : 0;
-  p.xn = ctx->xn; p.y = y; p.z = ctx->z; p.ticket = ctx->ticket; p.work = ctx->work; p.dev_status = ctx->dev_status;
+  p.residual = residual ? 1 : 0;
+  p.y = y; p.z = ctx->z; p.ticket = ctx->ticket; p.work = ctx->work; p.dev_status = ctx->dev_status;
   p.topk_ids = o.topk_ids; p.topk_w = o.topk_w;
   p.union_mask = (unsigned long long*)o.union_mask; p.union_ids = o.union_ids; p.union_count = o.union_count;
   p.offsets = o.offsets; p.perm = o.perm;
@@ -238,19 +246,27 @@ static dx_status do_route(dx_layer* L, const float* h, int K, float* y, const Ro
   return DX_OK;
 }
 
-static dx_status do_experts(dx_layer* L, const float* h, int K, float* y, bool residual, cudaStream_t st) {
+static dx_status do_experts(dx_layer* L, const float* h, int K, float* y, bool draft, bool residual,
+                            cudaStream_t st) {
   dx_ctx* ctx = L->ctx;
-  if (!h || !y) return DX_ERR_INVALID_ARG;
+  const dx_layer_desc& d = L->desc;
+  if (!h || !y || h == y) return DX_ERR_INVALID_ARG;
   if (K < 1 || K > DX_MAX_K) return DX_ERR_UNSUPPORTED;
   dx_status s = upload_table(L, st);
   if (s != DX_OK) return s;
   DxExpertParams p{};
-  p.x = residual ? ctx->xn : h;
+  p.x = h;
   p.y = y;
   p.table = L->table_dev;
   p.work = ctx->work;
   p.dev_status = ctx->dev_status;
-  p.H = L->desc.hidden;
+  p.H = d.hidden;
+  p.K = K;
+  p.rms_norm = residual ? 1 : 0;
+  p.n_shared = d.n_shared;
+  p.shared_tiles = d.n_shared ? d.shared_inter / DX_TILE_I : 0;
+  p.draft_tiles = draft ? d.draft_inter / DX_TILE_I : 0;
+  p.gamma = d.draft_gamma;
   DX_CUDA(ctx, dx_launch_experts(ctx, p, L->desc.weight_dtype, K, st));
   ctx->launches++;
   if (L->cache) dx_cache_note_use(L->cache, L->cache_layer, st);
@@ -264,16 +280,17 @@ extern "C" dx_status moe_draft_step(dx_layer* L, const float* h, float* y, int32
   RouteOut o{topk_ids, topk_w, nullptr, nullptr, nullptr, nullptr, nullptr};
   dx_status s = do_route(L, h, 1, y, o, true, false, st);
   if (s != DX_OK) return s;
-  return do_experts(L, h, 1, y, false, st);
+  return do_experts(L, h, 1, y, true, false, st);
 }
 
-extern "C" dx_status moe_draft_step_residual(dx_layer* L, float* h, int32_t* topk_ids, float* topk_w, void* stream) {
+extern "C" dx_status moe_draft_step_residual(dx_layer* L, const float* h_in, float* h_out, int32_t* topk_ids,
+                                             float* topk_w, void* stream) {
   if (!L) return DX_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;
   RouteOut o{topk_ids, topk_w, nullptr, nullptr, nullptr, nullptr, nullptr};
-  dx_status s = do_route(L, h, 1, h, o, true, true, st);
+  dx_status s = do_route(L, h_in, 1, h_out, o, true, true, st);
   if (s != DX_OK) return s;
-  return do_experts(L, h, 1, h, true, st);
+  return do_experts(L, h_in, 1, h_out, true, true, st);
 }
 
 extern "C" dx_status moe_verify_route(dx_layer* L, const float* h, int32_t K, float* y, int32_t* topk_ids,
@@ -286,7 +303,7 @@ extern "C" dx_status moe_verify_route(dx_layer* L, const float* h, int32_t K, fl
 
 extern "C" dx_status moe_verify_experts(dx_layer* L, const float* h, int32_t K, float* y, void* stream) {
   if (!L) return DX_ERR_INVALID_ARG;
-  return do_experts(L, h, K, y, false, (cudaStream_t)stream);
+  return do_experts(L, h, K, y, false, false, (cudaStream_t)stream);
 }
 
 extern "C" dx_status moe_verify_block(dx_layer* L, const float* h, int32_t K, float* y, int32_t* topk_ids,
@@ -298,15 +315,16 @@ extern "C" dx_status moe_verify_block(dx_layer* L, const float* h, int32_t K, fl
   return moe_verify_experts(L, h, K, y, stream);
 }
 
-extern "C" dx_status moe_verify_block_residual(dx_layer* L, float* h, int32_t K, int32_t* topk_ids, float* topk_w,
-                                               uint64_t* union_mask, int32_t* union_ids, int32_t* union_count,
-                                               int32_t* offsets, int32_t* perm, void* stream) {
+extern "C" dx_status moe_verify_block_residual(dx_layer* L, const float* h_in, float* h_out, int32_t K,
+                                               int32_t* topk_ids, float* topk_w, uint64_t* union_mask,
+                                               int32_t* union_ids, int32_t* union_count, int32_t* offsets,
+                                               int32_t* perm, void* stream) {
   if (!L) return DX_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;
   RouteOut o{topk_ids, topk_w, union_mask, union_ids, union_count, offsets, perm};
-  dx_status s = do_route(L, h, K, h, o, false, true, st);
+  dx_status s = do_route(L, h_in, K, h_out, o, false, true, st);
   if (s != DX_OK) return s;
-  return do_experts(L, h, K, h, true, st);
+  return do_experts(L, h_in, K, h_out, false, true, st);
 }
 
 extern "C" dx_status spec_accept(dx_ctx* ctx, const float* h, int32_t M, const void* W_lm, int32_t V, int32_t H,

@@ -101,6 +101,14 @@ __device__ __forceinline__ int find_entry(const DxWork* W, int n_entries, int u,
 // is one bulk copy, one ring slot, one full/empty mbarrier pair, and is read by
 // exactly one warp, so slots recycle warp by warp and the producer can run
 // more than two units ahead of the consumers.
+//
+// Overlap with routing.  The groups that do not depend on the router (the
+// shared experts, and the draft expert in draft mode) are known from the layer
+// description alone.  The kernel is launched with programmatic stream
+// serialization right behind the routing kernel and streams those groups
+// first; only then does it wait for the routing kernel (griddepcontrol.wait),
+// read the work list and stream the routed groups.  Nothing is written to y
+// before that wait, because the routing kernel is what initialises y.
 constexpr int kConsumerWarps = 8;
 constexpr int kThreads = (kConsumerWarps + 1) * 32;
 constexpr int kMaxSlots = 24;
@@ -110,12 +118,18 @@ struct SmemHeader {
   unsigned long long empty[kMaxSlots];
   int abort_flag;
   int n_entries;
-  int pad[2];
+  int total_units;
+  int pad;
+  float rstd[DX_MAX_K];
   int e_begin[DX_MAX_ENTRIES];       // first unit of each entry
   int e_tiles[DX_MAX_ENTRIES];
   int e_m[DX_MAX_ENTRIES];
   const unsigned char* e_blob[DX_MAX_ENTRIES];
 };
+
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void cta_bar() { asm volatile("bar.sync 2, 288;" ::: "memory"); }
 
 template <int H, int NT>
 __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertParams p, int n_slots) {
@@ -137,10 +151,11 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const DxWork* W = p.work;
-  const int n_entries = W->n_entries;
-  const long long total = W->total_units;
-  const int u_lo = (int)((total * blockIdx.x) / gridDim.x);
-  const int u_hi = (int)((total * (blockIdx.x + 1)) / gridDim.x);
+  const int G = gridDim.x, cta = blockIdx.x;
+  // groups that do not depend on routing: shared experts, then (draft mode) the draft expert
+  const int n_static = p.n_shared + (p.draft_tiles > 0 ? 1 : 0);
+  const int NS = p.n_shared * p.shared_tiles + p.draft_tiles;
+  const int s_lo = (int)(((long long)NS * cta) / G), s_hi = (int)(((long long)NS * (cta + 1)) / G);
   volatile int* abort_flag = &hdr->abort_flag;
 
   if (threadIdx.x == 0) {
@@ -151,25 +166,23 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
     hdr->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  for (int i = threadIdx.x; i < n_entries; i += kThreads) {
-    const DxEntry& en = W->entries[i];
-    const unsigned char* blob = reinterpret_cast<const unsigned char*>(p.table[en.table_index]);
-    hdr->e_begin[i] = en.unit_begin;
-    hdr->e_tiles[i] = en.n_tiles;
-    hdr->e_m[i] = en.m;
-    hdr->e_blob[i] = blob;
-    if (blob == nullptr && en.n_tiles > 0) atomicExch(p.dev_status, DX_DEV_BAD_EXPERT_ID);
+  if (threadIdx.x < n_static) {
+    const int i = threadIdx.x;
+    const bool is_draft = i >= p.n_shared;
+    hdr->e_begin[i] = is_draft ? p.n_shared * p.shared_tiles : i * p.shared_tiles;
+    hdr->e_tiles[i] = is_draft ? p.draft_tiles : p.shared_tiles;
+    hdr->e_m[i] = is_draft ? 1 : p.K;
+    hdr->e_blob[i] = reinterpret_cast<const unsigned char*>(p.table[i]);
   }
   __syncthreads();
-  if (u_lo >= u_hi) return;
 
   if (warp == kConsumerWarps) {
     // ------------------------------------------------------------ producer
-    if (lane == 0) {
-      uint32_t it = 0;   // chunk counter
-      for (int e = 0; e < n_entries; ++e) {
+    uint32_t it = 0;   // chunk counter
+    auto issue = [&](int e0, int e1, int lo_u, int hi_u) {
+      for (int e = e0; e < e1; ++e) {
         const int b = hdr->e_begin[e], nt = hdr->e_tiles[e];
-        const int lo = max(b, u_lo), hi = min(b + nt, u_hi);
+        const int lo = max(b, lo_u), hi = min(b + nt, hi_u);
         const unsigned char* blob = hdr->e_blob[e];
         if (lo >= hi || blob == nullptr) continue;
         for (int u = lo; u < hi; ++u) {
@@ -184,6 +197,27 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
           }
         }
       }
+    };
+    if (lane == 0) issue(0, n_static, s_lo, s_hi);
+    __syncwarp();
+    pdl_wait();
+    const int n_entries = W->n_entries;
+    for (int i = n_static + threadIdx.x; i < n_entries; i += kThreads) {
+      const DxEntry& en = W->entries[i];
+      const unsigned char* blob = reinterpret_cast<const unsigned char*>(p.table[en.table_index]);
+      hdr->e_begin[i] = en.unit_begin; hdr->e_tiles[i] = en.n_tiles; hdr->e_m[i] = en.m; hdr->e_blob[i] = blob;
+      if (blob == nullptr && en.n_tiles > 0) atomicExch(p.dev_status, DX_DEV_BAD_EXPERT_ID);
+    }
+    cta_bar();
+    if (lane == 0) {
+      const long long T = W->total_units, NR = T - NS;
+      long long r_lo, r_hi;
+      if (T / G >= (NS + G - 1) / G) {   // keep shared + routed balanced together
+        r_lo = (T * cta) / G - s_lo; r_hi = (T * (cta + 1)) / G - s_hi;
+      } else {
+        r_lo = (NR * cta) / G; r_hi = (NR * (cta + 1)) / G;
+      }
+      issue(n_static, n_entries, NS + (int)r_lo, NS + (int)r_hi);
       if (*abort_flag) {
         // something gave up: make sure no copy is still landing in this CTA's
         // shared memory before it is released (bounded, ignores the flag)
@@ -212,154 +246,207 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
   // {hi(k0,k1), hi(k2,k3), lo(k0,k1), lo(k2,k3)} of token slot g
   uint32_t breg[kRegB ? KW : 1][4];
 
+  // 1/rms of every block row when the experts see RMSNorm(x)
+  for (int r = warp; r < DX_MAX_K; r += kConsumerWarps) {
+    float rs = 1.0f;
+    if (p.rms_norm && r < p.K) {
+      float ss = 0.f;
+      for (int j = lane * 4; j < H; j += 128) {
+        const float4 v = *reinterpret_cast<const float4*>(p.x + (size_t)r * H + j);
+        ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+      rs = rsqrtf(ss / (float)H + 1e-6f);
+    }
+    if (lane == 0) hdr->rstd[r] = rs;
+  }
+  consumer_bar();
+
   uint32_t uc = 0;   // units consumed by this CTA so far
   int buf = 0;
   // partial-exchange source lanes: lane (g,c) ends up holding the sums of rows i = 2c and 2c+1 for token g
   const int src0 = (2 * c) * 4 + (g >> 1), src1 = src0 + 4;
   const bool odd = g & 1;
 
-  for (int e = 0; e < n_entries; ++e) {
-    const int eb = hdr->e_begin[e], etiles = hdr->e_tiles[e];
-    const int lo = max(eb, u_lo), hi = min(eb + etiles, u_hi);
-    if (lo >= hi || hdr->e_blob[e] == nullptr) continue;
-    const DxEntry& en = W->entries[e];
-    const int m = hdr->e_m[e];
+  auto entry_tok = [&](int e, int slot) -> int { return e < n_static ? slot : W->entries[e].tok[slot]; };
+  auto entry_w = [&](int e, int slot) -> float {
+    return e < n_static ? (e < p.n_shared ? 1.0f : p.gamma) : W->entries[e].w[slot];
+  };
 
-    // ---- token fragments of this group
-    if constexpr (kRegB) {
-      const bool valid = g < m;
-      const float* xrow = p.x + (size_t)(valid ? en.tok[g] : 0) * H + 4 * c;
+  auto process = [&](int e0, int e1, int lo_u, int hi_u) {
+    for (int e = e0; e < e1; ++e) {
+      const int eb = hdr->e_begin[e], etiles = hdr->e_tiles[e];
+      const int lo = max(eb, lo_u), hi = min(eb + etiles, hi_u);
+      if (lo >= hi || hdr->e_blob[e] == nullptr) continue;
+      const int m = hdr->e_m[e];
+
+      // ---- token fragments of this group
+      if constexpr (kRegB) {
+        const bool valid = g < m;
+        const int tk = valid ? entry_tok(e, g) : 0;
+        const float rs = hdr->rstd[tk];
+        const float* xrow = p.x + (size_t)tk * H + 4 * c;
 #pragma unroll
-      for (int i = 0; i < KW; ++i) {
-        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (valid) v = *reinterpret_cast<const float4*>(xrow + 16 * (warp * KW + i));
-        __nv_bfloat16 h0, h1, h2, h3, l0, l1, l2, l3;
-        split_bf16(v.x, h0, l0); split_bf16(v.y, h1, l1); split_bf16(v.z, h2, l2); split_bf16(v.w, h3, l3);
-        breg[i][0] = pack2(h0, h1); breg[i][1] = pack2(h2, h3);
-        breg[i][2] = pack2(l0, l1); breg[i][3] = pack2(l2, l3);
-      }
-    } else {
-      consumer_bar();   // everyone is done reading the previous group's fragments
-      for (int idx = threadIdx.x; idx < NT * KSTEPS * 32; idx += kConsumerWarps * 32) {
-        const int l = idx & 31, ks = (idx >> 5) % KSTEPS, nt = idx / (32 * KSTEPS);
-        const int slot = nt * 8 + (l >> 2);
-        uint4 o = make_uint4(0u, 0u, 0u, 0u);
-        if (slot < m) {
-          const float4 v = *reinterpret_cast<const float4*>(p.x + (size_t)en.tok[slot] * H + 16 * ks + 4 * (l & 3));
+        for (int i = 0; i < KW; ++i) {
+          float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (valid) v = *reinterpret_cast<const float4*>(xrow + 16 * (warp * KW + i));
           __nv_bfloat16 h0, h1, h2, h3, l0, l1, l2, l3;
-          split_bf16(v.x, h0, l0); split_bf16(v.y, h1, l1); split_bf16(v.z, h2, l2); split_bf16(v.w, h3, l3);
-          o = make_uint4(pack2(h0, h1), pack2(h2, h3), pack2(l0, l1), pack2(l2, l3));
+          split_bf16(v.x * rs, h0, l0); split_bf16(v.y * rs, h1, l1);
+          split_bf16(v.z * rs, h2, l2); split_bf16(v.w * rs, h3, l3);
+          breg[i][0] = pack2(h0, h1); breg[i][1] = pack2(h2, h3);
+          breg[i][2] = pack2(l0, l1); breg[i][3] = pack2(l2, l3);
         }
-        bfrag[idx] = o;
+      } else {
+        consumer_bar();   // everyone is done reading the previous group's fragments
+        for (int idx = threadIdx.x; idx < NT * KSTEPS * 32; idx += kConsumerWarps * 32) {
+          const int l = idx & 31, ks = (idx >> 5) % KSTEPS, nt = idx / (32 * KSTEPS);
+          const int slot = nt * 8 + (l >> 2);
+          uint4 o = make_uint4(0u, 0u, 0u, 0u);
+          if (slot < m) {
+            const int tk = entry_tok(e, slot);
+            const float rs = hdr->rstd[tk];
+            const float4 v = *reinterpret_cast<const float4*>(p.x + (size_t)tk * H + 16 * ks + 4 * (l & 3));
+            __nv_bfloat16 h0, h1, h2, h3, l0, l1, l2, l3;
+            split_bf16(v.x * rs, h0, l0); split_bf16(v.y * rs, h1, l1);
+            split_bf16(v.z * rs, h2, l2); split_bf16(v.w * rs, h3, l3);
+            o = make_uint4(pack2(h0, h1), pack2(h2, h3), pack2(l0, l1), pack2(l2, l3));
+          }
+          bfrag[idx] = o;
+        }
+        consumer_bar();
       }
-      consumer_bar();
-    }
 
-    for (int u = lo; u < hi; ++u, ++uc) {
-      const uint32_t it = uc * kConsumerWarps + warp;
-      const uint32_t s = it % (uint32_t)n_slots, ph = (it / (uint32_t)n_slots) & 1u;
-      const uint4* A = reinterpret_cast<const uint4*>(ring + (size_t)s * CHUNK) + lane;
-      mbar_wait(smem_u32(&hdr->full[s]), ph, abort_flag);
+      for (int u = lo; u < hi; ++u, ++uc) {
+        const uint32_t it = uc * kConsumerWarps + warp;
+        const uint32_t s = it % (uint32_t)n_slots, ph = (it / (uint32_t)n_slots) & 1u;
+        const uint4* A = reinterpret_cast<const uint4*>(ring + (size_t)s * CHUNK) + lane;
+        mbar_wait(smem_u32(&hdr->full[s]), ph, abort_flag);
 
-      // ---- phase 1: [8 gate rows ; 8 up rows] x tokens over this warp's slice of the contraction
-      float ch[NT][2][4], cl[NT][2][4];
+        // ---- phase 1: [8 gate rows ; 8 up rows] x tokens over this warp's slice of the contraction
+        float ch[NT][2][4], cl[NT][2][4];
 #pragma unroll
-      for (int nt = 0; nt < NT; ++nt)
+        for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-        for (int r = 0; r < 4; ++r) ch[nt][0][r] = ch[nt][1][r] = cl[nt][0][r] = cl[nt][1][r] = 0.f;
+          for (int r = 0; r < 4; ++r) ch[nt][0][r] = ch[nt][1][r] = cl[nt][0][r] = cl[nt][1][r] = 0.f;
 #pragma unroll
-      for (int i = 0; i < KW; ++i) {
-        const uint4 a = A[i * 32];
-        if constexpr (kRegB) {
-          mma_k16(ch[0][i & 1], a, breg[i][0], breg[i][1]);
-          mma_k16(cl[0][i & 1], a, breg[i][2], breg[i][3]);
-        } else {
+        for (int i = 0; i < KW; ++i) {
+          const uint4 a = A[i * 32];
+          if constexpr (kRegB) {
+            mma_k16(ch[0][i & 1], a, breg[i][0], breg[i][1]);
+            mma_k16(cl[0][i & 1], a, breg[i][2], breg[i][3]);
+          } else {
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+              if (nt > 0 && m <= 8 * nt) continue;
+              const uint4 b = bfrag[(nt * KSTEPS + warp * KW + i) * 32 + lane];
+              mma_k16(ch[nt][i & 1], a, b.x, b.y);
+              mma_k16(cl[nt][i & 1], a, b.z, b.w);
+            }
+          }
+        }
+        // re-fragment: C holds (gate|up row g, tokens 2c,2c+1); phase 2 wants rows (2c,2c+1) of token g
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+          float v[4];
+#pragma unroll
+          for (int r = 0; r < 4; ++r) v[r] = (ch[nt][0][r] + ch[nt][1][r]) + (cl[nt][0][r] + cl[nt][1][r]);
+          const float a0 = __shfl_sync(0xffffffffu, v[0], src0), a1 = __shfl_sync(0xffffffffu, v[1], src0);
+          const float a2 = __shfl_sync(0xffffffffu, v[2], src0), a3 = __shfl_sync(0xffffffffu, v[3], src0);
+          const float b0 = __shfl_sync(0xffffffffu, v[0], src1), b1 = __shfl_sync(0xffffffffu, v[1], src1);
+          const float b2 = __shfl_sync(0xffffffffu, v[2], src1), b3 = __shfl_sync(0xffffffffu, v[3], src1);
+          partial[((buf * 8 + warp) * NT + nt) * 32 + lane] =
+              make_float4(odd ? a1 : a0, odd ? a3 : a2, odd ? b1 : b0, odd ? b3 : b2);
+        }
+        consumer_bar();
+
+        // ---- sum the eight slices, activation, phase-2 token fragment
+        uint32_t bhi[NT], blo[NT];
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+          float4 t = partial[((buf * 8 + 0) * NT + nt) * 32 + lane];
+#pragma unroll
+          for (int w = 1; w < 8; ++w) {
+            const float4 q = partial[((buf * 8 + w) * NT + nt) * 32 + lane];
+            t.x += q.x; t.y += q.y; t.z += q.z; t.w += q.w;
+          }
+          const float a0 = dx_silu(t.x) * t.y, a1 = dx_silu(t.z) * t.w;
+          __nv_bfloat16 h0, l0, h1, l1;
+          split_bf16(a0, h0, l0);
+          split_bf16(a1, h1, l1);
+          bhi[nt] = pack2(h0, h1);
+          blo[nt] = pack2(l0, l1);
+        }
+        buf ^= 1;
+
+        // ---- phase 2: 8 columns of W_d x activations for this warp's output rows
+        const uint4* D = A + KW * 32;
+#pragma unroll
+        for (int q = 0; q < PW; ++q) {
+          const uint4 a = D[q * 32];
 #pragma unroll
           for (int nt = 0; nt < NT; ++nt) {
             if (nt > 0 && m <= 8 * nt) continue;
-            const uint4 b = bfrag[(nt * KSTEPS + warp * KW + i) * 32 + lane];
-            mma_k16(ch[nt][i & 1], a, b.x, b.y);
-            mma_k16(cl[nt][i & 1], a, b.z, b.w);
+            mma_k8(acc[nt][2 * q], a.x, a.y, bhi[nt]);
+            mma_k8(acc[nt][2 * q + 1], a.z, a.w, bhi[nt]);
+            mma_k8(acc[nt][2 * q], a.x, a.y, blo[nt]);
+            mma_k8(acc[nt][2 * q + 1], a.z, a.w, blo[nt]);
           }
         }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&hdr->empty[s]));
       }
-      // re-fragment: C holds (gate|up row g, tokens 2c,2c+1); phase 2 wants rows (2c,2c+1) of token g
+
+      // ---- add this group's partial output rows to y (scaled by each token's weight), reset.
+      // y is initialised by the routing kernel, so its completion is awaited first.
+      pdl_wait();
 #pragma unroll
       for (int nt = 0; nt < NT; ++nt) {
-        float v[4];
+        const int s0 = nt * 8 + 2 * c, s1 = s0 + 1;
+        const bool v0 = s0 < m, v1 = s1 < m;
+        if (v0) {
+          const float w0 = entry_w(e, s0), w1 = v1 ? entry_w(e, s1) : 0.f;
+          float* y0 = p.y + (size_t)entry_tok(e, s0) * H;
+          float* y1 = p.y + (size_t)(v1 ? entry_tok(e, s1) : 0) * H;
 #pragma unroll
-        for (int r = 0; r < 4; ++r) v[r] = (ch[nt][0][r] + ch[nt][1][r]) + (cl[nt][0][r] + cl[nt][1][r]);
-        const float a0 = __shfl_sync(0xffffffffu, v[0], src0), a1 = __shfl_sync(0xffffffffu, v[1], src0);
-        const float a2 = __shfl_sync(0xffffffffu, v[2], src0), a3 = __shfl_sync(0xffffffffu, v[3], src0);
-        const float b0 = __shfl_sync(0xffffffffu, v[0], src1), b1 = __shfl_sync(0xffffffffu, v[1], src1);
-        const float b2 = __shfl_sync(0xffffffffu, v[2], src1), b3 = __shfl_sync(0xffffffffu, v[3], src1);
-        partial[((buf * 8 + warp) * NT + nt) * 32 + lane] =
-            make_float4(odd ? a1 : a0, odd ? a3 : a2, odd ? b1 : b0, odd ? b3 : b2);
-      }
-      consumer_bar();
-
-      // ---- sum the eight slices, activation, phase-2 token fragment
-      uint32_t bhi[NT], blo[NT];
-#pragma unroll
-      for (int nt = 0; nt < NT; ++nt) {
-        float4 t = partial[((buf * 8 + 0) * NT + nt) * 32 + lane];
-#pragma unroll
-        for (int w = 1; w < 8; ++w) {
-          const float4 q = partial[((buf * 8 + w) * NT + nt) * 32 + lane];
-          t.x += q.x; t.y += q.y; t.z += q.z; t.w += q.w;
-        }
-        const float a0 = dx_silu(t.x) * t.y, a1 = dx_silu(t.z) * t.w;
-        __nv_bfloat16 h0, l0, h1, l1;
-        split_bf16(a0, h0, l0);
-        split_bf16(a1, h1, l1);
-        bhi[nt] = pack2(h0, h1);
-        blo[nt] = pack2(l0, l1);
-      }
-      buf ^= 1;
-
-      // ---- phase 2: 8 columns of W_d x activations for this warp's output rows
-      const uint4* D = A + KW * 32;
-#pragma unroll
-      for (int q = 0; q < PW; ++q) {
-        const uint4 a = D[q * 32];
-#pragma unroll
-        for (int nt = 0; nt < NT; ++nt) {
-          if (nt > 0 && m <= 8 * nt) continue;
-          mma_k8(acc[nt][2 * q], a.x, a.y, bhi[nt]);
-          mma_k8(acc[nt][2 * q + 1], a.z, a.w, bhi[nt]);
-          mma_k8(acc[nt][2 * q], a.x, a.y, blo[nt]);
-          mma_k8(acc[nt][2 * q + 1], a.z, a.w, blo[nt]);
-        }
-      }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&hdr->empty[s]));
-    }
-
-    // ---- add this group's partial output rows to y (scaled by each token's weight), reset
-#pragma unroll
-    for (int nt = 0; nt < NT; ++nt) {
-      const int s0 = nt * 8 + 2 * c, s1 = s0 + 1;
-      const bool v0 = s0 < m, v1 = s1 < m;
-      if (v0) {
-        const float w0 = en.w[s0], w1 = v1 ? en.w[s1] : 0.f;
-        float* y0 = p.y + (size_t)en.tok[s0] * H;
-        float* y1 = p.y + (size_t)(v1 ? en.tok[s1] : 0) * H;
-#pragma unroll
-        for (int j = 0; j < 2 * PW; ++j) {
-          const int hh = (warp * 2 * PW + j) * 16 + g;
-          atomicAdd(y0 + hh, w0 * acc[nt][j][0]);
-          atomicAdd(y0 + hh + 8, w0 * acc[nt][j][2]);
-          if (v1) {
-            atomicAdd(y1 + hh, w1 * acc[nt][j][1]);
-            atomicAdd(y1 + hh + 8, w1 * acc[nt][j][3]);
+          for (int j = 0; j < 2 * PW; ++j) {
+            const int hh = (warp * 2 * PW + j) * 16 + g;
+            atomicAdd(y0 + hh, w0 * acc[nt][j][0]);
+            atomicAdd(y0 + hh + 8, w0 * acc[nt][j][2]);
+            if (v1) {
+              atomicAdd(y1 + hh, w1 * acc[nt][j][1]);
+              atomicAdd(y1 + hh + 8, w1 * acc[nt][j][3]);
+            }
           }
         }
+#pragma unroll
+        for (int j = 0; j < 2 * PW; ++j)
+#pragma unroll
+          for (int r = 0; r < 4; ++r) acc[nt][j][r] = 0.f;
       }
-#pragma unroll
-      for (int j = 0; j < 2 * PW; ++j)
-#pragma unroll
-        for (int r = 0; r < 4; ++r) acc[nt][j][r] = 0.f;
     }
+  };
+
+  process(0, n_static, s_lo, s_hi);
+  pdl_wait();
+  pdl_launch_dependents();
+  const int n_entries = W->n_entries;
+  for (int i = n_static + threadIdx.x; i < n_entries; i += kThreads) {
+    const DxEntry& en = W->entries[i];
+    const unsigned char* blob = reinterpret_cast<const unsigned char*>(p.table[en.table_index]);
+    hdr->e_begin[i] = en.unit_begin; hdr->e_tiles[i] = en.n_tiles; hdr->e_m[i] = en.m; hdr->e_blob[i] = blob;
+    if (blob == nullptr && en.n_tiles > 0) atomicExch(p.dev_status, DX_DEV_BAD_EXPERT_ID);
+  }
+  cta_bar();
+  {
+    const long long T = W->total_units, NR = T - NS;
+    long long r_lo, r_hi;
+    if (T / G >= (NS + G - 1) / G) {
+      r_lo = (T * cta) / G - s_lo; r_hi = (T * (cta + 1)) / G - s_hi;
+    } else {
+      r_lo = (NR * cta) / G; r_hi = (NR * (cta + 1)) / G;
+    }
+    process(n_static, n_entries, NS + (int)r_lo, NS + (int)r_hi);
   }
   if (*abort_flag && threadIdx.x == 0) atomicExch(p.dev_status, DX_DEV_WAIT_EXPIRED);
 }
@@ -369,9 +456,24 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
 // warp w owns gate/up row w, then every thread owns output columns.
 __global__ void __launch_bounds__(256) dx_experts_fp32_kernel(DxExpertParams p) {
   __shared__ float s_act[DX_MAX_K][DX_TILE_I];
+  __shared__ float s_rstd[DX_MAX_K];
   const DxWork* W = p.work;
-  const int n_entries = W->n_entries, total = W->total_units, H = p.H;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  dx_pdl_wait();
+  dx_pdl_trigger();
+  const int n_entries = W->n_entries, total = W->total_units, H = p.H;
+  for (int r = warp; r < DX_MAX_K; r += 8) {
+    float rs = 1.0f;
+    if (p.rms_norm && r < p.K) {
+      float ss = 0.f;
+      for (int j = lane; j < H; j += 32) { const float v = p.x[(size_t)r * H + j]; ss += v * v; }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+      rs = rsqrtf(ss / (float)H + 1e-6f);
+    }
+    if (lane == 0) s_rstd[r] = rs;
+  }
+  __syncthreads();
   int ei = 0;
   for (int u = blockIdx.x; u < total; u += gridDim.x) {
     ei = find_entry(W, n_entries, u, ei);
@@ -386,9 +488,10 @@ __global__ void __launch_bounds__(256) dx_experts_fp32_kernel(DxExpertParams p) 
     const float* ur = unit + (size_t)(8 + warp) * H;
     for (int t = 0; t < en.m; ++t) {
       const float* x = p.x + (size_t)en.tok[t] * H;
+      const float rs = s_rstd[en.tok[t]];
       float ag = 0.f, au = 0.f;
       for (int j = lane; j < H; j += 32) {
-        const float xv = x[j];
+        const float xv = x[j] * rs;
         ag = fmaf(gr[j], xv, ag);
         au = fmaf(ur[j], xv, au);
       }
@@ -476,8 +579,7 @@ cudaError_t launch_bf16(dx_ctx* ctx, const DxExpertParams& p, cudaStream_t st) {
   cudaError_t e = cudaFuncSetAttribute(dx_experts_bf16_kernel<H, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)smem);
   if (e != cudaSuccess) return e;
-  dx_experts_bf16_kernel<H, NT><<<ctx->sm_count, kThreads, smem, st>>>(p, n_slots);
-  return cudaGetLastError();
+  return dx_launch_pdl(DX_PDL_EXPERTS, dx_experts_bf16_kernel<H, NT>, dim3(ctx->sm_count), dim3(kThreads), smem, st, p, n_slots);
 }
 
 template <int H>
@@ -491,8 +593,7 @@ bool dx_bf16_hidden_supported(int H) { return H == 256 || H == 512 || H == 1024 
 
 cudaError_t dx_launch_experts(dx_ctx* ctx, const DxExpertParams& p, int weight_dtype, int K, cudaStream_t st) {
   if (weight_dtype == DX_DTYPE_FP32) {
-    dx_experts_fp32_kernel<<<ctx->sm_count * 4, 256, 0, st>>>(p);
-    return cudaGetLastError();
+    return dx_launch_pdl(DX_PDL_EXPERTS, dx_experts_fp32_kernel, dim3(ctx->sm_count * 4), dim3(256), 0, st, p);
   }
   switch (p.H) {
     case 256: return launch_bf16_h<256>(ctx, p, K, st);

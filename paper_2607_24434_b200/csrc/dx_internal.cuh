@@ -46,7 +46,6 @@ struct dx_ctx {
   int64_t launches;
   // device scratch
   DxWork* work;        // work list
-  float* xn;           // [DX_MAX_K, DX_MAX_H] normalised block
   float* z;            // [DX_MAX_K, DX_MAX_E] router logits
   unsigned int* ticket;        // last-CTA tickets (route, accept)
   unsigned long long* keys;    // [DX_MAX_M] packed argmax keys
@@ -80,8 +79,7 @@ struct DxRouteParams {
   int draft_mode;   // 0: verify block, 1: drafter (shared + draft expert + top_r routed)
   int top_r;
   int rms_norm;     // 1: route and experts see RMSNorm(h)
-  int accumulate;   // 1: y is added to, not overwritten
-  float* xn;
+  int residual;     // 0: y starts at zero, 1: y starts as a copy of h (pre-norm residual form)
   float* y;
   float* z;
   unsigned int* ticket;
@@ -97,12 +95,16 @@ struct DxRouteParams {
 };
 
 struct DxExpertParams {
-  const float* x;            // [K,H] block the experts see (h or the normalised copy)
-  float* y;                  // [K,H] accumulated into
+  const float* x;            // [K,H] block input (never written while the kernel runs)
+  float* y;                  // [K,H] accumulated into; initialised by the routing kernel
   const void* const* table;  // layer blob table (device)
   const DxWork* work;
   int32_t* dev_status;
-  int H;
+  int H, K;
+  int rms_norm;              // 1: the experts see RMSNorm(x) (unit gain, eps 1e-6)
+  // groups known without routing: shared experts (all K rows, weight 1) and, in draft mode, the draft expert
+  int n_shared, shared_tiles, draft_tiles;
+  float gamma;
 };
 
 // launchers (each returns the cudaError_t of the launch)
@@ -118,6 +120,32 @@ cudaError_t dx_experts_prepare(dx_ctx* ctx);   // opt-in shared memory attribute
 // cache hooks used by the layer code
 const void** dx_cache_table(dx_cache* c, int layer);
 void dx_cache_note_use(dx_cache* c, int layer, cudaStream_t st);
+
+// Programmatic dependent launch: wait for the preceding kernel of the stream / let the next one start early.
+__device__ __forceinline__ void dx_pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void dx_pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+// Which kernels are launched with programmatic stream serialization: bit 0 routing, bit 1 experts, bit 2 accept.
+// Default from the library; DX_PDL_MASK in the environment overrides it (0 = plain stream order everywhere).
+int dx_pdl_mask();
+enum { DX_PDL_ROUTE = 1, DX_PDL_EXPERTS = 2, DX_PDL_ACCEPT = 4 };
+
+// Launch with programmatic stream serialization so that the kernel may begin while its predecessor drains.
+template <typename... KArgs, typename... Args>
+inline cudaError_t dx_launch_pdl(int which, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                                 cudaStream_t st, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = (dx_pdl_mask() & which) ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
 
 __device__ __forceinline__ float dx_silu(float x) { return x / (1.0f + expf(-x)); }
 

@@ -70,6 +70,9 @@ __global__ void __launch_bounds__(256) dx_route_kernel(DxRouteParams p) {
   const int t = blockIdx.x / EG, eg = blockIdx.x % EG;
   const int H = p.H;
   const float* hrow = p.h + (size_t)t * H;
+  // everything this kernel reads or writes may still be in use by the previous kernel of the stream
+  dx_pdl_wait();
+  dx_pdl_trigger();
 
   // 1/rms of the row (every warp recomputes it: H floats from L1/L2)
   float rstd = 1.0f;
@@ -87,6 +90,7 @@ __global__ void __launch_bounds__(256) dx_route_kernel(DxRouteParams p) {
   if (e < p.E) {
     const WT* wrow = reinterpret_cast<const WT*>(p.W_r) + (size_t)e * H;
     float acc = 0.f;
+#pragma unroll 4
     for (int j = lane * 8; j < H; j += 256) {
       float wv[8], hv[8];
       load8(wrow + j, wv);
@@ -98,13 +102,11 @@ __global__ void __launch_bounds__(256) dx_route_kernel(DxRouteParams p) {
     if (lane == 0) p.z[t * p.E + e] = acc * rstd + (p.bias ? p.bias[e] : 0.f);
   }
   if (eg == 0) {
+    // y starts at zero, or as a copy of the block in the residual form
     for (int j = threadIdx.x * 4; j < H; j += 1024) {
-      if (p.rms_norm) {
-        float4 v = *reinterpret_cast<const float4*>(hrow + j);
-        v.x *= rstd; v.y *= rstd; v.z *= rstd; v.w *= rstd;
-        *reinterpret_cast<float4*>(p.xn + (size_t)t * H + j) = v;
-      }
-      if (!p.accumulate) *reinterpret_cast<float4*>(p.y + (size_t)t * H + j) = make_float4(0.f, 0.f, 0.f, 0.f);
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (p.residual) v = *reinterpret_cast<const float4*>(hrow + j);
+      *reinterpret_cast<float4*>(p.y + (size_t)t * H + j) = v;
     }
   }
 
@@ -279,8 +281,6 @@ __global__ void __launch_bounds__(256) dx_route_kernel(DxRouteParams p) {
 cudaError_t dx_launch_route(const DxRouteParams& p, int weight_dtype, cudaStream_t st) {
   const int grid = p.K * ((p.E + 7) / 8);
   if (weight_dtype == DX_DTYPE_BF16)
-    dx_route_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(p);
-  else
-    dx_route_kernel<float><<<grid, 256, 0, st>>>(p);
-  return cudaGetLastError();
+    return dx_launch_pdl(DX_PDL_ROUTE, dx_route_kernel<__nv_bfloat16>, dim3(grid), dim3(256), 0, st, p);
+  return dx_launch_pdl(DX_PDL_ROUTE, dx_route_kernel<float>, dim3(grid), dim3(256), 0, st, p);
 }

@@ -161,17 +161,16 @@ def test_residual_forms(dx):
     L = binding.Layer.from_weights(ctx, layer)
     h = synth.hidden_block(6, SMALL.hidden, 61, 0.9, "cuda") * 3.0
     h_np = h.cpu().numpy().astype(np.float64)
-    hv = h.clone()
-    out = binding.moe_verify_block_residual(L, hv)
+    out = binding.moe_verify_block_residual(L, h)
     torch.cuda.synchronize()
     ids = out["topk_ids"].cpu().numpy()
     want = O.stack_layer_target(h_np, ref, forced_ids=ids)[0]
-    assert row_rel_err(hv.cpu().numpy(), want).max() <= Y_TIGHT
-    hd = h[:1].clone()
-    outd = binding.moe_draft_step_residual(L, hd)
+    assert row_rel_err(out["h"].cpu().numpy(), want).max() <= Y_TIGHT
+    assert torch.equal(h.cpu(), torch.from_numpy(h_np.astype(np.float32)))      # the input block is untouched
+    outd = binding.moe_draft_step_residual(L, h[:1])
     torch.cuda.synchronize()
     wantd = O.stack_layer_draft(h_np[:1], ref, forced_ids=outd["topk_ids"].cpu().numpy()[None])[0]
-    assert row_rel_err(hd.cpu().numpy(), wantd).max() <= Y_TIGHT
+    assert row_rel_err(outd["h"].cpu().numpy(), wantd).max() <= Y_TIGHT
     L.close()
 
 
