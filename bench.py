@@ -229,6 +229,42 @@ def run_gpu(args):
     draft_ms = float(np.mean([x.elapsed_time(y) for x, y in t_draft]))
     route_ms = float(np.mean([x.elapsed_time(y) for x, y in t_route]))
     acc_ms = float(np.mean([x.elapsed_time(y) for x, y in t_acc]))
+
+    # ---- each component replayed back to back from its own CUDA graph (no launch gaps, routing overlapped)
+    def graph_ms(fn, reps=200):
+        side = torch.cuda.Stream()
+        side.wait_stream(stream)
+        with torch.cuda.stream(side):
+            for i in range(NL):
+                fn(i)
+        stream.wait_stream(side)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            for i in range(NL):
+                fn(i)
+        g.replay()
+        torch.cuda.synchronize()
+        x0, x1 = ev(), ev()
+        x0.record(stream)
+        for _ in range(reps):
+            g.replay()
+        x1.record(stream)
+        torch.cuda.synchronize()
+        return x0.elapsed_time(x1) / (reps * NL)
+
+    comp = {}
+    if not args.no_graph:
+        comp["verify_block_ms"] = graph_ms(lambda i: binding.moe_verify_block(layers[i], blocks[i], ys[i], rb[i]))
+        comp["draft_step_ms"] = graph_ms(lambda i: binding.moe_draft_step(layers[i], blocks[i][:1], yd, dbuf))
+        comp["accept_ms"] = graph_ms(lambda i: binding.spec_accept(ctx, ys[i], W_lm, draft_tok, True, abuf))
+        vb = float(np.mean([(union[li] + shape.n_shared) * exp_bytes for li in range(NL)])) + shape.n_experts * H * 2
+        comp["verify_block_gbs"] = vb / (comp["verify_block_ms"] * 1e-3) / 1e9
+        comp["verify_block_frac_of_8TBs"] = comp["verify_block_gbs"] / NOMINAL_HBM_GBS
+        comp["verify_block_tokens_per_s"] = K / (comp["verify_block_ms"] * 1e-3)
+        comp["draft_step_gbs"] = ((shape.n_shared + 2) * exp_bytes + shape.n_experts * H * 2) / (
+            comp["draft_step_ms"] * 1e-3) / 1e9
+        comp["accept_gbs"] = V * H * 2 / (comp["accept_ms"] * 1e-3) / 1e9
     draft_bytes = (shape.n_shared + 2) * exp_bytes + shape.n_experts * H * 2
     acc_bytes = V * H * 2
 
@@ -307,6 +343,7 @@ def run_gpu(args):
                     "draft_frac_of_peak": draft_bytes / (draft_ms * 1e-3) / 1e9 / peak,
                     "accept_ms": acc_ms, "accept_gbs": acc_bytes / (acc_ms * 1e-3) / 1e9,
                     "accept_frac_of_peak": acc_bytes / (acc_ms * 1e-3) / 1e9 / peak},
+        "graph_components": comp,
         "clocks": clocks,
     }
     if world == 1 and not args.no_cpu_baseline:

@@ -251,7 +251,7 @@ cudaError_t dx_launch_accept(dx_ctx* ctx, const float* h, int M, const void* W_l
   if (w_dtype == DX_DTYPE_FP32) {
     int grid = (V + 7) / 8;
     if (grid > ctx->sm_count * 8) grid = ctx->sm_count * 8;
-    return dx_launch_pdl(DX_PDL_ACCEPT, dx_accept_fp32_kernel, dim3(grid), dim3(256), 0, st, p);
+    return dx_launch_pdl(DX_PDL_ACCEPT, dx_accept_fp32_kernel, dim3(grid), dim3(256), 0, st, 1, p);
   }
   const int NT = (M + 7) / 8;
   const size_t smem = (size_t)NT * (H / 32) * 32 * 16 * 2;
@@ -259,10 +259,10 @@ cudaError_t dx_launch_accept(dx_ctx* ctx, const float* h, int M, const void* W_l
   if (NT == 1) {
     e = cudaFuncSetAttribute(dx_accept_bf16_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    return dx_launch_pdl(DX_PDL_ACCEPT, dx_accept_bf16_kernel<1>, dim3(ctx->sm_count), dim3(512), smem, st, p);
+    return dx_launch_pdl(DX_PDL_ACCEPT, dx_accept_bf16_kernel<1>, dim3(ctx->sm_count), dim3(512), smem, st, 1, p);
   } else {
     e = cudaFuncSetAttribute(dx_accept_bf16_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    return dx_launch_pdl(DX_PDL_ACCEPT, dx_accept_bf16_kernel<2>, dim3(ctx->sm_count), dim3(512), smem, st, p);
+    return dx_launch_pdl(DX_PDL_ACCEPT, dx_accept_bf16_kernel<2>, dim3(ctx->sm_count), dim3(512), smem, st, 1, p);
   }
 }

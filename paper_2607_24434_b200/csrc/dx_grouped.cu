@@ -579,7 +579,7 @@ cudaError_t launch_bf16(dx_ctx* ctx, const DxExpertParams& p, cudaStream_t st) {
   cudaError_t e = cudaFuncSetAttribute(dx_experts_bf16_kernel<H, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)smem);
   if (e != cudaSuccess) return e;
-  return dx_launch_pdl(DX_PDL_EXPERTS, dx_experts_bf16_kernel<H, NT>, dim3(ctx->sm_count), dim3(kThreads), smem, st, p, n_slots);
+  return dx_launch_pdl(DX_PDL_EXPERTS, dx_experts_bf16_kernel<H, NT>, dim3(ctx->sm_count), dim3(kThreads), smem, st, 1, p, n_slots);
 }
 
 template <int H>
@@ -593,7 +593,7 @@ bool dx_bf16_hidden_supported(int H) { return H == 256 || H == 512 || H == 1024 
 
 cudaError_t dx_launch_experts(dx_ctx* ctx, const DxExpertParams& p, int weight_dtype, int K, cudaStream_t st) {
   if (weight_dtype == DX_DTYPE_FP32) {
-    return dx_launch_pdl(DX_PDL_EXPERTS, dx_experts_fp32_kernel, dim3(ctx->sm_count * 4), dim3(256), 0, st, p);
+    return dx_launch_pdl(DX_PDL_EXPERTS, dx_experts_fp32_kernel, dim3(ctx->sm_count * 4), dim3(256), 0, st, 1, p);
   }
   switch (p.H) {
     case 256: return launch_bf16_h<256>(ctx, p, K, st);

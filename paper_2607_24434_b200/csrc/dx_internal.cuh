@@ -80,6 +80,7 @@ struct DxRouteParams {
   int top_r;
   int rms_norm;     // 1: route and experts see RMSNorm(h)
   int residual;     // 0: y starts at zero, 1: y starts as a copy of h (pre-norm residual form)
+  int tok_group;    // block rows staged in shared memory per pass (set by the launcher)
   float* y;
   float* z;
   unsigned int* ticket;
@@ -133,17 +134,28 @@ enum { DX_PDL_ROUTE = 1, DX_PDL_EXPERTS = 2, DX_PDL_ACCEPT = 4 };
 // Launch with programmatic stream serialization so that the kernel may begin while its predecessor drains.
 template <typename... KArgs, typename... Args>
 inline cudaError_t dx_launch_pdl(int which, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
-                                 cudaStream_t st, Args... args) {
+                                 cudaStream_t st, int cluster, Args... args) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid;
   cfg.blockDim = block;
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchAttribute attr[2];
+  int n = 0;
+  if (cluster > 1) {   // the grid is made of thread-block clusters of this many CTAs
+    attr[n].id = cudaLaunchAttributeClusterDimension;
+    attr[n].val.clusterDim.x = cluster;
+    attr[n].val.clusterDim.y = 1;
+    attr[n].val.clusterDim.z = 1;
+    ++n;
+  }
+  if (dx_pdl_mask() & which) {
+    attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[n].val.programmaticStreamSerializationAllowed = 1;
+    ++n;
+  }
   cfg.attrs = attr;
-  cfg.numAttrs = (dx_pdl_mask() & which) ? 1 : 0;
+  cfg.numAttrs = n;
   return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 

@@ -2,28 +2,42 @@
 // g_{l,e} of Eq. 4), the block's expert union and the pair permutation grouped
 // by expert (Eq. 2 / Eq. 3), and the work list the expert kernels consume.
 //
-// Grid: one CTA per (token, group of 8 experts); each warp owns one router row
-// and reduces its dot product with shuffles.  The CTA that takes the last
-// ticket finalises: one warp per token runs k rounds of a warp-wide 64-bit max
-// over (orderable logit, ~expert id) keys, then the CTA builds the union with
-// ballot/popc compaction and a counting sort of the K*k (token, expert) pairs.
+// One thread-block cluster of 8 CTAs does all of it.  Each CTA owns an eighth
+// of the router rows: a warp loads a 2048-column slab of its row once (all
+// loads in flight together) and dots it with every block row, which sit in
+// shared memory.  The logits are written straight into CTA 0's shared memory
+// through distributed shared memory, so the hand-over is one hardware cluster
+// barrier: no fences, tickets or global round trips on the critical path.
+// CTA 0 then runs, one warp per token, k rounds of a warp-wide 64-bit max over
+// (orderable logit, ~expert id) keys, and builds the union with ballot/popc
+// compaction and a counting sort of the K*k (token, expert) pairs.
+#include <cooperative_groups.h>
+
 #include "dx_internal.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace {
 
-__device__ __forceinline__ void load8(const float* p, float (&v)[8]) {
-  float4 a = *reinterpret_cast<const float4*>(p);
-  float4 b = *reinterpret_cast<const float4*>(p + 4);
-  v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
-}
-__device__ __forceinline__ void load8(const __nv_bfloat16* p, float (&v)[8]) {
-  uint4 r = *reinterpret_cast<const uint4*>(p);
-  unsigned int u[4] = {r.x, r.y, r.z, r.w};
+constexpr int kRouteThreads = 256;
+constexpr int kRouteCluster = 8;
+constexpr int kRouteWarps = kRouteThreads / 32;
+
+__device__ __forceinline__ void unpack8(const uint4& r, float (&v)[8]) {
+  const unsigned int u[4] = {r.x, r.y, r.z, r.w};
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
     v[2 * i] = __uint_as_float(u[i] << 16);
     v[2 * i + 1] = __uint_as_float(u[i] & 0xffff0000u);
   }
+}
+
+__device__ __forceinline__ uint4 ldg_stream(const void* p) {
+  uint4 r;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
+               : "l"(p));
+  return r;
 }
 
 __device__ __forceinline__ float warp_sum(float v) {
@@ -40,7 +54,7 @@ __device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long v)
   return v;
 }
 
-// Exclusive scan over the 256 threads of the CTA; `total` receives the sum.
+// Exclusive scan over the threads of the CTA; `total` receives the sum.
 __device__ __forceinline__ int block_exclusive_scan(int v, int* s_warp, int& total) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   int inc = v;
@@ -53,7 +67,7 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int* s_warp, int& tot
   __syncthreads();
   int base = 0, tot = 0;
 #pragma unroll
-  for (int w = 0; w < 8; ++w) {
+  for (int w = 0; w < kRouteWarps; ++w) {
     int c = s_warp[w];
     if (w < warp) base += c;
     tot += c;
@@ -63,81 +77,147 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int* s_warp, int& tot
   return base + inc - v;
 }
 
+// Dot products of one router row with up to kTokGroup block rows (staged in
+// shared memory, row stride H) over a slab of <= 2048 columns; the lane owns
+// columns j0 + lane*8 + 256*i.
+constexpr int kTokGroup = 8;
+__device__ __forceinline__ void row_dots(const __nv_bfloat16* wrow, const float* h, int H, int K, int j0, int chunks,
+                                         int lane, float (&acc)[kTokGroup]) {
+  uint4 w[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i)
+    if (i < chunks) w[i] = ldg_stream(wrow + j0 + lane * 8 + 256 * i);
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    if (i < chunks) {
+      float wv[8];
+      unpack8(w[i], wv);
+      const float* hp = h + j0 + lane * 8 + 256 * i;
+#pragma unroll
+      for (int t = 0; t < kTokGroup; ++t) {
+        if (t < K) {
+          const float4 a = *reinterpret_cast<const float4*>(hp + (size_t)t * H);
+          const float4 b = *reinterpret_cast<const float4*>(hp + (size_t)t * H + 4);
+          float s = acc[t];
+          s = fmaf(wv[0], a.x, s); s = fmaf(wv[1], a.y, s); s = fmaf(wv[2], a.z, s); s = fmaf(wv[3], a.w, s);
+          s = fmaf(wv[4], b.x, s); s = fmaf(wv[5], b.y, s); s = fmaf(wv[6], b.z, s); s = fmaf(wv[7], b.w, s);
+          acc[t] = s;
+        }
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ void row_dots(const float* wrow, const float* h, int H, int K, int j0, int chunks, int lane,
+                                         float (&acc)[kTokGroup]) {
+#pragma unroll 2
+  for (int i = 0; i < chunks; ++i) {
+    const float* wp = wrow + j0 + lane * 8 + 256 * i;
+    const uint4 u0 = ldg_stream(wp), u1 = ldg_stream(wp + 4);
+    const float4 w0 = make_float4(__uint_as_float(u0.x), __uint_as_float(u0.y), __uint_as_float(u0.z), __uint_as_float(u0.w));
+    const float4 w1 = make_float4(__uint_as_float(u1.x), __uint_as_float(u1.y), __uint_as_float(u1.z), __uint_as_float(u1.w));
+    const float* hp = h + j0 + lane * 8 + 256 * i;
+#pragma unroll
+    for (int t = 0; t < kTokGroup; ++t) {
+      if (t < K) {
+        const float4 a = *reinterpret_cast<const float4*>(hp + (size_t)t * H);
+        const float4 b = *reinterpret_cast<const float4*>(hp + (size_t)t * H + 4);
+        float s = acc[t];
+        s = fmaf(w0.x, a.x, s); s = fmaf(w0.y, a.y, s); s = fmaf(w0.z, a.z, s); s = fmaf(w0.w, a.w, s);
+        s = fmaf(w1.x, b.x, s); s = fmaf(w1.y, b.y, s); s = fmaf(w1.z, b.z, s); s = fmaf(w1.w, b.w, s);
+        acc[t] = s;
+      }
+    }
+  }
+}
+
 template <typename WT>
-__global__ void __launch_bounds__(256) dx_route_kernel(DxRouteParams p) {
+__global__ void __launch_bounds__(kRouteThreads) dx_route_kernel(DxRouteParams p) {
+  __shared__ float s_z[DX_MAX_K * DX_MAX_E];
+  __shared__ float s_rstd[DX_MAX_K];
+  __shared__ int s_ids[DX_MAX_PAIRS];
+  __shared__ float s_w[DX_MAX_PAIRS];
+  __shared__ int s_perm[DX_MAX_PAIRS];
+  __shared__ int s_scan[kRouteWarps];
+  __shared__ unsigned int s_ballot[kRouteWarps];
+
+  cg::cluster_group cluster = cg::this_cluster();
+  const int crank = (int)cluster.block_rank();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int EG = (p.E + 7) >> 3;
-  const int t = blockIdx.x / EG, eg = blockIdx.x % EG;
-  const int H = p.H;
-  const float* hrow = p.h + (size_t)t * H;
-  // everything this kernel reads or writes may still be in use by the previous kernel of the stream
+  const int K = p.K, E = p.E, k = p.k, H = p.H, P = K * k;
+  const int epc = (E + kRouteCluster - 1) / kRouteCluster;   // router rows per CTA
+  const int e_lo = crank * epc, e_hi = min(E, e_lo + epc);
+  // the router matrix is constant: pull this CTA's rows into L2 while the previous kernel of the stream drains
+  if (e_lo < e_hi) {
+    const char* wb = reinterpret_cast<const char*>(p.W_r) + (size_t)e_lo * H * sizeof(WT);
+    const size_t bytes = (size_t)(e_hi - e_lo) * H * sizeof(WT);
+    for (size_t o = (size_t)threadIdx.x * 128; o < bytes; o += (size_t)kRouteThreads * 128)
+      asm volatile("prefetch.global.L2 [%0];" ::"l"(wb + o));
+  }
+  // everything else this kernel reads or writes may still be in use by the previous kernel of the stream;
+  // once that is over, let the expert kernel start on the groups that need no routing
   dx_pdl_wait();
   dx_pdl_trigger();
 
-  // 1/rms of the row (every warp recomputes it: H floats from L1/L2)
-  float rstd = 1.0f;
-  if (p.rms_norm) {
-    float ss = 0.f;
-    for (int j = lane * 4; j < H; j += 128) {
-      float4 v = *reinterpret_cast<const float4*>(hrow + j);
-      ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+  // 1/rms of every block row
+  for (int t = warp; t < DX_MAX_K; t += kRouteWarps) {
+    float rs = 1.0f;
+    if (p.rms_norm && t < K) {
+      float ss = 0.f;
+      for (int j = lane * 4; j < H; j += 128) {
+        const float4 v = *reinterpret_cast<const float4*>(p.h + (size_t)t * H + j);
+        ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+      }
+      rs = rsqrtf(warp_sum(ss) / (float)H + 1e-6f);
     }
-    ss = warp_sum(ss);
-    rstd = rsqrtf(ss / (float)H + 1e-6f);
+    if (lane == 0) s_rstd[t] = rs;
   }
+  __syncthreads();
 
-  const int e = eg * 8 + warp;
-  if (e < p.E) {
-    const WT* wrow = reinterpret_cast<const WT*>(p.W_r) + (size_t)e * H;
-    float acc = 0.f;
-#pragma unroll 4
-    for (int j = lane * 8; j < H; j += 256) {
-      float wv[8], hv[8];
-      load8(wrow + j, wv);
-      load8(hrow + j, hv);
+  // router logits z[t,e]; block rows go through shared memory in groups of up to `tg` rows
+  extern __shared__ __align__(16) float s_h[];
+  float* z0 = cluster.map_shared_rank(s_z, 0);   // CTA 0's logit table
+  const int tg = p.tok_group;
+  for (int t0 = 0; t0 < K; t0 += tg) {
+    const int kt = min(tg, K - t0);
+    __syncthreads();
+    for (int j = threadIdx.x * 4; j < kt * H; j += kRouteThreads * 4)
+      *reinterpret_cast<float4*>(s_h + j) = *reinterpret_cast<const float4*>(p.h + (size_t)t0 * H + j);
+    __syncthreads();
+    for (int e = e_lo + warp; e < e_hi; e += kRouteWarps) {
+      const WT* wrow = reinterpret_cast<const WT*>(p.W_r) + (size_t)e * H;
+      float acc[kTokGroup];
 #pragma unroll
-      for (int i = 0; i < 8; ++i) acc = fmaf(wv[i], hv[i], acc);
+      for (int t = 0; t < kTokGroup; ++t) acc[t] = 0.f;
+      for (int j0 = 0; j0 < H; j0 += 2048) row_dots(wrow, s_h, H, kt, j0, min(8, (H - j0) / 256), lane, acc);
+      const float b = p.bias ? p.bias[e] : 0.f;
+#pragma unroll
+      for (int t = 0; t < kTokGroup; ++t) {
+        if (t < kt) {
+          const float s = warp_sum(acc[t]);
+          if (lane == 0) z0[(t0 + t) * E + e] = s * s_rstd[t0 + t] + b;
+        }
+      }
     }
-    acc = warp_sum(acc);
-    if (lane == 0) p.z[t * p.E + e] = acc * rstd + (p.bias ? p.bias[e] : 0.f);
   }
-  if (eg == 0) {
-    // y starts at zero, or as a copy of the block in the residual form
-    for (int j = threadIdx.x * 4; j < H; j += 1024) {
-      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (p.residual) v = *reinterpret_cast<const float4*>(hrow + j);
-      *reinterpret_cast<float4*>(p.y + (size_t)t * H + j) = v;
-    }
+  // y starts at zero, or as a copy of the block in the residual form
+  for (int j = (crank * kRouteThreads + threadIdx.x) * 4; j < K * H; j += kRouteCluster * kRouteThreads * 4) {
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (p.residual) v = *reinterpret_cast<const float4*>(p.h + j);
+    *reinterpret_cast<float4*>(p.y + j) = v;
   }
+  cluster.sync();          // all logits have landed in CTA 0
+  if (crank != 0) return;
 
-  __shared__ int s_last;
-  __threadfence();
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    unsigned int tk = atomicAdd(p.ticket, 1u);
-    s_last = (tk == gridDim.x - 1);
-  }
-  __syncthreads();
-  if (!s_last) return;
-  if (threadIdx.x == 0) *p.ticket = 0u;
-  __threadfence();
-
-  // ------------------------------------------------------------- finalise
-  __shared__ int s_ids[DX_MAX_PAIRS];
-  __shared__ float s_w[DX_MAX_PAIRS];
-  __shared__ int s_scan[8];
-  __shared__ unsigned int s_ballot[8];
-  __shared__ int s_perm[DX_MAX_PAIRS];
-  const int K = p.K, E = p.E, k = p.k, P = K * k;
-
-  for (int tt = warp; tt < K; tt += 8) {
+  // top-k and gate weights, one warp per token
+  for (int tt = warp; tt < K; tt += kRouteWarps) {
     unsigned long long key[8];
     float zv[8];
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
       int ee = lane + 32 * j;
       if (ee < E) {
-        zv[j] = __ldcg(p.z + tt * E + ee);
+        zv[j] = s_z[tt * E + ee];
         key[j] = ((unsigned long long)dx_orderable(zv[j]) << 32) | (unsigned long long)(0xffffffffu - (unsigned)ee);
       } else {
         zv[j] = 0.f;
@@ -196,7 +276,7 @@ __global__ void __launch_bounds__(256) dx_route_kernel(DxRouteParams p) {
   const unsigned int bal = __ballot_sync(0xffffffffu, flag);
   if (lane == 0) s_ballot[warp] = bal;
   int ucount;
-  const int upos = block_exclusive_scan(flag, s_scan, ucount);   // also orders s_ballot
+  const int upos = block_exclusive_scan(flag, s_scan, ucount);   // its barriers also publish s_ballot
   if (me < E) {
     if (p.offsets) p.offsets[me] = off;
     int i = 0;
@@ -209,12 +289,12 @@ __global__ void __launch_bounds__(256) dx_route_kernel(DxRouteParams p) {
     if (p.union_count) *p.union_count = ucount;
   }
   if (p.union_mask && me < (E + 63) / 64) {
-    unsigned long long lo = s_ballot[2 * me], hi = (2 * me + 1 < 8) ? s_ballot[2 * me + 1] : 0u;
+    unsigned long long lo = s_ballot[2 * me], hi = (2 * me + 1 < kRouteWarps) ? s_ballot[2 * me + 1] : 0u;
     p.union_mask[me] = lo | (hi << 32);
   }
   __syncthreads();
   if (p.perm)
-    for (int q = me; q < P; q += 256) p.perm[q] = s_perm[q];
+    for (int q = me; q < P; q += kRouteThreads) p.perm[q] = s_perm[q];
 
   // work list
   DxWork* W = p.work;
@@ -278,9 +358,24 @@ __global__ void __launch_bounds__(256) dx_route_kernel(DxRouteParams p) {
 
 }  // namespace
 
-cudaError_t dx_launch_route(const DxRouteParams& p, int weight_dtype, cudaStream_t st) {
-  const int grid = p.K * ((p.E + 7) / 8);
-  if (weight_dtype == DX_DTYPE_BF16)
-    return dx_launch_pdl(DX_PDL_ROUTE, dx_route_kernel<__nv_bfloat16>, dim3(grid), dim3(256), 0, st, p);
-  return dx_launch_pdl(DX_PDL_ROUTE, dx_route_kernel<float>, dim3(grid), dim3(256), 0, st, p);
+cudaError_t dx_launch_route(const DxRouteParams& p_in, int weight_dtype, cudaStream_t st) {
+  DxRouteParams p = p_in;
+  // as many block rows per pass as fit in 64 KB of shared memory (at most kTokGroup)
+  int tg = (64 * 1024) / (p.H * 4);
+  if (tg > kTokGroup) tg = kTokGroup;
+  if (tg > p.K) tg = p.K;
+  if (tg < 1) tg = 1;
+  p.tok_group = tg;
+  const size_t smem = (size_t)tg * p.H * 4;
+  cudaError_t e;
+  if (weight_dtype == DX_DTYPE_BF16) {
+    e = cudaFuncSetAttribute(dx_route_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024);
+    if (e != cudaSuccess) return e;
+    return dx_launch_pdl(DX_PDL_ROUTE, dx_route_kernel<__nv_bfloat16>, dim3(kRouteCluster), dim3(kRouteThreads), smem,
+                         st, kRouteCluster, p);
+  }
+  e = cudaFuncSetAttribute(dx_route_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024);
+  if (e != cudaSuccess) return e;
+  return dx_launch_pdl(DX_PDL_ROUTE, dx_route_kernel<float>, dim3(kRouteCluster), dim3(kRouteThreads), smem, st,
+                       kRouteCluster, p);
 }
