@@ -17,7 +17,8 @@ import torch
 from .synth import DTYPE_BF16, LayerShape
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libdraftexpert.so")
+# DX_LIB_PATH in the environment points the binding at another build of the library (e.g. a debug build)
+LIB_PATH = os.environ.get("DX_LIB_PATH") or os.path.join(_HERE, "libdraftexpert.so")
 
 DX_OK = 0
 STATUS_NAMES = {0: "DX_OK", 1: "DX_ERR_INVALID_ARG", 2: "DX_ERR_SHAPE", 3: "DX_ERR_CUDA", 4: "DX_ERR_OOM",

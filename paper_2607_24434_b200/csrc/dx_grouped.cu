@@ -76,6 +76,8 @@ __device__ __forceinline__ void mma_k8(float (&d)[4], uint32_t a0, uint32_t a1, 
                : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
                : "r"(a0), "r"(a1), "r"(b0));
 }
+// silu with the hardware exponential and reciprocal (relative error ~1e-6, far inside the parity tolerance)
+__device__ __forceinline__ float fast_silu(float x) { return __fdividef(x, 1.0f + __expf(-x)); }
 // x = hi + lo with hi, lo bf16 (lo is the rounding residual of hi)
 __device__ __forceinline__ void split_bf16(float x, __nv_bfloat16& hi, __nv_bfloat16& lo) {
   hi = __float2bfloat16_rn(x);
@@ -364,13 +366,17 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
         uint32_t bhi[NT], blo[NT];
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
-          float4 t = partial[((buf * 8 + 0) * NT + nt) * 32 + lane];
+          float4 q[8];
 #pragma unroll
-          for (int w = 1; w < 8; ++w) {
-            const float4 q = partial[((buf * 8 + w) * NT + nt) * 32 + lane];
-            t.x += q.x; t.y += q.y; t.z += q.z; t.w += q.w;
-          }
-          const float a0 = dx_silu(t.x) * t.y, a1 = dx_silu(t.z) * t.w;
+          for (int w = 0; w < 8; ++w) q[w] = partial[((buf * 8 + w) * NT + nt) * 32 + lane];
+#pragma unroll
+          for (int st = 1; st < 8; st <<= 1)
+#pragma unroll
+            for (int w = 0; w < 8; w += 2 * st) {
+              q[w].x += q[w + st].x; q[w].y += q[w + st].y; q[w].z += q[w + st].z; q[w].w += q[w + st].w;
+            }
+          const float4 t = q[0];
+          const float a0 = fast_silu(t.x) * t.y, a1 = fast_silu(t.z) * t.w;
           __nv_bfloat16 h0, l0, h1, l1;
           split_bf16(a0, h0, l0);
           split_bf16(a1, h1, l1);
