@@ -175,6 +175,25 @@ dx_status spec_accept(dx_ctx* ctx, const float* h, int32_t M, const void* W_lm, 
                       int32_t w_dtype, const int32_t* draft, int32_t K, int32_t rms_norm,
                       int32_t* target, int32_t* n_accept, int32_t* next_token, void* stream);
 
+/* ---- greedy verification without any allocation ----------------------------------------------------------------
+ * (No counterpart in the paper: an addition for callers of this library that cannot allocate device memory --
+ * a serving thread whose memory pool was sized once at start-up and where a late cudaMalloc is forbidden or
+ * would stall every stream, a plugin that is handed buffers and a stream but no allocator.  dx_create
+ * allocates, so such callers cannot use a context.)  Same inputs, outputs and results as spec_accept, but without a context handle: the kernels' scratch
+ * (one packed 64-bit argmax key per row and a ticket) is a static device array inside the library, 256-byte
+ * aligned and sized for at most 16 rows, which every GPU that loads the library keeps until the process exits.
+ * The call performs no cudaMalloc / cudaFree and uses no allocating library routine.
+ *   - M > 16 (or any size spec_accept rejects) returns DX_ERR_UNSUPPORTED; nothing is truncated.
+ *   - The first call on a device resolves the array's device address (cudaGetSymbolAddress, with that device
+ *     current) and reads two device attributes; make that first call before any stream capture.
+ *   - All calls share the one array, which keeps the previous call's contents; each call clears it on `stream`
+ *     first.  Calls that overlap on the GPU (different streams, no ordering between them) race on it and give
+ *     undefined results: keep calls to this entry point on one stream or order them yourself.
+ * All tensor pointers are device pointers, as for spec_accept. */
+dx_status spec_accept_noalloc(const float* h, int32_t M, const void* W_lm, int32_t V, int32_t H, int32_t w_dtype,
+                              const int32_t* draft, int32_t K, int32_t rms_norm, int32_t* target,
+                              int32_t* n_accept, int32_t* next_token, void* stream);
+
 /* ---- accelerator expert cache: C and P of Algorithm 1, Sec. 3.5 ----------------------------------------------
  * A cache owns n_layers * slots_per_layer HBM slots of blob_bytes each (allocated in create), a side stream
  * for transfers and one event per slot.  Routed experts live in a host pool the caller registers blob by

@@ -69,6 +69,7 @@ SIGNATURES = {
     "moe_verify_experts": (_I, [_P, _P, _I, _P, _P]),
     "moe_verify_block_residual": (_I, [_P, _P, _P, _I, _P, _P, _P, _P, _P, _P, _P, _P]),
     "spec_accept": (_I, [_P, _P, _I, _P, _I, _I, _I, _P, _I, _I, _P, _P, _P, _P]),
+    "spec_accept_noalloc": (_I, [_P, _I, _P, _I, _I, _I, _P, _I, _I, _P, _P, _P, _P]),
     "expert_cache_create": (_I, [_P, _I, _I, _I, C.c_size_t, C.POINTER(_P)]),
     "expert_cache_destroy": (_I, [_P]),
     "expert_cache_register": (_I, [_P, _I, _I, _P]),
@@ -322,4 +323,18 @@ def spec_accept(ctx: Context, h: torch.Tensor, W_lm: torch.Tensor, draft: torch.
     _check(ctx.lib.spec_accept(ctx.handle, _ptr(h), M, _ptr(W_lm), V, H, wd, _ptr(draft), int(draft.shape[0]),
                                1 if rms_norm else 0, _ptr(out["target"]), _ptr(out["n_accept"]),
                                _ptr(out["next_token"]), _stream()), "spec_accept")
+    return out
+
+
+def spec_accept_noalloc(h: torch.Tensor, W_lm: torch.Tensor, draft: torch.Tensor, out: Dict[str, torch.Tensor],
+                        rms_norm: bool = False) -> Dict[str, torch.Tensor]:
+    """Greedy verification through the entry point that allocates nothing: no context, and the caller passes
+    the output tensors (``target`` [M], ``n_accept`` [1], ``next_token`` [1], int32, on the device) because
+    this wrapper does not allocate either.  For callers that cannot allocate device memory (a memory pool fixed
+    at start-up, or no allocator at hand).  At most 16 rows; calls must not overlap on the GPU."""
+    M, H = h.shape
+    wd = 1 if W_lm.dtype == torch.bfloat16 else 0
+    _check(load().spec_accept_noalloc(_ptr(h), M, _ptr(W_lm), W_lm.shape[0], H, wd, _ptr(draft), int(draft.shape[0]),
+                                      1 if rms_norm else 0, _ptr(out["target"]), _ptr(out["n_accept"]),
+                                      _ptr(out["next_token"]), _stream()), "spec_accept_noalloc")
     return out

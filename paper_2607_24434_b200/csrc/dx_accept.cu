@@ -266,3 +266,81 @@ cudaError_t dx_launch_accept(dx_ctx* ctx, const float* h, int M, const void* W_l
     return dx_launch_pdl(DX_PDL_ACCEPT, dx_accept_bf16_kernel<2>, dim3(ctx->sm_count), dim3(512), smem, st, 1, p);
   }
 }
+
+// ---------------------------------------------------------------------------------------------------------
+// spec_accept_noalloc: greedy verification for callers that must not allocate.
+//
+// Some callers cannot call cudaMalloc (or anything that does): a thread inside a serving loop whose memory
+// pool was sized once at start-up (a late cudaMalloc is forbidden there, or would stall every stream), a
+// plugin that is handed streams and buffers but no allocator.  For them this entry point needs no context handle: the scratch the
+// kernels use (the packed 64-bit argmax key of every row and the "last CTA" ticket) lives in the file-scope
+// device array below, which every GPU that loads the library holds until the process exits.
+//
+// The array's name is only a host-side stand-in in host code, not a device address, so the address is looked
+// up once per device with cudaGetSymbolAddress and that pointer is what the kernels get.
+constexpr int kNoAllocMaxRows = DX_MAX_M;                       // rows (M) the static scratch is sized for
+static __device__ __align__(256) unsigned long long g_noalloc_scratch[kNoAllocMaxRows + 2];   // keys, then ticket
+
+namespace {
+struct NoAllocDevice {
+  bool ready = false;
+  unsigned long long* scratch = nullptr;
+  int sm_count = 0;
+  int smem_optin = 0;
+};
+NoAllocDevice g_noalloc_dev[64];
+}  // namespace
+
+extern "C" dx_status spec_accept_noalloc(const float* h, int32_t M, const void* W_lm, int32_t V, int32_t H,
+                                         int32_t w_dtype, const int32_t* draft, int32_t K, int32_t rms_norm,
+                                         int32_t* target, int32_t* n_accept, int32_t* next_token, void* stream) {
+  if (!h || !W_lm || !target || !n_accept || !next_token) return DX_ERR_INVALID_ARG;
+  if (K > 0 && !draft) return DX_ERR_INVALID_ARG;
+  if (M < 1 || V < 1 || K < 0) return DX_ERR_SHAPE;
+  if (w_dtype != DX_DTYPE_FP32 && w_dtype != DX_DTYPE_BF16) return DX_ERR_INVALID_ARG;
+  // sizes beyond what the static scratch (and the kernels) are built for are refused, never truncated
+  if (M > kNoAllocMaxRows || K > DX_MAX_K || H <= 0 || H > DX_MAX_H || H % 256) return DX_ERR_UNSUPPORTED;
+  if (((uintptr_t)h) % 16 || ((uintptr_t)W_lm) % 16) return DX_ERR_INVALID_ARG;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return DX_ERR_CUDA;
+  NoAllocDevice& d = g_noalloc_dev[dev];
+  if (!d.ready) {
+    // first call on this device (with this device current): resolve the device address of the scratch array
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess || ptr == nullptr) return DX_ERR_CUDA;
+    if (cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return DX_ERR_CUDA;
+    if (cudaDeviceGetAttribute(&d.smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess)
+      return DX_ERR_CUDA;
+    d.scratch = static_cast<unsigned long long*>(ptr);
+    d.ready = true;
+  }
+  const int NT = (M + 7) / 8;
+  const size_t smem = (size_t)NT * (H / 32) * 32 * 16 * 2;
+  if (w_dtype == DX_DTYPE_BF16 && smem > (size_t)d.smem_optin) return DX_ERR_UNSUPPORTED;
+  cudaStream_t st = (cudaStream_t)stream;
+  // the array keeps whatever the last call left; keys and ticket must start at zero
+  if (cudaMemsetAsync(d.scratch, 0, sizeof(unsigned long long) * (kNoAllocMaxRows + 2), st) != cudaSuccess)
+    return DX_ERR_CUDA;
+  AcceptParams p{h, M, V, H, W_lm, draft, K, rms_norm, target, n_accept, next_token, d.scratch,
+                 reinterpret_cast<unsigned int*>(d.scratch + kNoAllocMaxRows)};
+  cudaError_t e;
+  if (w_dtype == DX_DTYPE_FP32) {
+    int grid = (V + 7) / 8;
+    if (grid > d.sm_count * 8) grid = d.sm_count * 8;
+    dx_accept_fp32_kernel<<<grid, 256, 0, st>>>(p);
+    e = cudaGetLastError();
+  } else if (NT == 1) {
+    e = cudaFuncSetAttribute(dx_accept_bf16_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e == cudaSuccess) {
+      dx_accept_bf16_kernel<1><<<d.sm_count, 512, smem, st>>>(p);
+      e = cudaGetLastError();
+    }
+  } else {
+    e = cudaFuncSetAttribute(dx_accept_bf16_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e == cudaSuccess) {
+      dx_accept_bf16_kernel<2><<<d.sm_count, 512, smem, st>>>(p);
+      e = cudaGetLastError();
+    }
+  }
+  return e == cudaSuccess ? DX_OK : DX_ERR_CUDA;
+}
