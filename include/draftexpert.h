@@ -153,6 +153,17 @@ dx_status moe_verify_route(dx_layer* layer, const float* h, int32_t K, float* y,
                            int32_t* topk_ids, float* topk_w, uint64_t* union_mask, int32_t* union_ids,
                            int32_t* union_count, int32_t* offsets, int32_t* perm, void* stream);
 dx_status moe_verify_experts(dx_layer* layer, const float* h, int32_t K, float* y, void* stream);
+/* The expert half restricted to a window of the union: union positions [first_union, first_union + n_union)
+ * of the ascending union_ids list, plus the shared experts iff include_shared != 0.  y is added to (the route
+ * half initialised it), so a union that does not fit the cache slots is evaluated in several windows ("waves"),
+ * each after staging its experts; exactly one window must include the shared experts. */
+dx_status moe_verify_experts_range(dx_layer* layer, const float* h, int32_t K, float* y, int32_t first_union,
+                                   int32_t n_union, int32_t include_shared, void* stream);
+/* The two halves of moe_draft_step, for layers whose routed experts are staged through a cache: after
+ * moe_draft_route the caller reads topk_ids[0] (= e1), makes that expert resident, then runs the experts. */
+dx_status moe_draft_route(dx_layer* layer, const float* h, float* y, int32_t* topk_ids, float* topk_w,
+                          void* stream);
+dx_status moe_draft_experts(dx_layer* layer, const float* h, float* y, void* stream);
 
 /* ---- pre-norm residual forms for layer stacks (synthetic stacks stub attention out) --------------------------
  * h_out = h_in + MoE(RMSNorm(h_in)) with unit gain and eps 1e-6, MoE = Eq. 4 (verify, [K,H]) or Eq. 5 (draft,
@@ -196,10 +207,13 @@ dx_status spec_accept_noalloc(const float* h, int32_t M, const void* W_lm, int32
 
 /* ---- accelerator expert cache: C and P of Algorithm 1, Sec. 3.5 ----------------------------------------------
  * A cache owns n_layers * slots_per_layer HBM slots of blob_bytes each (allocated in create), a side stream
- * for transfers and one event per slot.  Routed experts live in a host pool the caller registers blob by
+ * for transfers and one event per slot.  With ctx == NULL, create builds a bookkeeping-only cache (no device
+ * memory, no copies, streams ignored) that runs the same policy on the host, e.g. to plan or to test it.  Routed experts live in a host pool the caller registers blob by
  * blob (pinned host pointers, borrowed).  All id arrays are HOST pointers.
- *   prefetch: for each id not cached and not in flight, pick the least-recently-used free slot and start a
- *             non-blocking copy on the side stream (Algorithm 1: prefetch U_hat \ (C u P)); never blocks.
+ *   prefetch: for each id not cached and not in flight, take a free slot, else the least-recently-used slot
+ *             that is neither protected (prefetched this step and not used yet) nor pinned, and start a
+ *             non-blocking copy on the side stream (Algorithm 1: prefetch U_hat \ (C u P)); never blocks; a
+ *             hint that finds no slot is dropped.
  *   stage:    make ids resident now: cached ones are hits; in-flight ones are waited for; the rest are copied
  *             on demand.  `stream` is made to wait (cudaStreamWaitEvent) for exactly the copies it needs.
  *             n must not exceed slots_per_layer (DX_ERR_CACHE_FULL); larger unions are staged in waves.
@@ -221,6 +235,9 @@ dx_status expert_cache_create(dx_ctx* ctx, int32_t n_layers, int32_t n_experts, 
                               size_t blob_bytes, dx_cache** out);
 dx_status expert_cache_destroy(dx_cache* cache);
 dx_status expert_cache_register(dx_cache* cache, int32_t layer, int32_t expert, const void* pinned_host_blob);
+/* Start of a decode step (Algorithm 1, line 1: P <- empty): experts prefetched earlier and never used since
+ * are counted as wasted and stop being protected from eviction. */
+dx_status expert_cache_begin_step(dx_cache* cache);
 dx_status expert_cache_prefetch(dx_cache* cache, int32_t layer, const int32_t* host_ids, int32_t n);
 dx_status expert_cache_stage(dx_cache* cache, int32_t layer, const int32_t* host_ids, int32_t n, void* stream);
 dx_status expert_cache_wait(dx_cache* cache, int32_t layer, const int32_t* host_ids, int32_t n, void* stream,

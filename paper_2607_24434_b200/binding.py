@@ -67,12 +67,16 @@ SIGNATURES = {
     "moe_verify_block": (_I, [_P, _P, _I, _P, _P, _P, _P, _P, _P, _P, _P, _P]),
     "moe_verify_route": (_I, [_P, _P, _I, _P, _P, _P, _P, _P, _P, _P, _P, _P]),
     "moe_verify_experts": (_I, [_P, _P, _I, _P, _P]),
+    "moe_verify_experts_range": (_I, [_P, _P, _I, _P, _I, _I, _I, _P]),
+    "moe_draft_route": (_I, [_P, _P, _P, _P, _P, _P]),
+    "moe_draft_experts": (_I, [_P, _P, _P, _P]),
     "moe_verify_block_residual": (_I, [_P, _P, _P, _I, _P, _P, _P, _P, _P, _P, _P, _P]),
     "spec_accept": (_I, [_P, _P, _I, _P, _I, _I, _I, _P, _I, _I, _P, _P, _P, _P]),
     "spec_accept_noalloc": (_I, [_P, _I, _P, _I, _I, _I, _P, _I, _I, _P, _P, _P, _P]),
     "expert_cache_create": (_I, [_P, _I, _I, _I, C.c_size_t, C.POINTER(_P)]),
     "expert_cache_destroy": (_I, [_P]),
     "expert_cache_register": (_I, [_P, _I, _I, _P]),
+    "expert_cache_begin_step": (_I, [_P]),
     "expert_cache_prefetch": (_I, [_P, _I, _P, _I]),
     "expert_cache_stage": (_I, [_P, _I, _P, _I, _P]),
     "expert_cache_wait": (_I, [_P, _I, _P, _I, _P, C.c_double]),
@@ -337,4 +341,115 @@ def spec_accept_noalloc(h: torch.Tensor, W_lm: torch.Tensor, draft: torch.Tensor
     _check(load().spec_accept_noalloc(_ptr(h), M, _ptr(W_lm), W_lm.shape[0], H, wd, _ptr(draft), int(draft.shape[0]),
                                       1 if rms_norm else 0, _ptr(out["target"]), _ptr(out["n_accept"]),
                                       _ptr(out["next_token"]), _stream()), "spec_accept_noalloc")
+    return out
+
+
+class ExpertCache:
+    """Handle of an accelerator expert cache (Sec. 3.5).  ``ctx=None`` gives the bookkeeping-only cache."""
+
+    def __init__(self, ctx: Optional[Context], n_layers: int, n_experts: int, slots: int, blob_bytes: int):
+        self.lib = load()
+        self.ctx = ctx
+        self.n_layers, self.n_experts, self.slots, self.blob_bytes = n_layers, n_experts, slots, blob_bytes
+        h = _P()
+        _check(self.lib.expert_cache_create(ctx.handle if ctx else None, n_layers, n_experts, slots, blob_bytes,
+                                            C.byref(h)), "expert_cache_create")
+        self.handle = h
+        self._keep: List[object] = []
+
+    def close(self) -> None:
+        if self.handle:
+            self.lib.expert_cache_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    @staticmethod
+    def _ids(ids: Sequence[int]):
+        arr = (C.c_int32 * len(ids))(*[int(i) for i in ids])
+        return arr, len(ids)
+
+    def register(self, layer: int, expert: int, pinned_blob: torch.Tensor) -> None:
+        self._keep.append(pinned_blob)
+        _check(self.lib.expert_cache_register(self.handle, layer, expert, _ptr(pinned_blob)), "expert_cache_register")
+
+    def register_fake(self, layer: int, expert: int) -> None:
+        """Bookkeeping-only caches never read the blob; any non-null 16-byte-aligned address will do."""
+        _check(self.lib.expert_cache_register(self.handle, layer, expert, 4096), "expert_cache_register")
+
+    def attach(self, layer_handle: "Layer", layer: int) -> None:
+        _check(self.lib.dx_layer_attach_cache(layer_handle.handle, self.handle, layer), "dx_layer_attach_cache")
+
+    def begin_step(self) -> None:
+        _check(self.lib.expert_cache_begin_step(self.handle), "expert_cache_begin_step")
+
+    def prefetch(self, layer: int, ids: Sequence[int]) -> None:
+        arr, n = self._ids(ids)
+        _check(self.lib.expert_cache_prefetch(self.handle, layer, arr, n), "expert_cache_prefetch")
+
+    def stage(self, layer: int, ids: Sequence[int]) -> None:
+        arr, n = self._ids(ids)
+        st = _stream() if self.ctx else None
+        _check(self.lib.expert_cache_stage(self.handle, layer, arr, n, st), "expert_cache_stage")
+
+    def wait(self, layer: int, ids: Sequence[int], timeout_s: float = 0.0) -> None:
+        arr, n = self._ids(ids)
+        st = _stream() if self.ctx else None
+        _check(self.lib.expert_cache_wait(self.handle, layer, arr, n, st, timeout_s), "expert_cache_wait")
+
+    def stats(self) -> Dict[str, int]:
+        s = CacheStats()
+        _check(self.lib.expert_cache_stats(self.handle, C.byref(s)), "expert_cache_stats")
+        return {name: int(getattr(s, name)) for name, _ in CacheStats._fields_}
+
+    def query(self, layer: int, expert: int) -> Tuple[int, int]:
+        slot, infl = _I(0), _I(0)
+        _check(self.lib.expert_cache_query(self.handle, layer, expert, C.byref(slot), C.byref(infl)),
+               "expert_cache_query")
+        return slot.value, infl.value
+
+
+def moe_verify_experts_range(layer: Layer, h: torch.Tensor, y: torch.Tensor, first_union: int, n_union: int,
+                             include_shared: bool) -> None:
+    _check(layer.lib.moe_verify_experts_range(layer.handle, _ptr(h), h.shape[0], _ptr(y), first_union, n_union,
+                                              1 if include_shared else 0, _stream()), "moe_verify_experts_range")
+
+
+def moe_draft_route(layer: Layer, h: torch.Tensor, y: torch.Tensor, out: Dict[str, torch.Tensor]) -> None:
+    _check(layer.lib.moe_draft_route(layer.handle, _ptr(h), _ptr(y), _ptr(out["topk_ids"]), _ptr(out["topk_w"]),
+                                     _stream()), "moe_draft_route")
+
+
+def moe_draft_experts(layer: Layer, h: torch.Tensor, y: torch.Tensor) -> None:
+    _check(layer.lib.moe_draft_experts(layer.handle, _ptr(h), _ptr(y), _stream()), "moe_draft_experts")
+
+
+def moe_verify_block_cached(layer: Layer, cache: ExpertCache, layer_index: int, h: torch.Tensor,
+                            y: Optional[torch.Tensor] = None, out: Optional[Dict[str, torch.Tensor]] = None):
+    """Verify block on a layer whose routed experts come through ``cache``: route, read the union on the host
+    (the one host round trip on-demand loading needs), then stage and evaluate the union in waves of at most
+    ``cache.slots`` experts in ascending id order, shared experts with the first wave."""
+    K = h.shape[0]
+    if out is None:
+        out = _routing_buffers(layer.shape, K, h.device)
+    if y is None:
+        y = torch.empty_like(h)
+    moe_verify_route(layer, h, y, out)
+    n = int(out["union_count"].item())
+    ids = out["union_ids"][:n].tolist()
+    S = cache.slots
+    first = 0
+    while True:
+        wave = ids[first:first + S]
+        cache.stage(layer_index, wave)
+        moe_verify_experts_range(layer, h, y, first, len(wave), include_shared=(first == 0))
+        first += len(wave)
+        if first >= n:
+            break
+    out["y"] = y
+    out["union_list"] = ids
     return out

@@ -247,7 +247,7 @@ static dx_status do_route(dx_layer* L, const float* h, int K, float* y, const Ro
 }
 
 static dx_status do_experts(dx_layer* L, const float* h, int K, float* y, bool draft, bool residual,
-                            cudaStream_t st) {
+                            cudaStream_t st, int first_routed = 0, int n_routed = -1, bool do_static = true) {
   dx_ctx* ctx = L->ctx;
   const dx_layer_desc& d = L->desc;
   if (!h || !y || h == y) return DX_ERR_INVALID_ARG;
@@ -267,6 +267,9 @@ static dx_status do_experts(dx_layer* L, const float* h, int K, float* y, bool d
   p.shared_tiles = d.n_shared ? d.shared_inter / DX_TILE_I : 0;
   p.draft_tiles = draft ? d.draft_inter / DX_TILE_I : 0;
   p.gamma = d.draft_gamma;
+  p.first_routed = first_routed;
+  p.n_routed = n_routed;
+  p.do_static = do_static ? 1 : 0;
   DX_CUDA(ctx, dx_launch_experts(ctx, p, L->desc.weight_dtype, K, st));
   ctx->launches++;
   if (L->cache) dx_cache_note_use(L->cache, L->cache_layer, st);
@@ -304,6 +307,25 @@ extern "C" dx_status moe_verify_route(dx_layer* L, const float* h, int32_t K, fl
 extern "C" dx_status moe_verify_experts(dx_layer* L, const float* h, int32_t K, float* y, void* stream) {
   if (!L) return DX_ERR_INVALID_ARG;
   return do_experts(L, h, K, y, false, false, (cudaStream_t)stream);
+}
+
+extern "C" dx_status moe_verify_experts_range(dx_layer* L, const float* h, int32_t K, float* y, int32_t first_union,
+                                              int32_t n_union, int32_t include_shared, void* stream) {
+  if (!L) return DX_ERR_INVALID_ARG;
+  if (first_union < 0 || n_union < 0) return DX_ERR_INVALID_ARG;
+  return do_experts(L, h, K, y, false, false, (cudaStream_t)stream, first_union, n_union, include_shared != 0);
+}
+
+extern "C" dx_status moe_draft_route(dx_layer* L, const float* h, float* y, int32_t* topk_ids, float* topk_w,
+                                     void* stream) {
+  if (!L) return DX_ERR_INVALID_ARG;
+  RouteOut o{topk_ids, topk_w, nullptr, nullptr, nullptr, nullptr, nullptr};
+  return do_route(L, h, 1, y, o, true, false, (cudaStream_t)stream);
+}
+
+extern "C" dx_status moe_draft_experts(dx_layer* L, const float* h, float* y, void* stream) {
+  if (!L) return DX_ERR_INVALID_ARG;
+  return do_experts(L, h, 1, y, true, false, (cudaStream_t)stream);
 }
 
 extern "C" dx_status moe_verify_block(dx_layer* L, const float* h, int32_t K, float* y, int32_t* topk_ids,

@@ -1,15 +1,362 @@
-// Accelerator expert cache (Sec. 3.5, Algorithm 1: cache C, in-flight set P).
+// Accelerator expert cache (Sec. 3.5 and Algorithm 1: cache C, in-flight set P).
+//
+// Host-side state machine plus the transfers it drives.  Per layer there are S
+// HBM slots of one expert blob each.  Routed experts live in pinned host memory
+// (registered blob by blob) and are copied into slots with cudaMemcpyAsync on
+// one side stream, so transfers are ordered among themselves and overlap with
+// compute; one event per slot lets the compute stream wait for exactly the
+// copies it needs.  The layer's device blob table is patched on the compute
+// stream (tiny kernel, entries passed by value) right before the kernels that
+// read it.  Policy (deterministic given the call sequence):
+//   - stamp = global access counter; a hit, a prefetch and an on-demand load set stamp = now;
+//   - P = slots prefetched since the last begin_step and not used yet: they are "protected";
+//   - prefetch victim: free slot (lowest index), else least-recently-used unprotected slot, else drop the hint;
+//   - stage victim:    free slot, else LRU unprotected slot not pinned by this call, else LRU protected
+//                      slot not pinned by this call (counted as a wasted prefetch), else DX_ERR_CACHE_FULL;
+//   - an id already cached (landed or in flight) is never copied again.
+// With ctx == NULL the cache is bookkeeping only: the same policy without device memory or copies.
+#include <chrono>
+#include <new>
+#include <vector>
+
 #include "dx_internal.cuh"
 
-const void** dx_cache_table(dx_cache*, int) { return nullptr; }
-void dx_cache_note_use(dx_cache*, int, cudaStream_t) {}
+struct DxSlot {
+  int expert = -1;
+  unsigned long long stamp = 0;
+  bool prefetched = false;   // member of P: prefetched this step, not used yet
+  bool copy_pending = false; // a copy was issued and not yet seen complete
+  cudaEvent_t ev = nullptr;
+};
 
-extern "C" dx_status dx_layer_attach_cache(dx_layer*, dx_cache*, int32_t) { return DX_ERR_UNSUPPORTED; }
-extern "C" dx_status expert_cache_create(dx_ctx*, int32_t, int32_t, int32_t, size_t, dx_cache**) { return DX_ERR_UNSUPPORTED; }
-extern "C" dx_status expert_cache_destroy(dx_cache*) { return DX_ERR_UNSUPPORTED; }
-extern "C" dx_status expert_cache_register(dx_cache*, int32_t, int32_t, const void*) { return DX_ERR_UNSUPPORTED; }
-extern "C" dx_status expert_cache_prefetch(dx_cache*, int32_t, const int32_t*, int32_t) { return DX_ERR_UNSUPPORTED; }
-extern "C" dx_status expert_cache_stage(dx_cache*, int32_t, const int32_t*, int32_t, void*) { return DX_ERR_UNSUPPORTED; }
-extern "C" dx_status expert_cache_wait(dx_cache*, int32_t, const int32_t*, int32_t, void*, double) { return DX_ERR_UNSUPPORTED; }
-extern "C" dx_status expert_cache_stats(dx_cache*, dx_cache_stats*) { return DX_ERR_UNSUPPORTED; }
-extern "C" dx_status expert_cache_query(dx_cache*, int32_t, int32_t, int32_t*, int32_t*) { return DX_ERR_UNSUPPORTED; }
+struct DxTablePatch {
+  int n;
+  int idx[32];
+  const void* ptr[32];
+};
+
+struct dx_cache {
+  dx_ctx* ctx;
+  int L, E, S;
+  size_t blob_bytes;
+  unsigned char* slab;
+  cudaStream_t copy_stream;
+  unsigned long long clock;
+  dx_cache_stats stats;
+  std::vector<const void*> host_blob;   // [L*E]
+  std::vector<DxSlot> slots;            // [L*S]
+  std::vector<int> slot_of;             // [L*E] -> slot or -1
+  std::vector<dx_layer*> layer;         // attached layer per cache layer
+  std::vector<cudaEvent_t> used_ev;     // last compute use of the layer's slots
+  std::vector<char> used_valid;
+  std::vector<std::vector<std::pair<int, const void*>>> pending;   // table patches not yet applied, per layer
+};
+
+namespace {
+
+__global__ void dx_table_patch_kernel(const void** table, DxTablePatch patch) {
+  dx_pdl_wait();
+  if ((int)threadIdx.x < patch.n) table[patch.idx[threadIdx.x]] = patch.ptr[threadIdx.x];
+}
+
+inline DxSlot& slot_ref(dx_cache* c, int layer, int s) { return c->slots[(size_t)layer * c->S + s]; }
+inline void* slot_ptr(dx_cache* c, int layer, int s) {
+  return c->slab ? c->slab + ((size_t)layer * c->S + s) * c->blob_bytes : nullptr;
+}
+
+// victim search; protected_ok: may take a slot of P; pinned: slots of the call in progress
+int find_victim(dx_cache* c, int layer, const std::vector<char>& pinned, bool protected_ok, bool* was_protected) {
+  *was_protected = false;
+  for (int s = 0; s < c->S; ++s)
+    if (slot_ref(c, layer, s).expert < 0 && !pinned[s]) return s;
+  int best = -1;
+  for (int s = 0; s < c->S; ++s) {
+    const DxSlot& sl = slot_ref(c, layer, s);
+    if (pinned[s] || sl.prefetched) continue;
+    if (best < 0 || sl.stamp < slot_ref(c, layer, best).stamp) best = s;
+  }
+  if (best >= 0 || !protected_ok) return best;
+  for (int s = 0; s < c->S; ++s) {
+    const DxSlot& sl = slot_ref(c, layer, s);
+    if (pinned[s]) continue;
+    if (best < 0 || sl.stamp < slot_ref(c, layer, best).stamp) best = s;
+  }
+  if (best >= 0) *was_protected = true;
+  return best;
+}
+
+// puts expert e of `layer` into slot s (evicting what is there) and starts the copy
+dx_status load_into(dx_cache* c, int layer, int s, int e, bool as_prefetch) {
+  DxSlot& sl = slot_ref(c, layer, s);
+  if (sl.expert >= 0) {
+    c->stats.evictions++;
+    c->slot_of[(size_t)layer * c->E + sl.expert] = -1;
+    c->pending[layer].push_back({sl.expert, nullptr});
+  }
+  sl.expert = e;
+  sl.prefetched = as_prefetch;
+  sl.stamp = ++c->clock;
+  c->slot_of[(size_t)layer * c->E + e] = s;
+  c->pending[layer].push_back({e, slot_ptr(c, layer, s)});
+  c->stats.bytes_h2d += (int64_t)c->blob_bytes;
+  if (c->ctx) {
+    // the slot may still be read by kernels already enqueued on the compute stream
+    if (c->used_valid[layer]) {
+      cudaError_t e0 = cudaStreamWaitEvent(c->copy_stream, c->used_ev[layer], 0);
+      if (e0 != cudaSuccess) { c->ctx->last_cuda = e0; return DX_ERR_CUDA; }
+    }
+    cudaError_t e1 = cudaMemcpyAsync(slot_ptr(c, layer, s), c->host_blob[(size_t)layer * c->E + e], c->blob_bytes,
+                                     cudaMemcpyHostToDevice, c->copy_stream);
+    if (e1 == cudaSuccess) e1 = cudaEventRecord(sl.ev, c->copy_stream);
+    if (e1 != cudaSuccess) { c->ctx->last_cuda = e1; return DX_ERR_CUDA; }
+    sl.copy_pending = true;
+  }
+  return DX_OK;
+}
+
+bool copy_done(dx_cache* c, DxSlot& sl) {
+  if (!sl.copy_pending) return true;
+  if (!c->ctx) { sl.copy_pending = false; return true; }
+  if (cudaEventQuery(sl.ev) == cudaSuccess) { sl.copy_pending = false; return true; }
+  return false;
+}
+
+// applies the layer's pending table patches on `st`
+dx_status flush_patches(dx_cache* c, int layer, cudaStream_t st) {
+  auto& pend = c->pending[layer];
+  dx_layer* L = c->layer[layer];
+  if (!c->ctx || !L) { pend.clear(); return DX_OK; }
+  const int base = L->desc.n_shared + 1;
+  // several patches may name the same expert (evicted, then loaded again): only the last one counts, and one
+  // launch must not carry two writes to the same table entry
+  {
+    std::vector<std::pair<int, const void*>> last;
+    for (size_t a = 0; a < pend.size(); ++a) {
+      bool later = false;
+      for (size_t b = a + 1; b < pend.size(); ++b)
+        if (pend[b].first == pend[a].first) { later = true; break; }
+      if (!later) last.push_back(pend[a]);
+    }
+    pend.swap(last);
+  }
+  size_t i = 0;
+  while (i < pend.size()) {
+    DxTablePatch patch;
+    patch.n = 0;
+    while (i < pend.size() && patch.n < 32) {
+      patch.idx[patch.n] = base + pend[i].first;
+      patch.ptr[patch.n] = pend[i].second;
+      L->table_host[base + pend[i].first] = pend[i].second;
+      ++patch.n;
+      ++i;
+    }
+    dx_table_patch_kernel<<<1, 32, 0, st>>>(L->table_dev, patch);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) { c->ctx->last_cuda = e; return DX_ERR_CUDA; }
+    c->ctx->launches++;
+  }
+  pend.clear();
+  return DX_OK;
+}
+
+dx_status check_ids(dx_cache* c, int layer, const int32_t* ids, int n) {
+  if (!c || (n > 0 && !ids) || n < 0) return DX_ERR_INVALID_ARG;
+  if (layer < 0 || layer >= c->L) return DX_ERR_INVALID_ARG;
+  for (int i = 0; i < n; ++i)
+    if (ids[i] < 0 || ids[i] >= c->E) return DX_ERR_INVALID_ARG;
+  return DX_OK;
+}
+
+}  // namespace
+
+void dx_cache_note_use(dx_cache* c, int layer, cudaStream_t st) {
+  if (!c || !c->ctx || layer < 0 || layer >= c->L) return;
+  if (cudaEventRecord(c->used_ev[layer], st) == cudaSuccess) c->used_valid[layer] = 1;
+}
+
+extern "C" dx_status expert_cache_create(dx_ctx* ctx, int32_t n_layers, int32_t n_experts, int32_t slots_per_layer,
+                                         size_t blob_bytes, dx_cache** out) {
+  if (!out) return DX_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (n_layers < 1 || n_experts < 1 || slots_per_layer < 1 || blob_bytes == 0 || blob_bytes % 128)
+    return DX_ERR_INVALID_ARG;
+  if (n_experts > DX_MAX_E) return DX_ERR_UNSUPPORTED;
+  dx_cache* c = new (std::nothrow) dx_cache();
+  if (!c) return DX_ERR_OOM;
+  c->ctx = ctx;
+  c->L = n_layers; c->E = n_experts; c->S = slots_per_layer;
+  c->blob_bytes = blob_bytes;
+  c->slab = nullptr;
+  c->copy_stream = nullptr;
+  c->clock = 0;
+  c->stats = dx_cache_stats{};
+  c->host_blob.assign((size_t)n_layers * n_experts, nullptr);
+  c->slots.assign((size_t)n_layers * slots_per_layer, DxSlot());
+  c->slot_of.assign((size_t)n_layers * n_experts, -1);
+  c->layer.assign(n_layers, nullptr);
+  c->used_ev.assign(n_layers, nullptr);
+  c->used_valid.assign(n_layers, 0);
+  c->pending.resize(n_layers);
+  if (ctx) {
+    cudaError_t e = cudaSetDevice(ctx->device);
+    if (e == cudaSuccess) e = cudaMalloc(&c->slab, (size_t)n_layers * slots_per_layer * blob_bytes);
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking);
+    for (size_t i = 0; e == cudaSuccess && i < c->slots.size(); ++i)
+      e = cudaEventCreateWithFlags(&c->slots[i].ev, cudaEventDisableTiming);
+    for (int l = 0; e == cudaSuccess && l < n_layers; ++l)
+      e = cudaEventCreateWithFlags(&c->used_ev[l], cudaEventDisableTiming);
+    if (e != cudaSuccess) {
+      ctx->last_cuda = e;
+      expert_cache_destroy(c);
+      return e == cudaErrorMemoryAllocation ? DX_ERR_OOM : DX_ERR_CUDA;
+    }
+  }
+  *out = c;
+  return DX_OK;
+}
+
+extern "C" dx_status expert_cache_destroy(dx_cache* c) {
+  if (!c) return DX_ERR_INVALID_ARG;
+  if (c->ctx) {
+    if (c->copy_stream) cudaStreamSynchronize(c->copy_stream);
+    for (auto& s : c->slots)
+      if (s.ev) cudaEventDestroy(s.ev);
+    for (auto& e : c->used_ev)
+      if (e) cudaEventDestroy(e);
+    if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
+    cudaFree(c->slab);
+  }
+  for (auto* L : c->layer)
+    if (L) { L->cache = nullptr; L->cache_layer = -1; }
+  delete c;
+  return DX_OK;
+}
+
+extern "C" dx_status dx_layer_attach_cache(dx_layer* L, dx_cache* c, int32_t layer_index) {
+  if (!L || !c || layer_index < 0 || layer_index >= c->L) return DX_ERR_INVALID_ARG;
+  if (L->desc.n_experts != c->E) return DX_ERR_SHAPE;
+  size_t need = 0;
+  if (dx_expert_blob_bytes(&L->desc, L->desc.inter, &need) != DX_OK || need != c->blob_bytes) return DX_ERR_SHAPE;
+  L->cache = c;
+  L->cache_layer = layer_index;
+  c->layer[layer_index] = L;
+  // routed entries now follow the slots: nothing is resident until it is staged
+  const int base = L->desc.n_shared + 1;
+  for (int e = 0; e < c->E; ++e) {
+    const int s = c->slot_of[(size_t)layer_index * c->E + e];
+    L->table_host[base + e] = s >= 0 ? slot_ptr(c, layer_index, s) : nullptr;
+  }
+  L->dirty = true;
+  return DX_OK;
+}
+
+extern "C" dx_status expert_cache_register(dx_cache* c, int32_t layer, int32_t expert, const void* blob) {
+  if (!c || !blob || layer < 0 || layer >= c->L || expert < 0 || expert >= c->E) return DX_ERR_INVALID_ARG;
+  if (((uintptr_t)blob) % 16) return DX_ERR_INVALID_ARG;
+  c->host_blob[(size_t)layer * c->E + expert] = blob;
+  return DX_OK;
+}
+
+extern "C" dx_status expert_cache_begin_step(dx_cache* c) {
+  if (!c) return DX_ERR_INVALID_ARG;
+  for (auto& s : c->slots)
+    if (s.prefetched) { s.prefetched = false; c->stats.prefetch_wasted++; }
+  return DX_OK;
+}
+
+extern "C" dx_status expert_cache_prefetch(dx_cache* c, int32_t layer, const int32_t* ids, int32_t n) {
+  dx_status st = check_ids(c, layer, ids, n);
+  if (st != DX_OK) return st;
+  std::vector<char> pinned(c->S, 0);
+  for (int i = 0; i < n; ++i) {
+    const int e = ids[i];
+    if (c->slot_of[(size_t)layer * c->E + e] >= 0) continue;   // cached or in flight already
+    if (!c->host_blob[(size_t)layer * c->E + e]) return DX_ERR_NOT_RESIDENT;
+    bool was_protected;
+    const int s = find_victim(c, layer, pinned, false, &was_protected);
+    if (s < 0) continue;   // every slot is protected: drop the hint
+    st = load_into(c, layer, s, e, true);
+    if (st != DX_OK) return st;
+    c->stats.prefetch_issued++;
+  }
+  return DX_OK;
+}
+
+static dx_status resolve(dx_cache* c, int layer, const int32_t* ids, int n, cudaStream_t stream, bool may_load,
+                         double timeout_s) {
+  dx_status st = check_ids(c, layer, ids, n);
+  if (st != DX_OK) return st;
+  if (n > c->S) return DX_ERR_CACHE_FULL;
+  std::vector<char> pinned(c->S, 0);
+  // hits first (they pin their slots), then the misses in the order given
+  for (int i = 0; i < n; ++i) {
+    const int s = c->slot_of[(size_t)layer * c->E + ids[i]];
+    if (s < 0) continue;
+    DxSlot& sl = slot_ref(c, layer, s);
+    if (!pinned[s]) {
+      c->stats.lookups++;
+      c->stats.hits++;
+      if (sl.prefetched) { sl.prefetched = false; c->stats.prefetch_used++; }
+      sl.stamp = ++c->clock;
+      pinned[s] = 1;
+    }
+  }
+  for (int i = 0; i < n; ++i) {
+    const int e = ids[i];
+    if (c->slot_of[(size_t)layer * c->E + e] >= 0) continue;
+    if (!may_load) return DX_ERR_NOT_RESIDENT;
+    if (!c->host_blob[(size_t)layer * c->E + e]) return DX_ERR_NOT_RESIDENT;
+    bool was_protected;
+    const int s = find_victim(c, layer, pinned, true, &was_protected);
+    if (s < 0) return DX_ERR_CACHE_FULL;
+    if (was_protected) { c->stats.prefetch_wasted++; slot_ref(c, layer, s).prefetched = false; }
+    c->stats.lookups++;
+    c->stats.on_demand++;
+    st = load_into(c, layer, s, e, false);
+    if (st != DX_OK) return st;
+    pinned[s] = 1;
+  }
+  if (!c->ctx) { c->pending[layer].clear(); return DX_OK; }
+  // the compute stream waits for exactly the copies it needs that are not known to be complete
+  const auto t0 = std::chrono::steady_clock::now();
+  for (int s = 0; s < c->S; ++s) {
+    if (!pinned[s]) continue;
+    DxSlot& sl = slot_ref(c, layer, s);
+    if (copy_done(c, sl)) continue;
+    if (timeout_s > 0.0) {
+      // bounded host wait (expert_cache_wait): poll the copy's event up to the deadline
+      while (!copy_done(c, sl)) {
+        const double dt = std::chrono::duration<double>(std::chrono::steady_clock::now() - t0).count();
+        if (dt > timeout_s) return DX_ERR_TIMEOUT;
+      }
+    } else {
+      cudaError_t e = cudaStreamWaitEvent(stream, sl.ev, 0);
+      if (e != cudaSuccess) { c->ctx->last_cuda = e; return DX_ERR_CUDA; }
+    }
+  }
+  return flush_patches(c, layer, stream);
+}
+
+extern "C" dx_status expert_cache_stage(dx_cache* c, int32_t layer, const int32_t* ids, int32_t n, void* stream) {
+  return resolve(c, layer, ids, n, (cudaStream_t)stream, true, 0.0);
+}
+
+extern "C" dx_status expert_cache_wait(dx_cache* c, int32_t layer, const int32_t* ids, int32_t n, void* stream,
+                                       double timeout_s) {
+  return resolve(c, layer, ids, n, (cudaStream_t)stream, false, timeout_s);
+}
+
+extern "C" dx_status expert_cache_stats(dx_cache* c, dx_cache_stats* out) {
+  if (!c || !out) return DX_ERR_INVALID_ARG;
+  *out = c->stats;
+  return DX_OK;
+}
+
+extern "C" dx_status expert_cache_query(dx_cache* c, int32_t layer, int32_t expert, int32_t* slot_out,
+                                        int32_t* in_flight_out) {
+  if (!c || layer < 0 || layer >= c->L || expert < 0 || expert >= c->E) return DX_ERR_INVALID_ARG;
+  const int s = c->slot_of[(size_t)layer * c->E + expert];
+  if (slot_out) *slot_out = s;
+  if (in_flight_out) *in_flight_out = s >= 0 ? (copy_done(c, slot_ref(c, layer, s)) ? 0 : 1) : 0;
+  return DX_OK;
+}

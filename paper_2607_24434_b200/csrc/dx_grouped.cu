@@ -133,6 +133,29 @@ __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;"
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void cta_bar() { asm volatile("bar.sync 2, 288;" ::: "memory"); }
 
+// This CTA's share of the routed groups.  The launch may be restricted to a window of the routed entries
+// (a "wave" of union experts when the experts are staged through a cache); the units of the window, together
+// with the routing-independent units handled before (NSe of them, [s_lo,s_hi) on this CTA), are split evenly.
+__device__ __forceinline__ void routed_range(const DxWork* W, const DxExpertParams& p, int n_static, int NSe, int s_lo,
+                                             int s_hi, int& e_lo, int& e_hi, int& u_lo, int& u_hi) {
+  const int G = gridDim.x, cta = blockIdx.x;
+  const int n_all = W->n_entries;
+  e_lo = min(n_all, n_static + p.first_routed);
+  e_hi = p.n_routed < 0 ? n_all : min(n_all, e_lo + p.n_routed);
+  if (e_lo >= e_hi) { u_lo = u_hi = 0; return; }
+  const long long R0 = W->entries[e_lo].unit_begin;
+  const long long R1 = (long long)W->entries[e_hi - 1].unit_begin + W->entries[e_hi - 1].n_tiles;
+  const long long NR = R1 - R0, T = NSe + NR;
+  long long a, b;
+  if (T / G >= (NSe + G - 1) / G) {   // keep routing-independent + routed units balanced together
+    a = (T * cta) / G - s_lo; b = (T * (cta + 1)) / G - s_hi;
+  } else {
+    a = (NR * cta) / G; b = (NR * (cta + 1)) / G;
+  }
+  u_lo = (int)(R0 + a);
+  u_hi = (int)(R0 + b);
+}
+
 template <int H, int NT>
 __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertParams p, int n_slots) {
   constexpr int KW = H / 128;        // phase-1 contraction steps per consumer warp
@@ -156,7 +179,7 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
   const int G = gridDim.x, cta = blockIdx.x;
   // groups that do not depend on routing: shared experts, then (draft mode) the draft expert
   const int n_static = p.n_shared + (p.draft_tiles > 0 ? 1 : 0);
-  const int NS = p.n_shared * p.shared_tiles + p.draft_tiles;
+  const int NS = p.do_static ? p.n_shared * p.shared_tiles + p.draft_tiles : 0;
   const int s_lo = (int)(((long long)NS * cta) / G), s_hi = (int)(((long long)NS * (cta + 1)) / G);
   volatile int* abort_flag = &hdr->abort_flag;
 
@@ -203,8 +226,9 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
     if (lane == 0) issue(0, n_static, s_lo, s_hi);
     __syncwarp();
     pdl_wait();
-    const int n_entries = W->n_entries;
-    for (int i = n_static + threadIdx.x; i < n_entries; i += kThreads) {
+    int e_lo, e_hi, u_lo, u_hi;
+    routed_range(W, p, n_static, NS, s_lo, s_hi, e_lo, e_hi, u_lo, u_hi);
+    for (int i = e_lo + threadIdx.x; i < e_hi; i += kThreads) {
       const DxEntry& en = W->entries[i];
       const unsigned char* blob = reinterpret_cast<const unsigned char*>(p.table[en.table_index]);
       hdr->e_begin[i] = en.unit_begin; hdr->e_tiles[i] = en.n_tiles; hdr->e_m[i] = en.m; hdr->e_blob[i] = blob;
@@ -212,14 +236,7 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
     }
     cta_bar();
     if (lane == 0) {
-      const long long T = W->total_units, NR = T - NS;
-      long long r_lo, r_hi;
-      if (T / G >= (NS + G - 1) / G) {   // keep shared + routed balanced together
-        r_lo = (T * cta) / G - s_lo; r_hi = (T * (cta + 1)) / G - s_hi;
-      } else {
-        r_lo = (NR * cta) / G; r_hi = (NR * (cta + 1)) / G;
-      }
-      issue(n_static, n_entries, NS + (int)r_lo, NS + (int)r_hi);
+      issue(e_lo, e_hi, u_lo, u_hi);
       if (*abort_flag) {
         // something gave up: make sure no copy is still landing in this CTA's
         // shared memory before it is released (bounded, ignores the flag)
@@ -436,23 +453,17 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
   process(0, n_static, s_lo, s_hi);
   pdl_wait();
   pdl_launch_dependents();
-  const int n_entries = W->n_entries;
-  for (int i = n_static + threadIdx.x; i < n_entries; i += kThreads) {
-    const DxEntry& en = W->entries[i];
-    const unsigned char* blob = reinterpret_cast<const unsigned char*>(p.table[en.table_index]);
-    hdr->e_begin[i] = en.unit_begin; hdr->e_tiles[i] = en.n_tiles; hdr->e_m[i] = en.m; hdr->e_blob[i] = blob;
-    if (blob == nullptr && en.n_tiles > 0) atomicExch(p.dev_status, DX_DEV_BAD_EXPERT_ID);
-  }
-  cta_bar();
   {
-    const long long T = W->total_units, NR = T - NS;
-    long long r_lo, r_hi;
-    if (T / G >= (NS + G - 1) / G) {
-      r_lo = (T * cta) / G - s_lo; r_hi = (T * (cta + 1)) / G - s_hi;
-    } else {
-      r_lo = (NR * cta) / G; r_hi = (NR * (cta + 1)) / G;
+    int e_lo, e_hi, u_lo, u_hi;
+    routed_range(W, p, n_static, NS, s_lo, s_hi, e_lo, e_hi, u_lo, u_hi);
+    for (int i = e_lo + threadIdx.x; i < e_hi; i += kThreads) {
+      const DxEntry& en = W->entries[i];
+      const unsigned char* blob = reinterpret_cast<const unsigned char*>(p.table[en.table_index]);
+      hdr->e_begin[i] = en.unit_begin; hdr->e_tiles[i] = en.n_tiles; hdr->e_m[i] = en.m; hdr->e_blob[i] = blob;
+      if (blob == nullptr && en.n_tiles > 0) atomicExch(p.dev_status, DX_DEV_BAD_EXPERT_ID);
     }
-    process(n_static, n_entries, NS + (int)r_lo, NS + (int)r_hi);
+    cta_bar();
+    process(e_lo, e_hi, u_lo, u_hi);
   }
   if (*abort_flag && threadIdx.x == 0) atomicExch(p.dev_status, DX_DEV_WAIT_EXPIRED);
 }
@@ -480,8 +491,16 @@ __global__ void __launch_bounds__(256) dx_experts_fp32_kernel(DxExpertParams p) 
     if (lane == 0) s_rstd[r] = rs;
   }
   __syncthreads();
+  // window of the routed entries covered by this launch (see routed_range) and the routing-independent units
+  const int n_static = p.n_shared + (p.draft_tiles > 0 ? 1 : 0);
+  const int NS_all = p.n_shared * p.shared_tiles + p.draft_tiles;
+  const int we_lo = min(n_entries, n_static + p.first_routed);
+  const int we_hi = p.n_routed < 0 ? n_entries : min(n_entries, we_lo + p.n_routed);
+  const int wu_lo = we_lo < we_hi ? W->entries[we_lo].unit_begin : 0;
+  const int wu_hi = we_lo < we_hi ? W->entries[we_hi - 1].unit_begin + W->entries[we_hi - 1].n_tiles : 0;
   int ei = 0;
   for (int u = blockIdx.x; u < total; u += gridDim.x) {
+    if (u < NS_all ? !p.do_static : (u < wu_lo || u >= wu_hi)) continue;
     ei = find_entry(W, n_entries, u, ei);
     const DxEntry& en = W->entries[ei];
     const float* blob = reinterpret_cast<const float*>(p.table[en.table_index]);

@@ -106,6 +106,9 @@ struct DxExpertParams {
   // groups known without routing: shared experts (all K rows, weight 1) and, in draft mode, the draft expert
   int n_shared, shared_tiles, draft_tiles;
   float gamma;
+  // window of the routed entries this launch covers (position among them, count or -1 = all) and whether
+  // the routing-independent groups are part of it; a cache-staged union is processed in several windows
+  int first_routed, n_routed, do_static;
 };
 
 // launchers (each returns the cudaError_t of the launch)
@@ -119,7 +122,6 @@ cudaError_t dx_launch_accept(dx_ctx* ctx, const float* h, int M, const void* W_l
 cudaError_t dx_experts_prepare(dx_ctx* ctx);   // opt-in shared memory attributes, once per context
 
 // cache hooks used by the layer code
-const void** dx_cache_table(dx_cache* c, int layer);
 void dx_cache_note_use(dx_cache* c, int layer, cudaStream_t st);
 
 // Programmatic dependent launch: wait for the preceding kernel of the stream / let the next one start early.
