@@ -301,21 +301,17 @@ def run_gpu(args):
     barrier()
     e2e_ms = g0.elapsed_time(g1)
 
-    if world > 1:
-        import torch.distributed as dist
-        t = torch.tensor([total_ms, e2e_ms], device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms, e2e_ms = float(t[0]), float(t[1])
-        lt = torch.tensor([launches], device=device)
-        dist.all_reduce(lt)
-        launches = int(lt[0])
+    from paper_2607_24434_b200 import multi
+    agg = multi.aggregate({"step": total_ms, "e2e": e2e_ms}, units=K * args.steps, launches=launches, device=device)
+    total_ms, e2e_ms, launches = agg["step"], agg["e2e"], int(agg["launches"])
+    units_all = agg["units"]
 
     if rank != 0:
         if world > 1:
             torch.distributed.destroy_process_group()
         return
     peak, peak_kind = measured_peaks()
-    value = world * K * args.steps / (total_ms * 1e-3)
+    value = multi.throughput(units_all, total_ms)
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -329,7 +325,7 @@ def run_gpu(args):
                    "launch": "CUDA graph replay" if graph is not None else "eager launches",
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
         "gpu_launches": launches,
-        "e2e": {"value": world * K * args.steps / (e2e_ms * 1e-3), "unit": UNIT,
+        "e2e": {"value": multi.throughput(units_all, e2e_ms), "unit": UNIT,
                 "h2d_bytes_per_step": K * H * 4 + K * 4, "d2h_bytes_per_step": K * H * 4 + K * 4 + 8,
                 "ms_per_step": e2e_ms / args.steps},
         "roofline": {"kernel": "dx_experts_bf16_kernel (grouped SwiGLU of the verify block)", "bound": "hbm",

@@ -1,0 +1,72 @@
+"""Layer stacks (attention stubbed out, pre-norm residual MoE sub-layers): DeepSeek-V2-Lite-shaped and
+Moonlight-shaped stacks, teacher-forced per layer -- the checker evaluates layer l on the GPU's own layer-l input
+with the GPU's routing replayed, so one near-tie early on cannot turn the rest into a meaningless comparison --
+followed by greedy verification on the normalised final hidden states."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import moe_oracle as O
+from paper_2607_24434_b200 import synth
+from tests.helpers import GAP, Y_TIGHT, check_routing, check_union, row_rel_err
+
+pytestmark = pytest.mark.gpu
+
+
+def _run_stack(shape, n_layers, K, seed, zipf, vocab):
+    from paper_2607_24434_b200 import binding
+    ctx = binding.Context(0)
+    h = synth.hidden_block(K, shape.hidden, seed, 0.9, "cuda")
+    hd = h[:1].clone()
+    unions, near_total = [], 0
+    for l in range(n_layers):
+        layer = synth.make_layer(shape, seed + 10 * l, "cuda", zipf=zipf)
+        ref = synth.layer_to_numpy(layer)
+        L = binding.Layer.from_weights(ctx, layer)
+        del layer
+        out = binding.moe_verify_block_residual(L, h)
+        outd = binding.moe_draft_step_residual(L, hd)
+        torch.cuda.synchronize()
+        assert ctx.device_status() == 0
+        ids = out["topk_ids"].cpu().numpy()
+        h_np = h.cpu().numpy().astype(np.float64)
+        want, ids_ref, _, z_ref = O.stack_layer_target(h_np, ref)
+        near_total += check_routing(shape, z_ref, ids_ref, ids)
+        want = O.stack_layer_target(h_np, ref, forced_ids=ids)[0]
+        assert row_rel_err(out["h"].cpu().numpy(), want).max() <= Y_TIGHT, l
+        unions.append(check_union(shape, K, ids, out))
+        wantd = O.stack_layer_draft(hd.cpu().numpy().astype(np.float64), ref,
+                                    forced_ids=outd["topk_ids"].cpu().numpy()[None])[0]
+        assert row_rel_err(outd["h"].cpu().numpy(), wantd).max() <= Y_TIGHT, l
+        h, hd = out["h"], outd["h"]           # the stack alternates buffers: each layer's output feeds the next
+        L.close()
+    W = synth.lm_head(vocab, shape.hidden, seed + 999, torch.bfloat16, "cuda")
+    hn = O.rmsnorm(h.cpu().numpy().astype(np.float64))
+    tgt_ref, _, _, lg = O.greedy_accept_fast(hn, synth.to_numpy_f32(W).astype(np.float64), np.zeros(0, np.int32))
+    draft = synth.draft_tokens_from_target(tgt_ref, vocab, seed)
+    acc = binding.spec_accept(ctx, h, W, torch.from_numpy(draft).cuda(), rms_norm=True)
+    torch.cuda.synchronize()
+    tgt = acc["target"].cpu().numpy()
+    srt = np.sort(lg, axis=1)
+    for i in range(K):
+        if srt[i, -1] - srt[i, -2] > GAP:
+            assert tgt[i] == tgt_ref[i]
+    n = 0
+    while n < K and draft[n] == tgt[n]:
+        n += 1
+    assert int(acc["n_accept"].item()) == n
+    ctx.close()
+    return unions, near_total
+
+
+def test_v2lite_stack_correlated_block():
+    sh = synth.shape_v2lite()
+    unions, near = _run_stack(sh, 4, 8, seed=500, zipf=False, vocab=102400)
+    # correlated block rows (rho = 0.9) share experts: unions grow sublinearly, far below the 48 pairs of K = 8
+    assert all(sh.top_k <= u < 8 * sh.top_k for u in unions)
+    assert np.mean(unions) < 30
+
+
+def test_moonlight_stack_sigmoid_scaled():
+    unions, near = _run_stack(synth.shape_moonlight(), 3, 4, seed=600, zipf=True, vocab=163840)
+    assert all(6 <= u <= 24 for u in unions)
