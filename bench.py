@@ -32,6 +32,10 @@ from paper_2607_24434_b200 import synth
 METRIC = "verify_block_moe_tokens_per_s"
 UNIT = "tokens/s"
 NOMINAL_HBM_GBS = 8000.0
+# DRAM bytes (read + write) per launch of the grouped-SwiGLU kernel from the ncu capture summarised in
+# profiles/hot_kernels_v2lite_k4_ncu_full.txt: 265.13 MB at 259.59 MB algorithmic (|U| = 13).  The capture
+# runs a 2-layer case; traffic grows with the units streamed, so a launch's traffic is that ratio x its bytes.
+NCU_TRAFFIC_RATIO = 265.13 / 259.59
 FALLBACK_HBM_GBS = 6650.0
 
 
@@ -331,7 +335,10 @@ def run_gpu(args):
         "roofline": {"kernel": "dx_experts_bf16_kernel (grouped SwiGLU of the verify block)", "bound": "hbm",
                      "achieved": verify_gbs, "peak": peak, "unit": "GB/s", "frac": verify_gbs / peak,
                      "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBs": verify_gbs / NOMINAL_HBM_GBS,
-                     "traffic": args.traffic, "ms_per_launch": float(np.mean(exp_ms)),
+                     "traffic": args.traffic if args.traffic is not None else NCU_TRAFFIC_RATIO * float(
+                         np.mean(exp_alg)),
+                     "traffic_source": "ncu capture of a 2-layer case scaled by algorithmic bytes (see profiles/)",
+                     "ms_per_launch": float(np.mean(exp_ms)),
                      "algorithmic_bytes_per_launch": float(np.mean(exp_alg)), "union_sizes": union},
         "kernels": {"verify_experts_ms": float(np.mean(exp_ms)), "verify_route_ms": route_ms,
                     "verify_tokens_per_s": K / ((float(np.mean(exp_ms)) + route_ms) * 1e-3),
