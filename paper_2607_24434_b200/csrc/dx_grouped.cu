@@ -604,7 +604,10 @@ cudaError_t launch_bf16(dx_ctx* ctx, const DxExpertParams& p, cudaStream_t st) {
   cudaError_t e = cudaFuncSetAttribute(dx_experts_bf16_kernel<H, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)smem);
   if (e != cudaSuccess) return e;
-  return dx_launch_pdl(DX_PDL_EXPERTS, dx_experts_bf16_kernel<H, NT>, dim3(ctx->sm_count), dim3(kThreads), smem, st, 1, p, n_slots);
+  // One CTA per SM, minus the SMs the routing cluster (8 CTAs) runs on at the same time: a CTA of this kernel
+  // fills an SM, so a CTA that had to wait for a routing CTA's SM would start late and become the tail.
+  const int grid = ctx->sm_count > 16 ? ctx->sm_count - 8 : ctx->sm_count;
+  return dx_launch_pdl(DX_PDL_EXPERTS, dx_experts_bf16_kernel<H, NT>, dim3(grid), dim3(kThreads), smem, st, 1, p, n_slots);
 }
 
 template <int H>

@@ -81,12 +81,14 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int* s_warp, int& tot
 // shared memory, row stride H) over a slab of <= 2048 columns; the lane owns
 // columns j0 + lane*8 + 256*i.
 constexpr int kTokGroup = 8;
-__device__ __forceinline__ void row_dots(const __nv_bfloat16* wrow, const float* h, int H, int K, int j0, int chunks,
-                                         int lane, float (&acc)[kTokGroup]) {
-  uint4 w[8];
+__device__ __forceinline__ void row_load(const __nv_bfloat16* wrow, int j0, int chunks, int lane, uint4 (&w)[8]) {
 #pragma unroll
   for (int i = 0; i < 8; ++i)
     if (i < chunks) w[i] = ldg_stream(wrow + j0 + lane * 8 + 256 * i);
+}
+__device__ __forceinline__ void row_load(const float*, int, int, int, uint4 (&)[8]) {}
+__device__ __forceinline__ void row_dots(const __nv_bfloat16* wrow, const float* h, int H, int K, int j0, int chunks,
+                                         int lane, float (&acc)[kTokGroup], const uint4 (&w)[8]) {
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
     if (i < chunks) {
@@ -109,7 +111,7 @@ __device__ __forceinline__ void row_dots(const __nv_bfloat16* wrow, const float*
 }
 
 __device__ __forceinline__ void row_dots(const float* wrow, const float* h, int H, int K, int j0, int chunks, int lane,
-                                         float (&acc)[kTokGroup]) {
+                                         float (&acc)[kTokGroup], const uint4 (&)[8]) {
 #pragma unroll 2
   for (int i = 0; i < chunks; ++i) {
     const float* wp = wrow + j0 + lane * 8 + 256 * i;
@@ -159,20 +161,18 @@ __global__ void __launch_bounds__(kRouteThreads) dx_route_kernel(DxRouteParams p
   dx_pdl_wait();
   dx_pdl_trigger();
 
-  // 1/rms of every block row
-  for (int t = warp; t < DX_MAX_K; t += kRouteWarps) {
-    float rs = 1.0f;
-    if (p.rms_norm && t < K) {
-      float ss = 0.f;
-      for (int j = lane * 4; j < H; j += 128) {
-        const float4 v = *reinterpret_cast<const float4*>(p.h + (size_t)t * H + j);
-        ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
-      }
-      rs = rsqrtf(warp_sum(ss) / (float)H + 1e-6f);
-    }
-    if (lane == 0) s_rstd[t] = rs;
+  // the first router row of this warp is requested before anything else, so its latency overlaps the staging
+  uint4 wreg[8];
+  const int first_chunks = min(8, H / 256);
+  if (e_lo + warp < e_hi)
+    row_load(reinterpret_cast<const WT*>(p.W_r) + (size_t)(e_lo + warp) * H, 0, first_chunks, lane, wreg);
+
+  // y starts at zero, or as a copy of the block in the residual form (stores only complete in the background)
+  for (int j = (crank * kRouteThreads + threadIdx.x) * 4; j < K * H; j += kRouteCluster * kRouteThreads * 4) {
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (p.residual) v = *reinterpret_cast<const float4*>(p.h + j);
+    *reinterpret_cast<float4*>(p.y + j) = v;
   }
-  __syncthreads();
 
   // router logits z[t,e]; block rows go through shared memory in groups of up to `tg` rows
   extern __shared__ __align__(16) float s_h[];
@@ -181,15 +181,45 @@ __global__ void __launch_bounds__(kRouteThreads) dx_route_kernel(DxRouteParams p
   for (int t0 = 0; t0 < K; t0 += tg) {
     const int kt = min(tg, K - t0);
     __syncthreads();
-    for (int j = threadIdx.x * 4; j < kt * H; j += kRouteThreads * 4)
-      *reinterpret_cast<float4*>(s_h + j) = *reinterpret_cast<const float4*>(p.h + (size_t)t0 * H + j);
+    // stage the rows with eight loads in flight per thread
+    for (int base = threadIdx.x * 4; base < kt * H; base += kRouteThreads * 4 * 8) {
+      float4 v[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const int j = base + i * kRouteThreads * 4;
+        if (j < kt * H) v[i] = *reinterpret_cast<const float4*>(p.h + (size_t)t0 * H + j);
+      }
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const int j = base + i * kRouteThreads * 4;
+        if (j < kt * H) *reinterpret_cast<float4*>(s_h + j) = v[i];
+      }
+    }
+    __syncthreads();
+    // 1/rms of the staged rows
+    for (int t = warp; t < kt; t += kRouteWarps) {
+      float rs = 1.0f;
+      if (p.rms_norm) {
+        float ss = 0.f;
+        for (int j = lane * 4; j < H; j += 128) {
+          const float4 v = *reinterpret_cast<const float4*>(s_h + (size_t)t * H + j);
+          ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+        }
+        rs = rsqrtf(warp_sum(ss) / (float)H + 1e-6f);
+      }
+      if (lane == 0) s_rstd[t0 + t] = rs;
+    }
     __syncthreads();
     for (int e = e_lo + warp; e < e_hi; e += kRouteWarps) {
       const WT* wrow = reinterpret_cast<const WT*>(p.W_r) + (size_t)e * H;
       float acc[kTokGroup];
 #pragma unroll
       for (int t = 0; t < kTokGroup; ++t) acc[t] = 0.f;
-      for (int j0 = 0; j0 < H; j0 += 2048) row_dots(wrow, s_h, H, kt, j0, min(8, (H - j0) / 256), lane, acc);
+      for (int j0 = 0; j0 < H; j0 += 2048) {
+        const int chunks = min(8, (H - j0) / 256);
+        if (!(t0 == 0 && e == e_lo + warp && j0 == 0)) row_load(wrow, j0, chunks, lane, wreg);
+        row_dots(wrow, s_h, H, kt, j0, chunks, lane, acc, wreg);
+      }
       const float b = p.bias ? p.bias[e] : 0.f;
 #pragma unroll
       for (int t = 0; t < kTokGroup; ++t) {
@@ -199,12 +229,6 @@ __global__ void __launch_bounds__(kRouteThreads) dx_route_kernel(DxRouteParams p
         }
       }
     }
-  }
-  // y starts at zero, or as a copy of the block in the residual form
-  for (int j = (crank * kRouteThreads + threadIdx.x) * 4; j < K * H; j += kRouteCluster * kRouteThreads * 4) {
-    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (p.residual) v = *reinterpret_cast<const float4*>(p.h + j);
-    *reinterpret_cast<float4*>(p.y + j) = v;
   }
   cluster.sync();          // all logits have landed in CTA 0
   if (crank != 0) return;
@@ -227,11 +251,16 @@ __global__ void __launch_bounds__(kRouteThreads) dx_route_kernel(DxRouteParams p
     int my_e = 0;
     float my_z = 0.f, zmax = 0.f;
     for (int r = 0; r < k; ++r) {
-      unsigned long long best = 0ull;
+      // lane-local best (largest orderable logit, lowest id on ties), then two warp reductions:
+      // the maximum logit, and the lowest expert id among the lanes that hold it
+      unsigned int lbest = 0u, lid = 0xffffffffu;
 #pragma unroll
-      for (int j = 0; j < 8; ++j) best = key[j] > best ? key[j] : best;
-      best = warp_max_u64(best);
-      int be = (int)(0xffffffffu - (unsigned)(best & 0xffffffffull));
+      for (int j = 0; j < 8; ++j) {
+        const unsigned int hi = (unsigned int)(key[j] >> 32);
+        if (key[j] != 0ull && hi > lbest) { lbest = hi; lid = (unsigned int)(lane + 32 * j); }
+      }
+      const unsigned int wbest = __reduce_max_sync(0xffffffffu, lbest);
+      const int be = (int)__reduce_min_sync(0xffffffffu, lbest == wbest ? lid : 0xffffffffu);
       // the owning lane publishes the logit and retires the key
       float bz = 0.f;
 #pragma unroll
@@ -268,8 +297,10 @@ __global__ void __launch_bounds__(kRouteThreads) dx_route_kernel(DxRouteParams p
   // counting sort of the pairs by expert; thread e owns expert e
   const int me = threadIdx.x;
   int cnt = 0;
-  if (me < E)
+  if (me < E) {
+#pragma unroll 8
     for (int q = 0; q < P; ++q) cnt += (s_ids[q] == me);
+  }
   int total;
   const int off = block_exclusive_scan(cnt, s_scan, total);
   const int flag = cnt > 0;
