@@ -58,10 +58,19 @@ __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatil
   }
   *abort_flag = 1;
 }
-__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
-               "l"(src), "r"(bytes), "r"(bar)
-               : "memory");
+// Expert weights are read exactly once per launch: mark them evict-first in L2 so that they do not push out
+// what is reused (block rows, router matrix, work list, output rows).
+__device__ __forceinline__ uint64_t l2_evict_first_policy() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar, uint64_t pol) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(
+          dst),
+      "l"(src), "r"(bytes), "r"(bar), "l"(pol)
+      : "memory");
 }
 __device__ __forceinline__ void consumer_bar() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 
@@ -119,9 +128,8 @@ struct SmemHeader {
   unsigned long long full[kMaxSlots];
   unsigned long long empty[kMaxSlots];
   int abort_flag;
-  int n_entries;
-  int total_units;
-  int pad;
+  int r_e_lo, r_e_hi, r_u_lo;   // this CTA's routed entries and units, published by the producer warp
+  int r_u_hi;
   float rstd[DX_MAX_K];
   int e_begin[DX_MAX_ENTRIES];       // first unit of each entry
   int e_tiles[DX_MAX_ENTRIES];
@@ -204,6 +212,7 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
   if (warp == kConsumerWarps) {
     // ------------------------------------------------------------ producer
     uint32_t it = 0;   // chunk counter
+    const uint64_t l2pol = l2_evict_first_policy();
     auto issue = [&](int e0, int e1, int lo_u, int hi_u) {
       for (int e = e0; e < e1; ++e) {
         const int b = hdr->e_begin[e], nt = hdr->e_tiles[e];
@@ -218,7 +227,7 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
             mbar_wait(smem_u32(&hdr->empty[s]), ph ^ 1u, abort_flag);
             const uint32_t fb = smem_u32(&hdr->full[s]);
             mbar_arrive_expect_tx(fb, CHUNK);
-            bulk_g2s(smem_u32(ring + (size_t)s * CHUNK), src + (size_t)w * CHUNK, CHUNK, fb);
+            bulk_g2s(smem_u32(ring + (size_t)s * CHUNK), src + (size_t)w * CHUNK, CHUNK, fb, l2pol);
           }
         }
       }
@@ -226,15 +235,21 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
     if (lane == 0) issue(0, n_static, s_lo, s_hi);
     __syncwarp();
     pdl_wait();
+    // the producer warp alone copies the routed part of the work list into shared memory, signals the
+    // consumers (bar.arrive: it does not wait for them, they may still be busy with their first reductions)
+    // and goes straight on streaming the routed groups
     int e_lo, e_hi, u_lo, u_hi;
     routed_range(W, p, n_static, NS, s_lo, s_hi, e_lo, e_hi, u_lo, u_hi);
-    for (int i = e_lo + threadIdx.x; i < e_hi; i += kThreads) {
+    for (int i = e_lo + lane; i < e_hi; i += 32) {
       const DxEntry& en = W->entries[i];
       const unsigned char* blob = reinterpret_cast<const unsigned char*>(p.table[en.table_index]);
       hdr->e_begin[i] = en.unit_begin; hdr->e_tiles[i] = en.n_tiles; hdr->e_m[i] = en.m; hdr->e_blob[i] = blob;
       if (blob == nullptr && en.n_tiles > 0) atomicExch(p.dev_status, DX_DEV_BAD_EXPERT_ID);
     }
-    cta_bar();
+    if (lane == 0) { hdr->r_e_lo = e_lo; hdr->r_e_hi = e_hi; hdr->r_u_lo = u_lo; hdr->r_u_hi = u_hi; }
+    __threadfence_block();   // bar.arrive alone does not order the shared-memory writes above
+    __syncwarp();
+    asm volatile("bar.arrive 2, 288;" ::: "memory");
     if (lane == 0) {
       issue(e_lo, e_hi, u_lo, u_hi);
       if (*abort_flag) {
@@ -453,18 +468,8 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
   process(0, n_static, s_lo, s_hi);
   pdl_wait();
   pdl_launch_dependents();
-  {
-    int e_lo, e_hi, u_lo, u_hi;
-    routed_range(W, p, n_static, NS, s_lo, s_hi, e_lo, e_hi, u_lo, u_hi);
-    for (int i = e_lo + threadIdx.x; i < e_hi; i += kThreads) {
-      const DxEntry& en = W->entries[i];
-      const unsigned char* blob = reinterpret_cast<const unsigned char*>(p.table[en.table_index]);
-      hdr->e_begin[i] = en.unit_begin; hdr->e_tiles[i] = en.n_tiles; hdr->e_m[i] = en.m; hdr->e_blob[i] = blob;
-      if (blob == nullptr && en.n_tiles > 0) atomicExch(p.dev_status, DX_DEV_BAD_EXPERT_ID);
-    }
-    cta_bar();
-    process(e_lo, e_hi, u_lo, u_hi);
-  }
+  cta_bar();   // the producer warp has published the routed part of the work list
+  process(hdr->r_e_lo, hdr->r_e_hi, hdr->r_u_lo, hdr->r_u_hi);
   if (*abort_flag && threadIdx.x == 0) atomicExch(p.dev_status, DX_DEV_WAIT_EXPIRED);
 }
 

@@ -87,22 +87,29 @@ __device__ __forceinline__ void row_load(const __nv_bfloat16* wrow, int j0, int 
     if (i < chunks) w[i] = ldg_stream(wrow + j0 + lane * 8 + 256 * i);
 }
 __device__ __forceinline__ void row_load(const float*, int, int, int, uint4 (&)[8]) {}
-__device__ __forceinline__ void row_dots(const __nv_bfloat16* wrow, const float* h, int H, int K, int j0, int chunks,
-                                         int lane, float (&acc)[kTokGroup], const uint4 (&w)[8]) {
+// Staged rows are stored so that a lane's eight columns of a 256-column chunk sit in two conflict-free halves:
+// columns 8l..8l+3 at chunk*256 + 4l, columns 8l+4..8l+7 at chunk*256 + 128 + 4l.
+__device__ __forceinline__ int staged_index(int col) {
+  const int chunk = col >> 8, c4 = (col & 255) >> 2;   // float4 index inside the chunk
+  return (chunk << 8) + ((c4 & 1) << 7) + ((c4 >> 1) << 2) + (col & 3);
+}
+
+template <int KT>
+__device__ __forceinline__ void row_dots_kt(const float* h, int H, int K, int j0, int chunks, int lane,
+                                            float (&acc)[kTokGroup], const float (&wv)[8][8]) {
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
     if (i < chunks) {
-      float wv[8];
-      unpack8(w[i], wv);
-      const float* hp = h + j0 + lane * 8 + 256 * i;
+      const float* hp = h + j0 + 256 * i + lane * 4;
 #pragma unroll
-      for (int t = 0; t < kTokGroup; ++t) {
+      for (int t = 0; t < KT; ++t) {
         if (t < K) {
           const float4 a = *reinterpret_cast<const float4*>(hp + (size_t)t * H);
-          const float4 b = *reinterpret_cast<const float4*>(hp + (size_t)t * H + 4);
+          const float4 b = *reinterpret_cast<const float4*>(hp + (size_t)t * H + 128);
           float s = acc[t];
-          s = fmaf(wv[0], a.x, s); s = fmaf(wv[1], a.y, s); s = fmaf(wv[2], a.z, s); s = fmaf(wv[3], a.w, s);
-          s = fmaf(wv[4], b.x, s); s = fmaf(wv[5], b.y, s); s = fmaf(wv[6], b.z, s); s = fmaf(wv[7], b.w, s);
+          s = fmaf(wv[i][0], a.x, s); s = fmaf(wv[i][1], a.y, s); s = fmaf(wv[i][2], a.z, s);
+          s = fmaf(wv[i][3], a.w, s); s = fmaf(wv[i][4], b.x, s); s = fmaf(wv[i][5], b.y, s);
+          s = fmaf(wv[i][6], b.z, s); s = fmaf(wv[i][7], b.w, s);
           acc[t] = s;
         }
       }
@@ -110,27 +117,106 @@ __device__ __forceinline__ void row_dots(const __nv_bfloat16* wrow, const float*
   }
 }
 
+__device__ __forceinline__ void row_dots_any(const float* h, int H, int K, int j0, int chunks, int lane,
+                                             float (&acc)[kTokGroup], const float (&wv)[8][8]) {
+  if (K <= 1) row_dots_kt<1>(h, H, K, j0, chunks, lane, acc, wv);
+  else if (K <= 2) row_dots_kt<2>(h, H, K, j0, chunks, lane, acc, wv);
+  else if (K <= 4) row_dots_kt<4>(h, H, K, j0, chunks, lane, acc, wv);
+  else row_dots_kt<8>(h, H, K, j0, chunks, lane, acc, wv);
+}
+
+__device__ __forceinline__ void row_dots(const __nv_bfloat16*, const float* h, int H, int K, int j0, int chunks,
+                                         int lane, float (&acc)[kTokGroup], const uint4 (&w)[8]) {
+  float wv[8][8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i)
+    if (i < chunks) unpack8(w[i], wv[i]);
+  row_dots_any(h, H, K, j0, chunks, lane, acc, wv);
+}
+
 __device__ __forceinline__ void row_dots(const float* wrow, const float* h, int H, int K, int j0, int chunks, int lane,
                                          float (&acc)[kTokGroup], const uint4 (&)[8]) {
-#pragma unroll 2
-  for (int i = 0; i < chunks; ++i) {
-    const float* wp = wrow + j0 + lane * 8 + 256 * i;
-    const uint4 u0 = ldg_stream(wp), u1 = ldg_stream(wp + 4);
-    const float4 w0 = make_float4(__uint_as_float(u0.x), __uint_as_float(u0.y), __uint_as_float(u0.z), __uint_as_float(u0.w));
-    const float4 w1 = make_float4(__uint_as_float(u1.x), __uint_as_float(u1.y), __uint_as_float(u1.z), __uint_as_float(u1.w));
-    const float* hp = h + j0 + lane * 8 + 256 * i;
+  // fp32 router rows (small layers): two passes of four chunks keep the register footprint down
+  for (int half = 0; half < 2; ++half) {
+    float wv[8][8];
+    const int c0 = half * 4, nc = min(4, chunks - c0);
+    if (nc <= 0) break;
 #pragma unroll
-    for (int t = 0; t < kTokGroup; ++t) {
-      if (t < K) {
-        const float4 a = *reinterpret_cast<const float4*>(hp + (size_t)t * H);
-        const float4 b = *reinterpret_cast<const float4*>(hp + (size_t)t * H + 4);
-        float s = acc[t];
-        s = fmaf(w0.x, a.x, s); s = fmaf(w0.y, a.y, s); s = fmaf(w0.z, a.z, s); s = fmaf(w0.w, a.w, s);
-        s = fmaf(w1.x, b.x, s); s = fmaf(w1.y, b.y, s); s = fmaf(w1.z, b.z, s); s = fmaf(w1.w, b.w, s);
-        acc[t] = s;
+    for (int i = 0; i < 4; ++i) {
+      if (i < nc) {
+        const float* wp = wrow + j0 + lane * 8 + 256 * (c0 + i);
+        const uint4 u0 = ldg_stream(wp), u1 = ldg_stream(wp + 4);
+        wv[i][0] = __uint_as_float(u0.x); wv[i][1] = __uint_as_float(u0.y); wv[i][2] = __uint_as_float(u0.z);
+        wv[i][3] = __uint_as_float(u0.w); wv[i][4] = __uint_as_float(u1.x); wv[i][5] = __uint_as_float(u1.y);
+        wv[i][6] = __uint_as_float(u1.z); wv[i][7] = __uint_as_float(u1.w);
       }
     }
+    row_dots_any(h, H, K, j0 + 256 * c0, nc, lane, acc, wv);
   }
+}
+
+// Top-k of one token by one warp: k rounds of (lane-local best, warp max of the logit, warp min of the id among
+// the holders of that maximum); then softmax / sigmoid scores of the selected experts and their gate weights.
+template <int NK>
+__device__ __forceinline__ void topk_token(const DxRouteParams& p, const float* s_z, int* s_ids, float* s_w, int tt,
+                                           int lane) {
+  const int E = p.E, k = p.k;
+    unsigned long long key[NK];
+    float zv[NK];
+#pragma unroll
+    for (int j = 0; j < NK; ++j) {
+      int ee = lane + 32 * j;
+      if (ee < E) {
+        zv[j] = s_z[tt * E + ee];
+        key[j] = ((unsigned long long)dx_orderable(zv[j]) << 32) | (unsigned long long)(0xffffffffu - (unsigned)ee);
+      } else {
+        zv[j] = 0.f;
+        key[j] = 0ull;
+      }
+    }
+    int my_e = 0;
+    float my_z = 0.f, zmax = 0.f;
+    for (int r = 0; r < k; ++r) {
+      // lane-local best (largest orderable logit, lowest id on ties), then two warp reductions:
+      // the maximum logit, and the lowest expert id among the lanes that hold it
+      unsigned int lbest = 0u, lid = 0xffffffffu;
+#pragma unroll
+      for (int j = 0; j < NK; ++j) {
+        const unsigned int hi = (unsigned int)(key[j] >> 32);
+        if (key[j] != 0ull && hi > lbest) { lbest = hi; lid = (unsigned int)(lane + 32 * j); }
+      }
+      const unsigned int wbest = __reduce_max_sync(0xffffffffu, lbest);
+      const int be = (int)__reduce_min_sync(0xffffffffu, lbest == wbest ? lid : 0xffffffffu);
+      // the owning lane publishes the logit and retires the key
+      float bz = 0.f;
+#pragma unroll
+      for (int j = 0; j < NK; ++j)
+        if (lane + 32 * j == be) { bz = zv[j]; key[j] = 0ull; }
+      bz = __shfl_sync(0xffffffffu, bz, be & 31);
+      if (r == 0) zmax = bz;
+      if (lane == r) { my_e = be; my_z = bz; }
+    }
+    float psel;
+    if (p.score_fn == DX_SCORE_SOFTMAX) {
+      float s = 0.f;
+#pragma unroll
+      for (int j = 0; j < NK; ++j)
+        if (lane + 32 * j < E) s += expf(zv[j] - zmax);
+      s = warp_sum(s);
+      psel = expf(my_z - zmax) / s;
+    } else {
+      psel = 1.0f / (1.0f + expf(-my_z));
+    }
+    if (lane >= k) psel = 0.f;
+    float denom = warp_sum(psel);
+    float g = p.norm_topk ? psel / denom : psel;
+    g *= p.scale;
+    if (lane < k) {
+      s_ids[tt * k + lane] = my_e;
+      s_w[tt * k + lane] = g;
+      if (p.topk_ids) p.topk_ids[tt * k + lane] = my_e;
+      if (p.topk_w) p.topk_w[tt * k + lane] = g;
+    }
 }
 
 template <typename WT>
@@ -192,7 +278,7 @@ __global__ void __launch_bounds__(kRouteThreads) dx_route_kernel(DxRouteParams p
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
         const int j = base + i * kRouteThreads * 4;
-        if (j < kt * H) *reinterpret_cast<float4*>(s_h + j) = v[i];
+        if (j < kt * H) *reinterpret_cast<float4*>(s_h + (j / H) * H + staged_index(j % H)) = v[i];
       }
     }
     __syncthreads();
@@ -233,64 +319,12 @@ __global__ void __launch_bounds__(kRouteThreads) dx_route_kernel(DxRouteParams p
   cluster.sync();          // all logits have landed in CTA 0
   if (crank != 0) return;
 
-  // top-k and gate weights, one warp per token
+  // top-k and gate weights, one warp per token (NK = keys per lane, a power of two covering E)
   for (int tt = warp; tt < K; tt += kRouteWarps) {
-    unsigned long long key[8];
-    float zv[8];
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      int ee = lane + 32 * j;
-      if (ee < E) {
-        zv[j] = s_z[tt * E + ee];
-        key[j] = ((unsigned long long)dx_orderable(zv[j]) << 32) | (unsigned long long)(0xffffffffu - (unsigned)ee);
-      } else {
-        zv[j] = 0.f;
-        key[j] = 0ull;
-      }
-    }
-    int my_e = 0;
-    float my_z = 0.f, zmax = 0.f;
-    for (int r = 0; r < k; ++r) {
-      // lane-local best (largest orderable logit, lowest id on ties), then two warp reductions:
-      // the maximum logit, and the lowest expert id among the lanes that hold it
-      unsigned int lbest = 0u, lid = 0xffffffffu;
-#pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        const unsigned int hi = (unsigned int)(key[j] >> 32);
-        if (key[j] != 0ull && hi > lbest) { lbest = hi; lid = (unsigned int)(lane + 32 * j); }
-      }
-      const unsigned int wbest = __reduce_max_sync(0xffffffffu, lbest);
-      const int be = (int)__reduce_min_sync(0xffffffffu, lbest == wbest ? lid : 0xffffffffu);
-      // the owning lane publishes the logit and retires the key
-      float bz = 0.f;
-#pragma unroll
-      for (int j = 0; j < 8; ++j)
-        if (lane + 32 * j == be) { bz = zv[j]; key[j] = 0ull; }
-      bz = __shfl_sync(0xffffffffu, bz, be & 31);
-      if (r == 0) zmax = bz;
-      if (lane == r) { my_e = be; my_z = bz; }
-    }
-    float psel;
-    if (p.score_fn == DX_SCORE_SOFTMAX) {
-      float s = 0.f;
-#pragma unroll
-      for (int j = 0; j < 8; ++j)
-        if (lane + 32 * j < E) s += expf(zv[j] - zmax);
-      s = warp_sum(s);
-      psel = expf(my_z - zmax) / s;
-    } else {
-      psel = 1.0f / (1.0f + expf(-my_z));
-    }
-    if (lane >= k) psel = 0.f;
-    float denom = warp_sum(psel);
-    float g = p.norm_topk ? psel / denom : psel;
-    g *= p.scale;
-    if (lane < k) {
-      s_ids[tt * k + lane] = my_e;
-      s_w[tt * k + lane] = g;
-      if (p.topk_ids) p.topk_ids[tt * k + lane] = my_e;
-      if (p.topk_w) p.topk_w[tt * k + lane] = g;
-    }
+    if (E <= 32) topk_token<1>(p, s_z, s_ids, s_w, tt, lane);
+    else if (E <= 64) topk_token<2>(p, s_z, s_ids, s_w, tt, lane);
+    else if (E <= 128) topk_token<4>(p, s_z, s_ids, s_w, tt, lane);
+    else topk_token<8>(p, s_z, s_ids, s_w, tt, lane);
   }
   __syncthreads();
 
@@ -301,13 +335,13 @@ __global__ void __launch_bounds__(kRouteThreads) dx_route_kernel(DxRouteParams p
 #pragma unroll 8
     for (int q = 0; q < P; ++q) cnt += (s_ids[q] == me);
   }
-  int total;
-  const int off = block_exclusive_scan(cnt, s_scan, total);
+  // one scan carries both prefix sums: pair counts in the low half, union membership in the high half
   const int flag = cnt > 0;
   const unsigned int bal = __ballot_sync(0xffffffffu, flag);
   if (lane == 0) s_ballot[warp] = bal;
-  int ucount;
-  const int upos = block_exclusive_scan(flag, s_scan, ucount);   // its barriers also publish s_ballot
+  int total;
+  const int both = block_exclusive_scan(cnt | (flag << 16), s_scan, total);   // its barriers also publish s_ballot
+  const int off = both & 0xffff, upos = both >> 16, ucount = total >> 16;
   if (me < E) {
     if (p.offsets) p.offsets[me] = off;
     int i = 0;
