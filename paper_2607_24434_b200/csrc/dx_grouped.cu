@@ -303,9 +303,12 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
   const int src0 = (2 * c) * 4 + (g >> 1), src1 = src0 + 4;
   const bool odd = g & 1;
 
-  auto entry_tok = [&](int e, int slot) -> int { return e < n_static ? slot : W->entries[e].tok[slot]; };
-  auto entry_w = [&](int e, int slot) -> float {
-    return e < n_static ? (e < p.n_shared ? 1.0f : p.gamma) : W->entries[e].w[slot];
+  // weight of group e's output in block row `row` (0 = the row does not belong to the group).  Token slots of
+  // the MMAs are the block rows themselves, for every group alike, so the accumulators can stay in registers
+  // across groups (the weight is folded into the activations) and y is touched once, at the very end.
+  auto row_weight = [&](int e, int row) -> float {
+    if (e < n_static) return row < p.K ? (e < p.n_shared ? 1.0f : p.gamma) : 0.0f;
+    return W->entries[e].roww[row];
   };
 
   auto process = [&](int e0, int e1, int lo_u, int hi_u) {
@@ -313,12 +316,16 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
       const int eb = hdr->e_begin[e], etiles = hdr->e_tiles[e];
       const int lo = max(eb, lo_u), hi = min(eb + etiles, hi_u);
       if (lo >= hi || hdr->e_blob[e] == nullptr) continue;
-      const int m = hdr->e_m[e];
+      // this lane's block rows (one per token tile) and their weights in this group
+      float wrow[NT];
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) wrow[nt] = row_weight(e, nt * 8 + g);
+      const bool need_hi = NT > 1 && __any_sync(0xffffffffu, wrow[NT - 1] != 0.0f);   // any of rows 8..15 routed here
 
       // ---- token fragments of this group
       if constexpr (kRegB) {
-        const bool valid = g < m;
-        const int tk = valid ? entry_tok(e, g) : 0;
+        const bool valid = wrow[0] != 0.0f;
+        const int tk = g;
         const float rs = hdr->rstd[tk];
         const float* xrow = p.x + (size_t)tk * H + 4 * c;
 #pragma unroll
@@ -337,8 +344,8 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
           const int l = idx & 31, ks = (idx >> 5) % KSTEPS, nt = idx / (32 * KSTEPS);
           const int slot = nt * 8 + (l >> 2);
           uint4 o = make_uint4(0u, 0u, 0u, 0u);
-          if (slot < m) {
-            const int tk = entry_tok(e, slot);
+          if (row_weight(e, slot) != 0.0f) {
+            const int tk = slot;
             const float rs = hdr->rstd[tk];
             const float4 v = *reinterpret_cast<const float4*>(p.x + (size_t)tk * H + 16 * ks + 4 * (l & 3));
             __nv_bfloat16 h0, h1, h2, h3, l0, l1, l2, l3;
@@ -372,7 +379,7 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
           } else {
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) {
-              if (nt > 0 && m <= 8 * nt) continue;
+              if (nt > 0 && !need_hi) continue;
               const uint4 b = bfrag[(nt * KSTEPS + warp * KW + i) * 32 + lane];
               mma_k16(ch[nt][i & 1], a, b.x, b.y);
               mma_k16(cl[nt][i & 1], a, b.z, b.w);
@@ -408,7 +415,7 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
               q[w].x += q[w + st].x; q[w].y += q[w + st].y; q[w].z += q[w + st].z; q[w].w += q[w + st].w;
             }
           const float4 t = q[0];
-          const float a0 = fast_silu(t.x) * t.y, a1 = fast_silu(t.z) * t.w;
+          const float a0 = fast_silu(t.x) * t.y * wrow[nt], a1 = fast_silu(t.z) * t.w * wrow[nt];
           __nv_bfloat16 h0, l0, h1, l1;
           split_bf16(a0, h0, l0);
           split_bf16(a1, h1, l1);
@@ -424,7 +431,7 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
           const uint4 a = D[q * 32];
 #pragma unroll
           for (int nt = 0; nt < NT; ++nt) {
-            if (nt > 0 && m <= 8 * nt) continue;
+            if (nt > 0 && !need_hi) continue;
             mma_k8(acc[nt][2 * q], a.x, a.y, bhi[nt]);
             mma_k8(acc[nt][2 * q + 1], a.z, a.w, bhi[nt]);
             mma_k8(acc[nt][2 * q], a.x, a.y, blo[nt]);
@@ -435,33 +442,6 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
         if (lane == 0) mbar_arrive(smem_u32(&hdr->empty[s]));
       }
 
-      // ---- add this group's partial output rows to y (scaled by each token's weight), reset.
-      // y is initialised by the routing kernel, so its completion is awaited first.
-      pdl_wait();
-#pragma unroll
-      for (int nt = 0; nt < NT; ++nt) {
-        const int s0 = nt * 8 + 2 * c, s1 = s0 + 1;
-        const bool v0 = s0 < m, v1 = s1 < m;
-        if (v0) {
-          const float w0 = entry_w(e, s0), w1 = v1 ? entry_w(e, s1) : 0.f;
-          float* y0 = p.y + (size_t)entry_tok(e, s0) * H;
-          float* y1 = p.y + (size_t)(v1 ? entry_tok(e, s1) : 0) * H;
-#pragma unroll
-          for (int j = 0; j < 2 * PW; ++j) {
-            const int hh = (warp * 2 * PW + j) * 16 + g;
-            atomicAdd(y0 + hh, w0 * acc[nt][j][0]);
-            atomicAdd(y0 + hh + 8, w0 * acc[nt][j][2]);
-            if (v1) {
-              atomicAdd(y1 + hh, w1 * acc[nt][j][1]);
-              atomicAdd(y1 + hh + 8, w1 * acc[nt][j][3]);
-            }
-          }
-        }
-#pragma unroll
-        for (int j = 0; j < 2 * PW; ++j)
-#pragma unroll
-          for (int r = 0; r < 4; ++r) acc[nt][j][r] = 0.f;
-      }
     }
   };
 
@@ -470,6 +450,27 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
   pdl_launch_dependents();
   cta_bar();   // the producer warp has published the routed part of the work list
   process(hdr->r_e_lo, hdr->r_e_hi, hdr->r_u_lo, hdr->r_u_hi);
+
+  // ---- the CTA's partial output rows go to y (initialised by the routing kernel, which has completed)
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt) {
+    const int r0 = nt * 8 + 2 * c, r1 = r0 + 1;
+    if (r0 < p.K) {
+      float* y0 = p.y + (size_t)r0 * H;
+      float* y1 = p.y + (size_t)r1 * H;
+      const bool v1 = r1 < p.K;
+#pragma unroll
+      for (int j = 0; j < 2 * PW; ++j) {
+        const int hh = (warp * 2 * PW + j) * 16 + g;
+        atomicAdd(y0 + hh, acc[nt][j][0]);
+        atomicAdd(y0 + hh + 8, acc[nt][j][2]);
+        if (v1) {
+          atomicAdd(y1 + hh, acc[nt][j][1]);
+          atomicAdd(y1 + hh + 8, acc[nt][j][3]);
+        }
+      }
+    }
+  }
   if (*abort_flag && threadIdx.x == 0) atomicExch(p.dev_status, DX_DEV_WAIT_EXPIRED);
 }
 

@@ -28,6 +28,7 @@ struct DxEntry {
   int32_t m;             // tokens in the group (<= K)
   int32_t tok[DX_MAX_K]; // block row of each group token
   float w[DX_MAX_K];     // weight of this expert's output in that row (g, 1 or gamma)
+  float roww[DX_MAX_K];  // the same weights indexed by block row (0 = the row is not in this group)
 };
 
 struct DxWork {

@@ -369,6 +369,7 @@ __global__ void __launch_bounds__(kRouteThreads) dx_route_kernel(DxRouteParams p
     en.n_tiles = p.shared_tiles;
     en.unit_begin = me * p.shared_tiles;
     en.m = K;
+    for (int i = 0; i < DX_MAX_K; ++i) en.roww[i] = i < K ? 1.0f : 0.0f;
     for (int i = 0; i < K; ++i) { en.tok[i] = i; en.w[i] = 1.0f; }
   }
   int n_entries, total_units;
@@ -380,10 +381,12 @@ __global__ void __launch_bounds__(kRouteThreads) dx_route_kernel(DxRouteParams p
       en.n_tiles = p.routed_tiles;
       en.unit_begin = routed_base + upos * p.routed_tiles;
       en.m = cnt;
+      for (int i = 0; i < DX_MAX_K; ++i) en.roww[i] = 0.0f;
       for (int i = 0; i < cnt; ++i) {
         int q = s_perm[off + i];
         en.tok[i] = q / k;
         en.w[i] = s_w[q];
+        en.roww[q / k] = s_w[q];
       }
     }
     n_entries = p.n_shared + ucount;
@@ -399,6 +402,7 @@ __global__ void __launch_bounds__(kRouteThreads) dx_route_kernel(DxRouteParams p
         en.m = 1;
         en.tok[0] = 0;
         en.w[0] = p.gamma;
+        for (int i = 0; i < DX_MAX_K; ++i) en.roww[i] = i == 0 ? p.gamma : 0.0f;
       }
       base += 1;
     }
@@ -410,6 +414,7 @@ __global__ void __launch_bounds__(kRouteThreads) dx_route_kernel(DxRouteParams p
       en.m = 1;
       en.tok[0] = 0;
       en.w[0] = s_w[me];
+      for (int i = 0; i < DX_MAX_K; ++i) en.roww[i] = i == 0 ? s_w[me] : 0.0f;
     }
     n_entries = base + p.top_r;
     total_units = routed_base + p.draft_tiles + p.top_r * p.routed_tiles;
