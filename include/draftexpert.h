@@ -137,6 +137,12 @@ dx_status dx_layer_attach_cache(dx_layer* layer, dx_cache* cache, int32_t layer_
 dx_status moe_draft_step(dx_layer* layer, const float* h, float* y, int32_t* topk_ids, float* topk_w,
                          void* stream);
 
+/* The training-free shared + top-r self-drafter of Sec. 2.2 / Sec. 4 (r = 1, 2, 3 in the paper), and mixtures:
+ * y = S(h) + sum_{j<top_r} g_{e_j} E_{e_j}(h) (+ gamma E^d(h) iff use_draft_expert != 0), gate weights as in Eq. 4.
+ * top_r = 1 with the draft expert is moe_draft_step; 1 <= top_r <= k. */
+dx_status moe_draft_step_topr(dx_layer* layer, const float* h, float* y, int32_t top_r, int32_t use_draft_expert,
+                              int32_t* topk_ids, float* topk_w, void* stream);
+
 /* ---- verifier: Eq. 4 over a block, grouped by the union of Eq. 2 / Eq. 3 -----------------------------------
  * h [K,H] in, y [K,H] out (overwritten; must not overlap h).  Routing outputs (device pointers, each may be NULL if unwanted):
  *   topk_ids [K,k] int32, topk_w [K,k] fp32;

@@ -63,6 +63,7 @@ SIGNATURES = {
     "dx_layer_set_expert": (_I, [_P, _I, _P]),
     "dx_layer_attach_cache": (_I, [_P, _P, _I]),
     "moe_draft_step": (_I, [_P, _P, _P, _P, _P, _P]),
+    "moe_draft_step_topr": (_I, [_P, _P, _P, _I, _I, _P, _P, _P]),
     "moe_draft_step_residual": (_I, [_P, _P, _P, _P, _P, _P]),
     "moe_verify_block": (_I, [_P, _P, _I, _P, _P, _P, _P, _P, _P, _P, _P, _P]),
     "moe_verify_route": (_I, [_P, _P, _I, _P, _P, _P, _P, _P, _P, _P, _P, _P]),
@@ -452,4 +453,19 @@ def moe_verify_block_cached(layer: Layer, cache: ExpertCache, layer_index: int, 
             break
     out["y"] = y
     out["union_list"] = ids
+    return out
+
+
+def moe_draft_step_topr(layer: Layer, h: torch.Tensor, top_r: int, use_draft_expert: bool,
+                        y: Optional[torch.Tensor] = None) -> Dict[str, torch.Tensor]:
+    """Shared + top-r drafter (Sec. 2.2), optionally with the draft expert."""
+    sh = layer.shape
+    out = {"topk_ids": torch.empty((sh.top_k,), dtype=torch.int32, device=h.device),
+           "topk_w": torch.empty((sh.top_k,), dtype=torch.float32, device=h.device)}
+    if y is None:
+        y = torch.empty_like(h)
+    _check(layer.lib.moe_draft_step_topr(layer.handle, _ptr(h), _ptr(y), top_r, 1 if use_draft_expert else 0,
+                                         _ptr(out["topk_ids"]), _ptr(out["topk_w"]), _stream()),
+           "moe_draft_step_topr")
+    out["y"] = y
     return out

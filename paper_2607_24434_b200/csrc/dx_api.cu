@@ -213,7 +213,7 @@ struct RouteOut {
 };
 
 static dx_status do_route(dx_layer* L, const float* h, int K, float* y, const RouteOut& o, bool draft, bool residual,
-                          cudaStream_t st) {
+                          cudaStream_t st, int top_r = 1, bool use_draft_expert = true) {
   dx_ctx* ctx = L->ctx;
   const dx_layer_desc& d = L->desc;
   if (!h || !y || h == y) return DX_ERR_INVALID_ARG;
@@ -221,7 +221,8 @@ static dx_status do_route(dx_layer* L, const float* h, int K, float* y, const Ro
   if (!L->W_r) return DX_ERR_NOT_RESIDENT;
   for (int s = 0; s < d.n_shared; ++s)
     if (!L->table_host[s]) return DX_ERR_NOT_RESIDENT;
-  if (draft && d.draft_inter > 0 && !L->table_host[d.n_shared]) return DX_ERR_NOT_RESIDENT;
+  if (draft && use_draft_expert && d.draft_inter > 0 && !L->table_host[d.n_shared]) return DX_ERR_NOT_RESIDENT;
+  if (top_r < 1 || top_r > d.top_k) return DX_ERR_INVALID_ARG;
   if (((uintptr_t)h) % 16 || ((uintptr_t)y) % 16) return DX_ERR_INVALID_ARG;
   dx_status s = upload_table(L, st);
   if (s != DX_OK) return s;
@@ -232,9 +233,9 @@ static dx_status do_route(dx_layer* L, const float* h, int K, float* y, const Ro
   p.n_shared = d.n_shared;
   p.shared_tiles = d.n_shared ? d.shared_inter / DX_TILE_I : 0;
   p.routed_tiles = d.inter / DX_TILE_I;
-  p.draft_tiles = draft ? d.draft_inter / DX_TILE_I : 0;
+  p.draft_tiles = draft && use_draft_expert ? d.draft_inter / DX_TILE_I : 0;
   p.draft_mode = draft ? 1 : 0;
-  p.top_r = 1;
+  p.top_r = top_r;
   p.rms_norm = residual ? 1 : 0;
   p.residual = residual ? 1 : 0;
   p.y = y; p.z = ctx->z; p.ticket = ctx->ticket; p.work = ctx->work; p.dev_status = ctx->dev_status;
@@ -314,6 +315,16 @@ extern "C" dx_status moe_verify_experts_range(dx_layer* L, const float* h, int32
   if (!L) return DX_ERR_INVALID_ARG;
   if (first_union < 0 || n_union < 0) return DX_ERR_INVALID_ARG;
   return do_experts(L, h, K, y, false, false, (cudaStream_t)stream, first_union, n_union, include_shared != 0);
+}
+
+extern "C" dx_status moe_draft_step_topr(dx_layer* L, const float* h, float* y, int32_t top_r,
+                                         int32_t use_draft_expert, int32_t* topk_ids, float* topk_w, void* stream) {
+  if (!L) return DX_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  RouteOut o{topk_ids, topk_w, nullptr, nullptr, nullptr, nullptr, nullptr};
+  dx_status s = do_route(L, h, 1, y, o, true, false, st, top_r, use_draft_expert != 0);
+  if (s != DX_OK) return s;
+  return do_experts(L, h, 1, y, use_draft_expert != 0, false, st);
 }
 
 extern "C" dx_status moe_draft_route(dx_layer* L, const float* h, float* y, int32_t* topk_ids, float* topk_w,

@@ -154,6 +154,27 @@ def test_detached_expert_is_reported_not_trapped(dx):
     L.close()
 
 
+def test_shared_plus_top_r_drafter(dx):
+    """The training-free shared + top-r drafter of Sec. 2.2 (r = 1..3) and r = k, which is the target layer."""
+    binding, ctx = dx
+    for shape, std in ((SMALL, 0.08), (synth.shape_tiny(), 0.1)):
+        layer, ref = gpu_layer(shape, 33, std=std)
+        L = binding.Layer.from_weights(ctx, layer)
+        h = synth.hidden_block(1, shape.hidden, 34, 0.0, "cuda")
+        h_np = h.cpu().numpy().astype(np.float64)
+        for r, use_d in [(1, False), (2, False), (shape.top_k, False), (2, True)]:
+            out = binding.moe_draft_step_topr(L, h, r, use_d)
+            torch.cuda.synchronize()
+            ids = out["topk_ids"].cpu().numpy()[None]
+            want = O.moe_draft(h_np, ref, forced_ids=ids, top_r=r, gamma=None if use_d else 0.0)[0]
+            assert row_rel_err(out["y"].cpu().numpy(), want).max() <= Y_TIGHT, (r, use_d)
+            if r == shape.top_k and not use_d:
+                target = O.moe_target(h_np, ref, forced_ids=ids)[0]
+                assert row_rel_err(out["y"].cpu().numpy(), target).max() <= Y_TIGHT
+        assert ctx.device_status() == 0
+        L.close()
+
+
 # ------------------------------------------------------------------ residual (stack) forms
 def test_residual_forms(dx):
     binding, ctx = dx
