@@ -192,6 +192,32 @@ dx_status spec_accept(dx_ctx* ctx, const float* h, int32_t M, const void* W_lm, 
                       int32_t w_dtype, const int32_t* draft, int32_t K, int32_t rms_norm,
                       int32_t* target, int32_t* n_accept, int32_t* next_token, void* stream);
 
+/* ---- drafting one token: Algorithm 1 "Draft v_i" (its LM-head step) and "Compute confidence q_i" -------------------
+ * For each of the M rows of h: token[i] = argmax_v <W_lm[v], h_i> and confidence[i] = the softmax probability of
+ * that token, q = 1 / sum_v exp(l_v - l_max) (the paper asks only for "a confidence score from the draft logits";
+ * the maximum softmax probability is the reading taken).  Same kernels and limits as spec_accept, with an online
+ * (max, sum-of-exp) pair carried next to the running argmax.  token [M] int32 and confidence [M] fp32 are device
+ * pointers. */
+dx_status spec_draft_token(dx_ctx* ctx, const float* h, int32_t M, const void* W_lm, int32_t V, int32_t H,
+                           int32_t w_dtype, int32_t rms_norm, int32_t* token, float* confidence, void* stream);
+
+/* ---- confidence-expansion truncation: Sec. 3.4, Eq. 12-14, Algorithm 1 loop body ------------------------------------
+ * Host-only.  The controller keeps the predicted block-level verifier set U_hat (Eq. 12) as one bitmask per layer.
+ *   reset:   U_hat <- empty (start of a decode step, Algorithm 1 line 1).
+ *   propose: candidate token i with confidence q and draft-router predictions predicted[l*k + j] (host ints: the
+ *            topk_ids moe_draft_step returned in layer l).  Computes Delta_i = |U_hat_i| - |U_hat| (Eq. 13, counted
+ *            in (layer, expert) pairs).  If q < tau and Delta_i > budget (Eq. 14) the candidate is dropped:
+ *            *stop_out = 1, U_hat unchanged.  Otherwise *stop_out = 0, U_hat <- U_hat_i, and the new pairs -- the
+ *            ones to prefetch -- are listed in new_layers_out / new_experts_out (each sized L*k, may be NULL). */
+typedef struct dx_controller dx_controller;
+dx_status dx_controller_create(int32_t n_layers, int32_t n_experts, dx_controller** out);
+dx_status dx_controller_destroy(dx_controller* c);
+dx_status dx_controller_reset(dx_controller* c);
+dx_status dx_controller_size(dx_controller* c, int32_t* size_out);
+dx_status dx_controller_propose(dx_controller* c, const int32_t* predicted, int32_t k, float q, float tau,
+                                int32_t budget, int32_t* delta_out, int32_t* stop_out, int32_t* new_layers_out,
+                                int32_t* new_experts_out, int32_t* n_new_out);
+
 /* ---- greedy verification without any allocation ----------------------------------------------------------------
  * (No counterpart in the paper: an addition for callers of this library that cannot allocate device memory --
  * a serving thread whose memory pool was sized once at start-up and where a late cudaMalloc is forbidden or

@@ -267,3 +267,37 @@ def stack_layer_draft(h: np.ndarray, layer, dtype=np.float64, norm: bool = True,
     x = rmsnorm(h) if norm else h
     y, ids, g, z = moe_draft(x, layer, dtype, forced_ids)
     return h + y, ids, g, z
+
+
+# --------------------------------------------------------------------------
+# Sec. 3.4: confidence of a draft token and confidence-expansion truncation.
+# --------------------------------------------------------------------------
+def draft_confidence(h: np.ndarray, W_lm: np.ndarray, dtype=np.float64):
+    """Draft token = argmax of the draft logits; q = its softmax probability (the reading taken for
+    "a confidence score from the draft logits")."""
+    lg = lm_logits(h, W_lm, dtype)
+    e = np.exp(lg - lg.max(axis=1, keepdims=True))
+    prob = e / e.sum(axis=1, keepdims=True)
+    tok = lg.argmax(axis=1).astype(np.int32)
+    return tok, prob[np.arange(lg.shape[0]), tok], lg
+
+
+class TruncationController:
+    """U_hat_i = union_{j<=i} union_l E_hat_{l,j} (Eq. 12) as a set of (layer, expert) pairs;
+    Delta_i = |U_hat_i| - |U_hat_{i-1}| (Eq. 13); stop before appending token i when q_i < tau and
+    Delta_i > B_i (Eq. 14); a stopped candidate leaves U_hat as it was (Algorithm 1)."""
+
+    def __init__(self):
+        self.u_hat = set()
+
+    def reset(self):
+        self.u_hat = set()
+
+    def propose(self, predicted, q, tau, budget):
+        cand = self.u_hat | {(l, int(e)) for l, row in enumerate(predicted) for e in row}
+        delta = len(cand) - len(self.u_hat)
+        stop = (q < tau) and (delta > budget)
+        new = sorted(cand - self.u_hat)
+        if not stop:
+            self.u_hat = cand
+        return stop, delta, ([] if stop else new)

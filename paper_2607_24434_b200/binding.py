@@ -73,6 +73,13 @@ SIGNATURES = {
     "moe_draft_experts": (_I, [_P, _P, _P, _P]),
     "moe_verify_block_residual": (_I, [_P, _P, _P, _I, _P, _P, _P, _P, _P, _P, _P, _P]),
     "spec_accept": (_I, [_P, _P, _I, _P, _I, _I, _I, _P, _I, _I, _P, _P, _P, _P]),
+    "spec_draft_token": (_I, [_P, _P, _I, _P, _I, _I, _I, _I, _P, _P, _P]),
+    "dx_controller_create": (_I, [_I, _I, C.POINTER(_P)]),
+    "dx_controller_destroy": (_I, [_P]),
+    "dx_controller_reset": (_I, [_P]),
+    "dx_controller_size": (_I, [_P, C.POINTER(_I)]),
+    "dx_controller_propose": (_I, [_P, _P, _I, C.c_float, C.c_float, _I, C.POINTER(_I), C.POINTER(_I), _P, _P,
+                                   C.POINTER(_I)]),
     "spec_accept_noalloc": (_I, [_P, _I, _P, _I, _I, _I, _P, _I, _I, _P, _P, _P, _P]),
     "expert_cache_create": (_I, [_P, _I, _I, _I, C.c_size_t, C.POINTER(_P)]),
     "expert_cache_destroy": (_I, [_P]),
@@ -469,3 +476,56 @@ def moe_draft_step_topr(layer: Layer, h: torch.Tensor, top_r: int, use_draft_exp
            "moe_draft_step_topr")
     out["y"] = y
     return out
+
+
+def spec_draft_token(ctx: Context, h: torch.Tensor, W_lm: torch.Tensor, rms_norm: bool = False):
+    """Draft-side LM head: token [M] = argmax and confidence [M] = its softmax probability (Algorithm 1, q_i)."""
+    M, H = h.shape
+    token = torch.empty((M,), dtype=torch.int32, device=h.device)
+    conf = torch.empty((M,), dtype=torch.float32, device=h.device)
+    wd = 1 if W_lm.dtype == torch.bfloat16 else 0
+    _check(ctx.lib.spec_draft_token(ctx.handle, _ptr(h), M, _ptr(W_lm), W_lm.shape[0], H, wd, 1 if rms_norm else 0,
+                                    _ptr(token), _ptr(conf), _stream()), "spec_draft_token")
+    return token, conf
+
+
+class Controller:
+    """Confidence-expansion truncation (Sec. 3.4): host-side predicted verifier set and stop rule."""
+
+    def __init__(self, n_layers: int, n_experts: int):
+        self.lib = load()
+        self.n_layers = n_layers
+        h = _P()
+        _check(self.lib.dx_controller_create(n_layers, n_experts, C.byref(h)), "dx_controller_create")
+        self.handle = h
+
+    def close(self) -> None:
+        if self.handle:
+            self.lib.dx_controller_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def reset(self) -> None:
+        _check(self.lib.dx_controller_reset(self.handle), "dx_controller_reset")
+
+    def size(self) -> int:
+        n = _I(0)
+        _check(self.lib.dx_controller_size(self.handle, C.byref(n)), "dx_controller_size")
+        return n.value
+
+    def propose(self, predicted: Sequence[Sequence[int]], q: float, tau: float, budget: int):
+        """predicted[l] = the draft router's top-k ids in layer l.  Returns (stop, delta, new (layer, expert) pairs)."""
+        k = len(predicted[0])
+        flat = [int(e) for row in predicted for e in row]
+        arr = (C.c_int32 * len(flat))(*flat)
+        nl = (C.c_int32 * len(flat))()
+        ne = (C.c_int32 * len(flat))()
+        delta, stop, n_new = _I(0), _I(0), _I(0)
+        _check(self.lib.dx_controller_propose(self.handle, arr, k, q, tau, budget, C.byref(delta), C.byref(stop), nl,
+                                              ne, C.byref(n_new)), "dx_controller_propose")
+        return bool(stop.value), delta.value, [(nl[i], ne[i]) for i in range(n_new.value)]

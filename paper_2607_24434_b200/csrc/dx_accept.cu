@@ -56,9 +56,25 @@ struct AcceptParams {
   int32_t* next_token;
   unsigned long long* keys;
   unsigned int* ticket;
+  float* conf;          // [M] softmax probability of the argmax (only the CONF variants)
+  float2* conf_part;    // [grid][DX_MAX_M] per-CTA (running max, sum of exp) pairs
 };
 
+// online softmax bookkeeping: (m, s) with s = sum exp(l - m) over the logits seen so far
+__device__ __forceinline__ void conf_push(float& m, float& s, float l) {
+  if (l > m) { s = s * __expf(m - l) + 1.0f; m = l; }
+  else s += __expf(l - m);
+}
+__device__ __forceinline__ void conf_merge(float& m, float& s, float m2, float s2) {
+  if (s2 == 0.0f) return;
+  if (s == 0.0f) { m = m2; s = s2; return; }
+  const float mm = fmaxf(m, m2);
+  s = s * __expf(m - mm) + s2 * __expf(m2 - mm);
+  m = mm;
+}
+
 // Shared tail: merge CTA maxima into the global keys; the last CTA decodes.
+template <bool CONF>
 __device__ __forceinline__ void finish(const AcceptParams& p, unsigned long long* s_keys) {
   __shared__ int s_last;
   __syncthreads();
@@ -76,6 +92,15 @@ __device__ __forceinline__ void finish(const AcceptParams& p, unsigned long long
     s_tok[threadIdx.x] = tok;
     p.target[threadIdx.x] = tok;
     p.keys[threadIdx.x] = 0ull;
+    if constexpr (CONF) {
+      // max softmax probability = 1 / sum_v exp(l_v - l_max): merge every CTA's (max, sum) pair in CTA order
+      float m = -INFINITY, sum = 0.0f;
+      for (unsigned int cta = 0; cta < gridDim.x; ++cta) {
+        const float2 part = __ldcg(p.conf_part + (size_t)cta * DX_MAX_M + threadIdx.x);
+        conf_merge(m, sum, part.x, part.y);
+      }
+      p.conf[threadIdx.x] = 1.0f / sum;
+    }
   }
   __syncthreads();
   if (threadIdx.x == 0) {
@@ -87,7 +112,7 @@ __device__ __forceinline__ void finish(const AcceptParams& p, unsigned long long
   }
 }
 
-template <int NT>
+template <int NT, bool CONF>
 __global__ void __launch_bounds__(512, 1) dx_accept_bf16_kernel(AcceptParams p) {
   extern __shared__ __align__(16) unsigned char smem[];
   __shared__ float s_rstd[DX_MAX_M];
@@ -141,6 +166,9 @@ __global__ void __launch_bounds__(512, 1) dx_accept_bf16_kernel(AcceptParams p) 
   int best_i[NT][2];
 #pragma unroll
   for (int nt = 0; nt < NT; ++nt) { best_v[nt][0] = best_v[nt][1] = -INFINITY; best_i[nt][0] = best_i[nt][1] = -1; }
+  float cm[NT][2], cs[NT][2];   // online softmax state of the two rows this lane owns per tile (CONF only)
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt) { cm[nt][0] = cm[nt][1] = -INFINITY; cs[nt][0] = cs[nt][1] = 0.0f; }
 
   const int tiles = (p.V + 15) / 16;
   const int warps_total = gridDim.x * (blockDim.x >> 5);
@@ -175,11 +203,35 @@ __global__ void __launch_bounds__(512, 1) dx_accept_bf16_kernel(AcceptParams p) 
       if (r0 < p.V) {
         if (l00 > best_v[nt][0]) { best_v[nt][0] = l00; best_i[nt][0] = r0; }
         if (l01 > best_v[nt][1]) { best_v[nt][1] = l01; best_i[nt][1] = r0; }
+        if constexpr (CONF) { conf_push(cm[nt][0], cs[nt][0], l00); conf_push(cm[nt][1], cs[nt][1], l01); }
       }
       if (r1 < p.V) {
         if (l10 > best_v[nt][0]) { best_v[nt][0] = l10; best_i[nt][0] = r1; }
         if (l11 > best_v[nt][1]) { best_v[nt][1] = l11; best_i[nt][1] = r1; }
+        if constexpr (CONF) { conf_push(cm[nt][0], cs[nt][0], l10); conf_push(cm[nt][1], cs[nt][1], l11); }
       }
+    }
+  }
+  if constexpr (CONF) {
+    __shared__ float2 s_conf[16][DX_MAX_M];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+        float m = cm[nt][j], sum = cs[nt][j];
+#pragma unroll
+        for (int o = 4; o < 32; o <<= 1) {
+          const float m2 = __shfl_xor_sync(0xffffffffu, m, o), s2 = __shfl_xor_sync(0xffffffffu, sum, o);
+          conf_merge(m, sum, m2, s2);
+        }
+        const int row = nt * 8 + 2 * c + j;
+        if (g == 0 && row < DX_MAX_M) s_conf[warp][row] = make_float2(m, sum);
+      }
+    __syncthreads();
+    if (threadIdx.x < p.M) {
+      float m = -INFINITY, sum = 0.0f;
+      for (int w = 0; w < 16; ++w) conf_merge(m, sum, s_conf[w][threadIdx.x].x, s_conf[w][threadIdx.x].y);
+      p.conf_part[(size_t)blockIdx.x * DX_MAX_M + threadIdx.x] = make_float2(m, sum);
     }
   }
   // lanes with equal c hold the same token columns: merge over g
@@ -196,10 +248,11 @@ __global__ void __launch_bounds__(512, 1) dx_accept_bf16_kernel(AcceptParams p) 
       const int row = nt * 8 + 2 * c + j;
       if (g == 0 && row < p.M && key != 0ull) atomicMax(&s_keys[row], key);
     }
-  finish(p, s_keys);
+  finish<CONF>(p, s_keys);
 }
 
 // fp32 LM head (small vocabularies): one warp per vocabulary row.
+template <bool CONF>
 __global__ void __launch_bounds__(256) dx_accept_fp32_kernel(AcceptParams p) {
   __shared__ float s_rstd[DX_MAX_M];
   __shared__ unsigned long long s_keys[DX_MAX_M];
@@ -219,8 +272,13 @@ __global__ void __launch_bounds__(256) dx_accept_fp32_kernel(AcceptParams p) {
   const float* Wf = reinterpret_cast<const float*>(p.W);
   const int warps_total = gridDim.x * 8;
   unsigned long long best[DX_MAX_M];
+  float cm[CONF ? DX_MAX_M : 1], cs[CONF ? DX_MAX_M : 1];
 #pragma unroll
   for (int i = 0; i < DX_MAX_M; ++i) best[i] = 0ull;
+  if constexpr (CONF) {
+#pragma unroll
+    for (int i = 0; i < DX_MAX_M; ++i) { cm[i] = -INFINITY; cs[i] = 0.0f; }
+  }
   for (int v = blockIdx.x * 8 + warp; v < p.V; v += warps_total) {
     const float* wr = Wf + (size_t)v * H;
 #pragma unroll
@@ -231,6 +289,7 @@ __global__ void __launch_bounds__(256) dx_accept_fp32_kernel(AcceptParams p) {
         acc = warp_sum(acc);
         unsigned long long key = make_key(acc, v);
         best[i] = key > best[i] ? key : best[i];
+        if constexpr (CONF) conf_push(cm[i], cs[i], acc);
       }
     }
   }
@@ -239,32 +298,47 @@ __global__ void __launch_bounds__(256) dx_accept_fp32_kernel(AcceptParams p) {
     for (int i = 0; i < DX_MAX_M; ++i)
       if (i < p.M && best[i] != 0ull) atomicMax(&s_keys[i], best[i]);
   }
-  finish(p, s_keys);
+  if constexpr (CONF) {
+    __shared__ float2 s_conf[8][DX_MAX_M];
+    if (lane == 0) {
+#pragma unroll
+      for (int i = 0; i < DX_MAX_M; ++i) s_conf[warp][i] = make_float2(cm[i], cs[i]);
+    }
+    __syncthreads();
+    if (threadIdx.x < p.M) {
+      float m = -INFINITY, sum = 0.0f;
+      for (int w = 0; w < 8; ++w) conf_merge(m, sum, s_conf[w][threadIdx.x].x, s_conf[w][threadIdx.x].y);
+      p.conf_part[(size_t)blockIdx.x * DX_MAX_M + threadIdx.x] = make_float2(m, sum);
+    }
+  }
+  finish<CONF>(p, s_keys);
 }
 
 }  // namespace
 
+template <int NT, bool CONF>
+static cudaError_t launch_accept_bf16(dx_ctx* ctx, const AcceptParams& p, size_t smem, cudaStream_t st) {
+  cudaError_t e = cudaFuncSetAttribute(dx_accept_bf16_kernel<NT, CONF>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)smem);
+  if (e != cudaSuccess) return e;
+  return dx_launch_pdl(DX_PDL_ACCEPT, dx_accept_bf16_kernel<NT, CONF>, dim3(ctx->sm_count), dim3(512), smem, st, 1, p);
+}
+
 cudaError_t dx_launch_accept(dx_ctx* ctx, const float* h, int M, const void* W_lm, int V, int H, int w_dtype,
                              const int32_t* draft, int K, int rms_norm, int32_t* target, int32_t* n_accept,
-                             int32_t* next_token, cudaStream_t st) {
-  AcceptParams p{h, M, V, H, W_lm, draft, K, rms_norm, target, n_accept, next_token, ctx->keys, ctx->ticket + 1};
+                             int32_t* next_token, float* conf, cudaStream_t st) {
+  AcceptParams p{h, M, V, H, W_lm, draft, K, rms_norm, target, n_accept, next_token, ctx->keys, ctx->ticket + 1,
+                 conf, ctx->conf_part};
   if (w_dtype == DX_DTYPE_FP32) {
     int grid = (V + 7) / 8;
     if (grid > ctx->sm_count * 8) grid = ctx->sm_count * 8;
-    return dx_launch_pdl(DX_PDL_ACCEPT, dx_accept_fp32_kernel, dim3(grid), dim3(256), 0, st, 1, p);
+    if (conf) return dx_launch_pdl(DX_PDL_ACCEPT, dx_accept_fp32_kernel<true>, dim3(grid), dim3(256), 0, st, 1, p);
+    return dx_launch_pdl(DX_PDL_ACCEPT, dx_accept_fp32_kernel<false>, dim3(grid), dim3(256), 0, st, 1, p);
   }
   const int NT = (M + 7) / 8;
   const size_t smem = (size_t)NT * (H / 32) * 32 * 16 * 2;
-  cudaError_t e;
-  if (NT == 1) {
-    e = cudaFuncSetAttribute(dx_accept_bf16_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    return dx_launch_pdl(DX_PDL_ACCEPT, dx_accept_bf16_kernel<1>, dim3(ctx->sm_count), dim3(512), smem, st, 1, p);
-  } else {
-    e = cudaFuncSetAttribute(dx_accept_bf16_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    return dx_launch_pdl(DX_PDL_ACCEPT, dx_accept_bf16_kernel<2>, dim3(ctx->sm_count), dim3(512), smem, st, 1, p);
-  }
+  if (NT == 1) return conf ? launch_accept_bf16<1, true>(ctx, p, smem, st) : launch_accept_bf16<1, false>(ctx, p, smem, st);
+  return conf ? launch_accept_bf16<2, true>(ctx, p, smem, st) : launch_accept_bf16<2, false>(ctx, p, smem, st);
 }
 
 // ---------------------------------------------------------------------------------------------------------
@@ -322,23 +396,23 @@ extern "C" dx_status spec_accept_noalloc(const float* h, int32_t M, const void* 
   if (cudaMemsetAsync(d.scratch, 0, sizeof(unsigned long long) * (kNoAllocMaxRows + 2), st) != cudaSuccess)
     return DX_ERR_CUDA;
   AcceptParams p{h, M, V, H, W_lm, draft, K, rms_norm, target, n_accept, next_token, d.scratch,
-                 reinterpret_cast<unsigned int*>(d.scratch + kNoAllocMaxRows)};
+                 reinterpret_cast<unsigned int*>(d.scratch + kNoAllocMaxRows), nullptr, nullptr};
   cudaError_t e;
   if (w_dtype == DX_DTYPE_FP32) {
     int grid = (V + 7) / 8;
     if (grid > d.sm_count * 8) grid = d.sm_count * 8;
-    dx_accept_fp32_kernel<<<grid, 256, 0, st>>>(p);
+    dx_accept_fp32_kernel<false><<<grid, 256, 0, st>>>(p);
     e = cudaGetLastError();
   } else if (NT == 1) {
-    e = cudaFuncSetAttribute(dx_accept_bf16_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    e = cudaFuncSetAttribute(dx_accept_bf16_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e == cudaSuccess) {
-      dx_accept_bf16_kernel<1><<<d.sm_count, 512, smem, st>>>(p);
+      dx_accept_bf16_kernel<1, false><<<d.sm_count, 512, smem, st>>>(p);
       e = cudaGetLastError();
     }
   } else {
-    e = cudaFuncSetAttribute(dx_accept_bf16_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    e = cudaFuncSetAttribute(dx_accept_bf16_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e == cudaSuccess) {
-      dx_accept_bf16_kernel<2><<<d.sm_count, 512, smem, st>>>(p);
+      dx_accept_bf16_kernel<2, false><<<d.sm_count, 512, smem, st>>>(p);
       e = cudaGetLastError();
     }
   }

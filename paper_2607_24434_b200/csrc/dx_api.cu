@@ -59,6 +59,8 @@ extern "C" dx_status dx_create(int device, dx_ctx** out) {
   if (e == cudaSuccess) e = cudaMalloc(&ctx->ticket, sizeof(unsigned int) * 4);
   if (e == cudaSuccess) e = cudaMalloc(&ctx->keys, sizeof(unsigned long long) * DX_MAX_M);
   if (e == cudaSuccess) e = cudaMalloc(&ctx->dev_status, sizeof(int32_t));
+  if (e == cudaSuccess) e = cudaMalloc(&ctx->conf_part, sizeof(float2) * 8 * ctx->sm_count * DX_MAX_M);
+  if (e == cudaSuccess) e = cudaMalloc(&ctx->scratch_i32, sizeof(int32_t) * 2);
   if (e == cudaSuccess) e = cudaMemset(ctx->work, 0, sizeof(DxWork));
   if (e == cudaSuccess) e = cudaMemset(ctx->ticket, 0, sizeof(unsigned int) * 4);
   if (e == cudaSuccess) e = cudaMemset(ctx->keys, 0, sizeof(unsigned long long) * DX_MAX_M);
@@ -79,6 +81,8 @@ extern "C" dx_status dx_destroy(dx_ctx* ctx) {
   cudaFree(ctx->ticket);
   cudaFree(ctx->keys);
   cudaFree(ctx->dev_status);
+  cudaFree(ctx->conf_part);
+  cudaFree(ctx->scratch_i32);
   delete ctx;
   return DX_OK;
 }
@@ -374,7 +378,22 @@ extern "C" dx_status spec_accept(dx_ctx* ctx, const float* h, int32_t M, const v
     if (smem > (size_t)ctx->smem_optin) return DX_ERR_UNSUPPORTED;
   }
   DX_CUDA(ctx, dx_launch_accept(ctx, h, M, W_lm, V, H, w_dtype, draft, K, rms_norm, target, n_accept, next_token,
-                                (cudaStream_t)stream));
+                                nullptr, (cudaStream_t)stream));
+  ctx->launches++;
+  return DX_OK;
+}
+
+extern "C" dx_status spec_draft_token(dx_ctx* ctx, const float* h, int32_t M, const void* W_lm, int32_t V, int32_t H,
+                                      int32_t w_dtype, int32_t rms_norm, int32_t* token, float* confidence,
+                                      void* stream) {
+  if (!ctx || !h || !W_lm || !token || !confidence) return DX_ERR_INVALID_ARG;
+  if (M < 1 || V < 1) return DX_ERR_SHAPE;
+  if (w_dtype != DX_DTYPE_FP32 && w_dtype != DX_DTYPE_BF16) return DX_ERR_INVALID_ARG;
+  if (M > DX_MAX_M || H <= 0 || H > DX_MAX_H || H % 256) return DX_ERR_UNSUPPORTED;
+  if (((uintptr_t)h) % 16 || ((uintptr_t)W_lm) % 16) return DX_ERR_INVALID_ARG;
+  if (w_dtype == DX_DTYPE_BF16 && (size_t)((M + 7) / 8) * H * 32 > (size_t)ctx->smem_optin) return DX_ERR_UNSUPPORTED;
+  DX_CUDA(ctx, dx_launch_accept(ctx, h, M, W_lm, V, H, w_dtype, nullptr, 0, rms_norm, token, ctx->scratch_i32,
+                                ctx->scratch_i32 + 1, confidence, (cudaStream_t)stream));
   ctx->launches++;
   return DX_OK;
 }

@@ -51,6 +51,8 @@ struct dx_ctx {
   unsigned int* ticket;        // last-CTA tickets (route, accept)
   unsigned long long* keys;    // [DX_MAX_M] packed argmax keys
   int32_t* dev_status;
+  float2* conf_part;           // [8 * sm_count][DX_MAX_M] per-CTA online-softmax pairs of the confidence variant
+  int32_t* scratch_i32;        // two ints the draft-token entry point parks unused outputs in
 };
 
 struct dx_cache;
@@ -119,7 +121,7 @@ cudaError_t dx_launch_pack(int weight_dtype, int H, int I, const void* Wg, const
                            void* blob, cudaStream_t st);
 cudaError_t dx_launch_accept(dx_ctx* ctx, const float* h, int M, const void* W_lm, int V, int H, int w_dtype,
                              const int32_t* draft, int K, int rms_norm, int32_t* target, int32_t* n_accept,
-                             int32_t* next_token, cudaStream_t st);
+                             int32_t* next_token, float* conf, cudaStream_t st);
 cudaError_t dx_experts_prepare(dx_ctx* ctx);   // opt-in shared memory attributes, once per context
 
 // cache hooks used by the layer code

@@ -280,3 +280,28 @@ def test_accept_ties_take_lowest_index(dx):
 def test_accept_full_vocab_bf16(dx):
     _accept_case(dx, 5, 4, 102400, 2048, torch.bfloat16, 400, mode="geometric", rms=True)
     _accept_case(dx, 9, 8, 163840, 2048, torch.bfloat16, 401, mode="geometric", rms=True)
+
+
+# ------------------------------------------------------------------ draft token + confidence (Sec. 3.4, q_i)
+@pytest.mark.parametrize("M,V,H,dtype", [(1, 1000, 512, torch.bfloat16), (4, 4099, 256, torch.bfloat16),
+                                         (9, 3001, 1024, torch.bfloat16), (3, 1024, 256, torch.float32),
+                                         (1, 102400, 2048, torch.bfloat16)])
+def test_draft_token_confidence(dx, M, V, H, dtype):
+    binding, ctx = dx
+    W = synth.lm_head(V, H, 700 + M, dtype, "cuda", std=0.05)
+    h = synth.hidden_block(M, H, 701 + M, 0.3, "cuda") * 2.0
+    tok, conf = binding.spec_draft_token(ctx, h, W, rms_norm=True)
+    torch.cuda.synchronize()
+    hn = O.rmsnorm(h.cpu().numpy().astype(np.float64))
+    tok_ref, q_ref, lg = O.draft_confidence(hn, synth.to_numpy_f32(W).astype(np.float64))
+    srt = np.sort(lg, axis=1)
+    for i in range(M):
+        if srt[i, -1] - srt[i, -2] > GAP:
+            assert int(tok[i]) == int(tok_ref[i])
+    # q = 1 / sum exp(l - l_max): fp32 logits and hardware exp, compared with the fp64 checker
+    assert np.abs(conf.cpu().numpy() - q_ref).max() <= 1e-4 * max(1.0, q_ref.max()) + 2e-3 * q_ref.max()
+    assert np.all(conf.cpu().numpy() > 0) and np.all(conf.cpu().numpy() <= 1.0 + 1e-6)
+    # the plain accept kernel is unchanged by the confidence variant
+    acc = binding.spec_accept(ctx, h, W, tok, rms_norm=True)
+    torch.cuda.synchronize()
+    assert torch.equal(acc["target"], tok) and int(acc["n_accept"].item()) == M
