@@ -214,6 +214,22 @@ class Layer:
         self._keep[f"expert{e}"] = blob
         _check(self.lib.dx_layer_set_expert(self.handle, e, _ptr(blob)), "dx_layer_set_expert")
 
+    def share(self, ctx: "Context") -> "Layer":
+        """A second handle on the same weights under another context (its own scratch and work list), so that the
+        layer can be used from another stream, or several routed layers can be in flight at once."""
+        other = Layer(ctx, self.shape)
+        W_r, bias = self._keep["router"]
+        other.set_router(W_r, bias)
+        for name, blob in self._keep.items():
+            if name.startswith("shared"):
+                other.set_shared(int(name[6:]), blob)
+            elif name == "draft":
+                other.set_draft(blob)
+            elif name.startswith("expert") and blob is not None:
+                other.set_expert(int(name[6:]), blob)
+        other.blobs = getattr(self, "blobs", None)
+        return other
+
     @classmethod
     def from_weights(cls, ctx: Context, layer: Dict[str, object], routed_resident: bool = True) -> "Layer":
         """Packs a canonical-layout layer (see ``synth.make_layer``) that already sits on the GPU and
