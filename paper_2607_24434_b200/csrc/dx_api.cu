@@ -59,6 +59,8 @@ extern "C" dx_status dx_create(int device, dx_ctx** out) {
   if (e == cudaSuccess) e = cudaMalloc(&ctx->ticket, sizeof(unsigned int) * 4);
   if (e == cudaSuccess) e = cudaMalloc(&ctx->keys, sizeof(unsigned long long) * DX_MAX_M);
   if (e == cudaSuccess) e = cudaMalloc(&ctx->dev_status, sizeof(int32_t));
+  if (e == cudaSuccess) e = cudaMalloc(&ctx->handover, 4 * sizeof(unsigned int));
+  if (e == cudaSuccess) e = cudaMemset(ctx->handover, 0, 4 * sizeof(unsigned int));
   if (e == cudaSuccess) e = cudaMalloc(&ctx->conf_part, sizeof(float2) * 8 * ctx->sm_count * DX_MAX_M);
   if (e == cudaSuccess) e = cudaMalloc(&ctx->scratch_i32, sizeof(int32_t) * 2);
   if (e == cudaSuccess) e = cudaMemset(ctx->work, 0, sizeof(DxWork));
@@ -81,6 +83,7 @@ extern "C" dx_status dx_destroy(dx_ctx* ctx) {
   cudaFree(ctx->ticket);
   cudaFree(ctx->keys);
   cudaFree(ctx->dev_status);
+  cudaFree(ctx->handover);
   cudaFree(ctx->conf_part);
   cudaFree(ctx->scratch_i32);
   delete ctx;
@@ -217,7 +220,7 @@ struct RouteOut {
 };
 
 static dx_status do_route(dx_layer* L, const float* h, int K, float* y, const RouteOut& o, bool draft, bool residual,
-                          cudaStream_t st, int top_r = 1, bool use_draft_expert = true) {
+                          cudaStream_t st, int top_r = 1, bool use_draft_expert = true, bool paired = false) {
   dx_ctx* ctx = L->ctx;
   const dx_layer_desc& d = L->desc;
   if (!h || !y || h == y) return DX_ERR_INVALID_ARG;
@@ -243,6 +246,7 @@ static dx_status do_route(dx_layer* L, const float* h, int K, float* y, const Ro
   p.rms_norm = residual ? 1 : 0;
   p.residual = residual ? 1 : 0;
   p.y = y; p.z = ctx->z; p.ticket = ctx->ticket; p.work = ctx->work; p.dev_status = ctx->dev_status;
+  p.handover = paired ? ctx->handover : nullptr;
   p.topk_ids = o.topk_ids; p.topk_w = o.topk_w;
   p.union_mask = (unsigned long long*)o.union_mask; p.union_ids = o.union_ids; p.union_count = o.union_count;
   p.offsets = o.offsets; p.perm = o.perm;
@@ -252,7 +256,8 @@ static dx_status do_route(dx_layer* L, const float* h, int K, float* y, const Ro
 }
 
 static dx_status do_experts(dx_layer* L, const float* h, int K, float* y, bool draft, bool residual,
-                            cudaStream_t st, int first_routed = 0, int n_routed = -1, bool do_static = true) {
+                            cudaStream_t st, int first_routed = 0, int n_routed = -1, bool do_static = true,
+                            bool paired = false) {
   dx_ctx* ctx = L->ctx;
   const dx_layer_desc& d = L->desc;
   if (!h || !y || h == y) return DX_ERR_INVALID_ARG;
@@ -272,6 +277,7 @@ static dx_status do_experts(dx_layer* L, const float* h, int K, float* y, bool d
   p.shared_tiles = d.n_shared ? d.shared_inter / DX_TILE_I : 0;
   p.draft_tiles = draft ? d.draft_inter / DX_TILE_I : 0;
   p.gamma = d.draft_gamma;
+  p.handover = paired ? ctx->handover : nullptr;
   p.first_routed = first_routed;
   p.n_routed = n_routed;
   p.do_static = do_static ? 1 : 0;
@@ -281,14 +287,25 @@ static dx_status do_experts(dx_layer* L, const float* h, int K, float* y, bool d
   return DX_OK;
 }
 
+// Routing kernel and expert kernel of one layer call, launched back to back.  Only here the two kernels use the
+// device-side hand-over (bf16 blobs): the routing kernel sets the words, the expert kernel that is certain to
+// follow consumes and clears them.
+static dx_status do_pair(dx_layer* L, const float* h, int K, float* y, const RouteOut& o, bool draft, bool residual,
+                         cudaStream_t st, int top_r = 1, bool use_draft_expert = true) {
+  const bool paired = L->desc.weight_dtype == DX_DTYPE_BF16;
+  dx_status s = do_route(L, h, K, y, o, draft, residual, st, top_r, use_draft_expert, paired);
+  if (s != DX_OK) return s;
+  s = do_experts(L, h, K, y, draft && use_draft_expert, residual, st, 0, -1, true, paired);
+  if (s != DX_OK && paired) cudaMemsetAsync(L->ctx->handover, 0, 4 * sizeof(unsigned int), st);
+  return s;
+}
+
 extern "C" dx_status moe_draft_step(dx_layer* L, const float* h, float* y, int32_t* topk_ids, float* topk_w,
                                     void* stream) {
   if (!L) return DX_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;
   RouteOut o{topk_ids, topk_w, nullptr, nullptr, nullptr, nullptr, nullptr};
-  dx_status s = do_route(L, h, 1, y, o, true, false, st);
-  if (s != DX_OK) return s;
-  return do_experts(L, h, 1, y, true, false, st);
+  return do_pair(L, h, 1, y, o, true, false, st);
 }
 
 extern "C" dx_status moe_draft_step_residual(dx_layer* L, const float* h_in, float* h_out, int32_t* topk_ids,
@@ -296,9 +313,7 @@ extern "C" dx_status moe_draft_step_residual(dx_layer* L, const float* h_in, flo
   if (!L) return DX_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;
   RouteOut o{topk_ids, topk_w, nullptr, nullptr, nullptr, nullptr, nullptr};
-  dx_status s = do_route(L, h_in, 1, h_out, o, true, true, st);
-  if (s != DX_OK) return s;
-  return do_experts(L, h_in, 1, h_out, true, true, st);
+  return do_pair(L, h_in, 1, h_out, o, true, true, st);
 }
 
 extern "C" dx_status moe_verify_route(dx_layer* L, const float* h, int32_t K, float* y, int32_t* topk_ids,
@@ -326,9 +341,7 @@ extern "C" dx_status moe_draft_step_topr(dx_layer* L, const float* h, float* y, 
   if (!L) return DX_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;
   RouteOut o{topk_ids, topk_w, nullptr, nullptr, nullptr, nullptr, nullptr};
-  dx_status s = do_route(L, h, 1, y, o, true, false, st, top_r, use_draft_expert != 0);
-  if (s != DX_OK) return s;
-  return do_experts(L, h, 1, y, use_draft_expert != 0, false, st);
+  return do_pair(L, h, 1, y, o, true, false, st, top_r, use_draft_expert != 0);
 }
 
 extern "C" dx_status moe_draft_route(dx_layer* L, const float* h, float* y, int32_t* topk_ids, float* topk_w,
@@ -346,10 +359,9 @@ extern "C" dx_status moe_draft_experts(dx_layer* L, const float* h, float* y, vo
 extern "C" dx_status moe_verify_block(dx_layer* L, const float* h, int32_t K, float* y, int32_t* topk_ids,
                                       float* topk_w, uint64_t* union_mask, int32_t* union_ids, int32_t* union_count,
                                       int32_t* offsets, int32_t* perm, void* stream) {
-  dx_status s = moe_verify_route(L, h, K, y, topk_ids, topk_w, union_mask, union_ids, union_count, offsets, perm,
-                                 stream);
-  if (s != DX_OK) return s;
-  return moe_verify_experts(L, h, K, y, stream);
+  if (!L) return DX_ERR_INVALID_ARG;
+  RouteOut o{topk_ids, topk_w, union_mask, union_ids, union_count, offsets, perm};
+  return do_pair(L, h, K, y, o, false, false, (cudaStream_t)stream);
 }
 
 extern "C" dx_status moe_verify_block_residual(dx_layer* L, const float* h_in, float* h_out, int32_t K,
@@ -359,9 +371,7 @@ extern "C" dx_status moe_verify_block_residual(dx_layer* L, const float* h_in, f
   if (!L) return DX_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;
   RouteOut o{topk_ids, topk_w, union_mask, union_ids, union_count, offsets, perm};
-  dx_status s = do_route(L, h_in, K, h_out, o, false, true, st);
-  if (s != DX_OK) return s;
-  return do_experts(L, h_in, K, h_out, false, true, st);
+  return do_pair(L, h_in, K, h_out, o, false, true, st);
 }
 
 extern "C" dx_status spec_accept(dx_ctx* ctx, const float* h, int32_t M, const void* W_lm, int32_t V, int32_t H,

@@ -48,6 +48,16 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+// Bounded wait for a word that another kernel sets (release/acquire at gpu scope).
+__device__ __forceinline__ bool flag_wait(const unsigned int* word) {
+  for (uint32_t it = 0; it < (1u << 22); ++it) {
+    unsigned int v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(word) : "memory");
+    if (v != 0u) return true;
+    __nanosleep(32);
+  }
+  return false;
+}
 // Bounded wait.  Returns false when it gave up; callers raise the abort flag,
 // after which every wait of the CTA falls through so the CTA still terminates.
 #define DX_WAIT_LIMIT (1u << 22)
@@ -234,12 +244,22 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
     };
     if (lane == 0) issue(0, n_static, s_lo, s_hi);
     __syncwarp();
-    pdl_wait();
+    bool have_list = true;
+    if (p.handover) {
+      if (lane == 0) {   // one poller per CTA: the word sits in a single L2 line
+        have_list = flag_wait(p.handover + 1);
+        if (!have_list) { *abort_flag = 1; atomicExch(p.dev_status, DX_DEV_WAIT_EXPIRED); }
+      }
+      have_list = __shfl_sync(0xffffffffu, have_list, 0);
+    } else {
+      pdl_wait();
+    }
     // the producer warp alone copies the routed part of the work list into shared memory, signals the
     // consumers (bar.arrive: it does not wait for them, they may still be busy with their first reductions)
     // and goes straight on streaming the routed groups
     int e_lo, e_hi, u_lo, u_hi;
     routed_range(W, p, n_static, NS, s_lo, s_hi, e_lo, e_hi, u_lo, u_hi);
+    if (!have_list) e_lo = e_hi = u_lo = u_hi = 0;
     for (int i = e_lo + lane; i < e_hi; i += 32) {
       const DxEntry& en = W->entries[i];
       const unsigned char* blob = reinterpret_cast<const unsigned char*>(p.table[en.table_index]);
@@ -280,6 +300,14 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
   // {hi(k0,k1), hi(k2,k3), lo(k0,k1), lo(k2,k3)} of token slot g
   uint32_t breg[kRegB ? KW : 1][4];
 
+  // the producers are already streaming weights; the block itself may still be written by the kernel in front
+  // of the routing kernel, which publishes its call number once that kernel has completed
+  if (p.handover) {
+    if (threadIdx.x == 0 && !flag_wait(p.handover)) { *abort_flag = 1; atomicExch(p.dev_status, DX_DEV_WAIT_EXPIRED); }
+    consumer_bar();   // one poller per CTA; the others pick the acquire up through the barrier
+  } else {
+    pdl_wait();
+  }
   // 1/rms of every block row when the experts see RMSNorm(x)
   for (int r = warp; r < DX_MAX_K; r += kConsumerWarps) {
     float rs = 1.0f;
@@ -446,10 +474,12 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
   };
 
   process(0, n_static, s_lo, s_hi);
-  pdl_wait();
+  cta_bar();   // the producer warp has seen the routing call's work list and published its routed part
+  // Only now may the next kernel of the stream start: if it is a routing kernel it clears the hand-over words,
+  // and this CTA is done with both of them.
   pdl_launch_dependents();
-  cta_bar();   // the producer warp has published the routed part of the work list
   process(hdr->r_e_lo, hdr->r_e_hi, hdr->r_u_lo, hdr->r_u_hi);
+  pdl_wait();  // the routing kernel (which initialised y) has completed as a whole
 
   // ---- the CTA's partial output rows go to y (initialised by the routing kernel, which has completed)
 #pragma unroll

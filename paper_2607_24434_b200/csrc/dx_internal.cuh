@@ -51,6 +51,7 @@ struct dx_ctx {
   unsigned int* ticket;        // last-CTA tickets (route, accept)
   unsigned long long* keys;    // [DX_MAX_M] packed argmax keys
   int32_t* dev_status;
+  unsigned int* handover;      // device words {block input final, work list complete}: see DxExpertParams
   float2* conf_part;           // [8 * sm_count][DX_MAX_M] per-CTA online-softmax pairs of the confidence variant
   int32_t* scratch_i32;        // two ints the draft-token entry point parks unused outputs in
 };
@@ -84,6 +85,8 @@ struct DxRouteParams {
   int rms_norm;     // 1: route and experts see RMSNorm(h)
   int residual;     // 0: y starts at zero, 1: y starts as a copy of h (pre-norm residual form)
   int tok_group;    // block rows staged in shared memory per pass (set by the launcher)
+  unsigned int* handover; // not null: set word 0 once everything in front of this kernel in the stream has
+                          // completed, and word 1 once the work list is complete
   float* y;
   float* z;
   unsigned int* ticket;
@@ -112,6 +115,12 @@ struct DxExpertParams {
   // window of the routed entries this launch covers (position among them, count or -1 = all) and whether
   // the routing-independent groups are part of it; a cache-staged union is processed in several windows
   int first_routed, n_routed, do_static;
+  // Hand-over from the routing kernel launched right before this one (fused entry points only; null otherwise,
+  // and then the kernel simply waits for everything in front of it).  With the hand-over this kernel may be running
+  // before its inputs are final: consumers read the block only once word 0 is set, and the routed groups are
+  // read only once word 1 is set.  The routing kernel of the next pair clears both words before it lets its own
+  // expert kernel start; this kernel in turn lets that routing kernel start only when it is past both words.
+  unsigned int* handover;
 };
 
 // launchers (each returns the cudaError_t of the launch)

@@ -242,10 +242,28 @@ __global__ void __launch_bounds__(kRouteThreads) dx_route_kernel(DxRouteParams p
     for (size_t o = (size_t)threadIdx.x * 128; o < bytes; o += (size_t)kRouteThreads * 128)
       asm volatile("prefetch.global.L2 [%0];" ::"l"(wb + o));
   }
-  // everything else this kernel reads or writes may still be in use by the previous kernel of the stream;
-  // once that is over, let the expert kernel start on the groups that need no routing
-  dx_pdl_wait();
+  // Let the expert kernel be scheduled right away: its producers only touch constant weights, and its consumers
+  // hold back until this kernel publishes that the block input is final.  Everything else this kernel reads or
+  // writes may still be in use by the previous kernel of the stream, so wait for that kernel first.
+  if (p.handover && crank == 0) {
+    // words left set by the previous pair: every CTA of that pair's expert kernel is past them (it lets this
+    // kernel start only then), and the expert kernel of this pair cannot start before the trigger below
+    if (threadIdx.x == 0) {
+      atomicExch(p.handover, 0u);
+      atomicExch(p.handover + 1, 0u);
+      __threadfence();
+    }
+    __syncthreads();
+  }
   dx_pdl_trigger();
+  dx_pdl_wait();
+  if (p.handover && crank == 0 && threadIdx.x == 0) {
+    __threadfence();
+    atomicExch(p.handover, 1u);
+  }
+  // bias of the first router row of this warp: requested now, used after the dot products
+  float bias_first = 0.f;
+  if (p.bias && e_lo + warp < e_hi) bias_first = p.bias[e_lo + warp];
 
   // the first router row of this warp is requested before anything else, so its latency overlaps the staging
   uint4 wreg[8];
@@ -306,7 +324,7 @@ __global__ void __launch_bounds__(kRouteThreads) dx_route_kernel(DxRouteParams p
         if (!(t0 == 0 && e == e_lo + warp && j0 == 0)) row_load(wrow, j0, chunks, lane, wreg);
         row_dots(wrow, s_h, H, kt, j0, chunks, lane, acc, wreg);
       }
-      const float b = p.bias ? p.bias[e] : 0.f;
+      const float b = (e == e_lo + warp) ? bias_first : (p.bias ? p.bias[e] : 0.f);
 #pragma unroll
       for (int t = 0; t < kTokGroup; ++t) {
         if (t < kt) {
@@ -342,27 +360,29 @@ __global__ void __launch_bounds__(kRouteThreads) dx_route_kernel(DxRouteParams p
   int total;
   const int both = block_exclusive_scan(cnt | (flag << 16), s_scan, total);   // its barriers also publish s_ballot
   const int off = both & 0xffff, upos = both >> 16, ucount = total >> 16;
-  if (me < E) {
-    if (p.offsets) p.offsets[me] = off;
-    int i = 0;
-    for (int q = 0; q < P; ++q)
-      if (s_ids[q] == me) { s_perm[off + i] = q; ++i; }
-    if (flag && p.union_ids) p.union_ids[upos] = me;
-  }
-  if (me == 0) {
-    if (p.offsets) p.offsets[E] = P;
-    if (p.union_count) *p.union_count = ucount;
-  }
-  if (p.union_mask && me < (E + 63) / 64) {
-    unsigned long long lo = s_ballot[2 * me], hi = (2 * me + 1 < kRouteWarps) ? s_ballot[2 * me + 1] : 0u;
-    p.union_mask[me] = lo | (hi << 32);
-  }
-  __syncthreads();
-  if (p.perm)
-    for (int q = me; q < P; q += kRouteThreads) p.perm[q] = s_perm[q];
-
-  // work list
+  // ---- work list first (it is what the expert kernel is waiting for), user-facing outputs afterwards
   DxWork* W = p.work;
+  const int routed_base = p.n_shared * p.shared_tiles;
+  if (me < E) {
+    // this thread's segment of the pair permutation, and (verify mode) its expert's group
+    DxEntry* en = (!p.draft_mode && flag) ? &W->entries[p.n_shared + upos] : nullptr;
+    if (en) {
+      en->table_index = p.n_shared + 1 + me;
+      en->n_tiles = p.routed_tiles;
+      en->unit_begin = routed_base + upos * p.routed_tiles;
+      en->m = cnt;
+#pragma unroll
+      for (int i = 0; i < DX_MAX_K; ++i) en->roww[i] = 0.0f;
+    }
+    int i = 0, q = 0;
+    for (int t = 0; t < K; ++t)
+      for (int j = 0; j < k; ++j, ++q)
+        if (s_ids[q] == me) {
+          s_perm[off + i] = q;
+          if (en) { en->tok[i] = t; en->w[i] = s_w[q]; en->roww[t] = s_w[q]; }
+          ++i;
+        }
+  }
   if (me < p.n_shared) {
     DxEntry& en = W->entries[me];
     en.table_index = me;
@@ -373,22 +393,7 @@ __global__ void __launch_bounds__(kRouteThreads) dx_route_kernel(DxRouteParams p
     for (int i = 0; i < K; ++i) { en.tok[i] = i; en.w[i] = 1.0f; }
   }
   int n_entries, total_units;
-  const int routed_base = p.n_shared * p.shared_tiles;
   if (!p.draft_mode) {
-    if (me < E && flag) {
-      DxEntry& en = W->entries[p.n_shared + upos];
-      en.table_index = p.n_shared + 1 + me;
-      en.n_tiles = p.routed_tiles;
-      en.unit_begin = routed_base + upos * p.routed_tiles;
-      en.m = cnt;
-      for (int i = 0; i < DX_MAX_K; ++i) en.roww[i] = 0.0f;
-      for (int i = 0; i < cnt; ++i) {
-        int q = s_perm[off + i];
-        en.tok[i] = q / k;
-        en.w[i] = s_w[q];
-        en.roww[q / k] = s_w[q];
-      }
-    }
     n_entries = p.n_shared + ucount;
     total_units = routed_base + ucount * p.routed_tiles;
   } else {
@@ -424,6 +429,25 @@ __global__ void __launch_bounds__(kRouteThreads) dx_route_kernel(DxRouteParams p
     W->total_units = total_units;
     W->K = K;
   }
+  __threadfence();
+  __syncthreads();
+  if (p.handover && me == 0) atomicExch(p.handover + 1, 1u);   // the work list is complete and visible
+
+  // ---- routing outputs for the caller
+  if (me < E) {
+    if (p.offsets) p.offsets[me] = off;
+    if (flag && p.union_ids) p.union_ids[upos] = me;
+  }
+  if (me == 0) {
+    if (p.offsets) p.offsets[E] = P;
+    if (p.union_count) *p.union_count = ucount;
+  }
+  if (p.union_mask && me < (E + 63) / 64) {
+    unsigned long long lo = s_ballot[2 * me], hi = (2 * me + 1 < kRouteWarps) ? s_ballot[2 * me + 1] : 0u;
+    p.union_mask[me] = lo | (hi << 32);
+  }
+  if (p.perm)
+    for (int q = me; q < P; q += kRouteThreads) p.perm[q] = s_perm[q];
 }
 
 }  // namespace

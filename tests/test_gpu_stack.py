@@ -70,3 +70,61 @@ def test_v2lite_stack_correlated_block():
 def test_moonlight_stack_sigmoid_scaled():
     unions, near = _run_stack(synth.shape_moonlight(), 3, 4, seed=600, zipf=True, vocab=163840)
     assert all(6 <= u <= 24 for u in unions)
+
+
+def test_stack_graph_replay_handover():
+    """Back-to-back launches from a CUDA graph: each expert kernel starts while the previous layer is still running
+    and picks its block input and its routed groups up through the device-side hand-over.  Every replay gets a new
+    input block; each layer's output is checked against the checker on that layer's own input and routing, so a
+    kernel that ran ahead with the previous layer's work list or a half-written input fails."""
+    from paper_2607_24434_b200 import binding
+    sh = synth.shape_v2lite()
+    n_layers, K = 4, 4
+    ctx = binding.Context(0)
+    refs, Ls = [], []
+    for l in range(n_layers):
+        layer = synth.make_layer(sh, 700 + 10 * l, "cuda", zipf=True)
+        refs.append(synth.layer_to_numpy(layer))
+        Ls.append(binding.Layer.from_weights(ctx, layer))
+        del layer
+    hs = [torch.zeros((K, sh.hidden), device="cuda") for _ in range(n_layers + 1)]
+    hd = [torch.zeros((1, sh.hidden), device="cuda") for _ in range(n_layers + 1)]
+    rb = [binding._routing_buffers(sh, K, "cuda") for _ in range(n_layers)]
+    db = [{"topk_ids": torch.empty((sh.top_k,), dtype=torch.int32, device="cuda"),
+           "topk_w": torch.empty((sh.top_k,), device="cuda")} for _ in range(n_layers)]
+
+    def chain():
+        for l in range(n_layers):
+            binding.moe_draft_step_residual(Ls[l], hd[l], hd[l + 1], db[l])
+        for l in range(n_layers):
+            binding.moe_verify_block_residual(Ls[l], hs[l], hs[l + 1], rb[l])
+
+    stream = torch.cuda.current_stream()
+    side = torch.cuda.Stream()
+    side.wait_stream(stream)
+    with torch.cuda.stream(side):
+        chain()
+    stream.wait_stream(side)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=side):
+        chain()
+    for rep in range(3):
+        hs[0].copy_(synth.hidden_block(K, sh.hidden, 710 + rep, 0.5, "cuda"))
+        hd[0].copy_(hs[0][:1])
+        g.replay()
+        g.replay()          # two replays in a row: the second must not be confused by what the first left behind
+        torch.cuda.synchronize()
+        assert ctx.device_status() == 0
+        for l in range(n_layers):
+            h_np = hs[l].cpu().numpy().astype(np.float64)
+            ids = rb[l]["topk_ids"].cpu().numpy()
+            want = O.stack_layer_target(h_np, refs[l], forced_ids=ids)[0]
+            assert row_rel_err(hs[l + 1].cpu().numpy(), want).max() <= Y_TIGHT, (rep, l)
+            check_union(sh, K, ids, rb[l])
+            wantd = O.stack_layer_draft(hd[l].cpu().numpy().astype(np.float64), refs[l],
+                                        forced_ids=db[l]["topk_ids"].cpu().numpy()[None])[0]
+            assert row_rel_err(hd[l + 1].cpu().numpy(), wantd).max() <= Y_TIGHT, (rep, l)
+    for L in Ls:
+        L.close()
+    ctx.close()
