@@ -236,7 +236,7 @@ static dx_status do_route(dx_layer* L, const float* h, int K, float* y, const Ro
   DxRouteParams p{};
   p.h = h; p.K = K; p.H = d.hidden; p.E = d.n_experts; p.k = d.top_k;
   p.score_fn = d.score_fn; p.norm_topk = d.norm_topk; p.scale = d.routed_scale; p.gamma = d.draft_gamma;
-  p.W_r = L->W_r; p.bias = L->bias;
+  p.W_r = L->W_r; p.bias = L->bias; p.table = L->table_dev;
   p.n_shared = d.n_shared;
   p.shared_tiles = d.n_shared ? d.shared_inter / DX_TILE_I : 0;
   p.routed_tiles = d.inter / DX_TILE_I;
@@ -276,6 +276,7 @@ static dx_status do_experts(dx_layer* L, const float* h, int K, float* y, bool d
   p.n_shared = d.n_shared;
   p.shared_tiles = d.n_shared ? d.shared_inter / DX_TILE_I : 0;
   p.draft_tiles = draft ? d.draft_inter / DX_TILE_I : 0;
+  p.routed_tiles = d.inter / DX_TILE_I;
   p.gamma = d.draft_gamma;
   p.handover = paired ? ctx->handover : nullptr;
   p.first_routed = first_routed;

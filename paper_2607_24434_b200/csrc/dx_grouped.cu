@@ -106,14 +106,6 @@ __device__ __forceinline__ uint32_t pack2(__nv_bfloat16 lo16, __nv_bfloat16 hi16
   return (uint32_t)__bfloat16_as_ushort(lo16) | ((uint32_t)__bfloat16_as_ushort(hi16) << 16);
 }
 
-__device__ __forceinline__ int find_entry(const DxWork* W, int n_entries, int u, int start) {
-  int ei = start;
-  while (ei + 1 < n_entries && u >= W->entries[ei + 1].unit_begin) ++ei;
-  // entries with zero tiles share unit_begin with their successor; skip them
-  while (ei + 1 < n_entries && W->entries[ei].n_tiles == 0) ++ei;
-  return ei;
-}
-
 // ----------------------------------------------------- bf16 tensor-core path
 // Streaming layout.  A unit (8 gate rows, 8 up rows, 8 down columns; 48*H bytes)
 // is stored as eight equal "chunks", one per consumer warp: chunk w holds the
@@ -141,10 +133,13 @@ struct SmemHeader {
   int r_e_lo, r_e_hi, r_u_lo;   // this CTA's routed entries and units, published by the producer warp
   int r_u_hi;
   float rstd[DX_MAX_K];
-  int e_begin[DX_MAX_ENTRIES];       // first unit of each entry
+  int e_begin[DX_MAX_ENTRIES];       // first unit of each group (routing-independent groups first)
   int e_tiles[DX_MAX_ENTRIES];
-  int e_m[DX_MAX_ENTRIES];
+  int e_gid[DX_MAX_ENTRIES];         // expert id of a routed group
   const unsigned char* e_blob[DX_MAX_ENTRIES];
+  int kk;                            // selected experts per block row
+  int pair_id[DX_MAX_PAIRS];         // [K,kk] selected expert ids and gate weights of the block
+  float pair_w[DX_MAX_PAIRS];
 };
 
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
@@ -154,16 +149,17 @@ __device__ __forceinline__ void cta_bar() { asm volatile("bar.sync 2, 288;" ::: 
 // This CTA's share of the routed groups.  The launch may be restricted to a window of the routed entries
 // (a "wave" of union experts when the experts are staged through a cache); the units of the window, together
 // with the routing-independent units handled before (NSe of them, [s_lo,s_hi) on this CTA), are split evenly.
-__device__ __forceinline__ void routed_range(const DxWork* W, const DxExpertParams& p, int n_static, int NSe, int s_lo,
+__device__ __forceinline__ void routed_range(int n_groups, const DxExpertParams& p, int n_static, int NSe, int s_lo,
                                              int s_hi, int& e_lo, int& e_hi, int& u_lo, int& u_hi) {
   const int G = gridDim.x, cta = blockIdx.x;
-  const int n_all = W->n_entries;
-  e_lo = min(n_all, n_static + p.first_routed);
-  e_hi = p.n_routed < 0 ? n_all : min(n_all, e_lo + p.n_routed);
-  if (e_lo >= e_hi) { u_lo = u_hi = 0; return; }
-  const long long R0 = W->entries[e_lo].unit_begin;
-  const long long R1 = (long long)W->entries[e_hi - 1].unit_begin + W->entries[e_hi - 1].n_tiles;
-  const long long NR = R1 - R0, T = NSe + NR;
+  const int g_lo = min(n_groups, p.first_routed);
+  const int g_hi = p.n_routed < 0 ? n_groups : min(n_groups, g_lo + p.n_routed);
+  e_lo = n_static + g_lo;
+  e_hi = n_static + g_hi;
+  if (g_lo >= g_hi) { u_lo = u_hi = 0; return; }
+  const long long base = (long long)p.n_shared * p.shared_tiles + p.draft_tiles;
+  const long long R0 = base + (long long)g_lo * p.routed_tiles;
+  const long long NR = (long long)(g_hi - g_lo) * p.routed_tiles, T = NSe + NR;
   long long a, b;
   if (T / G >= (NSe + G - 1) / G) {   // keep routing-independent + routed units balanced together
     a = (T * cta) / G - s_lo; b = (T * (cta + 1)) / G - s_hi;
@@ -214,7 +210,6 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
     const bool is_draft = i >= p.n_shared;
     hdr->e_begin[i] = is_draft ? p.n_shared * p.shared_tiles : i * p.shared_tiles;
     hdr->e_tiles[i] = is_draft ? p.draft_tiles : p.shared_tiles;
-    hdr->e_m[i] = is_draft ? 1 : p.K;
     hdr->e_blob[i] = reinterpret_cast<const unsigned char*>(p.table[i]);
   }
   __syncthreads();
@@ -254,19 +249,49 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
     } else {
       pdl_wait();
     }
-    // the producer warp alone copies the routed part of the work list into shared memory, signals the
-    // consumers (bar.arrive: it does not wait for them, they may still be busy with their first reductions)
-    // and goes straight on streaming the routed groups
-    int e_lo, e_hi, u_lo, u_hi;
-    routed_range(W, p, n_static, NS, s_lo, s_hi, e_lo, e_hi, u_lo, u_hi);
-    if (!have_list) e_lo = e_hi = u_lo = u_hi = 0;
-    for (int i = e_lo + lane; i < e_hi; i += 32) {
-      const DxEntry& en = W->entries[i];
-      const unsigned char* blob = reinterpret_cast<const unsigned char*>(p.table[en.table_index]);
-      hdr->e_begin[i] = en.unit_begin; hdr->e_tiles[i] = en.n_tiles; hdr->e_m[i] = en.m; hdr->e_blob[i] = blob;
-      if (blob == nullptr && en.n_tiles > 0) atomicExch(p.dev_status, DX_DEV_BAD_EXPERT_ID);
+    // the producer warp alone copies the group list into shared memory, signals the consumers (bar.arrive: it
+    // does not wait for them, they may still be busy with their first reductions) and goes straight on streaming
+    // the routed groups.  Everything is requested in one round of loads, whatever the group count turns out to be.
+    constexpr int PER_LANE = DX_MAX_PAIRS / 32;
+    const int n_groups = have_list ? min(W->n_groups, DX_MAX_PAIRS) : 0;
+    const int kk = W->k;
+    int gid_l[PER_LANE], pid_l[PER_LANE];
+    float pw_l[PER_LANE];
+    const unsigned char* blob_l[PER_LANE];
+#pragma unroll
+    for (int i = 0; i < PER_LANE; ++i) {
+      const int idx = lane + 32 * i;
+      gid_l[i] = W->gid[idx];
+      pid_l[i] = W->pair_id[idx];
+      pw_l[i] = W->pair_w[idx];
+      blob_l[i] = reinterpret_cast<const unsigned char*>(W->gblob[idx]);
     }
-    if (lane == 0) { hdr->r_e_lo = e_lo; hdr->r_e_hi = e_hi; hdr->r_u_lo = u_lo; hdr->r_u_hi = u_hi; }
+    int e_lo, e_hi, u_lo, u_hi;
+    routed_range(n_groups, p, n_static, NS, s_lo, s_hi, e_lo, e_hi, u_lo, u_hi);
+    const int unit_base = p.n_shared * p.shared_tiles + p.draft_tiles;
+#pragma unroll
+    for (int i = 0; i < PER_LANE; ++i) {
+      const int idx = lane + 32 * i;
+      hdr->pair_id[idx] = pid_l[i];
+      hdr->pair_w[idx] = pw_l[i];
+      if (idx < n_groups) {
+        const unsigned char* blob = blob_l[i];
+        // without the hand-over the table may have changed since the routing kernel ran (experts staged by the
+        // cache in between): read it now
+        if (!p.handover && gid_l[i] >= 0 && gid_l[i] < DX_MAX_E)
+          blob = reinterpret_cast<const unsigned char*>(p.table[p.n_shared + 1 + gid_l[i]]);
+        const int e = n_static + idx;
+        hdr->e_begin[e] = unit_base + idx * p.routed_tiles;
+        hdr->e_tiles[e] = p.routed_tiles;
+        hdr->e_gid[e] = gid_l[i];
+        hdr->e_blob[e] = blob;
+        if (blob == nullptr && e >= e_lo && e < e_hi) atomicExch(p.dev_status, DX_DEV_BAD_EXPERT_ID);
+      }
+    }
+    if (lane == 0) {
+      hdr->kk = kk;
+      hdr->r_e_lo = e_lo; hdr->r_e_hi = e_hi; hdr->r_u_lo = u_lo; hdr->r_u_hi = u_hi;
+    }
     __threadfence_block();   // bar.arrive alone does not order the shared-memory writes above
     __syncwarp();
     asm volatile("bar.arrive 2, 288;" ::: "memory");
@@ -336,7 +361,12 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
   // across groups (the weight is folded into the activations) and y is touched once, at the very end.
   auto row_weight = [&](int e, int row) -> float {
     if (e < n_static) return row < p.K ? (e < p.n_shared ? 1.0f : p.gamma) : 0.0f;
-    return W->entries[e].roww[row];
+    if (row >= p.K) return 0.0f;
+    const int gid = hdr->e_gid[e], kk = hdr->kk;
+    float w = 0.0f;
+    for (int j = 0; j < kk; ++j)
+      if (hdr->pair_id[row * kk + j] == gid) w = hdr->pair_w[row * kk + j];
+    return w;
   };
 
   auto process = [&](int e0, int e1, int lo_u, int hi_u) {
@@ -514,7 +544,7 @@ __global__ void __launch_bounds__(256) dx_experts_fp32_kernel(DxExpertParams p) 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   dx_pdl_wait();
   dx_pdl_trigger();
-  const int n_entries = W->n_entries, total = W->total_units, H = p.H;
+  const int n_groups = min(W->n_groups, DX_MAX_PAIRS), kk = W->k, H = p.H;
   for (int r = warp; r < DX_MAX_K; r += 8) {
     float rs = 1.0f;
     if (p.rms_norm && r < p.K) {
@@ -527,29 +557,56 @@ __global__ void __launch_bounds__(256) dx_experts_fp32_kernel(DxExpertParams p) 
     if (lane == 0) s_rstd[r] = rs;
   }
   __syncthreads();
-  // window of the routed entries covered by this launch (see routed_range) and the routing-independent units
-  const int n_static = p.n_shared + (p.draft_tiles > 0 ? 1 : 0);
+  // window of the routed groups covered by this launch (see routed_range) and the routing-independent units
   const int NS_all = p.n_shared * p.shared_tiles + p.draft_tiles;
-  const int we_lo = min(n_entries, n_static + p.first_routed);
-  const int we_hi = p.n_routed < 0 ? n_entries : min(n_entries, we_lo + p.n_routed);
-  const int wu_lo = we_lo < we_hi ? W->entries[we_lo].unit_begin : 0;
-  const int wu_hi = we_lo < we_hi ? W->entries[we_hi - 1].unit_begin + W->entries[we_hi - 1].n_tiles : 0;
-  int ei = 0;
+  const int g_lo = min(n_groups, p.first_routed);
+  const int g_hi = p.n_routed < 0 ? n_groups : min(n_groups, g_lo + p.n_routed);
+  const int wu_lo = NS_all + g_lo * p.routed_tiles, wu_hi = NS_all + g_hi * p.routed_tiles;
+  const int total = NS_all + n_groups * p.routed_tiles;
+  __shared__ float s_roww[DX_MAX_K];
   for (int u = blockIdx.x; u < total; u += gridDim.x) {
     if (u < NS_all ? !p.do_static : (u < wu_lo || u >= wu_hi)) continue;
-    ei = find_entry(W, n_entries, u, ei);
-    const DxEntry& en = W->entries[ei];
-    const float* blob = reinterpret_cast<const float*>(p.table[en.table_index]);
+    // the group of this unit, its blob and its weight in every block row (0 = the row is not in the group)
+    int table_index, unit_begin, gid = -1;
+    float w_static = 1.0f;
+    if (u < p.n_shared * p.shared_tiles) {
+      table_index = u / p.shared_tiles;
+      unit_begin = table_index * p.shared_tiles;
+    } else if (u < NS_all) {
+      table_index = p.n_shared;
+      unit_begin = p.n_shared * p.shared_tiles;
+      w_static = p.gamma;
+    } else {
+      const int gi = (u - NS_all) / p.routed_tiles;
+      gid = W->gid[gi];
+      table_index = p.n_shared + 1 + gid;
+      unit_begin = NS_all + gi * p.routed_tiles;
+    }
+    if (threadIdx.x < DX_MAX_K) {
+      const int row = threadIdx.x;
+      float w = 0.0f;
+      if (row < p.K) {
+        if (gid < 0) w = w_static;
+        else
+          for (int j = 0; j < kk; ++j)
+            if (W->pair_id[row * kk + j] == gid) w = W->pair_w[row * kk + j];
+      }
+      s_roww[row] = w;
+    }
+    __syncthreads();
+    const float* blob = reinterpret_cast<const float*>(p.table[table_index]);
     if (blob == nullptr) {
       if (threadIdx.x == 0) atomicExch(p.dev_status, DX_DEV_BAD_EXPERT_ID);
+      __syncthreads();
       continue;
     }
-    const float* unit = blob + (size_t)(u - en.unit_begin) * 24 * H;
+    const float* unit = blob + (size_t)(u - unit_begin) * 24 * H;
     const float* gr = unit + (size_t)warp * H;
     const float* ur = unit + (size_t)(8 + warp) * H;
-    for (int t = 0; t < en.m; ++t) {
-      const float* x = p.x + (size_t)en.tok[t] * H;
-      const float rs = s_rstd[en.tok[t]];
+    for (int t = 0; t < p.K; ++t) {
+      if (s_roww[t] == 0.0f) continue;
+      const float* x = p.x + (size_t)t * H;
+      const float rs = s_rstd[t];
       float ag = 0.f, au = 0.f;
       for (int j = lane; j < H; j += 32) {
         const float xv = x[j] * rs;
@@ -569,11 +626,12 @@ __global__ void __launch_bounds__(256) dx_experts_fp32_kernel(DxExpertParams p) 
       float d[8];
 #pragma unroll
       for (int i = 0; i < 8; ++i) d[i] = dT[(size_t)i * H + hh];
-      for (int t = 0; t < en.m; ++t) {
+      for (int t = 0; t < p.K; ++t) {
+        if (s_roww[t] == 0.0f) continue;
         float s = 0.f;
 #pragma unroll
         for (int i = 0; i < 8; ++i) s = fmaf(s_act[t][i], d[i], s);
-        atomicAdd(p.y + (size_t)en.tok[t] * H + hh, en.w[t] * s);
+        atomicAdd(p.y + (size_t)t * H + hh, s_roww[t] * s);
       }
     }
     __syncthreads();

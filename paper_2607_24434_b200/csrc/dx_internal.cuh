@@ -19,24 +19,18 @@
 #define DX_TILE_I 8            // intermediate rows per streamed weight tile
 #define DX_MAX_M 16            // accept rows
 
-// One group of the grouped SwiGLU: an expert (by index into the layer's blob
-// table) together with the block tokens routed to it and their output weights.
-struct DxEntry {
-  int32_t table_index;   // index into the layer's device blob table
-  int32_t n_tiles;       // I / DX_TILE_I of this expert (0 = skip)
-  int32_t unit_begin;    // first global work-unit index of this entry
-  int32_t m;             // tokens in the group (<= K)
-  int32_t tok[DX_MAX_K]; // block row of each group token
-  float w[DX_MAX_K];     // weight of this expert's output in that row (g, 1 or gamma)
-  float roww[DX_MAX_K];  // the same weights indexed by block row (0 = the row is not in this group)
-};
-
+// What the routing kernel hands to the expert kernels.  The routing-independent groups (shared experts, draft
+// expert) follow from the launch parameters alone; the routed groups are listed here, one per expert that some
+// block row selected, in the order in which their work units are numbered.  A group's weight in block row t is
+// the gate weight of the pair (t, j) that selected its expert, or nothing if no pair of that row did.
 struct DxWork {
-  int32_t n_entries;
-  int32_t total_units;
-  int32_t K;
+  int32_t n_groups;                   // routed groups
+  int32_t K, k;                       // block rows and selected experts per row
   int32_t pad;
-  DxEntry entries[DX_MAX_ENTRIES];
+  int32_t gid[DX_MAX_PAIRS];          // expert id of group i
+  const void* gblob[DX_MAX_PAIRS];    // its blob as the layer's table had it when the routing kernel ran
+  int32_t pair_id[DX_MAX_PAIRS];      // [K,k] selected expert ids, row-major
+  float pair_w[DX_MAX_PAIRS];         // [K,k] their gate weights
 };
 
 struct dx_ctx {
@@ -79,6 +73,7 @@ struct DxRouteParams {
   float scale, gamma;
   const void* W_r;
   const float* bias;
+  const void* const* table;   // layer blob table (device)
   int n_shared, shared_tiles, routed_tiles, draft_tiles;
   int draft_mode;   // 0: verify block, 1: drafter (shared + draft expert + top_r routed)
   int top_r;
@@ -110,7 +105,7 @@ struct DxExpertParams {
   int H, K;
   int rms_norm;              // 1: the experts see RMSNorm(x) (unit gain, eps 1e-6)
   // groups known without routing: shared experts (all K rows, weight 1) and, in draft mode, the draft expert
-  int n_shared, shared_tiles, draft_tiles;
+  int n_shared, shared_tiles, draft_tiles, routed_tiles;
   float gamma;
   // window of the routed entries this launch covers (position among them, count or -1 = all) and whether
   // the routing-independent groups are part of it; a cache-staged union is processed in several windows

@@ -158,8 +158,8 @@ __device__ __forceinline__ void row_dots(const float* wrow, const float* h, int 
 // Top-k of one token by one warp: k rounds of (lane-local best, warp max of the logit, warp min of the id among
 // the holders of that maximum); then softmax / sigmoid scores of the selected experts and their gate weights.
 template <int NK>
-__device__ __forceinline__ void topk_token(const DxRouteParams& p, const float* s_z, int* s_ids, float* s_w, int tt,
-                                           int lane) {
+__device__ __forceinline__ void topk_token(const DxRouteParams& p, const float* s_z, int* s_ids, float* s_w,
+                                           unsigned int* s_mask, int tt, int lane) {
   const int E = p.E, k = p.k;
     unsigned long long key[NK];
     float zv[NK];
@@ -214,6 +214,7 @@ __device__ __forceinline__ void topk_token(const DxRouteParams& p, const float* 
     if (lane < k) {
       s_ids[tt * k + lane] = my_e;
       s_w[tt * k + lane] = g;
+      atomicOr(&s_mask[my_e >> 5], 1u << (my_e & 31));   // union of Eq. 2 / Eq. 3 as a bit mask
       if (p.topk_ids) p.topk_ids[tt * k + lane] = my_e;
       if (p.topk_w) p.topk_w[tt * k + lane] = g;
     }
@@ -227,7 +228,8 @@ __global__ void __launch_bounds__(kRouteThreads) dx_route_kernel(DxRouteParams p
   __shared__ float s_w[DX_MAX_PAIRS];
   __shared__ int s_perm[DX_MAX_PAIRS];
   __shared__ int s_scan[kRouteWarps];
-  __shared__ unsigned int s_ballot[kRouteWarps];
+  __shared__ unsigned int s_mask[DX_MAX_E / 32];
+  __shared__ const void* s_tab[DX_MAX_E];
 
   cg::cluster_group cluster = cg::this_cluster();
   const int crank = (int)cluster.block_rank();
@@ -260,6 +262,11 @@ __global__ void __launch_bounds__(kRouteThreads) dx_route_kernel(DxRouteParams p
   if (p.handover && crank == 0 && threadIdx.x == 0) {
     __threadfence();
     atomicExch(p.handover, 1u);
+  }
+  // routed part of the blob table (final now), for the group list at the end
+  if (crank == 0) {
+    if (threadIdx.x < E) s_tab[threadIdx.x] = p.table[p.n_shared + 1 + threadIdx.x];
+    if (threadIdx.x < DX_MAX_E / 32) s_mask[threadIdx.x] = 0u;
   }
   // bias of the first router row of this warp: requested now, used after the dot products
   float bias_first = 0.f;
@@ -339,102 +346,57 @@ __global__ void __launch_bounds__(kRouteThreads) dx_route_kernel(DxRouteParams p
 
   // top-k and gate weights, one warp per token (NK = keys per lane, a power of two covering E)
   for (int tt = warp; tt < K; tt += kRouteWarps) {
-    if (E <= 32) topk_token<1>(p, s_z, s_ids, s_w, tt, lane);
-    else if (E <= 64) topk_token<2>(p, s_z, s_ids, s_w, tt, lane);
-    else if (E <= 128) topk_token<4>(p, s_z, s_ids, s_w, tt, lane);
-    else topk_token<8>(p, s_z, s_ids, s_w, tt, lane);
+    if (E <= 32) topk_token<1>(p, s_z, s_ids, s_w, s_mask, tt, lane);
+    else if (E <= 64) topk_token<2>(p, s_z, s_ids, s_w, s_mask, tt, lane);
+    else if (E <= 128) topk_token<4>(p, s_z, s_ids, s_w, s_mask, tt, lane);
+    else topk_token<8>(p, s_z, s_ids, s_w, s_mask, tt, lane);
   }
   __syncthreads();
 
-  // counting sort of the pairs by expert; thread e owns expert e
+  // ---- group list for the expert kernel (it is waiting for it); the caller's outputs come afterwards
   const int me = threadIdx.x;
+  DxWork* W = p.work;
+  int flag = 0, upos = 0, ucount = 0;
+  {
+    const unsigned int mine = me < E ? s_mask[me >> 5] : 0u;
+    flag = (mine >> (me & 31)) & 1u;
+    for (int w2 = 0; w2 < (E + 31) / 32; ++w2) {
+      const int c = __popc(s_mask[w2]);
+      ucount += c;
+      if (w2 < (me >> 5)) upos += c;
+    }
+    upos += __popc(mine & ((1u << (me & 31)) - 1u));
+  }
+  if (!p.draft_mode) {
+    if (flag) { W->gid[upos] = me; W->gblob[upos] = s_tab[me]; }
+  } else if (me < p.top_r) {
+    W->gid[me] = s_ids[me];
+    W->gblob[me] = s_tab[s_ids[me]];
+  }
+  for (int q = me; q < P; q += kRouteThreads) { W->pair_id[q] = s_ids[q]; W->pair_w[q] = s_w[q]; }
+  if (me == 0) {
+    W->n_groups = p.draft_mode ? p.top_r : ucount;
+    W->K = K;
+    W->k = k;
+  }
+  __syncthreads();
+  if (p.handover && me == 0) {
+    __threadfence();   // cumulative: covers the other threads' stores ordered before the barrier
+    atomicExch(p.handover + 1, 1u);
+  }
+
+  // ---- routing outputs for the caller: pairs sorted by expert (counting sort; thread e owns expert e)
   int cnt = 0;
   if (me < E) {
 #pragma unroll 8
     for (int q = 0; q < P; ++q) cnt += (s_ids[q] == me);
   }
-  // one scan carries both prefix sums: pair counts in the low half, union membership in the high half
-  const int flag = cnt > 0;
-  const unsigned int bal = __ballot_sync(0xffffffffu, flag);
-  if (lane == 0) s_ballot[warp] = bal;
   int total;
-  const int both = block_exclusive_scan(cnt | (flag << 16), s_scan, total);   // its barriers also publish s_ballot
-  const int off = both & 0xffff, upos = both >> 16, ucount = total >> 16;
-  // ---- work list first (it is what the expert kernel is waiting for), user-facing outputs afterwards
-  DxWork* W = p.work;
-  const int routed_base = p.n_shared * p.shared_tiles;
+  const int off = block_exclusive_scan(cnt, s_scan, total);
   if (me < E) {
-    // this thread's segment of the pair permutation, and (verify mode) its expert's group
-    DxEntry* en = (!p.draft_mode && flag) ? &W->entries[p.n_shared + upos] : nullptr;
-    if (en) {
-      en->table_index = p.n_shared + 1 + me;
-      en->n_tiles = p.routed_tiles;
-      en->unit_begin = routed_base + upos * p.routed_tiles;
-      en->m = cnt;
-#pragma unroll
-      for (int i = 0; i < DX_MAX_K; ++i) en->roww[i] = 0.0f;
-    }
-    int i = 0, q = 0;
-    for (int t = 0; t < K; ++t)
-      for (int j = 0; j < k; ++j, ++q)
-        if (s_ids[q] == me) {
-          s_perm[off + i] = q;
-          if (en) { en->tok[i] = t; en->w[i] = s_w[q]; en->roww[t] = s_w[q]; }
-          ++i;
-        }
-  }
-  if (me < p.n_shared) {
-    DxEntry& en = W->entries[me];
-    en.table_index = me;
-    en.n_tiles = p.shared_tiles;
-    en.unit_begin = me * p.shared_tiles;
-    en.m = K;
-    for (int i = 0; i < DX_MAX_K; ++i) en.roww[i] = i < K ? 1.0f : 0.0f;
-    for (int i = 0; i < K; ++i) { en.tok[i] = i; en.w[i] = 1.0f; }
-  }
-  int n_entries, total_units;
-  if (!p.draft_mode) {
-    n_entries = p.n_shared + ucount;
-    total_units = routed_base + ucount * p.routed_tiles;
-  } else {
-    int base = p.n_shared;
-    if (p.draft_tiles > 0) {
-      if (me == 0) {
-        DxEntry& en = W->entries[base];
-        en.table_index = p.n_shared;
-        en.n_tiles = p.draft_tiles;
-        en.unit_begin = routed_base;
-        en.m = 1;
-        en.tok[0] = 0;
-        en.w[0] = p.gamma;
-        for (int i = 0; i < DX_MAX_K; ++i) en.roww[i] = i == 0 ? p.gamma : 0.0f;
-      }
-      base += 1;
-    }
-    if (me < p.top_r) {
-      DxEntry& en = W->entries[base + me];
-      en.table_index = p.n_shared + 1 + s_ids[me];
-      en.n_tiles = p.routed_tiles;
-      en.unit_begin = routed_base + p.draft_tiles + me * p.routed_tiles;
-      en.m = 1;
-      en.tok[0] = 0;
-      en.w[0] = s_w[me];
-      for (int i = 0; i < DX_MAX_K; ++i) en.roww[i] = i == 0 ? s_w[me] : 0.0f;
-    }
-    n_entries = base + p.top_r;
-    total_units = routed_base + p.draft_tiles + p.top_r * p.routed_tiles;
-  }
-  if (me == 0) {
-    W->n_entries = n_entries;
-    W->total_units = total_units;
-    W->K = K;
-  }
-  __threadfence();
-  __syncthreads();
-  if (p.handover && me == 0) atomicExch(p.handover + 1, 1u);   // the work list is complete and visible
-
-  // ---- routing outputs for the caller
-  if (me < E) {
+    int i = 0;
+    for (int q = 0; q < P; ++q)
+      if (s_ids[q] == me) s_perm[off + i++] = q;
     if (p.offsets) p.offsets[me] = off;
     if (flag && p.union_ids) p.union_ids[upos] = me;
   }
@@ -443,9 +405,10 @@ __global__ void __launch_bounds__(kRouteThreads) dx_route_kernel(DxRouteParams p
     if (p.union_count) *p.union_count = ucount;
   }
   if (p.union_mask && me < (E + 63) / 64) {
-    unsigned long long lo = s_ballot[2 * me], hi = (2 * me + 1 < kRouteWarps) ? s_ballot[2 * me + 1] : 0u;
+    const unsigned long long lo = s_mask[2 * me], hi = (2 * me + 1 < DX_MAX_E / 32) ? s_mask[2 * me + 1] : 0u;
     p.union_mask[me] = lo | (hi << 32);
   }
+  __syncthreads();
   if (p.perm)
     for (int q = me; q < P; q += kRouteThreads) p.perm[q] = s_perm[q];
 }
