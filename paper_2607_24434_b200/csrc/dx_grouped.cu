@@ -239,32 +239,49 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
     };
     if (lane == 0) issue(0, n_static, s_lo, s_hi);
     __syncwarp();
-    bool have_list = true;
-    if (p.handover) {
-      if (lane == 0) {   // one poller per CTA: the word sits in a single L2 line
-        have_list = flag_wait(p.handover + 1);
-        if (!have_list) { *abort_flag = 1; atomicExch(p.dev_status, DX_DEV_WAIT_EXPIRED); }
-      }
-      have_list = __shfl_sync(0xffffffffu, have_list, 0);
-    } else {
-      pdl_wait();
-    }
-    // the producer warp alone copies the group list into shared memory, signals the consumers (bar.arrive: it
-    // does not wait for them, they may still be busy with their first reductions) and goes straight on streaming
-    // the routed groups.  Everything is requested in one round of loads, whatever the group count turns out to be.
+    // The routed groups: the producer warp alone reads the work list, copies it into shared memory, signals the
+    // consumers (bar.arrive: it does not wait for them, they may still be busy with their first reductions) and
+    // goes straight on streaming.  With the hand-over the list is being written while this warp polls it; each
+    // word says by itself when it is there.  Otherwise the routing kernel has completed once the wait returns,
+    // and the first look succeeds.
+    if (!p.handover) pdl_wait();
     constexpr int PER_LANE = DX_MAX_PAIRS / 32;
-    const int n_groups = have_list ? min(W->n_groups, DX_MAX_PAIRS) : 0;
-    const int kk = W->k;
-    int gid_l[PER_LANE], pid_l[PER_LANE];
-    float pw_l[PER_LANE];
-    const unsigned char* blob_l[PER_LANE];
+    unsigned long long gw[PER_LANE], pw[PER_LANE];
 #pragma unroll
-    for (int i = 0; i < PER_LANE; ++i) {
+    for (int i = 0; i < PER_LANE; ++i) gw[i] = pw[i] = 0ull;
+    int n_groups = 0, kk = 1, n_pairs = 0;
+    bool have_list = false;
+    for (uint32_t look = 0; look < (1u << 22) && !have_list; ++look) {
+      const unsigned long long head = dx_word_load(&W->head);
+      gw[0] = dx_word_load(&W->group[lane]);
+      pw[0] = dx_word_load(&W->pair[lane]);
+      bool mine = false;
+      if (head & DX_WORD_VALID) {
+        n_groups = min((int)(head & 0xffffu), DX_MAX_PAIRS);
+        kk = (int)((head >> 16) & 0xffu);
+        n_pairs = min((int)((head >> 24) & 0xffu) * kk, DX_MAX_PAIRS);
+        mine = (lane >= n_groups || (gw[0] & DX_WORD_VALID)) && (lane >= n_pairs || (pw[0] & DX_WORD_VALID));
+      }
+      have_list = __all_sync(0xffffffffu, mine);
+    }
+    // larger blocks: the words beyond the first 32 of each kind
+#pragma unroll
+    for (int i = 1; i < PER_LANE; ++i) {
       const int idx = lane + 32 * i;
-      gid_l[i] = W->gid[idx];
-      pid_l[i] = W->pair_id[idx];
-      pw_l[i] = W->pair_w[idx];
-      blob_l[i] = reinterpret_cast<const unsigned char*>(W->gblob[idx]);
+      bool mine = !have_list;
+      for (uint32_t look = 0; look < (1u << 22); ++look) {
+        if (!mine) {
+          if (idx < n_groups) gw[i] = dx_word_load(&W->group[idx]);
+          if (idx < n_pairs) pw[i] = dx_word_load(&W->pair[idx]);
+          mine = (idx >= n_groups || (gw[i] & DX_WORD_VALID)) && (idx >= n_pairs || (pw[i] & DX_WORD_VALID));
+        }
+        if (__all_sync(0xffffffffu, mine)) break;
+        if (look + 1 == (1u << 22)) have_list = false;
+      }
+    }
+    if (!have_list) {
+      n_groups = 0;
+      if (lane == 0) { *abort_flag = 1; atomicExch(p.dev_status, DX_DEV_WAIT_EXPIRED); }
     }
     int e_lo, e_hi, u_lo, u_hi;
     routed_range(n_groups, p, n_static, NS, s_lo, s_hi, e_lo, e_hi, u_lo, u_hi);
@@ -272,18 +289,18 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
 #pragma unroll
     for (int i = 0; i < PER_LANE; ++i) {
       const int idx = lane + 32 * i;
-      hdr->pair_id[idx] = pid_l[i];
-      hdr->pair_w[idx] = pw_l[i];
+      hdr->pair_id[idx] = idx < n_pairs ? dx_pair_id(pw[i]) : -1;
+      hdr->pair_w[idx] = idx < n_pairs ? dx_pair_weight(pw[i]) : 0.0f;
       if (idx < n_groups) {
-        const unsigned char* blob = blob_l[i];
+        const int gid = dx_group_id(gw[i]);
+        const unsigned char* blob = reinterpret_cast<const unsigned char*>(dx_group_blob(gw[i]));
         // without the hand-over the table may have changed since the routing kernel ran (experts staged by the
         // cache in between): read it now
-        if (!p.handover && gid_l[i] >= 0 && gid_l[i] < DX_MAX_E)
-          blob = reinterpret_cast<const unsigned char*>(p.table[p.n_shared + 1 + gid_l[i]]);
+        if (!p.handover && gid < DX_MAX_E) blob = reinterpret_cast<const unsigned char*>(p.table[p.n_shared + 1 + gid]);
         const int e = n_static + idx;
         hdr->e_begin[e] = unit_base + idx * p.routed_tiles;
         hdr->e_tiles[e] = p.routed_tiles;
-        hdr->e_gid[e] = gid_l[i];
+        hdr->e_gid[e] = gid;
         hdr->e_blob[e] = blob;
         if (blob == nullptr && e >= e_lo && e < e_hi) atomicExch(p.dev_status, DX_DEV_BAD_EXPERT_ID);
       }
@@ -542,9 +559,11 @@ __global__ void __launch_bounds__(256) dx_experts_fp32_kernel(DxExpertParams p) 
   __shared__ float s_rstd[DX_MAX_K];
   const DxWork* W = p.work;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  // (no early trigger: the kernel reads the work list until its last unit, and a routing kernel that follows may
+  // clear the list as soon as it starts)
   dx_pdl_wait();
-  dx_pdl_trigger();
-  const int n_groups = min(W->n_groups, DX_MAX_PAIRS), kk = W->k, H = p.H;
+  const unsigned long long head = W->head;
+  const int n_groups = min((int)(head & 0xffffu), DX_MAX_PAIRS), kk = (int)((head >> 16) & 0xffu), H = p.H;
   for (int r = warp; r < DX_MAX_K; r += 8) {
     float rs = 1.0f;
     if (p.rms_norm && r < p.K) {
@@ -578,7 +597,7 @@ __global__ void __launch_bounds__(256) dx_experts_fp32_kernel(DxExpertParams p) 
       w_static = p.gamma;
     } else {
       const int gi = (u - NS_all) / p.routed_tiles;
-      gid = W->gid[gi];
+      gid = dx_group_id(W->group[gi]);
       table_index = p.n_shared + 1 + gid;
       unit_begin = NS_all + gi * p.routed_tiles;
     }
@@ -589,7 +608,7 @@ __global__ void __launch_bounds__(256) dx_experts_fp32_kernel(DxExpertParams p) 
         if (gid < 0) w = w_static;
         else
           for (int j = 0; j < kk; ++j)
-            if (W->pair_id[row * kk + j] == gid) w = W->pair_w[row * kk + j];
+            if (dx_pair_id(W->pair[row * kk + j]) == gid) w = dx_pair_weight(W->pair[row * kk + j]);
       }
       s_roww[row] = w;
     }

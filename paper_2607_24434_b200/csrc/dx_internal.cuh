@@ -23,15 +23,43 @@
 // expert) follow from the launch parameters alone; the routed groups are listed here, one per expert that some
 // block row selected, in the order in which their work units are numbered.  A group's weight in block row t is
 // the gate weight of the pair (t, j) that selected its expert, or nothing if no pair of that row did.
+//
+// Every item is one 64-bit word that carries its own "valid" bit (bit 63), so a reader that runs concurrently
+// with the routing kernel polls the words themselves: no flag, no fence, no second round trip.  The routing
+// kernel of a fused pair zeroes all words before it lets its expert kernel start.
+//   head : valid | K << 24 | k << 16 | number of routed groups
+//   group: valid | expert id << 48 | (blob address >> 4), the blob as the layer's table had it at routing time
+//   pair : valid | expert id << 32 | gate weight bits, index t * k + j
 struct DxWork {
-  int32_t n_groups;                   // routed groups
-  int32_t K, k;                       // block rows and selected experts per row
-  int32_t pad;
-  int32_t gid[DX_MAX_PAIRS];          // expert id of group i
-  const void* gblob[DX_MAX_PAIRS];    // its blob as the layer's table had it when the routing kernel ran
-  int32_t pair_id[DX_MAX_PAIRS];      // [K,k] selected expert ids, row-major
-  float pair_w[DX_MAX_PAIRS];         // [K,k] their gate weights
+  unsigned long long head;
+  unsigned long long group[DX_MAX_PAIRS];
+  unsigned long long pair[DX_MAX_PAIRS];
 };
+#define DX_WORD_VALID (1ull << 63)
+__host__ __device__ inline unsigned long long dx_head_word(int K, int k, int n_groups) {
+  return DX_WORD_VALID | ((unsigned long long)K << 24) | ((unsigned long long)k << 16) | (unsigned long long)n_groups;
+}
+__host__ __device__ inline unsigned long long dx_group_word(int gid, const void* blob) {
+  return DX_WORD_VALID | ((unsigned long long)gid << 48) | ((unsigned long long)(uintptr_t)blob >> 4);
+}
+__host__ __device__ inline int dx_group_id(unsigned long long w) { return (int)((w >> 48) & 0x7fff); }
+__host__ __device__ inline const void* dx_group_blob(unsigned long long w) {
+  return (const void*)(uintptr_t)((w & 0xffffffffffffull) << 4);
+}
+__device__ __forceinline__ unsigned long long dx_pair_word(int id, float w) {
+  return DX_WORD_VALID | ((unsigned long long)id << 32) | (unsigned long long)__float_as_uint(w);
+}
+__device__ __forceinline__ int dx_pair_id(unsigned long long w) { return (int)((w >> 32) & 0x7fffffff); }
+__device__ __forceinline__ float dx_pair_weight(unsigned long long w) { return __uint_as_float((unsigned int)w); }
+// 8-byte accesses that go to the L2 (the point where concurrently running kernels meet)
+__device__ __forceinline__ void dx_word_store(unsigned long long* p, unsigned long long v) {
+  asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+__device__ __forceinline__ unsigned long long dx_word_load(const unsigned long long* p) {
+  unsigned long long v;
+  asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+  return v;
+}
 
 struct dx_ctx {
   int device;
@@ -45,7 +73,7 @@ struct dx_ctx {
   unsigned int* ticket;        // last-CTA tickets (route, accept)
   unsigned long long* keys;    // [DX_MAX_M] packed argmax keys
   int32_t* dev_status;
-  unsigned int* handover;      // device words {block input final, work list complete}: see DxExpertParams
+  unsigned int* handover;      // device word {block input final}: see DxExpertParams
   float2* conf_part;           // [8 * sm_count][DX_MAX_M] per-CTA online-softmax pairs of the confidence variant
   int32_t* scratch_i32;        // two ints the draft-token entry point parks unused outputs in
 };
@@ -79,9 +107,9 @@ struct DxRouteParams {
   int top_r;
   int rms_norm;     // 1: route and experts see RMSNorm(h)
   int residual;     // 0: y starts at zero, 1: y starts as a copy of h (pre-norm residual form)
-  int tok_group;    // block rows staged in shared memory per pass (set by the launcher)
-  unsigned int* handover; // not null: set word 0 once everything in front of this kernel in the stream has
-                          // completed, and word 1 once the work list is complete
+  unsigned int* handover; // not null: the expert kernel of this call runs concurrently (fused entry points): zero
+                          // the hand-over words first, and set this word once everything in front of this
+                          // kernel in the stream has completed
   float* y;
   float* z;
   unsigned int* ticket;
@@ -112,9 +140,9 @@ struct DxExpertParams {
   int first_routed, n_routed, do_static;
   // Hand-over from the routing kernel launched right before this one (fused entry points only; null otherwise,
   // and then the kernel simply waits for everything in front of it).  With the hand-over this kernel may be running
-  // before its inputs are final: consumers read the block only once word 0 is set, and the routed groups are
-  // read only once word 1 is set.  The routing kernel of the next pair clears both words before it lets its own
-  // expert kernel start; this kernel in turn lets that routing kernel start only when it is past both words.
+  // before its inputs are final: consumers read the block only once this word is set, and the routed groups are
+  // polled out of the work list.  The routing kernel of the next pair clears the word and the list before it lets
+  // its own expert kernel start; this kernel in turn lets that routing kernel start only when it is past both.
   unsigned int* handover;
 };
 
