@@ -138,6 +138,7 @@ struct SmemHeader {
   int e_gid[DX_MAX_ENTRIES];         // expert id of a routed group
   const unsigned char* e_blob[DX_MAX_ENTRIES];
   int kk;                            // selected experts per block row
+  int n_pairs;                       // K * kk
   int pair_id[DX_MAX_PAIRS];         // [K,kk] selected expert ids and gate weights of the block
   float pair_w[DX_MAX_PAIRS];
 };
@@ -157,17 +158,19 @@ __device__ __forceinline__ void routed_range(int n_groups, const DxExpertParams&
   e_lo = n_static + g_lo;
   e_hi = n_static + g_hi;
   if (g_lo >= g_hi) { u_lo = u_hi = 0; return; }
-  const long long base = (long long)p.n_shared * p.shared_tiles + p.draft_tiles;
-  const long long R0 = base + (long long)g_lo * p.routed_tiles;
-  const long long NR = (long long)(g_hi - g_lo) * p.routed_tiles, T = NSe + NR;
-  long long a, b;
-  if (T / G >= (NSe + G - 1) / G) {   // keep routing-independent + routed units balanced together
-    a = (T * cta) / G - s_lo; b = (T * (cta + 1)) / G - s_hi;
+  // (unit counts are a few ten thousand at most, grids a few hundred CTAs: the products fit 32 bits)
+  const unsigned int base = (unsigned int)(p.n_shared * p.shared_tiles + p.draft_tiles);
+  const unsigned int R0 = base + (unsigned int)(g_lo * p.routed_tiles);
+  const unsigned int NR = (unsigned int)((g_hi - g_lo) * p.routed_tiles), T = (unsigned int)NSe + NR;
+  const unsigned int uG = (unsigned int)G, ucta = (unsigned int)cta;
+  int a, b;
+  if (T / uG >= ((unsigned int)NSe + uG - 1u) / uG) {   // keep routing-independent + routed units balanced together
+    a = (int)((T * ucta) / uG) - s_lo; b = (int)((T * (ucta + 1u)) / uG) - s_hi;
   } else {
-    a = (NR * cta) / G; b = (NR * (cta + 1)) / G;
+    a = (int)((NR * ucta) / uG); b = (int)((NR * (ucta + 1u)) / uG);
   }
-  u_lo = (int)(R0 + a);
-  u_hi = (int)(R0 + b);
+  u_lo = (int)R0 + a;
+  u_hi = (int)R0 + b;
 }
 
 template <int H, int NT>
@@ -246,34 +249,32 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
     // and the first look succeeds.
     if (!p.handover) pdl_wait();
     constexpr int PER_LANE = DX_MAX_PAIRS / 32;
-    unsigned long long gw[PER_LANE], pw[PER_LANE];
+    unsigned long long gw[PER_LANE];
 #pragma unroll
-    for (int i = 0; i < PER_LANE; ++i) gw[i] = pw[i] = 0ull;
+    for (int i = 0; i < PER_LANE; ++i) gw[i] = 0ull;
     int n_groups = 0, kk = 1, n_pairs = 0;
     bool have_list = false;
     for (uint32_t look = 0; look < (1u << 22) && !have_list; ++look) {
       const unsigned long long head = dx_word_load(&W->head);
       gw[0] = dx_word_load(&W->group[lane]);
-      pw[0] = dx_word_load(&W->pair[lane]);
       bool mine = false;
       if (head & DX_WORD_VALID) {
         n_groups = min((int)(head & 0xffffu), DX_MAX_PAIRS);
         kk = (int)((head >> 16) & 0xffu);
         n_pairs = min((int)((head >> 24) & 0xffu) * kk, DX_MAX_PAIRS);
-        mine = (lane >= n_groups || (gw[0] & DX_WORD_VALID)) && (lane >= n_pairs || (pw[0] & DX_WORD_VALID));
+        mine = lane >= n_groups || (gw[0] & DX_WORD_VALID);
       }
       have_list = __all_sync(0xffffffffu, mine);
     }
-    // larger blocks: the words beyond the first 32 of each kind
+    // larger unions: the group words beyond the first 32
 #pragma unroll
     for (int i = 1; i < PER_LANE; ++i) {
       const int idx = lane + 32 * i;
-      bool mine = !have_list;
+      bool mine = !have_list || idx >= n_groups;
       for (uint32_t look = 0; look < (1u << 22); ++look) {
         if (!mine) {
-          if (idx < n_groups) gw[i] = dx_word_load(&W->group[idx]);
-          if (idx < n_pairs) pw[i] = dx_word_load(&W->pair[idx]);
-          mine = (idx >= n_groups || (gw[i] & DX_WORD_VALID)) && (idx >= n_pairs || (pw[i] & DX_WORD_VALID));
+          gw[i] = dx_word_load(&W->group[idx]);
+          mine = (gw[i] & DX_WORD_VALID) != 0;
         }
         if (__all_sync(0xffffffffu, mine)) break;
         if (look + 1 == (1u << 22)) have_list = false;
@@ -289,8 +290,6 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
 #pragma unroll
     for (int i = 0; i < PER_LANE; ++i) {
       const int idx = lane + 32 * i;
-      hdr->pair_id[idx] = idx < n_pairs ? dx_pair_id(pw[i]) : -1;
-      hdr->pair_w[idx] = idx < n_pairs ? dx_pair_weight(pw[i]) : 0.0f;
       if (idx < n_groups) {
         const int gid = dx_group_id(gw[i]);
         const unsigned char* blob = reinterpret_cast<const unsigned char*>(dx_group_blob(gw[i]));
@@ -307,6 +306,7 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
     }
     if (lane == 0) {
       hdr->kk = kk;
+      hdr->n_pairs = n_pairs;
       hdr->r_e_lo = e_lo; hdr->r_e_hi = e_hi; hdr->r_u_lo = u_lo; hdr->r_u_hi = u_hi;
     }
     __threadfence_block();   // bar.arrive alone does not order the shared-memory writes above
@@ -525,6 +525,25 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
   // Only now may the next kernel of the stream start: if it is a routing kernel it clears the hand-over words,
   // and this CTA is done with both of them.
   pdl_launch_dependents();
+  // The (row, expert, gate) pairs come out of the gate arithmetic a little after the group list.  Every warp
+  // fetches all of them for itself (same values from every warp, so no barrier is needed beyond its own).
+  {
+    const int n_pairs = hdr->n_pairs;
+    bool ok = true;
+    for (int idx = lane; idx < n_pairs; idx += 32) {
+      unsigned long long w = 0ull;
+      uint32_t look = 0;
+      for (; look < (1u << 22); ++look) {
+        w = dx_word_load(&W->pair[idx]);
+        if (w & DX_WORD_VALID) break;
+      }
+      ok = ok && look < (1u << 22);
+      hdr->pair_id[idx] = dx_pair_id(w);
+      hdr->pair_w[idx] = dx_pair_weight(w);
+    }
+    if (!ok) { *abort_flag = 1; atomicExch(p.dev_status, DX_DEV_WAIT_EXPIRED); }
+    __syncwarp();
+  }
   process(hdr->r_e_lo, hdr->r_e_hi, hdr->r_u_lo, hdr->r_u_hi);
   pdl_wait();  // the routing kernel (which initialised y) has completed as a whole
 

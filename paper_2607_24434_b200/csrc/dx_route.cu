@@ -2,17 +2,19 @@
 // g_{l,e} of Eq. 4), the block's expert union and the pair permutation grouped
 // by expert (Eq. 2 / Eq. 3), and the work list the expert kernels consume.
 //
-// One thread-block cluster of 8 CTAs does all of it.  Each CTA owns an eighth
-// of the router rows; a warp dots its row with every block row, reading both
-// straight from global memory with all loads of a slab in flight together
-// (the block rows are shared by the warps of a CTA through L1).  The logits
-// are written into CTA 0's shared memory through distributed shared memory,
-// so the hand-over is one hardware cluster barrier: no fences, tickets or
-// global round trips on the critical path.  CTA 0 then selects, one warp per
-// token, by ranking every logit against all others (no selection rounds),
-// builds the union as a bit mask, publishes the group list the expert kernel
-// is waiting for, and only then sorts the K*k (token, expert) pairs by expert
-// for the caller's outputs.
+// One thread-block cluster of 8 CTAs does all of it.  The contraction is split
+// over the hidden dimension: CTA c owns a slice of the columns (and, for narrow
+// layers, a share of the router rows).  Its part of the router matrix is a
+// constant and sits in registers before the previous kernel of the stream has
+// finished; once the block is final a thread needs two 16-byte loads per block
+// row and slab, so a single memory round trip separates "block ready" from the
+// arithmetic.  Partial logits go into CTA 0's shared memory through distributed
+// shared memory (one table per slice, summed in a fixed order, so the result
+// does not depend on timing); the hand-over is one hardware cluster barrier.
+// CTA 0 then selects, one warp per token, by ranking every logit against all
+// others (no selection rounds), builds the union as a bit mask, publishes the
+// group list the expert kernel is waiting for, and only then sorts the K*k
+// (token, expert) pairs by expert for the caller's outputs.
 #include <cooperative_groups.h>
 
 #include "dx_internal.cuh"
@@ -70,11 +72,8 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int* s_warp, int& tot
   return base + inc - v;
 }
 
-// Dot products of one router row with TG block rows, everything read straight from global memory: the lane owns
-// columns 256*c + 8*lane .. +7 of every 256-column chunk c, and NB chunks (one row slab and TG block-row slabs
-// each, row stride hs) are requested together before any of them is used.  The block rows are shared by all warps of the CTA
-// and come out of L1 after the first touch.  With `rms`, the sums of squares of the block rows ride along.
-constexpr int kTokGroup = 8;
+// Eight router columns as stored (bf16: one 16-byte load, fp32: two).
+constexpr int kRowsPerBatch = 8;   // router rows a warp carries through one pass over its slice
 template <typename WT> struct RowRaw;
 template <> struct RowRaw<__nv_bfloat16> {
   uint4 r;
@@ -91,95 +90,84 @@ template <> struct RowRaw<float> {
   }
 };
 
-template <typename WT, int TG>
-__device__ __forceinline__ void row_dots_direct(const WT* wrow, const float* h, int hs, int H, int kt, int lane, bool rms,
-                                                float (&acc)[kTokGroup], float (&ss)[kTokGroup]) {
-  constexpr int NB = TG >= 8 ? 2 : (TG >= 4 ? 4 : 8);
-  const int chunks = H / 256;
-  for (int c0 = 0; c0 < chunks; c0 += NB) {
-    RowRaw<WT> wr[NB];
-    float4 ha[NB][TG], hb[NB][TG];
+// Sum N = 8, 16 or 32 per-lane values across the warp so that lane j (< N) ends up with the total of value j:
+// each step halves the number of live values by exchanging the half the partner lane keeps (N - 1 shuffles
+// instead of 5 N), and the lanes that share j then fold their subtotals.
+template <int N>
+__device__ __forceinline__ float warp_transpose_sum(float (&v)[N], int lane) {
 #pragma unroll
-    for (int i = 0; i < NB; ++i) {
-      if (c0 + i < chunks) {
-        const int col = 256 * (c0 + i) + 8 * lane;
-        wr[i].load(wrow + col);
+  for (int o = N / 2; o >= 1; o >>= 1) {
+    const bool upper = (lane & o) != 0;
 #pragma unroll
-        for (int t = 0; t < TG; ++t) {
-          if (t < kt) {
-            ha[i][t] = *reinterpret_cast<const float4*>(h + (size_t)t * hs + col);
-            hb[i][t] = *reinterpret_cast<const float4*>(h + (size_t)t * hs + col + 4);
-          }
-        }
-      }
-    }
-#pragma unroll
-    for (int i = 0; i < NB; ++i) {
-      if (c0 + i < chunks) {
-        float wv[8];
-        wr[i].unpack(wv);
-#pragma unroll
-        for (int t = 0; t < TG; ++t) {
-          if (t < kt) {
-            const float4 a = ha[i][t], b = hb[i][t];
-            float s = acc[t];
-            s = fmaf(wv[0], a.x, s); s = fmaf(wv[1], a.y, s); s = fmaf(wv[2], a.z, s); s = fmaf(wv[3], a.w, s);
-            s = fmaf(wv[4], b.x, s); s = fmaf(wv[5], b.y, s); s = fmaf(wv[6], b.z, s); s = fmaf(wv[7], b.w, s);
-            acc[t] = s;
-            if (rms) {
-              float q = ss[t];
-              q = fmaf(a.x, a.x, q); q = fmaf(a.y, a.y, q); q = fmaf(a.z, a.z, q); q = fmaf(a.w, a.w, q);
-              q = fmaf(b.x, b.x, q); q = fmaf(b.y, b.y, q); q = fmaf(b.z, b.z, q); q = fmaf(b.w, b.w, q);
-              ss[t] = q;
-            }
-          }
-        }
-      }
+    for (int i = 0; i < o; ++i) {
+      const float keep = upper ? v[i + o] : v[i];
+      const float send = upper ? v[i] : v[i + o];
+      v[i] = keep + __shfl_xor_sync(0xffffffffu, send, o);
     }
   }
+  float r = v[0];
+#pragma unroll
+  for (int o = N; o < 32; o <<= 1) r += __shfl_xor_sync(0xffffffffu, r, o);
+  return r;
 }
 
-// Top-k of one token by one warp.  Every lane ranks its own logits against all E of them (rank = number of
-// logits that are larger, or equal with a lower expert id), so there are no selection rounds: the k logits of
-// rank < k are the selection, in order.  Then softmax / sigmoid scores of the selected experts and their gates.
+// Top-k, in two steps so that the expert ids (all the expert kernel's producers need) are out before the gate
+// arithmetic starts.  Selection of one token by one warp: k rounds of (lane-local best, warp maximum of the
+// orderable logit, lowest expert id among the lanes that hold it); NK = logits per lane.
 template <int NK>
-__device__ __forceinline__ void topk_token(const DxRouteParams& p, const float* s_z, int* s_ids, float* s_w,
-                                           unsigned int* s_mask, int* s_sel_e, float* s_sel_z, int tt, int lane) {
+__device__ __forceinline__ void topk_select(const DxRouteParams& p, const float* s_z, int* s_ids, unsigned int* s_mask,
+                                            float* s_sel_z, int tt, int lane) {
   const int E = p.E, k = p.k;
   const float* zrow = s_z + tt * E;
+  unsigned int key[NK];   // orderable logit; 0 = retired or out of range (a real logit never maps to 0)
   float zv[NK];
-  int rank[NK];
 #pragma unroll
   for (int j = 0; j < NK; ++j) {
     const int ee = lane + 32 * j;
     zv[j] = ee < E ? zrow[ee] : 0.f;
-    rank[j] = 0;
+    key[j] = ee < E ? dx_orderable(zv[j]) : 0u;
+    if (ee < E && key[j] == 0u) key[j] = 1u;   // (only a NaN pattern maps to 0; keep it selectable)
   }
-  for (int o = 0; o < E; ++o) {
-    const float zo = zrow[o];
-#pragma unroll
-    for (int j = 0; j < NK; ++j) {
-      const int ee = lane + 32 * j;
-      rank[j] += (zo > zv[j]) || (zo == zv[j] && o < ee);
-    }
-  }
-#pragma unroll
-  for (int j = 0; j < NK; ++j) {
-    const int ee = lane + 32 * j;
-    if (ee < E && rank[j] < k) { s_sel_e[tt * DX_MAX_TOPK + rank[j]] = ee; s_sel_z[tt * DX_MAX_TOPK + rank[j]] = zv[j]; }
-  }
-  __syncwarp();
-  const float zmax = s_sel_z[tt * DX_MAX_TOPK];
   int my_e = 0;
   float my_z = 0.f;
-  if (lane < k) { my_e = s_sel_e[tt * DX_MAX_TOPK + lane]; my_z = s_sel_z[tt * DX_MAX_TOPK + lane]; }
-  my_e = min(max(my_e, 0), E - 1);   // whatever the logits were (NaNs rank nowhere), stay in range
+  for (int r = 0; r < k; ++r) {
+    unsigned int lbest = 0u, lid = 0xffffffffu;
+#pragma unroll
+    for (int j = 0; j < NK; ++j)
+      if (key[j] > lbest) { lbest = key[j]; lid = (unsigned int)(lane + 32 * j); }
+    const unsigned int wbest = __reduce_max_sync(0xffffffffu, lbest);
+    const int be = (int)__reduce_min_sync(0xffffffffu, lbest == wbest ? lid : 0xffffffffu);
+    // the owning lane publishes the logit and retires the key
+    float bz = 0.f;
+#pragma unroll
+    for (int j = 0; j < NK; ++j)
+      if (lane + 32 * j == be) { bz = zv[j]; key[j] = 0u; }
+    bz = __shfl_sync(0xffffffffu, bz, be & 31);
+    if (lane == r) { my_e = be; my_z = bz; }
+  }
+  if (lane < k) {
+    my_e = min(max(my_e, 0), E - 1);   // whatever the logits were, stay in range
+    s_sel_z[tt * DX_MAX_TOPK + lane] = my_z;
+    s_ids[tt * k + lane] = my_e;
+    atomicOr(&s_mask[my_e >> 5], 1u << (my_e & 31));   // union of Eq. 2 / Eq. 3 as a bit mask
+    if (p.topk_ids) p.topk_ids[tt * k + lane] = my_e;
+  }
+}
+
+// Softmax / sigmoid scores of the selected experts and their gate weights (the g_{l,e} of Eq. 4).
+template <int NK>
+__device__ __forceinline__ void topk_gates(const DxRouteParams& p, const float* s_z, const int* s_ids, float* s_w,
+                                           const float* s_sel_z, int tt, int lane) {
+  const int E = p.E, k = p.k;
+  const float* zrow = s_z + tt * E;
+  const float zmax = s_sel_z[tt * DX_MAX_TOPK];
+  const float my_z = lane < k ? s_sel_z[tt * DX_MAX_TOPK + lane] : 0.f;
   float psel;
   if (p.score_fn == DX_SCORE_SOFTMAX) {
     float s = 0.f;
 #pragma unroll
     for (int j = 0; j < NK; ++j)
-      if (lane + 32 * j < E) s += expf(zv[j] - zmax);
+      if (lane + 32 * j < E) s += expf(zrow[lane + 32 * j] - zmax);
     s = warp_sum(s);
     psel = expf(my_z - zmax) / s;
   } else {
@@ -190,20 +178,40 @@ __device__ __forceinline__ void topk_token(const DxRouteParams& p, const float* 
   float g = p.norm_topk ? psel / denom : psel;
   g *= p.scale;
   if (lane < k) {
-    s_ids[tt * k + lane] = my_e;
     s_w[tt * k + lane] = g;
-    atomicOr(&s_mask[my_e >> 5], 1u << (my_e & 31));   // union of Eq. 2 / Eq. 3 as a bit mask
-    dx_word_store(&p.work->pair[tt * k + lane], dx_pair_word(my_e, g));   // what the expert kernel waits for
-    if (p.topk_ids) p.topk_ids[tt * k + lane] = my_e;
+    dx_word_store(&p.work->pair[tt * k + lane], dx_pair_word(s_ids[tt * k + lane], g));   // for the consumers
     if (p.topk_w) p.topk_w[tt * k + lane] = g;
   }
 }
 
-// TG: block rows per pass of the logits phase (1, 2, 4 or 8; the launcher picks the smallest that covers K, or 8)
+// How the cluster divides the contraction: S column slices (the largest divisor of H/256 that is at most 8) of C
+// 256-column slabs each, times R = 8 / S shares of the router rows.
+struct RouteSplit {
+  int S, R, C, slice, share, e_lo, e_hi;
+  bool idle;
+};
+__device__ __forceinline__ RouteSplit route_split(int H, int E, int crank) {
+  RouteSplit q;
+  const int slabs = H / 256;
+  q.S = 1;
+  for (int s = 2; s <= kRouteCluster; ++s)
+    if (slabs % s == 0) q.S = s;
+  q.R = kRouteCluster / q.S;
+  q.C = slabs / q.S;
+  q.idle = crank >= q.S * q.R;
+  q.slice = crank % q.S;
+  q.share = crank / q.S;
+  const int per = (E + q.R - 1) / q.R;
+  q.e_lo = min(E, q.share * per);
+  q.e_hi = q.idle ? q.e_lo : min(E, q.e_lo + per);
+  return q;
+}
+
+// TG: block rows per pass of the logits phase (1, 2 or 4; the launcher picks the smallest that covers K, or 4)
 template <typename WT, int TG>
 __global__ void __launch_bounds__(kRouteThreads) dx_route_kernel(DxRouteParams p) {
-  __shared__ float s_z[DX_MAX_K * DX_MAX_E];
-  __shared__ int s_sel_e[DX_MAX_K * DX_MAX_TOPK];
+  __shared__ __align__(16) float s_z[DX_MAX_K * DX_MAX_E];
+  __shared__ float s_bias[DX_MAX_E];
   __shared__ float s_sel_z[DX_MAX_K * DX_MAX_TOPK];
   __shared__ int s_ids[DX_MAX_PAIRS];
   __shared__ float s_w[DX_MAX_PAIRS];
@@ -211,20 +219,29 @@ __global__ void __launch_bounds__(kRouteThreads) dx_route_kernel(DxRouteParams p
   __shared__ int s_scan[kRouteWarps];
   __shared__ unsigned int s_mask[DX_MAX_E / 32];
   __shared__ const void* s_tab[DX_MAX_E];
+  extern __shared__ __align__(16) float s_part[];   // CTA 0: [S][K*E + K] partial logits and sums of squares
 
   cg::cluster_group cluster = cg::this_cluster();
   const int crank = (int)cluster.block_rank();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int K = p.K, E = p.E, k = p.k, H = p.H, P = K * k;
-  const int epc = (E + kRouteCluster - 1) / kRouteCluster;   // router rows per CTA
-  const int e_lo = crank * epc, e_hi = min(E, e_lo + epc);
-  // the router matrix is constant: pull this CTA's rows into L2 while the previous kernel of the stream drains
-  if (e_lo < e_hi) {
-    const char* wb = reinterpret_cast<const char*>(p.W_r) + (size_t)e_lo * H * sizeof(WT);
-    const size_t bytes = (size_t)(e_hi - e_lo) * H * sizeof(WT);
-    for (size_t o = (size_t)threadIdx.x * 128; o < bytes; o += (size_t)kRouteThreads * 128)
-      asm volatile("prefetch.global.L2 [%0];" ::"l"(wb + o));
+  const RouteSplit sp = route_split(H, E, crank);
+  const int part_stride = K * E + K;
+  const int col0 = sp.slice * sp.C * 256 + 8 * lane;   // this lane's first column; slab c adds 256 c
+  const WT* Wr = reinterpret_cast<const WT*>(p.W_r);
+
+  // the first batch of this warp's router rows (first slab of the slice): constant data, fetched right away
+  RowRaw<WT> wpre[kRowsPerBatch];
+#pragma unroll
+  for (int i = 0; i < kRowsPerBatch; ++i) {
+    const int e = sp.e_lo + warp + kRouteWarps * i;
+    if (e < sp.e_hi) wpre[i].load(Wr + (size_t)e * H + col0);
   }
+  if (crank == 0)
+    for (int e = threadIdx.x; e < E; e += kRouteThreads) s_bias[e] = p.bias ? p.bias[e] : 0.f;
+  for (int i = threadIdx.x; i < DX_MAX_K * DX_MAX_TOPK; i += kRouteThreads) s_sel_z[i] = 0.f;
+  for (int i = threadIdx.x; i < DX_MAX_PAIRS; i += kRouteThreads) s_ids[i] = 0;
+
   // Let the expert kernel be scheduled right away: its producers only touch constant weights, and its consumers
   // hold back until this kernel publishes that the block input is final.
   if (p.handover && crank == 0) {
@@ -237,124 +254,201 @@ __global__ void __launch_bounds__(kRouteThreads) dx_route_kernel(DxRouteParams p
     __syncthreads();
   }
   dx_pdl_trigger();
-  for (int i = threadIdx.x; i < DX_MAX_K * DX_MAX_TOPK; i += kRouteThreads) { s_sel_e[i] = 0; s_sel_z[i] = 0.f; }
+  // everything this kernel reads or writes from here on may have been in use by the previous kernel
+  dx_pdl_wait();
+  if (p.handover && crank == 0 && threadIdx.x == 0) {
+    __threadfence();
+    atomicExch(p.handover, 1u);
+  }
+  if (crank == 0) {
+    // routed part of the blob table, for the group list at the end; empty union mask
+    if (threadIdx.x < E) s_tab[threadIdx.x] = p.table[p.n_shared + 1 + threadIdx.x];
+    if (threadIdx.x < DX_MAX_E / 32) s_mask[threadIdx.x] = 0u;
+  }
 
-  float* z0 = cluster.map_shared_rank(s_z, 0);
+  // ---- partial logits of this CTA's slice, into CTA 0's table for the slice
+  float* part0 = cluster.map_shared_rank(s_part, 0) + (size_t)sp.slice * part_stride;
   const bool rms = p.rms_norm != 0;
-  const int me = threadIdx.x;
-  DxWork* W = p.work;
-  {
-    // everything this kernel reads or writes from here on may have been in use by the previous kernel
-    dx_pdl_wait();
-    if (p.handover && crank == 0 && threadIdx.x == 0) {
-      __threadfence();
-      atomicExch(p.handover, 1u);
-    }
-    if (crank == 0) {
-      // routed part of the blob table, for the group list at the end; empty union mask
-      if (threadIdx.x < E) s_tab[threadIdx.x] = p.table[p.n_shared + 1 + threadIdx.x];
-      if (threadIdx.x < DX_MAX_E / 32) s_mask[threadIdx.x] = 0u;
-    }
-    // router logits z[t,e], written into CTA 0's table through distributed shared memory
-    for (int t0 = 0; t0 < K; t0 += TG) {
-      const int kt = min(TG, K - t0);
-      const float* hb = p.h + (size_t)t0 * H;
-      const int hs = H;
-      for (int e = e_lo + warp; e < e_hi; e += kRouteWarps) {
-        const WT* wrow = reinterpret_cast<const WT*>(p.W_r) + (size_t)e * H;
-        const float b = p.bias ? p.bias[e] : 0.f;
-        float acc[kTokGroup], ss[kTokGroup];
+  for (int t0 = 0; t0 < K; t0 += TG) {
+    const int kt = min(TG, K - t0);
+    float ss[TG];
 #pragma unroll
-        for (int t = 0; t < kTokGroup; ++t) { acc[t] = 0.f; ss[t] = 0.f; }
-        row_dots_direct<WT, TG>(wrow, hb, hs, H, kt, lane, rms, acc, ss);
+    for (int t = 0; t < TG; ++t) ss[t] = 0.f;
+    for (int r0 = sp.e_lo + warp; r0 < sp.e_hi; r0 += kRouteWarps * kRowsPerBatch) {
+      float acc[kRowsPerBatch * TG];
+#pragma unroll
+      for (int i = 0; i < kRowsPerBatch * TG; ++i) acc[i] = 0.f;
+      const bool first_rows = r0 == sp.e_lo + warp;
+      for (int c = 0; c < sp.C; ++c) {
+        // the block rows' part of this slab: two 16-byte loads per row, all in flight together
+        float4 ha[TG], hb[TG];
 #pragma unroll
         for (int t = 0; t < TG; ++t) {
           if (t < kt) {
-            const float s = warp_sum(acc[t]);
-            const float rs = rms ? rsqrtf(warp_sum(ss[t]) / (float)H + 1e-6f) : 1.0f;
-            if (lane == 0) z0[(t0 + t) * E + e] = s * rs + b;
+            const float* hp = p.h + (size_t)(t0 + t) * H + col0 + 256 * c;
+            ha[t] = *reinterpret_cast<const float4*>(hp);
+            hb[t] = *reinterpret_cast<const float4*>(hp + 4);
+          } else {
+            ha[t] = hb[t] = make_float4(0.f, 0.f, 0.f, 0.f);
+          }
+        }
+        RowRaw<WT> wr[kRowsPerBatch];
+        const bool pre = first_rows && c == 0;
+#pragma unroll
+        for (int i = 0; i < kRowsPerBatch; ++i) {
+          const int e = r0 + kRouteWarps * i;
+          if (pre) wr[i] = wpre[i];
+          else if (e < sp.e_hi) wr[i].load(Wr + (size_t)e * H + col0 + 256 * c);
+        }
+        if (rms && first_rows && warp == 0 && sp.share == 0) {
+#pragma unroll
+          for (int t = 0; t < TG; ++t) {
+            float q = ss[t];
+            q = fmaf(ha[t].x, ha[t].x, q); q = fmaf(ha[t].y, ha[t].y, q); q = fmaf(ha[t].z, ha[t].z, q);
+            q = fmaf(ha[t].w, ha[t].w, q); q = fmaf(hb[t].x, hb[t].x, q); q = fmaf(hb[t].y, hb[t].y, q);
+            q = fmaf(hb[t].z, hb[t].z, q); q = fmaf(hb[t].w, hb[t].w, q);
+            ss[t] = q;
+          }
+        }
+#pragma unroll
+        for (int i = 0; i < kRowsPerBatch; ++i) {
+          if (r0 + kRouteWarps * i < sp.e_hi) {
+            float wv[8];
+            wr[i].unpack(wv);
+#pragma unroll
+            for (int t = 0; t < TG; ++t) {
+              float s = acc[i * TG + t];
+              s = fmaf(wv[0], ha[t].x, s); s = fmaf(wv[1], ha[t].y, s); s = fmaf(wv[2], ha[t].z, s);
+              s = fmaf(wv[3], ha[t].w, s); s = fmaf(wv[4], hb[t].x, s); s = fmaf(wv[5], hb[t].y, s);
+              s = fmaf(wv[6], hb[t].z, s); s = fmaf(wv[7], hb[t].w, s);
+              acc[i * TG + t] = s;
+            }
           }
         }
       }
+      // lane j now gets the warp total of (row r0 + 8 (j / TG), block row t0 + j % TG)
+      const float tot = warp_transpose_sum<kRowsPerBatch * TG>(acc, lane);
+      const int e = r0 + kRouteWarps * (lane / TG), t = lane % TG;
+      if (lane < kRowsPerBatch * TG && e < sp.e_hi && t < kt) part0[(t0 + t) * E + e] = tot;
     }
-    {
-      // y starts at zero, or as a copy of the block in the residual form; nothing reads it before this kernel
-      // is over
-      for (int j = (crank * kRouteThreads + threadIdx.x) * 4; j < K * H; j += kRouteCluster * kRouteThreads * 4) {
-        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (p.residual) v = *reinterpret_cast<const float4*>(p.h + j);
-        *reinterpret_cast<float4*>(p.y + j) = v;
+    if (rms && warp == 0 && sp.share == 0 && !sp.idle) {
+#pragma unroll
+      for (int t = 0; t < TG; ++t) {
+        const float q = warp_sum(ss[t]);
+        if (lane == 0 && t < kt) part0[K * E + t0 + t] = q;
       }
-    }
-    cluster.sync();          // all logits have landed in CTA 0
-    if (crank == 0) {
-      // top-k and gate weights, one warp per token (NK = logits per lane, a power of two covering E)
-      for (int tt = warp; tt < K; tt += kRouteWarps) {
-        if (E <= 32) topk_token<1>(p, s_z, s_ids, s_w, s_mask, s_sel_e, s_sel_z, tt, lane);
-        else if (E <= 64) topk_token<2>(p, s_z, s_ids, s_w, s_mask, s_sel_e, s_sel_z, tt, lane);
-        else if (E <= 128) topk_token<4>(p, s_z, s_ids, s_w, s_mask, s_sel_e, s_sel_z, tt, lane);
-        else topk_token<8>(p, s_z, s_ids, s_w, s_mask, s_sel_e, s_sel_z, tt, lane);
-      }
-      __syncthreads();
-
-      // ---- group list for the expert kernel (it is waiting for it); the caller's outputs come afterwards
-      int flag = 0, upos = 0, ucount = 0;
-      {
-        const unsigned int mine = me < E ? s_mask[me >> 5] : 0u;
-        flag = (mine >> (me & 31)) & 1u;
-        for (int w2 = 0; w2 < (E + 31) / 32; ++w2) {
-          const int c = __popc(s_mask[w2]);
-          ucount += c;
-          if (w2 < (me >> 5)) upos += c;
-        }
-        upos += __popc(mine & ((1u << (me & 31)) - 1u));
-      }
-      if (!p.draft_mode) {
-        if (flag) dx_word_store(&W->group[upos], dx_group_word(me, s_tab[me]));
-      } else if (me < p.top_r) {
-        dx_word_store(&W->group[me], dx_group_word(s_ids[me], s_tab[s_ids[me]]));
-      }
-      if (me == 0) dx_word_store(&W->head, dx_head_word(K, k, p.draft_mode ? p.top_r : ucount));
-
-      // ---- routing outputs for the caller: pairs sorted by expert (counting sort; thread e owns expert e)
-      int cnt = 0;
-      if (me < E) {
-#pragma unroll 8
-        for (int q = 0; q < P; ++q) cnt += (s_ids[q] == me);
-      }
-      int total;
-      const int off = block_exclusive_scan(cnt, s_scan, total);
-      if (me < E) {
-        int i = 0;
-        for (int q = 0; q < P; ++q)
-          if (s_ids[q] == me) s_perm[off + i++] = q;
-        if (p.offsets) p.offsets[me] = off;
-        if (flag && p.union_ids) p.union_ids[upos] = me;
-      }
-      if (me == 0) {
-        if (p.offsets) p.offsets[E] = P;
-        if (p.union_count) *p.union_count = ucount;
-      }
-      if (p.union_mask && me < (E + 63) / 64) {
-        const unsigned long long lo = s_mask[2 * me], hi = (2 * me + 1 < DX_MAX_E / 32) ? s_mask[2 * me + 1] : 0u;
-        p.union_mask[me] = lo | (hi << 32);
-      }
-      __syncthreads();
-      if (p.perm)
-        for (int q = me; q < P; q += kRouteThreads) p.perm[q] = s_perm[q];
     }
   }
+  // y starts at zero, or as a copy of the block in the residual form; nothing reads it before this kernel is over
+  for (int j = (crank * kRouteThreads + threadIdx.x) * 4; j < K * H; j += kRouteCluster * kRouteThreads * 4) {
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (p.residual) v = *reinterpret_cast<const float4*>(p.h + j);
+    *reinterpret_cast<float4*>(p.y + j) = v;
+  }
+  cluster.sync();          // all partial logits have landed in CTA 0
+  if (crank != 0) return;
+
+  // logits: slices summed in a fixed order, RMSNorm scale and bias applied
+  for (int idx = threadIdx.x; idx < K * E; idx += kRouteThreads) {
+    const int t = idx / E, e = idx - t * E;
+    float z = 0.f, q = 0.f;
+#pragma unroll 8
+    for (int s2 = 0; s2 < sp.S; ++s2) {
+      z += s_part[s2 * part_stride + idx];
+      if (rms) q += s_part[s2 * part_stride + K * E + t];
+    }
+    const float rs = rms ? rsqrtf(q / (float)H + 1e-6f) : 1.0f;
+    s_z[idx] = z * rs + s_bias[e];
+  }
+  __syncthreads();
+
+  // selection, one warp per token
+  for (int tt = warp; tt < K; tt += kRouteWarps) {
+    if (E <= 32) topk_select<1>(p, s_z, s_ids, s_mask, s_sel_z, tt, lane);
+    else if (E <= 64) topk_select<2>(p, s_z, s_ids, s_mask, s_sel_z, tt, lane);
+    else if (E <= 128) topk_select<4>(p, s_z, s_ids, s_mask, s_sel_z, tt, lane);
+    else topk_select<8>(p, s_z, s_ids, s_mask, s_sel_z, tt, lane);
+  }
+  __syncthreads();
+
+  // ---- group list for the expert kernel (it is waiting for it); the caller's outputs come afterwards
+  const int me = threadIdx.x;
+  DxWork* W = p.work;
+  int flag = 0, upos = 0, ucount = 0;
+  {
+    const unsigned int mine = me < E ? s_mask[me >> 5] : 0u;
+    flag = (mine >> (me & 31)) & 1u;
+    for (int w2 = 0; w2 < (E + 31) / 32; ++w2) {
+      const int c = __popc(s_mask[w2]);
+      ucount += c;
+      if (w2 < (me >> 5)) upos += c;
+    }
+    upos += __popc(mine & ((1u << (me & 31)) - 1u));
+  }
+  if (!p.draft_mode) {
+    if (flag) dx_word_store(&W->group[upos], dx_group_word(me, s_tab[me]));
+  } else if (me < p.top_r) {
+    dx_word_store(&W->group[me], dx_group_word(s_ids[me], s_tab[s_ids[me]]));
+  }
+  if (me == 0) dx_word_store(&W->head, dx_head_word(K, k, p.draft_mode ? p.top_r : ucount));
+
+  // ---- gate weights: the expert kernel's consumers pick the pairs up when they reach the first routed group
+  for (int tt = warp; tt < K; tt += kRouteWarps) {
+    if (E <= 32) topk_gates<1>(p, s_z, s_ids, s_w, s_sel_z, tt, lane);
+    else if (E <= 64) topk_gates<2>(p, s_z, s_ids, s_w, s_sel_z, tt, lane);
+    else if (E <= 128) topk_gates<4>(p, s_z, s_ids, s_w, s_sel_z, tt, lane);
+    else topk_gates<8>(p, s_z, s_ids, s_w, s_sel_z, tt, lane);
+  }
+
+  // ---- routing outputs for the caller: pairs sorted by expert (counting sort; thread e owns expert e)
+  int cnt = 0;
+  if (me < E) {
+#pragma unroll 8
+    for (int q = 0; q < P; ++q) cnt += (s_ids[q] == me);
+  }
+  int total;
+  const int off = block_exclusive_scan(cnt, s_scan, total);
+  if (me < E) {
+    int i = 0;
+    for (int q = 0; q < P; ++q)
+      if (s_ids[q] == me) s_perm[off + i++] = q;
+    if (p.offsets) p.offsets[me] = off;
+    if (flag && p.union_ids) p.union_ids[upos] = me;
+  }
+  if (me == 0) {
+    if (p.offsets) p.offsets[E] = P;
+    if (p.union_count) *p.union_count = ucount;
+  }
+  if (p.union_mask && me < (E + 63) / 64) {
+    const unsigned long long lo = s_mask[2 * me], hi = (2 * me + 1 < DX_MAX_E / 32) ? s_mask[2 * me + 1] : 0u;
+    p.union_mask[me] = lo | (hi << 32);
+  }
+  __syncthreads();
+  if (p.perm)
+    for (int q = me; q < P; q += kRouteThreads) p.perm[q] = s_perm[q];
 }
 
 }  // namespace
 
+template <typename WT, int TG>
+static cudaError_t launch_route_one(const DxRouteParams& p, cudaStream_t st) {
+  // CTA 0 holds one partial table per column slice (at most 8)
+  const size_t smem = (size_t)kRouteCluster * ((size_t)p.K * p.E + p.K) * sizeof(float);
+  static size_t allowed = 48 * 1024;   // per instantiation: raise the opt-in limit only when a launch needs it
+  if (smem > allowed) {
+    cudaError_t e = cudaFuncSetAttribute(dx_route_kernel<WT, TG>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    allowed = smem;
+  }
+  return dx_launch_pdl(DX_PDL_ROUTE, dx_route_kernel<WT, TG>, dim3(kRouteCluster), dim3(kRouteThreads), smem, st,
+                       kRouteCluster, p);
+}
+
 template <typename WT>
 static cudaError_t launch_route_tg(const DxRouteParams& p, cudaStream_t st) {
-  const dim3 grid(kRouteCluster), block(kRouteThreads);
-  if (p.K <= 1) return dx_launch_pdl(DX_PDL_ROUTE, dx_route_kernel<WT, 1>, grid, block, 0, st, kRouteCluster, p);
-  if (p.K <= 2) return dx_launch_pdl(DX_PDL_ROUTE, dx_route_kernel<WT, 2>, grid, block, 0, st, kRouteCluster, p);
-  if (p.K <= 4) return dx_launch_pdl(DX_PDL_ROUTE, dx_route_kernel<WT, 4>, grid, block, 0, st, kRouteCluster, p);
-  return dx_launch_pdl(DX_PDL_ROUTE, dx_route_kernel<WT, 8>, grid, block, 0, st, kRouteCluster, p);
+  if (p.K <= 1) return launch_route_one<WT, 1>(p, st);
+  if (p.K <= 2) return launch_route_one<WT, 2>(p, st);
+  return launch_route_one<WT, 4>(p, st);
 }
 
 cudaError_t dx_launch_route(const DxRouteParams& p, int weight_dtype, cudaStream_t st) {
