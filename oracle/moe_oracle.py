@@ -177,6 +177,50 @@ def missing_residual(h: np.ndarray, layer: Dict[str, object], dtype=np.float64) 
     return y_star - y_top1
 
 
+def draft_expert_term(h: np.ndarray, layer: Dict[str, object], dtype=np.float64, gamma: Optional[float] = None):
+    """gamma_l * E^d_l(h_t) for every row -- the left operand of Eq. 7."""
+    sh = layer["shape"]
+    gam = sh.draft_gamma if gamma is None else gamma
+    h = np.asarray(h, dtype)
+    Wg, Wu, Wd = layer["draft"]
+    return np.stack([gam * swiglu_expert(h[t], Wg, Wu, Wd, dtype) for t in range(h.shape[0])])
+
+
+def residual_loss(h_draft: np.ndarray, h_star: np.ndarray, layer: Dict[str, object], dtype=np.float64) -> float:
+    """One layer's term of L_res (Eq. 7): sum_t || gamma E^d(h^d_t) - m*_t ||_2^2, the draft expert evaluated on
+    the drafter's hidden states and the missing residual (Eq. 6) on the teacher-forced ones."""
+    d = draft_expert_term(h_draft, layer, dtype) - missing_residual(h_star, layer, dtype)
+    return float((d * d).sum())
+
+
+def router_distribution(z: np.ndarray, score_fn: int) -> np.ndarray:
+    """R_l(h) as a distribution over the experts: the softmax itself, or -- for sigmoid routers, whose scores do
+    not sum to one -- the scores divided by their sum (a reading: Eq. 10 takes a KL between two R_l)."""
+    p = router_probs(z, score_fn)
+    if score_fn == SCORE_SIGMOID:
+        p = p / p.sum(axis=-1, keepdims=True)
+    return p
+
+
+def router_agreement(h_star: np.ndarray, h_draft: np.ndarray, layer: Dict[str, object], dtype=np.float64):
+    """Per row: KL( R_l(h*_t) || R_l(h^d_t) ), whose sum over rows and layers is L_router (Eq. 10), and the
+    number of experts that TopK_l(h*_t) and TopK_l(h^d_t) have in common (the top-k set agreement that Sec. 3.3
+    tracks as a validation metric).  Also returns the two selections."""
+    sh = layer["shape"]
+    zs = router_logits(h_star, layer["router"], layer["bias"], dtype)
+    zd = router_logits(h_draft, layer["router"], layer["bias"], dtype)
+    ps, pd = router_distribution(zs, sh.score_fn), router_distribution(zd, sh.score_fn)
+    kl = np.zeros(zs.shape[0], dtype)
+    for t in range(zs.shape[0]):
+        for e in range(zs.shape[1]):
+            if ps[t, e] > 0.0:
+                kl[t] += ps[t, e] * (np.log(ps[t, e]) - np.log(pd[t, e]))
+    ids_s = topk_select(router_probs(zs, sh.score_fn), sh.top_k)
+    ids_d = topk_select(router_probs(zd, sh.score_fn), sh.top_k)
+    agree = np.array([len(set(ids_s[t].tolist()) & set(ids_d[t].tolist())) for t in range(zs.shape[0])], np.int32)
+    return kl, agree, ids_s, ids_d
+
+
 # --------------------------------------------------------------------------
 # Eq. 2 / Eq. 3: the block's expert set and the pair permutation grouped by expert.
 # --------------------------------------------------------------------------

@@ -225,6 +225,69 @@ def test_draft_identities():
     assert np.allclose(O.moe_draft(h, L, gamma=0.0, top_r=sh.top_k)[0], y_star, rtol=1e-13)
 
 
+# ------------------------------------------------------ Sec. 3.3: evaluation terms (Eq. 6, 7, 10)
+def test_router_agreement_closed_forms():
+    TINY = synth.shape_tiny()
+    sh = dataclasses.replace(TINY, n_experts=2, top_k=1)
+    L = synth.layer_to_numpy(synth.make_layer(sh, 21, "cpu"))
+    # two experts, softmax: R = (s, 1 - s) with s = sigmoid(z0 - z1); KL of two Bernoullis in closed form
+    rng = np.random.default_rng(22)
+    hs, hd = rng.standard_normal((3, sh.hidden)), rng.standard_normal((3, sh.hidden))
+    kl, agree, ids_s, ids_d = O.router_agreement(hs, hd, L)
+    zs, zd = O.router_logits(hs, L["router"], L["bias"]), O.router_logits(hd, L["router"], L["bias"])
+    for t in range(3):
+        a = 1.0 / (1.0 + math.exp(-(zs[t, 0] - zs[t, 1])))
+        b = 1.0 / (1.0 + math.exp(-(zd[t, 0] - zd[t, 1])))
+        want = a * math.log(a / b) + (1 - a) * math.log((1 - a) / (1 - b))
+        assert abs(kl[t] - want) <= 1e-12 * max(1.0, abs(want))
+        assert agree[t] == int((zs[t, 0] >= zs[t, 1]) == (zd[t, 0] >= zd[t, 1]))
+    # identical hidden states: zero divergence, full agreement; KL is never negative and is not symmetric
+    sh6 = TINY
+    L6 = synth.layer_to_numpy(synth.make_layer(sh6, 23, "cpu"))
+    h = rng.standard_normal((4, sh6.hidden))
+    kl0, ag0, _, _ = O.router_agreement(h, h, L6)
+    assert np.all(np.abs(kl0) <= 1e-15) and np.all(ag0 == sh6.top_k)
+    h2 = h + 0.5 * rng.standard_normal(h.shape)
+    kl_ab, ag_ab, ia, ib = O.router_agreement(h, h2, L6)
+    kl_ba, ag_ba, _, _ = O.router_agreement(h2, h, L6)
+    assert np.all(kl_ab >= 0) and np.all(kl_ba >= 0) and not np.allclose(kl_ab, kl_ba)
+    assert np.array_equal(ag_ab, ag_ba) and np.all(ag_ab <= sh6.top_k)
+    for t in range(4):
+        assert ag_ab[t] == len(np.intersect1d(ia[t], ib[t]))
+    # against the library routine on the same distributions
+    from scipy.special import rel_entr, softmax
+    za = O.router_logits(h, L6["router"], L6["bias"]); zb = O.router_logits(h2, L6["router"], L6["bias"])
+    assert np.allclose(kl_ab, rel_entr(softmax(za, axis=1), softmax(zb, axis=1)).sum(axis=1), rtol=1e-10, atol=1e-14)
+    # sigmoid routers: scores normalised to a distribution first (the reading), so scaling has no effect
+    Ls = dict(L6); Ls["shape"] = dataclasses.replace(sh6, score_fn=synth.SCORE_SIGMOID)
+    kls, _, _, _ = O.router_agreement(h, h2, Ls)
+    pa = 1 / (1 + np.exp(-za)); pb = 1 / (1 + np.exp(-zb))
+    assert np.allclose(kls, rel_entr(pa / pa.sum(1, keepdims=True), pb / pb.sum(1, keepdims=True)).sum(axis=1),
+                       rtol=1e-10, atol=1e-14)
+
+
+def test_residual_loss_identities():
+    TINY = synth.shape_tiny()
+    sh = TINY
+    L = synth.layer_to_numpy(synth.make_layer(sh, 24, "cpu"))
+    rng = np.random.default_rng(25)
+    h = rng.standard_normal((3, sh.hidden))
+    # Eq. 7 with gamma = 0 is the squared norm of the missing residual; it is quadratic in gamma in general
+    m = O.missing_residual(h, L)
+    L0 = dict(L); L0["shape"] = dataclasses.replace(sh, draft_gamma=0.0)
+    assert abs(O.residual_loss(h, h, L0) - float((m * m).sum())) <= 1e-12 * float((m * m).sum())
+    d = np.stack([O.swiglu_expert(h[t], *L["draft"]) for t in range(3)])
+    for gam in (0.5, 1.0, -2.0):
+        Lg = dict(L); Lg["shape"] = dataclasses.replace(sh, draft_gamma=gam)
+        want = float(((gam * d - m) ** 2).sum())
+        assert abs(O.residual_loss(h, h, Lg) - want) <= 1e-12 * want
+        assert np.allclose(O.draft_expert_term(h, Lg), gam * d, rtol=1e-13)
+    # a draft expert that reproduces the residual exactly has zero loss: y_d == y* then (Eq. 5 vs Eq. 4)
+    y_star = O.moe_target(h, L)[0]
+    y_top1 = O.moe_draft(h, L, gamma=0.0)[0]
+    assert np.allclose(y_top1 + m, y_star, rtol=1e-12, atol=1e-14)
+
+
 # ------------------------------------------------------ union (Eq. 2, Eq. 3)
 def test_block_union_enumeration_and_invariants():
     rng = np.random.default_rng(6)
