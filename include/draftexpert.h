@@ -218,6 +218,28 @@ dx_status dx_controller_propose(dx_controller* c, const int32_t* predicted, int3
                                 int32_t budget, int32_t* delta_out, int32_t* stop_out, int32_t* new_layers_out,
                                 int32_t* new_experts_out, int32_t* n_new_out);
 
+/* ---- evaluation terms of the self-distillation section (Sec. 3.3); forward only, nothing is trained ---------
+ * All pointers are device pointers; K block rows, 1 <= K <= 16; asynchronous on `stream`.
+ *
+ * moe_missing_residual: Eq. 6 for a block, m[t] = y*_t - S(h_t) - g_{t,e1} E_{e1}(h_t), evaluated as what it is
+ *   equal to: the routed sum of Eq. 4 over each row's selected experts except the first, with the gate weights
+ *   of the full top-k.  h [K,H] in, m [K,H] out (overwritten); topk_ids [K,k] / topk_w [K,k] optional outputs
+ *   (NULL to skip) as in moe_verify_block.  Every routed expert of the layer must be resident.
+ * moe_draft_expert_term: gamma * E^d(h_t) for every row, the left operand of Eq. 7.  out [K,H] overwritten.
+ *   DX_ERR_UNSUPPORTED for a layer without a draft expert.
+ * moe_router_agreement: per row t, kl[t] = KL( R(h*_t) || R(h^d_t) ) -- the summand of Eq. 10 -- and
+ *   agree[t] = | TopK(h*_t) & TopK(h^d_t) |, the top-k set agreement tracked beside it.  R is the router's softmax;
+ *   for sigmoid routers the scores are divided by their sum first (they are not a distribution otherwise).
+ *   h_star, h_draft [K,H]; kl [K] fp32 and agree [K] int32, either may be NULL.  Any K >= 1.
+ * dx_squared_error: out[0] = sum_i (a[i] - b[i])^2 over n floats in a fixed order -- with the two calls above,
+ *   one layer's term of Eq. 7. */
+dx_status moe_missing_residual(dx_layer* layer, const float* h, int32_t K, float* m, int32_t* topk_ids, float* topk_w,
+                               void* stream);
+dx_status moe_draft_expert_term(dx_layer* layer, const float* h, int32_t K, float* out, void* stream);
+dx_status moe_router_agreement(dx_layer* layer, const float* h_star, const float* h_draft, int32_t K, float* kl,
+                               int32_t* agree, void* stream);
+dx_status dx_squared_error(dx_ctx* ctx, const float* a, const float* b, int64_t n, float* out, void* stream);
+
 /* ---- greedy verification without any allocation ----------------------------------------------------------------
  * (No counterpart in the paper: an addition for callers of this library that cannot allocate device memory --
  * a serving thread whose memory pool was sized once at start-up and where a late cudaMalloc is forbidden or

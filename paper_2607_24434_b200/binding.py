@@ -81,6 +81,10 @@ SIGNATURES = {
     "dx_controller_propose": (_I, [_P, _P, _I, C.c_float, C.c_float, _I, C.POINTER(_I), C.POINTER(_I), _P, _P,
                                    C.POINTER(_I)]),
     "spec_accept_noalloc": (_I, [_P, _I, _P, _I, _I, _I, _P, _I, _I, _P, _P, _P, _P]),
+    "moe_missing_residual": (_I, [_P, _P, _I, _P, _P, _P, _P]),
+    "moe_draft_expert_term": (_I, [_P, _P, _I, _P, _P]),
+    "moe_router_agreement": (_I, [_P, _P, _P, _I, _P, _P, _P]),
+    "dx_squared_error": (_I, [_P, _P, _P, C.c_int64, _P, _P]),
     "expert_cache_create": (_I, [_P, _I, _I, _I, C.c_size_t, C.POINTER(_P)]),
     "expert_cache_destroy": (_I, [_P]),
     "expert_cache_register": (_I, [_P, _I, _I, _P]),
@@ -503,6 +507,42 @@ def spec_draft_token(ctx: Context, h: torch.Tensor, W_lm: torch.Tensor, rms_norm
     _check(ctx.lib.spec_draft_token(ctx.handle, _ptr(h), M, _ptr(W_lm), W_lm.shape[0], H, wd, 1 if rms_norm else 0,
                                     _ptr(token), _ptr(conf), _stream()), "spec_draft_token")
     return token, conf
+
+
+def moe_missing_residual(layer: Layer, h: torch.Tensor) -> Dict[str, torch.Tensor]:
+    """Eq. 6 for a block: m[t] = y*_t - S(h_t) - g_{t,e1} E_{e1}(h_t).  Returns m and the routing it used."""
+    K, sh = h.shape[0], layer.shape
+    out = {"m": torch.empty_like(h),
+           "topk_ids": torch.empty((K, sh.top_k), dtype=torch.int32, device=h.device),
+           "topk_w": torch.empty((K, sh.top_k), dtype=torch.float32, device=h.device)}
+    _check(layer.lib.moe_missing_residual(layer.handle, _ptr(h), K, _ptr(out["m"]), _ptr(out["topk_ids"]),
+                                          _ptr(out["topk_w"]), _stream()), "moe_missing_residual")
+    return out
+
+
+def moe_draft_expert_term(layer: Layer, h: torch.Tensor) -> torch.Tensor:
+    """gamma * E^d(h_t) for every row (left operand of Eq. 7)."""
+    out = torch.empty_like(h)
+    _check(layer.lib.moe_draft_expert_term(layer.handle, _ptr(h), h.shape[0], _ptr(out), _stream()),
+           "moe_draft_expert_term")
+    return out
+
+
+def moe_router_agreement(layer: Layer, h_star: torch.Tensor, h_draft: torch.Tensor):
+    """Per row: KL(R(h*) || R(h^d)) (summand of Eq. 10) and the size of the top-k sets' intersection."""
+    K = h_star.shape[0]
+    kl = torch.empty((K,), dtype=torch.float32, device=h_star.device)
+    agree = torch.empty((K,), dtype=torch.int32, device=h_star.device)
+    _check(layer.lib.moe_router_agreement(layer.handle, _ptr(h_star), _ptr(h_draft), K, _ptr(kl), _ptr(agree),
+                                          _stream()), "moe_router_agreement")
+    return kl, agree
+
+
+def squared_error(ctx: Context, a: torch.Tensor, b: torch.Tensor) -> torch.Tensor:
+    """sum (a - b)^2 (with moe_draft_expert_term and moe_missing_residual: one layer's term of Eq. 7)."""
+    out = torch.empty((1,), dtype=torch.float32, device=a.device)
+    _check(ctx.lib.dx_squared_error(ctx.handle, _ptr(a), _ptr(b), a.numel(), _ptr(out), _stream()), "dx_squared_error")
+    return out
 
 
 class Controller:

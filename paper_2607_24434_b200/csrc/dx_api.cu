@@ -220,7 +220,8 @@ struct RouteOut {
 };
 
 static dx_status do_route(dx_layer* L, const float* h, int K, float* y, const RouteOut& o, bool draft, bool residual,
-                          cudaStream_t st, int top_r = 1, bool use_draft_expert = true, bool paired = false) {
+                          cudaStream_t st, int top_r = 1, bool use_draft_expert = true, bool paired = false,
+                          bool skip_top1 = false) {
   dx_ctx* ctx = L->ctx;
   const dx_layer_desc& d = L->desc;
   if (!h || !y || h == y) return DX_ERR_INVALID_ARG;
@@ -229,7 +230,7 @@ static dx_status do_route(dx_layer* L, const float* h, int K, float* y, const Ro
   for (int s = 0; s < d.n_shared; ++s)
     if (!L->table_host[s]) return DX_ERR_NOT_RESIDENT;
   if (draft && use_draft_expert && d.draft_inter > 0 && !L->table_host[d.n_shared]) return DX_ERR_NOT_RESIDENT;
-  if (top_r < 1 || top_r > d.top_k) return DX_ERR_INVALID_ARG;
+  if (top_r < 0 || top_r > d.top_k) return DX_ERR_INVALID_ARG;
   if (((uintptr_t)h) % 16 || ((uintptr_t)y) % 16) return DX_ERR_INVALID_ARG;
   dx_status s = upload_table(L, st);
   if (s != DX_OK) return s;
@@ -243,6 +244,7 @@ static dx_status do_route(dx_layer* L, const float* h, int K, float* y, const Ro
   p.draft_tiles = draft && use_draft_expert ? d.draft_inter / DX_TILE_I : 0;
   p.draft_mode = draft ? 1 : 0;
   p.top_r = top_r;
+  p.skip_top1 = skip_top1 ? 1 : 0;
   p.rms_norm = residual ? 1 : 0;
   p.residual = residual ? 1 : 0;
   p.y = y; p.z = ctx->z; p.ticket = ctx->ticket; p.work = ctx->work; p.dev_status = ctx->dev_status;
@@ -257,7 +259,7 @@ static dx_status do_route(dx_layer* L, const float* h, int K, float* y, const Ro
 
 static dx_status do_experts(dx_layer* L, const float* h, int K, float* y, bool draft, bool residual,
                             cudaStream_t st, int first_routed = 0, int n_routed = -1, bool do_static = true,
-                            bool paired = false) {
+                            bool paired = false, bool skip_shared = false) {
   dx_ctx* ctx = L->ctx;
   const dx_layer_desc& d = L->desc;
   if (!h || !y || h == y) return DX_ERR_INVALID_ARG;
@@ -282,6 +284,7 @@ static dx_status do_experts(dx_layer* L, const float* h, int K, float* y, bool d
   p.first_routed = first_routed;
   p.n_routed = n_routed;
   p.do_static = do_static ? 1 : 0;
+  p.skip_shared = skip_shared ? 1 : 0;
   DX_CUDA(ctx, dx_launch_experts(ctx, p, L->desc.weight_dtype, K, st));
   ctx->launches++;
   if (L->cache) dx_cache_note_use(L->cache, L->cache_layer, st);
@@ -342,6 +345,7 @@ extern "C" dx_status moe_draft_step_topr(dx_layer* L, const float* h, float* y, 
   if (!L) return DX_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;
   RouteOut o{topk_ids, topk_w, nullptr, nullptr, nullptr, nullptr, nullptr};
+  if (top_r < 1) return DX_ERR_INVALID_ARG;
   return do_pair(L, h, 1, y, o, true, false, st, top_r, use_draft_expert != 0);
 }
 
@@ -373,6 +377,49 @@ extern "C" dx_status moe_verify_block_residual(dx_layer* L, const float* h_in, f
   cudaStream_t st = (cudaStream_t)stream;
   RouteOut o{topk_ids, topk_w, union_mask, union_ids, union_count, offsets, perm};
   return do_pair(L, h_in, K, h_out, o, false, true, st);
+}
+
+// ---- evaluation terms of Sec. 3.3 (no training involved) -----------------------------------------------------
+extern "C" dx_status moe_missing_residual(dx_layer* L, const float* h, int32_t K, float* m, int32_t* topk_ids,
+                                          float* topk_w, void* stream) {
+  if (!L) return DX_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  RouteOut o{topk_ids, topk_w, nullptr, nullptr, nullptr, nullptr, nullptr};
+  // Eq. 6 is the routed sum of Eq. 4 without each row's first selected expert: same kernels, that pair's weight
+  // set to zero (and its expert left out of the union unless another pair selects it), shared experts skipped
+  dx_status s = do_route(L, h, K, m, o, false, false, st, 1, true, false, true);
+  if (s != DX_OK) return s;
+  return do_experts(L, h, K, m, false, false, st, 0, -1, false);
+}
+
+extern "C" dx_status moe_draft_expert_term(dx_layer* L, const float* h, int32_t K, float* out, void* stream) {
+  if (!L) return DX_ERR_INVALID_ARG;
+  if (L->desc.draft_inter <= 0) return DX_ERR_UNSUPPORTED;
+  cudaStream_t st = (cudaStream_t)stream;
+  RouteOut o{nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
+  // gamma * E^d(h_t) for K rows: the drafter's kernels with no routed group and the shared experts skipped
+  dx_status s = do_route(L, h, K, out, o, true, false, st, 0, true);
+  if (s != DX_OK) return s;
+  return do_experts(L, h, K, out, true, false, st, 0, -1, true, false, true);
+}
+
+extern "C" dx_status moe_router_agreement(dx_layer* L, const float* h_star, const float* h_draft, int32_t K, float* kl,
+                                          int32_t* agree, void* stream) {
+  if (!L || !h_star || !h_draft || (!kl && !agree)) return DX_ERR_INVALID_ARG;
+  if (K < 1) return DX_ERR_SHAPE;
+  if (!L->W_r) return DX_ERR_NOT_RESIDENT;
+  DX_CUDA(L->ctx, dx_launch_router_agreement(L, h_star, h_draft, K, kl, agree, (cudaStream_t)stream));
+  L->ctx->launches++;
+  return DX_OK;
+}
+
+extern "C" dx_status dx_squared_error(dx_ctx* ctx, const float* a, const float* b, int64_t n, float* out,
+                                      void* stream) {
+  if (!ctx || !a || !b || !out) return DX_ERR_INVALID_ARG;
+  if (n < 0) return DX_ERR_SHAPE;
+  DX_CUDA(ctx, dx_launch_squared_error(a, b, (long long)n, out, (cudaStream_t)stream));
+  ctx->launches++;
+  return DX_OK;
 }
 
 extern "C" dx_status spec_accept(dx_ctx* ctx, const float* h, int32_t M, const void* W_lm, int32_t V, int32_t H,

@@ -196,8 +196,9 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
   const int G = gridDim.x, cta = blockIdx.x;
   // groups that do not depend on routing: shared experts, then (draft mode) the draft expert
   const int n_static = p.n_shared + (p.draft_tiles > 0 ? 1 : 0);
-  const int NS = p.do_static ? p.n_shared * p.shared_tiles + p.draft_tiles : 0;
-  const int s_lo = (int)(((long long)NS * cta) / G), s_hi = (int)(((long long)NS * (cta + 1)) / G);
+  const int S0 = p.skip_shared ? p.n_shared * p.shared_tiles : 0;   // first routing-independent unit evaluated
+  const int NS = p.do_static ? p.n_shared * p.shared_tiles + p.draft_tiles - S0 : 0;
+  const int s_lo = S0 + (int)(((long long)NS * cta) / G), s_hi = S0 + (int)(((long long)NS * (cta + 1)) / G);
   volatile int* abort_flag = &hdr->abort_flag;
 
   if (threadIdx.x == 0) {
@@ -285,7 +286,7 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
       if (lane == 0) { *abort_flag = 1; atomicExch(p.dev_status, DX_DEV_WAIT_EXPIRED); }
     }
     int e_lo, e_hi, u_lo, u_hi;
-    routed_range(n_groups, p, n_static, NS, s_lo, s_hi, e_lo, e_hi, u_lo, u_hi);
+    routed_range(n_groups, p, n_static, NS, s_lo - S0, s_hi - S0, e_lo, e_hi, u_lo, u_hi);
     const int unit_base = p.n_shared * p.shared_tiles + p.draft_tiles;
 #pragma unroll
     for (int i = 0; i < PER_LANE; ++i) {
@@ -603,7 +604,8 @@ __global__ void __launch_bounds__(256) dx_experts_fp32_kernel(DxExpertParams p) 
   const int total = NS_all + n_groups * p.routed_tiles;
   __shared__ float s_roww[DX_MAX_K];
   for (int u = blockIdx.x; u < total; u += gridDim.x) {
-    if (u < NS_all ? !p.do_static : (u < wu_lo || u >= wu_hi)) continue;
+    if (u < NS_all ? (!p.do_static || (p.skip_shared && u < p.n_shared * p.shared_tiles)) : (u < wu_lo || u >= wu_hi))
+      continue;
     // the group of this unit, its blob and its weight in every block row (0 = the row is not in the group)
     int table_index, unit_begin, gid = -1;
     float w_static = 1.0f;

@@ -104,7 +104,8 @@ struct DxRouteParams {
   const void* const* table;   // layer blob table (device)
   int n_shared, shared_tiles, routed_tiles, draft_tiles;
   int draft_mode;   // 0: verify block, 1: drafter (shared + draft expert + top_r routed)
-  int top_r;
+  int top_r;        // drafter: routed groups taken from the top of the selection (0 = none)
+  int skip_top1;    // verify: leave every row's first selected expert out (the missing residual of Eq. 6)
   int rms_norm;     // 1: route and experts see RMSNorm(h)
   int residual;     // 0: y starts at zero, 1: y starts as a copy of h (pre-norm residual form)
   unsigned int* handover; // not null: the expert kernel of this call runs concurrently (fused entry points): zero
@@ -138,6 +139,7 @@ struct DxExpertParams {
   // window of the routed entries this launch covers (position among them, count or -1 = all) and whether
   // the routing-independent groups are part of it; a cache-staged union is processed in several windows
   int first_routed, n_routed, do_static;
+  int skip_shared;           // 1: of the routing-independent groups only the draft expert is evaluated
   // Hand-over from the routing kernel launched right before this one (fused entry points only; null otherwise,
   // and then the kernel simply waits for everything in front of it).  With the hand-over this kernel may be running
   // before its inputs are final: consumers read the block only once this word is set, and the routed groups are
@@ -154,6 +156,9 @@ cudaError_t dx_launch_pack(int weight_dtype, int H, int I, const void* Wg, const
 cudaError_t dx_launch_accept(dx_ctx* ctx, const float* h, int M, const void* W_lm, int V, int H, int w_dtype,
                              const int32_t* draft, int K, int rms_norm, int32_t* target, int32_t* n_accept,
                              int32_t* next_token, float* conf, cudaStream_t st);
+cudaError_t dx_launch_router_agreement(const dx_layer* L, const float* h_star, const float* h_draft, int K, float* kl,
+                                       int32_t* agree, cudaStream_t st);
+cudaError_t dx_launch_squared_error(const float* a, const float* b, long long n, float* out, cudaStream_t st);
 cudaError_t dx_experts_prepare(dx_ctx* ctx);   // opt-in shared memory attributes, once per context
 
 // cache hooks used by the layer code

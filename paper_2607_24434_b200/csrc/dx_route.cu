@@ -149,7 +149,8 @@ __device__ __forceinline__ void topk_select(const DxRouteParams& p, const float*
     my_e = min(max(my_e, 0), E - 1);   // whatever the logits were, stay in range
     s_sel_z[tt * DX_MAX_TOPK + lane] = my_z;
     s_ids[tt * k + lane] = my_e;
-    atomicOr(&s_mask[my_e >> 5], 1u << (my_e & 31));   // union of Eq. 2 / Eq. 3 as a bit mask
+    if (!(p.skip_top1 && lane == 0))
+      atomicOr(&s_mask[my_e >> 5], 1u << (my_e & 31));   // union of Eq. 2 / Eq. 3 as a bit mask
     if (p.topk_ids) p.topk_ids[tt * k + lane] = my_e;
   }
 }
@@ -179,7 +180,8 @@ __device__ __forceinline__ void topk_gates(const DxRouteParams& p, const float* 
   g *= p.scale;
   if (lane < k) {
     s_w[tt * k + lane] = g;
-    dx_word_store(&p.work->pair[tt * k + lane], dx_pair_word(s_ids[tt * k + lane], g));   // for the consumers
+    // for the consumers (the missing residual of Eq. 6 leaves the first selected expert's term out)
+    dx_word_store(&p.work->pair[tt * k + lane], dx_pair_word(s_ids[tt * k + lane], (p.skip_top1 && lane == 0) ? 0.0f : g));
     if (p.topk_w) p.topk_w[tt * k + lane] = g;
   }
 }
