@@ -177,6 +177,25 @@ def missing_residual(h: np.ndarray, layer: Dict[str, object], dtype=np.float64) 
     return y_star - y_top1
 
 
+def dequantize_q4_0(blocks: np.ndarray, dtype=np.float64) -> np.ndarray:
+    """Values of 4-bit block-quantised weights (the format of the paper's mobile runs, Sec. 4): ``blocks`` is
+    uint8 [R, C/32, 18]; bytes 0..1 of a block are the fp16 scale d (little endian), byte 2 + j holds the code of
+    weight j in its low nibble and of weight 16 + j in its high nibble; the weight is d * (code - 8).  Plain
+    loops over the block structure; returns [R, C]."""
+    blocks = np.asarray(blocks, np.uint8)
+    R, nb, nbytes = blocks.shape
+    assert nbytes == 18
+    out = np.zeros((R, nb * 32), dtype)
+    for r in range(R):
+        for b in range(nb):
+            blk = blocks[r, b]
+            d = dtype(np.frombuffer(blk[0:2].tobytes(), dtype="<f2")[0])
+            for j in range(16):
+                out[r, 32 * b + j] = d * (int(blk[2 + j] & 0x0F) - 8)
+                out[r, 32 * b + 16 + j] = d * (int(blk[2 + j] >> 4) - 8)
+    return out
+
+
 def draft_expert_term(h: np.ndarray, layer: Dict[str, object], dtype=np.float64, gamma: Optional[float] = None):
     """gamma_l * E^d_l(h_t) for every row -- the left operand of Eq. 7."""
     sh = layer["shape"]

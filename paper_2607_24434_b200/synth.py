@@ -173,6 +173,42 @@ def draft_tokens_from_target(target: np.ndarray, V: int, seed: int, p_accept: fl
     return out
 
 
+# --------------------------------------------------------------------------
+# 4-bit block-quantised routed experts (the mobile workload of Sec. 4 runs Q4_0 weights).  Quantising is input
+# preparation, like the bf16 rounding above: it is done once, here, and both sides consume the resulting bytes.
+# Format (the published Q4_0 block): 32 consecutive weights of a matrix row share one fp16 scale d; each weight is
+# stored as a 4-bit code q with value d * (q - 8); a block is 18 bytes, the scale first, then 16 bytes whose low
+# nibbles hold codes 0..15 and whose high nibbles hold codes 16..31.
+# --------------------------------------------------------------------------
+Q4_BLOCK = 32
+Q4_BLOCK_BYTES = 18
+
+
+def quantize_q4_0(w: torch.Tensor) -> torch.Tensor:
+    """[R, C] float weights (C a multiple of 32) -> uint8 [R, C/32, 18] of Q4_0 blocks.  Per block: d = m / -8
+    with m the entry of largest magnitude (the first one on ties), code = min(15, floor(x / d + 8.5)), and d is
+    stored rounded to fp16."""
+    R, Ccols = w.shape
+    assert Ccols % Q4_BLOCK == 0
+    x = w.detach().to(torch.float32).cpu().reshape(R, Ccols // Q4_BLOCK, Q4_BLOCK)
+    idx = x.abs().argmax(dim=2, keepdim=True)
+    m = torch.gather(x, 2, idx)
+    d = m / -8.0
+    inv = torch.where(d != 0, 1.0 / d, torch.zeros_like(d))
+    q = torch.clamp(torch.floor(x * inv + 8.5), max=15.0).to(torch.uint8)
+    d16 = d.to(torch.float16)
+    out = torch.empty((R, Ccols // Q4_BLOCK, Q4_BLOCK_BYTES), dtype=torch.uint8)
+    out[:, :, 0:2] = d16.view(torch.uint8).reshape(R, Ccols // Q4_BLOCK, 2)
+    out[:, :, 2:] = q[:, :, :16] | (q[:, :, 16:] << 4)
+    return out
+
+
+def q4_expert_blob(Wg: torch.Tensor, Wu: torch.Tensor, Wd: torch.Tensor) -> torch.Tensor:
+    """One routed expert as the host pool stores it when quantised: the Q4_0 blocks of W_g [I,H], W_u [I,H] and
+    W_d [H,I], row-major, one matrix after the other (uint8, 3*H*I*18/32 bytes)."""
+    return torch.cat([quantize_q4_0(Wg).reshape(-1), quantize_q4_0(Wu).reshape(-1), quantize_q4_0(Wd).reshape(-1)])
+
+
 def to_numpy_f32(t: torch.Tensor) -> np.ndarray:
     """Exact fp32 view of a (possibly bf16, possibly CUDA) tensor as a numpy array."""
     return t.detach().to("cpu", torch.float32).numpy()

@@ -288,6 +288,57 @@ def test_residual_loss_identities():
     assert np.allclose(y_top1 + m, y_star, rtol=1e-12, atol=1e-14)
 
 
+# ------------------------------------------------------ 4-bit block-quantised experts (Sec. 4, mobile runs)
+def test_q4_blocks_round_trip_and_error_bound():
+    rng = np.random.default_rng(30)
+    w = torch.from_numpy(rng.standard_normal((5, 96)).astype(np.float32) * 0.02)
+    w[0, :32] = 0.0                                  # an all-zero block: scale 0, every weight 0
+    w[1, 7] = -0.2                                   # a block whose extreme is negative: d > 0, code 0 is the extreme
+    w[2, 40] = 0.3                                   # ... and one whose extreme is positive: d < 0
+    blocks = synth.quantize_q4_0(w).numpy()
+    assert blocks.shape == (5, 3, 18)
+    deq = O.dequantize_q4_0(blocks)
+    x = w.numpy().astype(np.float64)
+    for r in range(5):
+        for b in range(3):
+            seg, got = x[r, 32 * b:32 * b + 32], deq[r, 32 * b:32 * b + 32]
+            d = float(np.frombuffer(blocks[r, b, :2].tobytes(), dtype="<f2")[0])
+            i_ext = int(np.argmax(np.abs(seg)))
+            if seg[i_ext] == 0.0:
+                assert d == 0.0 and np.all(got == 0.0)
+                continue
+            # the scale is the extreme over -8, rounded to fp16, and the extreme gets code 0
+            assert d == float(np.float16(seg[i_ext] / -8.0))
+            assert got[i_ext] == -8.0 * d
+            # every weight lies on the grid d * {-8..7}; the error is at most half a step, except where a value
+            # of the sign opposite to the extreme would need code 16 and is clipped to 15 (at most one step);
+            # rounding the scale to fp16 moves the grid by at most 8 * |d| * 2^-11
+            codes = got / d
+            assert np.all(codes == np.round(codes)) and codes.min() >= -8 and codes.max() <= 7
+            slack = 8 * abs(d) * 2.0 ** -11 + 1e-12
+            clipped = (seg / (seg[i_ext] / -8.0)) > 7.5
+            assert np.all(np.abs(got - seg)[~clipped] <= 0.5 * abs(d) + slack)
+            assert np.all(np.abs(got - seg)[clipped] <= 1.0 * abs(d) + slack)
+    # values already on a block's grid are reproduced exactly; blocks do not influence each other
+    d0 = float(np.float16(0.0123))
+    grid = torch.tensor([[d0 * (c - 8) for c in range(16)] * 2], dtype=torch.float32)
+    assert np.array_equal(O.dequantize_q4_0(synth.quantize_q4_0(grid).numpy())[0], grid.numpy()[0].astype(np.float64))
+    w2 = w.clone(); w2[3, 64:] *= 5.0
+    b2 = synth.quantize_q4_0(w2).numpy()
+    assert np.array_equal(b2[3, :2], blocks[3, :2]) and not np.array_equal(b2[3, 2], blocks[3, 2])
+    # nibble order: low nibbles are weights 0..15 of the block, high nibbles weights 16..31
+    ramp = torch.tensor([[-8.0 + (j % 16) for j in range(32)]], dtype=torch.float32)   # extreme -8 -> d = 1
+    rb = synth.quantize_q4_0(ramp).numpy()[0, 0]
+    assert float(np.frombuffer(rb[:2].tobytes(), dtype="<f2")[0]) == 1.0
+    assert [int(v & 15) for v in rb[2:]] == list(range(16)) and [int(v >> 4) for v in rb[2:]] == list(range(16))
+    # expert blob: three matrices one after the other, 18 bytes per 32 weights
+    Wg = torch.from_numpy(rng.standard_normal((8, 64)).astype(np.float32))
+    Wd = torch.from_numpy(rng.standard_normal((64, 32)).astype(np.float32))
+    blob = synth.q4_expert_blob(Wg, Wg * 2, Wd)
+    assert blob.numel() == (8 * 64 * 2 + 64 * 32) * 18 // 32
+    assert np.array_equal(blob[:8 * 2 * 18].numpy().reshape(8, 2, 18), synth.quantize_q4_0(Wg).numpy())
+
+
 # ------------------------------------------------------ union (Eq. 2, Eq. 3)
 def test_block_union_enumeration_and_invariants():
     rng = np.random.default_rng(6)
