@@ -401,11 +401,19 @@ def run_offload(args):
     layers, pools = [], []
     nbytes = binding.expert_blob_bytes(shape, shape.inter)
     cache = binding.ExpertCache(ctx, NLAY, shape.n_experts, S, nbytes)
+    if args.q4:
+        cache.set_q4(shape)      # host pool of 4-bit block-quantised experts, expanded into the slots after each copy
+    pool_bytes = binding.q4_expert_bytes(shape, shape.inter) if args.q4 else nbytes
     for l in range(NLAY):
         w = synth.make_layer(shape, 3000 + l, device, zipf=True)
         L = binding.Layer.from_weights(ctx, w, routed_resident=False)
         torch.cuda.synchronize()
-        host = L.blobs.cpu().pin_memory()
+        if args.q4:
+            Wg, Wu, Wd = w["experts"]
+            host = torch.stack([synth.q4_expert_blob(Wg[e].float().cpu(), Wu[e].float().cpu(), Wd[e].float().cpu())
+                                for e in range(shape.n_experts)]).pin_memory()
+        else:
+            host = L.blobs.cpu().pin_memory()
         L.blobs = None
         del w
         for e in range(shape.n_experts):
@@ -457,7 +465,9 @@ def run_offload(args):
         "warmup": args.warmup, "ms_per_step": dt / steps * 1e3, "higher_is_better": True, "data": "synthetic",
         "dtype": "bf16 weights, fp32 accumulate",
         "config": {"workload": f"configs[4]: offloaded V2-Lite-shaped stack, {NLAY} MoE layers, experts in pinned host "
-                               f"memory ({NLAY * shape.n_experts * nbytes / 1e9:.1f} GB), {S} HBM slots per layer (LRU), "
+                               f"memory ({NLAY * shape.n_experts * pool_bytes / 1e9:.1f} GB, "
+                               f"{'4-bit block-quantised, expanded to bf16 after each copy' if args.q4 else 'bf16 blobs'}), "
+                               f"{S} HBM slots per layer (LRU), "
                                f"draft K={K} + prefetch of the draft router's top-{shape.top_k} + verify in waves; "
                                "scripted geometric(0.85) acceptance", "layers": NLAY, "block_tokens": K},
         "emitted_tokens_per_s": (accepted + steps) / dt,
@@ -557,6 +567,8 @@ def main():
     ap.add_argument("--workload", default="layer", choices=["layer", "offload"],
                     help="layer: configs[1] (default, the driver's line); offload: configs[4] expert-cache workload")
     ap.add_argument("--offload-layers", type=int, default=4)
+    ap.add_argument("--q4", action="store_true",
+                    help="offload workload: keep the host pool 4-bit block-quantised (Q4_0 blocks)")
     ap.add_argument("--offload-steps", type=int, default=24)
     ap.add_argument("--traffic", type=float, default=None,
                     help="ncu DRAM bytes per launch of the dominant kernel, if known")

@@ -111,6 +111,21 @@ dx_status dx_expert_blob_bytes(const dx_layer_desc* desc, int32_t inter, size_t*
 dx_status dx_pack_expert(dx_ctx* ctx, const dx_layer_desc* desc, int32_t inter,
                          const void* Wg, const void* Wu, const void* Wd, void* blob_out, void* stream);
 
+/* ---- 4-bit block-quantised experts (the paper's mobile runs use Q4_0 weights, Sec. 4) ----------------------
+ * Format of a quantised expert: the Q4_0 blocks of W_g [inter,hidden], W_u [inter,hidden] and W_d [hidden,inter],
+ * row-major, one matrix after the other; a block covers 32 consecutive weights of a row and is 18 bytes: the fp16
+ * scale d (little endian), then 16 bytes whose low nibbles are the codes of weights 0..15 and whose high nibbles
+ * those of weights 16..31; weight = d * (code - 8).  inter must be a multiple of 32; bf16 layers only.
+ * On this hardware the quantised form is the *transport and storage* form: 180 GB of HBM hold expanded slots
+ * easily, the scarce link is host -> device.  dx_expand_q4_expert (device pointers, asynchronous on `stream`)
+ * writes the bf16 streaming blob of dx_expert_blob_bytes bytes (128-byte aligned), each weight rounded to bf16
+ * once: out = bf16(d * (code - 8)); the compute kernels are the bf16 ones, unchanged.  A cache switched with
+ * expert_cache_set_q4 takes quantised blobs in expert_cache_register and expands each copy on its copy stream
+ * (see the cache section). */
+dx_status dx_q4_expert_bytes(const dx_layer_desc* desc, int32_t inter, size_t* bytes_out);
+dx_status dx_expand_q4_expert(dx_ctx* ctx, const dx_layer_desc* desc, int32_t inter, const void* q4_blob,
+                              void* blob_out, void* stream);
+
 /* ---- layer ------------------------------------------------------------------------------------------------
  * dx_layer_create copies the description and allocates the layer's device pointer table.
  * set_router: W_r [E,H] in weight_dtype, optional fp32 bias[E] added to the router logits (NULL = none).
@@ -288,6 +303,10 @@ typedef struct {
 dx_status expert_cache_create(dx_ctx* ctx, int32_t n_layers, int32_t n_experts, int32_t slots_per_layer,
                               size_t blob_bytes, dx_cache** out);
 dx_status expert_cache_destroy(dx_cache* cache);
+/* Switch the host pool to 4-bit block-quantised blobs (dx_q4_expert_bytes each; see above): must be called before
+ * the first expert_cache_register; DX_ERR_SHAPE if desc/inter do not give the slot size the cache was created
+ * with.  bytes_h2d then counts the quantised bytes that actually cross the link. */
+dx_status expert_cache_set_q4(dx_cache* cache, const dx_layer_desc* desc, int32_t inter);
 dx_status expert_cache_register(dx_cache* cache, int32_t layer, int32_t expert, const void* pinned_host_blob);
 /* Start of a decode step (Algorithm 1, line 1: P <- empty): experts prefetched earlier and never used since
  * are counted as wasted and stop being protected from eviction. */

@@ -55,6 +55,8 @@ SIGNATURES = {
     "dx_kernel_launches": (C.c_int64, [_P]),
     "dx_expert_blob_bytes": (_I, [C.POINTER(LayerDesc), _I, C.POINTER(C.c_size_t)]),
     "dx_pack_expert": (_I, [_P, C.POINTER(LayerDesc), _I, _P, _P, _P, _P, _P]),
+    "dx_q4_expert_bytes": (_I, [C.POINTER(LayerDesc), _I, C.POINTER(C.c_size_t)]),
+    "dx_expand_q4_expert": (_I, [_P, C.POINTER(LayerDesc), _I, _P, _P, _P]),
     "dx_layer_create": (_I, [_P, C.POINTER(LayerDesc), C.POINTER(_P)]),
     "dx_layer_destroy": (_I, [_P]),
     "dx_layer_set_router": (_I, [_P, _P, _P]),
@@ -86,6 +88,7 @@ SIGNATURES = {
     "moe_router_agreement": (_I, [_P, _P, _P, _I, _P, _P, _P]),
     "dx_squared_error": (_I, [_P, _P, _P, C.c_int64, _P, _P]),
     "expert_cache_create": (_I, [_P, _I, _I, _I, C.c_size_t, C.POINTER(_P)]),
+    "expert_cache_set_q4": (_I, [_P, C.POINTER(LayerDesc), _I]),
     "expert_cache_destroy": (_I, [_P]),
     "expert_cache_register": (_I, [_P, _I, _I, _P]),
     "expert_cache_begin_step": (_I, [_P]),
@@ -177,6 +180,26 @@ def pack_expert(ctx: Context, shape: LayerShape, Wg: torch.Tensor, Wu: torch.Ten
     d = _desc(shape)
     _check(ctx.lib.dx_pack_expert(ctx.handle, C.byref(d), inter, _ptr(Wg.contiguous()), _ptr(Wu.contiguous()),
                                   _ptr(Wd.contiguous()), _ptr(out), _stream()), "dx_pack_expert")
+    return out
+
+
+def q4_expert_bytes(shape: LayerShape, inter: int) -> int:
+    n = C.c_size_t(0)
+    d = _desc(shape)
+    _check(load().dx_q4_expert_bytes(C.byref(d), inter, C.byref(n)), "dx_q4_expert_bytes")
+    return n.value
+
+
+def expand_q4_expert(ctx: Context, shape: LayerShape, inter: int, q4_blob: torch.Tensor,
+                     out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """dx_expand_q4_expert: a 4-bit block-quantised expert (uint8 device tensor) -> the bf16 streaming blob."""
+    if q4_blob.numel() != q4_expert_bytes(shape, inter):
+        raise ValueError("quantised blob has the wrong size")
+    if out is None:
+        out = torch.empty(expert_blob_bytes(shape, inter), dtype=torch.uint8, device=q4_blob.device)
+    d = _desc(shape)
+    _check(ctx.lib.dx_expand_q4_expert(ctx.handle, C.byref(d), inter, _ptr(q4_blob), _ptr(out), _stream()),
+           "dx_expand_q4_expert")
     return out
 
 
@@ -400,6 +423,11 @@ class ExpertCache:
     def _ids(ids: Sequence[int]):
         arr = (C.c_int32 * len(ids))(*[int(i) for i in ids])
         return arr, len(ids)
+
+    def set_q4(self, shape: LayerShape) -> None:
+        """The host pool holds 4-bit block-quantised blobs from now on (before the first register)."""
+        d = _desc(shape)
+        _check(self.lib.expert_cache_set_q4(self.handle, C.byref(d), shape.inter), "expert_cache_set_q4")
 
     def register(self, layer: int, expert: int, pinned_blob: torch.Tensor) -> None:
         self._keep.append(pinned_blob)

@@ -135,6 +135,27 @@ extern "C" dx_status dx_pack_expert(dx_ctx* ctx, const dx_layer_desc* desc, int3
   return DX_OK;
 }
 
+extern "C" dx_status dx_q4_expert_bytes(const dx_layer_desc* desc, int32_t inter, size_t* bytes_out) {
+  if (!desc || !bytes_out) return DX_ERR_INVALID_ARG;
+  if (desc->weight_dtype != DX_DTYPE_BF16) return DX_ERR_UNSUPPORTED;
+  // blocks of 32 along the rows of W_g, W_u [inter, hidden] and of W_d [hidden, inter]
+  if (inter <= 0 || inter % 32 || desc->hidden <= 0 || desc->hidden % 256) return DX_ERR_UNSUPPORTED;
+  *bytes_out = (size_t)3 * desc->hidden * inter / 32 * 18;
+  return DX_OK;
+}
+
+extern "C" dx_status dx_expand_q4_expert(dx_ctx* ctx, const dx_layer_desc* desc, int32_t inter, const void* q4_blob,
+                                         void* blob_out, void* stream) {
+  if (!ctx || !desc || !q4_blob || !blob_out) return DX_ERR_INVALID_ARG;
+  size_t need = 0;
+  dx_status s = dx_q4_expert_bytes(desc, inter, &need);
+  if (s != DX_OK) return s;
+  if (((uintptr_t)blob_out) % 128 || ((uintptr_t)q4_blob) % 2) return DX_ERR_INVALID_ARG;
+  DX_CUDA(ctx, dx_launch_expand_q4(desc->hidden, inter, q4_blob, blob_out, (cudaStream_t)stream));
+  ctx->launches++;
+  return DX_OK;
+}
+
 extern "C" dx_status dx_layer_create(dx_ctx* ctx, const dx_layer_desc* desc, dx_layer** out) {
   if (!ctx || !out) return DX_ERR_INVALID_ARG;
   *out = nullptr;

@@ -40,6 +40,11 @@ struct dx_cache {
   int L, E, S;
   size_t blob_bytes;
   unsigned char* slab;
+  // quantised host pool: registered blobs are 4-bit block-quantised (q4_bytes each); a copy lands in the slot's
+  // staging area and is expanded into the slot on the copy stream
+  size_t q4_bytes;
+  int q4_hidden, q4_inter;
+  unsigned char* staging;
   cudaStream_t copy_stream;
   unsigned long long clock;
   dx_cache_stats stats;
@@ -62,6 +67,9 @@ __global__ void dx_table_patch_kernel(const void** table, DxTablePatch patch) {
 inline DxSlot& slot_ref(dx_cache* c, int layer, int s) { return c->slots[(size_t)layer * c->S + s]; }
 inline void* slot_ptr(dx_cache* c, int layer, int s) {
   return c->slab ? c->slab + ((size_t)layer * c->S + s) * c->blob_bytes : nullptr;
+}
+inline void* staging_ptr(dx_cache* c, int layer, int s) {
+  return c->staging + ((size_t)layer * c->S + s) * ((c->q4_bytes + 255) / 256 * 256);
 }
 
 // victim search; protected_ok: may take a slot of P; pinned: slots of the call in progress
@@ -98,15 +106,26 @@ dx_status load_into(dx_cache* c, int layer, int s, int e, bool as_prefetch) {
   sl.stamp = ++c->clock;
   c->slot_of[(size_t)layer * c->E + e] = s;
   c->pending[layer].push_back({e, slot_ptr(c, layer, s)});
-  c->stats.bytes_h2d += (int64_t)c->blob_bytes;
+  c->stats.bytes_h2d += (int64_t)(c->q4_bytes ? c->q4_bytes : c->blob_bytes);
   if (c->ctx) {
     // the slot may still be read by kernels already enqueued on the compute stream
     if (c->used_valid[layer]) {
       cudaError_t e0 = cudaStreamWaitEvent(c->copy_stream, c->used_ev[layer], 0);
       if (e0 != cudaSuccess) { c->ctx->last_cuda = e0; return DX_ERR_CUDA; }
     }
-    cudaError_t e1 = cudaMemcpyAsync(slot_ptr(c, layer, s), c->host_blob[(size_t)layer * c->E + e], c->blob_bytes,
-                                     cudaMemcpyHostToDevice, c->copy_stream);
+    cudaError_t e1;
+    if (c->q4_bytes) {
+      // a quarter of the bytes cross the host link; the expansion to the streaming layout runs at HBM speed
+      e1 = cudaMemcpyAsync(staging_ptr(c, layer, s), c->host_blob[(size_t)layer * c->E + e], c->q4_bytes,
+                           cudaMemcpyHostToDevice, c->copy_stream);
+      if (e1 == cudaSuccess)
+        e1 = dx_launch_expand_q4(c->q4_hidden, c->q4_inter, staging_ptr(c, layer, s), slot_ptr(c, layer, s),
+                                 c->copy_stream);
+      if (e1 == cudaSuccess) c->ctx->launches++;
+    } else {
+      e1 = cudaMemcpyAsync(slot_ptr(c, layer, s), c->host_blob[(size_t)layer * c->E + e], c->blob_bytes,
+                           cudaMemcpyHostToDevice, c->copy_stream);
+    }
     if (e1 == cudaSuccess) e1 = cudaEventRecord(sl.ev, c->copy_stream);
     if (e1 != cudaSuccess) { c->ctx->last_cuda = e1; return DX_ERR_CUDA; }
     sl.copy_pending = true;
@@ -187,6 +206,9 @@ extern "C" dx_status expert_cache_create(dx_ctx* ctx, int32_t n_layers, int32_t 
   c->L = n_layers; c->E = n_experts; c->S = slots_per_layer;
   c->blob_bytes = blob_bytes;
   c->slab = nullptr;
+  c->q4_bytes = 0;
+  c->q4_hidden = c->q4_inter = 0;
+  c->staging = nullptr;
   c->copy_stream = nullptr;
   c->clock = 0;
   c->stats = dx_cache_stats{};
@@ -225,6 +247,7 @@ extern "C" dx_status expert_cache_destroy(dx_cache* c) {
       if (e) cudaEventDestroy(e);
     if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
     cudaFree(c->slab);
+    cudaFree(c->staging);
   }
   for (auto* L : c->layer)
     if (L) { L->cache = nullptr; L->cache_layer = -1; }
@@ -247,6 +270,30 @@ extern "C" dx_status dx_layer_attach_cache(dx_layer* L, dx_cache* c, int32_t lay
     L->table_host[base + e] = s >= 0 ? slot_ptr(c, layer_index, s) : nullptr;
   }
   L->dirty = true;
+  return DX_OK;
+}
+
+extern "C" dx_status expert_cache_set_q4(dx_cache* c, const dx_layer_desc* desc, int32_t inter) {
+  if (!c || !desc) return DX_ERR_INVALID_ARG;
+  size_t q4 = 0, full = 0;
+  dx_status s = dx_q4_expert_bytes(desc, inter, &q4);
+  if (s != DX_OK) return s;
+  if (dx_expert_blob_bytes(desc, inter, &full) != DX_OK || full != c->blob_bytes) return DX_ERR_SHAPE;
+  // only before anything is registered or resident: the pool's format is one for all experts
+  for (const void* b : c->host_blob)
+    if (b) return DX_ERR_INVALID_ARG;
+  if (c->q4_bytes) return DX_ERR_INVALID_ARG;
+  if (c->ctx) {
+    cudaError_t e = cudaSetDevice(c->ctx->device);
+    if (e == cudaSuccess) e = cudaMalloc(&c->staging, (size_t)c->L * c->S * ((q4 + 255) / 256 * 256));
+    if (e != cudaSuccess) {
+      c->ctx->last_cuda = e;
+      return e == cudaErrorMemoryAllocation ? DX_ERR_OOM : DX_ERR_CUDA;
+    }
+  }
+  c->q4_bytes = q4;
+  c->q4_hidden = desc->hidden;
+  c->q4_inter = inter;
   return DX_OK;
 }
 

@@ -20,6 +20,8 @@
 // the products carry ~16 mantissa bits.  The packed blob stores every tile in
 // the exact per-lane fragment order, which is why no ldmatrix or swizzle is
 // needed.  All waits are bounded; an expired wait sets the device status word.
+#include <cuda_fp16.h>
+
 #include "dx_internal.cuh"
 
 namespace {
@@ -711,6 +713,47 @@ __global__ void dx_pack_bf16_kernel(const __nv_bfloat16* Wg, const __nv_bfloat16
   }
 }
 
+// 4-bit block-quantised expert (three matrices of 18-byte blocks: fp16 scale, then 16 bytes of codes, low nibbles
+// = weights 0..15 of the block, high nibbles = weights 16..31; weight = scale * (code - 8)) expanded straight
+// into the bf16 streaming blob above, each value rounded to bf16 once.
+__device__ __forceinline__ __nv_bfloat16 q4_value(const unsigned char* mat, int row, int col, int cols) {
+  const unsigned char* blk = mat + ((size_t)row * (cols / 32) + col / 32) * 18;
+  const float d = __half2float(__ushort_as_half((unsigned short)(blk[0] | (blk[1] << 8))));
+  const int j = col & 31;
+  const int code = j < 16 ? (blk[2 + j] & 0x0F) : (blk[2 + j - 16] >> 4);
+  return __float2bfloat16_rn(d * (float)(code - 8));
+}
+
+__global__ void dx_expand_q4_kernel(const unsigned char* q4, __nv_bfloat16* blob, int H, int I) {
+  const size_t n = (size_t)3 * H * I;
+  const int KW = H / 128, PW = H / 256;
+  const size_t mat_gu = (size_t)I * (H / 32) * 18;   // bytes of W_g (and of W_u)
+  const unsigned char* Wg = q4;
+  const unsigned char* Wu = q4 + mat_gu;
+  const unsigned char* Wd = q4 + 2 * mat_gu;
+  for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < n; idx += (size_t)gridDim.x * blockDim.x) {
+    const int j = (int)(idx / (24 * (size_t)H));
+    const int r = (int)(idx % (24 * (size_t)H));
+    const int w = r / (3 * H), rr = r % (3 * H);
+    __nv_bfloat16 v;
+    if (rr < 2 * H) {
+      const int i = rr / 256, l = (rr % 256) / 8, el = rr % 8;
+      const int s = w * KW + i, g = l >> 2, c = l & 3;
+      const int col = 16 * s + 4 * c + (el & 1) + ((el >> 2) << 1);
+      const int row = 8 * j + g;
+      v = q4_value(((el >> 1) & 1) ? Wu : Wg, row, col, H);
+    } else {
+      const int r2 = rr - 2 * H;
+      const int i = r2 / 256, l = (r2 % 256) / 8, el = r2 % 8;
+      const int q = w * PW + i, g = l >> 2, c = l & 3;
+      const int row = 32 * q + 8 * (el >> 1) + g;
+      const int col = 8 * j + 2 * c + (el & 1);
+      v = q4_value(Wd, row, col, I);
+    }
+    blob[idx] = v;
+  }
+}
+
 // fp32 blob, unit j: Wg rows 8j..8j+7 [8][H], Wu rows [8][H], then W_d columns 8j..8j+7 transposed [8][H]
 __global__ void dx_pack_fp32_kernel(const float* Wg, const float* Wu, const float* Wd, float* blob, int H, int I) {
   const size_t n = (size_t)3 * H * I;
@@ -764,6 +807,14 @@ cudaError_t dx_launch_experts(dx_ctx* ctx, const DxExpertParams& p, int weight_d
     case 2048: return launch_bf16_h<2048>(ctx, p, K, st);
     default: return cudaErrorInvalidConfiguration;
   }
+}
+
+cudaError_t dx_launch_expand_q4(int H, int I, const void* q4, void* blob, cudaStream_t st) {
+  const size_t n = (size_t)3 * H * I;
+  int grid = (int)((n + 255) / 256);
+  if (grid > 4096) grid = 4096;
+  dx_expand_q4_kernel<<<grid, 256, 0, st>>>((const unsigned char*)q4, (__nv_bfloat16*)blob, H, I);
+  return cudaGetLastError();
 }
 
 cudaError_t dx_launch_pack(int weight_dtype, int H, int I, const void* Wg, const void* Wu, const void* Wd,

@@ -153,6 +153,7 @@ cudaError_t dx_launch_route(const DxRouteParams& p, int weight_dtype, cudaStream
 cudaError_t dx_launch_experts(dx_ctx* ctx, const DxExpertParams& p, int weight_dtype, int K, cudaStream_t st);
 cudaError_t dx_launch_pack(int weight_dtype, int H, int I, const void* Wg, const void* Wu, const void* Wd,
                            void* blob, cudaStream_t st);
+cudaError_t dx_launch_expand_q4(int H, int I, const void* q4, void* blob, cudaStream_t st);
 cudaError_t dx_launch_accept(dx_ctx* ctx, const float* h, int M, const void* W_lm, int V, int H, int w_dtype,
                              const int32_t* draft, int K, int rms_norm, int32_t* target, int32_t* n_accept,
                              int32_t* next_token, float* conf, cudaStream_t st);
