@@ -20,7 +20,7 @@ namespace {
 
 __device__ __forceinline__ uint4 ldg_stream(const void* p) {
   uint4 r;
-  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+  asm volatile("ld.global.nc.L1::no_allocate.L2::256B.v4.u32 {%0,%1,%2,%3}, [%4];"
                : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
                : "l"(p));
   return r;
@@ -182,7 +182,7 @@ __global__ void __launch_bounds__(512, 1) dx_accept_bf16_kernel(AcceptParams p) 
     for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
       for (int r = 0; r < 4; ++r) ch[nt][r] = cl[nt][r] = 0.f;
-#pragma unroll 8
+#pragma unroll 16
     for (int q = 0; q < Q; ++q) {
       const uint4 a0 = ldg_stream(w0 + 32 * q);
       const uint4 a1 = ldg_stream(w1 + 32 * q);
