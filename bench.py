@@ -296,26 +296,54 @@ def run_gpu(args):
     draft_bytes = (shape.n_shared + 2) * exp_bytes + shape.n_experts * H * 2
     acc_bytes = V * H * 2
 
-    # ---- end to end through the binding with host buffers (pinned), copies inside the timed region
-    h_host = [b.cpu().pin_memory() for b in blocks]
-    d_host = draft_tok.cpu().pin_memory()
-    y_host = torch.empty((K, H), dtype=torch.float32).pin_memory()
-    res_host = torch.empty((2,), dtype=torch.int32).pin_memory()
-    tgt_host = torch.empty((K,), dtype=torch.int32).pin_memory()
-    h_dev = torch.empty((K, H), device=device)
-    d_dev = torch.empty((K,), dtype=torch.int32, device=device)
+    # ---- end to end through the binding with host buffers (pinned), copies inside the timed region.  Inputs (block
+    # and draft tokens) sit in one pinned buffer and one device buffer, results (y, target tokens, accepted length,
+    # next token) in another pair, so a step moves them with one copy each way.
+    in_bytes, out_bytes = K * H * 4 + K * 4, K * H * 4 + K * 4 + 8
+    in_host = [torch.empty((in_bytes,), dtype=torch.uint8).pin_memory() for _ in range(NL)]
+    for li in range(NL):
+        in_host[li][:K * H * 4].view(torch.float32).copy_(blocks[li].cpu().reshape(-1))
+        in_host[li][K * H * 4:].view(torch.int32).copy_(draft_tok.cpu())
+    out_host = torch.empty((out_bytes,), dtype=torch.uint8).pin_memory()
+    in_dev = torch.empty((in_bytes,), dtype=torch.uint8, device=device)
+    out_dev = torch.empty((out_bytes,), dtype=torch.uint8, device=device)
+    h_dev = in_dev[:K * H * 4].view(torch.float32).view(K, H)
+    d_dev = in_dev[K * H * 4:].view(torch.int32)
+    y_e2e = out_dev[:K * H * 4].view(torch.float32).view(K, H)
+    res = out_dev[K * H * 4:].view(torch.int32)
+    abuf_e2e = {"target": res[:K], "n_accept": res[K:K + 1], "next_token": res[K + 1:K + 2]}
+
+    def e2e_body(li):
+        in_dev.copy_(in_host[li], non_blocking=True)
+        binding.moe_draft_step(layers[li], h_dev[:1], yd, dbuf)
+        binding.moe_verify_block(layers[li], h_dev, y_e2e, rb[li])
+        binding.spec_accept(ctx, y_e2e, W_lm, d_dev, True, abuf_e2e)
+        out_host.copy_(out_dev, non_blocking=True)
+
+    # one graph per layer: the host -> device copies of the step's inputs (from fixed pinned buffers a caller would
+    # fill), the five kernels, and the device -> host copies of the results; a step = one graph launch + one sync
+    e2e_graphs = None
+    if not args.no_graph:
+        side2 = torch.cuda.Stream(device=device)
+        side2.wait_stream(stream)
+        with torch.cuda.stream(side2):
+            for li in range(NL):
+                e2e_body(li)
+        stream.wait_stream(side2)
+        torch.cuda.synchronize()
+        e2e_graphs = []
+        for li in range(NL):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=side2):
+                e2e_body(li)
+            e2e_graphs.append(g)
 
     def e2e_step(i):
         li = i % NL
-        h_dev.copy_(h_host[li], non_blocking=True)
-        d_dev.copy_(d_host, non_blocking=True)
-        binding.moe_draft_step(layers[li], h_dev[:1], yd, dbuf)
-        binding.moe_verify_block(layers[li], h_dev, ys[li], rb[li])
-        binding.spec_accept(ctx, ys[li], W_lm, d_dev, True, abuf)
-        y_host.copy_(ys[li], non_blocking=True)
-        tgt_host.copy_(abuf["target"], non_blocking=True)
-        res_host[0:1].copy_(abuf["n_accept"], non_blocking=True)
-        res_host[1:2].copy_(abuf["next_token"], non_blocking=True)
+        if e2e_graphs is not None:
+            e2e_graphs[li].replay()
+        else:
+            e2e_body(li)
         stream.synchronize()
 
     for i in range(max(3, args.warmup)):
@@ -328,6 +356,16 @@ def run_gpu(args):
     g1.record(stream)
     barrier()
     e2e_ms = g0.elapsed_time(g1)
+    # what came back over the link must be what the device-resident loop produced for the same layer
+    li_last = (args.steps - 1) % NL
+    got_y = out_host[:K * H * 4].view(torch.float32).view(K, H)
+    got_t = out_host[K * H * 4:].view(torch.int32)[:K]
+    binding.moe_verify_block(layers[li_last], blocks[li_last], ys[li_last], rb[li_last])
+    binding.spec_accept(ctx, ys[li_last], W_lm, draft_tok, True, abuf)
+    torch.cuda.synchronize()
+    if not torch.equal(got_t, abuf["target"].cpu()) or \
+            (got_y - ys[li_last].cpu()).abs().max().item() > 1e-4 * ys[li_last].abs().max().item():
+        raise RuntimeError("end-to-end results differ from the device-resident run")
 
     from paper_2607_24434_b200 import multi
     agg = multi.aggregate({"step": total_ms, "e2e": e2e_ms}, units=K * args.steps, launches=launches, device=device)
@@ -355,7 +393,10 @@ def run_gpu(args):
         "gpu_launches": launches,
         "e2e": {"value": multi.throughput(units_all, e2e_ms), "unit": UNIT,
                 "h2d_bytes_per_step": K * H * 4 + K * 4, "d2h_bytes_per_step": K * H * 4 + K * 4 + 8,
-                "ms_per_step": e2e_ms / args.steps},
+                "ms_per_step": e2e_ms / args.steps,
+                "launch": ("one CUDA graph launch (input copies, five kernels, result copies) and one stream "
+                           "synchronisation per step") if e2e_graphs is not None else
+                          "eager calls and one stream synchronisation per step"},
         "roofline": {"kernel": "dx_experts_bf16_kernel (grouped SwiGLU of the verify block)", "bound": "hbm",
                      "achieved": verify_gbs, "peak": peak, "unit": "GB/s", "frac": verify_gbs / peak,
                      "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBs": verify_gbs / NOMINAL_HBM_GBS,
