@@ -153,8 +153,7 @@ __device__ __forceinline__ void cta_bar() { asm volatile("bar.sync 2, 288;" ::: 
 // (a "wave" of union experts when the experts are staged through a cache); the units of the window, together
 // with the routing-independent units handled before (NSe of them, [s_lo,s_hi) on this CTA), are split evenly.
 __device__ __forceinline__ void routed_range(int n_groups, const DxExpertParams& p, int n_static, int NSe, int s_lo,
-                                             int s_hi, int& e_lo, int& e_hi, int& u_lo, int& u_hi) {
-  const int G = gridDim.x, cta = blockIdx.x;
+                                             int s_hi, int G, int cta, int& e_lo, int& e_hi, int& u_lo, int& u_hi) {
   const int g_lo = min(n_groups, p.first_routed);
   const int g_hi = p.n_routed < 0 ? n_groups : min(n_groups, g_lo + p.n_routed);
   e_lo = n_static + g_lo;
@@ -175,7 +174,8 @@ __device__ __forceinline__ void routed_range(int n_groups, const DxExpertParams&
   u_hi = (int)R0 + b;
 }
 
-template <int H, int NT>
+// TILES = 2: CTA pairs, one tile of eight block rows each (see below); only with NT = 1
+template <int H, int NT, int TILES>
 __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertParams p, int n_slots) {
   constexpr int KW = H / 128;        // phase-1 contraction steps per consumer warp
   constexpr int PW = H / 256;        // phase-2 row-tile pairs per consumer warp
@@ -195,7 +195,12 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const DxWork* W = p.work;
-  const int G = gridDim.x, cta = blockIdx.x;
+  // Blocks of more than eight rows whose second token tile does not fit next to the ring (H = 2048): the CTAs work
+  // in pairs, both members stream the same share of the units (the second read of a unit comes out of L2, its
+  // partner having just fetched it) and each multiplies it with one tile of eight block rows.
+  constexpr int row_tiles = TILES;
+  const int row_base = row_tiles == 2 ? 8 * (int)(blockIdx.x & 1) : 0;
+  const int G = gridDim.x / row_tiles, cta = blockIdx.x / row_tiles;
   // groups that do not depend on routing: shared experts, then (draft mode) the draft expert
   const int n_static = p.n_shared + (p.draft_tiles > 0 ? 1 : 0);
   const int S0 = p.skip_shared ? p.n_shared * p.shared_tiles : 0;   // first routing-independent unit evaluated
@@ -288,7 +293,7 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
       if (lane == 0) { *abort_flag = 1; atomicExch(p.dev_status, DX_DEV_WAIT_EXPIRED); }
     }
     int e_lo, e_hi, u_lo, u_hi;
-    routed_range(n_groups, p, n_static, NS, s_lo - S0, s_hi - S0, e_lo, e_hi, u_lo, u_hi);
+    routed_range(n_groups, p, n_static, NS, s_lo - S0, s_hi - S0, G, cta, e_lo, e_hi, u_lo, u_hi);
     const int unit_base = p.n_shared * p.shared_tiles + p.draft_tiles;
 #pragma unroll
     for (int i = 0; i < PER_LANE; ++i) {
@@ -397,13 +402,13 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
       // this lane's block rows (one per token tile) and their weights in this group
       float wrow[NT];
 #pragma unroll
-      for (int nt = 0; nt < NT; ++nt) wrow[nt] = row_weight(e, nt * 8 + g);
+      for (int nt = 0; nt < NT; ++nt) wrow[nt] = row_weight(e, row_base + nt * 8 + g);
       const bool need_hi = NT > 1 && __any_sync(0xffffffffu, wrow[NT - 1] != 0.0f);   // any of rows 8..15 routed here
 
       // ---- token fragments of this group
       if constexpr (kRegB) {
         const bool valid = wrow[0] != 0.0f;
-        const int tk = g;
+        const int tk = row_base + g;
         const float rs = hdr->rstd[tk];
         const float* xrow = p.x + (size_t)tk * H + 4 * c;
 #pragma unroll
@@ -553,7 +558,7 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
   // ---- the CTA's partial output rows go to y (initialised by the routing kernel, which has completed)
 #pragma unroll
   for (int nt = 0; nt < NT; ++nt) {
-    const int r0 = nt * 8 + 2 * c, r1 = r0 + 1;
+    const int r0 = row_base + nt * 8 + 2 * c, r1 = r0 + 1;
     if (r0 < p.K) {
       float* y0 = p.y + (size_t)r0 * H;
       float* y1 = p.y + (size_t)r1 * H;
@@ -769,27 +774,37 @@ __global__ void dx_pack_fp32_kernel(const float* Wg, const float* Wu, const floa
   }
 }
 
-template <int H, int NT>
+template <int H, int NT, int TILES>
 cudaError_t launch_bf16(dx_ctx* ctx, const DxExpertParams& p, cudaStream_t st) {
   const size_t hdr = (sizeof(SmemHeader) + 127) / 128 * 128;
   const size_t fixed = hdr + (size_t)2 * 8 * NT * 32 * 16 + (NT == 1 ? 0 : (size_t)NT * (H / 16) * 32 * 16);
   const size_t chunk = (size_t)6 * H;
   int n_slots = (int)(((size_t)ctx->smem_optin - fixed) / chunk);
   if (n_slots > kMaxSlots) n_slots = kMaxSlots;
-  if (n_slots < 2) return cudaErrorInvalidConfiguration;
+  if (n_slots < kConsumerWarps + 1) return cudaErrorInvalidConfiguration;   // a unit needs all its chunks at once
   const size_t smem = fixed + (size_t)n_slots * chunk;
-  cudaError_t e = cudaFuncSetAttribute(dx_experts_bf16_kernel<H, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  cudaError_t e = cudaFuncSetAttribute(dx_experts_bf16_kernel<H, NT, TILES>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)smem);
   if (e != cudaSuccess) return e;
   // One CTA per SM, minus the SMs the routing cluster (8 CTAs) runs on at the same time: a CTA of this kernel
   // fills an SM, so a CTA that had to wait for a routing CTA's SM would start late and become the tail.
-  const int grid = ctx->sm_count > 16 ? ctx->sm_count - 8 : ctx->sm_count;
-  return dx_launch_pdl(DX_PDL_EXPERTS, dx_experts_bf16_kernel<H, NT>, dim3(grid), dim3(kThreads), smem, st, 1, p, n_slots);
+  int grid = ctx->sm_count > 16 ? ctx->sm_count - 8 : ctx->sm_count;
+  if (TILES == 2) grid &= ~1;
+  return dx_launch_pdl(DX_PDL_EXPERTS, dx_experts_bf16_kernel<H, NT, TILES>, dim3(grid), dim3(kThreads), smem, st, 1, p, n_slots);
 }
 
 template <int H>
-cudaError_t launch_bf16_h(dx_ctx* ctx, const DxExpertParams& p, int K, cudaStream_t st) {
-  return K > 8 ? launch_bf16<H, 2>(ctx, p, st) : launch_bf16<H, 1>(ctx, p, st);
+cudaError_t launch_bf16_h(dx_ctx* ctx, const DxExpertParams& p_in, int K, cudaStream_t st) {
+  DxExpertParams p = p_in;
+  p.row_tiles = 1;
+  if (K <= 8) return launch_bf16<H, 1, 1>(ctx, p, st);
+  // two token tiles: fragments of both in shared memory where they fit next to a ring of at least one slot per
+  // consumer warp and one to spare; otherwise CTA pairs with one tile each
+  const size_t hdr = (sizeof(SmemHeader) + 127) / 128 * 128;
+  const size_t fixed2 = hdr + (size_t)2 * 8 * 2 * 32 * 16 + (size_t)2 * (H / 16) * 32 * 16;
+  if (fixed2 + (size_t)(kConsumerWarps + 1) * 6 * H <= (size_t)ctx->smem_optin) return launch_bf16<H, 2, 1>(ctx, p, st);
+  p.row_tiles = 2;
+  return launch_bf16<H, 1, 2>(ctx, p, st);
 }
 
 }  // namespace

@@ -140,6 +140,7 @@ struct DxExpertParams {
   // the routing-independent groups are part of it; a cache-staged union is processed in several windows
   int first_routed, n_routed, do_static;
   int skip_shared;           // 1: of the routing-independent groups only the draft expert is evaluated
+  int row_tiles;             // set by the launcher: 2 = CTA pairs, one tile of eight block rows each (K > 8)
   // Hand-over from the routing kernel launched right before this one (fused entry points only; null otherwise,
   // and then the kernel simply waits for everything in front of it).  With the hand-over this kernel may be running
   // before its inputs are final: consumers read the block only once this word is set, and the routed groups are

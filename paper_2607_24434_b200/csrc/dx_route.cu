@@ -436,11 +436,13 @@ template <typename WT, int TG>
 static cudaError_t launch_route_one(const DxRouteParams& p, cudaStream_t st) {
   // CTA 0 holds one partial table per column slice (at most 8)
   const size_t smem = (size_t)kRouteCluster * ((size_t)p.K * p.E + p.K) * sizeof(float);
-  static size_t allowed = 48 * 1024;   // per instantiation: raise the opt-in limit only when a launch needs it
-  if (smem > allowed) {
-    cudaError_t e = cudaFuncSetAttribute(dx_route_kernel<WT, TG>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  // static + dynamic shared memory can pass the default 48 KB: opt in once per instantiation for the largest case
+  static bool opted_in = false;
+  if (!opted_in) {
+    const size_t most = (size_t)kRouteCluster * ((size_t)DX_MAX_K * DX_MAX_E + DX_MAX_K) * sizeof(float);
+    cudaError_t e = cudaFuncSetAttribute(dx_route_kernel<WT, TG>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)most);
     if (e != cudaSuccess) return e;
-    allowed = smem;
+    opted_in = true;
   }
   return dx_launch_pdl(DX_PDL_ROUTE, dx_route_kernel<WT, TG>, dim3(kRouteCluster), dim3(kRouteThreads), smem, st,
                        kRouteCluster, p);

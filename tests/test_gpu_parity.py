@@ -196,7 +196,7 @@ def test_residual_forms(dx):
 
 
 # ------------------------------------------------------------------ full DeepSeek-V2-Lite-shaped layer (config 1)
-@pytest.mark.parametrize("K,zipf,rho", [(4, True, 0.0), (8, False, 0.9)])
+@pytest.mark.parametrize("K,zipf,rho", [(4, True, 0.0), (8, False, 0.9), (16, True, 0.9)])
 def test_v2lite_layer_verify_and_draft(dx, K, zipf, rho):
     sh = synth.shape_v2lite()
     near, n_union = _verify_case(dx, sh, K, seed=100 + K, zipf=zipf, rho=rho)
