@@ -165,8 +165,13 @@ dx_status moe_draft_step_topr(dx_layer* layer, const float* h, float* y, int32_t
  *   union_count [1] int32 = |U|;
  *   offsets [E+1] int32 and perm [K*k] int32: the token-expert pairs p = t*k + j sorted by (expert, p);
  *   expert e owns perm[offsets[e] .. offsets[e+1]).
- * moe_verify_block = moe_verify_route followed by moe_verify_experts on the same stream; the two halves are
- * exported so that a caller with offloaded experts can make them resident in between. */
+ * moe_verify_block gives the results of moe_verify_route followed by moe_verify_experts on the same stream; the
+ * two halves are exported so that a caller with offloaded experts can make them resident in between.  The fused
+ * call (and moe_draft_step, the *_residual forms) overlaps the two kernels: the expert kernel is made resident by
+ * the routing kernel before either has its input, streams the shared experts, and picks the block and the routed
+ * groups up from device memory as the routing kernel publishes them.  Every wait in it is bounded: if the routing
+ * kernel never runs, the expert kernel gives up, records DX_DEV_WAIT_EXPIRED and returns.  The fused calls are safe
+ * to capture into CUDA graphs and to replay. */
 dx_status moe_verify_block(dx_layer* layer, const float* h, int32_t K, float* y,
                            int32_t* topk_ids, float* topk_w, uint64_t* union_mask, int32_t* union_ids,
                            int32_t* union_count, int32_t* offsets, int32_t* perm, void* stream);

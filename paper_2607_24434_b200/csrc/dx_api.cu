@@ -55,7 +55,6 @@ extern "C" dx_status dx_create(int device, dx_ctx** out) {
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, device);
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device);
   if (e == cudaSuccess) e = cudaMalloc(&ctx->work, sizeof(DxWork));
-  if (e == cudaSuccess) e = cudaMalloc(&ctx->z, sizeof(float) * DX_MAX_K * DX_MAX_E);
   if (e == cudaSuccess) e = cudaMalloc(&ctx->ticket, sizeof(unsigned int) * 4);
   if (e == cudaSuccess) e = cudaMalloc(&ctx->keys, sizeof(unsigned long long) * DX_MAX_M);
   if (e == cudaSuccess) e = cudaMalloc(&ctx->dev_status, sizeof(int32_t));
@@ -79,7 +78,6 @@ extern "C" dx_status dx_create(int device, dx_ctx** out) {
 extern "C" dx_status dx_destroy(dx_ctx* ctx) {
   if (!ctx) return DX_ERR_INVALID_ARG;
   cudaFree(ctx->work);
-  cudaFree(ctx->z);
   cudaFree(ctx->ticket);
   cudaFree(ctx->keys);
   cudaFree(ctx->dev_status);
@@ -268,7 +266,7 @@ static dx_status do_route(dx_layer* L, const float* h, int K, float* y, const Ro
   p.skip_top1 = skip_top1 ? 1 : 0;
   p.rms_norm = residual ? 1 : 0;
   p.residual = residual ? 1 : 0;
-  p.y = y; p.z = ctx->z; p.ticket = ctx->ticket; p.work = ctx->work; p.dev_status = ctx->dev_status;
+  p.y = y; p.work = ctx->work; p.dev_status = ctx->dev_status;
   p.handover = paired ? ctx->handover : nullptr;
   p.topk_ids = o.topk_ids; p.topk_w = o.topk_w;
   p.union_mask = (unsigned long long*)o.union_mask; p.union_ids = o.union_ids; p.union_count = o.union_count;

@@ -69,8 +69,7 @@ struct dx_ctx {
   int64_t launches;
   // device scratch
   DxWork* work;        // work list
-  float* z;            // [DX_MAX_K, DX_MAX_E] router logits
-  unsigned int* ticket;        // last-CTA tickets (route, accept)
+  unsigned int* ticket;        // last-CTA ticket of the accept kernels (second word)
   unsigned long long* keys;    // [DX_MAX_M] packed argmax keys
   int32_t* dev_status;
   unsigned int* handover;      // device word {block input final}: see DxExpertParams
@@ -112,8 +111,6 @@ struct DxRouteParams {
                           // the hand-over words first, and set this word once everything in front of this
                           // kernel in the stream has completed
   float* y;
-  float* z;
-  unsigned int* ticket;
   DxWork* work;
   int32_t* dev_status;
   int32_t* topk_ids;
