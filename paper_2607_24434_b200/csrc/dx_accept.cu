@@ -171,9 +171,12 @@ __global__ void __launch_bounds__(512, 1) dx_accept_bf16_kernel(AcceptParams p) 
   for (int nt = 0; nt < NT; ++nt) { cm[nt][0] = cm[nt][1] = -INFINITY; cs[nt][0] = cs[nt][1] = 0.0f; }
 
   const int tiles = (p.V + 15) / 16;
-  const int warps_total = gridDim.x * (blockDim.x >> 5);
+  // Tiles are dealt to the CTAs first (tile t belongs to CTA t mod gridDim.x) and to the warps inside a CTA second,
+  // so every CTA streams the same number of tiles to within one; dealing them warp by warp across the grid would
+  // give the first CTAs one whole tile per warp more than the last ones.
+  const int tiles_cta = gridDim.x;
   const __nv_bfloat16* Wb = reinterpret_cast<const __nv_bfloat16*>(p.W);
-  for (int tile = blockIdx.x * (blockDim.x >> 5) + warp; tile < tiles; tile += warps_total) {
+  for (int tile = blockIdx.x + tiles_cta * warp; tile < tiles; tile += tiles_cta * (int)(blockDim.x >> 5)) {
     const int r0 = tile * 16 + g, r1 = r0 + 8;
     const __nv_bfloat16* w0 = Wb + (size_t)min(r0, p.V - 1) * H + 8 * c;
     const __nv_bfloat16* w1 = Wb + (size_t)min(r1, p.V - 1) * H + 8 * c;
