@@ -375,6 +375,41 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
   }
   consumer_bar();
 
+  // ---- token fragments: the MMA token slots are the block rows themselves, the same for every group (a group's
+  // weight, zero for the rows outside it, multiplies the activations), so they are built once
+  if constexpr (kRegB) {
+    const int tk = row_base + g;
+    const bool valid = tk < p.K;
+    const float rs = hdr->rstd[tk];
+    const float* xrow = p.x + (size_t)tk * H + 4 * c;
+#pragma unroll
+    for (int i = 0; i < KW; ++i) {
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (valid) v = *reinterpret_cast<const float4*>(xrow + 16 * (warp * KW + i));
+      __nv_bfloat16 h0, h1, h2, h3, l0, l1, l2, l3;
+      split_bf16(v.x * rs, h0, l0); split_bf16(v.y * rs, h1, l1);
+      split_bf16(v.z * rs, h2, l2); split_bf16(v.w * rs, h3, l3);
+      breg[i][0] = pack2(h0, h1); breg[i][1] = pack2(h2, h3);
+      breg[i][2] = pack2(l0, l1); breg[i][3] = pack2(l2, l3);
+    }
+  } else {
+    for (int idx = threadIdx.x; idx < NT * KSTEPS * 32; idx += kConsumerWarps * 32) {
+      const int l = idx & 31, ks = (idx >> 5) % KSTEPS, nt = idx / (32 * KSTEPS);
+      const int tk = nt * 8 + (l >> 2);
+      uint4 o = make_uint4(0u, 0u, 0u, 0u);
+      if (tk < p.K) {
+        const float rs = hdr->rstd[tk];
+        const float4 v = *reinterpret_cast<const float4*>(p.x + (size_t)tk * H + 16 * ks + 4 * (l & 3));
+        __nv_bfloat16 h0, h1, h2, h3, l0, l1, l2, l3;
+        split_bf16(v.x * rs, h0, l0); split_bf16(v.y * rs, h1, l1);
+        split_bf16(v.z * rs, h2, l2); split_bf16(v.w * rs, h3, l3);
+        o = make_uint4(pack2(h0, h1), pack2(h2, h3), pack2(l0, l1), pack2(l2, l3));
+      }
+      bfrag[idx] = o;
+    }
+    consumer_bar();
+  }
+
   uint32_t uc = 0;   // units consumed by this CTA so far
   int buf = 0;
   // partial-exchange source lanes: lane (g,c) ends up holding the sums of rows i = 2c and 2c+1 for token g
@@ -383,7 +418,7 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
 
   // weight of group e's output in block row `row` (0 = the row does not belong to the group).  Token slots of
   // the MMAs are the block rows themselves, for every group alike, so the accumulators can stay in registers
-  // across groups (the weight is folded into the activations) and y is touched once, at the very end.
+  // across groups (the weight multiplies the activations) and y is touched once, at the very end.
   auto row_weight = [&](int e, int row) -> float {
     if (e < n_static) return row < p.K ? (e < p.n_shared ? 1.0f : p.gamma) : 0.0f;
     if (row >= p.K) return 0.0f;
@@ -404,42 +439,6 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
 #pragma unroll
       for (int nt = 0; nt < NT; ++nt) wrow[nt] = row_weight(e, row_base + nt * 8 + g);
       const bool need_hi = NT > 1 && __any_sync(0xffffffffu, wrow[NT - 1] != 0.0f);   // any of rows 8..15 routed here
-
-      // ---- token fragments of this group
-      if constexpr (kRegB) {
-        const bool valid = wrow[0] != 0.0f;
-        const int tk = row_base + g;
-        const float rs = hdr->rstd[tk];
-        const float* xrow = p.x + (size_t)tk * H + 4 * c;
-#pragma unroll
-        for (int i = 0; i < KW; ++i) {
-          float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-          if (valid) v = *reinterpret_cast<const float4*>(xrow + 16 * (warp * KW + i));
-          __nv_bfloat16 h0, h1, h2, h3, l0, l1, l2, l3;
-          split_bf16(v.x * rs, h0, l0); split_bf16(v.y * rs, h1, l1);
-          split_bf16(v.z * rs, h2, l2); split_bf16(v.w * rs, h3, l3);
-          breg[i][0] = pack2(h0, h1); breg[i][1] = pack2(h2, h3);
-          breg[i][2] = pack2(l0, l1); breg[i][3] = pack2(l2, l3);
-        }
-      } else {
-        consumer_bar();   // everyone is done reading the previous group's fragments
-        for (int idx = threadIdx.x; idx < NT * KSTEPS * 32; idx += kConsumerWarps * 32) {
-          const int l = idx & 31, ks = (idx >> 5) % KSTEPS, nt = idx / (32 * KSTEPS);
-          const int slot = nt * 8 + (l >> 2);
-          uint4 o = make_uint4(0u, 0u, 0u, 0u);
-          if (row_weight(e, slot) != 0.0f) {
-            const int tk = slot;
-            const float rs = hdr->rstd[tk];
-            const float4 v = *reinterpret_cast<const float4*>(p.x + (size_t)tk * H + 16 * ks + 4 * (l & 3));
-            __nv_bfloat16 h0, h1, h2, h3, l0, l1, l2, l3;
-            split_bf16(v.x * rs, h0, l0); split_bf16(v.y * rs, h1, l1);
-            split_bf16(v.z * rs, h2, l2); split_bf16(v.w * rs, h3, l3);
-            o = make_uint4(pack2(h0, h1), pack2(h2, h3), pack2(l0, l1), pack2(l2, l3));
-          }
-          bfrag[idx] = o;
-        }
-        consumer_bar();
-      }
 
       for (int u = lo; u < hi; ++u, ++uc) {
         const uint32_t it = uc * kConsumerWarps + warp;
