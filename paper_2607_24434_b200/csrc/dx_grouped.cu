@@ -7,9 +7,11 @@
 // same 8 rows of W_u and the matching 8 columns of W_d.  A unit is
 // self-contained (its 8 activations feed only its own 8 columns of W_d), so the
 // down projection is fused in and nothing intermediate ever reaches HBM.  The
-// global unit list is split into equal contiguous ranges, one per CTA, so a CTA
-// touches at most a few experts and keeps its partial y in registers until the
-// expert changes; partials are then added to y with fp32 reductions.
+// global unit list is split into equal contiguous ranges, one per CTA.  The MMA
+// token slots are the block rows themselves for every group (a group's weight,
+// zero for rows outside it, multiplies the activations), so a CTA keeps its
+// partial y in registers across all its groups and adds it to y once, at the
+// end, with fp32 reductions.
 //
 // bf16 path (sm_100a): one elected producer thread streams each unit through a
 // shared-memory ring with bulk asynchronous copies (cp.async.bulk, completion on
@@ -120,10 +122,14 @@ __device__ __forceinline__ uint32_t pack2(__nv_bfloat16 lo16, __nv_bfloat16 hi16
 // Overlap with routing.  The groups that do not depend on the router (the
 // shared experts, and the draft expert in draft mode) are known from the layer
 // description alone.  The kernel is launched with programmatic stream
-// serialization right behind the routing kernel and streams those groups
-// first; only then does it wait for the routing kernel (griddepcontrol.wait),
-// read the work list and stream the routed groups.  Nothing is written to y
-// before that wait, because the routing kernel is what initialises y.
+// serialization behind the routing kernel, which lets it start before either
+// kernel has its input: the producer streams those groups at once, the
+// consumers begin when the routing kernel has published that the block is
+// final, and the routed groups are polled out of the work list as the routing
+// kernel writes it (fused entry points; otherwise the kernel simply waits for
+// the routing kernel first).  Nothing is written to y before the routing
+// kernel has completed (griddepcontrol.wait in front of the final reductions),
+// because the routing kernel is what initialises y.
 constexpr int kConsumerWarps = 8;
 constexpr int kThreads = (kConsumerWarps + 1) * 32;
 constexpr int kMaxSlots = 24;
