@@ -791,9 +791,9 @@ cudaError_t launch_bf16(dx_ctx* ctx, const DxExpertParams& p, cudaStream_t st) {
   cudaError_t e = cudaFuncSetAttribute(dx_experts_bf16_kernel<H, NT, TILES>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)smem);
   if (e != cudaSuccess) return e;
-  // One CTA per SM, minus the SMs the routing cluster (8 CTAs) runs on at the same time: a CTA of this kernel
+  // One CTA per SM, minus the SMs the routing cluster runs on at the same time: a CTA of this kernel
   // fills an SM, so a CTA that had to wait for a routing CTA's SM would start late and become the tail.
-  int grid = ctx->sm_count > 16 ? ctx->sm_count - 8 : ctx->sm_count;
+  int grid = ctx->sm_count > 16 ? ctx->sm_count - DX_ROUTE_CLUSTER : ctx->sm_count;
   if (TILES == 2) grid &= ~1;
   return dx_launch_pdl(DX_PDL_EXPERTS, dx_experts_bf16_kernel<H, NT, TILES>, dim3(grid), dim3(kThreads), smem, st, 1, p, n_slots);
 }

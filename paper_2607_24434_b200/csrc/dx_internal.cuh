@@ -18,6 +18,7 @@
 #define DX_MAX_ENTRIES (DX_MAX_SHARED + 1 + DX_MAX_PAIRS)
 #define DX_TILE_I 8            // intermediate rows per streamed weight tile
 #define DX_MAX_M 16            // accept rows
+#define DX_ROUTE_CLUSTER 4     // CTAs (and SMs) of the routing kernel; the expert kernel leaves them free
 
 // What the routing kernel hands to the expert kernels.  The routing-independent groups (shared experts, draft
 // expert) follow from the launch parameters alone; the routed groups are listed here, one per expert that some

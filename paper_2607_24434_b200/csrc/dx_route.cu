@@ -2,7 +2,8 @@
 // g_{l,e} of Eq. 4), the block's expert union and the pair permutation grouped
 // by expert (Eq. 2 / Eq. 3), and the work list the expert kernels consume.
 //
-// One thread-block cluster of 8 CTAs does all of it.  The contraction is split
+// One thread-block cluster of 4 CTAs does all of it (few SMs, because the
+// expert kernel runs beside it on all the others).  The contraction is split
 // over the hidden dimension: CTA c owns a slice of the columns (and, for narrow
 // layers, a share of the router rows).  Its part of the router matrix is a
 // constant and sits in registers before the previous kernel of the stream has
@@ -24,7 +25,7 @@ namespace cg = cooperative_groups;
 namespace {
 
 constexpr int kRouteThreads = 256;
-constexpr int kRouteCluster = 8;
+constexpr int kRouteCluster = DX_ROUTE_CLUSTER;
 constexpr int kRouteWarps = kRouteThreads / 32;
 
 __device__ __forceinline__ void unpack8(const uint4& r, float (&v)[8]) {
@@ -186,8 +187,8 @@ __device__ __forceinline__ void topk_gates(const DxRouteParams& p, const float* 
   }
 }
 
-// How the cluster divides the contraction: S column slices (the largest divisor of H/256 that is at most 8) of C
-// 256-column slabs each, times R = 8 / S shares of the router rows.
+// How the cluster divides the contraction: S column slices (the largest divisor of H/256 that is at most the
+// cluster size) of C 256-column slabs each, times R = cluster size / S shares of the router rows.
 struct RouteSplit {
   int S, R, C, slice, share, e_lo, e_hi;
   bool idle;
@@ -232,13 +233,16 @@ __global__ void __launch_bounds__(kRouteThreads) dx_route_kernel(DxRouteParams p
   const int col0 = sp.slice * sp.C * 256 + 8 * lane;   // this lane's first column; slab c adds 256 c
   const WT* Wr = reinterpret_cast<const WT*>(p.W_r);
 
-  // the first batch of this warp's router rows (first slab of the slice): constant data, fetched right away
-  RowRaw<WT> wpre[kRowsPerBatch];
+  // the first batch of this warp's router rows (first kPreSlabs slabs of the slice): constant data, fetched right away
+  constexpr int kPreSlabs = 2;
+  RowRaw<WT> wpre[kPreSlabs][kRowsPerBatch];
 #pragma unroll
-  for (int i = 0; i < kRowsPerBatch; ++i) {
-    const int e = sp.e_lo + warp + kRouteWarps * i;
-    if (e < sp.e_hi) wpre[i].load(Wr + (size_t)e * H + col0);
-  }
+  for (int c = 0; c < kPreSlabs; ++c)
+#pragma unroll
+    for (int i = 0; i < kRowsPerBatch; ++i) {
+      const int e = sp.e_lo + warp + kRouteWarps * i;
+      if (c < sp.C && e < sp.e_hi) wpre[c][i].load(Wr + (size_t)e * H + col0 + 256 * c);
+    }
   if (crank == 0)
     for (int e = threadIdx.x; e < E; e += kRouteThreads) s_bias[e] = p.bias ? p.bias[e] : 0.f;
   for (int i = threadIdx.x; i < DX_MAX_K * DX_MAX_TOPK; i += kRouteThreads) s_sel_z[i] = 0.f;
@@ -295,11 +299,11 @@ __global__ void __launch_bounds__(kRouteThreads) dx_route_kernel(DxRouteParams p
           }
         }
         RowRaw<WT> wr[kRowsPerBatch];
-        const bool pre = first_rows && c == 0;
 #pragma unroll
         for (int i = 0; i < kRowsPerBatch; ++i) {
           const int e = r0 + kRouteWarps * i;
-          if (pre) wr[i] = wpre[i];
+          if (first_rows && c == 0) wr[i] = wpre[0][i];
+          else if (first_rows && c == 1) wr[i] = wpre[1][i];
           else if (e < sp.e_hi) wr[i].load(Wr + (size_t)e * H + col0 + 256 * c);
         }
         if (rms && first_rows && warp == 0 && sp.share == 0) {
@@ -434,7 +438,7 @@ __global__ void __launch_bounds__(kRouteThreads) dx_route_kernel(DxRouteParams p
 
 template <typename WT, int TG>
 static cudaError_t launch_route_one(const DxRouteParams& p, cudaStream_t st) {
-  // CTA 0 holds one partial table per column slice (at most 8)
+  // CTA 0 holds one partial table per column slice (at most one per CTA of the cluster)
   const size_t smem = (size_t)kRouteCluster * ((size_t)p.K * p.E + p.K) * sizeof(float);
   // static + dynamic shared memory can pass the default 48 KB: opt in once per instantiation for the largest case
   static bool opted_in = false;
