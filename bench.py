@@ -425,6 +425,109 @@ def run_gpu(args):
         torch.distributed.destroy_process_group()
 
 
+def run_stack(args):
+    """configs[2] / configs[3]: a stack of MoE sub-layers (attention stubbed out, pre-norm residual form) with all
+    experts resident.  The draft stack is timed per token; the verify stack (routing + grouped SwiGLU per layer,
+    then greedy accept on the normalised final rows) is timed for K in {1, 2, 4, 8, 16} with block rows that follow
+    an AR(1) process (rho 0.9), and the union sizes per layer are reported with the bytes they imply."""
+    from paper_2607_24434_b200 import binding
+    torch.cuda.set_device(0)
+    device = torch.device("cuda", 0)
+    shape = synth.shape_moonlight() if args.moonlight else synth.shape_v2lite()
+    V = 163840 if args.moonlight else args.vocab
+    NLAY, H = args.stack_layers, shape.hidden
+    ctx = binding.Context(0)
+    layers = []
+    for l in range(NLAY):
+        w = synth.make_layer(shape, 7000 + l, device, zipf=args.zipf)
+        layers.append(binding.Layer.from_weights(ctx, w))
+        torch.cuda.synchronize()
+        del w
+    torch.cuda.empty_cache()
+    W_lm = synth.lm_head(V, H, 7999, torch.bfloat16, device)
+    exp_bytes = binding.expert_blob_bytes(shape, shape.inter)
+    peak, peak_kind = measured_peaks()
+    stream = torch.cuda.current_stream()
+
+    def timed_graph(body, reps):
+        side = torch.cuda.Stream(device=device)
+        side.wait_stream(stream)
+        with torch.cuda.stream(side):
+            body()
+        stream.wait_stream(side)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            body()
+        for _ in range(3):
+            g.replay()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(reps):
+            g.replay()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps
+
+    # ---- draft stack: one token through all layers
+    hd = [torch.empty((1, H), device=device) for _ in range(NLAY + 1)]
+    hd[0].copy_(synth.hidden_block(1, H, 7100, 0.0, device))
+    db = [{"topk_ids": torch.empty((shape.top_k,), dtype=torch.int32, device=device),
+           "topk_w": torch.empty((shape.top_k,), dtype=torch.float32, device=device)} for _ in range(NLAY)]
+
+    def draft_body():
+        for l in range(NLAY):
+            binding.moe_draft_step_residual(layers[l], hd[l], hd[l + 1], db[l])
+
+    draft_ms = timed_graph(draft_body, args.stack_reps)
+    draft_bytes = NLAY * ((shape.n_shared + 2) * exp_bytes + shape.n_experts * H * 2)
+    out = {"metric": "draft_stack_us_per_token", "value": draft_ms * 1e3, "unit": "us/token", "n_gpus": 1,
+           "higher_is_better": False, "data": "synthetic", "dtype": "bf16 weights, fp32 accumulate",
+           "config": {"workload": f"{'configs[3] Moonlight' if args.moonlight else 'configs[2] DeepSeek-V2-Lite'}-shaped "
+                                  f"stack of {NLAY} MoE sub-layers, experts resident "
+                                  f"({NLAY * (shape.n_experts + shape.n_shared + 1) * exp_bytes / 1e9:.1f} GB), "
+                                  f"AR(1) block rows (rho 0.9), Zipf router bias {'on' if args.zipf else 'off'}, "
+                                  f"vocab {V}; CUDA graph replay, {args.stack_reps} timed replays per point",
+                      "layers": NLAY},
+           "draft_gbs": draft_bytes / (draft_ms * 1e-3) / 1e9,
+           "draft_frac_of_8TBs": draft_bytes / (draft_ms * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
+           "draft_us_per_layer": draft_ms * 1e3 / NLAY, "peak_gbs": peak, "peak_kind": peak_kind, "verify": []}
+    # ---- verify stack for every block length
+    for K in (1, 2, 4, 8, 16):
+        hs = [torch.empty((K, H), device=device) for _ in range(NLAY + 1)]
+        hs[0].copy_(synth.hidden_block(K, H, 7200 + K, 0.9, device))
+        rb = [binding._routing_buffers(shape, K, device) for _ in range(NLAY)]
+        draft_tok = torch.zeros((K,), dtype=torch.int32, device=device)
+        abuf = {"target": torch.empty((K,), dtype=torch.int32, device=device),
+                "n_accept": torch.empty((1,), dtype=torch.int32, device=device),
+                "next_token": torch.empty((1,), dtype=torch.int32, device=device)}
+
+        def layers_body():
+            for l in range(NLAY):
+                binding.moe_verify_block_residual(layers[l], hs[l], hs[l + 1], rb[l])
+
+        def accept_body():
+            binding.spec_accept(ctx, hs[NLAY], W_lm, draft_tok, True, abuf)
+
+        ms_layers = timed_graph(layers_body, args.stack_reps)
+        ms_accept = timed_graph(accept_body, args.stack_reps)
+        if ctx.device_status() != 0:
+            raise RuntimeError("device status word set during the stack run")
+        unions = [int(rb[l]["union_count"].item()) for l in range(NLAY)]
+        vbytes = sum((u + shape.n_shared) * exp_bytes + shape.n_experts * H * 2 for u in unions)
+        out["verify"].append({
+            "K": K, "stack_ms": ms_layers, "accept_ms": ms_accept,
+            "tokens_per_s": K / ((ms_layers + ms_accept) * 1e-3),
+            "union_mean": float(np.mean(unions)), "union_min": min(unions), "union_max": max(unions),
+            "layers_gbs": vbytes / (ms_layers * 1e-3) / 1e9,
+            "layers_frac_of_8TBs": vbytes / (ms_layers * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
+            "layers_frac_of_measured": vbytes / (ms_layers * 1e-3) / 1e9 / peak,
+            "accept_gbs": V * H * 2 / (ms_accept * 1e-3) / 1e9})
+        del hs, rb
+    print(json.dumps(out))
+
+
 def run_offload(args):
     """configs[4]: offloaded V2-Lite-shaped stack.  Routed experts live in pinned host memory; each layer has an HBM
     cache of 16 slots with LRU eviction; shared and draft experts are resident.  Per decode step: K draft tokens go
@@ -605,8 +708,13 @@ def main():
     ap.add_argument("--cpu-vocab", type=int, default=16384, help="vocabulary rows in the CPU-baseline sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="time eager launches instead of a CUDA graph replay")
-    ap.add_argument("--workload", default="layer", choices=["layer", "offload"],
-                    help="layer: configs[1] (default, the driver's line); offload: configs[4] expert-cache workload")
+    ap.add_argument("--stack-layers", type=int, default=26)
+    ap.add_argument("--stack-reps", type=int, default=20)
+    ap.add_argument("--moonlight", action="store_true", help="stack workload: Moonlight shapes (sigmoid router, vocab 163840)")
+    ap.add_argument("--zipf", action="store_true", help="stack workload: Zipf(1.1) router bias")
+    ap.add_argument("--workload", default="layer", choices=["layer", "offload", "stack"],
+                    help="layer: configs[1] (default, the driver's line); offload: configs[4] expert-cache workload; "
+                         "stack: configs[2] / configs[3] layer stacks, K sweep and draft us per token")
     ap.add_argument("--offload-layers", type=int, default=4)
     ap.add_argument("--q4", action="store_true",
                     help="offload workload: keep the host pool 4-bit block-quantised (Q4_0 blocks)")
@@ -618,6 +726,8 @@ def main():
         args.warmup = 3
     if args.workload == "offload" and args.impl != "reference":
         run_offload(args)
+    elif args.workload == "stack" and args.impl != "reference":
+        run_stack(args)
     elif args.impl == "reference":
         run_reference(args)
     else:
