@@ -201,6 +201,25 @@ dx_status moe_verify_block_residual(dx_layer* layer, const float* h_in, float* h
 dx_status moe_draft_step_residual(dx_layer* layer, const float* h_in, float* h_out, int32_t* topk_ids,
                                   float* topk_w, void* stream);
 
+/* ---- the drafter through a whole stack in one launch --------------------------------------------------------
+ * The chain  h_{l+1} = moe_draft_step_residual(layer_l, h_l),  l = 0 .. n_layers-1  (Eq. 5 per layer, one
+ * token), run by ONE persistent kernel: a draft step reads so few bytes per layer that the gaps between
+ * per-layer launches are a visible share of its time, and the weights of layer l+1 can stream while layer l is
+ * still being reduced.  dx_stack_create records the layer handles (host array of n_layers handles, all of one
+ * context and one shape, bf16 weights, no expert cache attached; DX_ERR_SHAPE / DX_ERR_UNSUPPORTED otherwise)
+ * and owns the scratch rows; the layers must outlive the stack.  moe_draft_stack: h_in, h_out [H] fp32 device,
+ * 16-byte aligned, distinct; topk_ids [n_layers, k] int32 and topk_w [n_layers, k] fp32 device or NULL (the
+ * selection of every layer, gates as in Eq. 4).  Every expert of every layer must be resident
+ * (DX_ERR_NOT_RESIDENT).  The kernel is launched cooperatively (one CTA per SM, all resident at once): a
+ * device that cannot place the grid fails the launch with DX_ERR_CUDA.  Its CTAs wait on one another with
+ * bounded polls; a wait that runs out sets DX_DEV_WAIT_EXPIRED in dx_device_status and the call's outputs are
+ * then undefined.  One call at a time per stack. */
+typedef struct dx_stack dx_stack;
+dx_status dx_stack_create(dx_ctx* ctx, dx_layer* const* layers, int32_t n_layers, dx_stack** out);
+dx_status dx_stack_destroy(dx_stack* stack);
+dx_status moe_draft_stack(dx_stack* stack, const float* h_in, float* h_out, int32_t* topk_ids, float* topk_w,
+                          void* stream);
+
 /* ---- exact greedy verification: Algorithm 1, "verify" and "accept the target-consistent prefix" -------------
  * h [M,H] fp32: row i is the hidden state that predicts draft token i (M = K, or K+1 to also get the token
  * after a fully accepted block).  W_lm [V,H] in w_dtype.  draft [K] int32.  Outputs (device):

@@ -67,6 +67,9 @@ SIGNATURES = {
     "moe_draft_step": (_I, [_P, _P, _P, _P, _P, _P]),
     "moe_draft_step_topr": (_I, [_P, _P, _P, _I, _I, _P, _P, _P]),
     "moe_draft_step_residual": (_I, [_P, _P, _P, _P, _P, _P]),
+    "dx_stack_create": (_I, [_P, C.POINTER(_P), C.c_int32, C.POINTER(_P)]),
+    "dx_stack_destroy": (_I, [_P]),
+    "moe_draft_stack": (_I, [_P, _P, _P, _P, _P, _P]),
     "moe_verify_block": (_I, [_P, _P, _I, _P, _P, _P, _P, _P, _P, _P, _P, _P]),
     "moe_verify_route": (_I, [_P, _P, _I, _P, _P, _P, _P, _P, _P, _P, _P, _P]),
     "moe_verify_experts": (_I, [_P, _P, _I, _P, _P]),
@@ -319,6 +322,43 @@ def moe_draft_step_residual(layer: Layer, h_in: torch.Tensor, h_out: Optional[to
         h_out = torch.empty_like(h_in)
     _check(layer.lib.moe_draft_step_residual(layer.handle, _ptr(h_in), _ptr(h_out), _ptr(out["topk_ids"]),
                                              _ptr(out["topk_w"]), _stream()), "moe_draft_step_residual")
+    out["h"] = h_out
+    return out
+
+
+class DraftStack:
+    """A stack of layers the drafter runs through in one persistent launch (Eq. 5 per layer, one token)."""
+
+    def __init__(self, ctx: Context, layers: Sequence[Layer]):
+        self.lib, self.ctx, self.layers = ctx.lib, ctx, list(layers)
+        arr = (_P * len(self.layers))(*[l.handle for l in self.layers])
+        h = _P()
+        _check(self.lib.dx_stack_create(ctx.handle, arr, len(self.layers), C.byref(h)), "dx_stack_create")
+        self.handle = h
+
+    def close(self) -> None:
+        if self.handle:
+            self.lib.dx_stack_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def moe_draft_stack(stack: DraftStack, h_in: torch.Tensor, h_out: Optional[torch.Tensor] = None,
+                    out: Optional[Dict[str, torch.Tensor]] = None) -> Dict[str, torch.Tensor]:
+    """h_out = the drafter's hidden row after every layer of the stack; topk_ids / topk_w [n_layers, k]."""
+    sh, n = stack.layers[0].shape, len(stack.layers)
+    if out is None:
+        out = {"topk_ids": torch.empty((n, sh.top_k), dtype=torch.int32, device=h_in.device),
+               "topk_w": torch.empty((n, sh.top_k), dtype=torch.float32, device=h_in.device)}
+    if h_out is None:
+        h_out = torch.empty_like(h_in)
+    _check(stack.lib.moe_draft_stack(stack.handle, _ptr(h_in), _ptr(h_out), _ptr(out["topk_ids"]),
+                                     _ptr(out["topk_w"]), _stream()), "moe_draft_stack")
     out["h"] = h_out
     return out
 

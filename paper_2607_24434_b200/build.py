@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libdraftexpert.so")
-SOURCES = ["dx_api.cu", "dx_route.cu", "dx_grouped.cu", "dx_accept.cu", "dx_cache.cu", "dx_controller.cu", "dx_eval.cu"]
+SOURCES = ["dx_api.cu", "dx_route.cu", "dx_grouped.cu", "dx_accept.cu", "dx_cache.cu", "dx_controller.cu", "dx_eval.cu", "dx_draft_stack.cu"]
 
 
 def _newest_source_mtime() -> float:

@@ -398,6 +398,110 @@ extern "C" dx_status moe_verify_block_residual(dx_layer* L, const float* h_in, f
   return do_pair(L, h_in, K, h_out, o, false, true, st);
 }
 
+// ---- draft stack: Eq. 5 through a whole stack of layers in one persistent kernel -----------------------------
+extern "C" dx_status dx_stack_create(dx_ctx* ctx, dx_layer* const* layers, int32_t n_layers, dx_stack** out) {
+  if (!ctx || !layers || !out) return DX_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (n_layers < 1 || n_layers > 1024) return DX_ERR_UNSUPPORTED;
+  for (int l = 0; l < n_layers; ++l) {
+    dx_layer* L = layers[l];
+    if (!L || L->ctx != ctx) return DX_ERR_INVALID_ARG;
+    const dx_layer_desc &d = L->desc, &d0 = layers[0]->desc;
+    if (d.weight_dtype != DX_DTYPE_BF16 || L->cache) return DX_ERR_UNSUPPORTED;   // resident bf16 experts only
+    if (d.hidden != d0.hidden || d.n_experts != d0.n_experts || d.top_k != d0.top_k || d.inter != d0.inter ||
+        d.n_shared != d0.n_shared || d.shared_inter != d0.shared_inter || d.draft_inter != d0.draft_inter ||
+        d.score_fn != d0.score_fn || d.norm_topk != d0.norm_topk || d.routed_scale != d0.routed_scale)
+      return DX_ERR_SHAPE;
+    if (!L->W_r) return DX_ERR_NOT_RESIDENT;
+  }
+  dx_stack* s = new (std::nothrow) dx_stack();
+  if (!s) return DX_ERR_OOM;
+  s->ctx = ctx;
+  s->n_layers = n_layers;
+  s->layers = new (std::nothrow) dx_layer*[n_layers];
+  s->desc_host = new (std::nothrow) DxStackLayer[n_layers]();
+  s->desc_dev = nullptr; s->scratch = nullptr;
+  if (!s->layers || !s->desc_host) { delete[] s->layers; delete[] s->desc_host; delete s; return DX_ERR_OOM; }
+  for (int l = 0; l < n_layers; ++l) s->layers[l] = layers[l];
+  const dx_layer_desc& d = layers[0]->desc;
+  cudaError_t e = cudaMalloc(&s->desc_dev, sizeof(DxStackLayer) * n_layers);
+  s->zword_off = sizeof(float) * (size_t)n_layers * d.hidden;
+  s->sync_off = s->zword_off + sizeof(unsigned long long) * (size_t)n_layers * d.n_experts;
+  s->scratch_bytes = s->sync_off + sizeof(unsigned int) * n_layers;
+  if (e == cudaSuccess) e = cudaMalloc(&s->scratch, s->scratch_bytes);
+  if (e != cudaSuccess) {
+    ctx->last_cuda = e;
+    dx_stack_destroy(s);
+    return e == cudaErrorMemoryAllocation ? DX_ERR_OOM : DX_ERR_CUDA;
+  }
+  *out = s;
+  return DX_OK;
+}
+
+extern "C" dx_status dx_stack_destroy(dx_stack* s) {
+  if (!s) return DX_ERR_INVALID_ARG;
+  cudaFree(s->desc_dev);
+  cudaFree(s->scratch);
+  delete[] s->layers;
+  delete[] s->desc_host;
+  delete s;
+  return DX_OK;
+}
+
+extern "C" dx_status moe_draft_stack(dx_stack* s, const float* h_in, float* h_out, int32_t* topk_ids, float* topk_w,
+                                     void* stream) {
+  if (!s || !h_in || !h_out || h_in == h_out) return DX_ERR_INVALID_ARG;
+  if (((uintptr_t)h_in) % 16 || ((uintptr_t)h_out) % 16) return DX_ERR_INVALID_ARG;
+  dx_ctx* ctx = s->ctx;
+  cudaStream_t st = (cudaStream_t)stream;
+  const dx_layer_desc& d = s->layers[0]->desc;
+  // every expert of every layer has to be resident, and the layers' tables and the descriptors up to date
+  bool changed = false;
+  for (int l = 0; l < s->n_layers; ++l) {
+    dx_layer* L = s->layers[l];
+    for (int i = 0; i < L->table_len; ++i)
+      if (!L->table_host[i] && !(i == d.n_shared && d.draft_inter == 0)) return DX_ERR_NOT_RESIDENT;
+    dx_status u = upload_table(L, st);
+    if (u != DX_OK) return u;
+    DxStackLayer now{};
+    now.table = L->table_dev;
+    now.W_r = L->W_r;
+    now.bias = L->bias;
+    now.gamma = L->desc.draft_gamma;
+    DxStackLayer& have = s->desc_host[l];
+    if (have.table != now.table || have.W_r != now.W_r || have.bias != now.bias || have.gamma != now.gamma) {
+      have = now;
+      changed = true;
+    }
+  }
+  // (the source outlives the copy: it belongs to the stack)
+  cudaError_t e = cudaSuccess;
+  if (changed)
+    e = cudaMemcpyAsync(s->desc_dev, s->desc_host, sizeof(DxStackLayer) * s->n_layers, cudaMemcpyHostToDevice, st);
+  if (e == cudaSuccess) e = cudaMemsetAsync(s->scratch, 0, s->scratch_bytes, st);
+  DX_CUDA(ctx, e);
+  DxStackParams p{};
+  p.layers = s->desc_dev;
+  p.n_layers = s->n_layers;
+  p.h_in = h_in;
+  p.h_out = h_out;
+  p.delta = reinterpret_cast<float*>(s->scratch);
+  p.zword = reinterpret_cast<unsigned long long*>(s->scratch + s->zword_off);
+  p.sync = reinterpret_cast<unsigned int*>(s->scratch + s->sync_off);
+  p.topk_ids = topk_ids;
+  p.topk_w = topk_w;
+  p.dev_status = ctx->dev_status;
+  p.H = d.hidden; p.E = d.n_experts; p.k = d.top_k; p.score_fn = d.score_fn; p.norm_topk = d.norm_topk;
+  p.scale = d.routed_scale;
+  p.n_shared = d.n_shared;
+  p.shared_tiles = d.n_shared ? d.shared_inter / DX_TILE_I : 0;
+  p.draft_tiles = d.draft_inter / DX_TILE_I;
+  p.routed_tiles = d.inter / DX_TILE_I;
+  DX_CUDA(ctx, dx_launch_draft_stack(ctx, p, st));
+  ctx->launches++;
+  return DX_OK;
+}
+
 // ---- evaluation terms of Sec. 3.3 (no training involved) -----------------------------------------------------
 extern "C" dx_status moe_missing_residual(dx_layer* L, const float* h, int32_t K, float* m, int32_t* topk_ids,
                                           float* topk_w, void* stream) {

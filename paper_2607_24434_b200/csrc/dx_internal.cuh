@@ -147,6 +147,42 @@ struct DxExpertParams {
   unsigned int* handover;
 };
 
+// Persistent draft stack (dx_draft_stack.cu): one descriptor per layer in device memory ...
+struct DxStackLayer {
+  const void* const* table;   // the layer's device blob table
+  const void* W_r;            // [E,H] bf16
+  const float* bias;          // [E] or null
+  float gamma;
+  int pad;
+};
+// ... and the launch parameters
+struct DxStackParams {
+  const DxStackLayer* layers;
+  int n_layers;
+  const float* h_in;          // [H]
+  float* h_out;               // [H]
+  // all zero at launch:
+  float* delta;               // [n_layers][H] what layer l adds to the hidden row
+  unsigned long long* zword;  // [n_layers][E] router logits exchanged between the CTAs, (1 << 32 | float bits)
+  unsigned int* sync;         // [n_layers] CTAs that have added all of their share of layer l
+  int32_t* topk_ids;          // [n_layers][k] or null
+  float* topk_w;              // [n_layers][k] or null
+  int32_t* dev_status;
+  int H, E, k, score_fn, norm_topk;
+  float scale;
+  int n_shared, shared_tiles, draft_tiles, routed_tiles;
+};
+struct dx_stack {
+  dx_ctx* ctx;
+  int n_layers;
+  dx_layer** layers;          // host copy of the handles
+  DxStackLayer* desc_host;    // what desc_dev holds (all zero at first)
+  DxStackLayer* desc_dev;
+  unsigned char* scratch;     // delta rows, logit words, arrival counters (cleared before every launch)
+  size_t scratch_bytes, zword_off, sync_off;
+};
+cudaError_t dx_launch_draft_stack(dx_ctx* ctx, const DxStackParams& p, cudaStream_t st);
+
 // launchers (each returns the cudaError_t of the launch)
 cudaError_t dx_launch_route(const DxRouteParams& p, int weight_dtype, cudaStream_t st);
 cudaError_t dx_launch_experts(dx_ctx* ctx, const DxExpertParams& p, int weight_dtype, int K, cudaStream_t st);

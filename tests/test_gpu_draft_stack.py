@@ -1,0 +1,91 @@
+"""The drafter through a whole stack in one persistent launch (Eq. 5 per layer, pre-norm residual form): checked
+layer by layer against the checker -- routing on the checker's own hidden row (exact outside near-ties), then the
+checker advanced with the selection the kernel reported -- and against the chain of per-layer launches."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import moe_oracle as O
+from paper_2607_24434_b200 import synth
+from tests.helpers import Y_TIGHT, check_routing, row_rel_err
+
+pytestmark = pytest.mark.gpu
+
+
+def _stack_case(shape, n_layers, seed, zipf=False, reps=1):
+    from paper_2607_24434_b200 import binding
+    ctx = binding.Context(0)
+    refs, layers = [], []
+    for l in range(n_layers):
+        w = synth.make_layer(shape, seed + 10 * l, "cuda", zipf=zipf)
+        refs.append(synth.layer_to_numpy(w))
+        layers.append(binding.Layer.from_weights(ctx, w))
+        del w
+    stack = binding.DraftStack(ctx, layers)
+    for rep in range(reps):
+        h0 = synth.hidden_block(1, shape.hidden, seed + 77 * rep, 0.0, "cuda")
+        out = binding.moe_draft_stack(stack, h0)
+        torch.cuda.synchronize()
+        assert ctx.device_status() == 0
+        ids = out["topk_ids"].cpu().numpy()
+        gates = out["topk_w"].cpu().numpy()
+        # the checker, advanced with the kernel's own selection
+        h = h0.cpu().numpy().astype(np.float64)
+        near = 0
+        for l in range(n_layers):
+            _, ids_ref, _, z_ref = O.stack_layer_draft(h, refs[l])
+            near += check_routing(shape, z_ref, ids_ref, ids[l][None])
+            h, _, g_ref, _ = O.stack_layer_draft(h, refs[l], forced_ids=ids[l][None])
+            assert np.allclose(gates[l], g_ref[0], rtol=2e-3, atol=1e-6), l
+        assert near <= max(1, n_layers // 4)
+        assert row_rel_err(out["h"].cpu().numpy(), h).max() <= Y_TIGHT
+        # the chain of per-layer launches takes the same path (same selection => same row up to summation order)
+        hc = h0
+        same = True
+        for l in range(n_layers):
+            o = binding.moe_draft_step_residual(layers[l], hc)
+            same = same and np.array_equal(o["topk_ids"].cpu().numpy(), ids[l])
+            hc = o["h"]
+        torch.cuda.synchronize()
+        if same:
+            assert row_rel_err(out["h"].cpu().numpy(), hc.cpu().numpy().astype(np.float64)).max() <= 2e-3
+    stack.close()
+    for L in layers:
+        L.close()
+    ctx.close()
+
+
+def test_draft_stack_small_bf16():
+    sh = dataclasses.replace(synth.shape_tiny(), weight_dtype=synth.DTYPE_BF16, n_experts=16, top_k=3)
+    _stack_case(sh, 7, seed=910, reps=3)
+
+
+def test_draft_stack_single_layer():
+    sh = dataclasses.replace(synth.shape_tiny(), weight_dtype=synth.DTYPE_BF16, hidden=512, inter=256, shared_inter=256)
+    _stack_case(sh, 1, seed=920)
+
+
+def test_draft_stack_v2lite():
+    _stack_case(synth.shape_v2lite(), 4, seed=930, reps=2)
+
+
+def test_draft_stack_moonlight_zipf():
+    _stack_case(synth.shape_moonlight(), 3, seed=940, zipf=True)
+
+
+def test_draft_stack_refuses_mixed_shapes_and_fp32():
+    from paper_2607_24434_b200 import binding
+    ctx = binding.Context(0)
+    a = binding.Layer.from_weights(ctx, synth.make_layer(synth.shape_tiny(), 1, "cuda"))
+    with pytest.raises(binding.DxError):
+        binding.DraftStack(ctx, [a])          # fp32 weights
+    shb = dataclasses.replace(synth.shape_tiny(), weight_dtype=synth.DTYPE_BF16)
+    b = binding.Layer.from_weights(ctx, synth.make_layer(shb, 2, "cuda"))
+    c = binding.Layer.from_weights(ctx, synth.make_layer(dataclasses.replace(shb, n_experts=16), 3, "cuda"))
+    with pytest.raises(binding.DxError):
+        binding.DraftStack(ctx, [b, c])
+    for L in (a, b, c):
+        L.close()
+    ctx.close()
