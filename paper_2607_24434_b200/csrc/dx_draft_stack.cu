@@ -124,36 +124,43 @@ __global__ void __launch_bounds__(kStackThreads, 1) dx_draft_stack_kernel(DxStac
 
   if (warp == kStackConsumers) {
     // ---------------------------------------------------------------- producer
-    uint32_t it = 0;
+    uint32_t it = 0, slot = 0, phase = 0;   // chunk counter, its ring slot and that slot's phase bit
     const uint64_t l2pol = l2_evict_first_policy();
-    auto push = [&](const unsigned char* blob, int j) {   // unit j of a blob: one chunk per consumer warp
-      const unsigned char* src = blob + (size_t)j * UNIT_BYTES;
-#pragma unroll 1
-      for (int w = 0; w < kStackConsumers; ++w, ++it) {
-        const uint32_t s = it % (uint32_t)n_slots, ph = (it / (uint32_t)n_slots) & 1u;
-        mbar_wait(smem_u32(&hdr->empty[s]), ph ^ 1u, abort_flag);
-        const uint32_t fb = smem_u32(&hdr->full[s]);
-        mbar_arrive_expect_tx(fb, CHUNK);
-        bulk_g2s(smem_u32(ring + (size_t)s * CHUNK), src + (size_t)w * CHUNK, CHUNK, fb, l2pol);
-      }
+    auto static_unit = [&](int l, int u) -> const unsigned char* {
+      const int grp = u < p.n_shared * p.shared_tiles ? u / p.shared_tiles : p.n_shared;
+      const int first = grp < p.n_shared ? grp * p.shared_tiles : p.n_shared * p.shared_tiles;
+      const unsigned char* blob = reinterpret_cast<const unsigned char*>(p.layers[l].table[grp]);
+      return blob ? blob + (size_t)(u - first) * UNIT_BYTES : nullptr;
+    };
+    auto push_chunk = [&](const unsigned char* src) {
+      mbar_wait(smem_u32(&hdr->empty[slot]), phase ^ 1u, abort_flag);
+      const uint32_t fb = smem_u32(&hdr->full[slot]);
+      mbar_arrive_expect_tx(fb, CHUNK);
+      bulk_g2s(smem_u32(ring + (size_t)slot * CHUNK), src, CHUNK, fb, l2pol);
+      ++it;
+      if (++slot == (uint32_t)n_slots) { slot = 0; phase ^= 1u; }
     };
     for (int l = 0; l < L; ++l) {
-      const void* const* table = p.layers[l].table;
       if (lane == 0) {
+#pragma unroll 1
         for (int u = s_lo; u < s_hi; ++u) {
-          const int grp = u < p.n_shared * p.shared_tiles ? u / p.shared_tiles : p.n_shared;
-          const int first = grp < p.n_shared ? grp * p.shared_tiles : p.n_shared * p.shared_tiles;
-          const unsigned char* blob = reinterpret_cast<const unsigned char*>(table[grp]);
-          if (blob) push(blob, u - first);
-          else *abort_flag = 1;   // (the entry point refuses stacks with missing experts; never expected)
+          const unsigned char* src = static_unit(l, u);
+          if (src) {
+#pragma unroll 1
+            for (int w = 0; w < kStackConsumers; ++w) push_chunk(src + (size_t)w * CHUNK);
+          } else {
+            *abort_flag = 1;   // (the entry point refuses stacks with missing experts; never expected)
+          }
         }
       }
       __syncwarp();
       asm volatile("bar.sync 2, 64;" ::: "memory");   // the router warp knows this layer's routed expert
       if (lane == 0) {
         const unsigned char* blob = hdr->r_blob;
-        for (int u = r_lo; u < r_hi; ++u)
-          if (blob) push(blob, u);
+        if (blob) {
+#pragma unroll 1
+          for (int c = r_lo * kStackConsumers; c < r_hi * kStackConsumers; ++c) push_chunk(blob + (size_t)c * CHUNK);
+        }
       }
       __syncwarp();
     }
@@ -336,7 +343,7 @@ __global__ void __launch_bounds__(kStackThreads, 1) dx_draft_stack_kernel(DxStac
 
   // ------------------------------------------------------------------ consumers
   const int g = lane >> 2, c = lane & 3;
-  uint32_t uc = 0;   // units consumed so far
+  uint32_t cslot = (uint32_t)warp, cphase = 0;   // ring slot (and its phase bit) of this warp's chunk of the next unit
   int buf = 0;
   for (int l = 0; l < L; ++l) {
     asm volatile("bar.sync 3, 288;" ::: "memory");   // the router warp has advanced the hidden row to this layer
@@ -360,8 +367,9 @@ __global__ void __launch_bounds__(kStackThreads, 1) dx_draft_stack_kernel(DxStac
 
     // one unit with weight wu
     auto unit = [&](float wu) {
-      const uint32_t it = uc * kStackConsumers + warp;
-      const uint32_t s = it % (uint32_t)n_slots, ph = (it / (uint32_t)n_slots) & 1u;
+      const uint32_t s = cslot, ph = cphase;
+      cslot += kStackConsumers;   // (a ring has more slots than a unit has chunks: at most one wrap)
+      if (cslot >= (uint32_t)n_slots) { cslot -= (uint32_t)n_slots; cphase ^= 1u; }
       const uint4* A = reinterpret_cast<const uint4*>(ring + (size_t)s * CHUNK) + lane;
       mbar_wait(smem_u32(&hdr->full[s]), ph, abort_flag);
       // gate (rows 0..7 of the tile) and up (rows 8..15) over this warp's slice of the hidden dimension
@@ -405,7 +413,6 @@ __global__ void __launch_bounds__(kStackThreads, 1) dx_draft_stack_kernel(DxStac
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&hdr->empty[s]));
-      ++uc;
     };
 
     const float gamma = p.layers[l].gamma;

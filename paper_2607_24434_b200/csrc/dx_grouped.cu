@@ -152,7 +152,7 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
 
   if (warp == kConsumerWarps) {
     // ------------------------------------------------------------ producer
-    uint32_t it = 0;   // chunk counter
+    uint32_t it = 0, slot = 0, phase = 0;   // chunk counter, its ring slot and that slot's phase bit
     const uint64_t l2pol = l2_evict_first_policy();
     auto issue = [&](int e0, int e1, int lo_u, int hi_u) {
       for (int e = e0; e < e1; ++e) {
@@ -164,11 +164,11 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
           const unsigned char* src = blob + (size_t)(u - b) * UNIT_BYTES;
 #pragma unroll 1
           for (int w = 0; w < kConsumerWarps; ++w, ++it) {
-            const uint32_t s = it % (uint32_t)n_slots, ph = (it / (uint32_t)n_slots) & 1u;
-            mbar_wait(smem_u32(&hdr->empty[s]), ph ^ 1u, abort_flag);
-            const uint32_t fb = smem_u32(&hdr->full[s]);
+            mbar_wait(smem_u32(&hdr->empty[slot]), phase ^ 1u, abort_flag);
+            const uint32_t fb = smem_u32(&hdr->full[slot]);
             mbar_arrive_expect_tx(fb, CHUNK);
-            bulk_g2s(smem_u32(ring + (size_t)s * CHUNK), src + (size_t)w * CHUNK, CHUNK, fb, l2pol);
+            bulk_g2s(smem_u32(ring + (size_t)slot * CHUNK), src + (size_t)w * CHUNK, CHUNK, fb, l2pol);
+            if (++slot == (uint32_t)n_slots) { slot = 0; phase ^= 1u; }
           }
         }
       }
@@ -335,7 +335,7 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
     consumer_bar();
   }
 
-  uint32_t uc = 0;   // units consumed by this CTA so far
+  uint32_t cslot = (uint32_t)warp, cphase = 0;   // ring slot (and its phase bit) of this warp's chunk of the next unit
   int buf = 0;
   // partial-exchange source lanes: lane (g,c) ends up holding the sums of rows i = 2c and 2c+1 for token g
   const int src0 = (2 * c) * 4 + (g >> 1), src1 = src0 + 4;
@@ -365,9 +365,10 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
       for (int nt = 0; nt < NT; ++nt) wrow[nt] = row_weight(e, row_base + nt * 8 + g);
       const bool need_hi = NT > 1 && __any_sync(0xffffffffu, wrow[NT - 1] != 0.0f);   // any of rows 8..15 routed here
 
-      for (int u = lo; u < hi; ++u, ++uc) {
-        const uint32_t it = uc * kConsumerWarps + warp;
-        const uint32_t s = it % (uint32_t)n_slots, ph = (it / (uint32_t)n_slots) & 1u;
+      for (int u = lo; u < hi; ++u) {
+        const uint32_t s = cslot, ph = cphase;
+        cslot += kConsumerWarps;   // (a ring has more slots than a unit has chunks: at most one wrap)
+        if (cslot >= (uint32_t)n_slots) { cslot -= (uint32_t)n_slots; cphase ^= 1u; }
         const uint4* A = reinterpret_cast<const uint4*>(ring + (size_t)s * CHUNK) + lane;
         mbar_wait(smem_u32(&hdr->full[s]), ph, abort_flag);
 

@@ -45,6 +45,7 @@ __device__ __forceinline__ bool flag_wait(const unsigned int* word) {
 // after which every wait of the CTA falls through so the CTA still terminates.
 #define DX_WAIT_LIMIT (1u << 22)
 __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try_wait(bar, parity)) return;   // the common case, kept out of the counted loop
   for (uint32_t it = 0; it < DX_WAIT_LIMIT; ++it) {
     if (mbar_try_wait(bar, parity)) return;
     if ((it & 63u) == 63u && *abort_flag) return;
