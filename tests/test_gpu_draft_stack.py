@@ -75,6 +75,45 @@ def test_draft_stack_moonlight_zipf():
     _stack_case(synth.shape_moonlight(), 3, seed=940, zipf=True)
 
 
+def test_draft_stack_wide_sigmoid_router_no_shared():
+    """256 experts (eight logit words per lane), top-8, sigmoid scores with a routed scale, no shared expert."""
+    sh = dataclasses.replace(synth.shape_tiny(), weight_dtype=synth.DTYPE_BF16, hidden=1024, n_experts=256, top_k=8,
+                             n_shared=0, shared_inter=0, score_fn=synth.SCORE_SIGMOID, routed_scale=2.5)
+    _stack_case(sh, 3, seed=950, zipf=True)
+
+
+def test_draft_stack_graph_replay():
+    """The launch (scratch clear + cooperative kernel) captured in a CUDA graph and replayed on new inputs."""
+    from paper_2607_24434_b200 import binding
+    sh = dataclasses.replace(synth.shape_tiny(), weight_dtype=synth.DTYPE_BF16, hidden=512, n_experts=32, top_k=4)
+    ctx = binding.Context(0)
+    refs, layers = [], []
+    for l in range(5):
+        w = synth.make_layer(sh, 960 + l, "cuda")
+        refs.append(synth.layer_to_numpy(w))
+        layers.append(binding.Layer.from_weights(ctx, w))
+    stack = binding.DraftStack(ctx, layers)
+    h_in = synth.hidden_block(1, sh.hidden, 1, 0.0, "cuda")
+    out = binding.moe_draft_stack(stack, h_in)           # warm-up outside the capture (descriptor upload)
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=side):
+        binding.moe_draft_stack(stack, h_in, out["h"], out)
+    for rep in range(3):
+        h_in.copy_(synth.hidden_block(1, sh.hidden, 970 + rep, 0.0, "cuda"))
+        g.replay()
+        torch.cuda.synchronize()
+        assert ctx.device_status() == 0
+        ids = out["topk_ids"].cpu().numpy()
+        h = h_in.cpu().numpy().astype(np.float64)
+        for l in range(5):
+            h = O.stack_layer_draft(h, refs[l], forced_ids=ids[l][None])[0]
+        assert row_rel_err(out["h"].cpu().numpy(), h).max() <= Y_TIGHT, rep
+    stack.close()
+    ctx.close()
+
+
 def test_draft_stack_refuses_mixed_shapes_and_fp32():
     from paper_2607_24434_b200 import binding
     ctx = binding.Context(0)
