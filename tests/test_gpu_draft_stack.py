@@ -125,6 +125,14 @@ def test_draft_stack_refuses_mixed_shapes_and_fp32():
     c = binding.Layer.from_weights(ctx, synth.make_layer(dataclasses.replace(shb, n_experts=16), 3, "cuda"))
     with pytest.raises(binding.DxError):
         binding.DraftStack(ctx, [b, c])
-    for L in (a, b, c):
+    # routed experts not resident: the call (not the kernel) reports it
+    d = binding.Layer.from_weights(ctx, synth.make_layer(shb, 4, "cuda"), routed_resident=False)
+    st = binding.DraftStack(ctx, [b, d])
+    with pytest.raises(binding.DxError):
+        binding.moe_draft_stack(st, synth.hidden_block(1, shb.hidden, 5, 0.0, "cuda"))
+    torch.cuda.synchronize()
+    assert ctx.device_status() == 0
+    st.close()
+    for L in (a, b, c, d):
         L.close()
     ctx.close()
