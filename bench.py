@@ -102,11 +102,13 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def build_workload(binding, ctx, shape, n_layers, K, V, seed0, device):
+def build_workload(binding, ctx, shape, n_layers, K, V, seed0, device, q4=False):
     """Packed layers, hidden blocks, LM head and draft tokens, all resident on the GPU."""
     layers, blocks, hosts = [], [], []
     for i in range(n_layers):
         w = synth.make_layer(shape, seed0 + i, device, zipf=True)
+        if q4:
+            w = synth.quantize_layer(w)      # experts 4-bit block-quantised, resident in that form
         L = binding.Layer.from_weights(ctx, w)
         torch.cuda.synchronize()
         del w
@@ -134,7 +136,7 @@ def run_gpu(args):
     shape = synth.shape_v2lite()
     K, V, NL = args.block, args.vocab, args.layers
     ctx = binding.Context(local)
-    layers, blocks, W_lm = build_workload(binding, ctx, shape, NL, K, V, 1000 + 50 * rank, device)
+    layers, blocks, W_lm = build_workload(binding, ctx, shape, NL, K, V, 1000 + 50 * rank, device, args.q4_resident)
     H = shape.hidden
     stream = torch.cuda.current_stream()
 
@@ -227,7 +229,7 @@ def run_gpu(args):
     torch.cuda.synchronize()
     clocks = sampler.stop() if rank == 0 else None
     union = [int(rb[li]["union_count"].item()) for li in range(NL)]
-    exp_bytes = shape.expert_bytes()
+    exp_bytes = binding.expert_blob_bytes(layers[0].shape, shape.inter)   # bytes of one expert as it is streamed
     exp_ms_isolated = [x.elapsed_time(y) for x, y, _ in t_exp]
     exp_alg = [(union[li] + shape.n_shared) * exp_bytes + 2 * K * H * 4 for _, _, li in t_exp]
 
@@ -381,41 +383,46 @@ def run_gpu(args):
     value = multi.throughput(units_all, total_ms)
     # the drafter through the rotating layers chained as a stack (Eq. 5 per layer, pre-norm residual form) in one
     # persistent launch: the "draft step us per token" figure, per layer
-    dstack = binding.DraftStack(ctx, layers)
+    dstack = binding.DraftStack(ctx, layers) if not args.q4_resident else None
     h_stack = torch.empty((1, H), device=device)
 
     def stack_once():
         binding.moe_draft_stack(dstack, blocks[0][:1], h_stack)
 
-    side3 = torch.cuda.Stream(device=device)
-    side3.wait_stream(stream)
-    with torch.cuda.stream(side3):
-        stack_once()
-    stream.wait_stream(side3)
-    torch.cuda.synchronize()
-    gs = torch.cuda.CUDAGraph()
-    with torch.cuda.graph(gs, stream=side3):
-        stack_once()
-    for _ in range(3):
-        gs.replay()
-    torch.cuda.synchronize()
-    s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    s0.record(stream)
-    for _ in range(50):
-        gs.replay()
-    s1.record(stream)
-    torch.cuda.synchronize()
-    stack_us = s0.elapsed_time(s1) * 1e3 / 50
-    if ctx.device_status() != 0:
-        raise RuntimeError("device status word set during the draft stack")
-    dstack.close()
+    stack_us = None
+    if dstack is not None:
+        side3 = torch.cuda.Stream(device=device)
+        side3.wait_stream(stream)
+        with torch.cuda.stream(side3):
+            stack_once()
+        stream.wait_stream(side3)
+        torch.cuda.synchronize()
+        gs = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(gs, stream=side3):
+            stack_once()
+        for _ in range(3):
+            gs.replay()
+        torch.cuda.synchronize()
+        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s0.record(stream)
+        for _ in range(50):
+            gs.replay()
+        s1.record(stream)
+        torch.cuda.synchronize()
+        stack_us = s0.elapsed_time(s1) * 1e3 / 50
+        if ctx.device_status() != 0:
+            raise RuntimeError("device status word set during the draft stack")
+        dstack.close()
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "bf16 weights, fp32 accumulate", "data": "synthetic",
+        "dtype": ("4-bit block-quantised experts (fp16 scale per 32 weights) de-quantised in the kernel, bf16 router "
+                  "and LM head, fp32 accumulate") if args.q4_resident else "bf16 weights, fp32 accumulate",
+        "data": "synthetic",
         "config": {"workload": "configs[1]: DeepSeek-V2-Lite-shaped MoE layer (H 2048, 64 experts x 1408, top-6, "
                                "2 shared + 1 draft expert, Zipf(1.1) router bias); step = draft step (1 token) + "
-                               f"verify block K={K} + greedy accept over vocab {V}",
+                               f"verify block K={K} + greedy accept over vocab {V}"
+                               + ("; experts resident in HBM as 4-bit blocks" if args.q4_resident else ""),
                    "block_tokens": K, "vocab": V, "layers_rotated": NL,
                    "l2": f"inputs larger than L2: steps rotate over {NL} independently seeded layers "
                          f"({NL * (shape.n_experts + shape.n_shared + 1) * exp_bytes / 1e9:.1f} GB of weights)",
@@ -431,8 +438,8 @@ def run_gpu(args):
         "roofline": {"kernel": "dx_experts_bf16_kernel (grouped SwiGLU of the verify block)", "bound": "hbm",
                      "achieved": verify_gbs, "peak": peak, "unit": "GB/s", "frac": verify_gbs / peak,
                      "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBs": verify_gbs / NOMINAL_HBM_GBS,
-                     "traffic": args.traffic if args.traffic is not None else NCU_TRAFFIC_RATIO * float(
-                         np.mean(exp_alg)),
+                     "traffic": args.traffic if args.traffic is not None else (
+                         None if args.q4_resident else NCU_TRAFFIC_RATIO * float(np.mean(exp_alg))),
                      "traffic_source": "ncu capture of a 2-layer case scaled by algorithmic bytes (see profiles/)",
                      "ms_per_launch": float(np.mean(exp_ms)),
                      "ms_per_launch_isolated": float(np.mean(exp_ms_isolated)),
@@ -447,14 +454,15 @@ def run_gpu(args):
                     "accept_ms": acc_ms, "accept_gbs": acc_bytes / (acc_ms * 1e-3) / 1e9,
                     "accept_frac_of_peak": acc_bytes / (acc_ms * 1e-3) / 1e9 / peak},
         "graph_components": comp,
-        "draft_stack": {"layers": NL, "us_per_token": stack_us, "us_per_layer": stack_us / NL,
-                        "gbs": NL * draft_bytes / (stack_us * 1e-6) / 1e9,
-                        "frac_of_nominal_8TBs": NL * draft_bytes / (stack_us * 1e-6) / 1e9 / NOMINAL_HBM_GBS,
-                        "path": "moe_draft_stack: the rotating layers chained as a stack, one persistent cooperative "
-                                "launch per token (CUDA graph replay, 50 tokens)"},
+        "draft_stack": None if stack_us is None else {
+            "layers": NL, "us_per_token": stack_us, "us_per_layer": stack_us / NL,
+            "gbs": NL * draft_bytes / (stack_us * 1e-6) / 1e9,
+            "frac_of_nominal_8TBs": NL * draft_bytes / (stack_us * 1e-6) / 1e9 / NOMINAL_HBM_GBS,
+            "path": "moe_draft_stack: the rotating layers chained as a stack, one persistent cooperative "
+                    "launch per token (CUDA graph replay, 50 tokens)"},
         "clocks": clocks,
     }
-    if world == 1 and not args.no_cpu_baseline:
+    if world == 1 and not args.no_cpu_baseline and not args.q4_resident:
         out["cpu_baseline"] = cpu_baseline(shape, K, V, sample_vocab=args.cpu_vocab)
     print(json.dumps(out))
     if world > 1:
@@ -771,6 +779,8 @@ def main():
     ap.add_argument("--offload-layers", type=int, default=4)
     ap.add_argument("--q4", action="store_true",
                     help="offload workload: keep the host pool 4-bit block-quantised (Q4_0 blocks)")
+    ap.add_argument("--q4-resident", action="store_true",
+                    help="layer workload: experts resident in HBM as 4-bit blocks, de-quantised in the expert kernel")
     ap.add_argument("--offload-steps", type=int, default=24)
     ap.add_argument("--traffic", type=float, default=None,
                     help="ncu DRAM bytes per launch of the dominant kernel, if known")

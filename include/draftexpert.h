@@ -22,7 +22,13 @@
  *   - A context carries one set of device scratch buffers; calls that share a context must be issued on one
  *     stream (or otherwise ordered).  Use one context per concurrent stream.
  *   - Matrices are row-major.  Hidden states, outputs, gate weights and logits are fp32; weights are fp32 or
- *     bf16 as stated by weight_dtype; all accumulation is fp32.
+ *     bf16 as stated by weight_dtype; all accumulation is fp32.  DX_DTYPE_Q4: the expert weights (shared, draft,
+ *     routed) are 4-bit block-quantised, the format of the paper's mobile runs (Sec. 4): every row of W_g, W_u
+ *     [inter, hidden] and W_d [hidden, inter] in blocks of 32 weights, 18 bytes each -- an fp16 scale d, then 16
+ *     bytes whose low / high nibbles are the codes of weights j / j + 16; weight = d * (code - 8), evaluated
+ *     exactly (no rounding of the product).  The router of such a layer is bf16.  The experts stay 4-bit in HBM
+ *     and are de-quantised inside the streaming loop of the expert kernel, so a Q4 expert costs 0.94 bytes per
+ *     weight of HBM traffic instead of 2.  Every intermediate size must then be a multiple of 32.
  *   - Limits: block length K <= 16, experts E <= 256, top-k <= 8, shared experts <= 8, every intermediate size
  *     a multiple of 8; hidden a multiple of 256 up to 8192 for fp32 weights and one of 256, 512, 1024, 2048
  *     for bf16 weights.  Outside them: DX_ERR_UNSUPPORTED.
@@ -53,7 +59,7 @@ enum {
 };
 
 enum { DX_SCORE_SOFTMAX = 0, DX_SCORE_SIGMOID = 1 };
-enum { DX_DTYPE_FP32 = 0, DX_DTYPE_BF16 = 1 };
+enum { DX_DTYPE_FP32 = 0, DX_DTYPE_BF16 = 1, DX_DTYPE_Q4 = 2 /* experts 4-bit, router bf16 */ };
 
 /* Codes a kernel may leave in the device status word (0 = clean). */
 enum {
@@ -106,7 +112,10 @@ int64_t dx_kernel_launches(dx_ctx* ctx);
  * The kernels stream each expert from ONE contiguous "blob" in a tile-major layout of the library's choosing
  * (the same number of bytes as the three matrices).  dx_expert_blob_bytes gives its size;
  * dx_pack_expert fills a blob from the three canonical row-major matrices (all device pointers; the blob must
- * be 128-byte aligned; runs on `stream`).  Blobs can be copied around freely (host pool, cache slots). */
+ * be 128-byte aligned; runs on `stream`).  Blobs can be copied around freely (host pool, cache slots).
+ * DX_DTYPE_Q4: Wg, Wu, Wd point to the matrices' 4-bit blocks (uint8 [rows][cols/32][18], device, 2-byte aligned)
+ * and the blob keeps the codes 4-bit (inter * (hidden/128*144 + hidden/256*192) bytes: the codes in the order the
+ * kernel's fragments want them, each 32-weight block's scale next to them). */
 dx_status dx_expert_blob_bytes(const dx_layer_desc* desc, int32_t inter, size_t* bytes_out);
 dx_status dx_pack_expert(dx_ctx* ctx, const dx_layer_desc* desc, int32_t inter,
                          const void* Wg, const void* Wu, const void* Wd, void* blob_out, void* stream);

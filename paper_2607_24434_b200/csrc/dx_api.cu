@@ -104,7 +104,8 @@ static dx_status check_desc(const dx_layer_desc* d) {
   if (!d) return DX_ERR_INVALID_ARG;
   if (d->hidden <= 0 || d->n_experts <= 0 || d->top_k <= 0 || d->inter <= 0 || d->n_shared < 0) return DX_ERR_SHAPE;
   if (d->top_k > d->n_experts) return DX_ERR_SHAPE;
-  if (d->weight_dtype != DX_DTYPE_FP32 && d->weight_dtype != DX_DTYPE_BF16) return DX_ERR_INVALID_ARG;
+  if (d->weight_dtype != DX_DTYPE_FP32 && d->weight_dtype != DX_DTYPE_BF16 && d->weight_dtype != DX_DTYPE_Q4)
+    return DX_ERR_INVALID_ARG;
   if (d->score_fn != DX_SCORE_SOFTMAX && d->score_fn != DX_SCORE_SIGMOID) return DX_ERR_INVALID_ARG;
   if (d->hidden > DX_MAX_H || d->hidden % 256 || d->n_experts > DX_MAX_E || d->top_k > DX_MAX_TOPK ||
       d->n_shared > DX_MAX_SHARED)
@@ -112,13 +113,22 @@ static dx_status check_desc(const dx_layer_desc* d) {
   if (d->inter % DX_TILE_I || (d->n_shared && (d->shared_inter <= 0 || d->shared_inter % DX_TILE_I)) ||
       d->draft_inter < 0 || d->draft_inter % DX_TILE_I)
     return DX_ERR_UNSUPPORTED;
-  if (d->weight_dtype == DX_DTYPE_BF16 && !dx_bf16_hidden_supported(d->hidden)) return DX_ERR_UNSUPPORTED;
+  if (d->weight_dtype != DX_DTYPE_FP32 && !dx_bf16_hidden_supported(d->hidden)) return DX_ERR_UNSUPPORTED;
+  // 4-bit experts: quantisation blocks of 32 along the rows of W_d [hidden, inter]
+  if (d->weight_dtype == DX_DTYPE_Q4 &&
+      (d->inter % 32 || (d->n_shared && d->shared_inter % 32) || d->draft_inter % 32))
+    return DX_ERR_UNSUPPORTED;
   return DX_OK;
 }
 
 extern "C" dx_status dx_expert_blob_bytes(const dx_layer_desc* desc, int32_t inter, size_t* bytes_out) {
   if (!desc || !bytes_out) return DX_ERR_INVALID_ARG;
   if (inter <= 0 || inter % DX_TILE_I || desc->hidden <= 0 || desc->hidden % 256) return DX_ERR_UNSUPPORTED;
+  if (desc->weight_dtype == DX_DTYPE_Q4) {
+    if (inter % 32 || !dx_bf16_hidden_supported(desc->hidden)) return DX_ERR_UNSUPPORTED;
+    *bytes_out = (size_t)inter * dx_chunk_bytes(desc->hidden, true);   // inter / 8 units of 8 chunks
+    return DX_OK;
+  }
   *bytes_out = (size_t)3 * desc->hidden * inter * (desc->weight_dtype == DX_DTYPE_BF16 ? 2 : 4);
   return DX_OK;
 }
@@ -128,14 +138,20 @@ extern "C" dx_status dx_pack_expert(dx_ctx* ctx, const dx_layer_desc* desc, int3
   if (!ctx || !desc || !Wg || !Wu || !Wd || !blob_out) return DX_ERR_INVALID_ARG;
   if (inter <= 0 || inter % DX_TILE_I || desc->hidden <= 0 || desc->hidden % 256) return DX_ERR_UNSUPPORTED;
   if (((uintptr_t)blob_out) % 128) return DX_ERR_INVALID_ARG;
-  DX_CUDA(ctx, dx_launch_pack(desc->weight_dtype, desc->hidden, inter, Wg, Wu, Wd, blob_out, (cudaStream_t)stream));
+  if (desc->weight_dtype == DX_DTYPE_Q4) {
+    if (inter % 32 || !dx_bf16_hidden_supported(desc->hidden)) return DX_ERR_UNSUPPORTED;
+    if (((uintptr_t)Wg) % 2 || ((uintptr_t)Wu) % 2 || ((uintptr_t)Wd) % 2) return DX_ERR_INVALID_ARG;
+    DX_CUDA(ctx, dx_launch_pack_q4(desc->hidden, inter, Wg, Wu, Wd, blob_out, (cudaStream_t)stream));
+  } else {
+    DX_CUDA(ctx, dx_launch_pack(desc->weight_dtype, desc->hidden, inter, Wg, Wu, Wd, blob_out, (cudaStream_t)stream));
+  }
   ctx->launches++;
   return DX_OK;
 }
 
 extern "C" dx_status dx_q4_expert_bytes(const dx_layer_desc* desc, int32_t inter, size_t* bytes_out) {
   if (!desc || !bytes_out) return DX_ERR_INVALID_ARG;
-  if (desc->weight_dtype != DX_DTYPE_BF16) return DX_ERR_UNSUPPORTED;
+  if (desc->weight_dtype != DX_DTYPE_BF16 && desc->weight_dtype != DX_DTYPE_Q4) return DX_ERR_UNSUPPORTED;
   // blocks of 32 along the rows of W_g, W_u [inter, hidden] and of W_d [hidden, inter]
   if (inter <= 0 || inter % 32 || desc->hidden <= 0 || desc->hidden % 256) return DX_ERR_UNSUPPORTED;
   *bytes_out = (size_t)3 * desc->hidden * inter / 32 * 18;
@@ -145,6 +161,7 @@ extern "C" dx_status dx_q4_expert_bytes(const dx_layer_desc* desc, int32_t inter
 extern "C" dx_status dx_expand_q4_expert(dx_ctx* ctx, const dx_layer_desc* desc, int32_t inter, const void* q4_blob,
                                          void* blob_out, void* stream) {
   if (!ctx || !desc || !q4_blob || !blob_out) return DX_ERR_INVALID_ARG;
+  if (desc->weight_dtype != DX_DTYPE_BF16) return DX_ERR_UNSUPPORTED;   // the result is a bf16 blob
   size_t need = 0;
   dx_status s = dx_q4_expert_bytes(desc, inter, &need);
   if (s != DX_OK) return s;
@@ -271,7 +288,8 @@ static dx_status do_route(dx_layer* L, const float* h, int K, float* y, const Ro
   p.topk_ids = o.topk_ids; p.topk_w = o.topk_w;
   p.union_mask = (unsigned long long*)o.union_mask; p.union_ids = o.union_ids; p.union_count = o.union_count;
   p.offsets = o.offsets; p.perm = o.perm;
-  DX_CUDA(ctx, dx_launch_route(p, d.weight_dtype, st));
+  // (the router of a layer with 4-bit experts is bf16)
+  DX_CUDA(ctx, dx_launch_route(p, d.weight_dtype == DX_DTYPE_Q4 ? DX_DTYPE_BF16 : d.weight_dtype, st));
   ctx->launches++;
   return DX_OK;
 }
@@ -315,7 +333,7 @@ static dx_status do_experts(dx_layer* L, const float* h, int K, float* y, bool d
 // follow consumes and clears them.
 static dx_status do_pair(dx_layer* L, const float* h, int K, float* y, const RouteOut& o, bool draft, bool residual,
                          cudaStream_t st, int top_r = 1, bool use_draft_expert = true) {
-  const bool paired = L->desc.weight_dtype == DX_DTYPE_BF16;
+  const bool paired = L->desc.weight_dtype != DX_DTYPE_FP32;
   dx_status s = do_route(L, h, K, y, o, draft, residual, st, top_r, use_draft_expert, paired);
   if (s != DX_OK) return s;
   s = do_experts(L, h, K, y, draft && use_draft_expert, residual, st, 0, -1, true, paired);

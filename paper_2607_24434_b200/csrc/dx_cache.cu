@@ -275,6 +275,7 @@ extern "C" dx_status dx_layer_attach_cache(dx_layer* L, dx_cache* c, int32_t lay
 
 extern "C" dx_status expert_cache_set_q4(dx_cache* c, const dx_layer_desc* desc, int32_t inter) {
   if (!c || !desc) return DX_ERR_INVALID_ARG;
+  if (desc->weight_dtype != DX_DTYPE_BF16) return DX_ERR_UNSUPPORTED;   // the slots hold expanded bf16 blobs
   size_t q4 = 0, full = 0;
   dx_status s = dx_q4_expert_bytes(desc, inter, &q4);
   if (s != DX_OK) return s;

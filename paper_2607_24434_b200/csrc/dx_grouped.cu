@@ -51,7 +51,7 @@ namespace {
 // because the routing kernel is what initialises y.
 constexpr int kConsumerWarps = 8;
 constexpr int kThreads = (kConsumerWarps + 1) * 32;
-constexpr int kMaxSlots = 24;
+constexpr int kMaxSlots = 48;
 
 struct SmemHeader {
   unsigned long long full[kMaxSlots];
@@ -100,12 +100,27 @@ __device__ __forceinline__ void routed_range(int n_groups, const DxExpertParams&
 }
 
 // TILES = 2: CTA pairs, one tile of eight block rows each (see below); only with NT = 1
-template <int H, int NT, int TILES>
+// Eight 4-bit codes -> four bf16 pairs (a lane's A fragment of one contraction step).  Pair p sits in bits
+// [4p, 4p+4) (first element) and [16+4p, 16+4p+4) (second): 0x4300 | code is the bf16 number 128 + code, and
+// subtracting 136 leaves code - 8 exactly.
+__device__ __forceinline__ uint32_t q4_pair(uint32_t w) {
+  const uint32_t v = (w & 0x000F000Fu) | 0x43004300u;
+  const __nv_bfloat162 r = __hsub2(*reinterpret_cast<const __nv_bfloat162*>(&v), __floats2bfloat162_rn(136.f, 136.f));
+  return *reinterpret_cast<const uint32_t*>(&r);
+}
+__device__ __forceinline__ uint4 q4_fragment(uint32_t w) {
+  return make_uint4(q4_pair(w), q4_pair(w >> 4), q4_pair(w >> 8), q4_pair(w >> 12));
+}
+
+// Q4: the units hold 4-bit codes with one fp16 scale per 32 weights along the contraction (see dx_pack_q4_kernel);
+// the codes become bf16 fragments in registers and the scales multiply the accumulators of their block.
+template <int H, int NT, int TILES, bool Q4 = false>
 __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertParams p, int n_slots) {
   constexpr int KW = H / 128;        // phase-1 contraction steps per consumer warp
   constexpr int PW = H / 256;        // phase-2 row-tile pairs per consumer warp
   constexpr int KSTEPS = H / 16;
-  constexpr uint32_t CHUNK_A = KW * 512u, CHUNK_D = PW * 512u, CHUNK = CHUNK_A + CHUNK_D;
+  constexpr uint32_t CHUNK_A = Q4 ? KW * 144u : KW * 512u, CHUNK_D = Q4 ? PW * 192u : PW * 512u;
+  constexpr uint32_t CHUNK = CHUNK_A + CHUNK_D;
   constexpr uint32_t UNIT_BYTES = 8u * CHUNK;
   constexpr bool kRegB = (NT == 1);  // token fragments live in registers (else in shared memory)
 
@@ -378,6 +393,41 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
         for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
           for (int r = 0; r < 4; ++r) ch[nt][0][r] = ch[nt][1][r] = cl[nt][0][r] = cl[nt][1][r] = 0.f;
+        if constexpr (Q4) {
+          // one 32-wide quantisation block = two contraction steps: codes -> exact bf16 fragments, the products of
+          // the block go to fresh accumulators, and the rows' scales (gate row g, up row g) are applied to those
+          const unsigned char* Cq = ring + (size_t)s * CHUNK;
+          const uint2* Aq = reinterpret_cast<const uint2*>(Cq) + lane;
+          const __half2* S1 = reinterpret_cast<const __half2*>(Cq + KW * 128) + g;
+#pragma unroll
+          for (int b = 0; b < KW / 2; ++b) {
+            const uint2 cw = Aq[b * 32];
+            const float2 sc = __half22float2(S1[b * 8]);
+            const uint4 a0 = q4_fragment(cw.x), a1 = q4_fragment(cw.y);
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+              if (nt > 0 && !need_hi) continue;
+              uint32_t b00, b01, b02, b03, b10, b11, b12, b13;
+              if constexpr (kRegB) {
+                b00 = breg[2 * b][0]; b01 = breg[2 * b][1]; b02 = breg[2 * b][2]; b03 = breg[2 * b][3];
+                b10 = breg[2 * b + 1][0]; b11 = breg[2 * b + 1][1]; b12 = breg[2 * b + 1][2]; b13 = breg[2 * b + 1][3];
+              } else {
+                const uint4 f0 = bfrag[(nt * KSTEPS + warp * KW + 2 * b) * 32 + lane];
+                const uint4 f1 = bfrag[(nt * KSTEPS + warp * KW + 2 * b + 1) * 32 + lane];
+                b00 = f0.x; b01 = f0.y; b02 = f0.z; b03 = f0.w;
+                b10 = f1.x; b11 = f1.y; b12 = f1.z; b13 = f1.w;
+              }
+              // (activations in bf16 without the low halves: with 4-bit weights the tensor pipe, not the stream,
+              // sets the pace, and the rounding is far below the quantisation's own error)
+              (void)b02; (void)b03; (void)b12; (void)b13;
+              float t0[4] = {0.f, 0.f, 0.f, 0.f}, t1[4] = {0.f, 0.f, 0.f, 0.f};
+              mma_k16(t0, a0, b00, b01);
+              mma_k16(t1, a1, b10, b11);
+              ch[nt][0][0] = fmaf(sc.x, t0[0] + t1[0], ch[nt][0][0]); ch[nt][0][1] = fmaf(sc.x, t0[1] + t1[1], ch[nt][0][1]);
+              ch[nt][0][2] = fmaf(sc.y, t0[2] + t1[2], ch[nt][0][2]); ch[nt][0][3] = fmaf(sc.y, t0[3] + t1[3], ch[nt][0][3]);
+            }
+          }
+        } else {
 #pragma unroll
         for (int i = 0; i < KW; ++i) {
           const uint4 a = A[i * 32];
@@ -393,6 +443,7 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
               mma_k16(cl[nt][i & 1], a, b.z, b.w);
             }
           }
+        }
         }
         // re-fragment: C holds (gate|up row g, tokens 2c,2c+1); phase 2 wants rows (2c,2c+1) of token g
 #pragma unroll
@@ -433,6 +484,34 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
         buf ^= 1;
 
         // ---- phase 2: 8 columns of W_d x activations for this warp's output rows
+        if constexpr (Q4) {
+          // the eight columns of a unit lie in one quantisation block of W_d: one scale per output row
+          const unsigned char* Cq = ring + (size_t)s * CHUNK + CHUNK_A;
+          const uint32_t* Dq = reinterpret_cast<const uint32_t*>(Cq) + lane;
+          const uint2* S2 = reinterpret_cast<const uint2*>(Cq + PW * 128) + g;
+#pragma unroll
+          for (int q = 0; q < PW; ++q) {
+            const uint4 a = q4_fragment(Dq[q * 32]);
+            const uint2 sw = S2[q * 8];
+            const float2 s01 = __half22float2(*reinterpret_cast<const __half2*>(&sw.x));   // tile 2q: rows g, g + 8
+            const float2 s23 = __half22float2(*reinterpret_cast<const __half2*>(&sw.y));   // tile 2q + 1
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+              if (nt > 0 && !need_hi) continue;
+              float t0[4] = {0.f, 0.f, 0.f, 0.f}, t1[4] = {0.f, 0.f, 0.f, 0.f};
+              mma_k8(t0, a.x, a.y, bhi[nt]);
+              mma_k8(t1, a.z, a.w, bhi[nt]);
+              acc[nt][2 * q][0] = fmaf(s01.x, t0[0], acc[nt][2 * q][0]);
+              acc[nt][2 * q][1] = fmaf(s01.x, t0[1], acc[nt][2 * q][1]);
+              acc[nt][2 * q][2] = fmaf(s01.y, t0[2], acc[nt][2 * q][2]);
+              acc[nt][2 * q][3] = fmaf(s01.y, t0[3], acc[nt][2 * q][3]);
+              acc[nt][2 * q + 1][0] = fmaf(s23.x, t1[0], acc[nt][2 * q + 1][0]);
+              acc[nt][2 * q + 1][1] = fmaf(s23.x, t1[1], acc[nt][2 * q + 1][1]);
+              acc[nt][2 * q + 1][2] = fmaf(s23.y, t1[2], acc[nt][2 * q + 1][2]);
+              acc[nt][2 * q + 1][3] = fmaf(s23.y, t1[3], acc[nt][2 * q + 1][3]);
+            }
+          }
+        } else {
         const uint4* D = A + KW * 32;
 #pragma unroll
         for (int q = 0; q < PW; ++q) {
@@ -445,6 +524,7 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
             mma_k8(acc[nt][2 * q], a.x, a.y, blo[nt]);
             mma_k8(acc[nt][2 * q + 1], a.z, a.w, blo[nt]);
           }
+        }
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&hdr->empty[s]));
@@ -699,37 +779,127 @@ __global__ void dx_pack_fp32_kernel(const float* Wg, const float* Wu, const floa
   }
 }
 
-template <int H, int NT, int TILES>
+template <int H, int NT, int TILES, bool Q4>
 cudaError_t launch_bf16(dx_ctx* ctx, const DxExpertParams& p, cudaStream_t st) {
   const size_t hdr = (sizeof(SmemHeader) + 127) / 128 * 128;
   const size_t fixed = hdr + (size_t)2 * 8 * NT * 32 * 16 + (NT == 1 ? 0 : (size_t)NT * (H / 16) * 32 * 16);
-  const size_t chunk = (size_t)6 * H;
+  const size_t chunk = dx_chunk_bytes(H, Q4);
   int n_slots = (int)(((size_t)ctx->smem_optin - fixed) / chunk);
   if (n_slots > kMaxSlots) n_slots = kMaxSlots;
   if (n_slots < kConsumerWarps + 1) return cudaErrorInvalidConfiguration;   // a unit needs all its chunks at once
   const size_t smem = fixed + (size_t)n_slots * chunk;
-  cudaError_t e = cudaFuncSetAttribute(dx_experts_bf16_kernel<H, NT, TILES>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)smem);
+  cudaError_t e = cudaFuncSetAttribute(dx_experts_bf16_kernel<H, NT, TILES, Q4>,
+                                       cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   // One CTA per SM, minus the SMs the routing cluster runs on at the same time: a CTA of this kernel
   // fills an SM, so a CTA that had to wait for a routing CTA's SM would start late and become the tail.
   int grid = ctx->sm_count > 16 ? ctx->sm_count - DX_ROUTE_CLUSTER : ctx->sm_count;
   if (TILES == 2) grid &= ~1;
-  return dx_launch_pdl(DX_PDL_EXPERTS, dx_experts_bf16_kernel<H, NT, TILES>, dim3(grid), dim3(kThreads), smem, st, 1, p, n_slots);
+  return dx_launch_pdl(DX_PDL_EXPERTS, dx_experts_bf16_kernel<H, NT, TILES, Q4>, dim3(grid), dim3(kThreads), smem, st, 1,
+                       p, n_slots);
 }
 
-template <int H>
+template <int H, bool Q4>
 cudaError_t launch_bf16_h(dx_ctx* ctx, const DxExpertParams& p_in, int K, cudaStream_t st) {
   DxExpertParams p = p_in;
   p.row_tiles = 1;
-  if (K <= 8) return launch_bf16<H, 1, 1>(ctx, p, st);
+  if (K <= 8) return launch_bf16<H, 1, 1, Q4>(ctx, p, st);
   // two token tiles: fragments of both in shared memory where they fit next to a ring of at least one slot per
   // consumer warp and one to spare; otherwise CTA pairs with one tile each
   const size_t hdr = (sizeof(SmemHeader) + 127) / 128 * 128;
   const size_t fixed2 = hdr + (size_t)2 * 8 * 2 * 32 * 16 + (size_t)2 * (H / 16) * 32 * 16;
-  if (fixed2 + (size_t)(kConsumerWarps + 1) * 6 * H <= (size_t)ctx->smem_optin) return launch_bf16<H, 2, 1>(ctx, p, st);
+  if (fixed2 + (size_t)(kConsumerWarps + 1) * dx_chunk_bytes(H, Q4) <= (size_t)ctx->smem_optin)
+    return launch_bf16<H, 2, 1, Q4>(ctx, p, st);
   p.row_tiles = 2;
-  return launch_bf16<H, 1, 2>(ctx, p, st);
+  return launch_bf16<H, 1, 2, Q4>(ctx, p, st);
+}
+
+template <bool Q4>
+cudaError_t launch_bf16_any(dx_ctx* ctx, const DxExpertParams& p, int K, cudaStream_t st) {
+  switch (p.H) {
+    case 256: return launch_bf16_h<256, Q4>(ctx, p, K, st);
+    case 512: return launch_bf16_h<512, Q4>(ctx, p, K, st);
+    case 1024: return launch_bf16_h<1024, Q4>(ctx, p, K, st);
+    case 2048: return launch_bf16_h<2048, Q4>(ctx, p, K, st);
+    default: return cudaErrorInvalidConfiguration;
+  }
+}
+
+// Packed 4-bit units from the three matrices' Q4_0 blocks (18 bytes: fp16 scale d, then 16 bytes whose low /
+// high nibbles are elements j / j + 16 of the block; value = d * (code - 8)).  One unit = the chunks of the eight
+// consumer warps; a chunk holds, for warp w of unit j,
+//   [KW/2][32 lanes] 8 bytes: the code words of contraction steps 2b and 2b+1 of the lane's gate / up fragment,
+//   [KW/2][8 rows g] 2 halves: scales of gate row 8j+g and up row 8j+g in hidden block (w KW + 2b) / 2,
+//   [PW][32 lanes]   4 bytes: the code word of the lane's W_d fragment for row-tile pair w PW + i,
+//   [PW][8 rows g]   4 halves: scales of output rows 32q+g, +8, +16, +24 in intermediate block j / 4.
+// A code word holds a fragment's four bf16 pairs as (first, second) = bits [4p, 4p+4), [16+4p, 16+4p+4).
+__device__ __forceinline__ uint32_t q4_code(const unsigned char* m, int row, int col, int ncols) {
+  const unsigned char* blk = m + ((size_t)row * (ncols / 32) + col / 32) * 18;
+  const int j = col & 31;
+  return j < 16 ? (blk[2 + j] & 0x0Fu) : (uint32_t)(blk[2 + j - 16] >> 4);
+}
+__device__ __forceinline__ unsigned short q4_scale_bits(const unsigned char* m, int row, int col, int ncols) {
+  const unsigned char* blk = m + ((size_t)row * (ncols / 32) + col / 32) * 18;
+  return (unsigned short)(blk[0] | (blk[1] << 8));
+}
+
+__global__ void dx_pack_q4_kernel(const unsigned char* Wg, const unsigned char* Wu, const unsigned char* Wd,
+                                  unsigned char* blob, int H, int I) {
+  const int KW = H / 128, PW = H / 256;
+  const size_t chunk = (size_t)KW * 144 + (size_t)PW * 192, unit = 8 * chunk;
+  const int per_chunk = KW * 32 + KW * 8 + PW * 32 + PW * 32;   // code words and scales of phase 1, then of phase 2
+  const size_t n = (size_t)(I / 8) * 8 * per_chunk;
+  for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < n; idx += (size_t)gridDim.x * blockDim.x) {
+    const int j = (int)(idx / ((size_t)8 * per_chunk));
+    const int r = (int)(idx % ((size_t)8 * per_chunk));
+    const int w = r / per_chunk;
+    int t = r % per_chunk;
+    unsigned char* out = blob + (size_t)j * unit + (size_t)w * chunk;
+    if (t < KW * 32) {                       // phase-1 code word of contraction step i, lane l
+      const int i = t / 32, l = t % 32, g = l >> 2, c = l & 3;
+      const int col = 16 * (w * KW + i) + 4 * c, row = 8 * j + g;
+      uint32_t word = 0;
+      // pairs: (gate col, col+1), (up col, col+1), (gate col+2, col+3), (up col+2, col+3)
+#pragma unroll
+      for (int pp = 0; pp < 4; ++pp) {
+        const unsigned char* m = (pp & 1) ? Wu : Wg;
+        const int cc = col + 2 * (pp >> 1);
+        word |= q4_code(m, row, cc, H) << (4 * pp);
+        word |= q4_code(m, row, cc + 1, H) << (16 + 4 * pp);
+      }
+      *reinterpret_cast<uint32_t*>(out + (size_t)(i / 2) * 256 + l * 8 + (i & 1) * 4) = word;
+      continue;
+    }
+    t -= KW * 32;
+    if (t < KW * 8) {                        // phase-1 scales of block pair b, row g, gate | up
+      const int b = t / 16, g = (t % 16) / 2, which = t & 1;
+      const int col = 16 * (w * KW + 2 * b);
+      *reinterpret_cast<unsigned short*>(out + (size_t)KW * 128 + b * 32 + g * 4 + which * 2) =
+          q4_scale_bits(which ? Wu : Wg, 8 * j + g, col, H);
+      continue;
+    }
+    t -= KW * 8;
+    if (t < PW * 32) {                       // phase-2 code word of row-tile pair i, lane l
+      const int i = t / 32, l = t % 32, g = l >> 2, c = l & 3;
+      const int q = w * PW + i, col = 8 * j + 2 * c;
+      uint32_t word = 0;
+#pragma unroll
+      for (int pp = 0; pp < 4; ++pp) {
+        const int row = 32 * q + 8 * pp + g;
+        word |= q4_code(Wd, row, col, I) << (4 * pp);
+        word |= q4_code(Wd, row, col + 1, I) << (16 + 4 * pp);
+      }
+      *reinterpret_cast<uint32_t*>(out + (size_t)KW * 144 + (size_t)i * 128 + l * 4) = word;
+      continue;
+    }
+    t -= PW * 32;
+    {                                        // phase-2 scales of row-tile pair i, row g, the four rows g + 8m
+      const int i = t / 32, g = (t % 32) / 4, m = t & 3;
+      const int q = w * PW + i;
+      *reinterpret_cast<unsigned short*>(out + (size_t)KW * 144 + (size_t)PW * 128 + (size_t)i * 64 + g * 8 + m * 2) =
+          q4_scale_bits(Wd, 32 * q + 8 * m + g, 8 * j, I);
+    }
+  }
 }
 
 }  // namespace
@@ -740,13 +910,18 @@ cudaError_t dx_launch_experts(dx_ctx* ctx, const DxExpertParams& p, int weight_d
   if (weight_dtype == DX_DTYPE_FP32) {
     return dx_launch_pdl(DX_PDL_EXPERTS, dx_experts_fp32_kernel, dim3(ctx->sm_count * 4), dim3(256), 0, st, 1, p);
   }
-  switch (p.H) {
-    case 256: return launch_bf16_h<256>(ctx, p, K, st);
-    case 512: return launch_bf16_h<512>(ctx, p, K, st);
-    case 1024: return launch_bf16_h<1024>(ctx, p, K, st);
-    case 2048: return launch_bf16_h<2048>(ctx, p, K, st);
-    default: return cudaErrorInvalidConfiguration;
-  }
+  if (weight_dtype == DX_DTYPE_Q4) return launch_bf16_any<true>(ctx, p, K, st);
+  return launch_bf16_any<false>(ctx, p, K, st);
+}
+
+cudaError_t dx_launch_pack_q4(int H, int I, const void* Wg, const void* Wu, const void* Wd, void* blob,
+                              cudaStream_t st) {
+  const size_t n = (size_t)I * ((size_t)(H / 128) * 40 + (size_t)(H / 256) * 64);
+  int grid = (int)((n + 255) / 256);
+  if (grid > 4096) grid = 4096;
+  dx_pack_q4_kernel<<<grid, 256, 0, st>>>((const unsigned char*)Wg, (const unsigned char*)Wu, (const unsigned char*)Wd,
+                                          (unsigned char*)blob, H, I);
+  return cudaGetLastError();
 }
 
 cudaError_t dx_launch_expand_q4(int H, int I, const void* q4, void* blob, cudaStream_t st) {

@@ -188,6 +188,12 @@ cudaError_t dx_launch_route(const DxRouteParams& p, int weight_dtype, cudaStream
 cudaError_t dx_launch_experts(dx_ctx* ctx, const DxExpertParams& p, int weight_dtype, int K, cudaStream_t st);
 cudaError_t dx_launch_pack(int weight_dtype, int H, int I, const void* Wg, const void* Wu, const void* Wd,
                            void* blob, cudaStream_t st);
+// bytes of one consumer warp's chunk of a unit (a unit = 8 chunks = 8 intermediate rows of an expert)
+inline size_t dx_chunk_bytes(int H, bool q4) {
+  return q4 ? (size_t)(H / 128) * 144 + (size_t)(H / 256) * 192 : (size_t)6 * H;
+}
+cudaError_t dx_launch_pack_q4(int H, int I, const void* Wg, const void* Wu, const void* Wd, void* blob,
+                              cudaStream_t st);
 cudaError_t dx_launch_expand_q4(int H, int I, const void* q4, void* blob, cudaStream_t st);
 cudaError_t dx_launch_accept(dx_ctx* ctx, const float* h, int M, const void* W_lm, int V, int H, int w_dtype,
                              const int32_t* draft, int K, int rms_norm, int32_t* target, int32_t* n_accept,

@@ -26,6 +26,7 @@ SCORE_SOFTMAX = 0
 SCORE_SIGMOID = 1
 DTYPE_FP32 = 0
 DTYPE_BF16 = 1
+DTYPE_Q4 = 2      # experts 4-bit block-quantised (18-byte blocks of 32 weights), router bf16
 
 
 @dataclasses.dataclass(frozen=True)
@@ -47,11 +48,11 @@ class LayerShape:
 
     @property
     def torch_dtype(self) -> torch.dtype:
-        return torch.bfloat16 if self.weight_dtype == DTYPE_BF16 else torch.float32
+        return torch.float32 if self.weight_dtype == DTYPE_FP32 else torch.bfloat16
 
     @property
     def elem_bytes(self) -> int:
-        return 2 if self.weight_dtype == DTYPE_BF16 else 4
+        return 4 if self.weight_dtype == DTYPE_FP32 else 2
 
     def expert_bytes(self, inter: Optional[int] = None) -> int:
         return 3 * self.hidden * (self.inter if inter is None else inter) * self.elem_bytes
@@ -184,20 +185,21 @@ Q4_BLOCK = 32
 Q4_BLOCK_BYTES = 18
 
 
-def quantize_q4_0(w: torch.Tensor) -> torch.Tensor:
+def quantize_q4_0(w: torch.Tensor, device=None) -> torch.Tensor:
     """[R, C] float weights (C a multiple of 32) -> uint8 [R, C/32, 18] of Q4_0 blocks.  Per block: d = m / -8
     with m the entry of largest magnitude (the first one on ties), code = min(15, floor(x / d + 8.5)), and d is
     stored rounded to fp16."""
     R, Ccols = w.shape
     assert Ccols % Q4_BLOCK == 0
-    x = w.detach().to(torch.float32).cpu().reshape(R, Ccols // Q4_BLOCK, Q4_BLOCK)
+    x = w.detach().to(torch.float32).to(device if device is not None else "cpu").reshape(
+        R, Ccols // Q4_BLOCK, Q4_BLOCK)
     idx = x.abs().argmax(dim=2, keepdim=True)
     m = torch.gather(x, 2, idx)
     d = m / -8.0
     inv = torch.where(d != 0, 1.0 / d, torch.zeros_like(d))
     q = torch.clamp(torch.floor(x * inv + 8.5), max=15.0).to(torch.uint8)
     d16 = d.to(torch.float16)
-    out = torch.empty((R, Ccols // Q4_BLOCK, Q4_BLOCK_BYTES), dtype=torch.uint8)
+    out = torch.empty((R, Ccols // Q4_BLOCK, Q4_BLOCK_BYTES), dtype=torch.uint8, device=x.device)
     out[:, :, 0:2] = d16.view(torch.uint8).reshape(R, Ccols // Q4_BLOCK, 2)
     out[:, :, 2:] = q[:, :, :16] | (q[:, :, 16:] << 4)
     return out
@@ -207,6 +209,26 @@ def q4_expert_blob(Wg: torch.Tensor, Wu: torch.Tensor, Wd: torch.Tensor) -> torc
     """One routed expert as the host pool stores it when quantised: the Q4_0 blocks of W_g [I,H], W_u [I,H] and
     W_d [H,I], row-major, one matrix after the other (uint8, 3*H*I*18/32 bytes)."""
     return torch.cat([quantize_q4_0(Wg).reshape(-1), quantize_q4_0(Wu).reshape(-1), quantize_q4_0(Wd).reshape(-1)])
+
+
+def quantize_layer(layer: Dict[str, object]) -> Dict[str, object]:
+    """The layer with every expert matrix (shared, draft, routed) replaced by its Q4_0 blocks (uint8
+    [rows, cols/32, 18], on the layer's device); router and bias unchanged; ``shape.weight_dtype`` = DTYPE_Q4."""
+    sh: LayerShape = layer["shape"]
+    dev = layer["router"].device
+
+    def q(w: torch.Tensor) -> torch.Tensor:
+        return quantize_q4_0(w, dev)
+
+    def q_stack(w: torch.Tensor) -> torch.Tensor:
+        return torch.stack([q(w[e]) for e in range(w.shape[0])])
+
+    out: Dict[str, object] = {"shape": dataclasses.replace(sh, weight_dtype=DTYPE_Q4), "router": layer["router"],
+                              "bias": layer["bias"]}
+    out["shared"] = [tuple(q(w) for w in tr) for tr in layer["shared"]]
+    out["draft"] = None if layer["draft"] is None else tuple(q(w) for w in layer["draft"])
+    out["experts"] = tuple(q_stack(w) for w in layer["experts"])
+    return out
 
 
 def to_numpy_f32(t: torch.Tensor) -> np.ndarray:
