@@ -417,7 +417,8 @@ def run_gpu(args):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": ("4-bit block-quantised experts (fp16 scale per 32 weights) de-quantised in the kernel, bf16 router "
-                  "and LM head, fp32 accumulate") if args.q4_resident else "bf16 weights, fp32 accumulate",
+                  "and LM head, fp32 accumulate") if args.q4_resident else (
+                      "bf16 weights, activations as bf16 tensor-core operands, fp32 accumulate"),
         "data": "synthetic",
         "config": {"workload": "configs[1]: DeepSeek-V2-Lite-shaped MoE layer (H 2048, 64 experts x 1408, top-6, "
                                "2 shared + 1 draft expert, Zipf(1.1) router bias); step = draft step (1 token) + "

@@ -101,6 +101,15 @@ dx_status dx_create(int device, dx_ctx** out);
 dx_status dx_destroy(dx_ctx* ctx);
 /* Reads (and clears) the device status word.  Synchronises `stream` first. */
 dx_status dx_last_device_status(dx_ctx* ctx, void* stream, int32_t* dev_status_out);
+/* How bf16 experts are evaluated (DX_DTYPE_BF16 layers; set before the calls it should affect).  Off (the
+ * default): the activations -- the block rows, then the SwiGLU products -- enter the tensor cores as bf16, one
+ * rounding of at most 2^-9 relative each, as a bf16 model does; layer outputs are then within ~5e-3 of the row
+ * maximum of exact arithmetic on the same weights (the stated tolerance is 2e-2).  On: every activation is fed
+ * as a bf16 high part plus a bf16 residual (two products per fragment), which brings the outputs to ~1e-5 at
+ * twice the tensor work (a few percent of the expert kernel's time for blocks of up to 8 rows, about twice the
+ * time above).  fp32 layers and the single-token stack kernel always use fp32 activations; 4-bit layers always
+ * plain bf16. */
+dx_status dx_set_activation_split(dx_ctx* ctx, int32_t on);
 /* Last cudaError_t seen by this context as an int (0 = none). */
 int32_t dx_last_cuda_error(dx_ctx* ctx);
 /* Number of kernels this context has launched so far (for launch accounting by a caller). */

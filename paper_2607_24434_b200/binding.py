@@ -51,6 +51,7 @@ SIGNATURES = {
     "dx_create": (_I, [C.c_int, C.POINTER(_P)]),
     "dx_destroy": (_I, [_P]),
     "dx_last_device_status": (_I, [_P, _P, C.POINTER(_I)]),
+    "dx_set_activation_split": (_I, [_P, _I]),
     "dx_last_cuda_error": (_I, [_P]),
     "dx_kernel_launches": (C.c_int64, [_P]),
     "dx_expert_blob_bytes": (_I, [C.POINTER(LayerDesc), _I, C.POINTER(C.c_size_t)]),
@@ -139,12 +140,19 @@ def _desc(shape: LayerShape) -> LayerDesc:
 
 
 class Context:
-    def __init__(self, device: int = 0):
+    def __init__(self, device: int = 0, act_split: bool = False):
+        """``act_split``: evaluate bf16 experts with high + residual activation fragments (see
+        ``dx_set_activation_split``); the default feeds plain bf16 activations to the tensor cores."""
         self.lib = load()
         self.device = device
         h = _P()
         _check(self.lib.dx_create(device, C.byref(h)), "dx_create")
         self.handle = h
+        if act_split:
+            self.set_activation_split(True)
+
+    def set_activation_split(self, on: bool) -> None:
+        _check(self.lib.dx_set_activation_split(self.handle, 1 if on else 0), "dx_set_activation_split")
 
     def close(self) -> None:
         if self.handle:

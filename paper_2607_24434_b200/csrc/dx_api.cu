@@ -97,6 +97,12 @@ extern "C" dx_status dx_last_device_status(dx_ctx* ctx, void* stream, int32_t* o
   return DX_OK;
 }
 
+extern "C" dx_status dx_set_activation_split(dx_ctx* ctx, int32_t on) {
+  if (!ctx) return DX_ERR_INVALID_ARG;
+  ctx->act_split = on ? 1 : 0;
+  return DX_OK;
+}
+
 extern "C" int32_t dx_last_cuda_error(dx_ctx* ctx) { return ctx ? (int32_t)ctx->last_cuda : 0; }
 extern "C" int64_t dx_kernel_launches(dx_ctx* ctx) { return ctx ? ctx->launches : 0; }
 

@@ -24,6 +24,8 @@
 // needed.  All waits are bounded; an expired wait sets the device status word.
 #include <cuda_fp16.h>
 
+#include <type_traits>
+
 #include "dx_internal.cuh"
 #include "dx_stream.cuh"
 
@@ -114,8 +116,13 @@ __device__ __forceinline__ uint4 q4_fragment(uint32_t w) {
 
 // Q4: the units hold 4-bit codes with one fp16 scale per 32 weights along the contraction (see dx_pack_q4_kernel);
 // the codes become bf16 fragments in registers and the scales multiply the accumulators of their block.
-template <int H, int NT, int TILES, bool Q4 = false>
+// SPLIT: the activations (block rows, then the SwiGLU products) enter the tensor cores as bf16 high part plus bf16
+// residual, two products per fragment: results to ~1e-5 of the row maximum.  Without it they are plain bf16 (one
+// rounding of at most 2^-9 relative each), which halves the tensor work -- on this part `mma.sync` is slow enough
+// that the split's products take about as long as streaming the weights.
+template <int H, int NT, int TILES, bool Q4 = false, bool SPLIT = true>
 __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertParams p, int n_slots) {
+  static_assert(!(Q4 && SPLIT), "4-bit units are evaluated with plain bf16 activations");
   constexpr int KW = H / 128;        // phase-1 contraction steps per consumer warp
   constexpr int PW = H / 256;        // phase-2 row-tile pairs per consumer warp
   constexpr int KSTEPS = H / 16;
@@ -129,8 +136,10 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
   constexpr size_t HDR = (sizeof(SmemHeader) + 127) / 128 * 128;
   float4* partial = reinterpret_cast<float4*>(smem + HDR);                         // [2][8][NT][32]
   constexpr size_t PART = (size_t)2 * 8 * NT * 32 * 16;
-  uint4* bfrag = reinterpret_cast<uint4*>(smem + HDR + PART);                       // [NT][KSTEPS][32] if !kRegB
-  constexpr size_t BF = kRegB ? 0 : (size_t)NT * KSTEPS * 32 * 16;
+  // token fragments in shared memory if !kRegB: [NT][KSTEPS][32] of {hi, hi, lo, lo} (SPLIT) or {hi, hi}
+  using FragT = typename std::conditional<SPLIT, uint4, uint2>::type;
+  FragT* bfrag = reinterpret_cast<FragT*>(smem + HDR + PART);
+  constexpr size_t BF = kRegB ? 0 : (size_t)NT * KSTEPS * 32 * sizeof(FragT);
   unsigned char* ring = smem + HDR + PART + BF;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -345,7 +354,8 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
         split_bf16(v.z * rs, h2, l2); split_bf16(v.w * rs, h3, l3);
         o = make_uint4(pack2(h0, h1), pack2(h2, h3), pack2(l0, l1), pack2(l2, l3));
       }
-      bfrag[idx] = o;
+      if constexpr (SPLIT) bfrag[idx] = o;
+      else bfrag[idx] = make_uint2(o.x, o.y);
     }
     consumer_bar();
   }
@@ -412,10 +422,10 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
                 b00 = breg[2 * b][0]; b01 = breg[2 * b][1]; b02 = breg[2 * b][2]; b03 = breg[2 * b][3];
                 b10 = breg[2 * b + 1][0]; b11 = breg[2 * b + 1][1]; b12 = breg[2 * b + 1][2]; b13 = breg[2 * b + 1][3];
               } else {
-                const uint4 f0 = bfrag[(nt * KSTEPS + warp * KW + 2 * b) * 32 + lane];
-                const uint4 f1 = bfrag[(nt * KSTEPS + warp * KW + 2 * b + 1) * 32 + lane];
-                b00 = f0.x; b01 = f0.y; b02 = f0.z; b03 = f0.w;
-                b10 = f1.x; b11 = f1.y; b12 = f1.z; b13 = f1.w;
+                const FragT f0 = bfrag[(nt * KSTEPS + warp * KW + 2 * b) * 32 + lane];
+                const FragT f1 = bfrag[(nt * KSTEPS + warp * KW + 2 * b + 1) * 32 + lane];
+                b00 = f0.x; b01 = f0.y; b02 = 0u; b03 = 0u;
+                b10 = f1.x; b11 = f1.y; b12 = 0u; b13 = 0u;
               }
               // (activations in bf16 without the low halves: with 4-bit weights the tensor pipe, not the stream,
               // sets the pace, and the rounding is far below the quantisation's own error)
@@ -433,14 +443,14 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
           const uint4 a = A[i * 32];
           if constexpr (kRegB) {
             mma_k16(ch[0][i & 1], a, breg[i][0], breg[i][1]);
-            mma_k16(cl[0][i & 1], a, breg[i][2], breg[i][3]);
+            if constexpr (SPLIT) mma_k16(cl[0][i & 1], a, breg[i][2], breg[i][3]);
           } else {
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) {
               if (nt > 0 && !need_hi) continue;
-              const uint4 b = bfrag[(nt * KSTEPS + warp * KW + i) * 32 + lane];
+              const FragT b = bfrag[(nt * KSTEPS + warp * KW + i) * 32 + lane];
               mma_k16(ch[nt][i & 1], a, b.x, b.y);
-              mma_k16(cl[nt][i & 1], a, b.z, b.w);
+              if constexpr (SPLIT) mma_k16(cl[nt][i & 1], a, b.z, b.w);
             }
           }
         }
@@ -521,8 +531,10 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
             if (nt > 0 && !need_hi) continue;
             mma_k8(acc[nt][2 * q], a.x, a.y, bhi[nt]);
             mma_k8(acc[nt][2 * q + 1], a.z, a.w, bhi[nt]);
-            mma_k8(acc[nt][2 * q], a.x, a.y, blo[nt]);
-            mma_k8(acc[nt][2 * q + 1], a.z, a.w, blo[nt]);
+            if constexpr (SPLIT) {
+              mma_k8(acc[nt][2 * q], a.x, a.y, blo[nt]);
+              mma_k8(acc[nt][2 * q + 1], a.z, a.w, blo[nt]);
+            }
           }
         }
         }
@@ -779,48 +791,48 @@ __global__ void dx_pack_fp32_kernel(const float* Wg, const float* Wu, const floa
   }
 }
 
-template <int H, int NT, int TILES, bool Q4>
+template <int H, int NT, int TILES, bool Q4, bool SPLIT>
 cudaError_t launch_bf16(dx_ctx* ctx, const DxExpertParams& p, cudaStream_t st) {
   const size_t hdr = (sizeof(SmemHeader) + 127) / 128 * 128;
-  const size_t fixed = hdr + (size_t)2 * 8 * NT * 32 * 16 + (NT == 1 ? 0 : (size_t)NT * (H / 16) * 32 * 16);
+  const size_t fixed = hdr + (size_t)2 * 8 * NT * 32 * 16 + (NT == 1 ? 0 : (size_t)NT * (H / 16) * 32 * (SPLIT ? 16 : 8));
   const size_t chunk = dx_chunk_bytes(H, Q4);
   int n_slots = (int)(((size_t)ctx->smem_optin - fixed) / chunk);
   if (n_slots > kMaxSlots) n_slots = kMaxSlots;
   if (n_slots < kConsumerWarps + 1) return cudaErrorInvalidConfiguration;   // a unit needs all its chunks at once
   const size_t smem = fixed + (size_t)n_slots * chunk;
-  cudaError_t e = cudaFuncSetAttribute(dx_experts_bf16_kernel<H, NT, TILES, Q4>,
+  cudaError_t e = cudaFuncSetAttribute(dx_experts_bf16_kernel<H, NT, TILES, Q4, SPLIT>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   // One CTA per SM, minus the SMs the routing cluster runs on at the same time: a CTA of this kernel
   // fills an SM, so a CTA that had to wait for a routing CTA's SM would start late and become the tail.
   int grid = ctx->sm_count > 16 ? ctx->sm_count - DX_ROUTE_CLUSTER : ctx->sm_count;
   if (TILES == 2) grid &= ~1;
-  return dx_launch_pdl(DX_PDL_EXPERTS, dx_experts_bf16_kernel<H, NT, TILES, Q4>, dim3(grid), dim3(kThreads), smem, st, 1,
+  return dx_launch_pdl(DX_PDL_EXPERTS, dx_experts_bf16_kernel<H, NT, TILES, Q4, SPLIT>, dim3(grid), dim3(kThreads), smem, st, 1,
                        p, n_slots);
 }
 
-template <int H, bool Q4>
+template <int H, bool Q4, bool SPLIT>
 cudaError_t launch_bf16_h(dx_ctx* ctx, const DxExpertParams& p_in, int K, cudaStream_t st) {
   DxExpertParams p = p_in;
   p.row_tiles = 1;
-  if (K <= 8) return launch_bf16<H, 1, 1, Q4>(ctx, p, st);
+  if (K <= 8) return launch_bf16<H, 1, 1, Q4, SPLIT>(ctx, p, st);
   // two token tiles: fragments of both in shared memory where they fit next to a ring of at least one slot per
   // consumer warp and one to spare; otherwise CTA pairs with one tile each
   const size_t hdr = (sizeof(SmemHeader) + 127) / 128 * 128;
-  const size_t fixed2 = hdr + (size_t)2 * 8 * 2 * 32 * 16 + (size_t)2 * (H / 16) * 32 * 16;
+  const size_t fixed2 = hdr + (size_t)2 * 8 * 2 * 32 * 16 + (size_t)2 * (H / 16) * 32 * (SPLIT ? 16 : 8);
   if (fixed2 + (size_t)(kConsumerWarps + 1) * dx_chunk_bytes(H, Q4) <= (size_t)ctx->smem_optin)
-    return launch_bf16<H, 2, 1, Q4>(ctx, p, st);
+    return launch_bf16<H, 2, 1, Q4, SPLIT>(ctx, p, st);
   p.row_tiles = 2;
-  return launch_bf16<H, 1, 2, Q4>(ctx, p, st);
+  return launch_bf16<H, 1, 2, Q4, SPLIT>(ctx, p, st);
 }
 
-template <bool Q4>
+template <bool Q4, bool SPLIT>
 cudaError_t launch_bf16_any(dx_ctx* ctx, const DxExpertParams& p, int K, cudaStream_t st) {
   switch (p.H) {
-    case 256: return launch_bf16_h<256, Q4>(ctx, p, K, st);
-    case 512: return launch_bf16_h<512, Q4>(ctx, p, K, st);
-    case 1024: return launch_bf16_h<1024, Q4>(ctx, p, K, st);
-    case 2048: return launch_bf16_h<2048, Q4>(ctx, p, K, st);
+    case 256: return launch_bf16_h<256, Q4, SPLIT>(ctx, p, K, st);
+    case 512: return launch_bf16_h<512, Q4, SPLIT>(ctx, p, K, st);
+    case 1024: return launch_bf16_h<1024, Q4, SPLIT>(ctx, p, K, st);
+    case 2048: return launch_bf16_h<2048, Q4, SPLIT>(ctx, p, K, st);
     default: return cudaErrorInvalidConfiguration;
   }
 }
@@ -910,8 +922,8 @@ cudaError_t dx_launch_experts(dx_ctx* ctx, const DxExpertParams& p, int weight_d
   if (weight_dtype == DX_DTYPE_FP32) {
     return dx_launch_pdl(DX_PDL_EXPERTS, dx_experts_fp32_kernel, dim3(ctx->sm_count * 4), dim3(256), 0, st, 1, p);
   }
-  if (weight_dtype == DX_DTYPE_Q4) return launch_bf16_any<true>(ctx, p, K, st);
-  return launch_bf16_any<false>(ctx, p, K, st);
+  if (weight_dtype == DX_DTYPE_Q4) return launch_bf16_any<true, false>(ctx, p, K, st);
+  return ctx->act_split ? launch_bf16_any<false, true>(ctx, p, K, st) : launch_bf16_any<false, false>(ctx, p, K, st);
 }
 
 cudaError_t dx_launch_pack_q4(int H, int I, const void* Wg, const void* Wu, const void* Wd, void* blob,

@@ -66,6 +66,7 @@ struct dx_ctx {
   int device;
   int sm_count;
   int smem_optin;
+  int act_split;              // 1: bf16 experts are evaluated with hi + residual activation fragments
   cudaError_t last_cuda;
   int64_t launches;
   // device scratch

@@ -6,11 +6,14 @@ from oracle import moe_oracle as O
 from paper_2607_24434_b200 import synth
 
 # Tolerances.  The stated bar for layer outputs is a max relative error of 2e-2 per row (bf16 weights, fp32
-# accumulate), measured as max_j |y_j - yhat_j| / max_j |yhat_j|.  The kernels accumulate in fp32 and feed
-# activations as bf16 high part + residual (~16 mantissa bits), so they sit orders of magnitude inside the
-# bar; TIGHT guards against regressions.
+# accumulate), measured as max_j |y_j - yhat_j| / max_j |yhat_j|.  The kernels accumulate in fp32.  With the
+# activation split on (bf16 high part + residual, ~16 mantissa bits) they sit orders of magnitude inside the bar:
+# TIGHT.  By default the activations enter the tensor cores as plain bf16, as a bf16 model feeds them: one rounding
+# of at most 2^-9 relative per element, twice in a row (block rows, SwiGLU products); measured up to 5e-3 of the
+# row maximum, asserted at half the stated bar: BF16.
 Y_TOL = 2e-2
 Y_TIGHT = 3e-4
+Y_BF16 = 1e-2
 GATE_TOL = 1e-5
 GAP = 1e-3          # integer outputs must be exact wherever the checker's logit gap exceeds this
 

@@ -31,7 +31,7 @@ def _offloaded_layer(binding, ctx, seed, slots):
 
 def test_cached_verify_matches_resident_and_checker():
     from paper_2607_24434_b200 import binding
-    ctx = binding.Context(0)
+    ctx = binding.Context(0, act_split=True)
     ref, resident, off, cache, host = _offloaded_layer(binding, ctx, 70, slots=4)
     model = ExpertCacheModel(1, SHAPE.n_experts, 4)
     for step, K in enumerate([6, 6, 3, 8]):
@@ -68,7 +68,7 @@ def test_cached_verify_matches_resident_and_checker():
 
 def test_cached_draft_step_and_errors():
     from paper_2607_24434_b200 import binding
-    ctx = binding.Context(0)
+    ctx = binding.Context(0, act_split=True)
     ref, resident, off, cache, host = _offloaded_layer(binding, ctx, 71, slots=2)
     h = synth.hidden_block(1, SHAPE.hidden, 90, 0.0, "cuda")
     y = torch.empty_like(h)

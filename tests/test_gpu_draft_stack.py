@@ -16,7 +16,7 @@ pytestmark = pytest.mark.gpu
 
 def _stack_case(shape, n_layers, seed, zipf=False, reps=1):
     from paper_2607_24434_b200 import binding
-    ctx = binding.Context(0)
+    ctx = binding.Context(0, act_split=True)
     refs, layers = [], []
     for l in range(n_layers):
         w = synth.make_layer(shape, seed + 10 * l, "cuda", zipf=zipf)
@@ -86,7 +86,7 @@ def test_draft_stack_graph_replay():
     """The launch (scratch clear + cooperative kernel) captured in a CUDA graph and replayed on new inputs."""
     from paper_2607_24434_b200 import binding
     sh = dataclasses.replace(synth.shape_tiny(), weight_dtype=synth.DTYPE_BF16, hidden=512, n_experts=32, top_k=4)
-    ctx = binding.Context(0)
+    ctx = binding.Context(0, act_split=True)
     refs, layers = [], []
     for l in range(5):
         w = synth.make_layer(sh, 960 + l, "cuda")
@@ -116,7 +116,7 @@ def test_draft_stack_graph_replay():
 
 def test_draft_stack_refuses_mixed_shapes_and_fp32():
     from paper_2607_24434_b200 import binding
-    ctx = binding.Context(0)
+    ctx = binding.Context(0, act_split=True)
     a = binding.Layer.from_weights(ctx, synth.make_layer(synth.shape_tiny(), 1, "cuda"))
     with pytest.raises(binding.DxError):
         binding.DraftStack(ctx, [a])          # fp32 weights

@@ -20,7 +20,7 @@ SMALL = synth.LayerShape(hidden=512, n_experts=16, top_k=4, inter=64, n_shared=1
 @pytest.fixture()
 def dx():
     from paper_2607_24434_b200 import binding
-    ctx = binding.Context(0)
+    ctx = binding.Context(0, act_split=True)
     yield binding, ctx
     assert ctx.device_status() == 0
     ctx.close()

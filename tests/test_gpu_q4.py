@@ -27,7 +27,7 @@ def _bf16_of(values: np.ndarray) -> torch.Tensor:
 @pytest.mark.parametrize("H,I", [(512, 64), (256, 32), (2048, 1408)])
 def test_expand_q4_is_pack_of_dequantised(H, I):
     from paper_2607_24434_b200 import binding
-    ctx = binding.Context(0)
+    ctx = binding.Context(0, act_split=True)
     sh = dataclasses.replace(SHAPE, hidden=H, inter=I)
     Wg = synth.normal((I, H), 0.02, 7, "q4.g", torch.float32)
     Wu = synth.normal((I, H), 0.02, 7, "q4.u", torch.float32)
@@ -71,7 +71,7 @@ def test_fast_dequantiser_used_above_matches_the_loops():
 
 def test_verify_block_from_quantised_host_pool():
     from paper_2607_24434_b200 import binding
-    ctx = binding.Context(0)
+    ctx = binding.Context(0, act_split=True)
     layer, ref = gpu_layer(SHAPE, 75, std=0.08)
     Wg, Wu, Wd = layer["experts"]
     E = SHAPE.n_experts

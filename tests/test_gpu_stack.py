@@ -15,7 +15,7 @@ pytestmark = pytest.mark.gpu
 
 def _run_stack(shape, n_layers, K, seed, zipf, vocab):
     from paper_2607_24434_b200 import binding
-    ctx = binding.Context(0)
+    ctx = binding.Context(0, act_split=True)
     h = synth.hidden_block(K, shape.hidden, seed, 0.9, "cuda")
     hd = h[:1].clone()
     unions, near_total = [], 0
@@ -80,7 +80,7 @@ def test_stack_graph_replay_handover():
     from paper_2607_24434_b200 import binding
     sh = synth.shape_v2lite()
     n_layers, K = 4, 4
-    ctx = binding.Context(0)
+    ctx = binding.Context(0, act_split=True)
     refs, Ls = [], []
     for l in range(n_layers):
         layer = synth.make_layer(sh, 700 + 10 * l, "cuda", zipf=True)

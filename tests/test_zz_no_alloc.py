@@ -26,7 +26,7 @@ def _outputs(M, device):
                                            (4, 4, 1024, 256, torch.float32)])
 def test_noalloc_matches_regular_entry_point_twice(M, K, V, H, dtype):
     from paper_2607_24434_b200 import binding
-    ctx = binding.Context(0)
+    ctx = binding.Context(0, act_split=True)
     W = synth.lm_head(V, H, 900 + M, dtype, "cuda")
     results = []
     for call in range(2):                       # two calls in a row on different inputs
