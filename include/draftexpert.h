@@ -224,7 +224,8 @@ dx_status moe_draft_step_residual(dx_layer* layer, const float* h_in, float* h_o
  * token), run by ONE persistent kernel: a draft step reads so few bytes per layer that the gaps between
  * per-layer launches are a visible share of its time, and the weights of layer l+1 can stream while layer l is
  * still being reduced.  dx_stack_create records the layer handles (host array of n_layers handles, all of one
- * context and one shape, bf16 weights, no expert cache attached; DX_ERR_SHAPE / DX_ERR_UNSUPPORTED otherwise)
+ * context and one shape, bf16 or 4-bit experts (one kind per stack), no expert cache attached; DX_ERR_SHAPE /
+ * DX_ERR_UNSUPPORTED otherwise)
  * and owns the scratch rows; the layers must outlive the stack.  moe_draft_stack: h_in, h_out [H] fp32 device,
  * 16-byte aligned, distinct; topk_ids [n_layers, k] int32 and topk_w [n_layers, k] fp32 device or NULL (the
  * selection of every layer, gates as in Eq. 4).  Every expert of every layer must be resident

@@ -431,7 +431,8 @@ extern "C" dx_status dx_stack_create(dx_ctx* ctx, dx_layer* const* layers, int32
     dx_layer* L = layers[l];
     if (!L || L->ctx != ctx) return DX_ERR_INVALID_ARG;
     const dx_layer_desc &d = L->desc, &d0 = layers[0]->desc;
-    if (d.weight_dtype != DX_DTYPE_BF16 || L->cache) return DX_ERR_UNSUPPORTED;   // resident bf16 experts only
+    if (d.weight_dtype == DX_DTYPE_FP32 || L->cache) return DX_ERR_UNSUPPORTED;   // resident bf16 / 4-bit experts only
+    if (d.weight_dtype != d0.weight_dtype) return DX_ERR_SHAPE;
     if (d.hidden != d0.hidden || d.n_experts != d0.n_experts || d.top_k != d0.top_k || d.inter != d0.inter ||
         d.n_shared != d0.n_shared || d.shared_inter != d0.shared_inter || d.draft_inter != d0.draft_inter ||
         d.score_fn != d0.score_fn || d.norm_topk != d0.norm_topk || d.routed_scale != d0.routed_scale)
@@ -521,6 +522,7 @@ extern "C" dx_status moe_draft_stack(dx_stack* s, const float* h_in, float* h_ou
   p.shared_tiles = d.n_shared ? d.shared_inter / DX_TILE_I : 0;
   p.draft_tiles = d.draft_inter / DX_TILE_I;
   p.routed_tiles = d.inter / DX_TILE_I;
+  p.q4 = d.weight_dtype == DX_DTYPE_Q4 ? 1 : 0;
   DX_CUDA(ctx, dx_launch_draft_stack(ctx, p, st));
   ctx->launches++;
   return DX_OK;

@@ -21,6 +21,7 @@
 // The kernel is launched cooperatively, which either places the whole grid at once or fails the launch.  Every
 // wait on another CTA is bounded and ends in the device status word.
 #include <cooperative_groups.h>
+#include <cuda_fp16.h>
 
 #include "dx_internal.cuh"
 #include "dx_stream.cuh"
@@ -30,7 +31,7 @@ namespace {
 
 constexpr int kStackConsumers = 8;
 constexpr int kStackThreads = (kStackConsumers + 2) * 32;   // consumers, producer warp, router warp
-constexpr int kStackMaxSlots = 24;
+constexpr int kStackMaxSlots = 48;
 constexpr int kStackPartialBytes = 2 * 8 * 8 * 8;   // [2][warp][row] (gate, up) partial sums
 
 struct StackSmem {
@@ -61,6 +62,12 @@ __device__ __forceinline__ bool counter_wait(const unsigned int* word, unsigned 
 }
 __device__ __forceinline__ float bf_lo(unsigned int u) { return __uint_as_float(u << 16); }
 __device__ __forceinline__ float bf_hi(unsigned int u) { return __uint_as_float(u & 0xffff0000u); }
+// Two 4-bit codes (bits [0,4) and [16,20)) -> the bf16 pair (code - 8): 0x4300 | code is 128 + code in bf16.
+__device__ __forceinline__ uint32_t q4s_pair(uint32_t w) {
+  const uint32_t v = (w & 0x000F000Fu) | 0x43004300u;
+  const __nv_bfloat162 r = __hsub2(*reinterpret_cast<const __nv_bfloat162*>(&v), __floats2bfloat162_rn(136.f, 136.f));
+  return *reinterpret_cast<const uint32_t*>(&r);
+}
 __device__ __forceinline__ void unpack8(const uint4& r, float (&v)[8]) {
   const unsigned int u[4] = {r.x, r.y, r.z, r.w};
 #pragma unroll
@@ -87,11 +94,12 @@ __device__ __forceinline__ void stack_shares(int NS, int NR, int G, int cta, int
   r_hi = min(max(r_hi, r_lo), NR);
 }
 
-template <int H>
+// Q4: units of 4-bit codes and fp16 block scales (the grouped kernel's packed 4-bit layout), converted in registers.
+template <int H, bool Q4>
 __global__ void __launch_bounds__(kStackThreads, 1) dx_draft_stack_kernel(DxStackParams p, int n_slots) {
   constexpr int KW = H / 128;        // phase-1 contraction steps per consumer warp
   constexpr int PW = H / 256;        // phase-2 row-tile pairs per consumer warp
-  constexpr uint32_t CHUNK = KW * 512u + PW * 512u;
+  constexpr uint32_t CHUNK = Q4 ? KW * 144u + PW * 192u : KW * 512u + PW * 512u;
   constexpr uint32_t UNIT_BYTES = 8u * CHUNK;
 
   extern __shared__ __align__(128) unsigned char smem[];
@@ -374,13 +382,38 @@ __global__ void __launch_bounds__(kStackThreads, 1) dx_draft_stack_kernel(DxStac
       mbar_wait(smem_u32(&hdr->full[s]), ph, abort_flag);
       // gate (rows 0..7 of the tile) and up (rows 8..15) over this warp's slice of the hidden dimension
       float ga = 0.f, gb = 0.f, ua = 0.f, ub = 0.f;
+      if constexpr (Q4) {
+        // a 32-wide quantisation block is two contraction steps; its sums are scaled by the rows' block scales
+        const unsigned char* Cq = ring + (size_t)s * CHUNK;
+        const uint2* Aq = reinterpret_cast<const uint2*>(Cq) + lane;
+        const __half2* S1 = reinterpret_cast<const __half2*>(Cq + KW * 128) + g;
 #pragma unroll
-      for (int i = 0; i < KW; ++i) {
-        const uint4 a = A[i * 32];
-        ga = fmaf(bf_lo(a.x), xr[i].x, ga); gb = fmaf(bf_hi(a.x), xr[i].y, gb);
-        ua = fmaf(bf_lo(a.y), xr[i].x, ua); ub = fmaf(bf_hi(a.y), xr[i].y, ub);
-        ga = fmaf(bf_lo(a.z), xr[i].z, ga); gb = fmaf(bf_hi(a.z), xr[i].w, gb);
-        ua = fmaf(bf_lo(a.w), xr[i].z, ua); ub = fmaf(bf_hi(a.w), xr[i].w, ub);
+        for (int b = 0; b < KW / 2; ++b) {
+          const uint2 cw = Aq[b * 32];
+          const float2 sc = __half22float2(S1[b * 8]);
+          float gs = 0.f, us = 0.f;
+#pragma unroll
+          for (int ks = 0; ks < 2; ++ks) {
+            const uint32_t w = ks ? cw.y : cw.x;
+            const float4 x4 = xr[2 * b + ks];
+            const uint32_t p0 = q4s_pair(w), p1 = q4s_pair(w >> 4), p2 = q4s_pair(w >> 8), p3 = q4s_pair(w >> 12);
+            gs = fmaf(bf_lo(p0), x4.x, gs); gs = fmaf(bf_hi(p0), x4.y, gs);
+            us = fmaf(bf_lo(p1), x4.x, us); us = fmaf(bf_hi(p1), x4.y, us);
+            gs = fmaf(bf_lo(p2), x4.z, gs); gs = fmaf(bf_hi(p2), x4.w, gs);
+            us = fmaf(bf_lo(p3), x4.z, us); us = fmaf(bf_hi(p3), x4.w, us);
+          }
+          if (b & 1) { gb = fmaf(sc.x, gs, gb); ub = fmaf(sc.y, us, ub); }
+          else { ga = fmaf(sc.x, gs, ga); ua = fmaf(sc.y, us, ua); }
+        }
+      } else {
+#pragma unroll
+        for (int i = 0; i < KW; ++i) {
+          const uint4 a = A[i * 32];
+          ga = fmaf(bf_lo(a.x), xr[i].x, ga); gb = fmaf(bf_hi(a.x), xr[i].y, gb);
+          ua = fmaf(bf_lo(a.y), xr[i].x, ua); ub = fmaf(bf_hi(a.y), xr[i].y, ub);
+          ga = fmaf(bf_lo(a.z), xr[i].z, ga); gb = fmaf(bf_hi(a.z), xr[i].w, gb);
+          ua = fmaf(bf_lo(a.w), xr[i].z, ua); ub = fmaf(bf_hi(a.w), xr[i].w, ub);
+        }
       }
       float gt = ga + gb, ut = ua + ub;
       gt += __shfl_xor_sync(0xffffffffu, gt, 1); ut += __shfl_xor_sync(0xffffffffu, ut, 1);
@@ -402,14 +435,33 @@ __global__ void __launch_bounds__(kStackThreads, 1) dx_draft_stack_kernel(DxStac
       const float act0 = __shfl_sync(0xffffffffu, act, 2 * c), act1 = __shfl_sync(0xffffffffu, act, 2 * c + 1);
       buf ^= 1;
       // down projection: a lane holds rows g and g + 8 of two 16-row tiles at intermediate rows 2c and 2c + 1
-      const uint4* D = A + KW * 32;
+      if constexpr (Q4) {
+        // the eight columns of a unit lie in one quantisation block of W_d: one scale per output row
+        const unsigned char* Cq = ring + (size_t)s * CHUNK + KW * 144;
+        const uint32_t* Dq = reinterpret_cast<const uint32_t*>(Cq) + lane;
+        const uint2* S2 = reinterpret_cast<const uint2*>(Cq + PW * 128) + g;
 #pragma unroll
-      for (int q2 = 0; q2 < PW; ++q2) {
-        const uint4 a = D[q2 * 32];
-        acc[2 * q2][0] = fmaf(bf_hi(a.x), act1, fmaf(bf_lo(a.x), act0, acc[2 * q2][0]));
-        acc[2 * q2][1] = fmaf(bf_hi(a.y), act1, fmaf(bf_lo(a.y), act0, acc[2 * q2][1]));
-        acc[2 * q2 + 1][0] = fmaf(bf_hi(a.z), act1, fmaf(bf_lo(a.z), act0, acc[2 * q2 + 1][0]));
-        acc[2 * q2 + 1][1] = fmaf(bf_hi(a.w), act1, fmaf(bf_lo(a.w), act0, acc[2 * q2 + 1][1]));
+        for (int q2 = 0; q2 < PW; ++q2) {
+          const uint32_t w = Dq[q2 * 32];
+          const uint2 sw = S2[q2 * 8];
+          const float2 s01 = __half22float2(*reinterpret_cast<const __half2*>(&sw.x));
+          const float2 s23 = __half22float2(*reinterpret_cast<const __half2*>(&sw.y));
+          const uint32_t p0 = q4s_pair(w), p1 = q4s_pair(w >> 4), p2 = q4s_pair(w >> 8), p3 = q4s_pair(w >> 12);
+          acc[2 * q2][0] = fmaf(s01.x, fmaf(bf_hi(p0), act1, bf_lo(p0) * act0), acc[2 * q2][0]);
+          acc[2 * q2][1] = fmaf(s01.y, fmaf(bf_hi(p1), act1, bf_lo(p1) * act0), acc[2 * q2][1]);
+          acc[2 * q2 + 1][0] = fmaf(s23.x, fmaf(bf_hi(p2), act1, bf_lo(p2) * act0), acc[2 * q2 + 1][0]);
+          acc[2 * q2 + 1][1] = fmaf(s23.y, fmaf(bf_hi(p3), act1, bf_lo(p3) * act0), acc[2 * q2 + 1][1]);
+        }
+      } else {
+        const uint4* D = A + KW * 32;
+#pragma unroll
+        for (int q2 = 0; q2 < PW; ++q2) {
+          const uint4 a = D[q2 * 32];
+          acc[2 * q2][0] = fmaf(bf_hi(a.x), act1, fmaf(bf_lo(a.x), act0, acc[2 * q2][0]));
+          acc[2 * q2][1] = fmaf(bf_hi(a.y), act1, fmaf(bf_lo(a.y), act0, acc[2 * q2][1]));
+          acc[2 * q2 + 1][0] = fmaf(bf_hi(a.z), act1, fmaf(bf_lo(a.z), act0, acc[2 * q2 + 1][0]));
+          acc[2 * q2 + 1][1] = fmaf(bf_hi(a.w), act1, fmaf(bf_lo(a.w), act0, acc[2 * q2 + 1][1]));
+        }
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&hdr->empty[s]));
@@ -454,16 +506,16 @@ __global__ void __launch_bounds__(kStackThreads, 1) dx_draft_stack_kernel(DxStac
   if (*abort_flag && threadIdx.x == 0) atomicExch(p.dev_status, DX_DEV_WAIT_EXPIRED);
 }
 
-template <int H>
+template <int H, bool Q4>
 cudaError_t launch_stack(dx_ctx* ctx, const DxStackParams& p, cudaStream_t st) {
   const size_t hdr = (sizeof(StackSmem) + 127) / 128 * 128;
   const size_t fixed = hdr + (size_t)kStackPartialBytes + (size_t)H * 4;
-  const size_t chunk = (size_t)6 * H;
+  const size_t chunk = dx_chunk_bytes(H, Q4);
   int n_slots = (int)(((size_t)ctx->smem_optin - fixed) / chunk);
   if (n_slots > kStackMaxSlots) n_slots = kStackMaxSlots;
   if (n_slots < kStackConsumers + 1) return cudaErrorInvalidConfiguration;
   const size_t smem = fixed + (size_t)n_slots * chunk;
-  cudaError_t e = cudaFuncSetAttribute(dx_draft_stack_kernel<H>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  cudaError_t e = cudaFuncSetAttribute(dx_draft_stack_kernel<H, Q4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(ctx->sm_count);
@@ -475,17 +527,17 @@ cudaError_t launch_stack(dx_ctx* ctx, const DxStackParams& p, cudaStream_t st) {
   attr[0].val.cooperative = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, dx_draft_stack_kernel<H>, p, n_slots);
+  return cudaLaunchKernelEx(&cfg, dx_draft_stack_kernel<H, Q4>, p, n_slots);
 }
 
 }  // namespace
 
 cudaError_t dx_launch_draft_stack(dx_ctx* ctx, const DxStackParams& p, cudaStream_t st) {
   switch (p.H) {
-    case 256: return launch_stack<256>(ctx, p, st);
-    case 512: return launch_stack<512>(ctx, p, st);
-    case 1024: return launch_stack<1024>(ctx, p, st);
-    case 2048: return launch_stack<2048>(ctx, p, st);
+    case 256: return p.q4 ? launch_stack<256, true>(ctx, p, st) : launch_stack<256, false>(ctx, p, st);
+    case 512: return p.q4 ? launch_stack<512, true>(ctx, p, st) : launch_stack<512, false>(ctx, p, st);
+    case 1024: return p.q4 ? launch_stack<1024, true>(ctx, p, st) : launch_stack<1024, false>(ctx, p, st);
+    case 2048: return p.q4 ? launch_stack<2048, true>(ctx, p, st) : launch_stack<2048, false>(ctx, p, st);
     default: return cudaErrorInvalidConfiguration;
   }
 }

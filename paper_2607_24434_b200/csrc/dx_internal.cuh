@@ -172,6 +172,7 @@ struct DxStackParams {
   int H, E, k, score_fn, norm_topk;
   float scale;
   int n_shared, shared_tiles, draft_tiles, routed_tiles;
+  int q4;                     // 1: the units are 4-bit codes with block scales
 };
 struct dx_stack {
   dx_ctx* ctx;

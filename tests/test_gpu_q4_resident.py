@@ -109,3 +109,35 @@ def test_q4_sizes_and_refusals():
     with pytest.raises(binding.DxError):
         binding.Layer(ctx, dataclasses.replace(q, draft_inter=24))
     ctx.close()
+
+
+@pytest.mark.parametrize("shape,n_layers", [(SMALL, 5), (dataclasses.replace(synth.shape_v2lite(), n_experts=16), 3)])
+def test_q4_draft_stack(shape, n_layers):
+    """The persistent draft stack on layers with 4-bit experts (fp32 activations, exact codes and scales)."""
+    from paper_2607_24434_b200 import binding
+    from tests.helpers import Y_TIGHT
+    ctx = binding.Context(0)
+    refs, layers = [], []
+    for l in range(n_layers):
+        lq = synth.quantize_layer(synth.make_layer(shape, 340 + 10 * l, "cuda", std=0.05 if shape is SMALL else 0.02))
+        refs.append(_reference(lq, _fast_dequant))
+        layers.append(binding.Layer.from_weights(ctx, lq))
+    stack = binding.DraftStack(ctx, layers)
+    h0 = synth.hidden_block(1, shape.hidden, 350, 0.0, "cuda")
+    out = binding.moe_draft_stack(stack, h0)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == 0
+    ids = out["topk_ids"].cpu().numpy()
+    h = h0.cpu().numpy().astype(np.float64)
+    near = 0
+    for l in range(n_layers):
+        _, ids_ref, _, z_ref = O.stack_layer_draft(h, refs[l])
+        near += check_routing(shape, z_ref, ids_ref, ids[l][None])
+        h = O.stack_layer_draft(h, refs[l], forced_ids=ids[l][None])[0]
+    assert row_rel_err(out["h"].cpu().numpy(), h).max() <= Y_TIGHT
+    # mixing 4-bit and bf16 layers in one stack is refused
+    b = binding.Layer.from_weights(ctx, synth.make_layer(shape, 399, "cuda"))
+    with pytest.raises(binding.DxError):
+        binding.DraftStack(ctx, [layers[0], b])
+    stack.close()
+    ctx.close()
