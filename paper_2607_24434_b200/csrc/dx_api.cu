@@ -307,6 +307,7 @@ static dx_status do_experts(dx_layer* L, const float* h, int K, float* y, bool d
   const dx_layer_desc& d = L->desc;
   if (!h || !y || h == y) return DX_ERR_INVALID_ARG;
   if (K < 1 || K > DX_MAX_K) return DX_ERR_UNSUPPORTED;
+  if (((uintptr_t)h) % 16 || ((uintptr_t)y) % 16) return DX_ERR_INVALID_ARG;   // 16-byte loads and reductions
   dx_status s = upload_table(L, st);
   if (s != DX_OK) return s;
   DxExpertParams p{};

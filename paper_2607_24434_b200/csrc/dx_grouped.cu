@@ -572,22 +572,42 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
   process(hdr->r_e_lo, hdr->r_e_hi, hdr->r_u_lo, hdr->r_u_hi);
   pdl_wait();  // the routing kernel (which initialised y) has completed as a whole
 
-  // ---- the CTA's partial output rows go to y (initialised by the routing kernel, which has completed)
+  // ---- the CTA's partial output rows go to y (initialised by the routing kernel, which has completed).
+  // A lane holds, per 16-row tile, rows g and g + 8 of block rows 2c and 2c + 1.  The four lanes g = 4q .. 4q+3 of a
+  // column pair transpose their 4 x 4 values (two butterfly steps over lane bits 2 and 3), after which lane i of
+  // the four holds four consecutive output rows of ONE (block row, half): one 16-byte reduction instead of four.
+  {
+    const int gi = g & 3;                       // this lane's place among the four, and the combination it ends up with:
+    const int tok = 2 * c + (gi & 1);           //   block row 2c or 2c + 1 ...
+    const int half = gi >> 1;                   //   ... rows g or g + 8 of the tile
 #pragma unroll
-  for (int nt = 0; nt < NT; ++nt) {
-    const int r0 = row_base + nt * 8 + 2 * c, r1 = r0 + 1;
-    if (r0 < p.K) {
-      float* y0 = p.y + (size_t)r0 * H;
-      float* y1 = p.y + (size_t)r1 * H;
-      const bool v1 = r1 < p.K;
+    for (int nt = 0; nt < NT; ++nt) {
+      const int row = row_base + nt * 8 + tok;
+      float* yrow = p.y + (size_t)row * H + (g >> 2) * 4 + half * 8;
 #pragma unroll
       for (int j = 0; j < 2 * PW; ++j) {
-        const int hh = (warp * 2 * PW + j) * 16 + g;
-        atomicAdd(y0 + hh, acc[nt][j][0]);
-        atomicAdd(y0 + hh + 8, acc[nt][j][2]);
-        if (v1) {
-          atomicAdd(y1 + hh, acc[nt][j][1]);
-          atomicAdd(y1 + hh + 8, acc[nt][j][3]);
+        // combination k of a lane: k = 0: (2c, g), 1: (2c+1, g), 2: (2c, g+8), 3: (2c+1, g+8)
+        float v0 = acc[nt][j][0], v1 = acc[nt][j][1], v2 = acc[nt][j][2], v3 = acc[nt][j][3];
+        // step 1 (partner differs in bit 0 of gi): keep combinations with my bit 0, get the partner's
+        {
+          const bool hi = gi & 1;
+          const float s0 = hi ? v0 : v1, s1 = hi ? v2 : v3;          // what the partner wants from me
+          const float r0 = __shfl_xor_sync(0xffffffffu, s0, 4), r1 = __shfl_xor_sync(0xffffffffu, s1, 4);
+          if (hi) { v0 = r0; v2 = r1; } else { v1 = r0; v3 = r1; }
+          // now (v0, v1) = combination (gi & 1) of lanes {gi & ~1, gi | 1}, rows g-pair order; (v2, v3) likewise + 2
+        }
+        // step 2 (partner differs in bit 1 of gi)
+        {
+          const bool hi = gi & 2;
+          const float s0 = hi ? v0 : v2, s1 = hi ? v1 : v3;
+          const float r0 = __shfl_xor_sync(0xffffffffu, s0, 8), r1 = __shfl_xor_sync(0xffffffffu, s1, 8);
+          if (hi) { v0 = r0; v1 = r1; } else { v2 = r0; v3 = r1; }
+        }
+        // (v0, v1, v2, v3) = this lane's combination at rows 4q, 4q+1, 4q+2, 4q+3 of the tile's half
+        if (row < p.K) {
+          float* dst = yrow + (warp * 2 * PW + j) * 16;
+          asm volatile("red.relaxed.gpu.global.add.v4.f32 [%0], {%1, %2, %3, %4};"
+                       :: "l"(dst), "f"(v0), "f"(v1), "f"(v2), "f"(v3) : "memory");
         }
       }
     }
