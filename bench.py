@@ -485,12 +485,14 @@ def run_stack(args):
     layers = []
     for l in range(NLAY):
         w = synth.make_layer(shape, 7000 + l, device, zipf=args.zipf)
+        if args.q4_resident:
+            w = synth.quantize_layer(w)
         layers.append(binding.Layer.from_weights(ctx, w))
         torch.cuda.synchronize()
         del w
     torch.cuda.empty_cache()
     W_lm = synth.lm_head(V, H, 7999, torch.bfloat16, device)
-    exp_bytes = binding.expert_blob_bytes(shape, shape.inter)
+    exp_bytes = binding.expert_blob_bytes(layers[0].shape, shape.inter)   # as streamed (bf16 or 4-bit units)
     peak, peak_kind = measured_peaks()
     stream = torch.cuda.current_stream()
 
@@ -542,7 +544,9 @@ def run_stack(args):
     drift = float(((h_stack - hd[NLAY]).norm() / hd[NLAY].norm()).item())
     draft_bytes = NLAY * ((shape.n_shared + 2) * exp_bytes + shape.n_experts * H * 2)
     out = {"metric": "draft_stack_us_per_token", "value": draft_ms * 1e3, "unit": "us/token", "n_gpus": 1,
-           "higher_is_better": False, "data": "synthetic", "dtype": "bf16 weights, fp32 accumulate",
+           "higher_is_better": False, "data": "synthetic",
+           "dtype": "4-bit block-quantised experts, fp32 accumulate" if args.q4_resident else
+                    "bf16 weights, fp32 accumulate",
            "config": {"workload": f"{'configs[3] Moonlight' if args.moonlight else 'configs[2] DeepSeek-V2-Lite'}-shaped "
                                   f"stack of {NLAY} MoE sub-layers, experts resident "
                                   f"({NLAY * (shape.n_experts + shape.n_shared + 1) * exp_bytes / 1e9:.1f} GB), "
