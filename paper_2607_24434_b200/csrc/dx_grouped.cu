@@ -62,6 +62,7 @@ struct SmemHeader {
   int r_e_lo, r_e_hi, r_u_lo;   // this CTA's routed entries and units, published by the producer warp
   int r_u_hi;
   float rstd[DX_MAX_K];
+  float ssq[8][8];                   // sums of squares of the block rows, per consumer warp's slice
   int e_begin[DX_MAX_ENTRIES];       // first unit of each group (routing-independent groups first)
   int e_tiles[DX_MAX_ENTRIES];
   int e_gid[DX_MAX_ENTRIES];         // expert id of a routed group
@@ -307,34 +308,56 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
   } else {
     pdl_wait();
   }
-  // 1/rms of every block row when the experts see RMSNorm(x)
-  for (int r = warp; r < DX_MAX_K; r += kConsumerWarps) {
-    float rs = 1.0f;
-    if (p.rms_norm && r < p.K) {
-      float ss = 0.f;
-      for (int j = lane * 4; j < H; j += 128) {
-        const float4 v = *reinterpret_cast<const float4*>(p.x + (size_t)r * H + j);
-        ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
-      }
+  // 1/rms of every block row when the experts see RMSNorm(x) (fragments in shared memory: every warp takes rows;
+  // fragments in registers: see below)
+  if constexpr (!kRegB) {
+    for (int r = warp; r < DX_MAX_K; r += kConsumerWarps) {
+      float rs = 1.0f;
+      if (p.rms_norm && r < p.K) {
+        float ss = 0.f;
+        for (int j = lane * 4; j < H; j += 128) {
+          const float4 v = *reinterpret_cast<const float4*>(p.x + (size_t)r * H + j);
+          ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+        }
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-      rs = rsqrtf(ss / (float)H + 1e-6f);
+        for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+        rs = rsqrtf(ss / (float)H + 1e-6f);
+      }
+      if (lane == 0) hdr->rstd[r] = rs;
     }
-    if (lane == 0) hdr->rstd[r] = rs;
+    consumer_bar();
   }
-  consumer_bar();
 
   // ---- token fragments: the MMA token slots are the block rows themselves, the same for every group (a group's
   // weight, zero for the rows outside it, multiplies the activations), so they are built once
   if constexpr (kRegB) {
+    // one pass over the block: a lane loads exactly the values of its fragments (row g, this warp's slice of the
+    // hidden dimension), the sum of squares of a row is put together from the eight warps' slices
     const int tk = row_base + g;
     const bool valid = tk < p.K;
-    const float rs = hdr->rstd[tk];
     const float* xrow = p.x + (size_t)tk * H + 4 * c;
+    float4 xv[KW];
+    float ss = 0.f;
 #pragma unroll
     for (int i = 0; i < KW; ++i) {
-      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (valid) v = *reinterpret_cast<const float4*>(xrow + 16 * (warp * KW + i));
+      xv[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (valid) xv[i] = *reinterpret_cast<const float4*>(xrow + 16 * (warp * KW + i));
+      ss += xv[i].x * xv[i].x + xv[i].y * xv[i].y + xv[i].z * xv[i].z + xv[i].w * xv[i].w;
+    }
+    float rs = 1.0f;
+    if (p.rms_norm) {
+      ss += __shfl_xor_sync(0xffffffffu, ss, 1);
+      ss += __shfl_xor_sync(0xffffffffu, ss, 2);
+      if (c == 0) hdr->ssq[warp][g] = ss;
+      consumer_bar();
+      float tot = 0.f;
+#pragma unroll
+      for (int w = 0; w < kConsumerWarps; ++w) tot += hdr->ssq[w][g];
+      rs = rsqrtf(tot / (float)H + 1e-6f);
+    }
+#pragma unroll
+    for (int i = 0; i < KW; ++i) {
+      const float4 v = xv[i];
       __nv_bfloat16 h0, h1, h2, h3, l0, l1, l2, l3;
       split_bf16(v.x * rs, h0, l0); split_bf16(v.y * rs, h1, l1);
       split_bf16(v.z * rs, h2, l2); split_bf16(v.w * rs, h3, l3);
