@@ -7,7 +7,7 @@ One *step* is one pass of the whole hot path over one block on one MoE layer:
 Steps rotate over independently seeded layers (default 8 x 1.16 GB of bf16 experts) so that no weight is
 ever re-read from L2 between timed iterations.
 
-Prints ONE JSON line (see README / DESIGN for the keys).  ``--impl reference`` times the CPU checker
+Prints ONE JSON line (keys: metric, value, roofline, e2e, cpu_baseline, clocks, ...).  ``--impl reference`` times the CPU checker
 (``oracle/``) on the host cores on the same configuration instead.
 """
 from __future__ import annotations
