@@ -210,6 +210,13 @@ def run_gpu(args):
     launches = (ctx.kernel_launches() - launches0) if graph is None else launches_per_step * args.steps
     total_ms = e0.elapsed_time(e1)
 
+    def check_status(where):
+        code = ctx.device_status()
+        if code != 0:
+            raise RuntimeError(f"device status word {code} set during {where}")
+
+    check_status("the timed steps")
+
     # ---- per-kernel timing of the dominant kernel (grouped SwiGLU of the verify block) and the others
     ev = lambda: torch.cuda.Event(enable_timing=True)
     t_exp, t_route, t_draft, t_acc = [], [], [], []
@@ -359,6 +366,7 @@ def run_gpu(args):
     g1.record(stream)
     barrier()
     e2e_ms = g0.elapsed_time(g1)
+    check_status("the component timings or the end-to-end steps")
     # what came back over the link must be what the device-resident loop produced for the same layer
     li_last = (args.steps - 1) % NL
     got_y = out_host[:K * H * 4].view(torch.float32).view(K, H)
@@ -410,8 +418,9 @@ def run_gpu(args):
         s1.record(stream)
         torch.cuda.synchronize()
         stack_us = s0.elapsed_time(s1) * 1e3 / 50
-        if ctx.device_status() != 0:
-            raise RuntimeError("device status word set during the draft stack")
+        dev_status = ctx.device_status()
+        if dev_status != 0:
+            raise RuntimeError(f"device status word {dev_status} set during the run (draft stack last)")
         dstack.close()
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,

@@ -570,11 +570,8 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
 
   process(0, n_static, s_lo, s_hi);
   cta_bar();   // the producer warp has seen the routing call's work list and published its routed part
-  // Only now may the next kernel of the stream start: if it is a routing kernel it clears the hand-over words,
-  // and this CTA is done with both of them.
-  pdl_launch_dependents();
   // The (row, expert, gate) pairs come out of the gate arithmetic a little after the group list.  Every warp
-  // fetches all of them for itself (same values from every warp, so no barrier is needed beyond its own).
+  // fetches all of them for itself (same values from every warp, so no barrier is needed to use them).
   {
     const int n_pairs = hdr->n_pairs;
     bool ok = true;
@@ -592,6 +589,13 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
     if (!ok) { *abort_flag = 1; atomicExch(p.dev_status, DX_DEV_WAIT_EXPIRED); }
     __syncwarp();
   }
+  // Only now may the next kernel of the stream start: if it is a routing kernel it clears the hand-over words
+  // (flag, group list, pairs) before its own wait, so every warp of this CTA has to be done with all of them.  (The
+  // trigger used to sit in front of the pair fetch: a routing kernel that started in that window wiped pairs that
+  // were still being polled -- rare, and seen as an expired wait on blocks of eight rows, whose gate arithmetic
+  // takes longest.)
+  consumer_bar();
+  pdl_launch_dependents();
   process(hdr->r_e_lo, hdr->r_e_hi, hdr->r_u_lo, hdr->r_u_hi);
   pdl_wait();  // the routing kernel (which initialised y) has completed as a whole
 

@@ -18,7 +18,10 @@
 // (token, expert) pairs by expert for the caller's outputs.
 #include <cooperative_groups.h>
 
+#include <type_traits>
+
 #include "dx_internal.cuh"
+#include "dx_stream.cuh"
 
 namespace cg = cooperative_groups;
 
@@ -233,16 +236,39 @@ __global__ void __launch_bounds__(kRouteThreads) dx_route_kernel(DxRouteParams p
   const int col0 = sp.slice * sp.C * 256 + 8 * lane;   // this lane's first column; slab c adds 256 c
   const WT* Wr = reinterpret_cast<const WT*>(p.W_r);
 
+  // bf16 router and blocks of more than two rows: the contraction runs on the tensor cores (one or two rows are
+  // quicker on the plain path: its arithmetic is small and it has no partial tables to merge)
+  constexpr bool kMma = std::is_same<WT, __nv_bfloat16>::value && TG == 4;
   // the first batch of this warp's router rows (first kPreSlabs slabs of the slice): constant data, fetched right away
   constexpr int kPreSlabs = 2;
-  RowRaw<WT> wpre[kPreSlabs][kRowsPerBatch];
+  constexpr int kPreTiles = 4;   // (tensor-core path) 16-row tiles of the router kept in registers
+  RowRaw<WT> wpre[kMma ? 1 : kPreSlabs][kMma ? 1 : kRowsPerBatch];
+  uint4 wa[kMma ? kPreTiles : 1][kMma ? kPreSlabs : 1][2];
+  const int mg = lane >> 2, mc = lane & 3;
+  // (tensor-core path) warp w owns the 32 columns [32 w, 32 w + 32) of every slab of the slice; a lane loads the
+  // 8 columns 8 mc .. 8 mc + 7 of rows mg and mg + 8 of a tile -- its operand fragment of two contraction steps
+  const int mcol0 = sp.slice * sp.C * 256 + 32 * warp + 8 * mc;
+  const int n_et = sp.idle ? 0 : (sp.e_hi - sp.e_lo + 15) / 16;
+  if constexpr (kMma) {
 #pragma unroll
-  for (int c = 0; c < kPreSlabs; ++c)
+    for (int et = 0; et < kPreTiles; ++et)
 #pragma unroll
-    for (int i = 0; i < kRowsPerBatch; ++i) {
-      const int e = sp.e_lo + warp + kRouteWarps * i;
-      if (c < sp.C && e < sp.e_hi) wpre[c][i].load(Wr + (size_t)e * H + col0 + 256 * c);
-    }
+      for (int c = 0; c < kPreSlabs; ++c) {
+        if (et < n_et && c < sp.C) {
+          const int e0 = min(sp.e_lo + 16 * et + mg, sp.e_hi - 1), e1 = min(sp.e_lo + 16 * et + mg + 8, sp.e_hi - 1);
+          wa[et][c][0] = ldg_stream(Wr + (size_t)e0 * H + mcol0 + 256 * c);
+          wa[et][c][1] = ldg_stream(Wr + (size_t)e1 * H + mcol0 + 256 * c);
+        }
+      }
+  } else {
+#pragma unroll
+    for (int c = 0; c < kPreSlabs; ++c)
+#pragma unroll
+      for (int i = 0; i < kRowsPerBatch; ++i) {
+        const int e = sp.e_lo + warp + kRouteWarps * i;
+        if (c < sp.C && e < sp.e_hi) wpre[c][i].load(Wr + (size_t)e * H + col0 + 256 * c);
+      }
+  }
   if (crank == 0)
     for (int e = threadIdx.x; e < E; e += kRouteThreads) s_bias[e] = p.bias ? p.bias[e] : 0.f;
   for (int i = threadIdx.x; i < DX_MAX_K * DX_MAX_TOPK; i += kRouteThreads) s_sel_z[i] = 0.f;
@@ -275,6 +301,105 @@ __global__ void __launch_bounds__(kRouteThreads) dx_route_kernel(DxRouteParams p
   // ---- partial logits of this CTA's slice, into CTA 0's table for the slice
   float* part0 = cluster.map_shared_rank(s_part, 0) + (size_t)sp.slice * part_stride;
   const bool rms = p.rms_norm != 0;
+  if constexpr (kMma) {
+    // Tensor-core contraction: the block rows are the eight (sixteen) token columns, split into bf16 high part and
+    // residual so that the logits keep fp32-like accuracy; a warp's products over its columns of every slab give
+    // one partial table per warp, the eight tables are added in a fixed order.
+    const int NTK = K > 8 ? 2 : 1, kpad = NTK * 8;
+    const int red_stride = ((E + 15) / 16) * 16 * kpad;
+    float* s_red = s_part + (size_t)kRouteCluster * part_stride;       // [8 warps][tiles * 16 rows][kpad tokens]
+    float* s_ssq = s_red + (size_t)kRouteWarps * red_stride;           // [8 warps][kpad]
+    uint4 bh[2][2], bl[2][2];   // [slab][token tile]
+    float ssq[2] = {0.f, 0.f};
+#pragma unroll
+    for (int c = 0; c < 2; ++c)
+#pragma unroll
+      for (int nt = 0; nt < 2; ++nt) {
+        bh[c][nt] = bl[c][nt] = make_uint4(0u, 0u, 0u, 0u);
+        const int tok = nt * 8 + mg;
+        if (c < sp.C && nt < NTK && tok < K && !sp.idle) {
+          const float* hp = p.h + (size_t)tok * H + mcol0 + 256 * c;
+          const float4 v0 = *reinterpret_cast<const float4*>(hp), v1 = *reinterpret_cast<const float4*>(hp + 4);
+          const float x[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+          __nv_bfloat16 hb[8], lb[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            ssq[nt] = fmaf(x[i], x[i], ssq[nt]);
+            split_bf16(x[i], hb[i], lb[i]);
+          }
+          bh[c][nt] = make_uint4(pack2(hb[0], hb[1]), pack2(hb[2], hb[3]), pack2(hb[4], hb[5]), pack2(hb[6], hb[7]));
+          bl[c][nt] = make_uint4(pack2(lb[0], lb[1]), pack2(lb[2], lb[3]), pack2(lb[4], lb[5]), pack2(lb[6], lb[7]));
+        }
+      }
+    // one 16-row tile of the router: products over this warp's columns of every slab, into the warp's table
+    auto do_tile = [&](int et, const uint4 (&aw)[2][2]) {
+      float cacc[2][4];
+#pragma unroll
+      for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+        for (int r = 0; r < 4; ++r) cacc[nt][r] = 0.f;
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        if (c >= sp.C) continue;
+        const uint4 a0 = aw[c][0], a1 = aw[c][1];
+        const uint4 f0 = make_uint4(a0.x, a1.x, a0.y, a1.y), f1 = make_uint4(a0.z, a1.z, a0.w, a1.w);
+#pragma unroll
+        for (int nt = 0; nt < 2; ++nt) {
+          if (nt >= NTK) continue;
+          mma_k16(cacc[nt], f0, bh[c][nt].x, bh[c][nt].y);
+          mma_k16(cacc[nt], f0, bl[c][nt].x, bl[c][nt].y);
+          mma_k16(cacc[nt], f1, bh[c][nt].z, bh[c][nt].w);
+          mma_k16(cacc[nt], f1, bl[c][nt].z, bl[c][nt].w);
+        }
+      }
+      // rows mg and mg + 8 of the tile, tokens 2 mc and 2 mc + 1 of each token tile
+#pragma unroll
+      for (int nt = 0; nt < 2; ++nt) {
+        if (nt >= NTK) continue;
+        float* dst = s_red + (size_t)warp * red_stride + (size_t)(16 * et + mg) * kpad + nt * 8 + 2 * mc;
+        *reinterpret_cast<float2*>(dst) = make_float2(cacc[nt][0], cacc[nt][1]);
+        *reinterpret_cast<float2*>(dst + 8 * kpad) = make_float2(cacc[nt][2], cacc[nt][3]);
+      }
+    };
+#pragma unroll
+    for (int et = 0; et < kPreTiles; ++et)   // (held in registers since before the wait)
+      if (et < n_et) do_tile(et, wa[et]);
+    for (int et = kPreTiles; et < n_et; ++et) {
+      uint4 aw[2][2];
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        aw[c][0] = aw[c][1] = make_uint4(0u, 0u, 0u, 0u);
+        if (c < sp.C) {
+          const int e0 = min(sp.e_lo + 16 * et + mg, sp.e_hi - 1), e1 = min(sp.e_lo + 16 * et + mg + 8, sp.e_hi - 1);
+          aw[c][0] = ldg_stream(Wr + (size_t)e0 * H + mcol0 + 256 * c);
+          aw[c][1] = ldg_stream(Wr + (size_t)e1 * H + mcol0 + 256 * c);
+        }
+      }
+      do_tile(et, aw);
+    }
+#pragma unroll
+    for (int nt = 0; nt < 2; ++nt) {
+      float q = ssq[nt];
+      q += __shfl_xor_sync(0xffffffffu, q, 1);
+      q += __shfl_xor_sync(0xffffffffu, q, 2);
+      if (mc == 0 && nt < NTK) s_ssq[warp * kpad + nt * 8 + mg] = q;
+    }
+    __syncthreads();
+    const int n_rows = sp.idle ? 0 : sp.e_hi - sp.e_lo;
+    for (int i = threadIdx.x; i < n_rows * K; i += kRouteThreads) {
+      const int el = i / K, t = i - el * K;
+      float z = 0.f;
+#pragma unroll
+      for (int w = 0; w < kRouteWarps; ++w) z += s_red[(size_t)w * red_stride + (size_t)el * kpad + t];
+      part0[t * E + sp.e_lo + el] = z;
+    }
+    if (rms && sp.share == 0 && !sp.idle && threadIdx.x < K) {
+      float q = 0.f;
+#pragma unroll
+      for (int w = 0; w < kRouteWarps; ++w) q += s_ssq[w * kpad + threadIdx.x];
+      part0[K * E + threadIdx.x] = q;
+    }
+  } else {
   for (int t0 = 0; t0 < K; t0 += TG) {
     const int kt = min(TG, K - t0);
     float ss[TG];
@@ -344,6 +469,7 @@ __global__ void __launch_bounds__(kRouteThreads) dx_route_kernel(DxRouteParams p
         if (lane == 0 && t < kt) part0[K * E + t0 + t] = q;
       }
     }
+  }
   }
   // y starts at zero, or as a copy of the block in the residual form; nothing reads it before this kernel is over
   for (int j = (crank * kRouteThreads + threadIdx.x) * 4; j < K * H; j += kRouteCluster * kRouteThreads * 4) {
@@ -439,11 +565,17 @@ __global__ void __launch_bounds__(kRouteThreads) dx_route_kernel(DxRouteParams p
 template <typename WT, int TG>
 static cudaError_t launch_route_one(const DxRouteParams& p, cudaStream_t st) {
   // CTA 0 holds one partial table per column slice (at most one per CTA of the cluster)
-  const size_t smem = (size_t)kRouteCluster * ((size_t)p.K * p.E + p.K) * sizeof(float);
+  size_t smem = (size_t)kRouteCluster * ((size_t)p.K * p.E + p.K) * sizeof(float);
+  // (tensor-core path) one partial table per warp: [8][tiles of 16 router rows][8 or 16 token columns], sums of squares
+  const size_t kpad = p.K > 8 ? 16 : 8;
+  if (std::is_same<WT, __nv_bfloat16>::value && TG == 4)
+    smem += (size_t)kRouteWarps * ((size_t)((p.E + 15) / 16) * 16 * kpad + kpad) * sizeof(float);
   // static + dynamic shared memory can pass the default 48 KB: opt in once per instantiation for the largest case
   static bool opted_in = false;
   if (!opted_in) {
-    const size_t most = (size_t)kRouteCluster * ((size_t)DX_MAX_K * DX_MAX_E + DX_MAX_K) * sizeof(float);
+    size_t most = (size_t)kRouteCluster * ((size_t)DX_MAX_K * DX_MAX_E + DX_MAX_K) * sizeof(float);
+    if (std::is_same<WT, __nv_bfloat16>::value && TG == 4)
+      most += (size_t)kRouteWarps * ((size_t)DX_MAX_E * 16 + 16) * sizeof(float);
     cudaError_t e = cudaFuncSetAttribute(dx_route_kernel<WT, TG>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)most);
     if (e != cudaSuccess) return e;
     opted_in = true;
