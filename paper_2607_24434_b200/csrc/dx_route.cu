@@ -9,13 +9,17 @@
 // constant and sits in registers before the previous kernel of the stream has
 // finished; once the block is final a thread needs two 16-byte loads per block
 // row and slab, so a single memory round trip separates "block ready" from the
-// arithmetic.  Partial logits go into CTA 0's shared memory through distributed
-// shared memory (one table per slice, summed in a fixed order, so the result
-// does not depend on timing); the hand-over is one hardware cluster barrier.
-// CTA 0 then selects, one warp per token, by ranking every logit against all
-// others (no selection rounds), builds the union as a bit mask, publishes the
-// group list the expert kernel is waiting for, and only then sorts the K*k
-// (token, expert) pairs by expert for the caller's outputs.
+// arithmetic.  For a bf16 router and blocks of more than two rows the products
+// run on the tensor cores (block rows as bf16 high part + residual, so the
+// logits keep fp32-like accuracy; one partial table per warp, added in a fixed
+// order); one or two rows and fp32 routers use plain FMAs.  Partial logits go
+// into CTA 0's shared memory through distributed shared memory (one table per
+// slice, summed in a fixed order, so the result does not depend on timing); the
+// hand-over is one hardware cluster barrier.  CTA 0 then selects, one warp per
+// token, in k rounds of warp-wide maximum on orderable keys, builds the union
+// as a bit mask, publishes the group list the expert kernel is waiting for, and
+// only then works out the gates and sorts the K*k (token, expert) pairs by
+// expert for the caller's outputs.
 #include <cooperative_groups.h>
 
 #include <type_traits>
