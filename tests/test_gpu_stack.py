@@ -128,3 +128,68 @@ def test_stack_graph_replay_handover():
     for L in Ls:
         L.close()
     ctx.close()
+
+
+@pytest.mark.parametrize("K", [8, 3])
+def test_many_overlapped_pairs_in_a_row(K):
+    """Hundreds of routing / expert kernel pairs back to back from a CUDA graph with nothing in between (draft step,
+    verify block and greedy accept on independent layers, as the benchmark's step): every pair's expert kernel lets
+    the next routing kernel start while it is still working, so anything of the hand-over that is read after that
+    point can be wiped under it (such a window is narrow: this is a soak, not a guaranteed catch).  No wait may
+    expire, and what the last replay leaves behind must be what the same calls give when each one is synchronised."""
+    from paper_2607_24434_b200 import binding
+    sh = synth.shape_v2lite()
+    n_layers = 3
+    ctx = binding.Context(0)
+    Ls, hs = [], []
+    for l in range(n_layers):
+        layer = synth.make_layer(sh, 800 + 10 * l, "cuda", zipf=True)
+        Ls.append(binding.Layer.from_weights(ctx, layer))
+        del layer
+        hs.append(synth.hidden_block(K, sh.hidden, 810 + l, 0.0, "cuda"))
+    W = synth.lm_head(4096, sh.hidden, 820, torch.bfloat16, "cuda")
+    rb = [binding._routing_buffers(sh, K, "cuda") for _ in range(n_layers)]
+    ys = [torch.empty((K, sh.hidden), device="cuda") for _ in range(n_layers)]
+    yd = torch.empty((1, sh.hidden), device="cuda")
+    db = {"topk_ids": torch.empty((sh.top_k,), dtype=torch.int32, device="cuda"),
+          "topk_w": torch.empty((sh.top_k,), device="cuda")}
+    dtok = torch.zeros((K,), dtype=torch.int32, device="cuda")
+    ab = {"target": torch.empty((K,), dtype=torch.int32, device="cuda"),
+          "n_accept": torch.empty((1,), dtype=torch.int32, device="cuda"),
+          "next_token": torch.empty((1,), dtype=torch.int32, device="cuda")}
+
+    def steps():
+        # verify blocks directly one after the other (the tightest overlap: routing kernel N + 1 starts the moment
+        # expert kernel N allows it), then the benchmark's step order
+        for rep in range(4):
+            for l in range(n_layers):
+                binding.moe_verify_block(Ls[l], hs[l], ys[l], rb[l])
+        for l in range(n_layers):
+            binding.moe_draft_step(Ls[l], hs[l][:1], yd, db)
+            binding.moe_verify_block(Ls[l], hs[l], ys[l], rb[l])
+            binding.spec_accept(ctx, ys[l], W, dtok, True, ab)
+
+    # reference: the same calls, one at a time
+    want = []
+    for l in range(n_layers):
+        o = binding.moe_verify_block(Ls[l], hs[l])
+        torch.cuda.synchronize()
+        want.append((o["y"].clone(), o["topk_ids"].clone()))
+    stream = torch.cuda.current_stream()
+    side = torch.cuda.Stream()
+    side.wait_stream(stream)
+    with torch.cuda.stream(side):
+        steps()
+    stream.wait_stream(side)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=side):
+        steps()
+    for _ in range(1000):
+        g.replay()
+    torch.cuda.synchronize()
+    assert ctx.device_status() == 0
+    for l in range(n_layers):
+        assert torch.equal(rb[l]["topk_ids"], want[l][1])
+        assert row_rel_err(ys[l].cpu().numpy(), want[l][0].cpu().numpy()).max() <= 1e-5
+    ctx.close()
