@@ -136,3 +136,40 @@ def test_draft_stack_refuses_mixed_shapes_and_fp32():
     for L in (a, b, c, d):
         L.close()
     ctx.close()
+
+
+def test_draft_stack_many_launches_in_a_row():
+    """Hundreds of persistent launches back to back (eager and from a CUDA graph): the scratch of one launch (delta
+    rows, logit words, arrival counters) is cleared in stream order before the next; no wait may expire and every
+    launch must leave the same row and the same selection."""
+    from paper_2607_24434_b200 import binding
+    sh = dataclasses.replace(synth.shape_v2lite(), n_experts=16)
+    ctx = binding.Context(0)
+    layers = [binding.Layer.from_weights(ctx, synth.make_layer(sh, 980 + l, "cuda")) for l in range(6)]
+    stack = binding.DraftStack(ctx, layers)
+    h0 = synth.hidden_block(1, sh.hidden, 990, 0.0, "cuda")
+    first = binding.moe_draft_stack(stack, h0)
+    torch.cuda.synchronize()
+    want_h, want_ids = first["h"].clone(), first["topk_ids"].clone()
+    out = {"topk_ids": torch.empty_like(want_ids), "topk_w": torch.empty_like(first["topk_w"])}
+    h_out = torch.empty_like(want_h)
+    for _ in range(200):
+        binding.moe_draft_stack(stack, h0, h_out, out)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == 0
+    assert torch.equal(out["topk_ids"], want_ids)
+    assert row_rel_err(h_out.cpu().numpy(), want_h.cpu().numpy().astype(np.float64)).max() <= 1e-5
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=side):
+        for _ in range(4):
+            binding.moe_draft_stack(stack, h0, h_out, out)
+    for _ in range(100):
+        g.replay()
+    torch.cuda.synchronize()
+    assert ctx.device_status() == 0
+    assert torch.equal(out["topk_ids"], want_ids)
+    assert row_rel_err(h_out.cpu().numpy(), want_h.cpu().numpy().astype(np.float64)).max() <= 1e-5
+    stack.close()
+    ctx.close()
