@@ -456,7 +456,17 @@ def run_gpu(args):
                      "timing": "CUDA events around back-to-back launches of the kernel alone over the rotating "
                                "layers (ms_per_launch); an event pair around single launches gives "
                                "ms_per_launch_isolated, which includes the launch gap",
-                     "algorithmic_bytes_per_launch": float(np.mean(exp_alg)), "union_sizes": union},
+                     "algorithmic_bytes_per_launch": float(np.mean(exp_alg)), "union_sizes": union,
+                     # the other kernels of the step, each timed back to back from its own graph, same peak
+                     "others": {
+                         "dx_accept_bf16_kernel (greedy accept, LM head streamed once)": {
+                             "ms_per_launch": comp.get("accept_ms", acc_ms),
+                             "achieved": acc_bytes / (comp.get("accept_ms", acc_ms) * 1e-3) / 1e9,
+                             "frac": acc_bytes / (comp.get("accept_ms", acc_ms) * 1e-3) / 1e9 / peak},
+                         "draft step (routing + expert kernel, one token)": {
+                             "ms_per_launch": comp.get("draft_step_ms", draft_ms),
+                             "achieved": draft_bytes / (comp.get("draft_step_ms", draft_ms) * 1e-3) / 1e9,
+                             "frac": draft_bytes / (comp.get("draft_step_ms", draft_ms) * 1e-3) / 1e9 / peak}}},
         "kernels": {"verify_experts_ms": float(np.mean(exp_ms)), "verify_route_ms": route_ms,
                     "verify_tokens_per_s": K / ((float(np.mean(exp_ms)) + route_ms) * 1e-3),
                     "draft_step_us": draft_ms * 1e3, "draft_gbs": draft_bytes / (draft_ms * 1e-3) / 1e9,
