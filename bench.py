@@ -173,9 +173,11 @@ def run_gpu(args):
         step(i)
     barrier()
     launches_per_step = 5
-    graph = None
+    graph = rem_graph = None
+    n_full, n_rem = divmod(args.steps, NL)
     if not args.no_graph:
-        # one CUDA graph holding a step on each of the NL layers; the timed loop replays it
+        # one CUDA graph holding a step on each of the NL layers, replayed steps // NL times, and a second graph with
+        # the remaining steps % NL steps: exactly --steps steps are timed
         side = torch.cuda.Stream()
         side.wait_stream(stream)
         with torch.cuda.stream(side):
@@ -189,7 +191,12 @@ def run_gpu(args):
             for i in range(NL):
                 step(i)
         launches_per_step = (ctx.kernel_launches() - l0) // NL
-        args.steps = max(NL, (args.steps + NL - 1) // NL * NL)
+        if n_rem:
+            rem_graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(rem_graph, stream=side):
+                for i in range(n_rem):
+                    step(i)
+            rem_graph.replay()
         for _ in range(2):
             graph.replay()
     barrier()
@@ -200,8 +207,10 @@ def run_gpu(args):
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
     if graph is not None:
-        for _ in range(args.steps // NL):
+        for _ in range(n_full):
             graph.replay()
+        if rem_graph is not None:
+            rem_graph.replay()
     else:
         for i in range(args.steps):
             step(i)
@@ -217,59 +226,13 @@ def run_gpu(args):
 
     check_status("the timed steps")
 
-    # ---- per-kernel timing of the dominant kernel (grouped SwiGLU of the verify block) and the others
+    # ---- per-kernel timings.  All of them use a fixed number of launches, whatever --steps is.
     ev = lambda: torch.cuda.Event(enable_timing=True)
-    t_exp, t_route, t_draft, t_acc = [], [], [], []
-    for i in range(min(args.steps, 400)):
-        li = i % NL
-        a, b, c, d, e, f = ev(), ev(), ev(), ev(), ev(), ev()
-        a.record(stream)
-        binding.moe_draft_step(layers[li], blocks[li][:1], yd, dbuf)
-        b.record(stream)
-        binding.moe_verify_route(layers[li], blocks[li], ys[li], rb[li])
-        c.record(stream)
-        binding.moe_verify_experts(layers[li], blocks[li], ys[li])
-        d.record(stream)
-        binding.spec_accept(ctx, ys[li], W_lm, draft_tok, True, abuf)
-        e.record(stream)
-        t_exp.append((c, d, li)); t_route.append((b, c)); t_draft.append((a, b)); t_acc.append((d, e))
-    torch.cuda.synchronize()
-    clocks = sampler.stop() if rank == 0 else None
-    union = [int(rb[li]["union_count"].item()) for li in range(NL)]
+    N_ISOLATED, N_BACK_TO_BACK = 200, 50          # event pairs around single launches; repetitions over the NL layers
     exp_bytes = binding.expert_blob_bytes(layers[0].shape, shape.inter)   # bytes of one expert as it is streamed
-    exp_ms_isolated = [x.elapsed_time(y) for x, y, _ in t_exp]
-    exp_alg = [(union[li] + shape.n_shared) * exp_bytes + 2 * K * H * 4 for _, _, li in t_exp]
 
-    # ---- the dominant kernel in a saturated stream: every layer gets its own context (own work list), is routed
-    # once, and then only the grouped-SwiGLU kernel is launched back to back over the rotating layers between two
-    # events, so the launch gap that an event pair around a single launch includes is not counted as kernel time
-    ctxs = [binding.Context(local) for _ in range(NL)]
-    twins = [layers[i].share(ctxs[i]) for i in range(NL)]
-    for i in range(NL):
-        binding.moe_verify_route(twins[i], blocks[i], ys[i], rb[i])
-    for i in range(NL):
-        binding.moe_verify_experts(twins[i], blocks[i], ys[i])
-    torch.cuda.synchronize()
-    reps = max(1, min(args.steps, 800) // NL)
-    x0, x1 = ev(), ev()
-    x0.record(stream)
-    for _ in range(reps):
-        for i in range(NL):
-            binding.moe_verify_experts(twins[i], blocks[i], ys[i])
-    x1.record(stream)
-    torch.cuda.synchronize()
-    exp_ms = [x0.elapsed_time(x1) / (reps * NL)] * len(exp_alg)
-    for t in twins:
-        t.close()
-    for c in ctxs:
-        c.close()
-    verify_gbs = sum(exp_alg) / (sum(exp_ms) * 1e-3) / 1e9
-    draft_ms = float(np.mean([x.elapsed_time(y) for x, y in t_draft]))
-    route_ms = float(np.mean([x.elapsed_time(y) for x, y in t_route]))
-    acc_ms = float(np.mean([x.elapsed_time(y) for x, y in t_acc]))
-
-    # ---- each component replayed back to back from its own CUDA graph (no launch gaps, routing overlapped)
     def graph_ms(fn, reps=200):
+        """fn(i) for the NL layers captured into one CUDA graph and replayed back to back: ms per call."""
         side = torch.cuda.Stream()
         side.wait_stream(stream)
         with torch.cuda.stream(side):
@@ -291,13 +254,101 @@ def run_gpu(args):
         torch.cuda.synchronize()
         return x0.elapsed_time(x1) / (reps * NL)
 
+    # every layer gets a second handle under its own context (own work list), so that back-to-back launches of the
+    # expert kernel alone never wait for another layer's routing
+    ctxs = [binding.Context(local) for _ in range(NL)]
+    twins = [layers[i].share(ctxs[i]) for i in range(NL)]
+
+    def measure_block(Kb, blocks_b, ys_b, rb_b):
+        """The grouped-SwiGLU kernel of a verify block of Kb rows, timed three ways (same bytes, same kernel):
+        pipelined  -- events around N_BACK_TO_BACK x NL back-to-back launches of the kernel alone over the rotating
+                      layers: the next launch's prologue overlaps the previous launch's tail;
+        isolated   -- an event pair around every single launch (launch gap and an empty pipeline included);
+        as_called  -- moe_verify_block (routing + experts, overlapped) replayed from a CUDA graph: what a caller
+                      gets, with the router's bytes added to the algorithmic bytes."""
+        iso = []
+        for i in range(N_ISOLATED):
+            li = i % NL
+            binding.moe_verify_route(layers[li], blocks_b[li], ys_b[li], rb_b[li])
+            c, d = ev(), ev()
+            c.record(stream)
+            binding.moe_verify_experts(layers[li], blocks_b[li], ys_b[li])
+            d.record(stream)
+            iso.append((c, d))
+        torch.cuda.synchronize()
+        union_b = [int(rb_b[li]["union_count"].item()) for li in range(NL)]
+        alg = float(np.mean([(u + shape.n_shared) * exp_bytes + 2 * Kb * H * 4 for u in union_b]))
+        iso_ms = float(np.mean([x.elapsed_time(y) for x, y in iso]))
+        for i in range(NL):
+            binding.moe_verify_route(twins[i], blocks_b[i], ys_b[i], rb_b[i])
+        for i in range(NL):
+            binding.moe_verify_experts(twins[i], blocks_b[i], ys_b[i])
+        torch.cuda.synchronize()
+        x0, x1 = ev(), ev()
+        x0.record(stream)
+        for _ in range(N_BACK_TO_BACK):
+            for i in range(NL):
+                binding.moe_verify_experts(twins[i], blocks_b[i], ys_b[i])
+        x1.record(stream)
+        torch.cuda.synchronize()
+        pipe_ms = x0.elapsed_time(x1) / (N_BACK_TO_BACK * NL)
+        res = {"K": Kb, "union_sizes": union_b, "algorithmic_bytes_per_launch": alg,
+               "launches_timed": {"pipelined": N_BACK_TO_BACK * NL, "isolated": N_ISOLATED},
+               "pipelined_ms": pipe_ms, "pipelined_gbs": alg / (pipe_ms * 1e-3) / 1e9,
+               "isolated_ms": iso_ms, "isolated_gbs": alg / (iso_ms * 1e-3) / 1e9}
+        if not args.no_graph:
+            blk_ms = graph_ms(lambda i: binding.moe_verify_block(layers[i], blocks_b[i], ys_b[i], rb_b[i]))
+            blk_alg = alg - 2 * Kb * H * 4 + shape.n_experts * H * 2
+            res.update({"as_called_ms": blk_ms, "as_called_gbs": blk_alg / (blk_ms * 1e-3) / 1e9,
+                        "as_called_tokens_per_s": Kb / (blk_ms * 1e-3)})
+        return res
+
+    blk = measure_block(K, blocks, ys, rb)
+    union = blk["union_sizes"]
+    # the other end of the block-length range the target is stated for
+    K8 = 8
+    blk8 = None
+    if K != K8 and not args.no_k8:
+        blocks8 = [synth.hidden_block(K8, H, 1000 + 50 * rank + 300 + i, 0.0, device) for i in range(NL)]
+        rb8 = [binding._routing_buffers(shape, K8, device) for _ in range(NL)]
+        ys8 = [torch.empty((K8, H), device=device) for _ in range(NL)]
+        blk8 = measure_block(K8, blocks8, ys8, rb8)
+    for t in twins:
+        t.close()
+    for c in ctxs:
+        c.close()
+
+    # the step's kernels one by one with an event pair around each call (launch gaps included)
+    t_route, t_draft, t_acc = [], [], []
+    for i in range(N_ISOLATED):
+        li = i % NL
+        a, b, c, d, e = ev(), ev(), ev(), ev(), ev()
+        a.record(stream)
+        binding.moe_draft_step(layers[li], blocks[li][:1], yd, dbuf)
+        b.record(stream)
+        binding.moe_verify_route(layers[li], blocks[li], ys[li], rb[li])
+        c.record(stream)
+        binding.moe_verify_experts(layers[li], blocks[li], ys[li])
+        d.record(stream)
+        binding.spec_accept(ctx, ys[li], W_lm, draft_tok, True, abuf)
+        e.record(stream)
+        t_route.append((b, c)); t_draft.append((a, b)); t_acc.append((d, e))
+    torch.cuda.synchronize()
+    clocks = sampler.stop() if rank == 0 else None
+    exp_alg = [blk["algorithmic_bytes_per_launch"]]
+    exp_ms = [blk["pipelined_ms"]]
+    verify_gbs = blk["pipelined_gbs"]
+    draft_ms = float(np.mean([x.elapsed_time(y) for x, y in t_draft]))
+    route_ms = float(np.mean([x.elapsed_time(y) for x, y in t_route]))
+    acc_ms = float(np.mean([x.elapsed_time(y) for x, y in t_acc]))
+
+    # ---- each component replayed back to back from its own CUDA graph (no launch gaps, routing overlapped)
     comp = {}
     if not args.no_graph:
-        comp["verify_block_ms"] = graph_ms(lambda i: binding.moe_verify_block(layers[i], blocks[i], ys[i], rb[i]))
+        comp["verify_block_ms"] = blk["as_called_ms"]
         comp["draft_step_ms"] = graph_ms(lambda i: binding.moe_draft_step(layers[i], blocks[i][:1], yd, dbuf))
         comp["accept_ms"] = graph_ms(lambda i: binding.spec_accept(ctx, ys[i], W_lm, draft_tok, True, abuf))
-        vb = float(np.mean([(union[li] + shape.n_shared) * exp_bytes for li in range(NL)])) + shape.n_experts * H * 2
-        comp["verify_block_gbs"] = vb / (comp["verify_block_ms"] * 1e-3) / 1e9
+        comp["verify_block_gbs"] = blk["as_called_gbs"]
         comp["verify_block_frac_of_8TBs"] = comp["verify_block_gbs"] / NOMINAL_HBM_GBS
         comp["verify_block_tokens_per_s"] = K / (comp["verify_block_ms"] * 1e-3)
         comp["draft_step_gbs"] = ((shape.n_shared + 2) * exp_bytes + shape.n_experts * H * 2) / (
@@ -422,6 +473,16 @@ def run_gpu(args):
         if dev_status != 0:
             raise RuntimeError(f"device status word {dev_status} set during the run (draft stack last)")
         dstack.close()
+
+    def fractions(b):
+        """The same kernel's three timings as fractions of the measured copy peak and of the nominal 8 TB/s."""
+        res = {}
+        for name in ("pipelined", "isolated", "as_called"):
+            if name + "_gbs" in b:
+                res[name] = {"ms": b[name + "_ms"], "gbs": b[name + "_gbs"], "of_peak": b[name + "_gbs"] / peak,
+                             "of_nominal_8TBs": b[name + "_gbs"] / NOMINAL_HBM_GBS}
+        return res
+
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -429,15 +490,8 @@ def run_gpu(args):
                   "and LM head, fp32 accumulate") if args.q4_resident else (
                       "bf16 weights, activations as bf16 tensor-core operands, fp32 accumulate"),
         "data": "synthetic",
-        "config": {"workload": "configs[1]: DeepSeek-V2-Lite-shaped MoE layer (H 2048, 64 experts x 1408, top-6, "
-                               "2 shared + 1 draft expert, Zipf(1.1) router bias); step = draft step (1 token) + "
-                               f"verify block K={K} + greedy accept over vocab {V}"
-                               + ("; experts resident in HBM as 4-bit blocks" if args.q4_resident else ""),
-                   "block_tokens": K, "vocab": V, "layers_rotated": NL,
-                   "l2": f"inputs larger than L2: steps rotate over {NL} independently seeded layers "
-                         f"({NL * (shape.n_experts + shape.n_shared + 1) * exp_bytes / 1e9:.1f} GB of weights)",
-                   "launch": "CUDA graph replay" if graph is not None else "eager launches",
-                   "parallelism": "replicas only" if world > 1 else "single GPU"},
+        "config": workload_config(shape, K, V, NL, exp_bytes, world, args.q4_resident),
+        "launch": "CUDA graph replay" if graph is not None else "eager launches",
         "gpu_launches": launches,
         "e2e": {"value": multi.throughput(units_all, e2e_ms), "unit": UNIT,
                 "h2d_bytes_per_step": K * H * 4 + K * 4, "d2h_bytes_per_step": K * H * 4 + K * 4 + 8,
@@ -447,16 +501,23 @@ def run_gpu(args):
                           "eager calls and one stream synchronisation per step"},
         "roofline": {"kernel": "dx_experts_bf16_kernel (grouped SwiGLU of the verify block)", "bound": "hbm",
                      "achieved": verify_gbs, "peak": peak, "unit": "GB/s", "frac": verify_gbs / peak,
+                     "frac_is": "pipelined: the kernel alone, back-to-back launches (see `fractions` for the other two "
+                                "ways of timing the same kernel; this is the most favourable of the three)",
                      "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBs": verify_gbs / NOMINAL_HBM_GBS,
+                     "fractions": fractions(blk),
                      "traffic": args.traffic if args.traffic is not None else (
                          None if args.q4_resident else NCU_TRAFFIC_RATIO * float(np.mean(exp_alg))),
                      "traffic_source": "ncu capture of a 2-layer case scaled by algorithmic bytes (see profiles/)",
-                     "ms_per_launch": float(np.mean(exp_ms)),
-                     "ms_per_launch_isolated": float(np.mean(exp_ms_isolated)),
-                     "timing": "CUDA events around back-to-back launches of the kernel alone over the rotating "
-                               "layers (ms_per_launch); an event pair around single launches gives "
-                               "ms_per_launch_isolated, which includes the launch gap",
+                     "ms_per_launch": blk["pipelined_ms"],
+                     "ms_per_launch_isolated": blk["isolated_ms"],
+                     "launches_timed": blk["launches_timed"],
+                     "timing": "CUDA events on the launch stream; a fixed number of launches whatever --steps is.  "
+                               "pipelined: events around back-to-back launches of the kernel alone over the rotating "
+                               "layers (the next launch's prologue overlaps the previous one's tail); isolated: an "
+                               "event pair around every single launch (launch gap included); as_called: "
+                               "moe_verify_block (routing + experts) replayed from a CUDA graph, router bytes added",
                      "algorithmic_bytes_per_launch": float(np.mean(exp_alg)), "union_sizes": union,
+                     "k8": None if blk8 is None else dict(blk8, fractions=fractions(blk8)),
                      # the other kernels of the step, each timed back to back from its own graph, same peak
                      "others": {
                          "dx_accept_bf16_kernel (greedy accept, LM head streamed once)": {
@@ -483,7 +544,7 @@ def run_gpu(args):
         "clocks": clocks,
     }
     if world == 1 and not args.no_cpu_baseline and not args.q4_resident:
-        out["cpu_baseline"] = cpu_baseline(shape, K, V, sample_vocab=args.cpu_vocab)
+        out["cpu_baseline"] = cpu_baseline(shape, K, V)
     print(json.dumps(out))
     if world > 1:
         torch.distributed.destroy_process_group()
@@ -614,78 +675,84 @@ def run_stack(args):
 
 
 def run_offload(args):
-    """configs[4]: offloaded V2-Lite-shaped stack.  Routed experts live in pinned host memory; each layer has an HBM
-    cache of 16 slots with LRU eviction; shared and draft experts are resident.  Per decode step: K draft tokens go
-    through the layers (the top-1 expert is staged on demand, the draft router's top-6 are prefetched on the side
-    stream), then the block is verified (route, read the union on the host, stage and evaluate it in waves) and
-    a scripted geometric(0.85) prefix is accepted.  Reports cache hit rate, prefetch hit / waste, host-to-device
-    GB/s and accepted tokens/s.  The routing decisions are read on the host (one sync per layer), which is the
-    serialisation on-demand loading inherently has; the workload is PCIe-bound by construction."""
-    from paper_2607_24434_b200 import binding
+    """configs[4]: offloaded V2-Lite-shaped stack, one exact DraftExpert decode step per iteration (Algorithm 1).
+    Routed experts live in pinned host memory; each layer has an HBM cache of 16 slots with LRU eviction; shared and
+    draft experts are resident.  Per step: draft tokens go one by one through the drafter's stack (chained residual
+    stream, top-1 expert staged on demand), each is scored by the draft LM head, the confidence-expansion controller
+    decides whether to keep it, and the newly predicted verifier experts are prefetched on the side stream; then the
+    block is verified through the target stack (route, read the union on the host, wait for useful transfers, load
+    misses on demand, waves if the union exceeds the slots) and greedily accepted.  The drafter's hidden states
+    differ from the verifier's from the second layer on, so its router's predictions can miss.  Two acceptance
+    modes: scripted geometric(0.85) (the draft experts are random, not trained) and closed-loop (the comparison's
+    own accepted length).  The routing decisions are read on the host (one sync per layer), which is the
+    serialisation on-demand loading inherently has; the workload is bound by the host link by construction."""
+    from paper_2607_24434_b200 import binding, decode
     torch.cuda.set_device(0)
     device = torch.device("cuda", 0)
     shape = synth.shape_v2lite()
-    K, NLAY, S = args.block, args.offload_layers, 16
+    NLAY, S, V, H = args.offload_layers, 16, args.vocab, shape.hidden
     ctx = binding.Context(0)
-    layers, pools = [], []
     nbytes = binding.expert_blob_bytes(shape, shape.inter)
+    pool_bytes = binding.q4_expert_bytes(shape, shape.inter) if args.q4 else nbytes
+    # the host pool first: if the box cannot pin it all, fewer layers are used (and reported)
+    pools = []
+    for l in range(NLAY):
+        try:
+            pools.append(torch.empty((shape.n_experts, pool_bytes), dtype=torch.uint8).pin_memory())
+        except RuntimeError:
+            break
+    if len(pools) < NLAY:
+        sys.stderr.write(f"could pin only {len(pools)} of {NLAY} layers' experts; running with that many\n")
+        NLAY = len(pools)
     cache = binding.ExpertCache(ctx, NLAY, shape.n_experts, S, nbytes)
     if args.q4:
         cache.set_q4(shape)      # host pool of 4-bit block-quantised experts, expanded into the slots after each copy
-    pool_bytes = binding.q4_expert_bytes(shape, shape.inter) if args.q4 else nbytes
+    layers = []
     for l in range(NLAY):
         w = synth.make_layer(shape, 3000 + l, device, zipf=True)
         L = binding.Layer.from_weights(ctx, w, routed_resident=False)
         torch.cuda.synchronize()
         if args.q4:
             Wg, Wu, Wd = w["experts"]
-            host = torch.stack([synth.q4_expert_blob(Wg[e].float().cpu(), Wu[e].float().cpu(), Wd[e].float().cpu())
-                                for e in range(shape.n_experts)]).pin_memory()
+            for e in range(shape.n_experts):
+                pools[l][e].copy_(synth.q4_expert_blob(Wg[e].float().cpu(), Wu[e].float().cpu(), Wd[e].float().cpu()))
         else:
-            host = L.blobs.cpu().pin_memory()
+            pools[l].copy_(L.blobs)
         L.blobs = None
         del w
         for e in range(shape.n_experts):
-            cache.register(l, e, host[e])
+            cache.register(l, e, pools[l][e])
         cache.attach(L, l)
-        layers.append(L); pools.append(host)
+        layers.append(L)
     torch.cuda.empty_cache()
-    H = shape.hidden
-    y = torch.empty((K, H), device=device)
-    yd = torch.empty((1, H), device=device)
-    rb = binding._routing_buffers(shape, K, device)
-    db = {"topk_ids": torch.empty((shape.top_k,), dtype=torch.int32, device=device),
-          "topk_w": torch.empty((shape.top_k,), dtype=torch.float32, device=device)}
+    emb = synth.embedding_table(V, H, 3998, device)
+    W_lm = synth.lm_head(V, H, 3999, torch.bfloat16, device)
+    dec = decode.OffloadedDecoder(ctx, layers, cache, emb, W_lm, k_max=args.k_max, tau=args.tau,
+                                  budget="cache" if args.budget < 0 else args.budget)
     rng = np.random.default_rng(11)
 
-    def step(i):
-        rows = synth.hidden_block(K, H, 5000 + i, 0.9, device)
-        cache.begin_step()
-        for t in range(K):                                   # draft phase
-            ht = rows[t:t + 1]
-            for l, L in enumerate(layers):
-                binding.moe_draft_route(L, ht, yd, db)
-                ids = db["topk_ids"].tolist()                # e1 and the predicted verifier experts
-                cache.stage(l, ids[:1])
-                binding.moe_draft_experts(L, ht, yd)
-                cache.prefetch(l, ids)
-        for l, L in enumerate(layers):                       # verify phase
-            binding.moe_verify_block_cached(L, cache, l, rows, y, rb)
+    def scripted():
         n = 0
-        while n < K and rng.random() < 0.85:
+        while n < args.k_max and rng.random() < 0.85:
             n += 1
         return n
 
+    closed = args.acceptance == "closed-loop"
+    t0_tok = 1
     for i in range(args.warmup):
-        step(i)
+        t0_tok = dec.step(t0_tok, scripted_accept=None if closed else scripted())["next"]
     torch.cuda.synchronize()
     st0 = cache.stats()
     t0 = time.perf_counter()
-    accepted = 0
+    accepted = emitted = drafted = rows = 0
     for i in range(args.offload_steps):
-        accepted += step(args.warmup + i)
+        r = dec.step(t0_tok, scripted_accept=None if closed else scripted())
+        t0_tok = r["next"]
+        accepted += r["n_accept"]; emitted += len(r["emitted"]); drafted += len(r["drafted"]); rows += r["block_rows"]
     torch.cuda.synchronize()
     dt = time.perf_counter() - t0
+    if ctx.device_status() != 0:
+        raise RuntimeError("device status word set during the offload run")
     st1 = cache.stats()
     d = {k: st1[k] - st0[k] for k in st1}
     steps = args.offload_steps
@@ -696,15 +763,25 @@ def run_offload(args):
         "config": {"workload": f"configs[4]: offloaded V2-Lite-shaped stack, {NLAY} MoE layers, experts in pinned host "
                                f"memory ({NLAY * shape.n_experts * pool_bytes / 1e9:.1f} GB, "
                                f"{'4-bit block-quantised, expanded to bf16 after each copy' if args.q4 else 'bf16 blobs'}), "
-                               f"{S} HBM slots per layer (LRU), "
-                               f"draft K={K} + prefetch of the draft router's top-{shape.top_k} + verify in waves; "
-                               "scripted geometric(0.85) acceptance", "layers": NLAY, "block_tokens": K},
-        "emitted_tokens_per_s": (accepted + steps) / dt,
+                               f"{S} HBM slots per layer (LRU); per step: draft up to {args.k_max} tokens through the "
+                               f"drafter's stack (chained residual stream), confidence-expansion controller "
+                               f"(tau {args.tau}, budget {'= free cache pairs' if args.budget < 0 else args.budget}), "
+                               f"prefetch of the newly predicted top-{shape.top_k} experts, verify through the target "
+                               f"stack in waves, greedy accept over vocab {V}",
+                   "layers": NLAY, "layers_requested": args.offload_layers, "k_max": args.k_max,
+                   "acceptance": "closed-loop (token chain through a seeded embedding table; random draft experts)"
+                                 if closed else "scripted geometric(0.85) prefix (stand-in for trained draft experts)"},
+        "emitted_tokens_per_s": emitted / dt,
+        "drafted_per_step": drafted / steps, "block_rows_per_step": rows / steps,
+        "acceptance_rate": accepted / max(1, drafted),
         "cache_hit_rate": d["hits"] / max(1, d["lookups"]),
         "prefetch_hit": d["prefetch_used"] / max(1, d["prefetch_issued"]),
         "prefetch_waste": d["prefetch_wasted"] / max(1, d["prefetch_issued"]),
-        "h2d_gbs": d["bytes_h2d"] / dt / 1e9, "cache": d,
+        "prefetch_note": "used / wasted are counted when they happen; experts prefetched in the last step and still "
+                         "pending are in neither",
+        "h2d_gbs": d["bytes_h2d"] / dt / 1e9, "waited_copies_per_step": d["waited_copies"] / steps, "cache": d,
     }))
+    dec.close()
 
 
 def _blas_threads() -> int:
@@ -722,14 +799,15 @@ def oracle_step(O, ref, h_np, W_np, draft, K):
     return O.greedy_accept_fast(O.rmsnorm(y), W_np, draft)
 
 
-def cpu_baseline(shape, K, V, sample_vocab, budget_s=12.0):
+def cpu_baseline(shape, K, V, budget_s=12.0):
     """Times the CPU checker, as it stands, on a bounded sample of the workload: whole steps (draft step + verify
-    block + greedy accept over a vocabulary slice) on one layer, repeated for about ``budget_s`` seconds."""
+    block + greedy accept over the full vocabulary) on one layer, repeated for about ``budget_s`` seconds."""
     from oracle import moe_oracle as O
     layer = synth.make_layer(shape, 4242, "cpu", zipf=True)
     ref = synth.layer_to_numpy(layer)
+    del layer
     h_np = synth.hidden_block(K, shape.hidden, 4243, 0.0).numpy().astype(np.float64)
-    W_np = synth.to_numpy_f32(synth.lm_head(sample_vocab, shape.hidden, 4244, torch.bfloat16))
+    W_np = synth.to_numpy_f32(synth.lm_head(V, shape.hidden, 4244, torch.bfloat16)).astype(np.float64)
     draft = np.zeros(K, np.int32)
     oracle_step(O, ref, h_np, W_np, draft, K)          # untimed first touch
     n, t0 = 0, time.perf_counter()
@@ -739,58 +817,91 @@ def cpu_baseline(shape, K, V, sample_vocab, budget_s=12.0):
         dt = time.perf_counter() - t0
         if dt >= budget_s or n >= 200:
             break
-    return {"value": K * n / dt, "unit": UNIT, "cores": _blas_threads(), "kind": "oracle",
+    return {"value": K * n / dt, "unit": UNIT, "cores": _blas_threads(), "kind": "oracle", "dtype": "f64",
             "seconds": dt, "steps": n,
-            "sample": f"{n} whole steps on one layer: draft step + verify block K={K} + greedy accept over the "
-                      f"first {sample_vocab} vocabulary rows (fp64 numpy, {dt:.1f} s of CPU work)"}
+            "sample": f"{n} whole steps on one layer of the {shape.n_experts}-expert shape: draft step + verify block "
+                      f"K={K} + greedy accept over all {V} vocabulary rows (the checker's default fp64 numpy "
+                      f"arithmetic, {dt:.1f} s of CPU work)"}
+
+
+def workload_config(shape, K, V, NL, exp_bytes, world=1, q4=False):
+    """The `config` object of the JSON line: the same for the GPU arm and the reference arm."""
+    return {"workload": "configs[1]: DeepSeek-V2-Lite-shaped MoE layer (H 2048, 64 experts x 1408, top-6, "
+                        "2 shared + 1 draft expert, Zipf(1.1) router bias); step = draft step (1 token) + "
+                        f"verify block K={K} + greedy accept over vocab {V}"
+                        + ("; experts resident in HBM as 4-bit blocks" if q4 else ""),
+            "block_tokens": K, "vocab": V, "layers_rotated": NL,
+            "l2": f"inputs larger than L2: steps rotate over {NL} independently seeded layers "
+                  f"({NL * (shape.n_experts + shape.n_shared + 1) * exp_bytes / 1e9:.1f} GB of weights)",
+            "parallelism": "replicas only" if world > 1 else "single GPU"}
 
 
 def run_reference(args):
-    """The reference arm: the CPU checker, as it stands, on the host cores (rank 0 only)."""
+    """The reference arm: the CPU checker, as it stands, on the host cores (rank 0 only), on the GPU arm's
+    configuration: the same seeded layers rotated in the same order, the same block length, the full vocabulary."""
     if int(os.environ.get("RANK", "0")) != 0:
         return
     from oracle import moe_oracle as O
     shape = synth.shape_v2lite()
-    K, V = args.block, args.cpu_vocab
-    n_layers = 1
-    refs = [synth.layer_to_numpy(synth.make_layer(shape, 1000 + i, "cpu", zipf=True)) for i in range(n_layers)]
-    hs = [synth.hidden_block(K, shape.hidden, 1100 + i, 0.0).numpy().astype(np.float64) for i in range(n_layers)]
-    W_np = synth.to_numpy_f32(synth.lm_head(V, shape.hidden, 1999, torch.bfloat16))
+    K, V, n_layers = args.block, args.vocab, args.layers
+    refs, hs = [], []
+    for i in range(n_layers):
+        layer = synth.make_layer(shape, 1000 + i, "cpu", zipf=True)
+        refs.append(synth.layer_to_numpy(layer))
+        del layer
+        hs.append(synth.hidden_block(K, shape.hidden, 1100 + i, 0.0).numpy().astype(np.float64))
+    W_np = synth.to_numpy_f32(synth.lm_head(V, shape.hidden, 1999, torch.bfloat16)).astype(np.float64)
     draft = np.zeros(K, np.int32)
     # bounded: the checker is slow by design, so at most ~2 minutes of it are timed
     budget_s, t_w = 120.0, time.perf_counter()
-    for i in range(min(args.warmup, 3)):
+    n_warm = max(1, min(args.warmup, n_layers))
+    for i in range(n_warm):
         oracle_step(O, refs[i % n_layers], hs[i % n_layers], W_np, draft, K)
-    per_step = (time.perf_counter() - t_w) / max(1, min(args.warmup, 3))
+    per_step = (time.perf_counter() - t_w) / n_warm
     timed = max(1, min(args.steps, int(budget_s / max(per_step, 1e-3))))
     t0 = time.perf_counter()
     for i in range(timed):
         oracle_step(O, refs[i % n_layers], hs[i % n_layers], W_np, draft, K)
     dt = time.perf_counter() - t0
     value = K * timed / dt
-    sample = (f"each step: draft step + verify block K={K} on one of {n_layers} layers + greedy accept over the "
-              f"first {V} vocabulary rows (fp64 numpy)")
+    sample = (f"each step: draft step + verify block K={K} on one of {n_layers} rotating layers + greedy accept over "
+              f"all {V} vocabulary rows (the checker's default fp64 numpy arithmetic)")
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": int(os.environ.get(
             "WORLD_SIZE", "1")), "steps": args.steps, "steps_timed": timed, "warmup": args.warmup, "ms_per_step": dt / timed * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": "configs[1]: DeepSeek-V2-Lite-shaped MoE layer; step = draft step + verify block "
-                               f"K={K} + greedy accept", "block_tokens": K, "vocab": V},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": _blas_threads(), "kind": "oracle", "sample": sample},
+        "config": workload_config(shape, K, V, n_layers, shape.expert_bytes()),
+        "launch": "host cores (numpy)",
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": _blas_threads(), "kind": "oracle", "dtype": "f64",
+                         "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
 
 
+def spawn_replicas(n: int) -> int:
+    """`python bench.py --gpus N` without a launcher: start N ranks of this script (one per GPU, replicas only)
+    under torch.distributed.run on this node and hand back its exit code."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
+
+
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--gpus", type=int, default=1,
+                    help="GPUs of this node, one replica each; under torchrun the ranks come from the environment, "
+                         "without a launcher N > 1 ranks are spawned here")
     ap.add_argument("--steps", type=int, default=8000)
     ap.add_argument("--warmup", type=int, default=16)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--block", type=int, default=4, help="verify block length K")
     ap.add_argument("--vocab", type=int, default=102400)
     ap.add_argument("--layers", type=int, default=8, help="independently seeded layers to rotate over")
-    ap.add_argument("--cpu-vocab", type=int, default=16384, help="vocabulary rows in the CPU-baseline sample")
+    ap.add_argument("--no-k8", action="store_true", help="skip the K = 8 figures of the dominant kernel")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="time eager launches instead of a CUDA graph replay")
     ap.add_argument("--stack-layers", type=int, default=26)
@@ -800,17 +911,24 @@ def main():
     ap.add_argument("--workload", default="layer", choices=["layer", "offload", "stack"],
                     help="layer: configs[1] (default, the driver's line); offload: configs[4] expert-cache workload; "
                          "stack: configs[2] / configs[3] layer stacks, K sweep and draft us per token")
-    ap.add_argument("--offload-layers", type=int, default=4)
+    ap.add_argument("--offload-layers", type=int, default=26)
+    ap.add_argument("--k-max", type=int, default=8, help="offload workload: most tokens drafted per step")
+    ap.add_argument("--tau", type=float, default=1.0, help="offload workload: confidence threshold of the stop rule")
+    ap.add_argument("--budget", type=int, default=-1,
+                    help="offload workload: layer-expert budget of the stop rule (-1: what is left of the cache)")
+    ap.add_argument("--acceptance", default="scripted", choices=["scripted", "closed-loop"])
     ap.add_argument("--q4", action="store_true",
                     help="offload workload: keep the host pool 4-bit block-quantised (Q4_0 blocks)")
     ap.add_argument("--q4-resident", action="store_true",
                     help="layer workload: experts resident in HBM as 4-bit blocks, de-quantised in the expert kernel")
-    ap.add_argument("--offload-steps", type=int, default=24)
+    ap.add_argument("--offload-steps", type=int, default=64)
     ap.add_argument("--traffic", type=float, default=None,
                     help="ncu DRAM bytes per launch of the dominant kernel, if known")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
+    if args.gpus > 1 and "RANK" not in os.environ and args.impl != "reference":
+        sys.exit(spawn_replicas(args.gpus))
     if args.workload == "offload" and args.impl != "reference":
         run_offload(args)
     elif args.workload == "stack" and args.impl != "reference":

@@ -66,7 +66,8 @@ enum {
   DX_DEV_OK = 0,
   DX_DEV_BAD_EXPERT_ID = 1,     /* a routed expert has no weight blob attached */
   DX_DEV_WAIT_EXPIRED = 2,      /* a bounded wait inside a kernel gave up */
-  DX_DEV_WORKLIST_OVERFLOW = 3
+  DX_DEV_WORKLIST_OVERFLOW = 3,
+  DX_DEV_BOUNDS = 4             /* checked build only (-DDX_CHECKED): an index left its range; the access was skipped */
 };
 
 typedef struct dx_ctx dx_ctx;
@@ -110,6 +111,21 @@ dx_status dx_last_device_status(dx_ctx* ctx, void* stream, int32_t* dev_status_o
  * time above).  fp32 layers and the single-token stack kernel always use fp32 activations; 4-bit layers always
  * plain bf16. */
 dx_status dx_set_activation_split(dx_ctx* ctx, int32_t on);
+/* Which kernels are launched so that they may begin while the kernel in front of them on the stream drains
+ * (programmatic stream serialization): bit 0 the routing kernel, bit 1 the expert kernels, bit 2 the greedy-accept
+ * kernels.  Default 3.  0 gives plain stream order everywhere; results never depend on the mask. */
+dx_status dx_set_launch_overlap(dx_ctx* ctx, int32_t mask);
+/* Every wait inside a kernel (for a word another kernel publishes, for a copy into shared memory, for the other CTAs
+ * of a cooperative launch) polls at most `polls` times, then records DX_DEV_WAIT_EXPIRED in the device status word and
+ * lets the kernel run to its end; the outputs of that call are then undefined, the context stays usable.  Default
+ * 2^22 polls (seconds); 0 restores it. */
+dx_status dx_set_wait_limit(dx_ctx* ctx, uint32_t polls);
+/* Exercises that give-up path without a fault: clears the hand-over words and launches the expert half of a verify
+ * block alone, as if the routing kernel it expects beside it never ran.  The kernel's waits run out, it returns, and
+ * dx_last_device_status reads DX_DEV_WAIT_EXPIRED; y is undefined afterwards.  Refused (DX_ERR_INVALID_ARG) unless the
+ * wait limit has been set to at most 2^16 polls, so that the kernel gives up within milliseconds; bf16 / 4-bit layers
+ * only.  h [K,H], y [K,H] device pointers as for moe_verify_block. */
+dx_status dx_selftest_wait_expiry(dx_layer* layer, const float* h, int32_t K, float* y, void* stream);
 /* Last cudaError_t seen by this context as an int (0 = none). */
 int32_t dx_last_cuda_error(dx_ctx* ctx);
 /* Number of kernels this context has launched so far (for launch accounting by a caller). */
@@ -153,6 +169,7 @@ dx_status dx_expand_q4_expert(dx_ctx* ctx, const dx_layer_desc* desc, int32_t in
  * The table is uploaded on the next compute call's stream, so set_* calls must not be interleaved with
  * compute calls that are still being captured into a CUDA graph. */
 dx_status dx_layer_create(dx_ctx* ctx, const dx_layer_desc* desc, dx_layer** out);
+/* (A layer attached to a cache may be destroyed before or after the cache: each side forgets the other.) */
 dx_status dx_layer_destroy(dx_layer* layer);
 dx_status dx_layer_set_router(dx_layer* layer, const void* W_r, const float* bias);
 dx_status dx_layer_set_shared(dx_layer* layer, int32_t s, const void* blob);
@@ -208,6 +225,27 @@ dx_status moe_verify_experts_range(dx_layer* layer, const float* h, int32_t K, f
 dx_status moe_draft_route(dx_layer* layer, const float* h, float* y, int32_t* topk_ids, float* topk_w,
                           void* stream);
 dx_status moe_draft_experts(dx_layer* layer, const float* h, float* y, void* stream);
+
+/* ---- the same two calls on a layer whose routed experts come through an expert cache (Sec. 3.5, Algorithm 1:
+ * "wait for useful in-flight prefetches", "any missed expert is still loaded on demand") ---------------------------
+ * The layer must be attached to a cache (dx_layer_attach_cache; DX_ERR_INVALID_ARG otherwise).  Both calls
+ * synchronise the host with `stream` once: the routing decision is made on the device, the copies are issued by
+ * the host.  residual != 0 selects the pre-norm residual form (h_out = h + MoE(RMSNorm(h))) of the next section.
+ *   moe_verify_block_cached: routes the block, reads the union back, and evaluates it in waves of at most
+ *     slots_per_layer experts -- first the experts the cache already holds (landed or in flight, so that no load
+ *     of this block evicts them before use), then the missing ones by ascending id -- each wave staged with
+ *     expert_cache_stage and evaluated by one launch of the expert kernel (shared experts with the first wave).
+ *     Routing outputs as for moe_verify_block (device, each may be NULL); host_union_ids [min(E,K*k)] /
+ *     host_union_count [1] (HOST pointers, may be NULL) receive the union the host read.
+ *   moe_draft_step_cached: routes the token, reads the k selected ids back (host_topk_ids [k], HOST pointer, may be
+ *     NULL: the predicted verifier experts to hand to dx_controller_propose / expert_cache_prefetch), stages e1 and
+ *     evaluates Eq. 5. */
+dx_status moe_verify_block_cached(dx_layer* layer, const float* h, int32_t K, float* y, int32_t residual,
+                                  int32_t* topk_ids, float* topk_w, uint64_t* union_mask, int32_t* union_ids,
+                                  int32_t* union_count, int32_t* offsets, int32_t* perm, int32_t* host_union_ids,
+                                  int32_t* host_union_count, void* stream);
+dx_status moe_draft_step_cached(dx_layer* layer, const float* h, float* y, int32_t residual, int32_t* topk_ids,
+                                float* topk_w, int32_t* host_topk_ids, void* stream);
 
 /* ---- pre-norm residual forms for layer stacks (synthetic stacks stub attention out) --------------------------
  * h_out = h_in + MoE(RMSNorm(h_in)) with unit gain and eps 1e-6, MoE = Eq. 4 (verify, [K,H]) or Eq. 5 (draft,
@@ -308,7 +346,8 @@ dx_status dx_squared_error(dx_ctx* ctx, const float* a, const float* b, int64_t 
  * The call performs no cudaMalloc / cudaFree and uses no allocating library routine.
  *   - M > 16 (or any size spec_accept rejects) returns DX_ERR_UNSUPPORTED; nothing is truncated.
  *   - The first call on a device resolves the array's device address (cudaGetSymbolAddress, with that device
- *     current) and reads two device attributes; make that first call before any stream capture.
+ *     current) and reads two device attributes; make that first call before any stream capture.  Host threads
+ *     that make the first call on a device at the same time are serialised inside (one does the set-up).
  *   - All calls share the one array, which keeps the previous call's contents; each call clears it on `stream`
  *     first.  Calls that overlap on the GPU (different streams, no ordering between them) race on it and give
  *     undefined results: keep calls to this entry point on one stream or order them yourself.
@@ -341,6 +380,8 @@ typedef struct {
   int64_t prefetch_wasted;  /* prefetched experts evicted before any use */
   int64_t evictions;
   int64_t bytes_h2d;
+  int64_t waited_copies;    /* experts asked for whose copy had not landed yet (the stream or the host waited) */
+  int64_t stall_ns;         /* host time spent polling for such copies in expert_cache_wait */
 } dx_cache_stats;
 
 dx_status expert_cache_create(dx_ctx* ctx, int32_t n_layers, int32_t n_experts, int32_t slots_per_layer,
@@ -359,6 +400,10 @@ dx_status expert_cache_stage(dx_cache* cache, int32_t layer, const int32_t* host
 dx_status expert_cache_wait(dx_cache* cache, int32_t layer, const int32_t* host_ids, int32_t n, void* stream,
                             double timeout_s);
 dx_status expert_cache_stats(dx_cache* cache, dx_cache_stats* out);
+/* Failure-detection aid: queues a host callback that sleeps `milliseconds` (at most 1000) on the cache's copy stream,
+ * so that copies issued after it complete that much later -- a slow link made on the host, with which the
+ * DX_ERR_TIMEOUT path of expert_cache_wait can be exercised.  Nothing on the GPU waits or spins meanwhile. */
+dx_status expert_cache_inject_transfer_delay(dx_cache* cache, int32_t milliseconds);
 /* Slot currently holding `expert` of `layer` (-1 if none) and whether its copy is still in flight. */
 dx_status expert_cache_query(dx_cache* cache, int32_t layer, int32_t expert, int32_t* slot_out,
                              int32_t* in_flight_out);

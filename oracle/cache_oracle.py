@@ -115,3 +115,17 @@ class ExpertCacheModel:
             touched.add(s)
             res["load"].append(e)
         return res
+
+    def stage_union(self, layer: int, union: Sequence[int]) -> List[List[int]]:
+        """A verification block whose expert set (Eq. 2, ascending ids) may exceed the slots: it is evaluated in
+        waves of at most S experts, the ones already held first (so that no load of this block can evict them
+        before they are used), then the missing ones by ascending id; each wave is one ``stage``.  Returns the
+        waves.  (The paper does not say what happens when a block needs more experts than the accelerator holds;
+        this is the stated reading.)"""
+        held = [e for e in union if self.slot_of(layer, e) >= 0]
+        missing = [e for e in union if self.slot_of(layer, e) < 0]
+        order = held + missing
+        waves = [order[i:i + self.S] for i in range(0, len(order), self.S)]
+        for w in waves:
+            self.stage(layer, w)
+        return waves

@@ -40,7 +40,7 @@ class LayerDesc(C.Structure):
 
 class CacheStats(C.Structure):
     _fields_ = [(n, C.c_int64) for n in ("lookups", "hits", "on_demand", "prefetch_issued", "prefetch_used",
-                                         "prefetch_wasted", "evictions", "bytes_h2d")]
+                                         "prefetch_wasted", "evictions", "bytes_h2d", "waited_copies", "stall_ns")]
 
 
 _P = C.c_void_p
@@ -52,6 +52,9 @@ SIGNATURES = {
     "dx_destroy": (_I, [_P]),
     "dx_last_device_status": (_I, [_P, _P, C.POINTER(_I)]),
     "dx_set_activation_split": (_I, [_P, _I]),
+    "dx_set_launch_overlap": (_I, [_P, _I]),
+    "dx_set_wait_limit": (_I, [_P, C.c_uint32]),
+    "dx_selftest_wait_expiry": (_I, [_P, _P, _I, _P, _P]),
     "dx_last_cuda_error": (_I, [_P]),
     "dx_kernel_launches": (C.c_int64, [_P]),
     "dx_expert_blob_bytes": (_I, [C.POINTER(LayerDesc), _I, C.POINTER(C.c_size_t)]),
@@ -77,6 +80,8 @@ SIGNATURES = {
     "moe_verify_experts_range": (_I, [_P, _P, _I, _P, _I, _I, _I, _P]),
     "moe_draft_route": (_I, [_P, _P, _P, _P, _P, _P]),
     "moe_draft_experts": (_I, [_P, _P, _P, _P]),
+    "moe_verify_block_cached": (_I, [_P, _P, _I, _P, _I, _P, _P, _P, _P, _P, _P, _P, _P, C.POINTER(_I), _P]),
+    "moe_draft_step_cached": (_I, [_P, _P, _P, _I, _P, _P, _P, _P]),
     "moe_verify_block_residual": (_I, [_P, _P, _P, _I, _P, _P, _P, _P, _P, _P, _P, _P]),
     "spec_accept": (_I, [_P, _P, _I, _P, _I, _I, _I, _P, _I, _I, _P, _P, _P, _P]),
     "spec_draft_token": (_I, [_P, _P, _I, _P, _I, _I, _I, _I, _P, _P, _P]),
@@ -100,6 +105,7 @@ SIGNATURES = {
     "expert_cache_stage": (_I, [_P, _I, _P, _I, _P]),
     "expert_cache_wait": (_I, [_P, _I, _P, _I, _P, C.c_double]),
     "expert_cache_stats": (_I, [_P, C.POINTER(CacheStats)]),
+    "expert_cache_inject_transfer_delay": (_I, [_P, _I]),
     "expert_cache_query": (_I, [_P, _I, _I, C.POINTER(_I), C.POINTER(_I)]),
 }
 
@@ -153,6 +159,12 @@ class Context:
 
     def set_activation_split(self, on: bool) -> None:
         _check(self.lib.dx_set_activation_split(self.handle, 1 if on else 0), "dx_set_activation_split")
+
+    def set_launch_overlap(self, mask: int) -> None:
+        _check(self.lib.dx_set_launch_overlap(self.handle, mask), "dx_set_launch_overlap")
+
+    def set_wait_limit(self, polls: int) -> None:
+        _check(self.lib.dx_set_wait_limit(self.handle, polls), "dx_set_wait_limit")
 
     def close(self) -> None:
         if self.handle:
@@ -505,6 +517,10 @@ class ExpertCache:
         st = _stream() if self.ctx else None
         _check(self.lib.expert_cache_wait(self.handle, layer, arr, n, st, timeout_s), "expert_cache_wait")
 
+    def inject_transfer_delay(self, milliseconds: int) -> None:
+        _check(self.lib.expert_cache_inject_transfer_delay(self.handle, milliseconds),
+               "expert_cache_inject_transfer_delay")
+
     def stats(self) -> Dict[str, int]:
         s = CacheStats()
         _check(self.lib.expert_cache_stats(self.handle, C.byref(s)), "expert_cache_stats")
@@ -533,30 +549,50 @@ def moe_draft_experts(layer: Layer, h: torch.Tensor, y: torch.Tensor) -> None:
 
 
 def moe_verify_block_cached(layer: Layer, cache: ExpertCache, layer_index: int, h: torch.Tensor,
-                            y: Optional[torch.Tensor] = None, out: Optional[Dict[str, torch.Tensor]] = None):
-    """Verify block on a layer whose routed experts come through ``cache``: route, read the union on the host
-    (the one host round trip on-demand loading needs), then stage and evaluate the union in waves of at most
-    ``cache.slots`` experts in ascending id order, shared experts with the first wave."""
+                            y: Optional[torch.Tensor] = None, out: Optional[Dict[str, torch.Tensor]] = None,
+                            residual: bool = False):
+    """Verify block on a layer whose routed experts come through ``cache`` (``moe_verify_block_cached`` of the
+    library: route, one read of the union on the host, waves of at most ``cache.slots`` experts -- cached ones
+    first, then misses by ascending id).  ``cache`` / ``layer_index`` are what the layer was attached with."""
     K = h.shape[0]
     if out is None:
         out = _routing_buffers(layer.shape, K, h.device)
     if y is None:
         y = torch.empty_like(h)
-    moe_verify_route(layer, h, y, out)
-    n = int(out["union_count"].item())
-    ids = out["union_ids"][:n].tolist()
-    S = cache.slots
-    first = 0
-    while True:
-        wave = ids[first:first + S]
-        cache.stage(layer_index, wave)
-        moe_verify_experts_range(layer, h, y, first, len(wave), include_shared=(first == 0))
-        first += len(wave)
-        if first >= n:
-            break
-    out["y"] = y
-    out["union_list"] = ids
+    cap = min(layer.shape.n_experts, K * layer.shape.top_k)
+    host_ids = (C.c_int32 * cap)()
+    host_n = _I(0)
+    _check(layer.lib.moe_verify_block_cached(layer.handle, _ptr(h), K, _ptr(y), 1 if residual else 0,
+                                             _ptr(out["topk_ids"]), _ptr(out["topk_w"]), _ptr(out["union_mask"]),
+                                             _ptr(out["union_ids"]), _ptr(out["union_count"]), _ptr(out["offsets"]),
+                                             _ptr(out["perm"]), host_ids, C.byref(host_n), _stream()),
+           "moe_verify_block_cached")
+    out["h" if residual else "y"] = y
+    out["union_list"] = [int(host_ids[i]) for i in range(host_n.value)]
     return out
+
+
+def moe_draft_step_cached(layer: Layer, h: torch.Tensor, y: Optional[torch.Tensor] = None,
+                          out: Optional[Dict[str, torch.Tensor]] = None, residual: bool = False):
+    """Draft step (Eq. 5) on a cache-attached layer: route, read the selection on the host, stage e1, experts.
+    ``out["host_ids"]`` is the router's top-k as a Python list (the predicted verifier experts)."""
+    sh = layer.shape
+    if out is None:
+        out = {"topk_ids": torch.empty((sh.top_k,), dtype=torch.int32, device=h.device),
+               "topk_w": torch.empty((sh.top_k,), dtype=torch.float32, device=h.device)}
+    if y is None:
+        y = torch.empty_like(h)
+    host_ids = (C.c_int32 * sh.top_k)()
+    _check(layer.lib.moe_draft_step_cached(layer.handle, _ptr(h), _ptr(y), 1 if residual else 0, _ptr(out["topk_ids"]),
+                                           _ptr(out["topk_w"]), host_ids, _stream()), "moe_draft_step_cached")
+    out["h" if residual else "y"] = y
+    out["host_ids"] = [int(host_ids[j]) for j in range(sh.top_k)]
+    return out
+
+
+def selftest_wait_expiry(layer: Layer, h: torch.Tensor, y: torch.Tensor) -> None:
+    _check(layer.lib.dx_selftest_wait_expiry(layer.handle, _ptr(h), h.shape[0], _ptr(y), _stream()),
+           "dx_selftest_wait_expiry")
 
 
 def moe_draft_step_topr(layer: Layer, h: torch.Tensor, top_r: int, use_draft_expert: bool,

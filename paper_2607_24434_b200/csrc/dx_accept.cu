@@ -14,6 +14,8 @@
 // merged as packed 64-bit keys (orderable logit << 32 | ~index) with
 // atomicMax, and the CTA that takes the last ticket turns the keys into
 // tokens, the accepted length and the next token.
+#include <mutex>
+
 #include "dx_internal.cuh"
 
 namespace {
@@ -58,6 +60,7 @@ struct AcceptParams {
   unsigned int* ticket;
   float* conf;          // [M] softmax probability of the argmax (only the CONF variants)
   float2* conf_part;    // [grid][DX_MAX_M] per-CTA (running max, sum of exp) pairs
+  int32_t* dev_status;  // the context's status word (null for the context-free entry point)
 };
 
 // online softmax bookkeeping: (m, s) with s = sum exp(l - m) over the logits seen so far
@@ -89,6 +92,9 @@ __device__ __forceinline__ void finish(const AcceptParams& p, unsigned long long
   if (threadIdx.x < p.M) {
     unsigned long long kk = __ldcg(p.keys + threadIdx.x);
     int tok = (int)(0xffffffffu - (unsigned)(kk & 0xffffffffull));
+#ifdef DX_CHECKED
+    if (p.dev_status && !(tok >= 0 && tok < p.V)) atomicExch(p.dev_status, (int32_t)DX_DEV_BOUNDS);
+#endif
     s_tok[threadIdx.x] = tok;
     p.target[threadIdx.x] = tok;
     p.keys[threadIdx.x] = 0ull;
@@ -324,19 +330,19 @@ static cudaError_t launch_accept_bf16(dx_ctx* ctx, const AcceptParams& p, size_t
   cudaError_t e = cudaFuncSetAttribute(dx_accept_bf16_kernel<NT, CONF>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)smem);
   if (e != cudaSuccess) return e;
-  return dx_launch_pdl(DX_PDL_ACCEPT, dx_accept_bf16_kernel<NT, CONF>, dim3(ctx->sm_count), dim3(512), smem, st, 1, p);
+  return dx_launch_pdl((ctx->pdl_mask & DX_PDL_ACCEPT) != 0, dx_accept_bf16_kernel<NT, CONF>, dim3(ctx->sm_count), dim3(512), smem, st, 1, p);
 }
 
 cudaError_t dx_launch_accept(dx_ctx* ctx, const float* h, int M, const void* W_lm, int V, int H, int w_dtype,
                              const int32_t* draft, int K, int rms_norm, int32_t* target, int32_t* n_accept,
                              int32_t* next_token, float* conf, cudaStream_t st) {
   AcceptParams p{h, M, V, H, W_lm, draft, K, rms_norm, target, n_accept, next_token, ctx->keys, ctx->ticket + 1,
-                 conf, ctx->conf_part};
+                 conf, ctx->conf_part, ctx->dev_status};
   if (w_dtype == DX_DTYPE_FP32) {
     int grid = (V + 7) / 8;
     if (grid > ctx->sm_count * 8) grid = ctx->sm_count * 8;
-    if (conf) return dx_launch_pdl(DX_PDL_ACCEPT, dx_accept_fp32_kernel<true>, dim3(grid), dim3(256), 0, st, 1, p);
-    return dx_launch_pdl(DX_PDL_ACCEPT, dx_accept_fp32_kernel<false>, dim3(grid), dim3(256), 0, st, 1, p);
+    if (conf) return dx_launch_pdl((ctx->pdl_mask & DX_PDL_ACCEPT) != 0, dx_accept_fp32_kernel<true>, dim3(grid), dim3(256), 0, st, 1, p);
+    return dx_launch_pdl((ctx->pdl_mask & DX_PDL_ACCEPT) != 0, dx_accept_fp32_kernel<false>, dim3(grid), dim3(256), 0, st, 1, p);
   }
   const int NT = (M + 7) / 8;
   const size_t smem = (size_t)NT * (H / 32) * 32 * 16 * 2;
@@ -360,7 +366,8 @@ static __device__ __align__(256) unsigned long long g_noalloc_scratch[kNoAllocMa
 
 namespace {
 struct NoAllocDevice {
-  bool ready = false;
+  std::once_flag once;     // the set-up below runs once per device, whichever host thread gets there first
+  bool ok = false;
   unsigned long long* scratch = nullptr;
   int sm_count = 0;
   int smem_optin = 0;
@@ -381,16 +388,17 @@ extern "C" dx_status spec_accept_noalloc(const float* h, int32_t M, const void* 
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return DX_ERR_CUDA;
   NoAllocDevice& d = g_noalloc_dev[dev];
-  if (!d.ready) {
-    // first call on this device (with this device current): resolve the device address of the scratch array
+  // first call on this device (with this device current): resolve the device address of the scratch array.  Host
+  // threads that arrive together are serialised here; the others see a fully initialised record.
+  std::call_once(d.once, [&d, dev] {
     void* ptr = nullptr;
-    if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess || ptr == nullptr) return DX_ERR_CUDA;
-    if (cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return DX_ERR_CUDA;
-    if (cudaDeviceGetAttribute(&d.smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess)
-      return DX_ERR_CUDA;
+    if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess || ptr == nullptr) return;
+    if (cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return;
+    if (cudaDeviceGetAttribute(&d.smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) return;
     d.scratch = static_cast<unsigned long long*>(ptr);
-    d.ready = true;
-  }
+    d.ok = true;
+  });
+  if (!d.ok) return DX_ERR_CUDA;
   const int NT = (M + 7) / 8;
   const size_t smem = (size_t)NT * (H / 32) * 32 * 16 * 2;
   if (w_dtype == DX_DTYPE_BF16 && smem > (size_t)d.smem_optin) return DX_ERR_UNSUPPORTED;
@@ -399,7 +407,7 @@ extern "C" dx_status spec_accept_noalloc(const float* h, int32_t M, const void* 
   if (cudaMemsetAsync(d.scratch, 0, sizeof(unsigned long long) * (kNoAllocMaxRows + 2), st) != cudaSuccess)
     return DX_ERR_CUDA;
   AcceptParams p{h, M, V, H, W_lm, draft, K, rms_norm, target, n_accept, next_token, d.scratch,
-                 reinterpret_cast<unsigned int*>(d.scratch + kNoAllocMaxRows), nullptr, nullptr};
+                 reinterpret_cast<unsigned int*>(d.scratch + kNoAllocMaxRows), nullptr, nullptr, nullptr};
   cudaError_t e;
   if (w_dtype == DX_DTYPE_FP32) {
     int grid = (V + 7) / 8;

@@ -5,17 +5,8 @@
 
 #include "dx_internal.cuh"
 
-#include <cstdlib>
-
 bool dx_bf16_hidden_supported(int H);
-
-int dx_pdl_mask() {
-  static const int mask = [] {
-    const char* v = std::getenv("DX_PDL_MASK");
-    return v ? std::atoi(v) : (DX_PDL_ROUTE | DX_PDL_EXPERTS);
-  }();
-  return mask;
-}
+void dx_cache_forget_layer(dx_cache* c, dx_layer* L);
 
 #define DX_CUDA(ctx, call)                 \
   do {                                     \
@@ -51,6 +42,8 @@ extern "C" dx_status dx_create(int device, dx_ctx** out) {
   ctx->device = device;
   ctx->last_cuda = cudaSuccess;
   ctx->launches = 0;
+  ctx->pdl_mask = DX_PDL_ROUTE | DX_PDL_EXPERTS;
+  ctx->wait_limit = DX_WAIT_LIMIT_DEFAULT;
   cudaError_t e = cudaSetDevice(device);
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, device);
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device);
@@ -62,6 +55,9 @@ extern "C" dx_status dx_create(int device, dx_ctx** out) {
   if (e == cudaSuccess) e = cudaMemset(ctx->handover, 0, 4 * sizeof(unsigned int));
   if (e == cudaSuccess) e = cudaMalloc(&ctx->conf_part, sizeof(float2) * 8 * ctx->sm_count * DX_MAX_M);
   if (e == cudaSuccess) e = cudaMalloc(&ctx->scratch_i32, sizeof(int32_t) * 2);
+  if (e == cudaSuccess) e = cudaMalloc(&ctx->union_dev, sizeof(int32_t) * (DX_MAX_E + 1 + DX_MAX_TOPK));
+  if (e == cudaSuccess) e = cudaHostAlloc((void**)&ctx->union_host, sizeof(int32_t) * (DX_MAX_E + 1 + DX_MAX_TOPK),
+                                          cudaHostAllocDefault);
   if (e == cudaSuccess) e = cudaMemset(ctx->work, 0, sizeof(DxWork));
   if (e == cudaSuccess) e = cudaMemset(ctx->ticket, 0, sizeof(unsigned int) * 4);
   if (e == cudaSuccess) e = cudaMemset(ctx->keys, 0, sizeof(unsigned long long) * DX_MAX_M);
@@ -84,6 +80,8 @@ extern "C" dx_status dx_destroy(dx_ctx* ctx) {
   cudaFree(ctx->handover);
   cudaFree(ctx->conf_part);
   cudaFree(ctx->scratch_i32);
+  cudaFree(ctx->union_dev);
+  if (ctx->union_host) cudaFreeHost(ctx->union_host);
   delete ctx;
   return DX_OK;
 }
@@ -100,6 +98,18 @@ extern "C" dx_status dx_last_device_status(dx_ctx* ctx, void* stream, int32_t* o
 extern "C" dx_status dx_set_activation_split(dx_ctx* ctx, int32_t on) {
   if (!ctx) return DX_ERR_INVALID_ARG;
   ctx->act_split = on ? 1 : 0;
+  return DX_OK;
+}
+
+extern "C" dx_status dx_set_launch_overlap(dx_ctx* ctx, int32_t mask) {
+  if (!ctx || mask < 0 || mask > (DX_PDL_ROUTE | DX_PDL_EXPERTS | DX_PDL_ACCEPT)) return DX_ERR_INVALID_ARG;
+  ctx->pdl_mask = mask;
+  return DX_OK;
+}
+
+extern "C" dx_status dx_set_wait_limit(dx_ctx* ctx, uint32_t polls) {
+  if (!ctx) return DX_ERR_INVALID_ARG;
+  ctx->wait_limit = polls ? polls : DX_WAIT_LIMIT_DEFAULT;
   return DX_OK;
 }
 
@@ -208,6 +218,7 @@ extern "C" dx_status dx_layer_create(dx_ctx* ctx, const dx_layer_desc* desc, dx_
 
 extern "C" dx_status dx_layer_destroy(dx_layer* L) {
   if (!L) return DX_ERR_INVALID_ARG;
+  if (L->cache) dx_cache_forget_layer(L->cache, L);   // the cache must not patch a table that is gone
   cudaFree((void*)L->table_dev);
   delete[] L->table_host;
   delete L;
@@ -295,14 +306,15 @@ static dx_status do_route(dx_layer* L, const float* h, int K, float* y, const Ro
   p.union_mask = (unsigned long long*)o.union_mask; p.union_ids = o.union_ids; p.union_count = o.union_count;
   p.offsets = o.offsets; p.perm = o.perm;
   // (the router of a layer with 4-bit experts is bf16)
-  DX_CUDA(ctx, dx_launch_route(p, d.weight_dtype == DX_DTYPE_Q4 ? DX_DTYPE_BF16 : d.weight_dtype, st));
+  DX_CUDA(ctx, dx_launch_route(ctx, p, d.weight_dtype == DX_DTYPE_Q4 ? DX_DTYPE_BF16 : d.weight_dtype, st));
   ctx->launches++;
   return DX_OK;
 }
 
 static dx_status do_experts(dx_layer* L, const float* h, int K, float* y, bool draft, bool residual,
                             cudaStream_t st, int first_routed = 0, int n_routed = -1, bool do_static = true,
-                            bool paired = false, bool skip_shared = false) {
+                            bool paired = false, bool skip_shared = false,
+                            const unsigned long long* subset = nullptr) {
   dx_ctx* ctx = L->ctx;
   const dx_layer_desc& d = L->desc;
   if (!h || !y || h == y) return DX_ERR_INVALID_ARG;
@@ -314,6 +326,7 @@ static dx_status do_experts(dx_layer* L, const float* h, int K, float* y, bool d
   p.x = h;
   p.y = y;
   p.table = L->table_dev;
+  p.table_len = L->table_len;
   p.work = ctx->work;
   p.dev_status = ctx->dev_status;
   p.H = d.hidden;
@@ -325,10 +338,13 @@ static dx_status do_experts(dx_layer* L, const float* h, int K, float* y, bool d
   p.routed_tiles = d.inter / DX_TILE_I;
   p.gamma = d.draft_gamma;
   p.handover = paired ? ctx->handover : nullptr;
+  p.wait_limit = ctx->wait_limit;
   p.first_routed = first_routed;
   p.n_routed = n_routed;
   p.do_static = do_static ? 1 : 0;
   p.skip_shared = skip_shared ? 1 : 0;
+  p.use_subset = subset ? 1 : 0;
+  for (int i = 0; i < DX_MAX_E / 64; ++i) p.subset[i] = subset ? subset[i] : 0ull;
   DX_CUDA(ctx, dx_launch_experts(ctx, p, L->desc.weight_dtype, K, st));
   ctx->launches++;
   if (L->cache) dx_cache_note_use(L->cache, L->cache_layer, st);
@@ -421,6 +437,102 @@ extern "C" dx_status moe_verify_block_residual(dx_layer* L, const float* h_in, f
   cudaStream_t st = (cudaStream_t)stream;
   RouteOut o{topk_ids, topk_w, union_mask, union_ids, union_count, offsets, perm};
   return do_pair(L, h_in, K, h_out, o, false, true, st);
+}
+
+// ---- layers whose routed experts come through an expert cache (Sec. 3.5, Algorithm 1) ------------------------
+int dx_cache_slot_of(const dx_cache* c, int layer, int expert);
+int dx_cache_slots(const dx_cache* c);
+
+// Device -> pinned host copy of `n` ints behind the routing kernel, then a host wait: the one round trip
+// on-demand loading needs (the routing decision is made on the device, the copies are issued by the host).
+static dx_status read_back(dx_ctx* ctx, const int32_t* dev, int n, int32_t* host_pinned, cudaStream_t st) {
+  DX_CUDA(ctx, cudaMemcpyAsync(host_pinned, dev, sizeof(int32_t) * n, cudaMemcpyDeviceToHost, st));
+  DX_CUDA(ctx, cudaStreamSynchronize(st));
+  return DX_OK;
+}
+
+extern "C" dx_status moe_verify_block_cached(dx_layer* L, const float* h, int32_t K, float* y, int32_t residual,
+                                             int32_t* topk_ids, float* topk_w, uint64_t* union_mask,
+                                             int32_t* union_ids, int32_t* union_count, int32_t* offsets,
+                                             int32_t* perm, int32_t* host_union_ids, int32_t* host_union_count,
+                                             void* stream) {
+  if (!L) return DX_ERR_INVALID_ARG;
+  if (!L->cache) return DX_ERR_INVALID_ARG;
+  dx_ctx* ctx = L->ctx;
+  dx_cache* c = L->cache;
+  cudaStream_t st = (cudaStream_t)stream;
+  const int E = L->desc.n_experts;
+  // the union goes to the context's scratch if the caller does not want it, and from there to the host
+  int32_t* uid = union_ids ? union_ids : ctx->union_dev;
+  int32_t* ucnt = union_count ? union_count : ctx->union_dev + DX_MAX_E;
+  RouteOut o{topk_ids, topk_w, union_mask, uid, ucnt, offsets, perm};
+  dx_status s = do_route(L, h, K, y, o, false, residual != 0, st);
+  if (s != DX_OK) return s;
+  const int cap = E < K * L->desc.top_k ? E : K * L->desc.top_k;
+  DX_CUDA(ctx, cudaMemcpyAsync(ctx->union_host, uid, sizeof(int32_t) * cap, cudaMemcpyDeviceToHost, st));
+  s = read_back(ctx, ucnt, 1, ctx->union_host + DX_MAX_E, st);
+  if (s != DX_OK) return s;
+  const int n = ctx->union_host[DX_MAX_E];
+  if (n < 0 || n > cap) return DX_ERR_CUDA;
+  if (host_union_count) *host_union_count = n;
+  if (host_union_ids)
+    for (int i = 0; i < n; ++i) host_union_ids[i] = ctx->union_host[i];
+  // Waves of at most S experts: the ones the cache already holds (landed or in flight) first, so that no load of
+  // this block can evict them before they are used, then the missing ones in ascending id order.
+  const int S = dx_cache_slots(c);
+  int32_t order[DX_MAX_E];
+  int m = 0;
+  for (int i = 0; i < n; ++i)
+    if (dx_cache_slot_of(c, L->cache_layer, ctx->union_host[i]) >= 0) order[m++] = ctx->union_host[i];
+  for (int i = 0; i < n; ++i)
+    if (dx_cache_slot_of(c, L->cache_layer, ctx->union_host[i]) < 0) order[m++] = ctx->union_host[i];
+  int first = 0;
+  do {
+    const int cnt = n - first < S ? n - first : S;
+    unsigned long long subset[DX_MAX_E / 64] = {};
+    for (int i = 0; i < cnt; ++i) subset[order[first + i] >> 6] |= 1ull << (order[first + i] & 63);
+    s = expert_cache_stage(c, L->cache_layer, order + first, cnt, stream);
+    if (s != DX_OK) return s;
+    s = do_experts(L, h, K, y, false, residual != 0, st, 0, -1, first == 0, false, false, subset);
+    if (s != DX_OK) return s;
+    first += cnt;
+  } while (first < n);
+  return DX_OK;
+}
+
+extern "C" dx_status moe_draft_step_cached(dx_layer* L, const float* h, float* y, int32_t residual,
+                                           int32_t* topk_ids, float* topk_w, int32_t* host_topk_ids, void* stream) {
+  if (!L) return DX_ERR_INVALID_ARG;
+  if (!L->cache) return DX_ERR_INVALID_ARG;
+  dx_ctx* ctx = L->ctx;
+  cudaStream_t st = (cudaStream_t)stream;
+  const int k = L->desc.top_k;
+  int32_t* ids = topk_ids ? topk_ids : ctx->union_dev + DX_MAX_E + 1;
+  RouteOut o{ids, topk_w, nullptr, nullptr, nullptr, nullptr, nullptr};
+  dx_status s = do_route(L, h, 1, y, o, true, residual != 0, st);
+  if (s != DX_OK) return s;
+  int32_t* host = ctx->union_host + DX_MAX_E + 1;
+  s = read_back(ctx, ids, k, host, st);
+  if (s != DX_OK) return s;
+  if (host_topk_ids)
+    for (int j = 0; j < k; ++j) host_topk_ids[j] = host[j];
+  const int32_t e1 = host[0];
+  s = expert_cache_stage(L->cache, L->cache_layer, &e1, 1, stream);   // hit, in flight (waited for) or on demand
+  if (s != DX_OK) return s;
+  return do_experts(L, h, 1, y, true, residual != 0, st);
+}
+
+// ---- exercising the bounded waits without a fault -------------------------------------------------------------
+extern "C" dx_status dx_selftest_wait_expiry(dx_layer* L, const float* h, int32_t K, float* y, void* stream) {
+  if (!L) return DX_ERR_INVALID_ARG;
+  dx_ctx* ctx = L->ctx;
+  if (L->desc.weight_dtype == DX_DTYPE_FP32) return DX_ERR_UNSUPPORTED;   // the fp32 kernels have no hand-over
+  if (ctx->wait_limit > (1u << 16)) return DX_ERR_INVALID_ARG;            // keep the give-up short: set a limit first
+  cudaStream_t st = (cudaStream_t)stream;
+  // hand-over words as a routing kernel leaves them before it publishes anything, and then no routing kernel
+  DX_CUDA(ctx, cudaMemsetAsync(ctx->handover, 0, 4 * sizeof(unsigned int), st));
+  DX_CUDA(ctx, cudaMemsetAsync(ctx->work, 0, sizeof(DxWork), st));
+  return do_experts(L, h, K, y, false, false, st, 0, -1, true, true);
 }
 
 // ---- draft stack: Eq. 5 through a whole stack of layers in one persistent kernel -----------------------------
@@ -524,6 +636,7 @@ extern "C" dx_status moe_draft_stack(dx_stack* s, const float* h_in, float* h_ou
   p.draft_tiles = d.draft_inter / DX_TILE_I;
   p.routed_tiles = d.inter / DX_TILE_I;
   p.q4 = d.weight_dtype == DX_DTYPE_Q4 ? 1 : 0;
+  p.wait_limit = ctx->wait_limit;
   DX_CUDA(ctx, dx_launch_draft_stack(ctx, p, st));
   ctx->launches++;
   return DX_OK;

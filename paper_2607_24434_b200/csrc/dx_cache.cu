@@ -17,6 +17,7 @@
 // With ctx == NULL the cache is bookkeeping only: the same policy without device memory or copies.
 #include <chrono>
 #include <new>
+#include <thread>
 #include <vector>
 
 #include "dx_internal.cuh"
@@ -59,9 +60,11 @@ struct dx_cache {
 
 namespace {
 
-__global__ void dx_table_patch_kernel(const void** table, DxTablePatch patch) {
+__global__ void dx_table_patch_kernel(const void** table, int table_len, int32_t* dev_status, DxTablePatch patch) {
   dx_pdl_wait();
-  if ((int)threadIdx.x < patch.n) table[patch.idx[threadIdx.x]] = patch.ptr[threadIdx.x];
+  if ((int)threadIdx.x < patch.n &&
+      DX_BOUNDS(patch.idx[threadIdx.x] >= 0 && patch.idx[threadIdx.x] < table_len, dev_status))
+    table[patch.idx[threadIdx.x]] = patch.ptr[threadIdx.x];
 }
 
 inline DxSlot& slot_ref(dx_cache* c, int layer, int s) { return c->slots[(size_t)layer * c->S + s]; }
@@ -169,7 +172,7 @@ dx_status flush_patches(dx_cache* c, int layer, cudaStream_t st) {
       ++patch.n;
       ++i;
     }
-    dx_table_patch_kernel<<<1, 32, 0, st>>>(L->table_dev, patch);
+    dx_table_patch_kernel<<<1, 32, 0, st>>>(L->table_dev, L->table_len, c->ctx->dev_status, patch);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { c->ctx->last_cuda = e; return DX_ERR_CUDA; }
     c->ctx->launches++;
@@ -187,6 +190,20 @@ dx_status check_ids(dx_cache* c, int layer, const int32_t* ids, int n) {
 }
 
 }  // namespace
+
+// A layer that is destroyed before its cache: drop the back pointer and the table patches queued for it.
+void dx_cache_forget_layer(dx_cache* c, dx_layer* L) {
+  if (!c || !L) return;
+  for (int l = 0; l < c->L; ++l)
+    if (c->layer[l] == L) { c->layer[l] = nullptr; c->pending[l].clear(); }
+}
+
+// Slot of `expert` in `layer` (-1: neither cached nor in flight); no statistics are touched.
+int dx_cache_slot_of(const dx_cache* c, int layer, int expert) {
+  if (!c || layer < 0 || layer >= c->L || expert < 0 || expert >= c->E) return -1;
+  return c->slot_of[(size_t)layer * c->E + expert];
+}
+int dx_cache_slots(const dx_cache* c) { return c ? c->S : 0; }
 
 void dx_cache_note_use(dx_cache* c, int layer, cudaStream_t st) {
   if (!c || !c->ctx || layer < 0 || layer >= c->L) return;
@@ -371,12 +388,16 @@ static dx_status resolve(dx_cache* c, int layer, const int32_t* ids, int n, cuda
     if (!pinned[s]) continue;
     DxSlot& sl = slot_ref(c, layer, s);
     if (copy_done(c, sl)) continue;
+    c->stats.waited_copies++;
     if (timeout_s > 0.0) {
-      // bounded host wait (expert_cache_wait): poll the copy's event up to the deadline
-      while (!copy_done(c, sl)) {
-        const double dt = std::chrono::duration<double>(std::chrono::steady_clock::now() - t0).count();
-        if (dt > timeout_s) return DX_ERR_TIMEOUT;
-      }
+      // bounded host wait (expert_cache_wait): poll the copy's event up to the deadline (counted from the call's start)
+      const auto ts = std::chrono::steady_clock::now();
+      bool late = false;
+      while (!late && !copy_done(c, sl))
+        late = std::chrono::duration<double>(std::chrono::steady_clock::now() - t0).count() > timeout_s;
+      c->stats.stall_ns += (int64_t)std::chrono::duration_cast<std::chrono::nanoseconds>(
+                               std::chrono::steady_clock::now() - ts).count();
+      if (late) return DX_ERR_TIMEOUT;
     } else {
       cudaError_t e = cudaStreamWaitEvent(stream, sl.ev, 0);
       if (e != cudaSuccess) { c->ctx->last_cuda = e; return DX_ERR_CUDA; }
@@ -392,6 +413,20 @@ extern "C" dx_status expert_cache_stage(dx_cache* c, int32_t layer, const int32_
 extern "C" dx_status expert_cache_wait(dx_cache* c, int32_t layer, const int32_t* ids, int32_t n, void* stream,
                                        double timeout_s) {
   return resolve(c, layer, ids, n, (cudaStream_t)stream, false, timeout_s);
+}
+
+namespace {
+void CUDART_CB sleep_on_host(void* ms) {
+  std::this_thread::sleep_for(std::chrono::milliseconds((long long)(intptr_t)ms));
+}
+}  // namespace
+
+extern "C" dx_status expert_cache_inject_transfer_delay(dx_cache* c, int32_t milliseconds) {
+  if (!c || milliseconds < 0 || milliseconds > 1000) return DX_ERR_INVALID_ARG;
+  if (!c->ctx) return DX_OK;
+  cudaError_t e = cudaLaunchHostFunc(c->copy_stream, sleep_on_host, (void*)(intptr_t)milliseconds);
+  if (e != cudaSuccess) { c->ctx->last_cuda = e; return DX_ERR_CUDA; }
+  return DX_OK;
 }
 
 extern "C" dx_status expert_cache_stats(dx_cache* c, dx_cache_stats* out) {

@@ -51,8 +51,8 @@ __device__ __forceinline__ float stack_warp_sum(float v) {
   return v;
 }
 // Bounded wait until a counter in global memory has reached `want`.
-__device__ __forceinline__ bool counter_wait(const unsigned int* word, unsigned int want) {
-  for (uint32_t it = 0; it < (1u << 22); ++it) {
+__device__ __forceinline__ bool counter_wait(const unsigned int* word, unsigned int want, uint32_t limit) {
+  for (uint32_t it = 0; it < limit; ++it) {
     unsigned int v;
     asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(word) : "memory");
     if (v >= want) return true;
@@ -141,7 +141,8 @@ __global__ void __launch_bounds__(kStackThreads, 1) dx_draft_stack_kernel(DxStac
       return blob ? blob + (size_t)(u - first) * UNIT_BYTES : nullptr;
     };
     auto push_chunk = [&](const unsigned char* src) {
-      mbar_wait(smem_u32(&hdr->empty[slot]), phase ^ 1u, abort_flag);
+      // nothing more is copied once anything has given up (see mbar_wait)
+      if (!mbar_wait(smem_u32(&hdr->empty[slot]), phase ^ 1u, abort_flag, p.wait_limit)) return;
       const uint32_t fb = smem_u32(&hdr->full[slot]);
       mbar_arrive_expect_tx(fb, CHUNK);
       bulk_g2s(smem_u32(ring + (size_t)slot * CHUNK), src, CHUNK, fb, l2pol);
@@ -177,7 +178,7 @@ __global__ void __launch_bounds__(kStackThreads, 1) dx_draft_stack_kernel(DxStac
       const uint32_t n_back = it < (uint32_t)n_slots ? it : (uint32_t)n_slots;
       for (uint32_t k = 1; k <= n_back; ++k) {
         const uint32_t j = it - k, s = j % (uint32_t)n_slots, ph = (j / (uint32_t)n_slots) & 1u;
-        for (uint32_t spin = 0; spin < DX_WAIT_LIMIT; ++spin)
+        for (uint32_t spin = 0; spin < DX_WAIT_LIMIT_DEFAULT; ++spin)
           if (mbar_try_wait(smem_u32(&hdr->full[s]), ph)) break;
       }
       atomicExch(p.dev_status, DX_DEV_WAIT_EXPIRED);
@@ -198,7 +199,7 @@ __global__ void __launch_bounds__(kStackThreads, 1) dx_draft_stack_kernel(DxStac
         for (int i = 0; i < WV; ++i) wreg[i] = wrow[lane + 32 * i];
       }
       bool ok = true;
-      if (l > 0 && lane == 0) ok = counter_wait(p.sync + (l - 1), (unsigned int)G);   // layer l-1 is complete
+      if (l > 0 && lane == 0) ok = counter_wait(p.sync + (l - 1), (unsigned int)G, p.wait_limit);   // layer l-1 is complete
       __syncwarp();   // orders the other lanes' reads of the delta row behind lane 0's acquire (a shuffle would not)
       ok = __shfl_sync(0xffffffffu, ok, 0);
       // advance the hidden row by the finished layer's delta; its mean square on the way
@@ -267,7 +268,7 @@ __global__ void __launch_bounds__(kStackThreads, 1) dx_draft_stack_kernel(DxStac
 #pragma unroll
         for (int j = 0; j < 8; ++j) zw[j] = 0ull;
         bool all = false;
-        for (uint32_t spin = 0; spin < (1u << 22) && !all; ++spin) {
+        for (uint32_t spin = 0; spin < p.wait_limit && !all; ++spin) {
           bool mine = true;
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
@@ -379,7 +380,7 @@ __global__ void __launch_bounds__(kStackThreads, 1) dx_draft_stack_kernel(DxStac
       cslot += kStackConsumers;   // (a ring has more slots than a unit has chunks: at most one wrap)
       if (cslot >= (uint32_t)n_slots) { cslot -= (uint32_t)n_slots; cphase ^= 1u; }
       const uint4* A = reinterpret_cast<const uint4*>(ring + (size_t)s * CHUNK) + lane;
-      mbar_wait(smem_u32(&hdr->full[s]), ph, abort_flag);
+      mbar_wait(smem_u32(&hdr->full[s]), ph, abort_flag, p.wait_limit);
       // gate (rows 0..7 of the tile) and up (rows 8..15) over this warp's slice of the hidden dimension
       float ga = 0.f, gb = 0.f, ua = 0.f, ub = 0.f;
       if constexpr (Q4) {
@@ -464,7 +465,7 @@ __global__ void __launch_bounds__(kStackThreads, 1) dx_draft_stack_kernel(DxStac
         }
       }
       __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&hdr->empty[s]));
+      if (lane == 0 && !*abort_flag) mbar_arrive(smem_u32(&hdr->empty[s]));   // (no slot is released after a give-up)
     };
 
     const float gamma = p.layers[l].gamma;

@@ -171,7 +171,7 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
     const bool is_draft = i >= p.n_shared;
     hdr->e_begin[i] = is_draft ? p.n_shared * p.shared_tiles : i * p.shared_tiles;
     hdr->e_tiles[i] = is_draft ? p.draft_tiles : p.shared_tiles;
-    hdr->e_blob[i] = reinterpret_cast<const unsigned char*>(p.table[i]);
+    hdr->e_blob[i] = DX_BOUNDS(i < p.table_len, p.dev_status) ? reinterpret_cast<const unsigned char*>(p.table[i]) : nullptr;
   }
   __syncthreads();
 
@@ -189,7 +189,9 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
           const unsigned char* src = blob + (size_t)(u - b) * UNIT_BYTES;
 #pragma unroll 1
           for (int w = 0; w < kConsumerWarps; ++w, ++it) {
-            mbar_wait(smem_u32(&hdr->empty[slot]), phase ^ 1u, abort_flag);
+            // once anything has given up nothing more is copied (see mbar_wait)
+            if (!mbar_wait(smem_u32(&hdr->empty[slot]), phase ^ 1u, abort_flag, p.wait_limit)) return;
+            if (!DX_BOUNDS(slot < (uint32_t)n_slots && u - b >= 0 && u - b < nt, p.dev_status)) { *abort_flag = 1; return; }
             const uint32_t fb = smem_u32(&hdr->full[slot]);
             mbar_arrive_expect_tx(fb, CHUNK);
             bulk_g2s(smem_u32(ring + (size_t)slot * CHUNK), src + (size_t)w * CHUNK, CHUNK, fb, l2pol);
@@ -212,7 +214,7 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
     for (int i = 0; i < PER_LANE; ++i) gw[i] = 0ull;
     int n_groups = 0, kk = 1, n_pairs = 0;
     bool have_list = false;
-    for (uint32_t look = 0; look < (1u << 22) && !have_list; ++look) {
+    for (uint32_t look = 0; look < p.wait_limit && !have_list; ++look) {
       const unsigned long long head = dx_word_load(&W->head);
       gw[0] = dx_word_load(&W->group[lane]);
       bool mine = false;
@@ -229,32 +231,49 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
     for (int i = 1; i < PER_LANE; ++i) {
       const int idx = lane + 32 * i;
       bool mine = !have_list || idx >= n_groups;
-      for (uint32_t look = 0; look < (1u << 22); ++look) {
+      for (uint32_t look = 0; look < p.wait_limit; ++look) {
         if (!mine) {
           gw[i] = dx_word_load(&W->group[idx]);
           mine = (gw[i] & DX_WORD_VALID) != 0;
         }
         if (__all_sync(0xffffffffu, mine)) break;
-        if (look + 1 == (1u << 22)) have_list = false;
+        if (look + 1 == p.wait_limit) have_list = false;
       }
     }
     if (!have_list) {
       n_groups = 0;
       if (lane == 0) { *abort_flag = 1; atomicExch(p.dev_status, DX_DEV_WAIT_EXPIRED); }
     }
+    // groups left out by the subset mask drop out of the list here: the rest keeps its order and closes up
+    int pos[PER_LANE];
+    {
+      int n_sel = 0;
+#pragma unroll
+      for (int i = 0; i < PER_LANE; ++i) {
+        const int idx = lane + 32 * i, gid = dx_group_id(gw[i]);
+        const bool in = idx < n_groups &&
+                        (!p.use_subset || (gid < DX_MAX_E && ((p.subset[gid >> 6] >> (gid & 63)) & 1ull)));
+        const unsigned int b = __ballot_sync(0xffffffffu, in);
+        pos[i] = in ? n_sel + __popc(b & ((1u << lane) - 1u)) : -1;
+        n_sel += __popc(b);
+      }
+      n_groups = n_sel;
+    }
     int e_lo, e_hi, u_lo, u_hi;
     routed_range(n_groups, p, n_static, NS, s_lo - S0, s_hi - S0, G, cta, e_lo, e_hi, u_lo, u_hi);
     const int unit_base = p.n_shared * p.shared_tiles + p.draft_tiles;
 #pragma unroll
     for (int i = 0; i < PER_LANE; ++i) {
-      const int idx = lane + 32 * i;
-      if (idx < n_groups) {
+      const int idx = pos[i];
+      if (idx >= 0) {
         const int gid = dx_group_id(gw[i]);
         const unsigned char* blob = reinterpret_cast<const unsigned char*>(dx_group_blob(gw[i]));
         // without the hand-over the table may have changed since the routing kernel ran (experts staged by the
         // cache in between): read it now
-        if (!p.handover && gid < DX_MAX_E) blob = reinterpret_cast<const unsigned char*>(p.table[p.n_shared + 1 + gid]);
+        if (!p.handover && gid < DX_MAX_E && DX_BOUNDS(p.n_shared + 1 + gid < p.table_len, p.dev_status))
+          blob = reinterpret_cast<const unsigned char*>(p.table[p.n_shared + 1 + gid]);
         const int e = n_static + idx;
+        if (!DX_BOUNDS(e < DX_MAX_ENTRIES, p.dev_status)) continue;
         hdr->e_begin[e] = unit_base + idx * p.routed_tiles;
         hdr->e_tiles[e] = p.routed_tiles;
         hdr->e_gid[e] = gid;
@@ -274,11 +293,12 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
       issue(e_lo, e_hi, u_lo, u_hi);
       if (*abort_flag) {
         // something gave up: make sure no copy is still landing in this CTA's
-        // shared memory before it is released (bounded, ignores the flag)
+        // shared memory before it is released (bounded, ignores the flag; the copies themselves take
+        // microseconds, so this uses the library's default limit whatever the context's limit is)
         const uint32_t n_back = it < (uint32_t)n_slots ? it : (uint32_t)n_slots;
         for (uint32_t k = 1; k <= n_back; ++k) {
           const uint32_t j = it - k, s = j % (uint32_t)n_slots, ph = (j / (uint32_t)n_slots) & 1u;
-          for (uint32_t spin = 0; spin < DX_WAIT_LIMIT; ++spin)
+          for (uint32_t spin = 0; spin < DX_WAIT_LIMIT_DEFAULT; ++spin)
             if (mbar_try_wait(smem_u32(&hdr->full[s]), ph)) break;
         }
         atomicExch(p.dev_status, DX_DEV_WAIT_EXPIRED);
@@ -303,7 +323,7 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
   // the producers are already streaming weights; the block itself may still be written by the kernel in front
   // of the routing kernel, which publishes its call number once that kernel has completed
   if (p.handover) {
-    if (threadIdx.x == 0 && !flag_wait(p.handover)) { *abort_flag = 1; atomicExch(p.dev_status, DX_DEV_WAIT_EXPIRED); }
+    if (threadIdx.x == 0 && !flag_wait(p.handover, p.wait_limit)) { *abort_flag = 1; atomicExch(p.dev_status, DX_DEV_WAIT_EXPIRED); }
     consumer_bar();   // one poller per CTA; the others pick the acquire up through the barrier
   } else {
     pdl_wait();
@@ -414,11 +434,14 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
       const bool need_hi = NT > 1 && __any_sync(0xffffffffu, wrow[NT - 1] != 0.0f);   // any of rows 8..15 routed here
 
       for (int u = lo; u < hi; ++u) {
-        const uint32_t s = cslot, ph = cphase;
+        uint32_t s = cslot;
+        const uint32_t ph = cphase;
         cslot += kConsumerWarps;   // (a ring has more slots than a unit has chunks: at most one wrap)
         if (cslot >= (uint32_t)n_slots) { cslot -= (uint32_t)n_slots; cphase ^= 1u; }
+        // (a slot out of range is reported and replaced: every warp has to keep taking part in the barriers below)
+        if (!DX_BOUNDS(s < (uint32_t)n_slots, p.dev_status)) { *abort_flag = 1; s = 0; }
         const uint4* A = reinterpret_cast<const uint4*>(ring + (size_t)s * CHUNK) + lane;
-        mbar_wait(smem_u32(&hdr->full[s]), ph, abort_flag);
+        mbar_wait(smem_u32(&hdr->full[s]), ph, abort_flag, p.wait_limit);
 
         // ---- phase 1: [8 gate rows ; 8 up rows] x tokens over this warp's slice of the contraction
         float ch[NT][2][4], cl[NT][2][4];
@@ -562,7 +585,7 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
         }
         }
         __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&hdr->empty[s]));
+        if (lane == 0 && !*abort_flag) mbar_arrive(smem_u32(&hdr->empty[s]));   // (no slot is released after a give-up)
       }
 
     }
@@ -578,11 +601,12 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
     for (int idx = lane; idx < n_pairs; idx += 32) {
       unsigned long long w = 0ull;
       uint32_t look = 0;
-      for (; look < (1u << 22); ++look) {
+      for (; look < p.wait_limit; ++look) {
         w = dx_word_load(&W->pair[idx]);
         if (w & DX_WORD_VALID) break;
       }
-      ok = ok && look < (1u << 22);
+      ok = ok && look < p.wait_limit;
+      if (!DX_BOUNDS(idx < DX_MAX_PAIRS, p.dev_status)) continue;
       hdr->pair_id[idx] = dx_pair_id(w);
       hdr->pair_w[idx] = dx_pair_weight(w);
     }
@@ -631,7 +655,7 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
           if (hi) { v0 = r0; v1 = r1; } else { v2 = r0; v3 = r1; }
         }
         // (v0, v1, v2, v3) = this lane's combination at rows 4q, 4q+1, 4q+2, 4q+3 of the tile's half
-        if (row < p.K) {
+        if (row < p.K && DX_BOUNDS((g >> 2) * 4 + half * 8 + (warp * 2 * PW + j) * 16 + 3 < H, p.dev_status)) {
           float* dst = yrow + (warp * 2 * PW + j) * 16;
           asm volatile("red.relaxed.gpu.global.add.v4.f32 [%0], {%1, %2, %3, %4};"
                        :: "l"(dst), "f"(v0), "f"(v1), "f"(v2), "f"(v3) : "memory");
@@ -690,6 +714,7 @@ __global__ void __launch_bounds__(256) dx_experts_fp32_kernel(DxExpertParams p) 
     } else {
       const int gi = (u - NS_all) / p.routed_tiles;
       gid = dx_group_id(W->group[gi]);
+      if (p.use_subset && !(gid < DX_MAX_E && ((p.subset[gid >> 6] >> (gid & 63)) & 1ull))) continue;
       table_index = p.n_shared + 1 + gid;
       unit_begin = NS_all + gi * p.routed_tiles;
     }
@@ -705,7 +730,8 @@ __global__ void __launch_bounds__(256) dx_experts_fp32_kernel(DxExpertParams p) 
       s_roww[row] = w;
     }
     __syncthreads();
-    const float* blob = reinterpret_cast<const float*>(p.table[table_index]);
+    const float* blob = DX_BOUNDS(table_index >= 0 && table_index < p.table_len, p.dev_status)
+                            ? reinterpret_cast<const float*>(p.table[table_index]) : nullptr;
     if (blob == nullptr) {
       if (threadIdx.x == 0) atomicExch(p.dev_status, DX_DEV_BAD_EXPERT_ID);
       __syncthreads();
@@ -854,7 +880,7 @@ cudaError_t launch_bf16(dx_ctx* ctx, const DxExpertParams& p, cudaStream_t st) {
   // fills an SM, so a CTA that had to wait for a routing CTA's SM would start late and become the tail.
   int grid = ctx->sm_count > 16 ? ctx->sm_count - DX_ROUTE_CLUSTER : ctx->sm_count;
   if (TILES == 2) grid &= ~1;
-  return dx_launch_pdl(DX_PDL_EXPERTS, dx_experts_bf16_kernel<H, NT, TILES, Q4, SPLIT>, dim3(grid), dim3(kThreads), smem, st, 1,
+  return dx_launch_pdl((ctx->pdl_mask & DX_PDL_EXPERTS) != 0, dx_experts_bf16_kernel<H, NT, TILES, Q4, SPLIT>, dim3(grid), dim3(kThreads), smem, st, 1,
                        p, n_slots);
 }
 
@@ -967,7 +993,7 @@ bool dx_bf16_hidden_supported(int H) { return H == 256 || H == 512 || H == 1024 
 
 cudaError_t dx_launch_experts(dx_ctx* ctx, const DxExpertParams& p, int weight_dtype, int K, cudaStream_t st) {
   if (weight_dtype == DX_DTYPE_FP32) {
-    return dx_launch_pdl(DX_PDL_EXPERTS, dx_experts_fp32_kernel, dim3(ctx->sm_count * 4), dim3(256), 0, st, 1, p);
+    return dx_launch_pdl((ctx->pdl_mask & DX_PDL_EXPERTS) != 0, dx_experts_fp32_kernel, dim3(ctx->sm_count * 4), dim3(256), 0, st, 1, p);
   }
   if (weight_dtype == DX_DTYPE_Q4) return launch_bf16_any<true, false>(ctx, p, K, st);
   return ctx->act_split ? launch_bf16_any<false, true>(ctx, p, K, st) : launch_bf16_any<false, false>(ctx, p, K, st);

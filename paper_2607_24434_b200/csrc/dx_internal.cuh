@@ -67,6 +67,8 @@ struct dx_ctx {
   int sm_count;
   int smem_optin;
   int act_split;              // 1: bf16 experts are evaluated with hi + residual activation fragments
+  int pdl_mask;               // DX_PDL_* bits: kernels launched with programmatic stream serialization
+  uint32_t wait_limit;        // polls after which a bounded wait inside a kernel gives up (dx_set_wait_limit)
   cudaError_t last_cuda;
   int64_t launches;
   // device scratch
@@ -77,6 +79,8 @@ struct dx_ctx {
   unsigned int* handover;      // device word {block input final}: see DxExpertParams
   float2* conf_part;           // [8 * sm_count][DX_MAX_M] per-CTA online-softmax pairs of the confidence variant
   int32_t* scratch_i32;        // two ints the draft-token entry point parks unused outputs in
+  int32_t* union_dev;          // [DX_MAX_E] union ids, [1] union count, [DX_MAX_TOPK] draft selection: what the
+  int32_t* union_host;         //   cached entry points read back (pinned host copy, same layout)
 };
 
 struct dx_cache;
@@ -128,6 +132,7 @@ struct DxExpertParams {
   const float* x;            // [K,H] block input (never written while the kernel runs)
   float* y;                  // [K,H] accumulated into; initialised by the routing kernel
   const void* const* table;  // layer blob table (device)
+  int table_len;             // entries of the table (bounds of the checked build)
   const DxWork* work;
   int32_t* dev_status;
   int H, K;
@@ -139,6 +144,10 @@ struct DxExpertParams {
   // the routing-independent groups are part of it; a cache-staged union is processed in several windows
   int first_routed, n_routed, do_static;
   int skip_shared;           // 1: of the routing-independent groups only the draft expert is evaluated
+  // of the routed groups (inside the window above) only those whose expert id has its bit set are evaluated: a wave
+  // of a cache-staged union need not be a contiguous run of the ascending id list
+  int use_subset;
+  unsigned long long subset[DX_MAX_E / 64];
   int row_tiles;             // set by the launcher: 2 = CTA pairs, one tile of eight block rows each (K > 8)
   // Hand-over from the routing kernel launched right before this one (fused entry points only; null otherwise,
   // and then the kernel simply waits for everything in front of it).  With the hand-over this kernel may be running
@@ -146,6 +155,7 @@ struct DxExpertParams {
   // polled out of the work list.  The routing kernel of the next pair clears the word and the list before it lets
   // its own expert kernel start; this kernel in turn lets that routing kernel start only when it is past both.
   unsigned int* handover;
+  uint32_t wait_limit;       // polls after which a bounded wait gives up (sets DX_DEV_WAIT_EXPIRED)
 };
 
 // Persistent draft stack (dx_draft_stack.cu): one descriptor per layer in device memory ...
@@ -173,6 +183,7 @@ struct DxStackParams {
   float scale;
   int n_shared, shared_tiles, draft_tiles, routed_tiles;
   int q4;                     // 1: the units are 4-bit codes with block scales
+  uint32_t wait_limit;        // polls after which a bounded wait gives up
 };
 struct dx_stack {
   dx_ctx* ctx;
@@ -186,7 +197,7 @@ struct dx_stack {
 cudaError_t dx_launch_draft_stack(dx_ctx* ctx, const DxStackParams& p, cudaStream_t st);
 
 // launchers (each returns the cudaError_t of the launch)
-cudaError_t dx_launch_route(const DxRouteParams& p, int weight_dtype, cudaStream_t st);
+cudaError_t dx_launch_route(dx_ctx* ctx, const DxRouteParams& p, int weight_dtype, cudaStream_t st);
 cudaError_t dx_launch_experts(dx_ctx* ctx, const DxExpertParams& p, int weight_dtype, int K, cudaStream_t st);
 cudaError_t dx_launch_pack(int weight_dtype, int H, int I, const void* Wg, const void* Wu, const void* Wd,
                            void* blob, cudaStream_t st);
@@ -212,14 +223,14 @@ void dx_cache_note_use(dx_cache* c, int layer, cudaStream_t st);
 __device__ __forceinline__ void dx_pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void dx_pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
-// Which kernels are launched with programmatic stream serialization: bit 0 routing, bit 1 experts, bit 2 accept.
-// Default from the library; DX_PDL_MASK in the environment overrides it (0 = plain stream order everywhere).
-int dx_pdl_mask();
+// Which kernels are launched with programmatic stream serialization (dx_ctx::pdl_mask, dx_set_launch_overlap):
+// bit 0 routing, bit 1 experts, bit 2 greedy accept.
 enum { DX_PDL_ROUTE = 1, DX_PDL_EXPERTS = 2, DX_PDL_ACCEPT = 4 };
+#define DX_WAIT_LIMIT_DEFAULT (1u << 22)
 
 // Launch with programmatic stream serialization so that the kernel may begin while its predecessor drains.
 template <typename... KArgs, typename... Args>
-inline cudaError_t dx_launch_pdl(int which, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+inline cudaError_t dx_launch_pdl(bool pdl, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
                                  cudaStream_t st, int cluster, Args... args) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid;
@@ -235,7 +246,7 @@ inline cudaError_t dx_launch_pdl(int which, void (*kernel)(KArgs...), dim3 grid,
     attr[n].val.clusterDim.z = 1;
     ++n;
   }
-  if (dx_pdl_mask() & which) {
+  if (pdl) {
     attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[n].val.programmaticStreamSerializationAllowed = 1;
     ++n;
@@ -244,6 +255,15 @@ inline cudaError_t dx_launch_pdl(int which, void (*kernel)(KArgs...), dim3 grid,
   cfg.numAttrs = n;
   return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
+
+// Bounds checks of the checked build (-DDX_CHECKED, the stand-in for a memory checker): `if (DX_BOUNDS(i < n, status))`
+// guards an indexed access; a violated bound records DX_DEV_BOUNDS in the status word and skips the access.  In the
+// normal build the condition is not evaluated.
+#ifdef DX_CHECKED
+#define DX_BOUNDS(cond, status) ((cond) ? true : (atomicExch((status), (int32_t)DX_DEV_BOUNDS), false))
+#else
+#define DX_BOUNDS(cond, status) (true)
+#endif
 
 __device__ __forceinline__ float dx_silu(float x) { return x / (1.0f + expf(-x)); }
 

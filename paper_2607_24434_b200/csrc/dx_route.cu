@@ -155,6 +155,7 @@ __device__ __forceinline__ void topk_select(const DxRouteParams& p, const float*
   }
   if (lane < k) {
     my_e = min(max(my_e, 0), E - 1);   // whatever the logits were, stay in range
+    if (!DX_BOUNDS(tt * k + lane < DX_MAX_PAIRS && tt * DX_MAX_TOPK + lane < DX_MAX_K * DX_MAX_TOPK, p.dev_status)) return;
     s_sel_z[tt * DX_MAX_TOPK + lane] = my_z;
     s_ids[tt * k + lane] = my_e;
     if (!(p.skip_top1 && lane == 0))
@@ -298,7 +299,8 @@ __global__ void __launch_bounds__(kRouteThreads) dx_route_kernel(DxRouteParams p
   }
   if (crank == 0) {
     // routed part of the blob table, for the group list at the end; empty union mask
-    if (threadIdx.x < E) s_tab[threadIdx.x] = p.table[p.n_shared + 1 + threadIdx.x];
+    if (threadIdx.x < E && DX_BOUNDS(E <= DX_MAX_E && E <= kRouteThreads, p.dev_status))
+      s_tab[threadIdx.x] = p.table[p.n_shared + 1 + threadIdx.x];
     if (threadIdx.x < DX_MAX_E / 32) s_mask[threadIdx.x] = 0u;
   }
 
@@ -522,8 +524,9 @@ __global__ void __launch_bounds__(kRouteThreads) dx_route_kernel(DxRouteParams p
     upos += __popc(mine & ((1u << (me & 31)) - 1u));
   }
   if (!p.draft_mode) {
-    if (flag) dx_word_store(&W->group[upos], dx_group_word(me, s_tab[me]));
-  } else if (me < p.top_r) {
+    if (flag && DX_BOUNDS(upos < DX_MAX_PAIRS && upos < K * k, p.dev_status))
+      dx_word_store(&W->group[upos], dx_group_word(me, s_tab[me]));
+  } else if (me < p.top_r && DX_BOUNDS(me < DX_MAX_PAIRS && s_ids[me] >= 0 && s_ids[me] < E, p.dev_status)) {
     dx_word_store(&W->group[me], dx_group_word(s_ids[me], s_tab[s_ids[me]]));
   }
   if (me == 0) dx_word_store(&W->head, dx_head_word(K, k, p.draft_mode ? p.top_r : ucount));
@@ -547,9 +550,9 @@ __global__ void __launch_bounds__(kRouteThreads) dx_route_kernel(DxRouteParams p
   if (me < E) {
     int i = 0;
     for (int q = 0; q < P; ++q)
-      if (s_ids[q] == me) s_perm[off + i++] = q;
+      if (s_ids[q] == me && DX_BOUNDS(off + i < P, p.dev_status)) s_perm[off + i++] = q;
     if (p.offsets) p.offsets[me] = off;
-    if (flag && p.union_ids) p.union_ids[upos] = me;
+    if (flag && p.union_ids && DX_BOUNDS(upos < min(E, P), p.dev_status)) p.union_ids[upos] = me;
   }
   if (me == 0) {
     if (p.offsets) p.offsets[E] = P;
@@ -567,7 +570,7 @@ __global__ void __launch_bounds__(kRouteThreads) dx_route_kernel(DxRouteParams p
 }  // namespace
 
 template <typename WT, int TG>
-static cudaError_t launch_route_one(const DxRouteParams& p, cudaStream_t st) {
+static cudaError_t launch_route_one(dx_ctx* ctx, const DxRouteParams& p, cudaStream_t st) {
   // CTA 0 holds one partial table per column slice (at most one per CTA of the cluster)
   size_t smem = (size_t)kRouteCluster * ((size_t)p.K * p.E + p.K) * sizeof(float);
   // (tensor-core path) one partial table per warp: [8][tiles of 16 router rows][8 or 16 token columns], sums of squares
@@ -584,18 +587,18 @@ static cudaError_t launch_route_one(const DxRouteParams& p, cudaStream_t st) {
     if (e != cudaSuccess) return e;
     opted_in = true;
   }
-  return dx_launch_pdl(DX_PDL_ROUTE, dx_route_kernel<WT, TG>, dim3(kRouteCluster), dim3(kRouteThreads), smem, st,
+  return dx_launch_pdl((ctx->pdl_mask & DX_PDL_ROUTE) != 0, dx_route_kernel<WT, TG>, dim3(kRouteCluster), dim3(kRouteThreads), smem, st,
                        kRouteCluster, p);
 }
 
 template <typename WT>
-static cudaError_t launch_route_tg(const DxRouteParams& p, cudaStream_t st) {
-  if (p.K <= 1) return launch_route_one<WT, 1>(p, st);
-  if (p.K <= 2) return launch_route_one<WT, 2>(p, st);
-  return launch_route_one<WT, 4>(p, st);
+static cudaError_t launch_route_tg(dx_ctx* ctx, const DxRouteParams& p, cudaStream_t st) {
+  if (p.K <= 1) return launch_route_one<WT, 1>(ctx, p, st);
+  if (p.K <= 2) return launch_route_one<WT, 2>(ctx, p, st);
+  return launch_route_one<WT, 4>(ctx, p, st);
 }
 
-cudaError_t dx_launch_route(const DxRouteParams& p, int weight_dtype, cudaStream_t st) {
-  if (weight_dtype == DX_DTYPE_BF16) return launch_route_tg<__nv_bfloat16>(p, st);
-  return launch_route_tg<float>(p, st);
+cudaError_t dx_launch_route(dx_ctx* ctx, const DxRouteParams& p, int weight_dtype, cudaStream_t st) {
+  if (weight_dtype == DX_DTYPE_BF16) return launch_route_tg<__nv_bfloat16>(ctx, p, st);
+  return launch_route_tg<float>(ctx, p, st);
 }

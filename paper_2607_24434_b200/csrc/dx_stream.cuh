@@ -32,8 +32,8 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 // Bounded wait for a word that another kernel sets (release/acquire at gpu scope).
-__device__ __forceinline__ bool flag_wait(const unsigned int* word) {
-  for (uint32_t it = 0; it < (1u << 22); ++it) {
+__device__ __forceinline__ bool flag_wait(const unsigned int* word, uint32_t limit) {
+  for (uint32_t it = 0; it < limit; ++it) {
     unsigned int v;
     asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(word) : "memory");
     if (v != 0u) return true;
@@ -41,16 +41,19 @@ __device__ __forceinline__ bool flag_wait(const unsigned int* word) {
   }
   return false;
 }
-// Bounded wait.  Returns false when it gave up; callers raise the abort flag,
-// after which every wait of the CTA falls through so the CTA still terminates.
-#define DX_WAIT_LIMIT (1u << 22)
-__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  if (mbar_try_wait(bar, parity)) return;   // the common case, kept out of the counted loop
-  for (uint32_t it = 0; it < DX_WAIT_LIMIT; ++it) {
-    if (mbar_try_wait(bar, parity)) return;
-    if ((it & 63u) == 63u && *abort_flag) return;
+// Bounded wait (`limit` polls, the context's wait limit).  Returns true once the barrier's phase has completed.
+// When it gives up it raises the abort flag and returns false; it also returns false, without waiting any longer,
+// once some other wait of the CTA has raised the flag, so that the CTA still terminates.  What the two sides of a
+// ring do with `false` keeps a slot from ever being armed again while its previous copy may still be landing: the
+// producer stops issuing, and a consumer that has seen the flag no longer releases slots.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t limit) {
+  if (mbar_try_wait(bar, parity)) return true;   // the common case, kept out of the counted loop
+  for (uint32_t it = 0; it < limit; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 63u) == 63u && *abort_flag) return false;
   }
   *abort_flag = 1;
+  return false;
 }
 // Expert weights are read exactly once per launch: mark them evict-first in L2 so that they do not push out
 // what is reused (block rows, router matrix, work list, output rows).

@@ -153,6 +153,11 @@ def lm_head(V: int, H: int, seed: int, dtype: torch.dtype, device="cpu", std: fl
     return normal((V, H), std, seed, "lm_head", dtype, device)
 
 
+def embedding_table(V: int, H: int, seed: int, device="cpu") -> torch.Tensor:
+    """Token embeddings for the closed-loop token chain of the offloaded-stack workload: bf16, N(0, 1) entries."""
+    return normal((V, H), 1.0, seed, "embedding", torch.bfloat16, device)
+
+
 def draft_tokens_from_target(target: np.ndarray, V: int, seed: int, p_accept: float = 0.85) -> np.ndarray:
     """Draft tokens that agree with ``target`` for a geometric(p) prefix.
 

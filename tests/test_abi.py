@@ -22,7 +22,8 @@ def test_header_symbols_exported_and_bound():
     names = _declared()
     assert len(names) >= 25
     for required in ("moe_draft_step", "moe_verify_block", "spec_accept", "expert_cache_prefetch",
-                     "expert_cache_stage", "dx_pack_expert"):
+                     "expert_cache_stage", "dx_pack_expert", "moe_verify_block_cached", "moe_draft_step_cached",
+                     "dx_set_wait_limit"):
         assert required in names
     for n in names:
         assert hasattr(lib, n), f"{n} declared in the header but not exported"
@@ -36,7 +37,7 @@ def test_header_symbols_exported_and_bound():
 def test_desc_struct_layout_matches_header():
     from paper_2607_24434_b200 import binding, synth
     assert ctypes.sizeof(binding.LayerDesc) == 12 * 4
-    assert ctypes.sizeof(binding.CacheStats) == 8 * 8
+    assert ctypes.sizeof(binding.CacheStats) == 10 * 8
     d = binding._desc(synth.shape_moonlight())
     assert (d.hidden, d.n_experts, d.top_k, d.inter, d.score_fn) == (2048, 64, 6, 1408, 1)
     assert abs(d.routed_scale - 2.446) < 1e-6
@@ -52,3 +53,6 @@ def test_argument_errors_without_a_device():
     assert lib.dx_destroy(None) == 1
     assert lib.moe_draft_step(None, None, None, None, None, None) == 1
     assert lib.spec_accept(None, None, 1, None, 1, 256, 1, None, 0, 0, None, None, None, None) == 1
+    assert lib.moe_verify_block_cached(None, None, 4, None, 0, None, None, None, None, None, None, None, None, None,
+                                       None) == 1
+    assert lib.dx_set_wait_limit(None, 100) == 1 and lib.dx_set_launch_overlap(None, 3) == 1

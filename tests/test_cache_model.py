@@ -120,3 +120,24 @@ def test_library_bookkeeping_cache_matches_model():
         fresh.prefetch(0, [99])
     assert err.value.status == 1
     cache.close(); fresh.close()
+
+
+def test_union_waves_keep_what_is_held():
+    """4 slots holding 1, 5, 9 (in that age order) and a block that needs 0..5: the held experts go first, so none of
+    them is evicted before it is used -- worked by hand: wave 1 = [1, 5, 0, 2] (two hits, two loads, the loads take
+    the free slot and then the oldest untouched one, 9), wave 2 = [3, 4] evicts the two oldest of wave 1."""
+    m = ExpertCacheModel(1, 16, 4)
+    for e in (1, 5, 9):
+        m.stage(0, [e])
+    base = dict(m.stats)
+    waves = m.stage_union(0, [0, 1, 2, 3, 4, 5])
+    assert waves == [[1, 5, 0, 2], [3, 4]]
+    assert m.stats["hits"] - base["hits"] == 2 and m.stats["on_demand"] - base["on_demand"] == 4
+    assert sorted(m.expert[0]) == [0, 2, 3, 4]             # 1 and 5 (oldest stamps of wave 1) made room for 3 and 4
+    # ascending waves would have been [0,1,2,3] then [4,5]: loading 0, 2, 3 evicts 5 before its wave -> one hit fewer
+    n = ExpertCacheModel(1, 16, 4)
+    for e in (1, 5, 9):
+        n.stage(0, [e])
+    b2 = dict(n.stats)
+    n.stage(0, [0, 1, 2, 3]); n.stage(0, [4, 5])
+    assert n.stats["hits"] - b2["hits"] == 1

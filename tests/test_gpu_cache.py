@@ -29,9 +29,11 @@ def _offloaded_layer(binding, ctx, seed, slots):
     return ref, resident, off, cache, host
 
 
-def test_cached_verify_matches_resident_and_checker():
+@pytest.mark.parametrize("act_split", [True, False])
+def test_cached_verify_matches_resident_and_checker(act_split):
     from paper_2607_24434_b200 import binding
-    ctx = binding.Context(0, act_split=True)
+    from tests.helpers import Y_BF16
+    ctx = binding.Context(0, act_split=act_split)
     ref, resident, off, cache, host = _offloaded_layer(binding, ctx, 70, slots=4)
     model = ExpertCacheModel(1, SHAPE.n_experts, 4)
     for step, K in enumerate([6, 6, 3, 8]):
@@ -53,10 +55,10 @@ def test_cached_verify_matches_resident_and_checker():
         # same arithmetic either way; only the order of the fp32 reductions into y differs between launches
         assert row_rel_err(out["y"].cpu().numpy(), want["y"].cpu().numpy()).max() <= 1e-5
         y_ref = O.moe_target(h.cpu().numpy().astype(np.float64), ref, forced_ids=ids)[0]
-        assert row_rel_err(out["y"].cpu().numpy(), y_ref).max() <= Y_TIGHT
+        assert row_rel_err(out["y"].cpu().numpy(), y_ref).max() <= (Y_TIGHT if act_split else Y_BF16)
         union = out["union_list"]
-        for first in range(0, len(union), 4):
-            model.stage(0, union[first:first + 4])
+        assert union == out["union_ids"].cpu().numpy()[:n].tolist()
+        model.stage_union(0, union)                          # held experts first, then the misses by ascending id
         for e in range(SHAPE.n_experts):                     # the library's slot table follows the host model
             assert cache.query(0, e)[0] == model.slot_of(0, e)
     st = cache.stats()
@@ -86,7 +88,63 @@ def test_cached_draft_step_and_errors():
     want = O.moe_draft(h.cpu().numpy().astype(np.float64), ref, forced_ids=out["topk_ids"].cpu().numpy()[None])[0]
     assert row_rel_err(y.cpu().numpy(), want).max() <= Y_TIGHT
     cache.wait(0, [e1], timeout_s=5.0)                       # resident now: returns at once
+    # the same step as one call of the library (route, read the selection on the host, stage e1, experts)
+    got = binding.moe_draft_step_cached(off, h)
+    torch.cuda.synchronize()
+    assert got["host_ids"] == out["topk_ids"].tolist()
+    assert row_rel_err(got["y"].cpu().numpy(), want).max() <= Y_TIGHT
+    # ... and in the pre-norm residual form the layer stacks use
+    got = binding.moe_draft_step_cached(off, h, residual=True)
+    res = binding.moe_draft_step_residual(resident, h)
+    torch.cuda.synchronize()
+    assert got["host_ids"] == res["topk_ids"].tolist()
+    assert row_rel_err(got["h"].cpu().numpy(), res["h"].cpu().numpy()).max() <= 1e-5
     # an expert that was never staged is reported through the status word, not by a fault
     other = (e1 + 1) % SHAPE.n_experts
     assert cache.query(0, other)[0] == -1
+    cache.close(); ctx.close()
+
+
+def test_slow_transfer_times_out_and_then_completes():
+    """A transfer that is slow (made on the host: a sleeping host callback queued on the copy stream in front of the
+    prefetch) makes the bounded wait of expert_cache_wait return DX_ERR_TIMEOUT; a later wait with time to spare
+    succeeds, and the results equal those of the resident layer."""
+    from paper_2607_24434_b200 import binding
+    ctx = binding.Context(0, act_split=True)
+    ref, resident, off, cache, host = _offloaded_layer(binding, ctx, 72, slots=4)
+    h = synth.hidden_block(1, SHAPE.hidden, 91, 0.0, "cuda")
+    want = binding.moe_draft_step(resident, h)
+    torch.cuda.synchronize()
+    ids = want["topk_ids"].tolist()
+    cache.begin_step()
+    cache.inject_transfer_delay(150)                         # the link stalls for 150 ms ...
+    cache.prefetch(0, ids[:1])                               # ... with the predicted expert's copy behind it
+    with pytest.raises(binding.DxError) as err:
+        cache.wait(0, ids[:1], timeout_s=0.005)
+    assert err.value.status == 6                             # DX_ERR_TIMEOUT
+    st = cache.stats()
+    assert st["waited_copies"] >= 1 and st["stall_ns"] >= 4_000_000
+    cache.wait(0, ids[:1], timeout_s=10.0)                   # the copy lands once the stall is over
+    y = torch.empty_like(h)
+    out = {"topk_ids": torch.empty((SHAPE.top_k,), dtype=torch.int32, device="cuda"),
+           "topk_w": torch.empty((SHAPE.top_k,), dtype=torch.float32, device="cuda")}
+    binding.moe_draft_route(off, h, y, out)
+    binding.moe_draft_experts(off, h, y)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == 0
+    assert out["topk_ids"].tolist() == ids
+    assert row_rel_err(y.cpu().numpy(), want["y"].cpu().numpy()).max() <= 1e-5
+    cache.close(); ctx.close()
+
+
+def test_layer_destroyed_before_its_cache():
+    """Either side may go first: a destroyed layer is forgotten by its cache (no patch is sent to a freed table)."""
+    from paper_2607_24434_b200 import binding
+    ctx = binding.Context(0)
+    ref, resident, off, cache, host = _offloaded_layer(binding, ctx, 73, slots=4)
+    cache.prefetch(0, [1, 2])
+    off.close()                                              # table patches for 1 and 2 were still pending
+    cache.stage(0, [3])
+    torch.cuda.synchronize()
+    assert cache.query(0, 3)[0] >= 0
     cache.close(); ctx.close()

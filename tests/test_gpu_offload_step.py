@@ -1,0 +1,142 @@
+"""One exact DraftExpert decode step (Algorithm 1) over an offloaded stack of full DeepSeek-V2-Lite-shaped layers
+with bf16 expert blobs in a pinned host pool, against the CPU checker:
+
+* every drafter layer (Eq. 5) and every verifier layer (Eq. 4 over the block's expert union) is compared with the
+  checker on that layer's own input rows with the library's routing replayed (teacher-forced per layer), and the
+  routing itself with the checker's wherever the logit gap exceeds 1e-3;
+* the stop rule (Sec. 3.4) with the checker's controller on the same predictions and confidences;
+* the expert cache's slot table and statistics (Sec. 3.5) with the host model replaying the same calls;
+* the target tokens and the accepted length with the checker's greedy verification on the final rows.
+
+Runs with plain bf16 activations (the library's default, what the benchmark times) and with the activation split."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import moe_oracle as O
+from oracle.cache_oracle import ExpertCacheModel
+from paper_2607_24434_b200 import synth
+from tests.helpers import GAP, Y_BF16, Y_TIGHT, check_routing, row_rel_err
+
+pytestmark = pytest.mark.gpu
+
+N_LAYERS, SLOTS, VOCAB, K_MAX = 3, 16, 4099, 6
+
+
+def _replay(model, calls):
+    for c in calls:
+        if c[0] == "begin_step":
+            model.begin_step()
+        elif c[0] == "stage":
+            model.stage(c[1], c[2])
+        elif c[0] == "prefetch":
+            model.prefetch(c[1], c[2])
+        elif c[0] == "stage_union":
+            model.stage_union(c[1], c[2])
+
+
+@pytest.mark.parametrize("act_split", [False, True])
+def test_offloaded_decode_step_full_shape(act_split):
+    from paper_2607_24434_b200 import binding, decode
+    shape = synth.shape_v2lite()
+    tol = Y_TIGHT if act_split else Y_BF16
+    ctx = binding.Context(0, act_split=act_split)
+    nbytes = binding.expert_blob_bytes(shape, shape.inter)
+    cache = binding.ExpertCache(ctx, N_LAYERS, shape.n_experts, SLOTS, nbytes)
+    layers, refs, pools = [], [], []
+    for l in range(N_LAYERS):
+        w = synth.make_layer(shape, 8100 + l, "cuda", zipf=True)
+        refs.append(synth.layer_to_numpy(w))
+        L = binding.Layer.from_weights(ctx, w, routed_resident=False)
+        torch.cuda.synchronize()
+        host = L.blobs.cpu().pin_memory()
+        L.blobs = None
+        del w
+        for e in range(shape.n_experts):
+            cache.register(l, e, host[e])
+        cache.attach(L, l)
+        layers.append(L); pools.append(host)
+    emb = synth.embedding_table(VOCAB, shape.hidden, 8198, "cuda")
+    W_lm = synth.lm_head(VOCAB, shape.hidden, 8199, torch.bfloat16, "cuda")
+    W_np = synth.to_numpy_f32(W_lm).astype(np.float64)
+    # a fixed budget below the second token's usual expansion would stop at once; the cache-derived one lets the
+    # block grow until the predictions no longer fit the 3 x 16 slots
+    dec = decode.OffloadedDecoder(ctx, layers, cache, emb, W_lm, k_max=K_MAX, tau=1.0, budget="cache")
+    model = ExpertCacheModel(N_LAYERS, shape.n_experts, SLOTS)
+    t0 = 7
+    for step in range(2):                                    # the second step starts from a warm cache
+        r = dec.step(t0, record=True)
+        torch.cuda.synchronize()
+        assert ctx.device_status() == 0
+        tr = r["trace"]
+        # ---- drafter: layer by layer on its own rows, routing replayed; the stop rule on the same numbers
+        ctl = O.TruncationController()
+        used = 0
+        for tok in tr["draft"]:
+            rows = tok["rows"] + [tok["final"]]
+            assert torch.equal(rows[0][0], emb[tok["prev"]].float())
+            for l in range(N_LAYERS):
+                pred = np.asarray(tok["pred"][l], np.int32)
+                h_np = rows[l].cpu().numpy().astype(np.float64)
+                want, ids_ref, _, z_ref = O.stack_layer_draft(h_np, refs[l])
+                check_routing(shape, z_ref, ids_ref, pred[None])
+                want = O.stack_layer_draft(h_np, refs[l], forced_ids=pred[None])[0]
+                assert row_rel_err(rows[l + 1].cpu().numpy(), want).max() <= tol, (step, l)
+            token_ref, q_ref = O.draft_confidence(O.rmsnorm(tok["final"].cpu().numpy().astype(np.float64)), W_np)
+            assert abs(tok["q"] - q_ref[0]) <= 1e-3 * q_ref[0] + 1e-7
+            budget = N_LAYERS * SLOTS - used
+            assert tok["budget"] == budget
+            stop, delta, new = ctl.propose(tok["pred"], tok["q"], 1.0, budget)
+            assert (stop, delta) == (tok["stop"], tok["delta"])
+            assert sorted(new) == sorted(tok["new"])
+            if not stop:
+                used += delta
+        kept = [t for t in tr["draft"] if not t["stop"]]
+        assert [t["token"] for t in kept] == r["drafted"] and 1 <= len(kept) <= K_MAX
+        assert len(tr["draft"]) == len(kept) + (1 if len(kept) < K_MAX else 0)      # the dropped candidate ended it
+        # ---- verifier: the rows are the embeddings of (t0, d_1 .. d_{K-1}); every layer against the checker
+        K = r["block_rows"]
+        assert K == len(kept)
+        inputs = [t0] + r["drafted"][:K - 1]
+        assert torch.equal(tr["verify"][0]["rows"], emb[torch.tensor(inputs, device="cuda")].float())
+        waves = 0
+        for l, v in enumerate(tr["verify"]):
+            ids = v["topk_ids"].cpu().numpy()
+            h_np = v["rows"].cpu().numpy().astype(np.float64)
+            want, ids_ref, _, z_ref = O.stack_layer_target(h_np, refs[l])
+            check_routing(shape, z_ref, ids_ref, ids)
+            want = O.stack_layer_target(h_np, refs[l], forced_ids=ids)[0]
+            assert row_rel_err(v["out"].cpu().numpy(), want).max() <= tol, (step, l)
+            assert v["union"] == O.block_union(ids, shape.n_experts)[1].tolist()
+            waves += -(-len(v["union"]) // SLOTS)
+            if l + 1 < N_LAYERS:
+                assert torch.equal(tr["verify"][l + 1]["rows"], v["out"])            # the residual stream is chained
+        # drafter and verifier see the same rows in the first layer only: later predictions can miss
+        if step == 0:
+            first_pred = set(tr["draft"][0]["pred"][0])
+            assert first_pred == set(tr["verify"][0]["topk_ids"][0].tolist())
+        # ---- greedy verification on the final rows
+        hn = O.rmsnorm(tr["verify"][-1]["out"].cpu().numpy().astype(np.float64))
+        t_ref, n_ref, next_ref, lg = O.greedy_accept_fast(hn, W_np, np.asarray(r["drafted"], np.int32))
+        srt = np.sort(lg, axis=1)
+        clear = (srt[:, -1] - srt[:, -2]) > GAP
+        assert np.array_equal(np.asarray(r["target"])[clear], t_ref[clear])
+        if clear.all():
+            assert r["n_accept"] == n_ref
+            assert r["emitted"] == r["drafted"][:n_ref] + ([int(t_ref[n_ref])] if n_ref < K else [])
+        # ---- the cache followed the host model call by call
+        _replay(model, tr["cache_calls"])
+        for l in range(N_LAYERS):
+            for e in range(shape.n_experts):
+                assert cache.query(l, e)[0] == model.slot_of(l, e), (step, l, e)
+        st = cache.stats()
+        for key in ("lookups", "hits", "on_demand", "prefetch_issued", "prefetch_used", "prefetch_wasted", "evictions"):
+            assert st[key] == model.stats[key], (step, key)
+        assert st["bytes_h2d"] == model.stats["loads"] * nbytes
+        t0 = r["next"]
+    # the predictions were neither perfect nor useless: some prefetched experts were used, some wasted or pending
+    assert 0 < st["prefetch_used"] < st["prefetch_issued"]
+    dec.close(); cache.close()
+    for L in layers:
+        L.close()
+    ctx.close()

@@ -240,7 +240,13 @@ def _accept_case(dx, M, K, V, H, dtype, seed, rms=False, mode="match"):
             assert tgt[i] == target_ref[i], (i, tgt[i], target_ref[i], gap[i])
         else:
             assert lg[i, tgt[i]] >= srt[i, -1] - GAP
-    # accepted length and next token follow exactly from the GPU's own target tokens
+    # accepted length and next token: the checker's own (n, next) for this draft wherever no row is near-tied ...
+    _, n_ref, next_ref, _ = O.greedy_accept(hn, W_np, draft, logits=lg) if V <= 8192 else \
+        O.greedy_accept_fast(hn, W_np, draft)
+    if (gap > GAP).all():
+        assert int(out["n_accept"].item()) == n_ref
+        assert int(out["next_token"].item()) == next_ref
+    # ... and in every case what the GPU's own target tokens imply (prefix rule restated on the device's tokens)
     n = 0
     while n < K and n < M and draft[n] == tgt[n]:
         n += 1
