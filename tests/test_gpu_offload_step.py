@@ -82,8 +82,11 @@ def test_offloaded_decode_step_full_shape(act_split):
                 check_routing(shape, z_ref, ids_ref, pred[None])
                 want = O.stack_layer_draft(h_np, refs[l], forced_ids=pred[None])[0]
                 assert row_rel_err(rows[l + 1].cpu().numpy(), want).max() <= tol, (step, l)
-            token_ref, q_ref = O.draft_confidence(O.rmsnorm(tok["final"].cpu().numpy().astype(np.float64)), W_np)
+            token_ref, q_ref, lg_d = O.draft_confidence(O.rmsnorm(tok["final"].cpu().numpy().astype(np.float64)), W_np)
             assert abs(tok["q"] - q_ref[0]) <= 1e-3 * q_ref[0] + 1e-7
+            top2 = np.sort(lg_d[0])[-2:]
+            if top2[1] - top2[0] > GAP:
+                assert tok["token"] == int(token_ref[0])
             budget = N_LAYERS * SLOTS - used
             assert tok["budget"] == budget
             stop, delta, new = ctl.propose(tok["pred"], tok["q"], 1.0, budget)
