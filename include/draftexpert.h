@@ -29,6 +29,12 @@
  *     exactly (no rounding of the product).  The router of such a layer is bf16.  The experts stay 4-bit in HBM
  *     and are de-quantised inside the streaming loop of the expert kernel, so a Q4 expert costs 0.94 bytes per
  *     weight of HBM traffic instead of 2.  Every intermediate size must then be a multiple of 32.
+ *     DX_DTYPE_BF16_WIDE: bf16 weights whose expert blobs are packed for the kernel that runs the grouped SwiGLU on
+ *     the 5th-generation tensor cores (tcgen05, accumulators in tensor memory) with the block rows as the 16-column
+ *     operand: its time does not depend on the block length, so it is the layout to choose when blocks of 9..16 rows
+ *     matter (Eq. 4 over longer verification blocks); the streaming layout of DX_DTYPE_BF16 is a little faster for
+ *     blocks of up to 8 rows.  Same blob size, same entry points; activations enter the tensor cores as plain bf16
+ *     (dx_set_activation_split does not apply); dx_stack_create and the 4-bit host pool refuse such layers.
  *   - Limits: block length K <= 16, experts E <= 256, top-k <= 8, shared experts <= 8, every intermediate size
  *     a multiple of 8; hidden a multiple of 256 up to 8192 for fp32 weights and one of 256, 512, 1024, 2048
  *     for bf16 weights.  Outside them: DX_ERR_UNSUPPORTED.
@@ -59,7 +65,12 @@ enum {
 };
 
 enum { DX_SCORE_SOFTMAX = 0, DX_SCORE_SIGMOID = 1 };
-enum { DX_DTYPE_FP32 = 0, DX_DTYPE_BF16 = 1, DX_DTYPE_Q4 = 2 /* experts 4-bit, router bf16 */ };
+enum {
+  DX_DTYPE_FP32 = 0,
+  DX_DTYPE_BF16 = 1,
+  DX_DTYPE_Q4 = 2,        /* experts 4-bit, router bf16 */
+  DX_DTYPE_BF16_WIDE = 3  /* bf16 router and experts, the experts packed for the tcgen05 kernel (see below) */
+};
 
 /* Codes a kernel may leave in the device status word (0 = clean). */
 enum {
@@ -256,6 +267,9 @@ dx_status moe_verify_block_residual(dx_layer* layer, const float* h_in, float* h
                                     int32_t* perm, void* stream);
 dx_status moe_draft_step_residual(dx_layer* layer, const float* h_in, float* h_out, int32_t* topk_ids,
                                   float* topk_w, void* stream);
+/* moe_draft_step_topr (the shared + top-r self-drafter of Sec. 2.2) in the same residual form. */
+dx_status moe_draft_step_topr_residual(dx_layer* layer, const float* h_in, float* h_out, int32_t top_r,
+                                       int32_t use_draft_expert, int32_t* topk_ids, float* topk_w, void* stream);
 
 /* ---- the drafter through a whole stack in one launch --------------------------------------------------------
  * The chain  h_{l+1} = moe_draft_step_residual(layer_l, h_l),  l = 0 .. n_layers-1  (Eq. 5 per layer, one

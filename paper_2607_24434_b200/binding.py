@@ -71,6 +71,7 @@ SIGNATURES = {
     "moe_draft_step": (_I, [_P, _P, _P, _P, _P, _P]),
     "moe_draft_step_topr": (_I, [_P, _P, _P, _I, _I, _P, _P, _P]),
     "moe_draft_step_residual": (_I, [_P, _P, _P, _P, _P, _P]),
+    "moe_draft_step_topr_residual": (_I, [_P, _P, _P, _I, _I, _P, _P, _P]),
     "dx_stack_create": (_I, [_P, C.POINTER(_P), C.c_int32, C.POINTER(_P)]),
     "dx_stack_destroy": (_I, [_P]),
     "moe_draft_stack": (_I, [_P, _P, _P, _P, _P, _P]),
@@ -608,6 +609,14 @@ def moe_draft_step_topr(layer: Layer, h: torch.Tensor, top_r: int, use_draft_exp
            "moe_draft_step_topr")
     out["y"] = y
     return out
+
+
+def moe_draft_step_topr_residual(layer: Layer, h_in: torch.Tensor, h_out: torch.Tensor, top_r: int,
+                                 use_draft_expert: bool, out: Dict[str, torch.Tensor]) -> None:
+    """h_out = h_in + (shared + top-r drafter, optionally with the draft expert) applied to RMSNorm(h_in)."""
+    _check(layer.lib.moe_draft_step_topr_residual(layer.handle, _ptr(h_in), _ptr(h_out), top_r,
+                                                  1 if use_draft_expert else 0, _ptr(out["topk_ids"]),
+                                                  _ptr(out["topk_w"]), _stream()), "moe_draft_step_topr_residual")
 
 
 def spec_draft_token(ctx: Context, h: torch.Tensor, W_lm: torch.Tensor, rms_norm: bool = False):

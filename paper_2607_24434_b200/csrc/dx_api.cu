@@ -120,7 +120,8 @@ static dx_status check_desc(const dx_layer_desc* d) {
   if (!d) return DX_ERR_INVALID_ARG;
   if (d->hidden <= 0 || d->n_experts <= 0 || d->top_k <= 0 || d->inter <= 0 || d->n_shared < 0) return DX_ERR_SHAPE;
   if (d->top_k > d->n_experts) return DX_ERR_SHAPE;
-  if (d->weight_dtype != DX_DTYPE_FP32 && d->weight_dtype != DX_DTYPE_BF16 && d->weight_dtype != DX_DTYPE_Q4)
+  if (d->weight_dtype != DX_DTYPE_FP32 && d->weight_dtype != DX_DTYPE_BF16 && d->weight_dtype != DX_DTYPE_Q4 &&
+      d->weight_dtype != DX_DTYPE_BF16_WIDE)
     return DX_ERR_INVALID_ARG;
   if (d->score_fn != DX_SCORE_SOFTMAX && d->score_fn != DX_SCORE_SIGMOID) return DX_ERR_INVALID_ARG;
   if (d->hidden > DX_MAX_H || d->hidden % 256 || d->n_experts > DX_MAX_E || d->top_k > DX_MAX_TOPK ||
@@ -145,7 +146,8 @@ extern "C" dx_status dx_expert_blob_bytes(const dx_layer_desc* desc, int32_t int
     *bytes_out = (size_t)inter * dx_chunk_bytes(desc->hidden, true);   // inter / 8 units of 8 chunks
     return DX_OK;
   }
-  *bytes_out = (size_t)3 * desc->hidden * inter * (desc->weight_dtype == DX_DTYPE_BF16 ? 2 : 4);
+  if (desc->weight_dtype == DX_DTYPE_BF16_WIDE && !dx_bf16_hidden_supported(desc->hidden)) return DX_ERR_UNSUPPORTED;
+  *bytes_out = (size_t)3 * desc->hidden * inter * (desc->weight_dtype == DX_DTYPE_FP32 ? 4 : 2);
   return DX_OK;
 }
 
@@ -158,6 +160,9 @@ extern "C" dx_status dx_pack_expert(dx_ctx* ctx, const dx_layer_desc* desc, int3
     if (inter % 32 || !dx_bf16_hidden_supported(desc->hidden)) return DX_ERR_UNSUPPORTED;
     if (((uintptr_t)Wg) % 2 || ((uintptr_t)Wu) % 2 || ((uintptr_t)Wd) % 2) return DX_ERR_INVALID_ARG;
     DX_CUDA(ctx, dx_launch_pack_q4(desc->hidden, inter, Wg, Wu, Wd, blob_out, (cudaStream_t)stream));
+  } else if (desc->weight_dtype == DX_DTYPE_BF16_WIDE) {
+    if (!dx_bf16_hidden_supported(desc->hidden)) return DX_ERR_UNSUPPORTED;
+    DX_CUDA(ctx, dx_launch_pack_wide(desc->hidden, inter, Wg, Wu, Wd, blob_out, (cudaStream_t)stream));
   } else {
     DX_CUDA(ctx, dx_launch_pack(desc->weight_dtype, desc->hidden, inter, Wg, Wu, Wd, blob_out, (cudaStream_t)stream));
   }
@@ -305,8 +310,8 @@ static dx_status do_route(dx_layer* L, const float* h, int K, float* y, const Ro
   p.topk_ids = o.topk_ids; p.topk_w = o.topk_w;
   p.union_mask = (unsigned long long*)o.union_mask; p.union_ids = o.union_ids; p.union_count = o.union_count;
   p.offsets = o.offsets; p.perm = o.perm;
-  // (the router of a layer with 4-bit experts is bf16)
-  DX_CUDA(ctx, dx_launch_route(ctx, p, d.weight_dtype == DX_DTYPE_Q4 ? DX_DTYPE_BF16 : d.weight_dtype, st));
+  // (the router of a layer with 4-bit experts, or with experts in the wide layout, is bf16)
+  DX_CUDA(ctx, dx_launch_route(ctx, p, d.weight_dtype == DX_DTYPE_FP32 ? DX_DTYPE_FP32 : DX_DTYPE_BF16, st));
   ctx->launches++;
   return DX_OK;
 }
@@ -356,7 +361,8 @@ static dx_status do_experts(dx_layer* L, const float* h, int K, float* y, bool d
 // follow consumes and clears them.
 static dx_status do_pair(dx_layer* L, const float* h, int K, float* y, const RouteOut& o, bool draft, bool residual,
                          cudaStream_t st, int top_r = 1, bool use_draft_expert = true) {
-  const bool paired = L->desc.weight_dtype != DX_DTYPE_FP32;
+  // (the wide-layout kernel takes the work list in plain stream order)
+  const bool paired = L->desc.weight_dtype == DX_DTYPE_BF16 || L->desc.weight_dtype == DX_DTYPE_Q4;
   dx_status s = do_route(L, h, K, y, o, draft, residual, st, top_r, use_draft_expert, paired);
   if (s != DX_OK) return s;
   s = do_experts(L, h, K, y, draft && use_draft_expert, residual, st, 0, -1, true, paired);
@@ -407,6 +413,15 @@ extern "C" dx_status moe_draft_step_topr(dx_layer* L, const float* h, float* y, 
   RouteOut o{topk_ids, topk_w, nullptr, nullptr, nullptr, nullptr, nullptr};
   if (top_r < 1) return DX_ERR_INVALID_ARG;
   return do_pair(L, h, 1, y, o, true, false, st, top_r, use_draft_expert != 0);
+}
+
+extern "C" dx_status moe_draft_step_topr_residual(dx_layer* L, const float* h_in, float* h_out, int32_t top_r,
+                                                  int32_t use_draft_expert, int32_t* topk_ids, float* topk_w,
+                                                  void* stream) {
+  if (!L) return DX_ERR_INVALID_ARG;
+  RouteOut o{topk_ids, topk_w, nullptr, nullptr, nullptr, nullptr, nullptr};
+  if (top_r < 1) return DX_ERR_INVALID_ARG;
+  return do_pair(L, h_in, 1, h_out, o, true, true, (cudaStream_t)stream, top_r, use_draft_expert != 0);
 }
 
 extern "C" dx_status moe_draft_route(dx_layer* L, const float* h, float* y, int32_t* topk_ids, float* topk_w,
@@ -526,7 +541,8 @@ extern "C" dx_status moe_draft_step_cached(dx_layer* L, const float* h, float* y
 extern "C" dx_status dx_selftest_wait_expiry(dx_layer* L, const float* h, int32_t K, float* y, void* stream) {
   if (!L) return DX_ERR_INVALID_ARG;
   dx_ctx* ctx = L->ctx;
-  if (L->desc.weight_dtype == DX_DTYPE_FP32) return DX_ERR_UNSUPPORTED;   // the fp32 kernels have no hand-over
+  if (L->desc.weight_dtype != DX_DTYPE_BF16 && L->desc.weight_dtype != DX_DTYPE_Q4)
+    return DX_ERR_UNSUPPORTED;   // only the streaming-layout kernels use the hand-over
   if (ctx->wait_limit > (1u << 16)) return DX_ERR_INVALID_ARG;            // keep the give-up short: set a limit first
   cudaStream_t st = (cudaStream_t)stream;
   // hand-over words as a routing kernel leaves them before it publishes anything, and then no routing kernel
@@ -544,7 +560,8 @@ extern "C" dx_status dx_stack_create(dx_ctx* ctx, dx_layer* const* layers, int32
     dx_layer* L = layers[l];
     if (!L || L->ctx != ctx) return DX_ERR_INVALID_ARG;
     const dx_layer_desc &d = L->desc, &d0 = layers[0]->desc;
-    if (d.weight_dtype == DX_DTYPE_FP32 || L->cache) return DX_ERR_UNSUPPORTED;   // resident bf16 / 4-bit experts only
+    if ((d.weight_dtype != DX_DTYPE_BF16 && d.weight_dtype != DX_DTYPE_Q4) || L->cache)
+      return DX_ERR_UNSUPPORTED;   // resident bf16 / 4-bit experts in the streaming layout only
     if (d.weight_dtype != d0.weight_dtype) return DX_ERR_SHAPE;
     if (d.hidden != d0.hidden || d.n_experts != d0.n_experts || d.top_k != d0.top_k || d.inter != d0.inter ||
         d.n_shared != d0.n_shared || d.shared_inter != d0.shared_inter || d.draft_inter != d0.draft_inter ||

@@ -151,7 +151,7 @@ cudaError_t dx_launch_router_agreement(const dx_layer* L, const float* h_star, c
                                        int32_t* agree, cudaStream_t st) {
   const dx_layer_desc& d = L->desc;
   AgreeParams p{h_star, h_draft, L->W_r, L->bias, d.hidden, d.n_experts, d.top_k, d.score_fn, kl, agree};
-  if (d.weight_dtype == DX_DTYPE_BF16)
+  if (d.weight_dtype != DX_DTYPE_FP32)   // (layers with 4-bit or wide-layout experts have a bf16 router)
     dx_router_agreement_kernel<__nv_bfloat16><<<K, kEvalThreads, 0, st>>>(p);
   else
     dx_router_agreement_kernel<float><<<K, kEvalThreads, 0, st>>>(p);

@@ -77,31 +77,6 @@ __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;"
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void cta_bar() { asm volatile("bar.sync 2, 288;" ::: "memory"); }
 
-// This CTA's share of the routed groups.  The launch may be restricted to a window of the routed entries
-// (a "wave" of union experts when the experts are staged through a cache); the units of the window, together
-// with the routing-independent units handled before (NSe of them, [s_lo,s_hi) on this CTA), are split evenly.
-__device__ __forceinline__ void routed_range(int n_groups, const DxExpertParams& p, int n_static, int NSe, int s_lo,
-                                             int s_hi, int G, int cta, int& e_lo, int& e_hi, int& u_lo, int& u_hi) {
-  const int g_lo = min(n_groups, p.first_routed);
-  const int g_hi = p.n_routed < 0 ? n_groups : min(n_groups, g_lo + p.n_routed);
-  e_lo = n_static + g_lo;
-  e_hi = n_static + g_hi;
-  if (g_lo >= g_hi) { u_lo = u_hi = 0; return; }
-  // (unit counts are a few ten thousand at most, grids a few hundred CTAs: the products fit 32 bits)
-  const unsigned int base = (unsigned int)(p.n_shared * p.shared_tiles + p.draft_tiles);
-  const unsigned int R0 = base + (unsigned int)(g_lo * p.routed_tiles);
-  const unsigned int NR = (unsigned int)((g_hi - g_lo) * p.routed_tiles), T = (unsigned int)NSe + NR;
-  const unsigned int uG = (unsigned int)G, ucta = (unsigned int)cta;
-  int a, b;
-  if (T / uG >= ((unsigned int)NSe + uG - 1u) / uG) {   // keep routing-independent + routed units balanced together
-    a = (int)((T * ucta) / uG) - s_lo; b = (int)((T * (ucta + 1u)) / uG) - s_hi;
-  } else {
-    a = (int)((NR * ucta) / uG); b = (int)((NR * (ucta + 1u)) / uG);
-  }
-  u_lo = (int)R0 + a;
-  u_hi = (int)R0 + b;
-}
-
 // TILES = 2: CTA pairs, one tile of eight block rows each (see below); only with NT = 1
 // Eight 4-bit codes -> four bf16 pairs (a lane's A fragment of one contraction step).  Pair p sits in bits
 // [4p, 4p+4) (first element) and [16+4p, 16+4p+4) (second): 0x4300 | code is the bf16 number 128 + code, and
@@ -260,7 +235,7 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
       n_groups = n_sel;
     }
     int e_lo, e_hi, u_lo, u_hi;
-    routed_range(n_groups, p, n_static, NS, s_lo - S0, s_hi - S0, G, cta, e_lo, e_hi, u_lo, u_hi);
+    dx_routed_range(n_groups, p, n_static, NS, s_lo - S0, s_hi - S0, G, cta, e_lo, e_hi, u_lo, u_hi);
     const int unit_base = p.n_shared * p.shared_tiles + p.draft_tiles;
 #pragma unroll
     for (int i = 0; i < PER_LANE; ++i) {
@@ -995,6 +970,7 @@ cudaError_t dx_launch_experts(dx_ctx* ctx, const DxExpertParams& p, int weight_d
   if (weight_dtype == DX_DTYPE_FP32) {
     return dx_launch_pdl((ctx->pdl_mask & DX_PDL_EXPERTS) != 0, dx_experts_fp32_kernel, dim3(ctx->sm_count * 4), dim3(256), 0, st, 1, p);
   }
+  if (weight_dtype == DX_DTYPE_BF16_WIDE) return dx_launch_experts_wide(ctx, p, st);
   if (weight_dtype == DX_DTYPE_Q4) return launch_bf16_any<true, false>(ctx, p, K, st);
   return ctx->act_split ? launch_bf16_any<false, true>(ctx, p, K, st) : launch_bf16_any<false, false>(ctx, p, K, st);
 }

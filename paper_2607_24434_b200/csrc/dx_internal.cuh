@@ -205,6 +205,9 @@ cudaError_t dx_launch_pack(int weight_dtype, int H, int I, const void* Wg, const
 inline size_t dx_chunk_bytes(int H, bool q4) {
   return q4 ? (size_t)(H / 128) * 144 + (size_t)(H / 256) * 192 : (size_t)6 * H;
 }
+cudaError_t dx_launch_experts_wide(dx_ctx* ctx, const DxExpertParams& p, cudaStream_t st);
+cudaError_t dx_launch_pack_wide(int H, int I, const void* Wg, const void* Wu, const void* Wd, void* blob,
+                                cudaStream_t st);
 cudaError_t dx_launch_pack_q4(int H, int I, const void* Wg, const void* Wu, const void* Wd, void* blob,
                               cudaStream_t st);
 cudaError_t dx_launch_expand_q4(int H, int I, const void* q4, void* blob, cudaStream_t st);
@@ -254,6 +257,31 @@ inline cudaError_t dx_launch_pdl(bool pdl, void (*kernel)(KArgs...), dim3 grid, 
   cfg.attrs = attr;
   cfg.numAttrs = n;
   return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
+// This CTA's share of the routed groups.  The launch may be restricted to a window of the routed entries
+// (a "wave" of union experts when the experts are staged through a cache); the units of the window, together
+// with the routing-independent units handled before (NSe of them, [s_lo,s_hi) on this CTA), are split evenly.
+__device__ __forceinline__ void dx_routed_range(int n_groups, const DxExpertParams& p, int n_static, int NSe, int s_lo,
+                                             int s_hi, int G, int cta, int& e_lo, int& e_hi, int& u_lo, int& u_hi) {
+  const int g_lo = min(n_groups, p.first_routed);
+  const int g_hi = p.n_routed < 0 ? n_groups : min(n_groups, g_lo + p.n_routed);
+  e_lo = n_static + g_lo;
+  e_hi = n_static + g_hi;
+  if (g_lo >= g_hi) { u_lo = u_hi = 0; return; }
+  // (unit counts are a few ten thousand at most, grids a few hundred CTAs: the products fit 32 bits)
+  const unsigned int base = (unsigned int)(p.n_shared * p.shared_tiles + p.draft_tiles);
+  const unsigned int R0 = base + (unsigned int)(g_lo * p.routed_tiles);
+  const unsigned int NR = (unsigned int)((g_hi - g_lo) * p.routed_tiles), T = (unsigned int)NSe + NR;
+  const unsigned int uG = (unsigned int)G, ucta = (unsigned int)cta;
+  int a, b;
+  if (T / uG >= ((unsigned int)NSe + uG - 1u) / uG) {   // keep routing-independent + routed units balanced together
+    a = (int)((T * ucta) / uG) - s_lo; b = (int)((T * (ucta + 1u)) / uG) - s_hi;
+  } else {
+    a = (int)((NR * ucta) / uG); b = (int)((NR * (ucta + 1u)) / uG);
+  }
+  u_lo = (int)R0 + a;
+  u_hi = (int)R0 + b;
 }
 
 // Bounds checks of the checked build (-DDX_CHECKED, the stand-in for a memory checker): `if (DX_BOUNDS(i < n, status))`

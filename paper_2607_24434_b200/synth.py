@@ -27,6 +27,7 @@ SCORE_SIGMOID = 1
 DTYPE_FP32 = 0
 DTYPE_BF16 = 1
 DTYPE_Q4 = 2      # experts 4-bit block-quantised (18-byte blocks of 32 weights), router bf16
+DTYPE_BF16_WIDE = 3   # bf16 weights, expert blobs packed for the tcgen05 kernel
 
 
 @dataclasses.dataclass(frozen=True)

@@ -197,6 +197,15 @@ def test_residual_forms(dx):
     torch.cuda.synchronize()
     wantd = O.stack_layer_draft(h_np[:1], ref, forced_ids=outd["topk_ids"].cpu().numpy()[None])[0]
     assert row_rel_err(outd["h"].cpu().numpy(), wantd).max() <= ctx.y_tol
+    # the shared + top-r self-drafter in the same form: h + drafter(RMSNorm(h)), r = 2, without the draft expert
+    buf = {"topk_ids": torch.empty((SMALL.top_k,), dtype=torch.int32, device="cuda"),
+           "topk_w": torch.empty((SMALL.top_k,), dtype=torch.float32, device="cuda")}
+    h1, h2 = h[:1].contiguous(), torch.empty((1, SMALL.hidden), device="cuda")
+    binding.moe_draft_step_topr_residual(L, h1, h2, 2, False, buf)
+    torch.cuda.synchronize()
+    y_r = O.moe_draft(O.rmsnorm(h_np[:1]), ref, forced_ids=buf["topk_ids"].cpu().numpy()[None], top_r=2, gamma=0.0)[0]
+    assert row_rel_err(h2.cpu().numpy(), h_np[:1] + y_r).max() <= ctx.y_tol
+    assert ctx.device_status() == 0
     L.close()
 
 
