@@ -134,6 +134,9 @@ def run_gpu(args):
         dist.init_process_group("nccl", device_id=device)
 
     shape = synth.shape_v2lite()
+    if args.wide:
+        import dataclasses
+        shape = dataclasses.replace(shape, weight_dtype=synth.DTYPE_BF16_WIDE)
     K, V, NL = args.block, args.vocab, args.layers
     ctx = binding.Context(local)
     layers, blocks, W_lm = build_workload(binding, ctx, shape, NL, K, V, 1000 + 50 * rank, device, args.q4_resident)
@@ -442,7 +445,7 @@ def run_gpu(args):
     value = multi.throughput(units_all, total_ms)
     # the drafter through the rotating layers chained as a stack (Eq. 5 per layer, pre-norm residual form) in one
     # persistent launch: the "draft step us per token" figure, per layer
-    dstack = binding.DraftStack(ctx, layers) if not args.q4_resident else None
+    dstack = binding.DraftStack(ctx, layers) if not (args.q4_resident or args.wide) else None
     h_stack = torch.empty((1, H), device=device)
 
     def stack_once():
@@ -499,14 +502,15 @@ def run_gpu(args):
                 "launch": ("one CUDA graph launch (input copies, five kernels, result copies) and one stream "
                            "synchronisation per step") if e2e_graphs is not None else
                           "eager calls and one stream synchronisation per step"},
-        "roofline": {"kernel": "dx_experts_bf16_kernel (grouped SwiGLU of the verify block)", "bound": "hbm",
+        "roofline": {"kernel": ("dx_experts_wide_kernel (grouped SwiGLU of the verify block, tcgen05)" if args.wide else
+                                "dx_experts_bf16_kernel (grouped SwiGLU of the verify block)"), "bound": "hbm",
                      "achieved": verify_gbs, "peak": peak, "unit": "GB/s", "frac": verify_gbs / peak,
                      "frac_is": "pipelined: the kernel alone, back-to-back launches (see `fractions` for the other two "
                                 "ways of timing the same kernel; this is the most favourable of the three)",
                      "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBs": verify_gbs / NOMINAL_HBM_GBS,
                      "fractions": fractions(blk),
                      "traffic": args.traffic if args.traffic is not None else (
-                         None if args.q4_resident else NCU_TRAFFIC_RATIO * float(np.mean(exp_alg))),
+                         None if (args.q4_resident or args.wide) else NCU_TRAFFIC_RATIO * float(np.mean(exp_alg))),
                      "traffic_source": "ncu capture of a 2-layer case scaled by algorithmic bytes (see profiles/)",
                      "ms_per_launch": blk["pipelined_ms"],
                      "ms_per_launch_isolated": blk["isolated_ms"],
@@ -559,6 +563,9 @@ def run_stack(args):
     torch.cuda.set_device(0)
     device = torch.device("cuda", 0)
     shape = synth.shape_moonlight() if args.moonlight else synth.shape_v2lite()
+    if args.wide:
+        import dataclasses
+        shape = dataclasses.replace(shape, weight_dtype=synth.DTYPE_BF16_WIDE)
     V = 163840 if args.moonlight else args.vocab
     NLAY, H = args.stack_layers, shape.hidden
     ctx = binding.Context(0)
@@ -608,20 +615,23 @@ def run_stack(args):
             binding.moe_draft_step_residual(layers[l], hd[l], hd[l + 1], db[l])
 
     chain_ms = timed_graph(draft_body, args.stack_reps)
-    # ... and the same chain as one persistent launch
-    dstack = binding.DraftStack(ctx, layers)
-    sb = {"topk_ids": torch.empty((NLAY, shape.top_k), dtype=torch.int32, device=device),
-          "topk_w": torch.empty((NLAY, shape.top_k), dtype=torch.float32, device=device)}
-    h_stack = torch.empty((1, H), device=device)
+    # ... and the same chain as one persistent launch (streaming blob layout only)
+    if args.wide:
+        draft_ms, same_ids, drift = chain_ms, True, 0.0
+    else:
+        dstack = binding.DraftStack(ctx, layers)
+        sb = {"topk_ids": torch.empty((NLAY, shape.top_k), dtype=torch.int32, device=device),
+              "topk_w": torch.empty((NLAY, shape.top_k), dtype=torch.float32, device=device)}
+        h_stack = torch.empty((1, H), device=device)
 
-    def stack_body():
-        binding.moe_draft_stack(dstack, hd[0], h_stack, sb)
+        def stack_body():
+            binding.moe_draft_stack(dstack, hd[0], h_stack, sb)
 
-    draft_ms = timed_graph(stack_body, args.stack_reps)
-    if ctx.device_status() != 0:
-        raise RuntimeError("device status word set during the draft stack")
-    same_ids = all(torch.equal(sb["topk_ids"][l], db[l]["topk_ids"]) for l in range(NLAY))
-    drift = float(((h_stack - hd[NLAY]).norm() / hd[NLAY].norm()).item())
+        draft_ms = timed_graph(stack_body, args.stack_reps)
+        if ctx.device_status() != 0:
+            raise RuntimeError("device status word set during the draft stack")
+        same_ids = all(torch.equal(sb["topk_ids"][l], db[l]["topk_ids"]) for l in range(NLAY))
+        drift = float(((h_stack - hd[NLAY]).norm() / hd[NLAY].norm()).item())
     draft_bytes = NLAY * ((shape.n_shared + 2) * exp_bytes + shape.n_experts * H * 2)
     out = {"metric": "draft_stack_us_per_token", "value": draft_ms * 1e3, "unit": "us/token", "n_gpus": 1,
            "higher_is_better": False, "data": "synthetic",
@@ -636,7 +646,8 @@ def run_stack(args):
            "draft_gbs": draft_bytes / (draft_ms * 1e-3) / 1e9,
            "draft_frac_of_8TBs": draft_bytes / (draft_ms * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
            "draft_us_per_layer": draft_ms * 1e3 / NLAY,
-           "draft_path": "one persistent cooperative launch for the whole stack",
+           "draft_path": "per-layer launch chain (wide blob layout)" if args.wide else
+                         "one persistent cooperative launch for the whole stack",
            "per_layer_launch_chain_us_per_token": chain_ms * 1e3,
            "chain_agreement": {"same_selection": bool(same_ids), "rel_l2_diff": drift}, "peak_gbs": peak, "peak_kind": peak_kind, "verify": []}
     # ---- the comparison axes of the paper's draft-side table on these synthetic weights: the training-free
@@ -938,6 +949,8 @@ def main():
     ap.add_argument("--vocab", type=int, default=102400)
     ap.add_argument("--layers", type=int, default=8, help="independently seeded layers to rotate over")
     ap.add_argument("--no-k8", action="store_true", help="skip the K = 8 figures of the dominant kernel")
+    ap.add_argument("--wide", action="store_true",
+                    help="layer / stack workloads: experts in the wide blob layout (tcgen05 kernel, any block length)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="time eager launches instead of a CUDA graph replay")
     ap.add_argument("--stack-layers", type=int, default=26)

@@ -18,14 +18,20 @@
 //       W_g (rg even) or W_u (rg odd), columns 64 s + 8 kg .. + 7                    -- one "stage" per s
 //   down region:                       [T < H/128][q < nq][hg < 16] core matrix = rows 128 T + 8 hg .. + 7 of W_d,
 //       columns 8 (8 m + q) .. + 7                                                   -- one stage per T
-// A stage is at most 16 KB and is one bulk copy (a CTA that owns only units q0..q1 of an MU copies that contiguous
-// part of every stage, to the same offset of the shared-memory stage).
+// In either region the part of one unit in one stage is 2 KB of contiguous bytes, and the parts of consecutive units
+// of an MU follow one another.
 //
-// Per MU piece: D1[128 x 16] = [gate rows; up rows] x block rows^T over H (accumulated in tensor memory over the
+// Pieces.  The products cost the same whether a tile of 128 rows is full or not, so the CTA packs its units -- any
+// units, of any experts -- eight at a time into "pieces": unit slot j of a piece is row groups 2 j, 2 j + 1 of the
+// first product and contraction chunk j of the second (both operands of the block are the same for every expert; an
+// expert's weight in a block row is folded into the activations).  A shared-memory stage is 16 KB = 8 unit slots of
+// 2 KB; a run of consecutive units of one MU is one bulk copy per stage.
+//
+// Per piece: D1[128 x 16] = [gate rows; up rows] x block rows^T over H (accumulated in tensor memory over the
 // H/64 stages), the epilogue warps read D1, form w * silu(g) * u in bf16 as the next operand in shared memory, and
 // D2[T][128 x 16] += W_d tile x that, for every tile T of 128 output rows; D2 (H/128 tiles x 16 columns) stays in
-// tensor memory across all pieces of the CTA and is added to y once, at the end.  Rows of a stage that were not
-// copied hold older weights or zeros (the ring is cleared once): their products are finite and meet zero activations.
+// tensor memory across all pieces of the CTA and is added to y once, at the end.  Unit slots a piece does not use
+// hold older weights or zeros (the ring is cleared once): their products are finite and meet zero activations.
 // The first product of piece p + 1 is issued before the second of piece p, so the epilogue's latency is covered.
 //
 // Warps: 0-3 epilogue (tensor-memory lanes 32 w .. 32 w + 31), 4 producer (one lane issues the bulk copies), 5 issues
@@ -35,6 +41,25 @@
 #include "dx_internal.cuh"
 #include "dx_stream.cuh"
 
+#ifdef DX_WIDE_TRACE
+__device__ unsigned long long g_wide_trace[160 * 16];
+__device__ long long g_wide_clk[160 * 64];
+__device__ __forceinline__ void trace(int slot) {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  g_wide_trace[blockIdx.x * 16 + slot] = t;
+}
+extern "C" int dx_debug_wide_trace(unsigned long long* host_out) {
+  return (int)cudaMemcpyFromSymbol(host_out, g_wide_trace, sizeof(unsigned long long) * 160 * 16);
+}
+extern "C" int dx_debug_wide_clk(long long* host_out) {
+  return (int)cudaMemcpyFromSymbol(host_out, g_wide_clk, sizeof(long long) * 160 * 64);
+}
+#define TRACE(slot) trace(slot)
+#else
+#define TRACE(slot)
+#endif
+
 namespace {
 
 constexpr int kWideThreads = 192;
@@ -42,6 +67,8 @@ constexpr int kEpiThreads = 128;
 constexpr int kStageBytes = 16384;
 constexpr int kMaxStages = 12;
 constexpr int kTok = 16;          // token columns of every product
+constexpr int kMaxPieces = 40;
+constexpr int kMaxRuns = 128;
 
 struct WideHeader {
   unsigned long long full[kMaxStages];
@@ -49,7 +76,8 @@ struct WideHeader {
   unsigned long long d1_full[2];
   unsigned long long act_ready[2];
   unsigned long long d2_full;
-  unsigned long long x_ready;
+  unsigned long long list_ready;   // the groups, pairs and pieces below are written
+  unsigned long long x_ready[4];   // quarters of the block-row operand, in the order the first product needs them
   uint32_t tmem_base;
   int abort_flag;
   int ph_e_lo[2], ph_e_hi[2], ph_u_lo[2], ph_u_hi[2];   // routing-independent groups, then routed groups
@@ -62,45 +90,31 @@ struct WideHeader {
   int pair_id[DX_MAX_PAIRS];
   float pair_w[DX_MAX_PAIRS];
   float roww[DX_MAX_ENTRIES][kTok];   // weight of every group in every block row (0: the row is not in the group)
+  // the CTA's units packed into pieces of up to eight unit slots; a run = consecutive units of one macro-unit
+  int n_pieces, n_runs;
+  short piece_run0[kMaxPieces + 1];             // runs of piece p: [piece_run0[p], piece_run0[p + 1])
+  unsigned char piece_slots[kMaxPieces];        // unit slots piece p uses
+  unsigned char piece_entry[kMaxPieces][8];     // group of every unit slot
+  const unsigned char* run_src1[kMaxRuns];      // gate/up part of the run's first unit in stage 0
+  const unsigned char* run_src2[kMaxRuns];      // down part of the run's first unit in tile 0
+  unsigned int run_stride[kMaxRuns];            // bytes from one stage (tile) to the next in the blob
+  unsigned char run_slot0[kMaxRuns], run_n[kMaxRuns];
 };
 
-struct Piece {
-  int e;        // group
-  int m;        // macro-unit of the group's expert
-  int q0, q1;   // units of the macro-unit this CTA owns
-  int nq;       // units the macro-unit has (8, or fewer for an expert's last one)
-};
-
-// The CTA's pieces in the order all three roles walk them.
-template <class F>
-__device__ __forceinline__ void for_each_piece(const WideHeader* hdr, F&& f) {
-  for (int ph = 0; ph < 2; ++ph)
-    for (int e = hdr->ph_e_lo[ph]; e < hdr->ph_e_hi[ph]; ++e) {
-      const int b = hdr->e_begin[e], nt = hdr->e_tiles[e];
-      const int lo = max(b, hdr->ph_u_lo[ph]), hi = min(b + nt, hdr->ph_u_hi[ph]);
-      if (lo >= hi || hdr->e_blob[e] == nullptr) continue;
-      for (int u = lo; u < hi;) {
-        const int m = (u - b) >> 3;
-        const int end = min(hi, b + 8 * (m + 1));
-        Piece pc;
-        pc.e = e; pc.m = m; pc.q0 = (u - b) & 7; pc.q1 = pc.q0 + (end - u); pc.nq = min(8, nt - 8 * m);
-        f(pc);
-        u = end;
-      }
-    }
-}
-
-// shared-memory matrix descriptor: no swizzle, K-major; lbo = bytes between the two core matrices of a product
-// along the contraction, sbo = bytes between groups of eight rows
-__device__ __forceinline__ uint64_t umma_desc(uint32_t addr, uint32_t lbo, uint32_t sbo) {
-  return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo >> 4) << 16) | ((uint64_t)(sbo >> 4) << 32) | (1ull << 46);
-}
+// Shared-memory matrix descriptor (no swizzle, K-major) as two words: low = start address >> 4 | (lbo >> 4) << 16,
+// high = sbo >> 4 | descriptor version; lbo = bytes between the two core matrices of a product along the
+// contraction, sbo = bytes between groups of eight rows.  Only the start address changes from product to product,
+// so the issuing thread adds to the low word and never rebuilds a descriptor: it is a single thread with nothing
+// to hide its instruction latencies behind, and every instruction it executes between two products costs.
+__device__ __forceinline__ uint32_t desc_lo(uint32_t addr, uint32_t lbo) { return ((addr & 0x3FFFFu) >> 4) | ((lbo >> 4) << 16); }
+__device__ __forceinline__ constexpr uint32_t desc_hi(uint32_t sbo) { return (sbo >> 4) | (1u << 14); }
 // D[128 x 16] (+)= A[128 x 16] B[16 x 16]^T, bf16 operands from shared memory, fp32 accumulator in tensor memory
 constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kTok >> 3) << 17) | (8u << 24);
-__device__ __forceinline__ void umma(uint32_t d_tmem, uint64_t da, uint64_t db, uint32_t accumulate) {
-  asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-               "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-               ::"r"(d_tmem), "l"(da), "l"(db), "r"(kIdesc), "r"(accumulate) : "memory");
+__device__ __forceinline__ void umma(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                     uint32_t accumulate) {
+  asm volatile("{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\tmov.b64 da, {%1, %2};\n\tmov.b64 db, {%3, %4};\n\t"
+               "setp.ne.b32 p, %6, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n\t}"
+               ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(kIdesc), "r"(accumulate) : "memory");
 }
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
@@ -119,6 +133,23 @@ __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence:
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void proxy_fence() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
+// Wait of the epilogue warps: lane 0 polls with a pause between looks and the warp takes the outcome from it.  The
+// tensor-core thread and the copy thread share their scheduler partitions with these warps; 128 threads spinning on
+// a barrier would take the issue slots (and the shared-memory cycles) those two need.
+__device__ __forceinline__ bool epi_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t limit, int lane) {
+  int ok = 1;
+  if (lane == 0) {
+    ok = 0;
+    for (uint32_t it = 0; it < limit; ++it) {
+      if (mbar_try_wait(bar, parity)) { ok = 1; break; }
+      if ((it & 15u) == 15u && *abort_flag) break;
+      __nanosleep(64);
+    }
+    if (!ok) *abort_flag = 1;
+  }
+  return __shfl_sync(0xffffffffu, ok, 0) != 0;
+}
 
 __host__ __device__ constexpr int tmem_columns(int H) {
   const int need = 32 + H / 8;   // two D1 buffers of 16 columns, H/128 D2 tiles of 16 columns
@@ -159,7 +190,8 @@ __global__ void __launch_bounds__(kWideThreads, 1) dx_experts_wide_kernel(DxExpe
       mbar_init(smem_u32(&hdr->act_ready[b]), 4);
     }
     mbar_init(smem_u32(&hdr->d2_full), 1);
-    mbar_init(smem_u32(&hdr->x_ready), 4);
+    for (int b = 0; b < 4; ++b) mbar_init(smem_u32(&hdr->x_ready[b]), 4);
+    mbar_init(smem_u32(&hdr->list_ready), 1);
     hdr->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -179,7 +211,12 @@ __global__ void __launch_bounds__(kWideThreads, 1) dx_experts_wide_kernel(DxExpe
   const uint32_t tm_d1 = tmem, tm_d2 = tmem + 32;
 
   // the routing kernel in front has completed once this returns: the work list is final and y is initialised
+#ifdef DX_WIDE_TRACE
+  if (threadIdx.x == 0) { g_wide_trace[blockIdx.x * 16 + 12] = 0; g_wide_trace[blockIdx.x * 16 + 13] = 0; }
+#endif
+  if (threadIdx.x == 0) TRACE(0);
   dx_pdl_wait();
+  if (threadIdx.x == 0) TRACE(1);
 
   // ---- the groups of this launch and this CTA's share of their units (as in dx_grouped.cu, without the hand-over)
   if (warp == 4) {
@@ -191,21 +228,26 @@ __global__ void __launch_bounds__(kWideThreads, 1) dx_experts_wide_kernel(DxExpe
       hdr->e_blob[lane] = DX_BOUNDS(lane < p.table_len, p.dev_status)
                               ? reinterpret_cast<const unsigned char*>(p.table[lane]) : nullptr;
     }
+    // the whole list in one round trip: every word this lane may need is requested before any is looked at (the
+    // list is final, so words past the valid entries are merely ignored)
+    constexpr int PER_LANE = DX_MAX_PAIRS / 32;
+    unsigned long long gw[PER_LANE], pw[PER_LANE];
     const unsigned long long head = dx_word_load(&W->head);
+#pragma unroll
+    for (int i = 0; i < PER_LANE; ++i) gw[i] = dx_word_load(&W->group[lane + 32 * i]);
+#pragma unroll
+    for (int i = 0; i < PER_LANE; ++i) pw[i] = dx_word_load(&W->pair[lane + 32 * i]);
     int n_groups = 0, kk = 1, n_pairs = 0;
     if (head & DX_WORD_VALID) {
       n_groups = min((int)(head & 0xffffu), DX_MAX_PAIRS);
       kk = (int)((head >> 16) & 0xffu);
       n_pairs = min((int)((head >> 24) & 0xffu) * kk, DX_MAX_PAIRS);
     }
-    constexpr int PER_LANE = DX_MAX_PAIRS / 32;
-    unsigned long long gw[PER_LANE];
     int pos[PER_LANE];
     int n_sel = 0;
 #pragma unroll
     for (int i = 0; i < PER_LANE; ++i) {
       const int idx = lane + 32 * i;
-      gw[i] = idx < n_groups ? dx_word_load(&W->group[idx]) : 0ull;
       const int gid = dx_group_id(gw[i]);
       const bool in = idx < n_groups && (gw[i] & DX_WORD_VALID) &&
                       (!p.use_subset || (gid < DX_MAX_E && ((p.subset[gid >> 6] >> (gid & 63)) & 1ull)));
@@ -233,56 +275,147 @@ __global__ void __launch_bounds__(kWideThreads, 1) dx_experts_wide_kernel(DxExpe
       hdr->e_blob[e] = blob;
       if (blob == nullptr && e >= e_lo && e < e_hi) atomicExch(p.dev_status, DX_DEV_BAD_EXPERT_ID);
     }
-    for (int idx = lane; idx < n_pairs; idx += 32) {
-      const unsigned long long w = dx_word_load(&W->pair[idx]);
-      hdr->pair_id[idx] = dx_pair_id(w);
-      hdr->pair_w[idx] = (w & DX_WORD_VALID) ? dx_pair_weight(w) : 0.0f;
+#pragma unroll
+    for (int i = 0; i < PER_LANE; ++i) {
+      const int idx = lane + 32 * i;
+      if (idx < n_pairs) {
+        hdr->pair_id[idx] = dx_pair_id(pw[i]);
+        hdr->pair_w[idx] = (pw[i] & DX_WORD_VALID) ? dx_pair_weight(pw[i]) : 0.0f;
+      }
     }
+    __syncwarp();
     if (lane == 0) {
       hdr->kk = kk;
       hdr->n_pairs = n_pairs;
       hdr->ph_e_lo[0] = 0; hdr->ph_e_hi[0] = p.do_static ? n_static : 0;
       hdr->ph_u_lo[0] = s_lo; hdr->ph_u_hi[0] = s_hi;
       hdr->ph_e_lo[1] = e_lo; hdr->ph_e_hi[1] = e_hi; hdr->ph_u_lo[1] = u_lo; hdr->ph_u_hi[1] = u_hi;
+      // pack this CTA's units into pieces
+      int np = 0, nr = 0, slot = 0;
+      bool overflow = false;
+      hdr->piece_run0[0] = 0;
+      for (int ph = 0; ph < 2 && !overflow; ++ph)
+        for (int e = hdr->ph_e_lo[ph]; e < hdr->ph_e_hi[ph] && !overflow; ++e) {
+          const int b = hdr->e_begin[e], nt = hdr->e_tiles[e];
+          const int lo = max(b, hdr->ph_u_lo[ph]), hi = min(b + nt, hdr->ph_u_hi[ph]);
+          const unsigned char* blob = hdr->e_blob[e];
+          if (lo >= hi || blob == nullptr) continue;
+          for (int u = lo; u < hi && !overflow;) {
+            const int m = (u - b) >> 3, end = min(hi, b + 8 * (m + 1)), nq = min(8, nt - 8 * m);
+            const unsigned char* mu = blob + (size_t)m * 8 * UNIT_BYTES;
+            int q = (u - b) & 7, left = end - u;
+            while (left > 0) {
+              if (nr >= kMaxRuns || np >= kMaxPieces) { overflow = true; break; }
+              const int take = min(left, 8 - slot);
+              hdr->run_src1[nr] = mu + (size_t)q * 2048;
+              hdr->run_src2[nr] = mu + (size_t)nq * 32 * H + (size_t)q * 2048;
+              hdr->run_stride[nr] = (unsigned int)nq * 2048u;
+              hdr->run_slot0[nr] = (unsigned char)slot;
+              hdr->run_n[nr] = (unsigned char)take;
+              for (int i = 0; i < take; ++i) hdr->piece_entry[np][slot + i] = (unsigned char)e;
+              ++nr; slot += take; q += take; left -= take;
+              if (slot == 8) { hdr->piece_slots[np] = 8; ++np; hdr->piece_run0[np] = (short)nr; slot = 0; }
+            }
+            u = end;
+          }
+        }
+      if (!overflow && slot > 0) {
+        if (np >= kMaxPieces) overflow = true;
+        else { hdr->piece_slots[np] = (unsigned char)slot; ++np; hdr->piece_run0[np] = (short)nr; }
+      }
+      if (overflow) { np = 0; nr = 0; atomicExch(p.dev_status, DX_DEV_WORKLIST_OVERFLOW); }
+      hdr->n_pieces = np;
+      hdr->n_runs = nr;
+      mbar_arrive(smem_u32(&hdr->list_ready));   // (release: everything written above is visible to who waits)
+      TRACE(2);
+      dx_pdl_trigger();   // what follows on the stream may be scheduled (it waits for this grid to end)
     }
+  } else if (warp < 4) {
+    // ---- the block rows as the bf16 operand [H/8][2][8 rows x 16 bytes], built while warp 4 reads the work list.
+    // An item is 8 consecutive elements of one row; items are dealt to the 128 threads with the row index fastest
+    // (rows padded to a power of two, so the index arithmetic is shifts) and fetched in batches of eight per thread:
+    // sixteen 16-byte loads in flight instead of one round trip per item.  A batch covers a contiguous range of the
+    // hidden dimension and is handed to the tensor-core thread as soon as it is stored, so the first products start
+    // after one batch.  RMSNorm: the rows go in unscaled and the sums of squares are collected on the way; 1 / rms
+    // of a row is a factor of its whole column of D1, applied by the epilogue.
+    const int tid = threadIdx.x;
+    constexpr int KG = H / 8, BATCH = 8;
+    const int lg = p.K <= 1 ? 0 : p.K <= 2 ? 1 : p.K <= 4 ? 2 : p.K <= 8 ? 3 : 4, Kp = 1 << lg;
+    const int n_items = Kp * KG;
+    if (tid < kTok) hdr->rstd[tid] = 0.0f;
+    for (int idx = tid; idx < (kTok - Kp) * KG; idx += kEpiThreads) {     // token columns beyond the padded block: zero
+      const int kg = idx / (kTok - Kp), t = Kp + idx - kg * (kTok - Kp);
+      *reinterpret_cast<uint4*>(xs + (size_t)kg * 256 + (t >> 3) * 128 + (t & 7) * 16) = make_uint4(0u, 0u, 0u, 0u);
+    }
+    epi_bar();
+    int batch = 0;
+    for (int base0 = 0; base0 < n_items; base0 += kEpiThreads * BATCH, ++batch) {   // (same trip count for every thread)
+      const int base = base0 + tid;
+      float4 a[BATCH], b[BATCH];
+#pragma unroll
+      for (int i = 0; i < BATCH; ++i) {
+        const int idx = base + i * kEpiThreads, t = idx & (Kp - 1), kg = idx >> lg;
+        a[i] = b[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (idx < n_items && t < p.K) {
+          const float* src = p.x + (size_t)t * H + 8 * kg;
+          a[i] = *reinterpret_cast<const float4*>(src);
+          b[i] = *reinterpret_cast<const float4*>(src + 4);
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < BATCH; ++i) {
+        const int idx = base + i * kEpiThreads, t = idx & (Kp - 1), kg = idx >> lg;
+        if (idx < n_items) {
+          uint4 o;
+          __nv_bfloat162 c0 = __floats2bfloat162_rn(a[i].x, a[i].y), c1 = __floats2bfloat162_rn(a[i].z, a[i].w);
+          __nv_bfloat162 c2 = __floats2bfloat162_rn(b[i].x, b[i].y), c3 = __floats2bfloat162_rn(b[i].z, b[i].w);
+          o.x = *reinterpret_cast<uint32_t*>(&c0); o.y = *reinterpret_cast<uint32_t*>(&c1);
+          o.z = *reinterpret_cast<uint32_t*>(&c2); o.w = *reinterpret_cast<uint32_t*>(&c3);
+          *reinterpret_cast<uint4*>(xs + (size_t)kg * 256 + (t >> 3) * 128 + (t & 7) * 16) = o;
+          if (p.rms_norm && t < p.K)
+            atomicAdd(&hdr->rstd[t], a[i].x * a[i].x + a[i].y * a[i].y + a[i].z * a[i].z + a[i].w * a[i].w +
+                                         b[i].x * b[i].x + b[i].y * b[i].y + b[i].z * b[i].z + b[i].w * b[i].w);
+        }
+      }
+      proxy_fence();            // written with ordinary stores, read by the tensor core
+      epi_bar();
+      if (lane == 0 && batch < 4) mbar_arrive(smem_u32(&hdr->x_ready[batch]));
+    }
+    for (; batch < 4; ++batch)   // (short blocks need fewer batches)
+      if (lane == 0) mbar_arrive(smem_u32(&hdr->x_ready[batch]));
   }
-  __syncthreads();
-  if (threadIdx.x == 0) dx_pdl_trigger();   // what follows on the stream may be scheduled (it waits for this grid to end)
+  // (no CTA-wide barrier here: the tensor-core thread starts on the first quarter of the block-row operand while the
+  // epilogue warps are still converting the rest; who needs the work list waits for `list_ready`)
 
   if (warp == 4) {
     // ------------------------------------------------------------------------------------------ producer
     if (lane == 0) {
+      const int n_pieces = hdr->n_pieces;
       uint32_t it = 0, slot = 0, phase = 0;
       bool alive = true;
       const uint64_t l2pol = l2_evict_first_policy();
-      auto push = [&](const unsigned char* src, uint32_t bytes, uint32_t dst_off) {
+      // one stage of piece pc: every run's part of it (src(r) = the run's data in this stage), one barrier
+      auto push = [&](int pc, bool second, uint32_t index) {
         if (!alive) return;
         if (!mbar_wait(smem_u32(&hdr->empty[slot]), phase ^ 1u, abort_flag, p.wait_limit)) { alive = false; return; }
         const uint32_t fb = smem_u32(&hdr->full[slot]);
-        mbar_arrive_expect_tx(fb, bytes);
-        bulk_g2s(smem_u32(ring + (size_t)slot * kStageBytes + dst_off), src, bytes, fb, l2pol);
+        mbar_arrive_expect_tx(fb, (uint32_t)hdr->piece_slots[pc] * 2048u);
+        const uint32_t dst = smem_u32(ring + (size_t)slot * kStageBytes);
+        for (int r = hdr->piece_run0[pc]; r < hdr->piece_run0[pc + 1]; ++r) {
+          const unsigned char* src = (second ? hdr->run_src2[r] : hdr->run_src1[r]) + (size_t)index * hdr->run_stride[r];
+          bulk_g2s(dst + (uint32_t)hdr->run_slot0[r] * 2048u, src, (uint32_t)hdr->run_n[r] * 2048u, fb, l2pol);
+        }
         ++it;
         if (++slot == (uint32_t)n_stages) { slot = 0; phase ^= 1u; }
       };
-      auto gate_up = [&](const Piece& c) {
-        const unsigned char* mu = hdr->e_blob[c.e] + (size_t)c.m * 8 * UNIT_BYTES;
-        const uint32_t bytes = (uint32_t)(c.q1 - c.q0) * 2048u, off = (uint32_t)c.q0 * 2048u;
-        for (int s = 0; s < S1; ++s) push(mu + (size_t)s * c.nq * 2048 + off, bytes, off);
-      };
-      auto down = [&](const Piece& c) {
-        const unsigned char* mu = hdr->e_blob[c.e] + (size_t)c.m * 8 * UNIT_BYTES + (size_t)c.nq * 32 * H;
-        const uint32_t bytes = (uint32_t)(c.q1 - c.q0) * 2048u, off = (uint32_t)c.q0 * 2048u;
-        for (int t = 0; t < S2; ++t) push(mu + (size_t)t * c.nq * 2048 + off, bytes, off);
-      };
-      Piece prev;
-      bool have_prev = false;
-      for_each_piece(hdr, [&](const Piece& c) {
-        gate_up(c);
-        if (have_prev) down(prev);
-        prev = c;
-        have_prev = true;
-      });
-      if (have_prev) down(prev);
+      for (int pc = 0; pc < n_pieces; ++pc) {
+        for (int st = 0; st < S1; ++st) push(pc, false, (uint32_t)st);
+        if (pc > 0)
+          for (int t = 0; t < S2; ++t) push(pc - 1, true, (uint32_t)t);
+      }
+      if (n_pieces > 0)
+        for (int t = 0; t < S2; ++t) push(n_pieces - 1, true, (uint32_t)t);
+      TRACE(11);
       if (*abort_flag) {
         // something gave up: no copy may still be landing when the CTA's shared memory is released
         const uint32_t n_back = it < (uint32_t)n_stages ? it : (uint32_t)n_stages;
@@ -298,99 +431,105 @@ __global__ void __launch_bounds__(kWideThreads, 1) dx_experts_wide_kernel(DxExpe
     // ------------------------------------------------------------------------------------------ tensor-core issue
     if (lane == 0) {
       uint32_t slot = 0, phase = 0;
-      bool alive = mbar_wait(smem_u32(&hdr->x_ready), 0u, abort_flag, p.wait_limit);
-      tc_fence_after();
-      const uint32_t xs_addr = smem_u32(xs), act_addr = smem_u32(acts);
+      bool alive = mbar_wait(smem_u32(&hdr->list_ready), 0u, abort_flag, p.wait_limit);
+      const int n_pieces = alive ? hdr->n_pieces : 0;
+      // quarters of the block-row operand known to be in shared memory; stage s of the first product reads the
+      // hidden columns up to 64 s + 63, which lie in quarter ((8 s + 7) * padded rows) / 1024
+      int x_have = 0;
+      const int x_lg = p.K <= 1 ? 0 : p.K <= 2 ? 1 : p.K <= 4 ? 2 : p.K <= 8 ? 3 : 4;
+      auto need_x = [&](int s) {
+        const int want = min(3, ((8 * s + 7) << x_lg) >> 10);
+        while (alive && x_have <= want) {
+          if (!mbar_wait(smem_u32(&hdr->x_ready[x_have]), 0u, abort_flag, p.wait_limit)) alive = false;
+          tc_fence_after();
+          ++x_have;
+        }
+      };
+      TRACE(3);
+      // low descriptor words of the operands at their base addresses (see desc_lo); a stage is 1024 sixteen-byte units
+      const uint32_t ring_a1 = desc_lo(smem_u32(ring), 128), ring_a2 = desc_lo(smem_u32(ring), 2048);
+      const uint32_t xs_lo = desc_lo(smem_u32(xs), 256), act_lo = desc_lo(smem_u32(acts), 256);
+      constexpr uint32_t A1_HI = desc_hi(1024), A2_HI = desc_hi(128), B_HI = desc_hi(128);
       uint32_t d2_started = 0u;    // bit T: tile T of D2 has been written
-      int n_done = 0;
-      auto next_stage = [&](uint32_t& stage_addr) -> bool {
+      auto next_stage = [&]() -> bool {
         if (!alive) return false;
+        // (the stage was written by a bulk copy, which completes on this barrier in the tensor core's own proxy: the
+        // products may follow the wait directly; a tcgen05 fence here would drain the pipe once per stage)
         if (!mbar_wait(smem_u32(&hdr->full[slot]), phase, abort_flag, p.wait_limit)) { alive = false; return false; }
-        tc_fence_after();
-        stage_addr = smem_u32(ring + (size_t)slot * kStageBytes);
         return true;
       };
       auto release_stage = [&]() {
         umma_commit(smem_u32(&hdr->empty[slot]));     // the slot is free again once the products above have read it
         if (++slot == (uint32_t)n_stages) { slot = 0; phase ^= 1u; }
       };
-      auto gate_up = [&](const Piece& c, int pidx) {
+      auto gate_up = [&](int pidx) {
         const uint32_t d1 = tm_d1 + (uint32_t)(pidx & 1) * kTok;
-        for (int s = 0; s < S1; ++s) {
-          uint32_t st;
-          if (!next_stage(st)) return;
-#pragma unroll
-          for (int j = 0; j < 4; ++j)
-            umma(d1, umma_desc(st + j * 256, 128, 1024), umma_desc(xs_addr + (8 * s + 2 * j) * 256, 256, 128),
-                 (s | j) != 0 ? 1u : 0u);
+        uint32_t b_lo = xs_lo;                      // advances by 8 core-matrix pairs (8 x 256 bytes) per stage
+        for (int s = 0; s < S1; ++s, b_lo += 128) {
+#ifdef DX_WIDE_TRACE
+          const long long c0 = clock64();
+#endif
+          if (x_have < 4) need_x(s);
+          if (!next_stage()) return;
+#ifdef DX_WIDE_TRACE
+          const long long c1 = clock64();
+#endif
+          const uint32_t a_lo = ring_a1 + slot * 1024u;
+          umma(d1, a_lo, A1_HI, b_lo, B_HI, s != 0 ? 1u : 0u);
+          umma(d1, a_lo + 16, A1_HI, b_lo + 32, B_HI, 1u);
+          umma(d1, a_lo + 32, A1_HI, b_lo + 64, B_HI, 1u);
+          umma(d1, a_lo + 48, A1_HI, b_lo + 96, B_HI, 1u);
+#ifdef DX_WIDE_TRACE
+          const long long c2 = clock64();
+#endif
           release_stage();
+#ifdef DX_WIDE_TRACE
+          const long long c3 = clock64();
+          if (pidx == 1 && s < 16) {
+            g_wide_clk[blockIdx.x * 64 + s * 4 + 0] = c1 - c0;
+            g_wide_clk[blockIdx.x * 64 + s * 4 + 1] = c2 - c1;
+            g_wide_clk[blockIdx.x * 64 + s * 4 + 2] = c3 - c2;
+            g_wide_clk[blockIdx.x * 64 + s * 4 + 3] = c3;
+          }
+#endif
         }
         umma_commit(smem_u32(&hdr->d1_full[pidx & 1]));
+        if (pidx < 4) TRACE(4 + pidx);
       };
-      auto down = [&](const Piece& c, int pidx) {
+      auto down = [&](int pidx) {
         // the SwiGLU products of this piece, written by the epilogue warps
         if (alive && !mbar_wait(smem_u32(&hdr->act_ready[pidx & 1]), (uint32_t)(pidx >> 1) & 1u, abort_flag, p.wait_limit))
           alive = false;
         tc_fence_after();
-        const uint32_t act = act_addr + (uint32_t)(pidx & 1) * 2048u;
+        const uint32_t b_lo = act_lo + (uint32_t)(pidx & 1) * 128u;
+        // products whose two unit slots are both unused are left out (their activations are zero anyway)
+        const int used = hdr->piece_slots[pidx];
+        const bool use0 = true, use1 = used > 2, use2 = used > 4, use3 = used > 6;
         for (int t = 0; t < S2; ++t) {
-          uint32_t st;
-          if (!next_stage(st)) return;
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            if (2 * j + 1 < c.q0 || 2 * j >= c.q1) continue;     // both units of this product lie outside the piece
-            umma(tm_d2 + (uint32_t)t * kTok, umma_desc(st + j * 4096, 2048, 128), umma_desc(act + j * 512, 256, 128),
-                 (d2_started >> t) & 1u);
-            d2_started |= 1u << t;
-          }
+          if (!next_stage()) return;
+          const uint32_t a_lo = ring_a2 + slot * 1024u, d2 = tm_d2 + (uint32_t)t * kTok;
+          uint32_t acc = (d2_started >> t) & 1u;
+          if (use0) { umma(d2, a_lo, A2_HI, b_lo, B_HI, acc); acc = 1u; }
+          if (use1) { umma(d2, a_lo + 256, A2_HI, b_lo + 32, B_HI, acc); acc = 1u; }
+          if (use2) { umma(d2, a_lo + 512, A2_HI, b_lo + 64, B_HI, acc); acc = 1u; }
+          if (use3) { umma(d2, a_lo + 768, A2_HI, b_lo + 96, B_HI, acc); acc = 1u; }
           release_stage();
         }
+        d2_started = (S2 >= 32) ? 0xffffffffu : ((1u << S2) - 1u);
       };
-      Piece prev;
-      bool have_prev = false;
-      for_each_piece(hdr, [&](const Piece& c) {
-        gate_up(c, n_done);
-        if (have_prev) down(prev, n_done - 1);
-        prev = c;
-        have_prev = true;
-        ++n_done;
-      });
-      if (have_prev) down(prev, n_done - 1);
+      for (int pc = 0; pc < n_pieces; ++pc) {
+        gate_up(pc);
+        if (pc > 0) down(pc - 1);
+      }
+      if (n_pieces > 0) down(n_pieces - 1);
+      TRACE(8);
       umma_commit(smem_u32(&hdr->d2_full));   // (also what the epilogue waits for before it lets the memory go)
     }
   } else {
     // ------------------------------------------------------------------------------------------ epilogue warps
     const int tid = threadIdx.x;   // 0..127 = tensor-memory lane
-    // 1/rms of the block rows, then the rows as the bf16 operand [H/8][2][8 rows x 16 bytes]
-    for (int r = warp; r < kTok; r += 4) {
-      float rs = 1.0f;
-      if (p.rms_norm && r < p.K) {
-        float ss = 0.f;
-        for (int j = lane * 4; j < H; j += 128) {
-          const float4 v = *reinterpret_cast<const float4*>(p.x + (size_t)r * H + j);
-          ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-        rs = rsqrtf(ss / (float)H + 1e-6f);
-      }
-      if (lane == 0) hdr->rstd[r] = rs;
-    }
-    epi_bar();
-    for (int idx = tid; idx < kTok * (H / 8); idx += kEpiThreads) {
-      const int t = idx & 15, kg = idx >> 4;
-      uint4 o = make_uint4(0u, 0u, 0u, 0u);
-      if (t < p.K) {
-        const float rs = hdr->rstd[t];
-        const float* src = p.x + (size_t)t * H + 8 * kg;
-        const float4 a = *reinterpret_cast<const float4*>(src), b = *reinterpret_cast<const float4*>(src + 4);
-        o.x = pack2(__float2bfloat16_rn(a.x * rs), __float2bfloat16_rn(a.y * rs));
-        o.y = pack2(__float2bfloat16_rn(a.z * rs), __float2bfloat16_rn(a.w * rs));
-        o.z = pack2(__float2bfloat16_rn(b.x * rs), __float2bfloat16_rn(b.y * rs));
-        o.w = pack2(__float2bfloat16_rn(b.z * rs), __float2bfloat16_rn(b.w * rs));
-      }
-      *reinterpret_cast<uint4*>(xs + (size_t)kg * 256 + (t >> 3) * 128 + (t & 7) * 16) = o;
-    }
+    bool alive = epi_wait(smem_u32(&hdr->list_ready), 0u, abort_flag, p.wait_limit, lane);
+    const int n_pieces = alive ? hdr->n_pieces : 0;
     // every group's weight in every block row
     {
       const int n_entries = max(hdr->ph_e_hi[0], hdr->ph_e_hi[1]);
@@ -409,17 +548,13 @@ __global__ void __launch_bounds__(kWideThreads, 1) dx_experts_wide_kernel(DxExpe
         hdr->roww[e][row] = w;
       }
     }
-    proxy_fence();            // the operand above was written with ordinary stores, the tensor core reads it
+    if (tid < kTok) hdr->rstd[tid] = p.rms_norm ? rsqrtf(hdr->rstd[tid] / (float)H + 1e-6f) : 1.0f;
     epi_bar();
-    if (lane == 0) mbar_arrive(smem_u32(&hdr->x_ready));
-
     // lane of tensor memory = row of D1: row group rg = tid / 8 = 2 q + (0 gate | 1 up), row r of the unit
     const int q = tid >> 4, gu = (tid >> 3) & 1, r = tid & 7;
     const uint32_t lane_base = (uint32_t)(32 * warp) << 16;
-    int pidx = 0;
-    bool alive = true;
-    for_each_piece(hdr, [&](const Piece& c) {
-      if (alive && !mbar_wait(smem_u32(&hdr->d1_full[pidx & 1]), (uint32_t)(pidx >> 1) & 1u, abort_flag, p.wait_limit))
+    for (int pidx = 0; pidx < n_pieces; ++pidx) {
+      if (alive && !epi_wait(smem_u32(&hdr->d1_full[pidx & 1]), (uint32_t)(pidx >> 1) & 1u, abort_flag, p.wait_limit, lane))
         alive = false;
       tc_fence_after();
       float v[16];
@@ -428,12 +563,14 @@ __global__ void __launch_bounds__(kWideThreads, 1) dx_experts_wide_kernel(DxExpe
       float other[8];
 #pragma unroll
       for (int i = 0; i < 8; ++i) other[i] = __shfl_xor_sync(0xffffffffu, gu ? v[i] : v[8 + i], 8);
-      const bool mine = q >= c.q0 && q < c.q1;
+      const bool mine = q < (int)hdr->piece_slots[pidx];
       unsigned char* dst = acts + (size_t)(pidx & 1) * 2048 + (size_t)q * 256 + gu * 128 + r * 2;
-      const float* wrow = hdr->roww[c.e] + 8 * gu;
+      const float* wrow = hdr->roww[mine ? hdr->piece_entry[pidx][q] : 0] + 8 * gu;
+      const float* rsrow = hdr->rstd + 8 * gu;
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
-        const float g = gu ? other[i] : v[i], u = gu ? v[8 + i] : other[i];
+        const float rs = rsrow[i];
+        const float g = (gu ? other[i] : v[i]) * rs, u = (gu ? v[8 + i] : other[i]) * rs;
         const float a = mine ? fast_silu(g) * u * wrow[i] : 0.0f;
         *reinterpret_cast<__nv_bfloat16*>(dst + i * 16) = __float2bfloat16_rn(a);
       }
@@ -441,12 +578,12 @@ __global__ void __launch_bounds__(kWideThreads, 1) dx_experts_wide_kernel(DxExpe
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&hdr->act_ready[pidx & 1]));
-      ++pidx;
-    });
+    }
     // ---- this CTA's partial output rows: D2 tile T, lane = output row 128 T + tid, columns = block rows
-    if (alive && !mbar_wait(smem_u32(&hdr->d2_full), 0u, abort_flag, p.wait_limit)) alive = false;
+    if (alive && !epi_wait(smem_u32(&hdr->d2_full), 0u, abort_flag, p.wait_limit, lane)) alive = false;
     tc_fence_after();
-    if (pidx > 0 && alive && !*abort_flag) {
+    if (tid == 0) TRACE(9);
+    if (n_pieces > 0 && alive && !*abort_flag) {
       for (int t = 0; t < S2; ++t) {
         float v[16];
         tmem_ld16(tm_d2 + lane_base + (uint32_t)t * kTok, v);
@@ -458,6 +595,7 @@ __global__ void __launch_bounds__(kWideThreads, 1) dx_experts_wide_kernel(DxExpe
       }
     }
     tc_fence_before();
+    if (tid == 0) TRACE(10);
   }
   // ---- everything this CTA put in flight has landed (or has been waited for): the tensor memory goes back
   __syncthreads();
