@@ -361,8 +361,7 @@ static dx_status do_experts(dx_layer* L, const float* h, int K, float* y, bool d
 // follow consumes and clears them.
 static dx_status do_pair(dx_layer* L, const float* h, int K, float* y, const RouteOut& o, bool draft, bool residual,
                          cudaStream_t st, int top_r = 1, bool use_draft_expert = true) {
-  // (the wide-layout kernel takes the work list in plain stream order)
-  const bool paired = L->desc.weight_dtype == DX_DTYPE_BF16 || L->desc.weight_dtype == DX_DTYPE_Q4;
+  const bool paired = L->desc.weight_dtype != DX_DTYPE_FP32;
   dx_status s = do_route(L, h, K, y, o, draft, residual, st, top_r, use_draft_expert, paired);
   if (s != DX_OK) return s;
   s = do_experts(L, h, K, y, draft && use_draft_expert, residual, st, 0, -1, true, paired);
@@ -541,8 +540,7 @@ extern "C" dx_status moe_draft_step_cached(dx_layer* L, const float* h, float* y
 extern "C" dx_status dx_selftest_wait_expiry(dx_layer* L, const float* h, int32_t K, float* y, void* stream) {
   if (!L) return DX_ERR_INVALID_ARG;
   dx_ctx* ctx = L->ctx;
-  if (L->desc.weight_dtype != DX_DTYPE_BF16 && L->desc.weight_dtype != DX_DTYPE_Q4)
-    return DX_ERR_UNSUPPORTED;   // only the streaming-layout kernels use the hand-over
+  if (L->desc.weight_dtype == DX_DTYPE_FP32) return DX_ERR_UNSUPPORTED;   // the fp32 kernels have no hand-over
   if (ctx->wait_limit > (1u << 16)) return DX_ERR_INVALID_ARG;            // keep the give-up short: set a limit first
   cudaStream_t st = (cudaStream_t)stream;
   // hand-over words as a routing kernel leaves them before it publishes anything, and then no routing kernel

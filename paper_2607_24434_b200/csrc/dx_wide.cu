@@ -41,24 +41,6 @@
 #include "dx_internal.cuh"
 #include "dx_stream.cuh"
 
-#ifdef DX_WIDE_TRACE
-__device__ unsigned long long g_wide_trace[160 * 16];
-__device__ long long g_wide_clk[160 * 64];
-__device__ __forceinline__ void trace(int slot) {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  g_wide_trace[blockIdx.x * 16 + slot] = t;
-}
-extern "C" int dx_debug_wide_trace(unsigned long long* host_out) {
-  return (int)cudaMemcpyFromSymbol(host_out, g_wide_trace, sizeof(unsigned long long) * 160 * 16);
-}
-extern "C" int dx_debug_wide_clk(long long* host_out) {
-  return (int)cudaMemcpyFromSymbol(host_out, g_wide_clk, sizeof(long long) * 160 * 64);
-}
-#define TRACE(slot) trace(slot)
-#else
-#define TRACE(slot)
-#endif
 
 namespace {
 
@@ -68,7 +50,7 @@ constexpr int kStageBytes = 16384;
 constexpr int kMaxStages = 12;
 constexpr int kTok = 16;          // token columns of every product
 constexpr int kMaxPieces = 40;
-constexpr int kMaxRuns = 128;
+constexpr int kMaxRuns = 72;
 
 struct WideHeader {
   unsigned long long full[kMaxStages];
@@ -77,6 +59,7 @@ struct WideHeader {
   unsigned long long act_ready[2];
   unsigned long long d2_full;
   unsigned long long list_ready;   // the groups, pairs and pieces below are written
+  unsigned long long static_ready; // (hand-over) the pieces of the routing-independent groups are written
   unsigned long long x_ready[4];   // quarters of the block-row operand, in the order the first product needs them
   uint32_t tmem_base;
   int abort_flag;
@@ -84,14 +67,15 @@ struct WideHeader {
   int kk, n_pairs;
   float rstd[DX_MAX_K];
   int e_begin[DX_MAX_ENTRIES];
-  int e_tiles[DX_MAX_ENTRIES];
-  int e_gid[DX_MAX_ENTRIES];
+  short e_tiles[DX_MAX_ENTRIES];
+  short e_gid[DX_MAX_ENTRIES];
   const unsigned char* e_blob[DX_MAX_ENTRIES];
-  int pair_id[DX_MAX_PAIRS];
+  short pair_id[DX_MAX_PAIRS];
   float pair_w[DX_MAX_PAIRS];
   float roww[DX_MAX_ENTRIES][kTok];   // weight of every group in every block row (0: the row is not in the group)
   // the CTA's units packed into pieces of up to eight unit slots; a run = consecutive units of one macro-unit
   int n_pieces, n_runs;
+  int n_pieces_a;                               // (hand-over) pieces that do not depend on routing: [0, n_pieces_a)
   short piece_run0[kMaxPieces + 1];             // runs of piece p: [piece_run0[p], piece_run0[p + 1])
   unsigned char piece_slots[kMaxPieces];        // unit slots piece p uses
   unsigned char piece_entry[kMaxPieces][8];     // group of every unit slot
@@ -192,6 +176,7 @@ __global__ void __launch_bounds__(kWideThreads, 1) dx_experts_wide_kernel(DxExpe
     mbar_init(smem_u32(&hdr->d2_full), 1);
     for (int b = 0; b < 4; ++b) mbar_init(smem_u32(&hdr->x_ready[b]), 4);
     mbar_init(smem_u32(&hdr->list_ready), 1);
+    mbar_init(smem_u32(&hdr->static_ready), 1);
     hdr->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -210,16 +195,16 @@ __global__ void __launch_bounds__(kWideThreads, 1) dx_experts_wide_kernel(DxExpe
   const uint32_t tmem = hdr->tmem_base;
   const uint32_t tm_d1 = tmem, tm_d2 = tmem + 32;
 
-  // the routing kernel in front has completed once this returns: the work list is final and y is initialised
-#ifdef DX_WIDE_TRACE
-  if (threadIdx.x == 0) { g_wide_trace[blockIdx.x * 16 + 12] = 0; g_wide_trace[blockIdx.x * 16 + 13] = 0; }
-#endif
-  if (threadIdx.x == 0) TRACE(0);
-  dx_pdl_wait();
-  if (threadIdx.x == 0) TRACE(1);
+  // Two ways to be launched.  Plain: the routing kernel in front has completed once the wait below returns (the work
+  // list is final, y is initialised).  Hand-over (fused entry points): this kernel was made resident by the routing
+  // kernel before either has its input; it streams and multiplies the routing-independent groups while the routing
+  // kernel works, takes the block from memory once a word says it is final, and polls the routed groups and the
+  // (row, expert, gate) pairs out of the work list as they are written (every word carries its own valid bit).
+  const bool paired = p.handover != nullptr;
+  if (!paired) dx_pdl_wait();
 
-  // ---- the groups of this launch and this CTA's share of their units (as in dx_grouped.cu, without the hand-over)
   if (warp == 4) {
+    // ------------------------------------------------------------------------------------------ work list + copies
     if (lane < n_static) {
       const bool is_draft = lane >= p.n_shared;
       hdr->e_begin[lane] = is_draft ? p.n_shared * p.shared_tiles : lane * p.shared_tiles;
@@ -228,15 +213,124 @@ __global__ void __launch_bounds__(kWideThreads, 1) dx_experts_wide_kernel(DxExpe
       hdr->e_blob[lane] = DX_BOUNDS(lane < p.table_len, p.dev_status)
                               ? reinterpret_cast<const unsigned char*>(p.table[lane]) : nullptr;
     }
-    // the whole list in one round trip: every word this lane may need is requested before any is looked at (the
-    // list is final, so words past the valid entries are merely ignored)
+    __syncwarp();
+    // packing state and copy state (used by lane 0 only)
+    int np = 0, nr = 0, pslot = 0;
+    bool overflow = false;
+    uint32_t it = 0, slot = 0, phase = 0;
+    bool alive = true;
+    const uint64_t l2pol = l2_evict_first_policy();
+    if (lane == 0) hdr->piece_run0[0] = 0;
+    // units [u_lo, u_hi) of the groups [e_lo, e_hi) into unit slots, eight to a piece
+    auto pack = [&](int e_lo, int e_hi, int u_lo, int u_hi) {
+      for (int e = e_lo; e < e_hi && !overflow; ++e) {
+        const int b = hdr->e_begin[e], nt = hdr->e_tiles[e];
+        const int lo = max(b, u_lo), hi = min(b + nt, u_hi);
+        const unsigned char* blob = hdr->e_blob[e];
+        if (lo >= hi || blob == nullptr) continue;
+        for (int u = lo; u < hi && !overflow;) {
+          const int m = (u - b) >> 3, end = min(hi, b + 8 * (m + 1)), nq = min(8, nt - 8 * m);
+          const unsigned char* mu = blob + (size_t)m * 8 * UNIT_BYTES;
+          int q = (u - b) & 7, left = end - u;
+          while (left > 0) {
+            if (nr >= kMaxRuns || np >= kMaxPieces) { overflow = true; break; }
+            const int take = min(left, 8 - pslot);
+            hdr->run_src1[nr] = mu + (size_t)q * 2048;
+            hdr->run_src2[nr] = mu + (size_t)nq * 32 * H + (size_t)q * 2048;
+            hdr->run_stride[nr] = (unsigned int)nq * 2048u;
+            hdr->run_slot0[nr] = (unsigned char)pslot;
+            hdr->run_n[nr] = (unsigned char)take;
+            for (int i = 0; i < take; ++i) hdr->piece_entry[np][pslot + i] = (unsigned char)e;
+            ++nr; pslot += take; q += take; left -= take;
+            if (pslot == 8) { hdr->piece_slots[np] = 8; ++np; hdr->piece_run0[np] = (short)nr; pslot = 0; }
+          }
+          u = end;
+        }
+      }
+    };
+    auto close_piece = [&]() {   // a partly filled piece ends here
+      if (!overflow && pslot > 0) {
+        if (np >= kMaxPieces) overflow = true;
+        else { hdr->piece_slots[np] = (unsigned char)pslot; ++np; hdr->piece_run0[np] = (short)nr; pslot = 0; }
+      }
+    };
+    // one stage of piece pc: every run's part of it, completing on one barrier
+    auto push = [&](int pc, bool second, uint32_t index) {
+      if (!alive) return;
+      if (!mbar_wait(smem_u32(&hdr->empty[slot]), phase ^ 1u, abort_flag, p.wait_limit)) { alive = false; return; }
+      const uint32_t fb = smem_u32(&hdr->full[slot]);
+      mbar_arrive_expect_tx(fb, (uint32_t)hdr->piece_slots[pc] * 2048u);
+      const uint32_t dst = smem_u32(ring + (size_t)slot * kStageBytes);
+      for (int r = hdr->piece_run0[pc]; r < hdr->piece_run0[pc + 1]; ++r) {
+        const unsigned char* src = (second ? hdr->run_src2[r] : hdr->run_src1[r]) + (size_t)index * hdr->run_stride[r];
+        bulk_g2s(dst + (uint32_t)hdr->run_slot0[r] * 2048u, src, (uint32_t)hdr->run_n[r] * 2048u, fb, l2pol);
+      }
+      ++it;
+      if (++slot == (uint32_t)n_stages) { slot = 0; phase ^= 1u; }
+    };
+    // pieces [lo, hi): gate/up stages of a piece, then the down stages of the piece before it
+    auto stream = [&](int lo, int hi) {
+      for (int pc = lo; pc < hi; ++pc) {
+        for (int st = 0; st < S1; ++st) push(pc, false, (uint32_t)st);
+        if (pc > lo)
+          for (int t = 0; t < S2; ++t) push(pc - 1, true, (uint32_t)t);
+      }
+      if (hi > lo)
+        for (int t = 0; t < S2; ++t) push(hi - 1, true, (uint32_t)t);
+    };
+    // Hand-over: the routing-independent groups could be multiplied at once, but a CTA's share of them is a few
+    // units -- a piece of their own costs a full piece's products and keeps this warp from polling the list -- so
+    // they wait for the routed groups and are packed with them (measured: 30 us for 2.4 units in a dependent stack).
+    // What overlaps with the routing kernel is this kernel's set-up and the conversion of the block rows.
+    const int n_a = 0;
+    if (lane == 0) {
+      hdr->n_pieces_a = 0;
+      if (paired) mbar_arrive(smem_u32(&hdr->static_ready));
+    }
+    // ---- the routed groups.  Plain launch: the whole list in one round trip (it is final, words past the valid
+    // entries are merely ignored).  Hand-over: polled until the head and every group word it announces are valid.
     constexpr int PER_LANE = DX_MAX_PAIRS / 32;
     unsigned long long gw[PER_LANE], pw[PER_LANE];
-    const unsigned long long head = dx_word_load(&W->head);
+    unsigned long long head = 0ull;
+    // the routed part of the blob table goes to shared memory in the same round trip as the list (the loads are
+    // issued here and consumed after the list has been looked at)
+    const void* tab[DX_MAX_E / 32];
 #pragma unroll
-    for (int i = 0; i < PER_LANE; ++i) gw[i] = dx_word_load(&W->group[lane + 32 * i]);
+    for (int i = 0; i < DX_MAX_E / 32; ++i) {
+      const int e = lane + 32 * i;
+      tab[i] = (p.n_shared + 1 + e < p.table_len)
+                   ? reinterpret_cast<const void*>((uintptr_t)__ldcg(
+                         reinterpret_cast<const unsigned long long*>(p.table + p.n_shared + 1 + e)))
+                   : nullptr;
+    }
+    if (!paired) {
+      head = dx_word_load(&W->head);
 #pragma unroll
-    for (int i = 0; i < PER_LANE; ++i) pw[i] = dx_word_load(&W->pair[lane + 32 * i]);
+      for (int i = 0; i < PER_LANE; ++i) gw[i] = dx_word_load(&W->group[lane + 32 * i]);
+#pragma unroll
+      for (int i = 0; i < PER_LANE; ++i) pw[i] = dx_word_load(&W->pair[lane + 32 * i]);
+    } else {
+      bool have = false;
+      for (uint32_t look = 0; look < p.wait_limit && !have; ++look) {
+        head = dx_word_load(&W->head);
+#pragma unroll
+        for (int i = 0; i < PER_LANE; ++i) gw[i] = dx_word_load(&W->group[lane + 32 * i]);
+        bool mine = false;
+        if (head & DX_WORD_VALID) {
+          const int ng = min((int)(head & 0xffffu), DX_MAX_PAIRS);
+          mine = true;
+#pragma unroll
+          for (int i = 0; i < PER_LANE; ++i) mine = mine && (lane + 32 * i >= ng || (gw[i] & DX_WORD_VALID));
+        }
+        have = __all_sync(0xffffffffu, mine);
+      }
+      if (!have) {
+        head = 0ull;
+        if (lane == 0) { *abort_flag = 1; atomicExch(p.dev_status, DX_DEV_WAIT_EXPIRED); }
+      }
+#pragma unroll
+      for (int i = 0; i < PER_LANE; ++i) pw[i] = 0ull;   // (the pairs are fetched by the epilogue warps)
+    }
     int n_groups = 0, kk = 1, n_pairs = 0;
     if (head & DX_WORD_VALID) {
       n_groups = min((int)(head & 0xffffu), DX_MAX_PAIRS);
@@ -262,11 +356,18 @@ __global__ void __launch_bounds__(kWideThreads, 1) dx_experts_wide_kernel(DxExpe
 #pragma unroll
     for (int i = 0; i < PER_LANE; ++i) {
       const int idx = pos[i];
-      if (idx < 0) continue;
       const int gid = dx_group_id(gw[i]);
+      // the blob of expert gid sits in lane gid % 32, register gid / 32 of the prefetched table
+      unsigned long long got = 0ull;
+#pragma unroll
+      for (int j = 0; j < DX_MAX_E / 32; ++j) {
+        const unsigned long long v = __shfl_sync(0xffffffffu, (unsigned long long)(uintptr_t)tab[j], gid & 31);
+        if ((gid >> 5) == j) got = v;
+      }
+      if (idx < 0) continue;
       const unsigned char* blob = nullptr;
       if (gid < DX_MAX_E && DX_BOUNDS(p.n_shared + 1 + gid < p.table_len, p.dev_status))
-        blob = reinterpret_cast<const unsigned char*>(p.table[p.n_shared + 1 + gid]);
+        blob = reinterpret_cast<const unsigned char*>((uintptr_t)got);
       const int e = n_static + idx;
       if (!DX_BOUNDS(e < DX_MAX_ENTRIES, p.dev_status)) continue;
       hdr->e_begin[e] = unit_base + idx * p.routed_tiles;
@@ -275,62 +376,139 @@ __global__ void __launch_bounds__(kWideThreads, 1) dx_experts_wide_kernel(DxExpe
       hdr->e_blob[e] = blob;
       if (blob == nullptr && e >= e_lo && e < e_hi) atomicExch(p.dev_status, DX_DEV_BAD_EXPERT_ID);
     }
+    if (!paired) {
 #pragma unroll
-    for (int i = 0; i < PER_LANE; ++i) {
-      const int idx = lane + 32 * i;
-      if (idx < n_pairs) {
-        hdr->pair_id[idx] = dx_pair_id(pw[i]);
-        hdr->pair_w[idx] = (pw[i] & DX_WORD_VALID) ? dx_pair_weight(pw[i]) : 0.0f;
+      for (int i = 0; i < PER_LANE; ++i) {
+        const int idx = lane + 32 * i;
+        if (idx < n_pairs) {
+          hdr->pair_id[idx] = dx_pair_id(pw[i]);
+          hdr->pair_w[idx] = (pw[i] & DX_WORD_VALID) ? dx_pair_weight(pw[i]) : 0.0f;
+        }
       }
     }
     __syncwarp();
     if (lane == 0) {
       hdr->kk = kk;
       hdr->n_pairs = n_pairs;
-      hdr->ph_e_lo[0] = 0; hdr->ph_e_hi[0] = p.do_static ? n_static : 0;
-      hdr->ph_u_lo[0] = s_lo; hdr->ph_u_hi[0] = s_hi;
-      hdr->ph_e_lo[1] = e_lo; hdr->ph_e_hi[1] = e_hi; hdr->ph_u_lo[1] = u_lo; hdr->ph_u_hi[1] = u_hi;
-      // pack this CTA's units into pieces
-      int np = 0, nr = 0, slot = 0;
-      bool overflow = false;
-      hdr->piece_run0[0] = 0;
-      for (int ph = 0; ph < 2 && !overflow; ++ph)
-        for (int e = hdr->ph_e_lo[ph]; e < hdr->ph_e_hi[ph] && !overflow; ++e) {
-          const int b = hdr->e_begin[e], nt = hdr->e_tiles[e];
-          const int lo = max(b, hdr->ph_u_lo[ph]), hi = min(b + nt, hdr->ph_u_hi[ph]);
-          const unsigned char* blob = hdr->e_blob[e];
-          if (lo >= hi || blob == nullptr) continue;
-          for (int u = lo; u < hi && !overflow;) {
-            const int m = (u - b) >> 3, end = min(hi, b + 8 * (m + 1)), nq = min(8, nt - 8 * m);
-            const unsigned char* mu = blob + (size_t)m * 8 * UNIT_BYTES;
-            int q = (u - b) & 7, left = end - u;
-            while (left > 0) {
-              if (nr >= kMaxRuns || np >= kMaxPieces) { overflow = true; break; }
-              const int take = min(left, 8 - slot);
-              hdr->run_src1[nr] = mu + (size_t)q * 2048;
-              hdr->run_src2[nr] = mu + (size_t)nq * 32 * H + (size_t)q * 2048;
-              hdr->run_stride[nr] = (unsigned int)nq * 2048u;
-              hdr->run_slot0[nr] = (unsigned char)slot;
-              hdr->run_n[nr] = (unsigned char)take;
-              for (int i = 0; i < take; ++i) hdr->piece_entry[np][slot + i] = (unsigned char)e;
-              ++nr; slot += take; q += take; left -= take;
-              if (slot == 8) { hdr->piece_slots[np] = 8; ++np; hdr->piece_run0[np] = (short)nr; slot = 0; }
-            }
-            u = end;
-          }
-        }
-      if (!overflow && slot > 0) {
-        if (np >= kMaxPieces) overflow = true;
-        else { hdr->piece_slots[np] = (unsigned char)slot; ++np; hdr->piece_run0[np] = (short)nr; }
-      }
-      if (overflow) { np = 0; nr = 0; atomicExch(p.dev_status, DX_DEV_WORKLIST_OVERFLOW); }
+      hdr->ph_e_hi[0] = p.do_static ? n_static : 0;
+      hdr->ph_e_hi[1] = e_hi;
+      if (p.do_static) pack(0, n_static, s_lo, s_hi);
+      pack(e_lo, e_hi, u_lo, u_hi);
+      close_piece();
+      if (overflow) { np = n_a; atomicExch(p.dev_status, DX_DEV_WORKLIST_OVERFLOW); }
       hdr->n_pieces = np;
       hdr->n_runs = nr;
       mbar_arrive(smem_u32(&hdr->list_ready));   // (release: everything written above is visible to who waits)
-      TRACE(2);
-      dx_pdl_trigger();   // what follows on the stream may be scheduled (it waits for this grid to end)
+      if (!paired) dx_pdl_trigger();   // what follows on the stream may be scheduled (it waits for this grid to end)
+      stream(n_a, np);
+      if (*abort_flag) {
+        // something gave up: no copy may still be landing when the CTA's shared memory is released
+        const uint32_t n_back = it < (uint32_t)n_stages ? it : (uint32_t)n_stages;
+        for (uint32_t k = 1; k <= n_back; ++k) {
+          const uint32_t j = it - k, s = j % (uint32_t)n_stages, ph = (j / (uint32_t)n_stages) & 1u;
+          for (uint32_t spin = 0; spin < DX_WAIT_LIMIT_DEFAULT; ++spin)
+            if (mbar_try_wait(smem_u32(&hdr->full[s]), ph)) break;
+        }
+        atomicExch(p.dev_status, DX_DEV_WAIT_EXPIRED);
+      }
     }
-  } else if (warp < 4) {
+  } else if (warp == 5) {
+    // ------------------------------------------------------------------------------------------ tensor-core issue
+    if (lane == 0) {
+      uint32_t slot = 0, phase = 0;
+      bool alive = true;
+      // quarters of the block-row operand known to be in shared memory; stage s of the first product reads the
+      // hidden columns up to 64 s + 63, which lie in quarter ((8 s + 7) * padded rows) / 1024
+      int x_have = 0;
+      const int x_lg = p.K <= 1 ? 0 : p.K <= 2 ? 1 : p.K <= 4 ? 2 : p.K <= 8 ? 3 : 4;
+      auto need_x = [&](int s) {
+        const int want = min(3, ((8 * s + 7) << x_lg) >> 10);
+        while (alive && x_have <= want) {
+          if (!mbar_wait(smem_u32(&hdr->x_ready[x_have]), 0u, abort_flag, p.wait_limit)) alive = false;
+          tc_fence_after();
+          ++x_have;
+        }
+      };
+      // low descriptor words of the operands at their base addresses (see desc_lo); a stage is 1024 sixteen-byte units
+      const uint32_t ring_a1 = desc_lo(smem_u32(ring), 128), ring_a2 = desc_lo(smem_u32(ring), 2048);
+      const uint32_t xs_lo = desc_lo(smem_u32(xs), 256), act_lo = desc_lo(smem_u32(acts), 256);
+      constexpr uint32_t A1_HI = desc_hi(1024), A2_HI = desc_hi(128), B_HI = desc_hi(128);
+      uint32_t d2_started = 0u;    // bit T: tile T of D2 has been written
+      auto next_stage = [&]() -> bool {
+        if (!alive) return false;
+        // (the stage was written by a bulk copy, which completes on this barrier in the tensor core's own proxy: the
+        // products may follow the wait directly; a tcgen05 fence here would drain the pipe once per stage)
+        if (!mbar_wait(smem_u32(&hdr->full[slot]), phase, abort_flag, p.wait_limit)) { alive = false; return false; }
+        return true;
+      };
+      auto release_stage = [&]() {
+        umma_commit(smem_u32(&hdr->empty[slot]));     // the slot is free again once the products above have read it
+        if (++slot == (uint32_t)n_stages) { slot = 0; phase ^= 1u; }
+      };
+      auto gate_up = [&](int pidx) {
+        const uint32_t d1 = tm_d1 + (uint32_t)(pidx & 1) * kTok;
+        uint32_t b_lo = xs_lo;                      // advances by 8 core-matrix pairs (8 x 256 bytes) per stage
+        for (int s = 0; s < S1; ++s, b_lo += 128) {
+          if (x_have < 4) need_x(s);
+          if (!next_stage()) return;
+          const uint32_t a_lo = ring_a1 + slot * 1024u;
+          umma(d1, a_lo, A1_HI, b_lo, B_HI, s != 0 ? 1u : 0u);
+          umma(d1, a_lo + 16, A1_HI, b_lo + 32, B_HI, 1u);
+          umma(d1, a_lo + 32, A1_HI, b_lo + 64, B_HI, 1u);
+          umma(d1, a_lo + 48, A1_HI, b_lo + 96, B_HI, 1u);
+          release_stage();
+        }
+        umma_commit(smem_u32(&hdr->d1_full[pidx & 1]));
+      };
+      auto down = [&](int pidx) {
+        // the SwiGLU products of this piece, written by the epilogue warps
+        if (alive && !mbar_wait(smem_u32(&hdr->act_ready[pidx & 1]), (uint32_t)(pidx >> 1) & 1u, abort_flag, p.wait_limit))
+          alive = false;
+        tc_fence_after();
+        const uint32_t b_lo = act_lo + (uint32_t)(pidx & 1) * 128u;
+        // products whose two unit slots are both unused are left out (their activations are zero anyway)
+        const int used = hdr->piece_slots[pidx];
+        const bool use0 = true, use1 = used > 2, use2 = used > 4, use3 = used > 6;
+        for (int t = 0; t < S2; ++t) {
+          if (!next_stage()) return;
+          const uint32_t a_lo = ring_a2 + slot * 1024u, d2 = tm_d2 + (uint32_t)t * kTok;
+          uint32_t acc = (d2_started >> t) & 1u;
+          if (use0) { umma(d2, a_lo, A2_HI, b_lo, B_HI, acc); acc = 1u; }
+          if (use1) { umma(d2, a_lo + 256, A2_HI, b_lo + 32, B_HI, acc); acc = 1u; }
+          if (use2) { umma(d2, a_lo + 512, A2_HI, b_lo + 64, B_HI, acc); acc = 1u; }
+          if (use3) { umma(d2, a_lo + 768, A2_HI, b_lo + 96, B_HI, acc); acc = 1u; }
+          release_stage();
+        }
+        d2_started = (S2 >= 32) ? 0xffffffffu : ((1u << S2) - 1u);
+      };
+      // pieces [lo, hi): first product of a piece, then the second product of the piece before it
+      auto run = [&](int lo, int hi) {
+        for (int pc = lo; pc < hi; ++pc) {
+          gate_up(pc);
+          if (pc > lo) down(pc - 1);
+        }
+        if (hi > lo) down(hi - 1);
+      };
+      int n_a = 0;
+      if (paired) {   // the routing-independent pieces, while the routing kernel is still at work
+        if (!mbar_wait(smem_u32(&hdr->static_ready), 0u, abort_flag, p.wait_limit)) alive = false;
+        n_a = alive ? hdr->n_pieces_a : 0;
+        run(0, n_a);
+      }
+      if (alive && !mbar_wait(smem_u32(&hdr->list_ready), 0u, abort_flag, p.wait_limit)) alive = false;
+      run(n_a, alive ? hdr->n_pieces : n_a);
+      umma_commit(smem_u32(&hdr->d2_full));   // (also what the epilogue waits for before it lets the memory go)
+    }
+  } else {
+    // ------------------------------------------------------------------------------------------ epilogue warps
+    bool alive = true;
+    if (paired) {
+      // the block itself may still be written by the kernel in front of the routing kernel, which sets this word
+      // once that kernel has completed
+      if (threadIdx.x == 0 && !flag_wait(p.handover, p.wait_limit)) { *abort_flag = 1; atomicExch(p.dev_status, DX_DEV_WAIT_EXPIRED); }
+      epi_bar();   // one poller per CTA; the others pick the acquire up through the barrier
+    }
+    {
     // ---- the block rows as the bf16 operand [H/8][2][8 rows x 16 bytes], built while warp 4 reads the work list.
     // An item is 8 consecutive elements of one row; items are dealt to the 128 threads with the row index fastest
     // (rows padded to a power of two, so the index arithmetic is shifts) and fetched in batches of eight per thread:
@@ -338,7 +516,7 @@ __global__ void __launch_bounds__(kWideThreads, 1) dx_experts_wide_kernel(DxExpe
     // hidden dimension and is handed to the tensor-core thread as soon as it is stored, so the first products start
     // after one batch.  RMSNorm: the rows go in unscaled and the sums of squares are collected on the way; 1 / rms
     // of a row is a factor of its whole column of D1, applied by the epilogue.
-    const int tid = threadIdx.x;
+    const int tid = threadIdx.x;   // 0..127 = tensor-memory lane
     constexpr int KG = H / 8, BATCH = 8;
     const int lg = p.K <= 1 ? 0 : p.K <= 2 ? 1 : p.K <= 4 ? 2 : p.K <= 8 ? 3 : 4, Kp = 1 << lg;
     const int n_items = Kp * KG;
@@ -383,158 +561,15 @@ __global__ void __launch_bounds__(kWideThreads, 1) dx_experts_wide_kernel(DxExpe
     }
     for (; batch < 4; ++batch)   // (short blocks need fewer batches)
       if (lane == 0) mbar_arrive(smem_u32(&hdr->x_ready[batch]));
-  }
-  // (no CTA-wide barrier here: the tensor-core thread starts on the first quarter of the block-row operand while the
-  // epilogue warps are still converting the rest; who needs the work list waits for `list_ready`)
-
-  if (warp == 4) {
-    // ------------------------------------------------------------------------------------------ producer
-    if (lane == 0) {
-      const int n_pieces = hdr->n_pieces;
-      uint32_t it = 0, slot = 0, phase = 0;
-      bool alive = true;
-      const uint64_t l2pol = l2_evict_first_policy();
-      // one stage of piece pc: every run's part of it (src(r) = the run's data in this stage), one barrier
-      auto push = [&](int pc, bool second, uint32_t index) {
-        if (!alive) return;
-        if (!mbar_wait(smem_u32(&hdr->empty[slot]), phase ^ 1u, abort_flag, p.wait_limit)) { alive = false; return; }
-        const uint32_t fb = smem_u32(&hdr->full[slot]);
-        mbar_arrive_expect_tx(fb, (uint32_t)hdr->piece_slots[pc] * 2048u);
-        const uint32_t dst = smem_u32(ring + (size_t)slot * kStageBytes);
-        for (int r = hdr->piece_run0[pc]; r < hdr->piece_run0[pc + 1]; ++r) {
-          const unsigned char* src = (second ? hdr->run_src2[r] : hdr->run_src1[r]) + (size_t)index * hdr->run_stride[r];
-          bulk_g2s(dst + (uint32_t)hdr->run_slot0[r] * 2048u, src, (uint32_t)hdr->run_n[r] * 2048u, fb, l2pol);
-        }
-        ++it;
-        if (++slot == (uint32_t)n_stages) { slot = 0; phase ^= 1u; }
-      };
-      for (int pc = 0; pc < n_pieces; ++pc) {
-        for (int st = 0; st < S1; ++st) push(pc, false, (uint32_t)st);
-        if (pc > 0)
-          for (int t = 0; t < S2; ++t) push(pc - 1, true, (uint32_t)t);
-      }
-      if (n_pieces > 0)
-        for (int t = 0; t < S2; ++t) push(n_pieces - 1, true, (uint32_t)t);
-      TRACE(11);
-      if (*abort_flag) {
-        // something gave up: no copy may still be landing when the CTA's shared memory is released
-        const uint32_t n_back = it < (uint32_t)n_stages ? it : (uint32_t)n_stages;
-        for (uint32_t k = 1; k <= n_back; ++k) {
-          const uint32_t j = it - k, s = j % (uint32_t)n_stages, ph = (j / (uint32_t)n_stages) & 1u;
-          for (uint32_t spin = 0; spin < DX_WAIT_LIMIT_DEFAULT; ++spin)
-            if (mbar_try_wait(smem_u32(&hdr->full[s]), ph)) break;
-        }
-        atomicExch(p.dev_status, DX_DEV_WAIT_EXPIRED);
-      }
     }
-  } else if (warp == 5) {
-    // ------------------------------------------------------------------------------------------ tensor-core issue
-    if (lane == 0) {
-      uint32_t slot = 0, phase = 0;
-      bool alive = mbar_wait(smem_u32(&hdr->list_ready), 0u, abort_flag, p.wait_limit);
-      const int n_pieces = alive ? hdr->n_pieces : 0;
-      // quarters of the block-row operand known to be in shared memory; stage s of the first product reads the
-      // hidden columns up to 64 s + 63, which lie in quarter ((8 s + 7) * padded rows) / 1024
-      int x_have = 0;
-      const int x_lg = p.K <= 1 ? 0 : p.K <= 2 ? 1 : p.K <= 4 ? 2 : p.K <= 8 ? 3 : 4;
-      auto need_x = [&](int s) {
-        const int want = min(3, ((8 * s + 7) << x_lg) >> 10);
-        while (alive && x_have <= want) {
-          if (!mbar_wait(smem_u32(&hdr->x_ready[x_have]), 0u, abort_flag, p.wait_limit)) alive = false;
-          tc_fence_after();
-          ++x_have;
-        }
-      };
-      TRACE(3);
-      // low descriptor words of the operands at their base addresses (see desc_lo); a stage is 1024 sixteen-byte units
-      const uint32_t ring_a1 = desc_lo(smem_u32(ring), 128), ring_a2 = desc_lo(smem_u32(ring), 2048);
-      const uint32_t xs_lo = desc_lo(smem_u32(xs), 256), act_lo = desc_lo(smem_u32(acts), 256);
-      constexpr uint32_t A1_HI = desc_hi(1024), A2_HI = desc_hi(128), B_HI = desc_hi(128);
-      uint32_t d2_started = 0u;    // bit T: tile T of D2 has been written
-      auto next_stage = [&]() -> bool {
-        if (!alive) return false;
-        // (the stage was written by a bulk copy, which completes on this barrier in the tensor core's own proxy: the
-        // products may follow the wait directly; a tcgen05 fence here would drain the pipe once per stage)
-        if (!mbar_wait(smem_u32(&hdr->full[slot]), phase, abort_flag, p.wait_limit)) { alive = false; return false; }
-        return true;
-      };
-      auto release_stage = [&]() {
-        umma_commit(smem_u32(&hdr->empty[slot]));     // the slot is free again once the products above have read it
-        if (++slot == (uint32_t)n_stages) { slot = 0; phase ^= 1u; }
-      };
-      auto gate_up = [&](int pidx) {
-        const uint32_t d1 = tm_d1 + (uint32_t)(pidx & 1) * kTok;
-        uint32_t b_lo = xs_lo;                      // advances by 8 core-matrix pairs (8 x 256 bytes) per stage
-        for (int s = 0; s < S1; ++s, b_lo += 128) {
-#ifdef DX_WIDE_TRACE
-          const long long c0 = clock64();
-#endif
-          if (x_have < 4) need_x(s);
-          if (!next_stage()) return;
-#ifdef DX_WIDE_TRACE
-          const long long c1 = clock64();
-#endif
-          const uint32_t a_lo = ring_a1 + slot * 1024u;
-          umma(d1, a_lo, A1_HI, b_lo, B_HI, s != 0 ? 1u : 0u);
-          umma(d1, a_lo + 16, A1_HI, b_lo + 32, B_HI, 1u);
-          umma(d1, a_lo + 32, A1_HI, b_lo + 64, B_HI, 1u);
-          umma(d1, a_lo + 48, A1_HI, b_lo + 96, B_HI, 1u);
-#ifdef DX_WIDE_TRACE
-          const long long c2 = clock64();
-#endif
-          release_stage();
-#ifdef DX_WIDE_TRACE
-          const long long c3 = clock64();
-          if (pidx == 1 && s < 16) {
-            g_wide_clk[blockIdx.x * 64 + s * 4 + 0] = c1 - c0;
-            g_wide_clk[blockIdx.x * 64 + s * 4 + 1] = c2 - c1;
-            g_wide_clk[blockIdx.x * 64 + s * 4 + 2] = c3 - c2;
-            g_wide_clk[blockIdx.x * 64 + s * 4 + 3] = c3;
-          }
-#endif
-        }
-        umma_commit(smem_u32(&hdr->d1_full[pidx & 1]));
-        if (pidx < 4) TRACE(4 + pidx);
-      };
-      auto down = [&](int pidx) {
-        // the SwiGLU products of this piece, written by the epilogue warps
-        if (alive && !mbar_wait(smem_u32(&hdr->act_ready[pidx & 1]), (uint32_t)(pidx >> 1) & 1u, abort_flag, p.wait_limit))
-          alive = false;
-        tc_fence_after();
-        const uint32_t b_lo = act_lo + (uint32_t)(pidx & 1) * 128u;
-        // products whose two unit slots are both unused are left out (their activations are zero anyway)
-        const int used = hdr->piece_slots[pidx];
-        const bool use0 = true, use1 = used > 2, use2 = used > 4, use3 = used > 6;
-        for (int t = 0; t < S2; ++t) {
-          if (!next_stage()) return;
-          const uint32_t a_lo = ring_a2 + slot * 1024u, d2 = tm_d2 + (uint32_t)t * kTok;
-          uint32_t acc = (d2_started >> t) & 1u;
-          if (use0) { umma(d2, a_lo, A2_HI, b_lo, B_HI, acc); acc = 1u; }
-          if (use1) { umma(d2, a_lo + 256, A2_HI, b_lo + 32, B_HI, acc); acc = 1u; }
-          if (use2) { umma(d2, a_lo + 512, A2_HI, b_lo + 64, B_HI, acc); acc = 1u; }
-          if (use3) { umma(d2, a_lo + 768, A2_HI, b_lo + 96, B_HI, acc); acc = 1u; }
-          release_stage();
-        }
-        d2_started = (S2 >= 32) ? 0xffffffffu : ((1u << S2) - 1u);
-      };
-      for (int pc = 0; pc < n_pieces; ++pc) {
-        gate_up(pc);
-        if (pc > 0) down(pc - 1);
-      }
-      if (n_pieces > 0) down(n_pieces - 1);
-      TRACE(8);
-      umma_commit(smem_u32(&hdr->d2_full));   // (also what the epilogue waits for before it lets the memory go)
-    }
-  } else {
-    // ------------------------------------------------------------------------------------------ epilogue warps
-    const int tid = threadIdx.x;   // 0..127 = tensor-memory lane
-    bool alive = epi_wait(smem_u32(&hdr->list_ready), 0u, abort_flag, p.wait_limit, lane);
-    const int n_pieces = alive ? hdr->n_pieces : 0;
-    // every group's weight in every block row
-    {
-      const int n_entries = max(hdr->ph_e_hi[0], hdr->ph_e_hi[1]);
+    const int tid = threadIdx.x;
+    // lane of tensor memory = row of D1: row group rg = tid / 8 = 2 q + (0 gate | 1 up), row r of the unit
+    const int q = tid >> 4, gu = (tid >> 3) & 1, r = tid & 7;
+    const uint32_t lane_base = (uint32_t)(32 * warp) << 16;
+    // weight of the groups [e_lo, e_hi) in every block row
+    auto row_weights = [&](int e_lo, int e_hi) {
       const int kk = hdr->kk;
-      for (int idx = tid; idx < n_entries * kTok; idx += kEpiThreads) {
+      for (int idx = tid + e_lo * kTok; idx < e_hi * kTok; idx += kEpiThreads) {
         const int e = idx >> 4, row = idx & 15;
         float w = 0.0f;
         if (row < p.K) {
@@ -547,42 +582,78 @@ __global__ void __launch_bounds__(kWideThreads, 1) dx_experts_wide_kernel(DxExpe
         }
         hdr->roww[e][row] = w;
       }
-    }
-    if (tid < kTok) hdr->rstd[tid] = p.rms_norm ? rsqrtf(hdr->rstd[tid] / (float)H + 1e-6f) : 1.0f;
-    epi_bar();
-    // lane of tensor memory = row of D1: row group rg = tid / 8 = 2 q + (0 gate | 1 up), row r of the unit
-    const int q = tid >> 4, gu = (tid >> 3) & 1, r = tid & 7;
-    const uint32_t lane_base = (uint32_t)(32 * warp) << 16;
-    for (int pidx = 0; pidx < n_pieces; ++pidx) {
-      if (alive && !epi_wait(smem_u32(&hdr->d1_full[pidx & 1]), (uint32_t)(pidx >> 1) & 1u, abort_flag, p.wait_limit, lane))
-        alive = false;
-      tc_fence_after();
-      float v[16];
-      tmem_ld16(tm_d1 + lane_base + (uint32_t)(pidx & 1) * kTok, v);
-      // a gate row takes block rows 0..7, its up row (8 lanes on) block rows 8..15: swap the halves each needs
-      float other[8];
+    };
+    // pieces [lo, hi): D1 -> w * silu(gate) * up as the bf16 operand of the second product
+    auto pieces = [&](int lo, int hi) {
+      for (int pidx = lo; pidx < hi; ++pidx) {
+        if (alive && !epi_wait(smem_u32(&hdr->d1_full[pidx & 1]), (uint32_t)(pidx >> 1) & 1u, abort_flag, p.wait_limit, lane))
+          alive = false;
+        tc_fence_after();
+        float v[16];
+        tmem_ld16(tm_d1 + lane_base + (uint32_t)(pidx & 1) * kTok, v);
+        // a gate row takes block rows 0..7, its up row (8 lanes on) block rows 8..15: swap the halves each needs
+        float other[8];
 #pragma unroll
-      for (int i = 0; i < 8; ++i) other[i] = __shfl_xor_sync(0xffffffffu, gu ? v[i] : v[8 + i], 8);
-      const bool mine = q < (int)hdr->piece_slots[pidx];
-      unsigned char* dst = acts + (size_t)(pidx & 1) * 2048 + (size_t)q * 256 + gu * 128 + r * 2;
-      const float* wrow = hdr->roww[mine ? hdr->piece_entry[pidx][q] : 0] + 8 * gu;
-      const float* rsrow = hdr->rstd + 8 * gu;
+        for (int i = 0; i < 8; ++i) other[i] = __shfl_xor_sync(0xffffffffu, gu ? v[i] : v[8 + i], 8);
+        const bool mine = q < (int)hdr->piece_slots[pidx];
+        unsigned char* dst = acts + (size_t)(pidx & 1) * 2048 + (size_t)q * 256 + gu * 128 + r * 2;
+        const float* wrow = hdr->roww[mine ? hdr->piece_entry[pidx][q] : 0] + 8 * gu;
+        const float* rsrow = hdr->rstd + 8 * gu;
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        const float rs = rsrow[i];
-        const float g = (gu ? other[i] : v[i]) * rs, u = (gu ? v[8 + i] : other[i]) * rs;
-        const float a = mine ? fast_silu(g) * u * wrow[i] : 0.0f;
-        *reinterpret_cast<__nv_bfloat16*>(dst + i * 16) = __float2bfloat16_rn(a);
+        for (int i = 0; i < 8; ++i) {
+          const float rs = rsrow[i];
+          const float g = (gu ? other[i] : v[i]) * rs, u = (gu ? v[8 + i] : other[i]) * rs;
+          const float a = mine ? fast_silu(g) * u * wrow[i] : 0.0f;
+          *reinterpret_cast<__nv_bfloat16*>(dst + i * 16) = __float2bfloat16_rn(a);
+        }
+        proxy_fence();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&hdr->act_ready[pidx & 1]));
       }
-      proxy_fence();
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&hdr->act_ready[pidx & 1]));
+    };
+    if (tid < kTok) hdr->rstd[tid] = p.rms_norm ? rsqrtf(hdr->rstd[tid] / (float)H + 1e-6f) : 1.0f;
+    int n_a = 0;
+    if (paired) {
+      if (!epi_wait(smem_u32(&hdr->static_ready), 0u, abort_flag, p.wait_limit, lane)) alive = false;
+      n_a = alive ? hdr->n_pieces_a : 0;
+      row_weights(0, n_static);
+      epi_bar();
+      pieces(0, n_a);
     }
+    if (alive && !epi_wait(smem_u32(&hdr->list_ready), 0u, abort_flag, p.wait_limit, lane)) alive = false;
+    const int n_pieces = alive ? hdr->n_pieces : n_a;
+    if (paired) {
+      // the (row, expert, gate) pairs come out of the gate arithmetic a little after the group list
+      const int n_pairs = alive ? hdr->n_pairs : 0;
+      bool ok = true;
+      for (int idx = tid; idx < n_pairs; idx += kEpiThreads) {
+        unsigned long long w = 0ull;
+        uint32_t look = 0;
+        for (; look < p.wait_limit; ++look) {
+          w = dx_word_load(&W->pair[idx]);
+          if (w & DX_WORD_VALID) break;
+        }
+        ok = ok && look < p.wait_limit;
+        hdr->pair_id[idx] = dx_pair_id(w);
+        hdr->pair_w[idx] = dx_pair_weight(w);
+      }
+      if (!ok) { *abort_flag = 1; atomicExch(p.dev_status, DX_DEV_WAIT_EXPIRED); }
+      epi_bar();
+      // Only now may the next kernel of the stream start: if it is a routing kernel it clears the hand-over words
+      // before its own wait, so every thread of this CTA has to be done with all of them (warp 4 was done with the
+      // group words before it signalled the list).
+      dx_pdl_trigger();
+      row_weights(n_static, hdr->ph_e_hi[1]);
+    } else {
+      row_weights(0, max(hdr->ph_e_hi[0], hdr->ph_e_hi[1]));
+    }
+    epi_bar();
+    pieces(n_a, n_pieces);
+    if (paired) dx_pdl_wait();   // the routing kernel (which initialised y) has completed as a whole
     // ---- this CTA's partial output rows: D2 tile T, lane = output row 128 T + tid, columns = block rows
     if (alive && !epi_wait(smem_u32(&hdr->d2_full), 0u, abort_flag, p.wait_limit, lane)) alive = false;
     tc_fence_after();
-    if (tid == 0) TRACE(9);
     if (n_pieces > 0 && alive && !*abort_flag) {
       for (int t = 0; t < S2; ++t) {
         float v[16];
@@ -595,7 +666,6 @@ __global__ void __launch_bounds__(kWideThreads, 1) dx_experts_wide_kernel(DxExpe
       }
     }
     tc_fence_before();
-    if (tid == 0) TRACE(10);
   }
   // ---- everything this CTA put in flight has landed (or has been waited for): the tensor memory goes back
   __syncthreads();

@@ -143,10 +143,75 @@ def test_wide_refusals(dxw):
     with pytest.raises(binding.DxError) as err:
         binding.DraftStack(ctx, [L])                         # the persistent draft stack reads the streaming layout
     assert err.value.status == 8
-    h = synth.hidden_block(4, SMALL.hidden, 91, 0.0, "cuda")
-    ctx.set_wait_limit(100)
-    with pytest.raises(binding.DxError) as err:
-        binding.selftest_wait_expiry(L, h, torch.empty_like(h))
-    assert err.value.status == 8
-    ctx.set_wait_limit(0)
     L.close()
+
+
+def test_wide_wait_for_a_routing_kernel_that_never_runs_expires(dxw):
+    """The give-up path of the tcgen05 kernel: launched alone in hand-over mode, its bounded waits run out, it frees
+    its tensor memory and returns with DX_DEV_WAIT_EXPIRED; the next ordinary block on the context is correct."""
+    binding, ctx = dxw
+    layer, ref = gpu_layer(SMALL, 92, std=0.08)
+    L = binding.Layer.from_weights(ctx, layer)
+    h = synth.hidden_block(12, SMALL.hidden, 93, 0.0, "cuda")
+    ctx.set_wait_limit(2000)
+    binding.selftest_wait_expiry(L, h, torch.empty_like(h))
+    torch.cuda.synchronize()
+    assert ctx.device_status() == 2
+    ctx.set_wait_limit(0)
+    out = binding.moe_verify_block(L, h)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == 0
+    y_ref = O.moe_target(h.cpu().numpy().astype(np.float64), ref, forced_ids=out["topk_ids"].cpu().numpy())[0]
+    assert row_rel_err(out["y"].cpu().numpy(), y_ref).max() <= Y_BF16
+    L.close()
+
+
+def test_wide_overlapped_pairs_in_a_row(dxw):
+    """Routing / expert kernel pairs back to back from a CUDA graph (stack of residual layers, verify and draft): each
+    expert kernel starts beside its routing kernel and takes block, groups and pairs through the hand-over."""
+    binding, ctx = dxw
+    sh = dataclasses.replace(SMALL, inter=200, shared_inter=72, draft_inter=64)
+    n_layers, K = 4, 11
+    refs, Ls = [], []
+    for l in range(n_layers):
+        layer, ref = gpu_layer(sh, 700 + 10 * l, std=0.08)
+        refs.append(ref); Ls.append(binding.Layer.from_weights(ctx, layer))
+    hs = [torch.zeros((K, sh.hidden), device="cuda") for _ in range(n_layers + 1)]
+    hd = [torch.zeros((1, sh.hidden), device="cuda") for _ in range(n_layers + 1)]
+    rb = [binding._routing_buffers(sh, K, "cuda") for _ in range(n_layers)]
+    db = [{"topk_ids": torch.empty((sh.top_k,), dtype=torch.int32, device="cuda"),
+           "topk_w": torch.empty((sh.top_k,), device="cuda")} for _ in range(n_layers)]
+
+    def chain():
+        for l in range(n_layers):
+            binding.moe_draft_step_residual(Ls[l], hd[l], hd[l + 1], db[l])
+        for l in range(n_layers):
+            binding.moe_verify_block_residual(Ls[l], hs[l], hs[l + 1], rb[l])
+
+    stream = torch.cuda.current_stream()
+    side = torch.cuda.Stream()
+    side.wait_stream(stream)
+    with torch.cuda.stream(side):
+        chain()
+    stream.wait_stream(side)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=side):
+        chain()
+    for rep in range(3):
+        hs[0].copy_(synth.hidden_block(K, sh.hidden, 710 + rep, 0.5, "cuda"))
+        hd[0].copy_(hs[0][:1])
+        for _ in range(20):
+            g.replay()
+        torch.cuda.synchronize()
+        assert ctx.device_status() == 0
+        for l in range(n_layers):
+            ids = rb[l]["topk_ids"].cpu().numpy()
+            want = O.stack_layer_target(hs[l].cpu().numpy().astype(np.float64), refs[l], forced_ids=ids)[0]
+            assert row_rel_err(hs[l + 1].cpu().numpy(), want).max() <= Y_BF16, (rep, l)
+            check_union(sh, K, ids, rb[l])
+            wantd = O.stack_layer_draft(hd[l].cpu().numpy().astype(np.float64), refs[l],
+                                        forced_ids=db[l]["topk_ids"].cpu().numpy()[None])[0]
+            assert row_rel_err(hd[l + 1].cpu().numpy(), wantd).max() <= Y_BF16, (rep, l)
+    for L in Ls:
+        L.close()
