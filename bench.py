@@ -33,10 +33,10 @@ METRIC = "verify_block_moe_tokens_per_s"
 UNIT = "tokens/s"
 NOMINAL_HBM_GBS = 8000.0
 # DRAM bytes (read + write) per launch of the grouped-SwiGLU kernel from the ncu capture summarised in
-# profiles/hot_kernels_v2lite_k4_ncu_full.txt: 259.66 MB read + 3.51 MB written at 259.59 MB algorithmic
+# profiles/hot_kernels_v2lite_k4_ncu_full.txt: 259.63 MB read + 3.56 MB written at 259.59 MB algorithmic
 # (|U| = 13).  The capture runs a 2-layer case; traffic grows with the units streamed, so a launch's traffic is
 # that ratio x its bytes.
-NCU_TRAFFIC_RATIO = (259.655 + 3.507) / 259.59
+NCU_TRAFFIC_RATIO = (259.635 + 3.561) / 259.59
 FALLBACK_HBM_GBS = 6650.0
 
 
