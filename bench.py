@@ -792,9 +792,11 @@ def run_offload(args):
     st0 = cache.stats()
     t0 = time.perf_counter()
     accepted = emitted = drafted = rows = 0
+    union_sum = np.zeros(NLAY)
     for i in range(args.offload_steps):
         r = dec.step(t0_tok, scripted_accept=None if closed else scripted())
         t0_tok = r["next"]
+        union_sum += np.asarray(r["union_sizes"])
         accepted += r["n_accept"]; emitted += len(r["emitted"]); drafted += len(r["drafted"]); rows += r["block_rows"]
     torch.cuda.synchronize()
     dt = time.perf_counter() - t0
@@ -827,6 +829,7 @@ def run_offload(args):
         "prefetch_note": "used / wasted are counted when they happen; experts prefetched in the last step and still "
                          "pending are in neither",
         "h2d_gbs": d["bytes_h2d"] / dt / 1e9, "waited_copies_per_step": d["waited_copies"] / steps, "cache": d,
+        "union_size_per_layer_mean": [round(float(u) / steps, 2) for u in union_sum],
     }))
     dec.close()
 

@@ -102,11 +102,13 @@ class OffloadedDecoder:
         inputs = [int(t0)] + drafted[:K - 1]
         hv = self._hv[0][:K]
         hv.copy_(self.emb[torch.tensor(inputs, device=self.emb.device)].float())
+        union_sizes: List[int] = []
         for l, layer in enumerate(self.layers):
             hv_out = self._hv[(l + 1) & 1][:K]
             if record:
                 rows_in = hv.clone()
             out = binding.moe_verify_block_cached(layer, self.cache, l, hv, hv_out, residual=True)
+            union_sizes.append(len(out["union_list"]))
             if record:
                 trace["verify"].append({"rows": rows_in, "out": hv_out.clone(), "topk_ids": out["topk_ids"].clone(),
                                         "topk_w": out["topk_w"].clone(), "union": out["union_list"]})
@@ -122,7 +124,7 @@ class OffloadedDecoder:
         # row is left for it (with the whole block accepted the next step starts from d_K)
         emitted = drafted[:n] + ([target[n]] if n < K else [])
         res = {"drafted": drafted, "n_accept": n, "emitted": emitted, "next": emitted[-1], "target": target,
-               "block_rows": K, "final": hv}
+               "block_rows": K, "final": hv, "union_sizes": union_sizes}
         if record:
             res["trace"] = trace
         return res
