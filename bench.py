@@ -139,6 +139,8 @@ def run_gpu(args):
         shape = dataclasses.replace(shape, weight_dtype=synth.DTYPE_BF16_WIDE)
     K, V, NL = args.block, args.vocab, args.layers
     ctx = binding.Context(local)
+    if args.launch_overlap is not None:
+        ctx.set_launch_overlap(args.launch_overlap)
     layers, blocks, W_lm = build_workload(binding, ctx, shape, NL, K, V, 1000 + 50 * rank, device, args.q4_resident)
     H = shape.hidden
     stream = torch.cuda.current_stream()
@@ -952,6 +954,8 @@ def main():
     ap.add_argument("--vocab", type=int, default=102400)
     ap.add_argument("--layers", type=int, default=8, help="independently seeded layers to rotate over")
     ap.add_argument("--no-k8", action="store_true", help="skip the K = 8 figures of the dominant kernel")
+    ap.add_argument("--launch-overlap", type=int, default=None,
+                    help="dx_set_launch_overlap mask (bit 0 routing, 1 experts, 2 greedy accept; library default 3)")
     ap.add_argument("--wide", action="store_true",
                     help="layer / stack workloads: experts in the wide blob layout (tcgen05 kernel, any block length)")
     ap.add_argument("--no-cpu-baseline", action="store_true")

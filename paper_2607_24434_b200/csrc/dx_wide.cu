@@ -393,7 +393,12 @@ __global__ void __launch_bounds__(kWideThreads, 1) dx_experts_wide_kernel(DxExpe
       hdr->ph_e_hi[0] = p.do_static ? n_static : 0;
       hdr->ph_e_hi[1] = e_hi;
       if (p.do_static) pack(0, n_static, s_lo, s_hi);
-      pack(e_lo, e_hi, u_lo, u_hi);
+      // (the routed groups all have routed_tiles units: only the few whose units meet this CTA's range are walked)
+      if (u_hi > u_lo && p.routed_tiles > 0) {
+        const int first = n_static + max(0, u_lo - unit_base) / p.routed_tiles;
+        const int last = n_static + max(0, u_hi - 1 - unit_base) / p.routed_tiles;
+        pack(max(e_lo, first), min(e_hi, last + 1), u_lo, u_hi);
+      }
       close_piece();
       if (overflow) { np = n_a; atomicExch(p.dev_status, DX_DEV_WORKLIST_OVERFLOW); }
       hdr->n_pieces = np;
@@ -540,6 +545,7 @@ __global__ void __launch_bounds__(kWideThreads, 1) dx_experts_wide_kernel(DxExpe
           b[i] = *reinterpret_cast<const float4*>(src + 4);
         }
       }
+      float ssq = 0.f;   // (all of a thread's items belong to one row: 128 is a multiple of the padded row count)
 #pragma unroll
       for (int i = 0; i < BATCH; ++i) {
         const int idx = base + i * kEpiThreads, t = idx & (Kp - 1), kg = idx >> lg;
@@ -550,10 +556,15 @@ __global__ void __launch_bounds__(kWideThreads, 1) dx_experts_wide_kernel(DxExpe
           o.x = *reinterpret_cast<uint32_t*>(&c0); o.y = *reinterpret_cast<uint32_t*>(&c1);
           o.z = *reinterpret_cast<uint32_t*>(&c2); o.w = *reinterpret_cast<uint32_t*>(&c3);
           *reinterpret_cast<uint4*>(xs + (size_t)kg * 256 + (t >> 3) * 128 + (t & 7) * 16) = o;
-          if (p.rms_norm && t < p.K)
-            atomicAdd(&hdr->rstd[t], a[i].x * a[i].x + a[i].y * a[i].y + a[i].z * a[i].z + a[i].w * a[i].w +
-                                         b[i].x * b[i].x + b[i].y * b[i].y + b[i].z * b[i].z + b[i].w * b[i].w);
+          ssq += a[i].x * a[i].x + a[i].y * a[i].y + a[i].z * a[i].z + a[i].w * a[i].w +
+                 b[i].x * b[i].x + b[i].y * b[i].y + b[i].z * b[i].z + b[i].w * b[i].w;
         }
+      }
+      if (p.rms_norm) {
+        // lanes that share a row (equal lane mod padded rows) fold their sums; one shared-memory addition per row
+        // and warp (an addition per item made the rows' four to sixteen words a serial bottleneck: 11 us at K = 4)
+        for (int off = 16; off >= Kp; off >>= 1) ssq += __shfl_xor_sync(0xffffffffu, ssq, off);
+        if (lane < Kp && lane < p.K) atomicAdd(&hdr->rstd[lane], ssq);
       }
       proxy_fence();            // written with ordinary stores, read by the tensor core
       epi_bar();
