@@ -293,15 +293,24 @@ __global__ void __launch_bounds__(kRouteThreads) dx_route_kernel(DxRouteParams p
   dx_pdl_trigger();
   // everything this kernel reads or writes from here on may have been in use by the previous kernel
   dx_pdl_wait();
-  if (p.handover && crank == 0 && threadIdx.x == 0) {
-    __threadfence();
-    atomicExch(p.handover, 1u);
-  }
+  // "the block is final", for the expert kernel that is already resident.  The fence in front of the word costs
+  // most of a microsecond; on the tensor-core path it is issued behind this thread's loads of the block rows, so the
+  // two latencies overlap instead of adding up on the way to the group list.
+  auto publish_block_final = [&]() {
+    if (p.handover && crank == 0 && threadIdx.x == 0) {
+      __threadfence();
+      atomicExch(p.handover, 1u);
+    }
+  };
+  if (!kMma) publish_block_final();
+  // routed part of the blob table, for the group list at the end: fetched here, put into shared memory after the
+  // partial logits (a store right away would hold these warps back for a memory round trip, in front of the loads
+  // of the block rows everything else waits for)
+  const void* tab_mine = nullptr;
   if (crank == 0) {
-    // routed part of the blob table, for the group list at the end; empty union mask
     if (threadIdx.x < E && DX_BOUNDS(E <= DX_MAX_E && E <= kRouteThreads, p.dev_status))
-      s_tab[threadIdx.x] = p.table[p.n_shared + 1 + threadIdx.x];
-    if (threadIdx.x < DX_MAX_E / 32) s_mask[threadIdx.x] = 0u;
+      tab_mine = p.table[p.n_shared + 1 + threadIdx.x];
+    if (threadIdx.x < DX_MAX_E / 32) s_mask[threadIdx.x] = 0u;   // empty union mask
   }
 
   // ---- partial logits of this CTA's slice, into CTA 0's table for the slice
@@ -317,6 +326,20 @@ __global__ void __launch_bounds__(kRouteThreads) dx_route_kernel(DxRouteParams p
     float* s_ssq = s_red + (size_t)kRouteWarps * red_stride;           // [8 warps][kpad]
     uint4 bh[2][2], bl[2][2];   // [slab][token tile]
     float ssq[2] = {0.f, 0.f};
+    float4 raw[2][2][2];
+#pragma unroll
+    for (int c = 0; c < 2; ++c)
+#pragma unroll
+      for (int nt = 0; nt < 2; ++nt) {
+        const int tok = nt * 8 + mg;
+        raw[c][nt][0] = raw[c][nt][1] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (c < sp.C && nt < NTK && tok < K && !sp.idle) {
+          const float* hp = p.h + (size_t)tok * H + mcol0 + 256 * c;
+          raw[c][nt][0] = *reinterpret_cast<const float4*>(hp);
+          raw[c][nt][1] = *reinterpret_cast<const float4*>(hp + 4);
+        }
+      }
+    publish_block_final();
 #pragma unroll
     for (int c = 0; c < 2; ++c)
 #pragma unroll
@@ -324,8 +347,7 @@ __global__ void __launch_bounds__(kRouteThreads) dx_route_kernel(DxRouteParams p
         bh[c][nt] = bl[c][nt] = make_uint4(0u, 0u, 0u, 0u);
         const int tok = nt * 8 + mg;
         if (c < sp.C && nt < NTK && tok < K && !sp.idle) {
-          const float* hp = p.h + (size_t)tok * H + mcol0 + 256 * c;
-          const float4 v0 = *reinterpret_cast<const float4*>(hp), v1 = *reinterpret_cast<const float4*>(hp + 4);
+          const float4 v0 = raw[c][nt][0], v1 = raw[c][nt][1];
           const float x[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
           __nv_bfloat16 hb[8], lb[8];
 #pragma unroll
@@ -477,14 +499,30 @@ __global__ void __launch_bounds__(kRouteThreads) dx_route_kernel(DxRouteParams p
     }
   }
   }
-  // y starts at zero, or as a copy of the block in the residual form; nothing reads it before this kernel is over
-  for (int j = (crank * kRouteThreads + threadIdx.x) * 4; j < K * H; j += kRouteCluster * kRouteThreads * 4) {
-    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (p.residual) v = *reinterpret_cast<const float4*>(p.h + j);
-    *reinterpret_cast<float4*>(p.y + j) = v;
-  }
+  if (crank == 0 && threadIdx.x < E && threadIdx.x < DX_MAX_E) s_tab[threadIdx.x] = tab_mine;
   cluster.sync();          // all partial logits have landed in CTA 0
-  if (crank != 0) return;
+  if (crank != 0) {
+    // y starts at zero, or as a copy of the block in the residual form; nothing reads it before this kernel is over,
+    // so the CTAs that are done fill it while CTA 0 selects (in front of the barrier the copy -- one memory round
+    // trip per 16 bytes and thread -- held the group list back by up to 3 us at sixteen rows)
+    constexpr int kFill = 4;
+    const int n_fill = (kRouteCluster - 1) * kRouteThreads;
+    for (int j0 = ((crank - 1) * kRouteThreads + threadIdx.x) * 4; j0 < K * H; j0 += n_fill * 4 * kFill) {
+      float4 v[kFill];
+#pragma unroll
+      for (int i = 0; i < kFill; ++i) {
+        const int j = j0 + i * n_fill * 4;
+        v[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (p.residual && j < K * H) v[i] = *reinterpret_cast<const float4*>(p.h + j);
+      }
+#pragma unroll
+      for (int i = 0; i < kFill; ++i) {
+        const int j = j0 + i * n_fill * 4;
+        if (j < K * H) *reinterpret_cast<float4*>(p.y + j) = v[i];
+      }
+    }
+    return;
+  }
 
   // logits: slices summed in a fixed order, RMSNorm scale and bias applied
   for (int idx = threadIdx.x; idx < K * E; idx += kRouteThreads) {
