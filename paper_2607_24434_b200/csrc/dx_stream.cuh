@@ -69,12 +69,6 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
       "l"(src), "r"(bytes), "r"(bar), "l"(pol)
       : "memory");
 }
-// Asks L2 to fetch [src, src + bytes) from memory (16-byte aligned, a multiple of 16 bytes): no destination and
-// nothing to wait for.  Used where a ring is full but it is already known what will be copied next, so that HBM
-// keeps working while the CTA waits for something else (a routing decision, a grid-wide sum).
-__device__ __forceinline__ void bulk_prefetch_l2(const void* src, uint32_t bytes) {
-  asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
-}
 __device__ __forceinline__ void consumer_bar() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 
 __device__ __forceinline__ void mma_k16(float (&d)[4], const uint4& a, uint32_t b0, uint32_t b1) {

@@ -287,21 +287,6 @@ __global__ void __launch_bounds__(kWideThreads, 1) dx_experts_wide_kernel(DxExpe
       hdr->n_pieces_a = 0;
       if (paired) mbar_arrive(smem_u32(&hdr->static_ready));
     }
-    // (hand-over) ... but their bytes can already be on their way from HBM to L2 while the routing kernel works:
-    // the macro-units this CTA's routing-independent units lie in, 64 KB per request, dealt over the lanes
-    if (paired && p.do_static) {
-      int piece = 0;
-      for (int e = 0; e < n_static; ++e) {
-        const int b = hdr->e_begin[e], nt = hdr->e_tiles[e];
-        const int lo = max(b, s_lo), hi = min(b + nt, s_hi);
-        const unsigned char* blob = hdr->e_blob[e];
-        if (lo >= hi || blob == nullptr) continue;
-        const size_t first = (size_t)((lo - b) >> 3) * 8 * UNIT_BYTES;
-        const size_t last = min((size_t)nt, (size_t)(((hi - 1 - b) >> 3) + 1) * 8) * UNIT_BYTES;
-        for (size_t off = first; off < last; off += 65536, ++piece)
-          if ((piece & 31) == lane) bulk_prefetch_l2(blob + off, (uint32_t)min((size_t)65536, last - off));
-      }
-    }
     // ---- the routed groups.  Plain launch: the whole list in one round trip (it is final, words past the valid
     // entries are merely ignored).  Hand-over: polled until the head and every group word it announces are valid.
     constexpr int PER_LANE = DX_MAX_PAIRS / 32;
