@@ -578,7 +578,7 @@ extern "C" dx_status dx_stack_create(dx_ctx* ctx, dx_layer* const* layers, int32
   for (int l = 0; l < n_layers; ++l) s->layers[l] = layers[l];
   const dx_layer_desc& d = layers[0]->desc;
   cudaError_t e = cudaMalloc(&s->desc_dev, sizeof(DxStackLayer) * n_layers);
-  s->zword_off = sizeof(float) * (size_t)n_layers * d.hidden;
+  s->zword_off = sizeof(float) * (size_t)n_layers * DX_STACK_COPIES * d.hidden;
   s->sync_off = s->zword_off + sizeof(unsigned long long) * (size_t)n_layers * d.n_experts;
   s->scratch_bytes = s->sync_off + sizeof(unsigned int) * n_layers;
   if (e == cudaSuccess) e = cudaMalloc(&s->scratch, s->scratch_bytes);

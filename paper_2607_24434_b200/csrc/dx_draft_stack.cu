@@ -5,9 +5,10 @@
 // token, so a layer lasts ~10 us at HBM speed and every microsecond between two layers shows.  One launch per layer
 // pays a kernel boundary each time; here one cooperative grid (one CTA per SM) stays resident for all layers:
 //   * every CTA keeps the hidden row in shared memory.  A layer's contributions are added (vector reductions in
-//     L2) to that layer's own delta row in global memory, zero at launch; once the layer's arrival counter shows
-//     all CTAs, each CTA adds the delta row to its copy.  No row is ever initialised or copied between layers,
-//     and the counter is the only grid-wide wait of a layer;
+//     L2) to that layer's own delta rows in global memory, zero at launch -- a few partial rows per layer, CTA c
+//     into row c mod DX_STACK_COPIES, because additions to one address are serial in L2; once the layer's arrival
+//     counter shows all CTAs, each CTA (all its warps but the producer) adds the partial rows to its copy.  No row
+//     is ever initialised or copied between layers, and the counter is the only grid-wide wait of a layer;
 //   * the producer warp of every CTA streams its share of the layer's routing-independent units (shared experts,
 //     draft expert) and, because weights are constants, runs ahead into the next layer while the current one is
 //     still being reduced -- the ring does not drain at a layer boundary;
@@ -38,7 +39,7 @@ struct StackSmem {
   unsigned long long full[kStackMaxSlots];
   unsigned long long empty[kStackMaxSlots];
   int abort_flag;
-  float rstd;   // 1/rms of the current hidden row
+  float ssq[kStackConsumers];   // sums of squares of the current hidden row, one per consumer warp
   // what the router warp found for the current layer
   int r_have;                    // 0: the routed expert has no blob (reported; the layer goes on without it)
   float r_w;                     // its gate
@@ -130,6 +131,48 @@ __global__ void __launch_bounds__(kStackThreads, 1) dx_draft_stack_kernel(DxStac
     *reinterpret_cast<float4*>(x_s + j) = *reinterpret_cast<const float4*>(p.h_in + j);
   __syncthreads();
 
+  // Advance the hidden row by the finished layer's partial rows (layer l - 1; nothing to add for l = 0) and collect
+  // its sum of squares.  Done by the eight consumer warps together (they have nothing else to do at this point, and
+  // the router warp keeps its registers for the router rows it has fetched): every thread owns one or two 16-byte
+  // pieces of the row and has the pieces of all partial rows in flight at once (one memory round trip).
+  constexpr int kAdvThreads = kStackConsumers * 32;
+  constexpr int kAdvPieces = (H / 4 + kAdvThreads - 1) / kAdvThreads;
+  auto advance_row = [&](int l, int q) {   // q: 0 .. kAdvThreads - 1 (the consumer's thread index)
+    float4 part[kAdvPieces][DX_STACK_COPIES];
+    if (l > 0) {
+#pragma unroll
+      for (int n = 0; n < kAdvPieces; ++n) {
+        const int j = (q + n * kAdvThreads) * 4;
+#pragma unroll
+        for (int c = 0; c < DX_STACK_COPIES; ++c)
+          part[n][c] = j < H ? __ldcg(reinterpret_cast<const float4*>(p.delta + ((size_t)(l - 1) * DX_STACK_COPIES + c) * H + j))
+                             : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+    }
+    float ss = 0.f;
+#pragma unroll
+    for (int n = 0; n < kAdvPieces; ++n) {
+      const int j = (q + n * kAdvThreads) * 4;
+      if (j < H) {
+        float4 v = *reinterpret_cast<float4*>(x_s + j);
+        if (l > 0) {
+#pragma unroll
+          for (int c = 0; c < DX_STACK_COPIES; ++c) { v.x += part[n][c].x; v.y += part[n][c].y; v.z += part[n][c].z; v.w += part[n][c].w; }
+          *reinterpret_cast<float4*>(x_s + j) = v;
+        }
+        ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+      }
+    }
+    ss = stack_warp_sum(ss);
+    if ((q & 31) == 0) hdr->ssq[q >> 5] = ss;
+  };
+  auto row_rstd = [&]() {
+    float t = 0.f;
+#pragma unroll
+    for (int w = 0; w < kStackConsumers; ++w) t += hdr->ssq[w];
+    return rsqrtf(t / (float)H + 1e-6f);
+  };
+
   if (warp == kStackConsumers) {
     // ---------------------------------------------------------------- producer
     uint32_t it = 0, slot = 0, phase = 0;   // chunk counter, its ring slot and that slot's phase bit
@@ -202,28 +245,10 @@ __global__ void __launch_bounds__(kStackThreads, 1) dx_draft_stack_kernel(DxStac
       if (l > 0 && lane == 0) ok = counter_wait(p.sync + (l - 1), (unsigned int)G, p.wait_limit);   // layer l-1 is complete
       __syncwarp();   // orders the other lanes' reads of the delta row behind lane 0's acquire (a shuffle would not)
       ok = __shfl_sync(0xffffffffu, ok, 0);
-      // advance the hidden row by the finished layer's delta; its mean square on the way
-      float ss = 0.f;
-      {
-        float4 dlt[H / 128];
-        if (l > 0) {
-          const float* dl = p.delta + (size_t)(l - 1) * H + lane * 4;
-#pragma unroll
-          for (int i = 0; i < H / 128; ++i) dlt[i] = __ldcg(reinterpret_cast<const float4*>(dl + 128 * i));
-        }
-#pragma unroll
-        for (int i = 0; i < H / 128; ++i) {
-          float4 v = *reinterpret_cast<float4*>(x_s + lane * 4 + 128 * i);
-          if (l > 0) {
-            v.x += dlt[i].x; v.y += dlt[i].y; v.z += dlt[i].z; v.w += dlt[i].w;
-            *reinterpret_cast<float4*>(x_s + lane * 4 + 128 * i) = v;
-          }
-          ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
-        }
-      }
+      asm volatile("bar.sync 5, 288;" ::: "memory");   // the finished layer's sums are complete: the consumers advance the row
+      asm volatile("bar.sync 3, 288;" ::: "memory");   // the row is advanced, its sums of squares are in place
       if (l == L) {   // past the last layer: the row is the result
         if (cta == 0) {
-          __syncwarp();
           for (int j = lane * 4; j < H; j += 128)
             *reinterpret_cast<float4*>(p.h_out + j) = *reinterpret_cast<const float4*>(x_s + j);
         }
@@ -231,11 +256,7 @@ __global__ void __launch_bounds__(kStackThreads, 1) dx_draft_stack_kernel(DxStac
         break;
       }
       const DxStackLayer& ly = p.layers[l];
-      const float rstd = rsqrtf(stack_warp_sum(ss) / (float)H + 1e-6f);
-      if (lane == 0) hdr->rstd = rstd;
-      __threadfence_block();
-      __syncwarp();
-      asm volatile("bar.sync 3, 288;" ::: "memory");   // the consumers may read the row
+      const float rstd = row_rstd();
       // this CTA's router rows, each logit published as (1 << 32 | float bits)
       for (int e = cta; e < E; e += G) {
         float acc = 0.f;
@@ -354,11 +375,14 @@ __global__ void __launch_bounds__(kStackThreads, 1) dx_draft_stack_kernel(DxStac
   const int g = lane >> 2, c = lane & 3;
   uint32_t cslot = (uint32_t)warp, cphase = 0;   // ring slot (and its phase bit) of this warp's chunk of the next unit
   int buf = 0;
-  for (int l = 0; l < L; ++l) {
-    asm volatile("bar.sync 3, 288;" ::: "memory");   // the router warp has advanced the hidden row to this layer
+  for (int l = 0; l <= L; ++l) {
+    asm volatile("bar.sync 5, 288;" ::: "memory");   // the router warp has seen every CTA's arrival for layer l - 1
+    advance_row(l, threadIdx.x);
+    asm volatile("bar.sync 3, 288;" ::: "memory");   // the hidden row stands at layer l
+    if (l == L) break;   // (the router warp of CTA 0 writes the result)
     // the token fragments of this warp's contraction slice: token slot 0 is the normalised row, the other seven
     // slots are zero
-    const float rs = hdr->rstd;
+    const float rs = row_rstd();
     // One token only: the tensor cores would spend seven of their eight token columns (and a second pass for the
     // low halves of the activations) on nothing, and at one token their issue rate, not the stream, sets the
     // pace.  The same fragments are consumed with plain FMAs instead: a lane holds rows g and g + 8 of a
@@ -478,7 +502,7 @@ __global__ void __launch_bounds__(kStackThreads, 1) dx_draft_stack_kernel(DxStac
     // the layer's partial output row goes to the layer's delta row.  The four lanes of a row group first add
     // their contraction columns up (lane 4g then has rows g and g + 8 of each 16-row tile); four neighbouring
     // rows are gathered into one lane so that the additions go out as 16-byte vector reductions
-    float* dl = p.delta + (size_t)l * H;
+    float* dl = p.delta + ((size_t)l * DX_STACK_COPIES + (cta % DX_STACK_COPIES)) * H;
     constexpr int NV = 4 * PW;   // (tile, half) values of this warp
 #pragma unroll
     for (int v0 = 0; v0 < NV; v0 += 16) {

@@ -167,13 +167,17 @@ struct DxStackLayer {
   int pad;
 };
 // ... and the launch parameters
+// Partial sums a layer's contributions to the hidden row are spread over (CTA c adds into copy c mod this): every
+// word of a single row would take one addition from every CTA, and additions to one address are carried out one
+// after the other in L2 -- with 148 CTAs the last CTA's release waited 2.5 us for them.
+#define DX_STACK_COPIES 4
 struct DxStackParams {
   const DxStackLayer* layers;
   int n_layers;
   const float* h_in;          // [H]
   float* h_out;               // [H]
   // all zero at launch:
-  float* delta;               // [n_layers][H] what layer l adds to the hidden row
+  float* delta;               // [n_layers][DX_STACK_COPIES][H] what layer l adds to the hidden row, in partial sums
   unsigned long long* zword;  // [n_layers][E] router logits exchanged between the CTAs, (1 << 32 | float bits)
   unsigned int* sync;         // [n_layers] CTAs that have added all of their share of layer l
   int32_t* topk_ids;          // [n_layers][k] or null
