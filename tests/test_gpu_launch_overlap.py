@@ -1,0 +1,83 @@
+"""Every setting of the launch-overlap mask (dx_set_launch_overlap: which kernels are launched with programmatic
+stream serialization) gives the same results: the mask moves launches in time, never what they compute.  The default
+(routing + expert kernels) is what all other tests run; here the verify block, the draft step, the residual chain and
+the greedy accept are compared with the CPU checker under no overlap at all, each kernel kind alone, and all three."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import moe_oracle as O
+from paper_2607_24434_b200 import synth
+from tests.helpers import Y_BF16, gpu_layer, row_rel_err
+from tests.test_gpu_parity import SMALL, _accept_case, _draft_case, _verify_case
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", params=[0, 1, 2, 4, 7])
+def dxm(request):
+    from paper_2607_24434_b200 import binding
+    ctx = binding.Context(0)
+    ctx.set_launch_overlap(request.param)
+    ctx.y_tol = Y_BF16
+    yield binding, ctx
+    assert ctx.device_status() == 0
+    ctx.close()
+
+
+def test_refused_masks():
+    from paper_2607_24434_b200 import binding
+    ctx = binding.Context(0)
+    for bad in (-1, 8):
+        with pytest.raises(binding.DxError) as err:
+            ctx.set_launch_overlap(bad)
+        assert err.value.status == 1
+    ctx.close()
+
+
+def test_block_draft_and_accept_under_the_mask(dxm):
+    for K in (1, 4, 11):
+        _verify_case(dxm, SMALL, K, seed=300 + K, std=0.08)
+    _draft_case(dxm, SMALL, seed=310, std=0.08)
+    wide = dataclasses.replace(SMALL, weight_dtype=synth.DTYPE_BF16_WIDE)
+    _verify_case(dxm, wide, 9, seed=320, std=0.08)
+    _draft_case(dxm, wide, seed=321, std=0.08)
+    assert _accept_case(dxm, 5, 4, 4099, 256, torch.bfloat16, 330, rms=True, mode="mid") == 2
+
+
+def test_back_to_back_steps_under_the_mask(dxm):
+    """Draft step -> verify block -> accept, three times in a row on one stream without a host wait in between (the
+    arrangement in which the overlap matters), on a DeepSeek-V2-Lite-shaped layer; every result against the checker."""
+    binding, ctx = dxm
+    shape = synth.shape_v2lite()
+    layer, ref = gpu_layer(shape, 340, zipf=True)
+    L = binding.Layer.from_weights(ctx, layer)
+    V, K = 4099, 4
+    W = synth.lm_head(V, shape.hidden, 341, torch.bfloat16, "cuda")
+    W_np = synth.to_numpy_f32(W).astype(np.float64)
+    blocks = [synth.hidden_block(K, shape.hidden, 342 + i, 0.5, "cuda") for i in range(3)]
+    draft = torch.zeros((K,), dtype=torch.int32, device="cuda")
+    outs = []
+    for h in blocks:
+        d = binding.moe_draft_step(L, h[:1])
+        v = binding.moe_verify_block_residual(L, h)
+        a = binding.spec_accept(ctx, v["h"], W, draft, rms_norm=True)
+        outs.append((d, v, a))
+    torch.cuda.synchronize()
+    assert ctx.device_status() == 0
+    for h, (d, v, a) in zip(blocks, outs):
+        h_np = h.cpu().numpy().astype(np.float64)
+        y_d = O.moe_draft(h_np[:1], ref, forced_ids=d["topk_ids"].cpu().numpy()[None])[0]
+        assert row_rel_err(d["y"].cpu().numpy(), y_d).max() <= Y_BF16
+        want = O.stack_layer_target(h_np, ref, forced_ids=v["topk_ids"].cpu().numpy())[0]
+        assert row_rel_err(v["h"].cpu().numpy(), want).max() <= Y_BF16
+        hn = O.rmsnorm(v["h"].cpu().numpy().astype(np.float64))
+        t_ref, n_ref, next_ref, lg = O.greedy_accept_fast(hn, W_np, draft.cpu().numpy())
+        srt = np.sort(lg, axis=1)
+        clear = (srt[:, -1] - srt[:, -2]) > 1e-3
+        assert np.array_equal(a["target"].cpu().numpy()[clear], t_ref[clear])
+        if clear.all():
+            assert int(a["n_accept"].item()) == n_ref and int(a["next_token"].item()) == next_ref
+    L.close()
