@@ -141,6 +141,8 @@ def run_gpu(args):
     ctx = binding.Context(local)
     if args.launch_overlap is not None:
         ctx.set_launch_overlap(args.launch_overlap)
+    if args.accept_l2_mb is not None:
+        ctx.set_accept_l2_keep(int(args.accept_l2_mb * 1e6))
     layers, blocks, W_lm = build_workload(binding, ctx, shape, NL, K, V, 1000 + 50 * rank, device, args.q4_resident)
     H = shape.hidden
     stream = torch.cuda.current_stream()
@@ -956,6 +958,8 @@ def main():
     ap.add_argument("--no-k8", action="store_true", help="skip the K = 8 figures of the dominant kernel")
     ap.add_argument("--launch-overlap", type=int, default=None,
                     help="dx_set_launch_overlap mask (bit 0 routing, 1 experts, 2 greedy accept; library default 3)")
+    ap.add_argument("--accept-l2-mb", type=float, default=None,
+                    help="dx_set_accept_l2_keep: MB at the head of the LM head kept in L2 between steps (library default 0)")
     ap.add_argument("--wide", action="store_true",
                     help="layer / stack workloads: experts in the wide blob layout (tcgen05 kernel, any block length)")
     ap.add_argument("--no-cpu-baseline", action="store_true")

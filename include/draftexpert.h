@@ -131,6 +131,11 @@ dx_status dx_set_launch_overlap(dx_ctx* ctx, int32_t mask);
  * lets the kernel run to its end; the outputs of that call are then undefined, the context stays usable.  Default
  * 2^22 polls (seconds); 0 restores it. */
 dx_status dx_set_wait_limit(dx_ctx* ctx, uint32_t polls);
+/* spec_accept / spec_draft_token with a bf16 head: the leading `bytes` of W_lm are read with an L2 evict-last hint and
+ * the rest with evict-first, so that the head of the matrix (the same in every decode step, and larger than L2 as a
+ * whole) is still in L2 at the next call and only the rest comes from HBM again.  0 (the default) reads the whole
+ * matrix as a plain stream.  Results do not depend on it. */
+dx_status dx_set_accept_l2_keep(dx_ctx* ctx, size_t bytes);
 /* Exercises that give-up path without a fault: clears the hand-over words and launches the expert half of a verify
  * block alone, as if the routing kernel it expects beside it never ran.  The kernel's waits run out, it returns, and
  * dx_last_device_status reads DX_DEV_WAIT_EXPIRED; y is undefined afterwards.  Refused (DX_ERR_INVALID_ARG) unless the

@@ -54,6 +54,7 @@ SIGNATURES = {
     "dx_set_activation_split": (_I, [_P, _I]),
     "dx_set_launch_overlap": (_I, [_P, _I]),
     "dx_set_wait_limit": (_I, [_P, C.c_uint32]),
+    "dx_set_accept_l2_keep": (_I, [_P, C.c_size_t]),
     "dx_selftest_wait_expiry": (_I, [_P, _P, _I, _P, _P]),
     "dx_last_cuda_error": (_I, [_P]),
     "dx_kernel_launches": (C.c_int64, [_P]),
@@ -166,6 +167,10 @@ class Context:
 
     def set_wait_limit(self, polls: int) -> None:
         _check(self.lib.dx_set_wait_limit(self.handle, polls), "dx_set_wait_limit")
+
+    def set_accept_l2_keep(self, nbytes: int) -> None:
+        """Leading bytes of a bf16 LM head that spec_accept asks L2 to retain between calls (0: plain stream)."""
+        _check(self.lib.dx_set_accept_l2_keep(self.handle, nbytes), "dx_set_accept_l2_keep")
 
     def close(self) -> None:
         if self.handle:

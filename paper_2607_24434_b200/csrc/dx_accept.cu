@@ -27,6 +27,13 @@ __device__ __forceinline__ uint4 ldg_stream(const void* p) {
                : "l"(p));
   return r;
 }
+__device__ __forceinline__ uint4 ldg_hint(const void* p, uint64_t pol) {
+  uint4 r;
+  asm volatile("ld.global.nc.L1::no_allocate.L2::cache_hint.L2::256B.v4.u32 {%0,%1,%2,%3}, [%4], %5;"
+               : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
+               : "l"(p), "l"(pol));
+  return r;
+}
 __device__ __forceinline__ void mma_k16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                         uint32_t b0, uint32_t b1) {
   asm volatile(
@@ -60,6 +67,7 @@ struct AcceptParams {
   unsigned int* ticket;
   float* conf;          // [M] softmax probability of the argmax (only the CONF variants)
   float2* conf_part;    // [grid][DX_MAX_M] per-CTA (running max, sum of exp) pairs
+  int keep_tiles;       // 16-row tiles at the head of the matrix that L2 is asked to retain from call to call
   int32_t* dev_status;  // the context's status word (null for the context-free entry point)
 };
 
@@ -182,7 +190,15 @@ __global__ void __launch_bounds__(512, 1) dx_accept_bf16_kernel(AcceptParams p) 
   // give the first CTAs one whole tile per warp more than the last ones.
   const int tiles_cta = gridDim.x;
   const __nv_bfloat16* Wb = reinterpret_cast<const __nv_bfloat16*>(p.W);
+  // The LM head is the same matrix in every decode step and larger than L2, so a plain stream leaves nothing of it
+  // behind.  The first keep_tiles tiles are read with an evict-last hint, everything else with evict-first: the
+  // head of the matrix stays in L2 between two calls (expert weights are streamed evict-first as well) and only the
+  // rest comes from HBM again.
+  uint64_t pol_keep, pol_stream;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_keep));
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_stream));
   for (int tile = blockIdx.x + tiles_cta * warp; tile < tiles; tile += tiles_cta * (int)(blockDim.x >> 5)) {
+    const uint64_t pol = tile < p.keep_tiles ? pol_keep : pol_stream;
     const int r0 = tile * 16 + g, r1 = r0 + 8;
     const __nv_bfloat16* w0 = Wb + (size_t)min(r0, p.V - 1) * H + 8 * c;
     const __nv_bfloat16* w1 = Wb + (size_t)min(r1, p.V - 1) * H + 8 * c;
@@ -193,8 +209,8 @@ __global__ void __launch_bounds__(512, 1) dx_accept_bf16_kernel(AcceptParams p) 
       for (int r = 0; r < 4; ++r) ch[nt][r] = cl[nt][r] = 0.f;
 #pragma unroll 16
     for (int q = 0; q < Q; ++q) {
-      const uint4 a0 = ldg_stream(w0 + 32 * q);
-      const uint4 a1 = ldg_stream(w1 + 32 * q);
+      const uint4 a0 = p.keep_tiles ? ldg_hint(w0 + 32 * q, pol) : ldg_stream(w0 + 32 * q);
+      const uint4 a1 = p.keep_tiles ? ldg_hint(w1 + 32 * q, pol) : ldg_stream(w1 + 32 * q);
 #pragma unroll
       for (int nt = 0; nt < NT; ++nt) {
         const uint4 bh = hiF[(nt * Q + q) * 32 + lane];
@@ -337,7 +353,8 @@ cudaError_t dx_launch_accept(dx_ctx* ctx, const float* h, int M, const void* W_l
                              const int32_t* draft, int K, int rms_norm, int32_t* target, int32_t* n_accept,
                              int32_t* next_token, float* conf, cudaStream_t st) {
   AcceptParams p{h, M, V, H, W_lm, draft, K, rms_norm, target, n_accept, next_token, ctx->keys, ctx->ticket + 1,
-                 conf, ctx->conf_part, ctx->dev_status};
+                 conf, ctx->conf_part, 0, ctx->dev_status};
+  if (w_dtype != DX_DTYPE_FP32) p.keep_tiles = (int)(ctx->accept_keep_bytes / ((size_t)16 * H * 2));
   if (w_dtype == DX_DTYPE_FP32) {
     int grid = (V + 7) / 8;
     if (grid > ctx->sm_count * 8) grid = ctx->sm_count * 8;
@@ -407,7 +424,7 @@ extern "C" dx_status spec_accept_noalloc(const float* h, int32_t M, const void* 
   if (cudaMemsetAsync(d.scratch, 0, sizeof(unsigned long long) * (kNoAllocMaxRows + 2), st) != cudaSuccess)
     return DX_ERR_CUDA;
   AcceptParams p{h, M, V, H, W_lm, draft, K, rms_norm, target, n_accept, next_token, d.scratch,
-                 reinterpret_cast<unsigned int*>(d.scratch + kNoAllocMaxRows), nullptr, nullptr, nullptr};
+                 reinterpret_cast<unsigned int*>(d.scratch + kNoAllocMaxRows), nullptr, nullptr, 0, nullptr};
   cudaError_t e;
   if (w_dtype == DX_DTYPE_FP32) {
     int grid = (V + 7) / 8;

@@ -43,6 +43,7 @@ extern "C" dx_status dx_create(int device, dx_ctx** out) {
   ctx->last_cuda = cudaSuccess;
   ctx->launches = 0;
   ctx->pdl_mask = DX_PDL_ROUTE | DX_PDL_EXPERTS;
+  ctx->accept_keep_bytes = 0;
   ctx->wait_limit = DX_WAIT_LIMIT_DEFAULT;
   cudaError_t e = cudaSetDevice(device);
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, device);
@@ -110,6 +111,12 @@ extern "C" dx_status dx_set_launch_overlap(dx_ctx* ctx, int32_t mask) {
 extern "C" dx_status dx_set_wait_limit(dx_ctx* ctx, uint32_t polls) {
   if (!ctx) return DX_ERR_INVALID_ARG;
   ctx->wait_limit = polls ? polls : DX_WAIT_LIMIT_DEFAULT;
+  return DX_OK;
+}
+
+extern "C" dx_status dx_set_accept_l2_keep(dx_ctx* ctx, size_t bytes) {
+  if (!ctx) return DX_ERR_INVALID_ARG;
+  ctx->accept_keep_bytes = bytes;
   return DX_OK;
 }
 

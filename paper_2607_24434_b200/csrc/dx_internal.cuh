@@ -69,6 +69,7 @@ struct dx_ctx {
   int act_split;              // 1: bf16 experts are evaluated with hi + residual activation fragments
   int pdl_mask;               // DX_PDL_* bits: kernels launched with programmatic stream serialization
   uint32_t wait_limit;        // polls after which a bounded wait inside a kernel gives up (dx_set_wait_limit)
+  size_t accept_keep_bytes;   // leading bytes of the LM head the accept kernel asks L2 to retain (dx_set_accept_l2_keep)
   cudaError_t last_cuda;
   int64_t launches;
   // device scratch

@@ -1,7 +1,9 @@
-"""Every setting of the launch-overlap mask (dx_set_launch_overlap: which kernels are launched with programmatic
-stream serialization) gives the same results: the mask moves launches in time, never what they compute.  The default
-(routing + expert kernels) is what all other tests run; here the verify block, the draft step, the residual chain and
-the greedy accept are compared with the CPU checker under no overlap at all, each kernel kind alone, and all three."""
+"""Context settings that move work in time or in the memory hierarchy, never what is computed.
+
+Every setting of the launch-overlap mask (dx_set_launch_overlap: which kernels are launched with programmatic stream
+serialization) gives the same results.  The default (routing + expert kernels) is what all other tests run; here the
+verify block, the draft step, the residual chain and the greedy accept are compared with the CPU checker under no
+overlap at all, each kernel kind alone, and all three.  Likewise dx_set_accept_l2_keep (cache hints of the LM head)."""
 import dataclasses
 
 import numpy as np
@@ -81,3 +83,19 @@ def test_back_to_back_steps_under_the_mask(dxm):
         if clear.all():
             assert int(a["n_accept"].item()) == n_ref and int(a["next_token"].item()) == next_ref
     L.close()
+
+
+@pytest.mark.parametrize("keep_bytes", [1 << 20, 5 << 20, 1 << 30])
+def test_accept_with_part_of_the_head_kept_in_l2(keep_bytes):
+    """dx_set_accept_l2_keep only changes the cache hints of the loads: part of the matrix, a boundary inside it, and
+    more than the whole matrix give the checker's tokens, repeatedly (the second and third calls are the ones that
+    find lines in L2)."""
+    from paper_2607_24434_b200 import binding
+    ctx = binding.Context(0)
+    ctx.set_accept_l2_keep(keep_bytes)
+    ctx.y_tol = Y_BF16
+    for rep in range(3):
+        assert _accept_case((binding, ctx), 9, 8, 3001, 1024, torch.bfloat16, 350, rms=True, mode="mid") == 4
+    _accept_case((binding, ctx), 4, 4, 4099, 256, torch.bfloat16, 351, mode="geometric")
+    assert ctx.device_status() == 0
+    ctx.close()
