@@ -136,6 +136,13 @@ dx_status dx_set_wait_limit(dx_ctx* ctx, uint32_t polls);
  * whole) is still in L2 at the next call and only the rest comes from HBM again.  0 (the default) reads the whole
  * matrix as a plain stream.  Results do not depend on it. */
 dx_status dx_set_accept_l2_keep(dx_ctx* ctx, size_t bytes);
+/* Host -> device transfer of a step's inputs (a block of hidden rows, draft tokens): dst (device, any alignment) <-
+ * src_host (page-locked host memory; DX_ERR_INVALID_ARG otherwise), in stream order.  Up to 1 MB with both addresses
+ * 16-byte aligned is moved by a kernel that reads the host buffer through its device mapping (no copy-engine set-up;
+ * the host may rewrite the buffer once the call's work has completed); anything else goes through cudaMemcpyAsync.
+ * The result pointers of spec_accept / spec_draft_token may point into page-locked host memory as well: the kernel
+ * then writes the few result words straight to the host and no device -> host copy is needed. */
+dx_status dx_stage_block(dx_ctx* ctx, void* dst, const void* src_host, size_t bytes, void* stream);
 /* Exercises that give-up path without a fault: clears the hand-over words and launches the expert half of a verify
  * block alone, as if the routing kernel it expects beside it never ran.  The kernel's waits run out, it returns, and
  * dx_last_device_status reads DX_DEV_WAIT_EXPIRED; y is undefined afterwards.  Refused (DX_ERR_INVALID_ARG) unless the

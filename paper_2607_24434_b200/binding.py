@@ -55,6 +55,7 @@ SIGNATURES = {
     "dx_set_launch_overlap": (_I, [_P, _I]),
     "dx_set_wait_limit": (_I, [_P, C.c_uint32]),
     "dx_set_accept_l2_keep": (_I, [_P, C.c_size_t]),
+    "dx_stage_block": (_I, [_P, _P, _P, C.c_size_t, _P]),
     "dx_selftest_wait_expiry": (_I, [_P, _P, _I, _P, _P]),
     "dx_last_cuda_error": (_I, [_P]),
     "dx_kernel_launches": (C.c_int64, [_P]),
@@ -429,6 +430,14 @@ def moe_verify_block_residual(layer: Layer, h_in: torch.Tensor, h_out: Optional[
                                                _stream()), "moe_verify_block_residual")
     out["h"] = h_out
     return out
+
+
+def stage_block(ctx: Context, dst: torch.Tensor, src_pinned: torch.Tensor) -> None:
+    """dst (device) <- src_pinned (page-locked host tensor of the same byte size), in stream order."""
+    nbytes = src_pinned.numel() * src_pinned.element_size()
+    if nbytes != dst.numel() * dst.element_size():
+        raise ValueError("stage_block: sizes differ")
+    _check(ctx.lib.dx_stage_block(ctx.handle, _ptr(dst), _ptr(src_pinned), nbytes, _stream()), "dx_stage_block")
 
 
 def spec_accept(ctx: Context, h: torch.Tensor, W_lm: torch.Tensor, draft: torch.Tensor, rms_norm: bool = False,

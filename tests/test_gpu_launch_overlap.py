@@ -99,3 +99,43 @@ def test_accept_with_part_of_the_head_kept_in_l2(keep_bytes):
     _accept_case((binding, ctx), 4, 4, 4099, 256, torch.bfloat16, 351, mode="geometric")
     assert ctx.device_status() == 0
     ctx.close()
+
+
+def test_stage_block_and_results_written_to_the_host():
+    """dx_stage_block moves pinned host bytes to the device (kernel path for small aligned sizes, copy engine
+    otherwise, a page-able source refused), and the accept kernel may write its result words straight into pinned
+    host memory: same tokens as with device outputs."""
+    from paper_2607_24434_b200 import binding
+    ctx = binding.Context(0)
+    for nbytes, offset in [(16, 0), (4 * 2048 * 4 + 16, 0), (1000, 0), (37, 0), (4096, 8), (3 << 20, 0)]:
+        host = torch.empty((nbytes + offset,), dtype=torch.uint8).pin_memory()
+        host.copy_(torch.randint(0, 256, (nbytes + offset,), dtype=torch.uint8))
+        dst = torch.zeros((nbytes + 64,), dtype=torch.uint8, device="cuda")
+        binding.stage_block(ctx, dst[:nbytes], host[offset:])
+        torch.cuda.synchronize()
+        assert torch.equal(dst[:nbytes].cpu(), host[offset:]) and int(dst[nbytes:].sum().item()) == 0, (nbytes, offset)
+        # the host rewrites the buffer: the next transfer sees the new bytes
+        host.add_(1)
+        binding.stage_block(ctx, dst[:nbytes], host[offset:])
+        torch.cuda.synchronize()
+        assert torch.equal(dst[:nbytes].cpu(), host[offset:])
+    with pytest.raises(binding.DxError) as err:
+        binding.stage_block(ctx, torch.zeros((64,), dtype=torch.uint8, device="cuda"), torch.zeros((64,), dtype=torch.uint8))
+    assert err.value.status == 1
+    # greedy accept with its three outputs in pinned host memory
+    M, K, V, H = 5, 4, 4099, 512
+    W = synth.lm_head(V, H, 360, torch.bfloat16, "cuda")
+    h = synth.hidden_block(M, H, 361, 0.5, "cuda")
+    dev = binding.spec_accept(ctx, h, W, torch.zeros((K,), dtype=torch.int32, device="cuda"), rms_norm=True)
+    torch.cuda.synchronize()
+    draft = dev["target"][:K].clone()
+    draft[2] = (draft[2] + 1) % V
+    dev = binding.spec_accept(ctx, h, W, draft, rms_norm=True)
+    res = torch.full((M + 2,), -7, dtype=torch.int32).pin_memory()
+    out = {"target": res[:M], "n_accept": res[M:M + 1], "next_token": res[M + 1:M + 2]}
+    binding.spec_accept(ctx, h, W, draft, rms_norm=True, out=out)
+    torch.cuda.synchronize()
+    assert torch.equal(res[:M], dev["target"].cpu())
+    assert int(res[M]) == int(dev["n_accept"].item()) == 2 and int(res[M + 1]) == int(dev["next_token"].item())
+    assert ctx.device_status() == 0
+    ctx.close()
