@@ -127,6 +127,9 @@ namespace {
 __global__ void dx_stage_block_kernel(uint4* dst, const uint4* src, size_t n16, unsigned char* dst_tail,
                                       const unsigned char* src_tail, int n_tail) {
   const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  // a routing kernel behind this one may become resident and fetch its router rows while the link is read; it waits
+  // for this grid's completion before it touches the block
+  dx_pdl_trigger();
   if (i < n16) {
     uint4 v;   // (a volatile load: the host rewrites the buffer between two calls, nothing may be served from a cache)
     asm volatile("ld.volatile.global.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(src + i));
