@@ -27,6 +27,7 @@ struct DxSlot {
   unsigned long long stamp = 0;
   bool prefetched = false;   // member of P: prefetched this step, not used yet
   bool copy_pending = false; // a copy was issued and not yet seen complete
+  bool ev_valid = false;     // the event has been recorded at least once
   cudaEvent_t ev = nullptr;
 };
 
@@ -42,11 +43,13 @@ struct dx_cache {
   size_t blob_bytes;
   unsigned char* slab;
   // quantised host pool: registered blobs are 4-bit block-quantised (q4_bytes each); a copy lands in the slot's
-  // staging area and is expanded into the slot on the copy stream
+  // staging area and is expanded into the slot on a stream of its own, so that the link goes on with the next copy
   size_t q4_bytes;
   int q4_hidden, q4_inter;
   unsigned char* staging;
   cudaStream_t copy_stream;
+  cudaStream_t expand_stream;           // (quantised pool) staging area -> slot
+  cudaEvent_t staged_ev;                // (quantised pool) the copy in front of an expansion has landed
   unsigned long long clock;
   dx_cache_stats stats;
   std::vector<const void*> host_blob;   // [L*E]
@@ -118,13 +121,24 @@ dx_status load_into(dx_cache* c, int layer, int s, int e, bool as_prefetch) {
     }
     cudaError_t e1;
     if (c->q4_bytes) {
-      // a quarter of the bytes cross the host link; the expansion to the streaming layout runs at HBM speed
-      e1 = cudaMemcpyAsync(staging_ptr(c, layer, s), c->host_blob[(size_t)layer * c->E + e], c->q4_bytes,
-                           cudaMemcpyHostToDevice, c->copy_stream);
+      // a quarter of the bytes cross the host link; the expansion to the streaming layout runs at HBM speed, behind
+      // the copy but on the expansion stream (the staging area of a slot is overwritten by the copy stream only
+      // after the slot's previous expansion, which the slot's event marks, has run)
+      e1 = sl.ev_valid ? cudaStreamWaitEvent(c->copy_stream, sl.ev, 0) : cudaSuccess;
+      if (e1 == cudaSuccess)
+        e1 = cudaMemcpyAsync(staging_ptr(c, layer, s), c->host_blob[(size_t)layer * c->E + e], c->q4_bytes,
+                             cudaMemcpyHostToDevice, c->copy_stream);
+      if (e1 == cudaSuccess) e1 = cudaEventRecord(c->staged_ev, c->copy_stream);
+      if (e1 == cudaSuccess) e1 = cudaStreamWaitEvent(c->expand_stream, c->staged_ev, 0);
       if (e1 == cudaSuccess)
         e1 = dx_launch_expand_q4(c->q4_hidden, c->q4_inter, staging_ptr(c, layer, s), slot_ptr(c, layer, s),
-                                 c->copy_stream);
+                                 c->expand_stream);
       if (e1 == cudaSuccess) c->ctx->launches++;
+      if (e1 == cudaSuccess) e1 = cudaEventRecord(sl.ev, c->expand_stream);
+      if (e1 != cudaSuccess) { c->ctx->last_cuda = e1; return DX_ERR_CUDA; }
+      sl.ev_valid = true;
+      sl.copy_pending = true;
+      return DX_OK;
     } else {
       e1 = cudaMemcpyAsync(slot_ptr(c, layer, s), c->host_blob[(size_t)layer * c->E + e], c->blob_bytes,
                            cudaMemcpyHostToDevice, c->copy_stream);
@@ -227,6 +241,8 @@ extern "C" dx_status expert_cache_create(dx_ctx* ctx, int32_t n_layers, int32_t 
   c->q4_hidden = c->q4_inter = 0;
   c->staging = nullptr;
   c->copy_stream = nullptr;
+  c->expand_stream = nullptr;
+  c->staged_ev = nullptr;
   c->clock = 0;
   c->stats = dx_cache_stats{};
   c->host_blob.assign((size_t)n_layers * n_experts, nullptr);
@@ -240,6 +256,8 @@ extern "C" dx_status expert_cache_create(dx_ctx* ctx, int32_t n_layers, int32_t 
     cudaError_t e = cudaSetDevice(ctx->device);
     if (e == cudaSuccess) e = cudaMalloc(&c->slab, (size_t)n_layers * slots_per_layer * blob_bytes);
     if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&c->expand_stream, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->staged_ev, cudaEventDisableTiming);
     for (size_t i = 0; e == cudaSuccess && i < c->slots.size(); ++i)
       e = cudaEventCreateWithFlags(&c->slots[i].ev, cudaEventDisableTiming);
     for (int l = 0; e == cudaSuccess && l < n_layers; ++l)
@@ -258,6 +276,9 @@ extern "C" dx_status expert_cache_destroy(dx_cache* c) {
   if (!c) return DX_ERR_INVALID_ARG;
   if (c->ctx) {
     if (c->copy_stream) cudaStreamSynchronize(c->copy_stream);
+    if (c->expand_stream) cudaStreamSynchronize(c->expand_stream);
+    if (c->staged_ev) cudaEventDestroy(c->staged_ev);
+    if (c->expand_stream) cudaStreamDestroy(c->expand_stream);
     for (auto& s : c->slots)
       if (s.ev) cudaEventDestroy(s.ev);
     for (auto& e : c->used_ev)

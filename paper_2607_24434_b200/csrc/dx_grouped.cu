@@ -786,41 +786,71 @@ __global__ void dx_pack_bf16_kernel(const __nv_bfloat16* Wg, const __nv_bfloat16
 // 4-bit block-quantised expert (three matrices of 18-byte blocks: fp16 scale, then 16 bytes of codes, low nibbles
 // = weights 0..15 of the block, high nibbles = weights 16..31; weight = scale * (code - 8)) expanded straight
 // into the bf16 streaming blob above, each value rounded to bf16 once.
-__device__ __forceinline__ __nv_bfloat16 q4_value(const unsigned char* mat, int row, int col, int cols) {
-  const unsigned char* blk = mat + ((size_t)row * (cols / 32) + col / 32) * 18;
-  const float d = __half2float(__ushort_as_half((unsigned short)(blk[0] | (blk[1] << 8))));
-  const int j = col & 31;
-  const int code = j < 16 ? (blk[2 + j] & 0x0F) : (blk[2 + j - 16] >> 4);
-  return __float2bfloat16_rn(d * (float)(code - 8));
-}
 
+// One thread writes one 16-byte fragment (eight values): the expansion sits between a host -> device copy and the
+// first use of a cache slot, once per loaded expert, and an element-by-element version (index arithmetic and three
+// byte loads per value) took as long as the copy itself.
+//   first product: the fragment of lane (g, c), step s holds columns 16 s + 4 c .. + 3 of gate row 8 j + g and of up
+//   row 8 j + g, as (g0 g1 u0 u1 g2 g3 u2 u3): four consecutive codes of one quantisation block per matrix;
+//   second product: rows 32 q + g, + 8, + 16, + 24 of W_d at columns 8 j + 2 c, + 1: two consecutive codes of four
+//   blocks.
+__device__ __forceinline__ float q4_scale(const unsigned char* blk) {
+  return __half2float(__ushort_as_half(*reinterpret_cast<const unsigned short*>(blk)));   // (blocks are 18 bytes: 2-byte aligned)
+}
+__device__ __forceinline__ uint32_t bf16_pair(float lo, float hi) {
+  return (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(lo)) | ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(hi)) << 16);
+}
 __global__ void dx_expand_q4_kernel(const unsigned char* q4, __nv_bfloat16* blob, int H, int I) {
-  const size_t n = (size_t)3 * H * I;
   const int KW = H / 128, PW = H / 256;
   const size_t mat_gu = (size_t)I * (H / 32) * 18;   // bytes of W_g (and of W_u)
   const unsigned char* Wg = q4;
   const unsigned char* Wu = q4 + mat_gu;
   const unsigned char* Wd = q4 + 2 * mat_gu;
+  const int per_unit = 3 * H, per_chunk = 3 * H / 8, p1 = H / 4;   // 16-byte fragments per unit / per chunk / of the first product
+  const size_t n = (size_t)(I / 8) * per_unit;
+  uint4* out = reinterpret_cast<uint4*>(blob);
   for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < n; idx += (size_t)gridDim.x * blockDim.x) {
-    const int j = (int)(idx / (24 * (size_t)H));
-    const int r = (int)(idx % (24 * (size_t)H));
-    const int w = r / (3 * H), rr = r % (3 * H);
-    __nv_bfloat16 v;
-    if (rr < 2 * H) {
-      const int i = rr / 256, l = (rr % 256) / 8, el = rr % 8;
-      const int s = w * KW + i, g = l >> 2, c = l & 3;
-      const int col = 16 * s + 4 * c + (el & 1) + ((el >> 2) << 1);
-      const int row = 8 * j + g;
-      v = q4_value(((el >> 1) & 1) ? Wu : Wg, row, col, H);
+    const int j = (int)(idx / per_unit);
+    const int u4 = (int)(idx - (size_t)j * per_unit);
+    const int w = u4 / per_chunk, r4 = u4 - w * per_chunk;
+    uint4 v;
+    if (r4 < p1) {
+      const int i = r4 >> 5, l = r4 & 31, g = l >> 2, c = l & 3;
+      const int col0 = 16 * (w * KW + i) + 4 * c, row = 8 * j + g;
+      const size_t off = ((size_t)row * (H / 32) + col0 / 32) * 18;
+      const int jj = col0 & 31, sh = (jj & 16) ? 4 : 0;
+      float gv[4], uv[4];
+#pragma unroll
+      for (int m = 0; m < 2; ++m) {
+        const unsigned char* blk = (m ? Wu : Wg) + off;
+        const float d = q4_scale(blk);
+        // four consecutive code bytes, 2-byte aligned
+        const unsigned short b01 = *reinterpret_cast<const unsigned short*>(blk + 2 + (jj & 15));
+        const unsigned short b23 = *reinterpret_cast<const unsigned short*>(blk + 4 + (jj & 15));
+        float* dst = m ? uv : gv;
+        dst[0] = d * (float)((int)((b01 >> sh) & 0xF) - 8);
+        dst[1] = d * (float)((int)((b01 >> (8 + sh)) & 0xF) - 8);
+        dst[2] = d * (float)((int)((b23 >> sh) & 0xF) - 8);
+        dst[3] = d * (float)((int)((b23 >> (8 + sh)) & 0xF) - 8);
+      }
+      v = make_uint4(bf16_pair(gv[0], gv[1]), bf16_pair(uv[0], uv[1]), bf16_pair(gv[2], gv[3]), bf16_pair(uv[2], uv[3]));
     } else {
-      const int r2 = rr - 2 * H;
-      const int i = r2 / 256, l = (r2 % 256) / 8, el = r2 % 8;
-      const int q = w * PW + i, g = l >> 2, c = l & 3;
-      const int row = 32 * q + 8 * (el >> 1) + g;
-      const int col = 8 * j + 2 * c + (el & 1);
-      v = q4_value(Wd, row, col, I);
+      const int r2 = r4 - p1;
+      const int i = r2 >> 5, l = r2 & 31, g = l >> 2, c = l & 3;
+      const int q = w * PW + i, col = 8 * j + 2 * c;
+      const int jj = col & 31, sh = (jj & 16) ? 4 : 0;
+      uint32_t o[4];
+#pragma unroll
+      for (int m = 0; m < 4; ++m) {
+        const int row = 32 * q + 8 * m + g;
+        const unsigned char* blk = Wd + ((size_t)row * (I / 32) + col / 32) * 18;
+        const float d = q4_scale(blk);
+        const unsigned short b01 = *reinterpret_cast<const unsigned short*>(blk + 2 + (jj & 15));
+        o[m] = bf16_pair(d * (float)((int)((b01 >> sh) & 0xF) - 8), d * (float)((int)((b01 >> (8 + sh)) & 0xF) - 8));
+      }
+      v = make_uint4(o[0], o[1], o[2], o[3]);
     }
-    blob[idx] = v;
+    out[idx] = v;
   }
 }
 
@@ -986,9 +1016,9 @@ cudaError_t dx_launch_pack_q4(int H, int I, const void* Wg, const void* Wu, cons
 }
 
 cudaError_t dx_launch_expand_q4(int H, int I, const void* q4, void* blob, cudaStream_t st) {
-  const size_t n = (size_t)3 * H * I;
+  const size_t n = (size_t)3 * H * I / 8;   // 16-byte fragments
   int grid = (int)((n + 255) / 256);
-  if (grid > 4096) grid = 4096;
+  if (grid > 8192) grid = 8192;
   dx_expand_q4_kernel<<<grid, 256, 0, st>>>((const unsigned char*)q4, (__nv_bfloat16*)blob, H, I);
   return cudaGetLastError();
 }
