@@ -58,7 +58,8 @@ extern "C" dx_status dx_create(int device, dx_ctx** out) {
   if (e == cudaSuccess) e = cudaMalloc(&ctx->scratch_i32, sizeof(int32_t) * 2);
   if (e == cudaSuccess) e = cudaMalloc(&ctx->union_dev, sizeof(int32_t) * (DX_MAX_E + 1 + DX_MAX_TOPK));
   if (e == cudaSuccess) e = cudaHostAlloc((void**)&ctx->union_host, sizeof(int32_t) * (DX_MAX_E + 1 + DX_MAX_TOPK),
-                                          cudaHostAllocDefault);
+                                          cudaHostAllocMapped);
+  if (e == cudaSuccess) e = cudaHostGetDevicePointer((void**)&ctx->union_host_dev, ctx->union_host, 0);
   if (e == cudaSuccess) e = cudaMemset(ctx->work, 0, sizeof(DxWork));
   if (e == cudaSuccess) e = cudaMemset(ctx->ticket, 0, sizeof(unsigned int) * 4);
   if (e == cudaSuccess) e = cudaMemset(ctx->keys, 0, sizeof(unsigned long long) * DX_MAX_M);
@@ -330,7 +331,7 @@ struct RouteOut {
 
 static dx_status do_route(dx_layer* L, const float* h, int K, float* y, const RouteOut& o, bool draft, bool residual,
                           cudaStream_t st, int top_r = 1, bool use_draft_expert = true, bool paired = false,
-                          bool skip_top1 = false) {
+                          bool skip_top1 = false, bool mirror_to_host = false) {
   dx_ctx* ctx = L->ctx;
   const dx_layer_desc& d = L->desc;
   if (!h || !y || h == y) return DX_ERR_INVALID_ARG;
@@ -361,6 +362,7 @@ static dx_status do_route(dx_layer* L, const float* h, int K, float* y, const Ro
   p.topk_ids = o.topk_ids; p.topk_w = o.topk_w;
   p.union_mask = (unsigned long long*)o.union_mask; p.union_ids = o.union_ids; p.union_count = o.union_count;
   p.offsets = o.offsets; p.perm = o.perm;
+  p.host_mirror = mirror_to_host ? ctx->union_host_dev : nullptr;
   // (the router of a layer with 4-bit experts, or with experts in the wide layout, is bf16)
   DX_CUDA(ctx, dx_launch_route(ctx, p, d.weight_dtype == DX_DTYPE_FP32 ? DX_DTYPE_FP32 : DX_DTYPE_BF16, st));
   ctx->launches++;
@@ -508,10 +510,10 @@ extern "C" dx_status moe_verify_block_residual(dx_layer* L, const float* h_in, f
 int dx_cache_slot_of(const dx_cache* c, int layer, int expert);
 int dx_cache_slots(const dx_cache* c);
 
-// Device -> pinned host copy of `n` ints behind the routing kernel, then a host wait: the one round trip
-// on-demand loading needs (the routing decision is made on the device, the copies are issued by the host).
-static dx_status read_back(dx_ctx* ctx, const int32_t* dev, int n, int32_t* host_pinned, cudaStream_t st) {
-  DX_CUDA(ctx, cudaMemcpyAsync(host_pinned, dev, sizeof(int32_t) * n, cudaMemcpyDeviceToHost, st));
+// The one round trip on-demand loading needs (the routing decision is made on the device, the copies are issued by
+// the host): the routing kernel itself writes what the host needs into page-locked host memory (a device -> host copy
+// behind it costs ~10 us of copy-engine set-up for a few ten bytes), and the host waits for the stream.
+static dx_status wait_for_routing(dx_ctx* ctx, cudaStream_t st) {
   DX_CUDA(ctx, cudaStreamSynchronize(st));
   return DX_OK;
 }
@@ -531,11 +533,10 @@ extern "C" dx_status moe_verify_block_cached(dx_layer* L, const float* h, int32_
   int32_t* uid = union_ids ? union_ids : ctx->union_dev;
   int32_t* ucnt = union_count ? union_count : ctx->union_dev + DX_MAX_E;
   RouteOut o{topk_ids, topk_w, union_mask, uid, ucnt, offsets, perm};
-  dx_status s = do_route(L, h, K, y, o, false, residual != 0, st);
+  dx_status s = do_route(L, h, K, y, o, false, residual != 0, st, 1, true, false, false, true);
   if (s != DX_OK) return s;
   const int cap = E < K * L->desc.top_k ? E : K * L->desc.top_k;
-  DX_CUDA(ctx, cudaMemcpyAsync(ctx->union_host, uid, sizeof(int32_t) * cap, cudaMemcpyDeviceToHost, st));
-  s = read_back(ctx, ucnt, 1, ctx->union_host + DX_MAX_E, st);
+  s = wait_for_routing(ctx, st);
   if (s != DX_OK) return s;
   const int n = ctx->union_host[DX_MAX_E];
   if (n < 0 || n > cap) return DX_ERR_CUDA;
@@ -574,10 +575,10 @@ extern "C" dx_status moe_draft_step_cached(dx_layer* L, const float* h, float* y
   const int k = L->desc.top_k;
   int32_t* ids = topk_ids ? topk_ids : ctx->union_dev + DX_MAX_E + 1;
   RouteOut o{ids, topk_w, nullptr, nullptr, nullptr, nullptr, nullptr};
-  dx_status s = do_route(L, h, 1, y, o, true, residual != 0, st);
+  dx_status s = do_route(L, h, 1, y, o, true, residual != 0, st, 1, true, false, false, true);
   if (s != DX_OK) return s;
   int32_t* host = ctx->union_host + DX_MAX_E + 1;
-  s = read_back(ctx, ids, k, host, st);
+  s = wait_for_routing(ctx, st);
   if (s != DX_OK) return s;
   if (host_topk_ids)
     for (int j = 0; j < k; ++j) host_topk_ids[j] = host[j];

@@ -82,6 +82,7 @@ struct dx_ctx {
   int32_t* scratch_i32;        // two ints the draft-token entry point parks unused outputs in
   int32_t* union_dev;          // [DX_MAX_E] union ids, [1] union count, [DX_MAX_TOPK] draft selection: what the
   int32_t* union_host;         //   cached entry points read back (pinned host copy, same layout)
+  int32_t* union_host_dev;     //   ... and its device mapping, which the routing kernel writes
 };
 
 struct dx_cache;
@@ -127,6 +128,10 @@ struct DxRouteParams {
   int32_t* union_count;
   int32_t* offsets;
   int32_t* perm;
+  // not null: page-locked host memory (through its device mapping) that gets a copy of what the host needs to go on
+  // after this kernel -- [0, DX_MAX_E) the union's expert ids, [DX_MAX_E] their count, [DX_MAX_E + 1, + k) the
+  // selection of block row 0 -- so that no device -> host copy has to follow the kernel
+  int32_t* host_mirror;
 };
 
 struct DxExpertParams {

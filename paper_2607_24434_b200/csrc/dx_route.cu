@@ -161,6 +161,7 @@ __device__ __forceinline__ void topk_select(const DxRouteParams& p, const float*
     if (!(p.skip_top1 && lane == 0))
       atomicOr(&s_mask[my_e >> 5], 1u << (my_e & 31));   // union of Eq. 2 / Eq. 3 as a bit mask
     if (p.topk_ids) p.topk_ids[tt * k + lane] = my_e;
+    if (p.host_mirror && tt == 0) p.host_mirror[DX_MAX_E + 1 + lane] = my_e;
   }
 }
 
@@ -631,10 +632,12 @@ __global__ void __launch_bounds__(kRouteThreads) dx_route_kernel(DxRouteParams p
       if (s_ids[q] == me && DX_BOUNDS(off + i < P, p.dev_status)) s_perm[off + i++] = q;
     if (p.offsets) p.offsets[me] = off;
     if (flag && p.union_ids && DX_BOUNDS(upos < min(E, P), p.dev_status)) p.union_ids[upos] = me;
+    if (flag && p.host_mirror && DX_BOUNDS(upos < min(E, P), p.dev_status)) p.host_mirror[upos] = me;
   }
   if (me == 0) {
     if (p.offsets) p.offsets[E] = P;
     if (p.union_count) *p.union_count = ucount;
+    if (p.host_mirror) p.host_mirror[DX_MAX_E] = ucount;
   }
   if (p.union_mask && me < (E + 63) / 64) {
     const unsigned long long lo = s_mask[2 * me], hi = (2 * me + 1 < DX_MAX_E / 32) ? s_mask[2 * me + 1] : 0u;
