@@ -748,7 +748,7 @@ def run_offload(args):
     torch.cuda.set_device(0)
     device = torch.device("cuda", 0)
     shape = synth.shape_v2lite()
-    NLAY, S, V, H = args.offload_layers, 16, args.vocab, shape.hidden
+    NLAY, S, V, H = args.offload_layers, args.slots, args.vocab, shape.hidden
     ctx = binding.Context(0)
     nbytes = binding.expert_blob_bytes(shape, shape.inter)
     pool_bytes = binding.q4_expert_bytes(shape, shape.inter) if args.q4 else nbytes
@@ -991,6 +991,7 @@ def main():
     ap.add_argument("--q4-resident", action="store_true",
                     help="layer workload: experts resident in HBM as 4-bit blocks, de-quantised in the expert kernel")
     ap.add_argument("--offload-steps", type=int, default=64)
+    ap.add_argument("--slots", type=int, default=16, help="offload workload: HBM cache slots per layer")
     ap.add_argument("--traffic", type=float, default=None,
                     help="ncu DRAM bytes per launch of the dominant kernel, if known")
     args = ap.parse_args()
