@@ -81,7 +81,7 @@ struct dx_ctx {
   float2* conf_part;           // [8 * sm_count][DX_MAX_M] per-CTA online-softmax pairs of the confidence variant
   int32_t* scratch_i32;        // two ints the draft-token entry point parks unused outputs in
   int32_t* union_dev;          // [DX_MAX_E] union ids, [1] union count, [DX_MAX_TOPK] draft selection: what the
-  int32_t* union_host;         //   cached entry points read back (pinned host copy, same layout)
+  int32_t* union_host;         //   cached entry points read on the host (page-locked and mapped; the routing kernel writes it)
   int32_t* union_host_dev;     //   ... and its device mapping, which the routing kernel writes
 };
 
