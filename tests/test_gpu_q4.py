@@ -93,9 +93,12 @@ def test_verify_block_from_quantised_host_pool():
         cache.register(0, e, host[e])
     cache.attach(off, 0)
     loads = 0
-    for step, K in enumerate([6, 3, 8]):
+    for step, K in enumerate([6, 3, 8, 5, 7]):
         h = synth.hidden_block(K, SHAPE.hidden, 85 + step, 0.5, "cuda")
         cache.begin_step()
+        if step >= 2:
+            # copies (and their expansions, on a stream of their own) still in flight when the block asks for them
+            cache.prefetch(0, [(3 * step + j) % E for j in range(3)])
         out = binding.moe_verify_block_cached(off, cache, 0, h)
         torch.cuda.synchronize()
         assert ctx.device_status() == 0
