@@ -361,6 +361,13 @@ def run_gpu(args):
         comp["draft_step_gbs"] = ((shape.n_shared + 2) * exp_bytes + shape.n_experts * H * 2) / (
             comp["draft_step_ms"] * 1e-3) / 1e9
         comp["accept_gbs"] = V * H * 2 / (comp["accept_ms"] * 1e-3) / 1e9
+        if args.accept_l2_mb is None:
+            # the same step with the head of the LM head kept in L2 from step to step (dx_set_accept_l2_keep, off by
+            # default and not part of the line's headline): reported beside it
+            ctx.set_accept_l2_keep(64 * 1000 * 1000)
+            graph_ms(step, reps=100)        # (what L2 holds settles over a few hundred steps)
+            comp["step_ms_with_64MB_of_lm_head_kept_in_l2"] = graph_ms(step, reps=100)
+            ctx.set_accept_l2_keep(0)
     draft_bytes = (shape.n_shared + 2) * exp_bytes + shape.n_experts * H * 2
     acc_bytes = V * H * 2
 
