@@ -793,7 +793,7 @@ def run_offload(args):
     emb = synth.embedding_table(V, H, 3998, device)
     W_lm = synth.lm_head(V, H, 3999, torch.bfloat16, device)
     dec = decode.OffloadedDecoder(ctx, layers, cache, emb, W_lm, k_max=args.k_max, tau=args.tau,
-                                  budget="cache" if args.budget < 0 else args.budget)
+                                  budget="cache" if args.budget < 0 else args.budget, native=not args.python_loop)
     rng = np.random.default_rng(11)
 
     def scripted():
@@ -999,6 +999,8 @@ def main():
                     help="layer workload: experts resident in HBM as 4-bit blocks, de-quantised in the expert kernel")
     ap.add_argument("--offload-steps", type=int, default=64)
     ap.add_argument("--slots", type=int, default=16, help="offload workload: HBM cache slots per layer")
+    ap.add_argument("--python-loop", action="store_true",
+                    help="offload workload: the decode step's host loop in Python (decode.py) instead of dx_decoder_step")
     ap.add_argument("--traffic", type=float, default=None,
                     help="ncu DRAM bytes per launch of the dominant kernel, if known")
     args = ap.parse_args()

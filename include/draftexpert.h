@@ -340,6 +340,30 @@ dx_status dx_controller_propose(dx_controller* c, const int32_t* predicted, int3
                                 int32_t budget, int32_t* delta_out, int32_t* stop_out, int32_t* new_layers_out,
                                 int32_t* new_experts_out, int32_t* n_new_out);
 
+/* ---- one decode step of Algorithm 1 over an offloaded stack, as a host loop inside the library -------------------
+ * dx_decoder_create: layers[l] must be attached to `cache` as cache layer l (bf16 layers of one shape; shared and
+ *   draft experts resident, routed experts registered with the cache).  emb [V,H] bf16 token embeddings (device,
+ *   16-byte aligned), W_lm [V,H] bf16 LM head (device); k_max <= 16 tokens drafted per step; tau and budget are the
+ *   threshold and the layer-expert budget B_i of Eq. 14 (budget < 0: what is left of the cache's n_layers * slots
+ *   pairs once the predictions accepted so far are counted).  Attention is not part of the path: a token's hidden
+ *   states depend on its own embedding alone.
+ * dx_decoder_step: from the last emitted token t0 -- draft candidates one by one through the drafter's stack (Eq. 5,
+ *   moe_draft_step_cached in the residual form; spec_draft_token on RMSNorm of the final row), apply the stop rule
+ *   (dx_controller_propose), prefetch the newly predicted experts (expert_cache_prefetch), verify the block through
+ *   the target stack (moe_verify_block_cached, residual form) and accept greedily (spec_accept on RMSNorm of the
+ *   final rows).  Exactly the calls, in the order, a caller of those entry points would make; the host waits for
+ *   `stream` after every routing decision and token.  HOST outputs: drafted [k_max] / n_drafted, n_accept (the
+ *   comparison's, or min(scripted_accept, n_drafted) if scripted_accept >= 0 -- for untrained draft experts),
+ *   emitted [k_max + 1] / n_emitted (d_1 .. d_n, then the target's token for position n + 1 if a row is left for it),
+ *   target [max(1, n_drafted)] (may be NULL), union_sizes [n_layers] (may be NULL). */
+typedef struct dx_decoder dx_decoder;
+dx_status dx_decoder_create(dx_ctx* ctx, dx_layer* const* layers, int32_t n_layers, dx_cache* cache, const void* emb,
+                            const void* W_lm, int32_t V, int32_t k_max, float tau, int32_t budget, dx_decoder** out);
+dx_status dx_decoder_destroy(dx_decoder* d);
+dx_status dx_decoder_step(dx_decoder* d, int32_t t0, int32_t scripted_accept, int32_t* drafted, int32_t* n_drafted,
+                          int32_t* n_accept, int32_t* emitted, int32_t* n_emitted, int32_t* target,
+                          int32_t* union_sizes, void* stream);
+
 /* ---- evaluation terms of the self-distillation section (Sec. 3.3); forward only, nothing is trained ---------
  * All pointers are device pointers; K block rows, 1 <= K <= 16; asynchronous on `stream`.
  *

@@ -94,6 +94,9 @@ SIGNATURES = {
     "dx_controller_size": (_I, [_P, C.POINTER(_I)]),
     "dx_controller_propose": (_I, [_P, _P, _I, C.c_float, C.c_float, _I, C.POINTER(_I), C.POINTER(_I), _P, _P,
                                    C.POINTER(_I)]),
+    "dx_decoder_create": (_I, [_P, _P, _I, _P, _P, _P, _I, _I, C.c_float, _I, C.POINTER(_P)]),
+    "dx_decoder_destroy": (_I, [_P]),
+    "dx_decoder_step": (_I, [_P, _I, _I, _P, C.POINTER(_I), C.POINTER(_I), _P, C.POINTER(_I), _P, _P, _P]),
     "spec_accept_noalloc": (_I, [_P, _I, _P, _I, _I, _I, _P, _I, _I, _P, _P, _P, _P]),
     "moe_missing_residual": (_I, [_P, _P, _I, _P, _P, _P, _P]),
     "moe_draft_expert_term": (_I, [_P, _P, _I, _P, _P]),
@@ -678,6 +681,52 @@ def squared_error(ctx: Context, a: torch.Tensor, b: torch.Tensor) -> torch.Tenso
     out = torch.empty((1,), dtype=torch.float32, device=a.device)
     _check(ctx.lib.dx_squared_error(ctx.handle, _ptr(a), _ptr(b), a.numel(), _ptr(out), _stream()), "dx_squared_error")
     return out
+
+
+class Decoder:
+    """One decode step of Algorithm 1 over an offloaded stack as a host loop inside the library (``dx_decoder_step``).
+    ``layers[l]`` must be attached to ``cache`` as cache layer l; ``emb`` / ``W_lm`` are bf16 device tensors [V, H];
+    ``budget`` < 0 derives B_i of Eq. 14 from the cache's free pairs."""
+
+    def __init__(self, ctx: "Context", layers: Sequence["Layer"], cache: "ExpertCache", emb: torch.Tensor,
+                 W_lm: torch.Tensor, k_max: int = 8, tau: float = 1.0, budget: int = -1):
+        if emb.dtype != torch.bfloat16 or W_lm.dtype != torch.bfloat16:
+            raise ValueError("Decoder: emb and W_lm must be bf16")
+        self.lib, self.ctx, self.k_max, self.n_layers = ctx.lib, ctx, k_max, len(layers)
+        self._keep = (list(layers), cache, emb, W_lm)        # (the library keeps raw pointers to all of them)
+        arr = (_P * len(layers))(*[l.handle for l in layers])
+        h = _P()
+        _check(self.lib.dx_decoder_create(ctx.handle, arr, len(layers), cache.handle, _ptr(emb), _ptr(W_lm),
+                                          int(W_lm.shape[0]), k_max, float(tau), int(budget), C.byref(h)),
+               "dx_decoder_create")
+        self.handle = h
+        self._drafted = (C.c_int32 * k_max)()
+        self._emitted = (C.c_int32 * (k_max + 1))()
+        self._target = (C.c_int32 * k_max)()
+        self._unions = (C.c_int32 * self.n_layers)()
+
+    def close(self) -> None:
+        if self.handle:
+            self.lib.dx_decoder_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def step(self, t0: int, scripted_accept: Optional[int] = None) -> Dict[str, object]:
+        nd, na, ne = _I(0), _I(0), _I(0)
+        _check(self.lib.dx_decoder_step(self.handle, int(t0), -1 if scripted_accept is None else int(scripted_accept),
+                                        self._drafted, C.byref(nd), C.byref(na), self._emitted, C.byref(ne),
+                                        self._target, self._unions, _stream()), "dx_decoder_step")
+        drafted = [int(self._drafted[i]) for i in range(nd.value)]
+        emitted = [int(self._emitted[i]) for i in range(ne.value)]
+        K = max(1, nd.value)
+        return {"drafted": drafted, "n_accept": na.value, "emitted": emitted, "next": emitted[-1],
+                "target": [int(self._target[i]) for i in range(K)], "block_rows": K,
+                "union_sizes": [int(self._unions[l]) for l in range(self.n_layers)]}
 
 
 class Controller:

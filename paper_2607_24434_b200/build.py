@@ -18,7 +18,7 @@ CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libdraftexpert.so")
 LIB_CHECKED = os.path.join(HERE, "libdraftexpert_checked.so")
 SOURCES = ["dx_api.cu", "dx_route.cu", "dx_grouped.cu", "dx_wide.cu", "dx_accept.cu", "dx_cache.cu", "dx_controller.cu",
-           "dx_eval.cu", "dx_draft_stack.cu"]
+           "dx_eval.cu", "dx_draft_stack.cu", "dx_decode.cu"]
 
 
 def _headers_mtime() -> float:

@@ -8,15 +8,6 @@
 bool dx_bf16_hidden_supported(int H);
 void dx_cache_forget_layer(dx_cache* c, dx_layer* L);
 
-#define DX_CUDA(ctx, call)                 \
-  do {                                     \
-    cudaError_t e__ = (call);              \
-    if (e__ != cudaSuccess) {              \
-      if (ctx) (ctx)->last_cuda = e__;     \
-      return DX_ERR_CUDA;                  \
-    }                                      \
-  } while (0)
-
 extern "C" const char* dx_status_string(dx_status s) {
   switch (s) {
     case DX_OK: return "ok";

@@ -85,6 +85,16 @@ struct dx_ctx {
   int32_t* union_host_dev;     //   ... and its device mapping, which the routing kernel writes
 };
 
+// a CUDA runtime call inside an entry point: the error goes to the context, the entry point returns DX_ERR_CUDA
+#define DX_CUDA(ctx, call)                 \
+  do {                                     \
+    cudaError_t e__ = (call);              \
+    if (e__ != cudaSuccess) {              \
+      if (ctx) (ctx)->last_cuda = e__;     \
+      return DX_ERR_CUDA;                  \
+    }                                      \
+  } while (0)
+
 struct dx_cache;
 
 struct dx_layer {

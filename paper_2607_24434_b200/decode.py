@@ -26,8 +26,13 @@ class OffloadedDecoder:
     is the one that is expensive to verify).  ``tau`` is the confidence threshold of Eq. 14."""
 
     def __init__(self, ctx: binding.Context, layers: Sequence[binding.Layer], cache: binding.ExpertCache,
-                 emb: torch.Tensor, W_lm: torch.Tensor, k_max: int = 8, tau: float = 1.0, budget="cache"):
+                 emb: torch.Tensor, W_lm: torch.Tensor, k_max: int = 8, tau: float = 1.0, budget="cache",
+                 native: bool = False):
+        """``native``: steps that are not recorded run as one library call (``dx_decoder_step``: the same calls in
+        the same order from a host loop inside the library, no interpreter between them)."""
         self.ctx, self.layers, self.cache = ctx, list(layers), cache
+        self._native = binding.Decoder(ctx, layers, cache, emb, W_lm, k_max, tau,
+                                       -1 if budget == "cache" else int(budget)) if native else None
         self.emb, self.W_lm = emb, W_lm
         self.k_max, self.tau, self.budget = k_max, tau, budget
         sh = self.layers[0].shape
@@ -43,6 +48,8 @@ class OffloadedDecoder:
 
     def close(self) -> None:
         self.controller.close()
+        if self._native is not None:
+            self._native.close()
 
     def _budget_now(self) -> int:
         if self.budget == "cache":
@@ -55,6 +62,8 @@ class OffloadedDecoder:
         the step (every layer's input rows, the routing the library used, the cache calls in order).
         ``scripted_accept``: take this accepted length (capped at the block length) instead of the comparison's
         -- for synthetic weights, whose random draft experts agree with the target almost never."""
+        if self._native is not None and not record:
+            return self._native.step(t0, scripted_accept)
         L = len(self.layers)
         trace: Dict[str, object] = {"draft": [], "verify": [], "cache_calls": []} if record else {}
         self.cache.begin_step()

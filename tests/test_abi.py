@@ -23,7 +23,7 @@ def test_header_symbols_exported_and_bound():
     assert len(names) >= 25
     for required in ("moe_draft_step", "moe_verify_block", "spec_accept", "expert_cache_prefetch",
                      "expert_cache_stage", "dx_pack_expert", "moe_verify_block_cached", "moe_draft_step_cached",
-                     "dx_set_wait_limit", "dx_set_accept_l2_keep", "dx_stage_block"):
+                     "dx_set_wait_limit", "dx_set_accept_l2_keep", "dx_stage_block", "dx_decoder_step"):
         assert required in names
     for n in names:
         assert hasattr(lib, n), f"{n} declared in the header but not exported"
@@ -58,3 +58,5 @@ def test_argument_errors_without_a_device():
     assert lib.dx_set_wait_limit(None, 100) == 1 and lib.dx_set_launch_overlap(None, 3) == 1
     assert lib.dx_set_accept_l2_keep(None, 1 << 20) == 1
     assert lib.dx_stage_block(None, None, None, 16, None) == 1
+    assert lib.dx_decoder_destroy(None) == 1
+    assert lib.dx_decoder_step(None, 0, -1, None, None, None, None, None, None, None, None) == 1
