@@ -262,7 +262,9 @@ dx_status moe_draft_experts(dx_layer* layer, const float* h, float* y, void* str
  *     host_union_count [1] (HOST pointers, may be NULL) receive the union the host read.
  *   moe_draft_step_cached: routes the token, reads the k selected ids back (host_topk_ids [k], HOST pointer, may be
  *     NULL: the predicted verifier experts to hand to dx_controller_propose / expert_cache_prefetch), stages e1 and
- *     evaluates Eq. 5. */
+ *     evaluates Eq. 5.  (bf16 / 4-bit units: the expert kernel is launched with the routing kernel, on the blob table
+ *     as the cache has it; if e1 turns out not to be held it is loaded and evaluated by a second launch.  The cache
+ *     sees one expert_cache_stage(e1) per call either way.) */
 dx_status moe_verify_block_cached(dx_layer* layer, const float* h, int32_t K, float* y, int32_t residual,
                                   int32_t* topk_ids, float* topk_w, uint64_t* union_mask, int32_t* union_ids,
                                   int32_t* union_count, int32_t* offsets, int32_t* perm, int32_t* host_union_ids,

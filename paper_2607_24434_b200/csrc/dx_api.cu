@@ -363,7 +363,7 @@ static dx_status do_route(dx_layer* L, const float* h, int K, float* y, const Ro
 static dx_status do_experts(dx_layer* L, const float* h, int K, float* y, bool draft, bool residual,
                             cudaStream_t st, int first_routed = 0, int n_routed = -1, bool do_static = true,
                             bool paired = false, bool skip_shared = false,
-                            const unsigned long long* subset = nullptr) {
+                            const unsigned long long* subset = nullptr, bool tolerate_missing = false) {
   dx_ctx* ctx = L->ctx;
   const dx_layer_desc& d = L->desc;
   if (!h || !y || h == y) return DX_ERR_INVALID_ARG;
@@ -393,6 +393,7 @@ static dx_status do_experts(dx_layer* L, const float* h, int K, float* y, bool d
   p.do_static = do_static ? 1 : 0;
   p.skip_shared = skip_shared ? 1 : 0;
   p.use_subset = subset ? 1 : 0;
+  p.tolerate_missing = tolerate_missing ? 1 : 0;
   for (int i = 0; i < DX_MAX_E / 64; ++i) p.subset[i] = subset ? subset[i] : 0ull;
   DX_CUDA(ctx, dx_launch_experts(ctx, p, L->desc.weight_dtype, K, st));
   ctx->launches++;
@@ -566,9 +567,34 @@ extern "C" dx_status moe_draft_step_cached(dx_layer* L, const float* h, float* y
   const int k = L->desc.top_k;
   int32_t* ids = topk_ids ? topk_ids : ctx->union_dev + DX_MAX_E + 1;
   RouteOut o{ids, topk_w, nullptr, nullptr, nullptr, nullptr, nullptr};
-  dx_status s = do_route(L, h, 1, y, o, true, residual != 0, st, 1, true, false, false, true);
-  if (s != DX_OK) return s;
   int32_t* host = ctx->union_host + DX_MAX_E + 1;
+  dx_status s;
+  const int dt = L->desc.weight_dtype;
+  if (dt == DX_DTYPE_BF16 || dt == DX_DTYPE_Q4) {
+    // Most selections are of experts the cache already holds, so the expert kernel is launched beside the routing
+    // kernel, as for a resident layer, before the host knows the selection: the blob table is first brought up to date
+    // (it then names exactly what the cache holds, and the stream has waited for copies still in flight), the kernel
+    // leaves a routed expert out if the table has no blob for it, and only in that case the expert is loaded and
+    // evaluated by a second launch.  The cache sees the same calls in the same order either way.
+    s = dx_cache_prepare_layer(L->cache, L->cache_layer, st);
+    if (s != DX_OK) return s;
+    s = do_route(L, h, 1, y, o, true, residual != 0, st, 1, true, true, false, true);
+    if (s != DX_OK) return s;
+    s = do_experts(L, h, 1, y, true, residual != 0, st, 0, -1, true, true, false, nullptr, true);
+    if (s != DX_OK) { cudaMemsetAsync(ctx->handover, 0, 4 * sizeof(unsigned int), st); return s; }
+    s = wait_for_routing(ctx, st);
+    if (s != DX_OK) return s;
+    if (host_topk_ids)
+      for (int j = 0; j < k; ++j) host_topk_ids[j] = host[j];
+    const int32_t e1 = host[0];
+    if (e1 < 0 || e1 >= L->desc.n_experts) return DX_ERR_CUDA;
+    const bool was_resident = dx_cache_slot_of(L->cache, L->cache_layer, e1) >= 0;
+    s = expert_cache_stage(L->cache, L->cache_layer, &e1, 1, stream);   // the bookkeeping of a hit, or the load
+    if (s != DX_OK || was_resident) return s;
+    return do_experts(L, h, 1, y, true, residual != 0, st, 0, -1, false);   // the routed expert alone, now that it is there
+  }
+  s = do_route(L, h, 1, y, o, true, residual != 0, st, 1, true, false, false, true);
+  if (s != DX_OK) return s;
   s = wait_for_routing(ctx, st);
   if (s != DX_OK) return s;
   if (host_topk_ids)

@@ -219,6 +219,18 @@ int dx_cache_slot_of(const dx_cache* c, int layer, int expert) {
 }
 int dx_cache_slots(const dx_cache* c) { return c ? c->S : 0; }
 
+dx_status dx_cache_prepare_layer(dx_cache* c, int layer, cudaStream_t st) {
+  if (!c || layer < 0 || layer >= c->L) return DX_ERR_INVALID_ARG;
+  if (!c->ctx) return DX_OK;
+  for (int s = 0; s < c->S; ++s) {
+    DxSlot& sl = slot_ref(c, layer, s);
+    if (sl.expert < 0 || copy_done(c, sl)) continue;
+    cudaError_t e = cudaStreamWaitEvent(st, sl.ev, 0);
+    if (e != cudaSuccess) { c->ctx->last_cuda = e; return DX_ERR_CUDA; }
+  }
+  return flush_patches(c, layer, st);
+}
+
 void dx_cache_note_use(dx_cache* c, int layer, cudaStream_t st) {
   if (!c || !c->ctx || layer < 0 || layer >= c->L) return;
   if (cudaEventRecord(c->used_ev[layer], st) == cudaSuccess) c->used_valid[layer] = 1;

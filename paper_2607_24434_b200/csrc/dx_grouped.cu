@@ -253,7 +253,7 @@ __global__ void __launch_bounds__(kThreads, 1) dx_experts_bf16_kernel(DxExpertPa
         hdr->e_tiles[e] = p.routed_tiles;
         hdr->e_gid[e] = gid;
         hdr->e_blob[e] = blob;
-        if (blob == nullptr && e >= e_lo && e < e_hi) atomicExch(p.dev_status, DX_DEV_BAD_EXPERT_ID);
+        if (blob == nullptr && e >= e_lo && e < e_hi && !p.tolerate_missing) atomicExch(p.dev_status, DX_DEV_BAD_EXPERT_ID);
       }
     }
     if (lane == 0) {

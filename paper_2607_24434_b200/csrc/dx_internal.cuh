@@ -96,6 +96,9 @@ struct dx_ctx {
   } while (0)
 
 struct dx_cache;
+// (cached layer calls) the compute stream waits for the layer's copies that are still in flight and the layer's blob
+// table is brought up to date: after this the table names exactly the experts the cache holds
+dx_status dx_cache_prepare_layer(dx_cache* c, int layer, cudaStream_t st);
 
 struct dx_layer {
   dx_ctx* ctx;
@@ -164,6 +167,10 @@ struct DxExpertParams {
   // of a cache-staged union need not be a contiguous run of the ascending id list
   int use_subset;
   unsigned long long subset[DX_MAX_E / 64];
+  // 1: a routed group whose blob-table entry is null is left out without a word in the status (the caller launched
+  // this kernel before it knew which expert the router would select, and evaluates the group afterwards if it was
+  // not resident); 0: such a group is reported as DX_DEV_BAD_EXPERT_ID
+  int tolerate_missing;
   int row_tiles;             // set by the launcher: 2 = CTA pairs, one tile of eight block rows each (K > 8)
   // Hand-over from the routing kernel launched right before this one (fused entry points only; null otherwise,
   // and then the kernel simply waits for everything in front of it).  With the hand-over this kernel may be running
