@@ -846,7 +846,8 @@ def run_offload(args):
         "prefetch_waste": d["prefetch_wasted"] / max(1, d["prefetch_issued"]),
         "prefetch_note": "used / wasted are counted when they happen; experts prefetched in the last step and still "
                          "pending are in neither",
-        "h2d_gbs": d["bytes_h2d"] / dt / 1e9, "waited_copies_per_step": d["waited_copies"] / steps, "cache": d,
+        "h2d_gbs": d["bytes_h2d"] / dt / 1e9, "waited_copies_per_step": d["waited_copies"] / steps,
+        "stream_wait_for_copies_ms_per_step": d["stream_stall_ns"] / steps / 1e6, "cache": d,
         "union_size_per_layer_mean": [round(float(u) / steps, 2) for u in union_sum],
     }))
     dec.close()

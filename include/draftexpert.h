@@ -432,8 +432,13 @@ typedef struct {
   int64_t prefetch_wasted;  /* prefetched experts evicted before any use */
   int64_t evictions;
   int64_t bytes_h2d;
-  int64_t waited_copies;    /* experts asked for whose copy had not landed yet (the stream or the host waited) */
+  int64_t waited_copies;    /* copies that had not landed yet when a call needed them -- or, for the drafter's layer
+                             * call, which runs its kernels before the selection is known, might need them (the
+                             * stream or the host waited) */
   int64_t stall_ns;         /* host time spent polling for such copies in expert_cache_wait */
+  int64_t stream_stall_ns;  /* time the compute stream spent waiting for such copies, measured on the device (an event
+                             * in front of the waits and one behind them; counted once both have completed, so a
+                             * call's waits show up in the statistics read after its work has run) */
 } dx_cache_stats;
 
 dx_status expert_cache_create(dx_ctx* ctx, int32_t n_layers, int32_t n_experts, int32_t slots_per_layer,

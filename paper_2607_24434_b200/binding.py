@@ -40,7 +40,8 @@ class LayerDesc(C.Structure):
 
 class CacheStats(C.Structure):
     _fields_ = [(n, C.c_int64) for n in ("lookups", "hits", "on_demand", "prefetch_issued", "prefetch_used",
-                                         "prefetch_wasted", "evictions", "bytes_h2d", "waited_copies", "stall_ns")]
+                                         "prefetch_wasted", "evictions", "bytes_h2d", "waited_copies", "stall_ns",
+                                         "stream_stall_ns")]
 
 
 _P = C.c_void_p

@@ -59,6 +59,10 @@ struct dx_cache {
   std::vector<cudaEvent_t> used_ev;     // last compute use of the layer's slots
   std::vector<char> used_valid;
   std::vector<std::vector<std::pair<int, const void*>>> pending;   // table patches not yet applied, per layer
+  // the compute stream's waits for copies, timed on the device: (event in front, event behind) pairs not yet read,
+  // and events free for reuse
+  std::vector<std::pair<cudaEvent_t, cudaEvent_t>> stall_open;
+  std::vector<cudaEvent_t> stall_free;
 };
 
 namespace {
@@ -157,6 +161,56 @@ bool copy_done(dx_cache* c, DxSlot& sl) {
   return false;
 }
 
+// A timed event (from the free list, or a new one); null if none can be had (the wait is then simply not timed).
+cudaEvent_t stall_event(dx_cache* c) {
+  if (!c->stall_free.empty()) { cudaEvent_t e = c->stall_free.back(); c->stall_free.pop_back(); return e; }
+  cudaEvent_t e = nullptr;
+  if (cudaEventCreate(&e) != cudaSuccess) { (void)cudaGetLastError(); return nullptr; }
+  return e;
+}
+// Makes `st` wait for the copies of the slots `want` marks that are still in flight, with an event in front of the
+// waits and one behind them.  Returns how many copies were waited for.
+int wait_for_copies(dx_cache* c, int layer, const std::vector<char>* want, cudaStream_t st, cudaError_t* err) {
+  *err = cudaSuccess;
+  int n = 0;
+  cudaEvent_t a = nullptr;
+  for (int s = 0; s < c->S; ++s) {
+    if (want && !(*want)[s]) continue;
+    DxSlot& sl = slot_ref(c, layer, s);
+    if (sl.expert < 0 || copy_done(c, sl)) continue;
+    if (n == 0) {
+      a = stall_event(c);
+      if (a && cudaEventRecord(a, st) != cudaSuccess) { (void)cudaGetLastError(); c->stall_free.push_back(a); a = nullptr; }
+    }
+    *err = cudaStreamWaitEvent(st, sl.ev, 0);
+    if (*err != cudaSuccess) break;
+    ++n;
+  }
+  if (a) {
+    cudaEvent_t b = stall_event(c);
+    if (b && cudaEventRecord(b, st) == cudaSuccess) c->stall_open.push_back({a, b});
+    else { (void)cudaGetLastError(); c->stall_free.push_back(a); if (b) c->stall_free.push_back(b); }
+  }
+  return n;
+}
+// Adds the waits that have run to the statistics.
+void harvest_stalls(dx_cache* c) {
+  size_t keep = 0;
+  for (size_t i = 0; i < c->stall_open.size(); ++i) {
+    auto pr = c->stall_open[i];
+    if (cudaEventQuery(pr.second) == cudaSuccess) {
+      float ms = 0.f;
+      if (cudaEventElapsedTime(&ms, pr.first, pr.second) == cudaSuccess) c->stats.stream_stall_ns += (int64_t)(ms * 1e6f);
+      c->stall_free.push_back(pr.first);
+      c->stall_free.push_back(pr.second);
+    } else {
+      (void)cudaGetLastError();
+      c->stall_open[keep++] = pr;
+    }
+  }
+  c->stall_open.resize(keep);
+}
+
 // applies the layer's pending table patches on `st`
 dx_status flush_patches(dx_cache* c, int layer, cudaStream_t st) {
   auto& pend = c->pending[layer];
@@ -222,12 +276,9 @@ int dx_cache_slots(const dx_cache* c) { return c ? c->S : 0; }
 dx_status dx_cache_prepare_layer(dx_cache* c, int layer, cudaStream_t st) {
   if (!c || layer < 0 || layer >= c->L) return DX_ERR_INVALID_ARG;
   if (!c->ctx) return DX_OK;
-  for (int s = 0; s < c->S; ++s) {
-    DxSlot& sl = slot_ref(c, layer, s);
-    if (sl.expert < 0 || copy_done(c, sl)) continue;
-    cudaError_t e = cudaStreamWaitEvent(st, sl.ev, 0);
-    if (e != cudaSuccess) { c->ctx->last_cuda = e; return DX_ERR_CUDA; }
-  }
+  cudaError_t e;
+  c->stats.waited_copies += wait_for_copies(c, layer, nullptr, st, &e);
+  if (e != cudaSuccess) { c->ctx->last_cuda = e; return DX_ERR_CUDA; }
   return flush_patches(c, layer, st);
 }
 
@@ -290,6 +341,8 @@ extern "C" dx_status expert_cache_destroy(dx_cache* c) {
     if (c->copy_stream) cudaStreamSynchronize(c->copy_stream);
     if (c->expand_stream) cudaStreamSynchronize(c->expand_stream);
     if (c->staged_ev) cudaEventDestroy(c->staged_ev);
+    for (auto& pr : c->stall_open) { cudaEventDestroy(pr.first); cudaEventDestroy(pr.second); }
+    for (auto& ev : c->stall_free) cudaEventDestroy(ev);
     if (c->expand_stream) cudaStreamDestroy(c->expand_stream);
     for (auto& s : c->slots)
       if (s.ev) cudaEventDestroy(s.ev);
@@ -359,6 +412,7 @@ extern "C" dx_status expert_cache_begin_step(dx_cache* c) {
   if (!c) return DX_ERR_INVALID_ARG;
   for (auto& s : c->slots)
     if (s.prefetched) { s.prefetched = false; c->stats.prefetch_wasted++; }
+  if (c->ctx) harvest_stalls(c);   // (keeps the list of timed waits short)
   return DX_OK;
 }
 
@@ -416,14 +470,14 @@ static dx_status resolve(dx_cache* c, int layer, const int32_t* ids, int n, cuda
   }
   if (!c->ctx) { c->pending[layer].clear(); return DX_OK; }
   // the compute stream waits for exactly the copies it needs that are not known to be complete
-  const auto t0 = std::chrono::steady_clock::now();
-  for (int s = 0; s < c->S; ++s) {
-    if (!pinned[s]) continue;
-    DxSlot& sl = slot_ref(c, layer, s);
-    if (copy_done(c, sl)) continue;
-    c->stats.waited_copies++;
-    if (timeout_s > 0.0) {
-      // bounded host wait (expert_cache_wait): poll the copy's event up to the deadline (counted from the call's start)
+  if (timeout_s > 0.0) {
+    // bounded host wait (expert_cache_wait): poll the copies' events up to the deadline (counted from the call's start)
+    const auto t0 = std::chrono::steady_clock::now();
+    for (int s = 0; s < c->S; ++s) {
+      if (!pinned[s]) continue;
+      DxSlot& sl = slot_ref(c, layer, s);
+      if (copy_done(c, sl)) continue;
+      c->stats.waited_copies++;
       const auto ts = std::chrono::steady_clock::now();
       bool late = false;
       while (!late && !copy_done(c, sl))
@@ -431,10 +485,11 @@ static dx_status resolve(dx_cache* c, int layer, const int32_t* ids, int n, cuda
       c->stats.stall_ns += (int64_t)std::chrono::duration_cast<std::chrono::nanoseconds>(
                                std::chrono::steady_clock::now() - ts).count();
       if (late) return DX_ERR_TIMEOUT;
-    } else {
-      cudaError_t e = cudaStreamWaitEvent(stream, sl.ev, 0);
-      if (e != cudaSuccess) { c->ctx->last_cuda = e; return DX_ERR_CUDA; }
     }
+  } else {
+    cudaError_t e;
+    c->stats.waited_copies += wait_for_copies(c, layer, &pinned, stream, &e);
+    if (e != cudaSuccess) { c->ctx->last_cuda = e; return DX_ERR_CUDA; }
   }
   return flush_patches(c, layer, stream);
 }
@@ -464,6 +519,7 @@ extern "C" dx_status expert_cache_inject_transfer_delay(dx_cache* c, int32_t mil
 
 extern "C" dx_status expert_cache_stats(dx_cache* c, dx_cache_stats* out) {
   if (!c || !out) return DX_ERR_INVALID_ARG;
+  if (c->ctx) harvest_stalls(c);
   *out = c->stats;
   return DX_OK;
 }

@@ -37,7 +37,7 @@ def test_header_symbols_exported_and_bound():
 def test_desc_struct_layout_matches_header():
     from paper_2607_24434_b200 import binding, synth
     assert ctypes.sizeof(binding.LayerDesc) == 12 * 4
-    assert ctypes.sizeof(binding.CacheStats) == 10 * 8
+    assert ctypes.sizeof(binding.CacheStats) == 11 * 8
     d = binding._desc(synth.shape_moonlight())
     assert (d.hidden, d.n_experts, d.top_k, d.inter, d.score_fn) == (2048, 64, 6, 1408, 1)
     assert abs(d.routed_scale - 2.446) < 1e-6

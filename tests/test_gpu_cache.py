@@ -137,6 +137,31 @@ def test_slow_transfer_times_out_and_then_completes():
     cache.close(); ctx.close()
 
 
+def test_stream_wait_for_a_slow_copy_is_timed_on_the_device():
+    """A block that needs an expert whose copy is stuck behind a 60 ms stall of the link: the compute stream waits for
+    it (no host wait), the result is right, and the statistics show the wait -- at least most of the stall, measured by
+    events on the stream."""
+    from paper_2607_24434_b200 import binding
+    ctx = binding.Context(0, act_split=True)
+    ref, resident, off, cache, host = _offloaded_layer(binding, ctx, 74, slots=4)
+    h = synth.hidden_block(1, SHAPE.hidden, 92, 0.0, "cuda")
+    want = binding.moe_draft_step(resident, h)
+    torch.cuda.synchronize()
+    ids = want["topk_ids"].tolist()
+    cache.begin_step()
+    assert cache.stats()["stream_stall_ns"] == 0
+    cache.inject_transfer_delay(60)
+    cache.prefetch(0, ids[:1])
+    out = binding.moe_draft_step_cached(off, h)              # returns once its kernels are queued behind the copy
+    torch.cuda.synchronize()
+    assert ctx.device_status() == 0
+    assert out["host_ids"] == ids
+    assert row_rel_err(out["y"].cpu().numpy(), want["y"].cpu().numpy()).max() <= 1e-5
+    st = cache.stats()
+    assert st["waited_copies"] >= 1 and 30_000_000 <= st["stream_stall_ns"] <= 500_000_000, st
+    cache.close(); ctx.close()
+
+
 def test_layer_destroyed_before_its_cache():
     """Either side may go first: a destroyed layer is forgotten by its cache (no patch is sent to a freed table)."""
     from paper_2607_24434_b200 import binding
