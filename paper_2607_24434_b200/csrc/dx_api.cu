@@ -570,12 +570,13 @@ extern "C" dx_status moe_draft_step_cached(dx_layer* L, const float* h, float* y
   int32_t* host = ctx->union_host + DX_MAX_E + 1;
   dx_status s;
   const int dt = L->desc.weight_dtype;
-  if (dt == DX_DTYPE_BF16 || dt == DX_DTYPE_Q4) {
-    // Most selections are of experts the cache already holds, so the expert kernel is launched beside the routing
-    // kernel, as for a resident layer, before the host knows the selection: the blob table is first brought up to date
-    // (it then names exactly what the cache holds, and the stream has waited for copies still in flight), the kernel
-    // leaves a routed expert out if the table has no blob for it, and only in that case the expert is loaded and
-    // evaluated by a second launch.  The cache sees the same calls in the same order either way.
+  if ((dt == DX_DTYPE_BF16 || dt == DX_DTYPE_Q4) && dx_cache_layer_quiet(L->cache, L->cache_layer)) {
+    // Most selections are of experts the cache already holds, so -- while none of the layer's copies is in flight:
+    // otherwise the stream would have to wait for all of them, not just for the one it may need -- the expert kernel
+    // is launched beside the routing kernel, as for a resident layer, before the host knows the selection: the blob
+    // table is first brought up to date (it then names exactly what the cache holds), the kernel leaves a routed
+    // expert out if the table has no blob for it, and only in that case the expert is loaded and evaluated by a
+    // second launch.  The cache sees the same calls in the same order either way.
     s = dx_cache_prepare_layer(L->cache, L->cache_layer, st);
     if (s != DX_OK) return s;
     s = do_route(L, h, 1, y, o, true, residual != 0, st, 1, true, true, false, true);

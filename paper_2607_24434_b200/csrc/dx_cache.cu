@@ -273,6 +273,16 @@ int dx_cache_slot_of(const dx_cache* c, int layer, int expert) {
 }
 int dx_cache_slots(const dx_cache* c) { return c ? c->S : 0; }
 
+bool dx_cache_layer_quiet(dx_cache* c, int layer) {
+  if (!c || layer < 0 || layer >= c->L) return false;
+  if (!c->ctx) return true;
+  for (int s = 0; s < c->S; ++s) {
+    DxSlot& sl = slot_ref(c, layer, s);
+    if (sl.expert >= 0 && !copy_done(c, sl)) return false;
+  }
+  return true;
+}
+
 dx_status dx_cache_prepare_layer(dx_cache* c, int layer, cudaStream_t st) {
   if (!c || layer < 0 || layer >= c->L) return DX_ERR_INVALID_ARG;
   if (!c->ctx) return DX_OK;

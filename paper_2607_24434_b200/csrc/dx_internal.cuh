@@ -99,6 +99,8 @@ struct dx_cache;
 // (cached layer calls) the compute stream waits for the layer's copies that are still in flight and the layer's blob
 // table is brought up to date: after this the table names exactly the experts the cache holds
 dx_status dx_cache_prepare_layer(dx_cache* c, int layer, cudaStream_t st);
+// true if none of the layer's copies is still in flight
+bool dx_cache_layer_quiet(dx_cache* c, int layer);
 
 struct dx_layer {
   dx_ctx* ctx;
