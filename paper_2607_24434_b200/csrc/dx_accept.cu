@@ -17,6 +17,7 @@
 #include <mutex>
 
 #include "dx_internal.cuh"
+#include "dx_stream.cuh"
 
 namespace {
 
@@ -40,9 +41,6 @@ __device__ __forceinline__ void mma_k16(float (&d)[4], uint32_t a0, uint32_t a1,
       "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
       : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
-__device__ __forceinline__ uint32_t pack2(__nv_bfloat16 lo16, __nv_bfloat16 hi16) {
-  return (uint32_t)__bfloat16_as_ushort(lo16) | ((uint32_t)__bfloat16_as_ushort(hi16) << 16);
 }
 __device__ __forceinline__ unsigned long long make_key(float v, int idx) {
   return ((unsigned long long)dx_orderable(v) << 32) | (unsigned long long)(0xffffffffu - (unsigned)idx);
@@ -276,6 +274,188 @@ __global__ void __launch_bounds__(512, 1) dx_accept_bf16_kernel(AcceptParams p) 
   finish<CONF>(p, s_keys);
 }
 
+// ---------------------------------------------------------------------------------------------------------
+// Ring variant (blocks of at most eight rows, H = 1024 / 2048, no confidence output).  Same arithmetic as the
+// kernel above; what differs is how the LM head reaches the tensor cores.  A producer thread streams whole
+// vocabulary rows (one bulk asynchronous copy each) into a ring of three 16-row tiles in shared memory; the eight
+// consumer warps split the contraction (warp w owns hidden columns [w H/8, (w+1) H/8), its hidden-row fragments
+// live in registers), add their partial logits up through shared memory once per tile, and 128 threads keep the
+// running maxima.  The LM head does not depend on the kernel in front, so when the launch is a programmatic one
+// the producer fills the ring while that kernel's last CTAs are still working, and the consumers wait for the
+// hidden rows only where they read them.  Loads that go to shared memory are also indifferent to how much of the
+// SM's memory is left for L1 -- the register-direct kernel loses a third of its rate on an SM that an expert CTA
+// has just left configured for 227 KB of shared memory.
+constexpr int kRingConsumers = 8;
+constexpr int kRingThreads = (kRingConsumers + 1) * 32;
+constexpr int kRingSlots = 3;
+
+struct RingHeader {
+  unsigned long long full[kRingSlots];
+  unsigned long long empty[kRingSlots];
+  unsigned long long keys[DX_MAX_M];
+  float ssq[kRingConsumers][8];
+  int abort_flag;
+};
+constexpr size_t kRingHdr = (sizeof(RingHeader) + 127) / 128 * 128;
+constexpr size_t kRingPartial = (size_t)2 * kRingConsumers * 32 * 16;   // [2][warp][lane] float4
+// a row of the tile is padded by 64 bytes: the eight rows a quarter-warp reads side by side fall into distinct banks
+template <int H> __host__ __device__ constexpr uint32_t ring_row_stride() { return (uint32_t)H * 2u + 64u; }
+template <int H> constexpr size_t ring_smem_bytes() { return kRingHdr + kRingPartial + (size_t)kRingSlots * 16 * ring_row_stride<H>(); }
+
+template <int H, bool CONF>
+__global__ void __launch_bounds__(kRingThreads, 1) dx_accept_ring_kernel(AcceptParams p, uint32_t wait_limit) {
+  constexpr int QW = H / 256;                    // 32-column steps of the contraction per consumer warp
+  constexpr uint32_t ROW = (uint32_t)H * 2u, STRIDE = ring_row_stride<H>(), TILE = 16u * STRIDE;
+  extern __shared__ __align__(128) unsigned char smem[];
+  RingHeader* hdr = reinterpret_cast<RingHeader*>(smem);
+  float4* partial = reinterpret_cast<float4*>(smem + kRingHdr);
+  unsigned char* ring = smem + kRingHdr + kRingPartial;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, c = lane & 3;
+  const int tiles = (p.V + 15) / 16;
+  volatile int* abort_flag = &hdr->abort_flag;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kRingSlots; ++s) {
+      mbar_init(smem_u32(&hdr->full[s]), 1);
+      mbar_init(smem_u32(&hdr->empty[s]), kRingConsumers);
+    }
+    hdr->abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (threadIdx.x < DX_MAX_M) hdr->keys[threadIdx.x] = 0ull;
+  __syncthreads();
+  dx_pdl_trigger();
+
+  if (warp == kRingConsumers) {
+    // ------------------------------------------------------------ producer: tile t of this CTA is tile blockIdx.x + t gridDim.x
+    if (lane == 0) {
+      // (tiles at the head of the matrix may be marked for retention in L2, see dx_set_accept_l2_keep)
+      const uint64_t pol_stream = l2_evict_first_policy();
+      uint64_t pol_keep;
+      asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_keep));
+      const unsigned char* Wb = reinterpret_cast<const unsigned char*>(p.W);
+      uint32_t issued = 0, slot = 0, phase = 0;
+      for (int tile = blockIdx.x; tile < tiles; tile += gridDim.x, ++issued) {
+        if (!mbar_wait(smem_u32(&hdr->empty[slot]), phase ^ 1u, abort_flag, wait_limit)) break;
+        const int rows = min(16, p.V - tile * 16);
+        const uint32_t fb = smem_u32(&hdr->full[slot]);
+        const uint64_t pol = tile < p.keep_tiles ? pol_keep : pol_stream;
+        mbar_arrive_expect_tx(fb, (uint32_t)rows * ROW);
+        for (int r = 0; r < rows; ++r)
+          bulk_g2s(smem_u32(ring + (size_t)slot * TILE + (size_t)r * STRIDE), Wb + ((size_t)tile * 16 + r) * ROW, ROW, fb, pol);
+        if (++slot == (uint32_t)kRingSlots) { slot = 0; phase ^= 1u; }
+      }
+      if (*abort_flag) {
+        // something gave up: no copy may still be landing in this CTA's shared memory when it is released
+        const uint32_t n_back = issued < (uint32_t)kRingSlots ? issued : (uint32_t)kRingSlots;
+        for (uint32_t k = 1; k <= n_back; ++k) {
+          const uint32_t j = issued - k, s = j % (uint32_t)kRingSlots, ph = (j / (uint32_t)kRingSlots) & 1u;
+          for (uint32_t spin = 0; spin < DX_WAIT_LIMIT_DEFAULT; ++spin)
+            if (mbar_try_wait(smem_u32(&hdr->full[s]), ph)) break;
+        }
+        if (p.dev_status) atomicExch(p.dev_status, (int32_t)DX_DEV_WAIT_EXPIRED);
+      }
+    }
+    __syncwarp();
+  } else {
+    // ------------------------------------------------------------ consumers
+    dx_pdl_wait();   // the hidden rows are usually the previous kernel's output
+    // this lane's fragments of hidden row g over the warp's columns: values of columns 32 q + 8 c .. + 7, as bf16 high
+    // part and residual (the contraction index is permuted the same way on both operands, see the kernel above)
+    uint4 bh[QW], bl[QW];
+    {
+      float4 xv[QW][2];
+      float ss = 0.f;
+      const bool valid = g < p.M;
+#pragma unroll
+      for (int q = 0; q < QW; ++q) {
+        xv[q][0] = xv[q][1] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (valid) {
+          const float* src = p.h + (size_t)g * H + 32 * (warp * QW + q) + 8 * c;
+          xv[q][0] = *reinterpret_cast<const float4*>(src);
+          xv[q][1] = *reinterpret_cast<const float4*>(src + 4);
+        }
+        ss += xv[q][0].x * xv[q][0].x + xv[q][0].y * xv[q][0].y + xv[q][0].z * xv[q][0].z + xv[q][0].w * xv[q][0].w;
+        ss += xv[q][1].x * xv[q][1].x + xv[q][1].y * xv[q][1].y + xv[q][1].z * xv[q][1].z + xv[q][1].w * xv[q][1].w;
+      }
+      float rs = 1.0f;
+      if (p.rms_norm) {
+        ss += __shfl_xor_sync(0xffffffffu, ss, 1);
+        ss += __shfl_xor_sync(0xffffffffu, ss, 2);
+        if (c == 0) hdr->ssq[warp][g] = ss;
+        consumer_bar();
+        float tot = 0.f;
+#pragma unroll
+        for (int w = 0; w < kRingConsumers; ++w) tot += hdr->ssq[w][g];
+        rs = rsqrtf(tot / (float)H + 1e-6f);
+      }
+#pragma unroll
+      for (int q = 0; q < QW; ++q) {
+        const float x[8] = {xv[q][0].x * rs, xv[q][0].y * rs, xv[q][0].z * rs, xv[q][0].w * rs,
+                            xv[q][1].x * rs, xv[q][1].y * rs, xv[q][1].z * rs, xv[q][1].w * rs};
+        __nv_bfloat16 hb[8], lb[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) split_bf16(x[i], hb[i], lb[i]);
+        bh[q] = make_uint4(pack2(hb[0], hb[1]), pack2(hb[2], hb[3]), pack2(hb[4], hb[5]), pack2(hb[6], hb[7]));
+        bl[q] = make_uint4(pack2(lb[0], lb[1]), pack2(lb[2], lb[3]), pack2(lb[4], lb[5]), pack2(lb[6], lb[7]));
+      }
+    }
+    // threads 0 .. 127 each own one (row within the tile, block row) pair of the summed logits: element e of the
+    // C fragments, e = 4 lane + r: tile row (lane >> 2) + 8 (r >> 1), block row 2 (lane & 3) + (r & 1)
+    const int e_row = (threadIdx.x >> 4) + ((threadIdx.x & 2) ? 8 : 0), e_tok = 2 * ((threadIdx.x >> 2) & 3) + (threadIdx.x & 1);
+    float best_v = -INFINITY;
+    int best_i = -1;
+    float cm = -INFINITY, cs = 0.0f;   // online softmax state of this thread's share of its block row (CONF only)
+    uint32_t slot = 0, phase = 0;
+    int buf = 0;
+    for (int tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
+      mbar_wait(smem_u32(&hdr->full[slot]), phase, abort_flag, wait_limit);
+      const unsigned char* T = ring + (size_t)slot * TILE + (size_t)g * STRIDE + (size_t)(warp * QW) * 64 + c * 16;
+      float ch[4] = {0.f, 0.f, 0.f, 0.f}, cl[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int q = 0; q < QW; ++q) {
+        const uint4 a0 = *reinterpret_cast<const uint4*>(T + q * 64);
+        const uint4 a1 = *reinterpret_cast<const uint4*>(T + 8 * STRIDE + q * 64);
+        mma_k16(ch, a0.x, a1.x, a0.y, a1.y, bh[q].x, bh[q].y);
+        mma_k16(cl, a0.x, a1.x, a0.y, a1.y, bl[q].x, bl[q].y);
+        mma_k16(ch, a0.z, a1.z, a0.w, a1.w, bh[q].z, bh[q].w);
+        mma_k16(cl, a0.z, a1.z, a0.w, a1.w, bl[q].z, bl[q].w);
+      }
+      __syncwarp();
+      if (lane == 0 && !*abort_flag) mbar_arrive(smem_u32(&hdr->empty[slot]));   // (no slot is released after a give-up)
+      if (++slot == (uint32_t)kRingSlots) { slot = 0; phase ^= 1u; }
+      partial[(buf * kRingConsumers + warp) * 32 + lane] = make_float4(ch[0] + cl[0], ch[1] + cl[1], ch[2] + cl[2], ch[3] + cl[3]);
+      consumer_bar();
+      if (threadIdx.x < 128) {
+        const float* ps = reinterpret_cast<const float*>(partial) + (size_t)buf * kRingConsumers * 128 + threadIdx.x;
+        float v = 0.f;
+#pragma unroll
+        for (int w = 0; w < kRingConsumers; ++w) v += ps[w * 128];
+        const int row = tile * 16 + e_row;
+        if (row < p.V) {
+          if (v > best_v) { best_v = v; best_i = row; }
+          if constexpr (CONF) conf_push(cm, cs, v);
+        }
+      }
+      buf ^= 1;
+    }
+    if (threadIdx.x < 128 && e_tok < p.M && best_i >= 0) atomicMax(&hdr->keys[e_tok], make_key(best_v, best_i));
+    if constexpr (CONF) {
+      // sixteen threads share a block row: their (max, sum) pairs meet in the (now idle) partial buffer
+      float2* sc = reinterpret_cast<float2*>(partial);
+      consumer_bar();
+      if (threadIdx.x < 128) sc[threadIdx.x] = make_float2(cm, cs);
+      consumer_bar();
+      if (threadIdx.x < p.M && threadIdx.x < 8) {
+        float m = -INFINITY, sum = 0.0f;
+        for (int e = 0; e < 128; ++e)
+          if (2 * ((e >> 2) & 3) + (e & 1) == (int)threadIdx.x) conf_merge(m, sum, sc[e].x, sc[e].y);
+        p.conf_part[(size_t)blockIdx.x * DX_MAX_M + threadIdx.x] = make_float2(m, sum);
+      }
+    }
+  }
+  finish<CONF>(p, hdr->keys);
+}
+
 // fp32 LM head (small vocabularies): one warp per vocabulary row.
 template <bool CONF>
 __global__ void __launch_bounds__(256) dx_accept_fp32_kernel(AcceptParams p) {
@@ -349,6 +529,15 @@ static cudaError_t launch_accept_bf16(dx_ctx* ctx, const AcceptParams& p, size_t
   return dx_launch_pdl((ctx->pdl_mask & DX_PDL_ACCEPT) != 0, dx_accept_bf16_kernel<NT, CONF>, dim3(ctx->sm_count), dim3(512), smem, st, 1, p);
 }
 
+template <int H, bool CONF>
+static cudaError_t launch_accept_ring(dx_ctx* ctx, const AcceptParams& p, cudaStream_t st) {
+  const size_t smem = ring_smem_bytes<H>();
+  cudaError_t e = cudaFuncSetAttribute(dx_accept_ring_kernel<H, CONF>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  return dx_launch_pdl((ctx->pdl_mask & DX_PDL_ACCEPT) != 0, dx_accept_ring_kernel<H, CONF>, dim3(ctx->sm_count), dim3(kRingThreads), smem, st, 1,
+                       p, ctx->wait_limit);
+}
+
 cudaError_t dx_launch_accept(dx_ctx* ctx, const float* h, int M, const void* W_lm, int V, int H, int w_dtype,
                              const int32_t* draft, int K, int rms_norm, int32_t* target, int32_t* n_accept,
                              int32_t* next_token, float* conf, cudaStream_t st) {
@@ -362,6 +551,11 @@ cudaError_t dx_launch_accept(dx_ctx* ctx, const float* h, int M, const void* W_l
     return dx_launch_pdl((ctx->pdl_mask & DX_PDL_ACCEPT) != 0, dx_accept_fp32_kernel<false>, dim3(grid), dim3(256), 0, st, 1, p);
   }
   const int NT = (M + 7) / 8;
+  // blocks of at most eight rows at the two large hidden sizes: the shared-memory ring variant
+  if (NT == 1 && H == 2048 && ring_smem_bytes<2048>() <= (size_t)ctx->smem_optin)
+    return conf ? launch_accept_ring<2048, true>(ctx, p, st) : launch_accept_ring<2048, false>(ctx, p, st);
+  if (NT == 1 && H == 1024 && ring_smem_bytes<1024>() <= (size_t)ctx->smem_optin)
+    return conf ? launch_accept_ring<1024, true>(ctx, p, st) : launch_accept_ring<1024, false>(ctx, p, st);
   const size_t smem = (size_t)NT * (H / 32) * 32 * 16 * 2;
   if (NT == 1) return conf ? launch_accept_bf16<1, true>(ctx, p, smem, st) : launch_accept_bf16<1, false>(ctx, p, smem, st);
   return conf ? launch_accept_bf16<2, true>(ctx, p, smem, st) : launch_accept_bf16<2, false>(ctx, p, smem, st);

@@ -47,3 +47,31 @@ def test_wait_for_a_routing_kernel_that_never_runs_expires():
     assert ctx.device_status() == 0
     assert row_rel_err(out["y"].cpu().numpy(), y_ref).max() <= Y_BF16
     L.close(); ctx.close()
+
+
+def test_accept_ring_gives_up_when_its_waits_are_cut_short():
+    """The ring variant of the accept kernel (blocks of at most eight rows, H = 2048) waits on mbarriers for its bulk
+    copies.  With a limit of a single poll those waits run out before the first tile has landed: the kernel records
+    DX_DEV_WAIT_EXPIRED, stops copying, waits (bounded) for what is still in flight and returns; with the default limit
+    restored the same call gives the checker's tokens."""
+    from paper_2607_24434_b200 import binding
+    ctx = binding.Context(0)
+    M, K, V, H = 5, 4, 148 * 16 * 4 + 3, 2048
+    W = synth.lm_head(V, H, 70, torch.bfloat16, "cuda")
+    h = synth.hidden_block(M, H, 71, 0.5, "cuda")
+    draft = torch.zeros((K,), dtype=torch.int32, device="cuda")
+    ctx.set_wait_limit(1)
+    binding.spec_accept(ctx, h, W, draft, rms_norm=True)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == DX_DEV_WAIT_EXPIRED
+    assert ctx.device_status() == 0
+    ctx.set_wait_limit(0)
+    out = binding.spec_accept(ctx, h, W, draft, rms_norm=True)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == 0
+    hn = O.rmsnorm(h.cpu().numpy().astype(np.float64))
+    t_ref, _, _, lg = O.greedy_accept_fast(hn, synth.to_numpy_f32(W).astype(np.float64), np.zeros(0, np.int32))
+    srt = np.sort(lg, axis=1)
+    clear = (srt[:, -1] - srt[:, -2]) > 1e-3
+    assert np.array_equal(out["target"].cpu().numpy()[clear], t_ref[clear])
+    ctx.close()

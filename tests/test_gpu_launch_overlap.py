@@ -47,6 +47,7 @@ def test_block_draft_and_accept_under_the_mask(dxm):
     _verify_case(dxm, wide, 9, seed=320, std=0.08)
     _draft_case(dxm, wide, seed=321, std=0.08)
     assert _accept_case(dxm, 5, 4, 4099, 256, torch.bfloat16, 330, rms=True, mode="mid") == 2
+    assert _accept_case(dxm, 5, 4, 4099, 2048, torch.bfloat16, 331, rms=True, mode="mid") == 2   # (ring variant)
 
 
 def test_back_to_back_steps_under_the_mask(dxm):
@@ -97,6 +98,9 @@ def test_accept_with_part_of_the_head_kept_in_l2(keep_bytes):
     for rep in range(3):
         assert _accept_case((binding, ctx), 9, 8, 3001, 1024, torch.bfloat16, 350, rms=True, mode="mid") == 4
     _accept_case((binding, ctx), 4, 4, 4099, 256, torch.bfloat16, 351, mode="geometric")
+    # (blocks of at most eight rows at H = 2048 go through the ring variant of the kernel: hints on its bulk copies)
+    for rep in range(2):
+        assert _accept_case((binding, ctx), 5, 4, 148 * 16 * 3 + 9, 2048, torch.bfloat16, 352, rms=True, mode="mid") == 2
     assert ctx.device_status() == 0
     ctx.close()
 

@@ -297,6 +297,34 @@ def test_accept_ties_take_lowest_index(dx):
     assert int(out["next_token"].item()) == -1
 
 
+@pytest.mark.parametrize("M,K,V,H", [(5, 4, 4099, 2048), (8, 8, 3001, 1024), (1, 1, 17, 2048), (3, 2, 2367 * 16 + 5, 1024),
+                                     (8, 7, 148 * 16 * 3 + 16, 2048)])
+def test_accept_ring_bf16(dx, M, K, V, H):
+    """Blocks of at most eight rows at H = 1024 / 2048 take the shared-memory ring variant of the accept kernel:
+    ragged last tile, fewer tiles than CTAs, several rounds of the three-slot ring."""
+    assert _accept_case(dx, M, K, V, H, torch.bfloat16, 500 + M, mode="match") == K
+    _accept_case(dx, M, K, V, H, torch.bfloat16, 510 + M, mode="geometric", rms=True)
+    if K > 1:
+        assert _accept_case(dx, M, K, V, H, torch.bfloat16, 520 + M, mode="mid", rms=True) == K // 2
+
+
+def test_accept_ring_ties_take_lowest_index(dx):
+    binding, ctx = dx
+    V, H = 148 * 16 * 2 + 40, 2048
+    W = torch.zeros((V, H), dtype=torch.bfloat16, device="cuda")
+    W[37, 0] = 1.0
+    W[4000, 0] = 1.0          # exact duplicate rows in different tiles / CTAs
+    W[V - 1, 1900] = 2.0      # in the ragged last tile, in the last warp's columns
+    W[5, 1900] = 2.0
+    h = torch.zeros((2, H), device="cuda")
+    h[0, 0] = 1.5
+    h[1, 1900] = 0.75
+    out = binding.spec_accept(ctx, h, W, torch.tensor([37, 5], dtype=torch.int32, device="cuda"))
+    torch.cuda.synchronize()
+    assert out["target"].tolist() == [37, 5] and int(out["n_accept"].item()) == 2
+    assert int(out["next_token"].item()) == -1
+
+
 def test_accept_full_vocab_bf16(dx):
     _accept_case(dx, 5, 4, 102400, 2048, torch.bfloat16, 400, mode="geometric", rms=True)
     _accept_case(dx, 9, 8, 163840, 2048, torch.bfloat16, 401, mode="geometric", rms=True)
@@ -305,7 +333,8 @@ def test_accept_full_vocab_bf16(dx):
 # ------------------------------------------------------------------ draft token + confidence (Sec. 3.4, q_i)
 @pytest.mark.parametrize("M,V,H,dtype", [(1, 1000, 512, torch.bfloat16), (4, 4099, 256, torch.bfloat16),
                                          (9, 3001, 1024, torch.bfloat16), (3, 1024, 256, torch.float32),
-                                         (1, 102400, 2048, torch.bfloat16)])
+                                         (1, 102400, 2048, torch.bfloat16), (8, 4099, 2048, torch.bfloat16),
+                                         (5, 148 * 16 + 7, 1024, torch.bfloat16)])
 def test_draft_token_confidence(dx, M, V, H, dtype):
     binding, ctx = dx
     W = synth.lm_head(V, H, 700 + M, dtype, "cuda", std=0.05)
