@@ -293,23 +293,23 @@ struct RingHeader {
   unsigned long long full[kRingSlots];
   unsigned long long empty[kRingSlots];
   unsigned long long keys[DX_MAX_M];
-  float ssq[kRingConsumers][8];
+  float ssq[kRingConsumers][DX_MAX_M];
   int abort_flag;
 };
 constexpr size_t kRingHdr = (sizeof(RingHeader) + 127) / 128 * 128;
-constexpr size_t kRingPartial = (size_t)2 * kRingConsumers * 32 * 16;   // [2][warp][lane] float4
+constexpr size_t kRingPartial = (size_t)2 * kRingConsumers * 32 * 16;   // [2][warp][lane] float4, per token tile
 // a row of the tile is padded by 64 bytes: the eight rows a quarter-warp reads side by side fall into distinct banks
 template <int H> __host__ __device__ constexpr uint32_t ring_row_stride() { return (uint32_t)H * 2u + 64u; }
-template <int H> constexpr size_t ring_smem_bytes() { return kRingHdr + kRingPartial + (size_t)kRingSlots * 16 * ring_row_stride<H>(); }
+template <int H, int NT> constexpr size_t ring_smem_bytes() { return kRingHdr + (size_t)NT * kRingPartial + (size_t)kRingSlots * 16 * ring_row_stride<H>(); }
 
-template <int H, bool CONF>
+template <int H, int NT, bool CONF>
 __global__ void __launch_bounds__(kRingThreads, 1) dx_accept_ring_kernel(AcceptParams p, uint32_t wait_limit) {
   constexpr int QW = H / 256;                    // 32-column steps of the contraction per consumer warp
   constexpr uint32_t ROW = (uint32_t)H * 2u, STRIDE = ring_row_stride<H>(), TILE = 16u * STRIDE;
   extern __shared__ __align__(128) unsigned char smem[];
   RingHeader* hdr = reinterpret_cast<RingHeader*>(smem);
-  float4* partial = reinterpret_cast<float4*>(smem + kRingHdr);
-  unsigned char* ring = smem + kRingHdr + kRingPartial;
+  float4* partial = reinterpret_cast<float4*>(smem + kRingHdr);            // [2][warp][NT][lane]
+  unsigned char* ring = smem + kRingHdr + (size_t)NT * kRingPartial;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, c = lane & 3;
   const int tiles = (p.V + 15) / 16;
   volatile int* abort_flag = &hdr->abort_flag;
@@ -359,49 +359,59 @@ __global__ void __launch_bounds__(kRingThreads, 1) dx_accept_ring_kernel(AcceptP
   } else {
     // ------------------------------------------------------------ consumers
     dx_pdl_wait();   // the hidden rows are usually the previous kernel's output
-    // this lane's fragments of hidden row g over the warp's columns: values of columns 32 q + 8 c .. + 7, as bf16 high
-    // part and residual (the contraction index is permuted the same way on both operands, see the kernel above)
-    uint4 bh[QW], bl[QW];
-    {
-      float4 xv[QW][2];
-      float ss = 0.f;
-      const bool valid = g < p.M;
+    // this lane's fragments of hidden rows g (and 8 + g) over the warp's columns: values of columns 32 q + 8 c .. + 7,
+    // as bf16 high part and residual (the contraction index is permuted the same way on both operands, see the
+    // kernel above)
+    uint4 bh[NT][QW], bl[NT][QW];
+    if (p.rms_norm) {
 #pragma unroll
-      for (int q = 0; q < QW; ++q) {
-        xv[q][0] = xv[q][1] = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (valid) {
-          const float* src = p.h + (size_t)g * H + 32 * (warp * QW + q) + 8 * c;
-          xv[q][0] = *reinterpret_cast<const float4*>(src);
-          xv[q][1] = *reinterpret_cast<const float4*>(src + 4);
+      for (int nt = 0; nt < NT; ++nt) {
+        float ss = 0.f;
+        if (nt * 8 + g < p.M) {
+#pragma unroll
+          for (int q = 0; q < QW; ++q) {
+            const float* src = p.h + (size_t)(nt * 8 + g) * H + 32 * (warp * QW + q) + 8 * c;
+            const float4 v0 = *reinterpret_cast<const float4*>(src), v1 = *reinterpret_cast<const float4*>(src + 4);
+            ss += v0.x * v0.x + v0.y * v0.y + v0.z * v0.z + v0.w * v0.w + v1.x * v1.x + v1.y * v1.y + v1.z * v1.z + v1.w * v1.w;
+          }
         }
-        ss += xv[q][0].x * xv[q][0].x + xv[q][0].y * xv[q][0].y + xv[q][0].z * xv[q][0].z + xv[q][0].w * xv[q][0].w;
-        ss += xv[q][1].x * xv[q][1].x + xv[q][1].y * xv[q][1].y + xv[q][1].z * xv[q][1].z + xv[q][1].w * xv[q][1].w;
-      }
-      float rs = 1.0f;
-      if (p.rms_norm) {
         ss += __shfl_xor_sync(0xffffffffu, ss, 1);
         ss += __shfl_xor_sync(0xffffffffu, ss, 2);
-        if (c == 0) hdr->ssq[warp][g] = ss;
-        consumer_bar();
+        if (c == 0) hdr->ssq[warp][nt * 8 + g] = ss;
+      }
+      consumer_bar();
+    }
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+      float rs = 1.0f;
+      if (p.rms_norm) {
         float tot = 0.f;
 #pragma unroll
-        for (int w = 0; w < kRingConsumers; ++w) tot += hdr->ssq[w][g];
+        for (int w = 0; w < kRingConsumers; ++w) tot += hdr->ssq[w][nt * 8 + g];
         rs = rsqrtf(tot / (float)H + 1e-6f);
       }
+      const bool valid = nt * 8 + g < p.M;
 #pragma unroll
       for (int q = 0; q < QW; ++q) {
-        const float x[8] = {xv[q][0].x * rs, xv[q][0].y * rs, xv[q][0].z * rs, xv[q][0].w * rs,
-                            xv[q][1].x * rs, xv[q][1].y * rs, xv[q][1].z * rs, xv[q][1].w * rs};
+        float4 v0 = make_float4(0.f, 0.f, 0.f, 0.f), v1 = v0;
+        if (valid) {
+          const float* src = p.h + (size_t)(nt * 8 + g) * H + 32 * (warp * QW + q) + 8 * c;
+          v0 = *reinterpret_cast<const float4*>(src);
+          v1 = *reinterpret_cast<const float4*>(src + 4);
+        }
+        const float x[8] = {v0.x * rs, v0.y * rs, v0.z * rs, v0.w * rs, v1.x * rs, v1.y * rs, v1.z * rs, v1.w * rs};
         __nv_bfloat16 hb[8], lb[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) split_bf16(x[i], hb[i], lb[i]);
-        bh[q] = make_uint4(pack2(hb[0], hb[1]), pack2(hb[2], hb[3]), pack2(hb[4], hb[5]), pack2(hb[6], hb[7]));
-        bl[q] = make_uint4(pack2(lb[0], lb[1]), pack2(lb[2], lb[3]), pack2(lb[4], lb[5]), pack2(lb[6], lb[7]));
+        bh[nt][q] = make_uint4(pack2(hb[0], hb[1]), pack2(hb[2], hb[3]), pack2(hb[4], hb[5]), pack2(hb[6], hb[7]));
+        bl[nt][q] = make_uint4(pack2(lb[0], lb[1]), pack2(lb[2], lb[3]), pack2(lb[4], lb[5]), pack2(lb[6], lb[7]));
       }
     }
-    // threads 0 .. 127 each own one (row within the tile, block row) pair of the summed logits: element e of the
-    // C fragments, e = 4 lane + r: tile row (lane >> 2) + 8 (r >> 1), block row 2 (lane & 3) + (r & 1)
-    const int e_row = (threadIdx.x >> 4) + ((threadIdx.x & 2) ? 8 : 0), e_tok = 2 * ((threadIdx.x >> 2) & 3) + (threadIdx.x & 1);
+    // threads 0 .. 128 NT - 1 each own one (row within the tile, block row) pair of the summed logits: element e of
+    // token tile nt's C fragments, e = 4 lane + r: tile row (lane >> 2) + 8 (r >> 1), block row 8 nt + 2 (lane & 3) + (r & 1)
+    const int e_el = threadIdx.x & 127, e_nt = threadIdx.x >> 7;
+    const int e_row = (e_el >> 4) + ((e_el & 2) ? 8 : 0), e_tok = 8 * e_nt + 2 * ((e_el >> 2) & 3) + (e_el & 1);
+    const bool owner = threadIdx.x < 128 * NT;
     float best_v = -INFINITY;
     int best_i = -1;
     float cm = -INFINITY, cs = 0.0f;   // online softmax state of this thread's share of its block row (CONF only)
@@ -410,26 +420,36 @@ __global__ void __launch_bounds__(kRingThreads, 1) dx_accept_ring_kernel(AcceptP
     for (int tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
       mbar_wait(smem_u32(&hdr->full[slot]), phase, abort_flag, wait_limit);
       const unsigned char* T = ring + (size_t)slot * TILE + (size_t)g * STRIDE + (size_t)(warp * QW) * 64 + c * 16;
-      float ch[4] = {0.f, 0.f, 0.f, 0.f}, cl[4] = {0.f, 0.f, 0.f, 0.f};
+      float ch[NT][4], cl[NT][4];
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+        for (int r = 0; r < 4; ++r) ch[nt][r] = cl[nt][r] = 0.f;
 #pragma unroll
       for (int q = 0; q < QW; ++q) {
         const uint4 a0 = *reinterpret_cast<const uint4*>(T + q * 64);
         const uint4 a1 = *reinterpret_cast<const uint4*>(T + 8 * STRIDE + q * 64);
-        mma_k16(ch, a0.x, a1.x, a0.y, a1.y, bh[q].x, bh[q].y);
-        mma_k16(cl, a0.x, a1.x, a0.y, a1.y, bl[q].x, bl[q].y);
-        mma_k16(ch, a0.z, a1.z, a0.w, a1.w, bh[q].z, bh[q].w);
-        mma_k16(cl, a0.z, a1.z, a0.w, a1.w, bl[q].z, bl[q].w);
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+          mma_k16(ch[nt], a0.x, a1.x, a0.y, a1.y, bh[nt][q].x, bh[nt][q].y);
+          mma_k16(cl[nt], a0.x, a1.x, a0.y, a1.y, bl[nt][q].x, bl[nt][q].y);
+          mma_k16(ch[nt], a0.z, a1.z, a0.w, a1.w, bh[nt][q].z, bh[nt][q].w);
+          mma_k16(cl[nt], a0.z, a1.z, a0.w, a1.w, bl[nt][q].z, bl[nt][q].w);
+        }
       }
       __syncwarp();
       if (lane == 0 && !*abort_flag) mbar_arrive(smem_u32(&hdr->empty[slot]));   // (no slot is released after a give-up)
       if (++slot == (uint32_t)kRingSlots) { slot = 0; phase ^= 1u; }
-      partial[(buf * kRingConsumers + warp) * 32 + lane] = make_float4(ch[0] + cl[0], ch[1] + cl[1], ch[2] + cl[2], ch[3] + cl[3]);
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt)
+        partial[((buf * kRingConsumers + warp) * NT + nt) * 32 + lane] =
+            make_float4(ch[nt][0] + cl[nt][0], ch[nt][1] + cl[nt][1], ch[nt][2] + cl[nt][2], ch[nt][3] + cl[nt][3]);
       consumer_bar();
-      if (threadIdx.x < 128) {
-        const float* ps = reinterpret_cast<const float*>(partial) + (size_t)buf * kRingConsumers * 128 + threadIdx.x;
+      if (owner) {
+        const float* ps = reinterpret_cast<const float*>(partial) + ((size_t)buf * kRingConsumers * NT + e_nt) * 128 + e_el;
         float v = 0.f;
 #pragma unroll
-        for (int w = 0; w < kRingConsumers; ++w) v += ps[w * 128];
+        for (int w = 0; w < kRingConsumers; ++w) v += ps[w * NT * 128];
         const int row = tile * 16 + e_row;
         if (row < p.V) {
           if (v > best_v) { best_v = v; best_i = row; }
@@ -438,17 +458,17 @@ __global__ void __launch_bounds__(kRingThreads, 1) dx_accept_ring_kernel(AcceptP
       }
       buf ^= 1;
     }
-    if (threadIdx.x < 128 && e_tok < p.M && best_i >= 0) atomicMax(&hdr->keys[e_tok], make_key(best_v, best_i));
+    if (owner && e_tok < p.M && best_i >= 0) atomicMax(&hdr->keys[e_tok], make_key(best_v, best_i));
     if constexpr (CONF) {
       // sixteen threads share a block row: their (max, sum) pairs meet in the (now idle) partial buffer
       float2* sc = reinterpret_cast<float2*>(partial);
       consumer_bar();
-      if (threadIdx.x < 128) sc[threadIdx.x] = make_float2(cm, cs);
+      if (owner) sc[threadIdx.x] = make_float2(cm, cs);
       consumer_bar();
-      if (threadIdx.x < p.M && threadIdx.x < 8) {
+      if (threadIdx.x < p.M && threadIdx.x < 8 * NT) {
         float m = -INFINITY, sum = 0.0f;
-        for (int e = 0; e < 128; ++e)
-          if (2 * ((e >> 2) & 3) + (e & 1) == (int)threadIdx.x) conf_merge(m, sum, sc[e].x, sc[e].y);
+        for (int e = 0; e < 128 * NT; ++e)
+          if (8 * (e >> 7) + 2 * (((e & 127) >> 2) & 3) + (e & 1) == (int)threadIdx.x) conf_merge(m, sum, sc[e].x, sc[e].y);
         p.conf_part[(size_t)blockIdx.x * DX_MAX_M + threadIdx.x] = make_float2(m, sum);
       }
     }
@@ -529,13 +549,18 @@ static cudaError_t launch_accept_bf16(dx_ctx* ctx, const AcceptParams& p, size_t
   return dx_launch_pdl((ctx->pdl_mask & DX_PDL_ACCEPT) != 0, dx_accept_bf16_kernel<NT, CONF>, dim3(ctx->sm_count), dim3(512), smem, st, 1, p);
 }
 
-template <int H, bool CONF>
+template <int H, int NT, bool CONF>
 static cudaError_t launch_accept_ring(dx_ctx* ctx, const AcceptParams& p, cudaStream_t st) {
-  const size_t smem = ring_smem_bytes<H>();
-  cudaError_t e = cudaFuncSetAttribute(dx_accept_ring_kernel<H, CONF>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  const size_t smem = ring_smem_bytes<H, NT>();
+  cudaError_t e = cudaFuncSetAttribute(dx_accept_ring_kernel<H, NT, CONF>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  return dx_launch_pdl((ctx->pdl_mask & DX_PDL_ACCEPT) != 0, dx_accept_ring_kernel<H, CONF>, dim3(ctx->sm_count), dim3(kRingThreads), smem, st, 1,
-                       p, ctx->wait_limit);
+  return dx_launch_pdl((ctx->pdl_mask & DX_PDL_ACCEPT) != 0, dx_accept_ring_kernel<H, NT, CONF>, dim3(ctx->sm_count), dim3(kRingThreads), smem,
+                       st, 1, p, ctx->wait_limit);
+}
+template <int H>
+static cudaError_t launch_accept_ring_h(dx_ctx* ctx, const AcceptParams& p, int NT, bool conf, cudaStream_t st) {
+  if (NT == 1) return conf ? launch_accept_ring<H, 1, true>(ctx, p, st) : launch_accept_ring<H, 1, false>(ctx, p, st);
+  return conf ? launch_accept_ring<H, 2, true>(ctx, p, st) : launch_accept_ring<H, 2, false>(ctx, p, st);
 }
 
 cudaError_t dx_launch_accept(dx_ctx* ctx, const float* h, int M, const void* W_lm, int V, int H, int w_dtype,
@@ -551,11 +576,9 @@ cudaError_t dx_launch_accept(dx_ctx* ctx, const float* h, int M, const void* W_l
     return dx_launch_pdl((ctx->pdl_mask & DX_PDL_ACCEPT) != 0, dx_accept_fp32_kernel<false>, dim3(grid), dim3(256), 0, st, 1, p);
   }
   const int NT = (M + 7) / 8;
-  // blocks of at most eight rows at the two large hidden sizes: the shared-memory ring variant
-  if (NT == 1 && H == 2048 && ring_smem_bytes<2048>() <= (size_t)ctx->smem_optin)
-    return conf ? launch_accept_ring<2048, true>(ctx, p, st) : launch_accept_ring<2048, false>(ctx, p, st);
-  if (NT == 1 && H == 1024 && ring_smem_bytes<1024>() <= (size_t)ctx->smem_optin)
-    return conf ? launch_accept_ring<1024, true>(ctx, p, st) : launch_accept_ring<1024, false>(ctx, p, st);
+  // the two large hidden sizes: the shared-memory ring variant
+  if (H == 2048 && ring_smem_bytes<2048, 2>() <= (size_t)ctx->smem_optin) return launch_accept_ring_h<2048>(ctx, p, NT, conf != nullptr, st);
+  if (H == 1024 && ring_smem_bytes<1024, 2>() <= (size_t)ctx->smem_optin) return launch_accept_ring_h<1024>(ctx, p, NT, conf != nullptr, st);
   const size_t smem = (size_t)NT * (H / 32) * 32 * 16 * 2;
   if (NT == 1) return conf ? launch_accept_bf16<1, true>(ctx, p, smem, st) : launch_accept_bf16<1, false>(ctx, p, smem, st);
   return conf ? launch_accept_bf16<2, true>(ctx, p, smem, st) : launch_accept_bf16<2, false>(ctx, p, smem, st);

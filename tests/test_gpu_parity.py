@@ -298,10 +298,11 @@ def test_accept_ties_take_lowest_index(dx):
 
 
 @pytest.mark.parametrize("M,K,V,H", [(5, 4, 4099, 2048), (8, 8, 3001, 1024), (1, 1, 17, 2048), (3, 2, 2367 * 16 + 5, 1024),
-                                     (8, 7, 148 * 16 * 3 + 16, 2048)])
+                                     (8, 7, 148 * 16 * 3 + 16, 2048), (16, 16, 148 * 16 * 2 + 1, 2048),
+                                     (9, 8, 5003, 2048), (13, 12, 4099, 1024)])
 def test_accept_ring_bf16(dx, M, K, V, H):
-    """Blocks of at most eight rows at H = 1024 / 2048 take the shared-memory ring variant of the accept kernel:
-    ragged last tile, fewer tiles than CTAs, several rounds of the three-slot ring."""
+    """H = 1024 / 2048 take the shared-memory ring variant of the accept kernel (one or two tiles of eight block
+    rows): ragged last tile, fewer tiles than CTAs, several rounds of the three-slot ring."""
     assert _accept_case(dx, M, K, V, H, torch.bfloat16, 500 + M, mode="match") == K
     _accept_case(dx, M, K, V, H, torch.bfloat16, 510 + M, mode="geometric", rms=True)
     if K > 1:
@@ -334,7 +335,7 @@ def test_accept_full_vocab_bf16(dx):
 @pytest.mark.parametrize("M,V,H,dtype", [(1, 1000, 512, torch.bfloat16), (4, 4099, 256, torch.bfloat16),
                                          (9, 3001, 1024, torch.bfloat16), (3, 1024, 256, torch.float32),
                                          (1, 102400, 2048, torch.bfloat16), (8, 4099, 2048, torch.bfloat16),
-                                         (5, 148 * 16 + 7, 1024, torch.bfloat16)])
+                                         (5, 148 * 16 + 7, 1024, torch.bfloat16), (11, 4099, 2048, torch.bfloat16)])
 def test_draft_token_confidence(dx, M, V, H, dtype):
     binding, ctx = dx
     W = synth.lm_head(V, H, 700 + M, dtype, "cuda", std=0.05)
