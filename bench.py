@@ -542,7 +542,7 @@ def run_gpu(args):
                      "k8": None if blk8 is None else dict(blk8, fractions=fractions(blk8)),
                      # the other kernels of the step, each timed back to back from its own graph, same peak
                      "others": {
-                         "dx_accept_bf16_kernel (greedy accept, LM head streamed once)": {
+                         "dx_accept_ring_kernel (greedy accept, LM head streamed once)": {
                              "ms_per_launch": comp.get("accept_ms", acc_ms),
                              "achieved": acc_bytes / (comp.get("accept_ms", acc_ms) * 1e-3) / 1e9,
                              "frac": acc_bytes / (comp.get("accept_ms", acc_ms) * 1e-3) / 1e9 / peak},

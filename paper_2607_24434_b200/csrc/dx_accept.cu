@@ -3,8 +3,10 @@
 // the lowest v winning ties, accepted length n = longest prefix with
 // t_i == d_i, next token = t_n.
 //
-// The LM head [V,H] is streamed from HBM exactly once for all M rows.  bf16
-// path: each warp owns 16 vocabulary rows at a time and multiplies them with
+// The LM head [V,H] is streamed from HBM exactly once for all M rows.  Two bf16
+// kernels share the arithmetic described here; the ring variant further down
+// (H = 1024 / 2048) brings the rows in through shared memory instead.  Register-
+// direct kernel: each warp owns 16 vocabulary rows at a time and multiplies them with
 // the M hidden rows on the tensor cores (mma.sync m16n8k16, vocabulary rows as
 // the 16-row operand, hidden rows as the 8-column operand, hidden rows fed as
 // bf16 high part + bf16 residual).  A lane loads 16 contiguous bytes of two
@@ -275,12 +277,12 @@ __global__ void __launch_bounds__(512, 1) dx_accept_bf16_kernel(AcceptParams p) 
 }
 
 // ---------------------------------------------------------------------------------------------------------
-// Ring variant (blocks of at most eight rows, H = 1024 / 2048, no confidence output).  Same arithmetic as the
+// Ring variant (H = 1024 / 2048; one or two tiles of eight block rows).  Same arithmetic as the
 // kernel above; what differs is how the LM head reaches the tensor cores.  A producer thread streams whole
 // vocabulary rows (one bulk asynchronous copy each) into a ring of three 16-row tiles in shared memory; the eight
 // consumer warps split the contraction (warp w owns hidden columns [w H/8, (w+1) H/8), its hidden-row fragments
-// live in registers), add their partial logits up through shared memory once per tile, and 128 threads keep the
-// running maxima.  The LM head does not depend on the kernel in front, so when the launch is a programmatic one
+// live in registers), add their partial logits up through shared memory once per tile, and 128 threads per token
+// tile keep the running maxima.  The LM head does not depend on the kernel in front, so when the launch is a programmatic one
 // the producer fills the ring while that kernel's last CTAs are still working, and the consumers wait for the
 // hidden rows only where they read them.  Loads that go to shared memory are also indifferent to how much of the
 // SM's memory is left for L1 -- the register-direct kernel loses a third of its rate on an SM that an expert CTA
