@@ -339,6 +339,10 @@ __global__ void __launch_bounds__(kRingThreads, 1) dx_accept_ring_kernel(AcceptP
       for (int tile = blockIdx.x; tile < tiles; tile += gridDim.x, ++issued) {
         if (!mbar_wait(smem_u32(&hdr->empty[slot]), phase ^ 1u, abort_flag, wait_limit)) break;
         const int rows = min(16, p.V - tile * 16);
+        if (!DX_BOUNDS(slot < (uint32_t)kRingSlots && rows >= 1 && (long long)tile * 16 + rows <= (long long)p.V, p.dev_status)) {
+          *abort_flag = 1;
+          break;
+        }
         const uint32_t fb = smem_u32(&hdr->full[slot]);
         const uint64_t pol = tile < p.keep_tiles ? pol_keep : pol_stream;
         mbar_arrive_expect_tx(fb, (uint32_t)rows * ROW);
@@ -420,6 +424,8 @@ __global__ void __launch_bounds__(kRingThreads, 1) dx_accept_ring_kernel(AcceptP
     uint32_t slot = 0, phase = 0;
     int buf = 0;
     for (int tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
+      // (a slot out of range is reported and replaced: every warp has to keep taking part in the barriers below)
+      if (!DX_BOUNDS(slot < (uint32_t)kRingSlots, p.dev_status)) { *abort_flag = 1; slot = 0; }
       mbar_wait(smem_u32(&hdr->full[slot]), phase, abort_flag, wait_limit);
       const unsigned char* T = ring + (size_t)slot * TILE + (size_t)g * STRIDE + (size_t)(warp * QW) * 64 + c * 16;
       float ch[NT][4], cl[NT][4];
@@ -460,7 +466,8 @@ __global__ void __launch_bounds__(kRingThreads, 1) dx_accept_ring_kernel(AcceptP
       }
       buf ^= 1;
     }
-    if (owner && e_tok < p.M && best_i >= 0) atomicMax(&hdr->keys[e_tok], make_key(best_v, best_i));
+    if (owner && e_tok < p.M && best_i >= 0 && DX_BOUNDS(e_tok < DX_MAX_M && best_i < p.V, p.dev_status))
+      atomicMax(&hdr->keys[e_tok], make_key(best_v, best_i));
     if constexpr (CONF) {
       // sixteen threads share a block row: their (max, sum) pairs meet in the (now idle) partial buffer
       float2* sc = reinterpret_cast<float2*>(partial);
