@@ -143,3 +143,70 @@ def test_stage_block_and_results_written_to_the_host():
     assert int(res[M]) == int(dev["n_accept"].item()) == 2 and int(res[M + 1]) == int(dev["next_token"].item())
     assert ctx.device_status() == 0
     ctx.close()
+
+
+@pytest.mark.parametrize("mask", [3, 7])
+def test_step_graph_replays_are_stable(mask):
+    """The benchmark's arrangement — draft step, verify block and greedy accept over the full 102 400-row vocabulary,
+    captured once in a CUDA graph and replayed — gives, on every one of several hundred replays, the results of the
+    first eager run (integer outputs bit for bit), and that run's target tokens are the checker's.  A race in one of
+    the hand-overs between neighbouring kernels would show up as an occasional odd replay."""
+    from paper_2607_24434_b200 import binding
+    ctx = binding.Context(0)
+    ctx.set_launch_overlap(mask)
+    shape = synth.shape_v2lite()
+    K, V, NL = 4, 102400, 2
+    layers = []
+    for l in range(NL):
+        w = synth.make_layer(shape, 380 + l, "cuda", zipf=True)
+        layers.append(binding.Layer.from_weights(ctx, w))
+        del w
+    W = synth.lm_head(V, shape.hidden, 383, torch.bfloat16, "cuda")
+    blocks = [synth.hidden_block(K, shape.hidden, 384 + l, 0.0, "cuda") for l in range(NL)]
+    rb = [binding._routing_buffers(shape, K, "cuda") for _ in range(NL)]
+    ys = [torch.empty((K, shape.hidden), device="cuda") for _ in range(NL)]
+    yd = torch.empty((1, shape.hidden), device="cuda")
+    dbuf = {"topk_ids": torch.empty((shape.top_k,), dtype=torch.int32, device="cuda"),
+            "topk_w": torch.empty((shape.top_k,), device="cuda")}
+    res = [torch.zeros((K + 2,), dtype=torch.int32, device="cuda") for _ in range(NL)]
+    draft = torch.zeros((K,), dtype=torch.int32, device="cuda")
+
+    def step(li):
+        binding.moe_draft_step(layers[li], blocks[li][:1], yd, dbuf)
+        binding.moe_verify_block(layers[li], blocks[li], ys[li], rb[li])
+        binding.spec_accept(ctx, ys[li], W, draft, True,
+                            {"target": res[li][:K], "n_accept": res[li][K:K + 1], "next_token": res[li][K + 1:K + 2]})
+
+    for li in range(NL):
+        step(li)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == 0
+    want_res, want_y = [r.clone() for r in res], [y.clone() for y in ys]
+    W_np = synth.to_numpy_f32(W).astype(np.float64)
+    for li in range(NL):
+        hn = O.rmsnorm(ys[li].cpu().numpy().astype(np.float64))
+        t_ref, _, _, lg = O.greedy_accept_fast(hn, W_np, np.zeros(0, np.int32))
+        srt = np.sort(lg, axis=1)
+        clear = (srt[:, -1] - srt[:, -2]) > 1e-3
+        assert np.array_equal(res[li][:K].cpu().numpy()[clear], t_ref[clear])
+    stream = torch.cuda.current_stream()
+    side = torch.cuda.Stream()
+    side.wait_stream(stream)
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(g, stream=side):
+            for li in range(NL):
+                step(li)
+    stream.wait_stream(side)
+    for it in range(300):
+        for r in res:
+            r.fill_(-9)
+        g.replay()
+        torch.cuda.synchronize()
+        for li in range(NL):
+            assert torch.equal(res[li], want_res[li]), (it, li)
+            assert (ys[li] - want_y[li]).abs().max().item() <= 1e-4 * want_y[li].abs().max().item(), (it, li)
+    assert ctx.device_status() == 0
+    for L in layers:
+        L.close()
+    ctx.close()
